@@ -1,0 +1,200 @@
+/*
+ * metis.h - C ABI of the B200 (sm_100a) spectral-split NVFP4 linear layer.
+ *
+ * The library implements the hot path of "Metis: Training LLMs with FP4 Quantization":
+ * every GEMM operand T (activation X, weight W, output gradient D) is written as
+ *
+ *        T = L diag(sigma) R^T + Res                        (Section 3.2, Eq. 1)
+ *
+ * with the top-k factors found by sparse row sampling plus a Gaussian random projection
+ * (Section 3.1), the factors and the residual are quantized independently to NVFP4
+ * (Section 2.3, Appendix C.1) and the products of Eq. 2 (forward), Eq. 3 (input gradient) and
+ * the weight gradient of Section 3.2 are evaluated with block-scaled FP4 tensor-core GEMMs
+ * accumulating in FP32.
+ *
+ * General rules
+ *  - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns every
+ *    buffer (inputs, outputs, workspace); the library allocates device memory only inside
+ *    metis_create (a 128 KiB quantile table and a status word) and frees it in metis_destroy.
+ *  - All work is enqueued on the caller's stream (a cudaStream_t passed as void*); calls return
+ *    without synchronising.  Host-detectable errors (null or misaligned pointer, unsupported shape,
+ *    workspace too small) are returned at once and nothing is enqueued.  Device-detected conditions
+ *    (a bounded wait that expired, a Cholesky breakdown) are OR-ed into the handle's device status
+ *    word, read with metis_last_device_status after the caller has synchronised the stream.
+ *  - Matrices are row-major.  "K-major" below means the contraction axis is the contiguous axis.
+ *  - No function throws, aborts or calls exit.
+ *
+ * NVFP4 storage (metis_nvfp4_t)
+ *  - codes: 4-bit E2M1 codes, sign in bit 3, two per byte, element 2j in the low nibble; the tensor
+ *    is stored K-major: `rows` x `k_len`/2 bytes where the 16-element blocks lie along k_len.
+ *    Quantizing with blocks along the ROWS of a source matrix therefore stores the transposed
+ *    matrix (rows = source cols, k_len = source rows).
+ *  - scales: one unsigned E4M3 byte per block.  METIS_SF_LINEAR: scales[r][b], b = k/16.
+ *    METIS_SF_TILED: the tensor-core layout: tiles of 128 rows x 4 blocks, 512 bytes each, tile
+ *    (r/128, b/4) at offset ((r/128)*(k_len/64) + b/4)*512, byte (r%32)*16 + ((r%128)/32)*4 + b%4
+ *    inside it.  Needs k_len % 64 == 0; rows are padded to a multiple of 128 (metis_sf_bytes).
+ *  - tensor_scale: one FP32 device scalar; value = E2M1(code) * E4M3(scale) * tensor_scale.
+ */
+#ifndef METIS_H_
+#define METIS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct metis_context* metis_handle_t;
+typedef void* metis_stream_t;                 /* a cudaStream_t */
+
+typedef enum {
+  METIS_OK = 0,
+  METIS_ERR_INVALID_ARG = 1,
+  METIS_ERR_SHAPE = 2,
+  METIS_ERR_ALIGNMENT = 3,
+  METIS_ERR_WORKSPACE = 4,
+  METIS_ERR_ARCH = 5,
+  METIS_ERR_CUDA = 6,
+  METIS_ERR_NONFINITE = 7,
+  METIS_ERR_NUMERIC = 8,
+  METIS_ERR_TIMEOUT = 9
+} metis_status_t;
+
+/* bits of the device status word */
+#define METIS_DEV_TIMEOUT 1u     /* a bounded wait inside a kernel expired                      */
+#define METIS_DEV_NUMERIC 2u     /* Cholesky breakdown / non-positive pivot in the orthonormaliser */
+
+typedef enum { METIS_BF16 = 0, METIS_FP32 = 1 } metis_dtype_t;
+typedef enum { METIS_ROUND_RNE = 0, METIS_ROUND_SR = 1 } metis_round_t;
+typedef enum { METIS_BLOCKS_ALONG_COLS = 1, METIS_BLOCKS_ALONG_ROWS = 2, METIS_BLOCKS_BOTH = 3 } metis_axis_t;
+typedef enum { METIS_TSCALE_AMAX_SELF = 0, METIS_TSCALE_GIVEN = 1 } metis_tscale_t;
+typedef enum { METIS_SKETCH_FULL = 0, METIS_SKETCH_SAMPLED = 1 } metis_sketch_t;
+typedef enum { METIS_SF_LINEAR = 0, METIS_SF_TILED = 1 } metis_sf_layout_t;
+
+/* Philox stream identifiers (third counter word) used by the library's own draws. */
+#define METIS_STREAM_RESIDUAL 0x10u
+#define METIS_STREAM_LEFT     0x11u
+#define METIS_STREAM_RIGHT    0x12u
+#define METIS_STREAM_OMEGA    0x100u
+#define METIS_STREAM_SAMPLING 0x200u
+
+typedef struct {
+  uint8_t* codes;          /* rows * k_len / 2 bytes, K-major, 16-byte aligned                        */
+  uint8_t* scales;         /* metis_sf_bytes(rows, k_len, sf_layout) bytes, 16-byte aligned           */
+  float*   tensor_scale;   /* one device float                                                        */
+  int64_t  rows;           /* stored rows                                                             */
+  int64_t  k_len;          /* stored contraction length (multiple of 16; of 64 for METIS_SF_TILED)    */
+  int32_t  sf_layout;      /* metis_sf_layout_t                                                       */
+  int32_t  reserved;
+} metis_nvfp4_t;
+
+/* One split + quantized operand T (rows x cols) = left diag(sigma) right^T + residual.
+ * k == 0 means plain NVFP4: the factor fields are ignored.
+ * left / right are the FP32 factors stored TRANSPOSED (k x rows, k x cols: each factor vector
+ * contiguous); left_q / right_q their NVFP4 forms (rows = k, k_len = rows resp. cols), i.e. blocks
+ * along the long dimension.  res_by_cols is the residual with blocks along its columns (stored
+ * rows x cols), res_by_rows with blocks along its rows (stored cols x rows).  Either residual may
+ * be absent (codes == NULL) if no product needs it. */
+typedef struct {
+  int32_t k;
+  int32_t reserved;
+  int64_t rows, cols;
+  float* left;             /* k x rows  */
+  float* sigma;            /* k         */
+  float* right;            /* k x cols  */
+  metis_nvfp4_t left_q, right_q;
+  metis_nvfp4_t res_by_cols, res_by_rows;
+} metis_operand_t;
+
+/* ---- life cycle -------------------------------------------------------------------------- */
+
+/* Creates a context on `device` (cudaSetDevice is called; the device stays current).  Builds the
+ * 65536-entry standard-normal quantile table used by the sketch (Section 3.1).  Fails with
+ * METIS_ERR_ARCH unless the device has compute capability 10.x. */
+metis_status_t metis_create(metis_handle_t* out, int device);
+metis_status_t metis_destroy(metis_handle_t h);
+
+/* Copies the device status word (METIS_DEV_* bits, 0 = clean) to *out (host) and clears it.
+ * Synchronises `stream` first. */
+metis_status_t metis_last_device_status(metis_handle_t h, uint32_t* out, metis_stream_t stream);
+
+/* Test hook: copies the 65536 bfloat16 quantile-table entries (bit patterns) to host memory.
+ * Entry u is the standard normal quantile at level (u + 0.5)/65536 (Section 3.1: the Gaussian test
+ * matrix of the random projection is drawn through this table). */
+metis_status_t metis_debug_quantile_table(metis_handle_t h, uint16_t* host_out);
+
+/* Bytes of scale storage for a stored rows x k_len NVFP4 tensor (host-only helper, no handle). */
+size_t metis_sf_bytes(int64_t rows, int64_t k_len, int32_t sf_layout);
+
+/* Workspace sizes (host-only helpers).  op: 0 quantize, 1 split, 2 linear_fwd, 3 linear_bwd.
+ * rows/cols describe the largest operand (for the linear ops: rows = max(l, n), cols = max(m, n)). */
+metis_status_t metis_workspace_bytes(int32_t op, int64_t rows, int64_t cols, int32_t k, int32_t p, size_t* bytes);
+
+/* Number of rows the SAMPLED sketch reads for a rows-row operand with k+p sketch columns
+ * (Section 3.1: "less than 1 % of sequences"; at least 4(k+p), multiple of 16). */
+int64_t metis_default_sample_count(int64_t rows, int32_t q);
+
+/* ---- NVFP4 quantizer (Section 2.3; value set of Appendix C.1) ----------------------------- */
+
+/* Quantizes x (rows x cols, leading dimension ld elements, BF16 or FP32) into blocks of 16 along
+ * its columns (out_by_cols) and/or its rows (out_by_rows); an output pointer may be NULL.
+ * Block scale = smallest E4M3 value >= block amax / (6 * tensor_scale) ("rounded up"), elements
+ * rounded to nearest even or stochastically (16 random bits per element from Philox4x32-10 keyed
+ * by (seed, stream_id, row*cols + col), so both orientations use the same draw).
+ * tscale == METIS_TSCALE_AMAX_SELF: tensor_scale <- amax(x)/2688 (1 if x == 0), written to both
+ * outputs' tensor_scale; METIS_TSCALE_GIVEN: the outputs' tensor_scale already hold the value.
+ * Requires cols % 16 == 0 (by cols), rows % 16 == 0 (by rows); tiled scales need % 64.
+ * Workspace: metis_workspace_bytes(0, ...). */
+metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dtype, int64_t rows, int64_t cols,
+                                    int64_t ld, int32_t rounding, uint64_t seed, uint32_t stream_id,
+                                    int32_t tscale, metis_nvfp4_t* out_by_cols, metis_nvfp4_t* out_by_rows,
+                                    void* ws, size_t ws_bytes, metis_stream_t stream);
+
+/* ---- split (Sections 3.1, 3.2) ------------------------------------------------------------ */
+
+/* Splits x (rows x cols BF16, contiguous) into rank-k factors and a residual and quantizes all of
+ * them into `out` (whose buffers the caller has allocated; out->k, rows, cols are checked).
+ *  sketch = METIS_SKETCH_FULL:    Z = x Omega, thin QR, M = H^T x, small SVD, top k, residual
+ *                                 x - A Lambda B^T.
+ *  sketch = METIS_SKETCH_SAMPLED: the same on n_sample sampled rows (0 = default rule) to get the
+ *                                 right basis B, then C = x B for all rows, Rayleigh-Ritz on C^T C,
+ *                                 residual x - C B^T.
+ * Omega (cols x (k+p)) is generated on the fly from Philox (seed, METIS_STREAM_OMEGA) through the
+ * quantile table; it never exists in global memory.  The residual is quantized with the tensor
+ * scale amax(x)/2688 of the SOURCE tensor; factors with their own.  `residual_axes` selects which
+ * residual orientations are produced.  `residual_dense` (optional, rows x cols FP32) receives the
+ * unquantized residual the quantizer saw.  k == 0 quantizes x itself.
+ * Requires rows % 16 == 0, cols % 64 == 0 (tiled scales), k + p <= 64, k % 4 == 0.
+ * Workspace: metis_workspace_bytes(1, rows, cols, k, p). */
+metis_status_t metis_split(metis_handle_t h, const void* x, int64_t rows, int64_t cols, int32_t k, int32_t p,
+                           int32_t sketch, int64_t n_sample, uint64_t seed, int32_t rounding,
+                           int32_t residual_axes, metis_operand_t* out, float* residual_dense,
+                           void* ws, size_t ws_bytes, metis_stream_t stream);
+
+/* ---- linear layer (Eq. 2, Eq. 3, weight gradient) ----------------------------------------- */
+
+/* y (l x n, ldy) = Xq Wq^T, Eq. 2.  x: l x m operand with res_by_cols; w: W_t, n x m operand with
+ * res_by_cols.  y is BF16 or FP32.  Scales must be METIS_SF_TILED. */
+metis_status_t metis_linear_fwd(metis_handle_t h, const metis_operand_t* x, const metis_operand_t* w,
+                                void* y, int32_t y_dtype, int64_t ldy, void* ws, size_t ws_bytes,
+                                metis_stream_t stream);
+
+/* dx (l x m) = Dq Wq' (Eq. 3; needs dy->res_by_cols, w->res_by_rows) and
+ * dw (n x m) = Dq''^T Xq'' (weight gradient; needs dy->res_by_rows, x->res_by_rows).
+ * Either output may be NULL to skip it. */
+metis_status_t metis_linear_bwd(metis_handle_t h, const metis_operand_t* dy, const metis_operand_t* x,
+                                const metis_operand_t* w, void* dx, int32_t dx_dtype, int64_t lddx,
+                                void* dw, int32_t dw_dtype, int64_t lddw, void* ws, size_t ws_bytes,
+                                metis_stream_t stream);
+
+/* Plain block-scaled FP4 GEMM on already quantized tensors: d (M x N, ldd) = a b^T * (a.ts * b.ts),
+ * a: M x K, b: N x K, both K-major with METIS_SF_TILED scales.  Exposed for tests and benchmarks of
+ * the tensor-core kernel on identical codes.  impl: 0 = tcgen05 kernel, 1 = scalar check kernel. */
+metis_status_t metis_gemm_nvfp4(metis_handle_t h, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d,
+                                int32_t d_dtype, int64_t ldd, int32_t impl, metis_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* METIS_H_ */

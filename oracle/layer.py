@@ -62,8 +62,12 @@ def quantize_operand(x, k, p, mode, seed, rounding=nvfp4.ROUND_RNE):
     res_c = nvfp4.dequantize(*rc)
     res_r = nvfp4.dequantize(*rr).T
     if k:
-        lq = nvfp4.quantize(sp.left.astype(np.float32), nvfp4.AXIS_ROWS, rounding, seed, philox.STREAM_LEFT)
-        rq = nvfp4.quantize(sp.right.astype(np.float32), nvfp4.AXIS_ROWS, rounding, seed, philox.STREAM_RIGHT)
+        # factors are held transposed (k x rows, k x cols: one factor vector per stored row), so their
+        # blocks of 16 run along the long dimension and the draw of element (j, i) is keyed by j*len + i
+        lq = nvfp4.quantize(np.ascontiguousarray(sp.left.T).astype(np.float32), nvfp4.AXIS_COLS, rounding, seed,
+                            philox.STREAM_LEFT)
+        rq = nvfp4.quantize(np.ascontiguousarray(sp.right.T).astype(np.float32), nvfp4.AXIS_COLS, rounding, seed,
+                            philox.STREAM_RIGHT)
         raw["left"], raw["right"] = lq, rq
         left_q, right_q = nvfp4.dequantize(*lq).T, nvfp4.dequantize(*rq).T
     else:

@@ -3,9 +3,9 @@
 Test infrastructure: a slow restatement used to check the CUDA library; never on the product path.
 
 Format as the paper states it: values are partitioned into blocks of 16; each block gets one
-E4M3 scale "set by the block's maximum magnitude and rounded up to the nearest representable
-FP8 value"; each element becomes round(e/s)*s with round() onto the E2M1 set
-+-{0, 0.5, 1, 1.5, 2, 3, 4, 6}.  Added on top (the paper has block scales only): one FP32 scale
+E4M3 scale derived from the largest magnitude in the block and rounded UP to the next
+representable E4M3 value, so the block is always covered; each element becomes round(e/s)*s
+with round() onto the E2M1 set +-{0, 0.5, 1, 1.5, 2, 3, 4, 6}.  Added on top (the paper has block scales only): one FP32 scale
 per tensor, s_T = amax/(6*448), so the E4M3 block scales use their whole range.
 
 The defined arithmetic is IEEE binary32, round to nearest even, no fused multiply-add, denormals

@@ -1,0 +1,159 @@
+// Context life cycle, host-side argument checks and the C entry points that do not live with their kernels.
+#include <cuda.h>
+#include <math.h>
+#include <stdlib.h>
+
+#include "common.cuh"
+
+size_t metis_split_ws_bytes(int64_t rows, int64_t cols, int k, int p);
+size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k);
+
+namespace {
+
+// Standard normal quantile for 0 < p <= 0.5 by Newton iteration on the complementary error function,
+// started from the classical rational approximation (Abramowitz & Stegun 26.2.23).
+double inv_norm_cdf_lower(double p) {
+  const double t = sqrt(-2.0 * log(p));
+  double x = -(t - (2.515517 + 0.802853 * t + 0.010328 * t * t) / (1.0 + 1.432788 * t + 0.189269 * t * t + 0.001308 * t * t * t));
+  for (int it = 0; it < 8; ++it) {
+    const double f = 0.5 * erfc(-x * 0.70710678118654752440) - p;
+    const double df = 0.39894228040143267794 * exp(-0.5 * x * x);
+    const double step = f / df;
+    x -= step / (1.0 + 0.5 * x * step);             // Halley correction
+  }
+  return x;
+}
+
+}  // namespace
+
+extern "C" {
+
+metis_status_t metis_create(metis_handle_t* out, int device) {
+  if (!out) return METIS_ERR_INVALID_ARG;
+  *out = nullptr;
+  METIS_CUDA_TRY(cudaSetDevice(device));
+  cudaDeviceProp prop;
+  METIS_CUDA_TRY(cudaGetDeviceProperties(&prop, device));
+  if (prop.major != 10) return METIS_ERR_ARCH;
+  metis_context* ctx = static_cast<metis_context*>(calloc(1, sizeof(metis_context)));
+  if (!ctx) return METIS_ERR_INVALID_ARG;
+  ctx->device = device;
+  ctx->sm_count = prop.multiProcessorCount;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !ctx->encode_tiled) {
+    free(ctx);
+    return METIS_ERR_CUDA;
+  }
+  __nv_bfloat16* host = static_cast<__nv_bfloat16*>(malloc(65536 * sizeof(__nv_bfloat16)));
+  if (!host) { free(ctx); return METIS_ERR_INVALID_ARG; }
+  for (int u = 0; u < 32768; ++u) {
+    const double v = inv_norm_cdf_lower((u + 0.5) / 65536.0);
+    host[u] = __float2bfloat16_rn((float)v);
+    host[65535 - u] = __float2bfloat16_rn((float)(-v));
+  }
+  cudaError_t e = cudaMalloc(&ctx->quantile_lut, 65536 * sizeof(__nv_bfloat16));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, 256);
+  if (e == cudaSuccess) e = cudaMemcpy(ctx->quantile_lut, host, 65536 * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, 256);
+  free(host);
+  if (e != cudaSuccess) {
+    cudaFree(ctx->quantile_lut); cudaFree(ctx->dev_status); free(ctx);
+    return METIS_ERR_CUDA;
+  }
+  *out = ctx;
+  return METIS_OK;
+}
+
+metis_status_t metis_destroy(metis_handle_t h) {
+  if (!h) return METIS_OK;
+  cudaFree(h->quantile_lut);
+  cudaFree(h->dev_status);
+  free(h);
+  return METIS_OK;
+}
+
+metis_status_t metis_last_device_status(metis_handle_t h, uint32_t* out, metis_stream_t stream) {
+  if (!h || !out) return METIS_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  METIS_CUDA_TRY(cudaMemcpyAsync(out, h->dev_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s));
+  METIS_CUDA_TRY(cudaMemsetAsync(h->dev_status, 0, sizeof(uint32_t), s));
+  METIS_CUDA_TRY(cudaStreamSynchronize(s));
+  return METIS_OK;
+}
+
+metis_status_t metis_debug_quantile_table(metis_handle_t h, uint16_t* host_out) {
+  if (!h || !host_out) return METIS_ERR_INVALID_ARG;
+  METIS_CUDA_TRY(cudaMemcpy(host_out, h->quantile_lut, 65536 * sizeof(uint16_t), cudaMemcpyDeviceToHost));
+  return METIS_OK;
+}
+
+size_t metis_sf_bytes(int64_t rows, int64_t k_len, int32_t sf_layout) {
+  if (rows <= 0 || k_len <= 0) return 0;
+  if (sf_layout == METIS_SF_TILED) return (size_t)(metis_ceil_div(rows, 128) * metis_ceil_div(k_len, 64) * 512);
+  return (size_t)(rows * metis_ceil_div(k_len, 16));
+}
+
+metis_status_t metis_workspace_bytes(int32_t op, int64_t rows, int64_t cols, int32_t k, int32_t p, size_t* bytes) {
+  if (!bytes || rows <= 0 || cols <= 0 || k < 0 || p < 0) return METIS_ERR_INVALID_ARG;
+  switch (op) {
+    case 0: *bytes = 256; return METIS_OK;
+    case 1: *bytes = metis_split_ws_bytes(rows, cols, k, p); return METIS_OK;
+    case 2:
+    case 3: *bytes = metis_linear_ws_bytes(rows, cols, k); return METIS_OK;
+    default: return METIS_ERR_INVALID_ARG;
+  }
+}
+
+metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dtype, int64_t rows, int64_t cols,
+                                    int64_t ld, int32_t rounding, uint64_t seed, uint32_t stream_id, int32_t tscale,
+                                    metis_nvfp4_t* out_by_cols, metis_nvfp4_t* out_by_rows, void* ws, size_t ws_bytes,
+                                    metis_stream_t stream) {
+  if (!h || !x || (!out_by_cols && !out_by_rows)) return METIS_ERR_INVALID_ARG;
+  if (dtype != METIS_BF16 && dtype != METIS_FP32) return METIS_ERR_INVALID_ARG;
+  if (rounding != METIS_ROUND_RNE && rounding != METIS_ROUND_SR) return METIS_ERR_INVALID_ARG;
+  if (tscale != METIS_TSCALE_AMAX_SELF && tscale != METIS_TSCALE_GIVEN) return METIS_ERR_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || ld < cols) return METIS_ERR_SHAPE;
+  if (!metis_aligned16(x)) return METIS_ERR_ALIGNMENT;
+  metis_nvfp4_t* outs[2] = {out_by_cols, out_by_rows};
+  for (int i = 0; i < 2; ++i) {
+    metis_nvfp4_t* o = outs[i];
+    if (!o) continue;
+    if (!o->codes || !o->scales || !o->tensor_scale) return METIS_ERR_INVALID_ARG;
+    if (!metis_aligned16(o->codes) || !metis_aligned16(o->scales)) return METIS_ERR_ALIGNMENT;
+    const int64_t klen = i == 0 ? cols : rows;
+    if (klen % 16) return METIS_ERR_SHAPE;
+    if (o->sf_layout == METIS_SF_TILED && klen % 64) return METIS_ERR_SHAPE;
+    if (o->sf_layout != METIS_SF_TILED && o->sf_layout != METIS_SF_LINEAR) return METIS_ERR_INVALID_ARG;
+    o->rows = i == 0 ? rows : cols;
+    o->k_len = klen;
+  }
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const float* ts_src;
+  int is_amax = 0;
+  if (tscale == METIS_TSCALE_AMAX_SELF) {
+    if (!ws || ws_bytes < 256) return METIS_ERR_WORKSPACE;
+    float* amax = static_cast<float*>(ws);
+    METIS_TRY(metis_launch_amax(x, dtype, rows, cols, ld, amax, s));
+    ts_src = amax;
+    is_amax = 1;
+  } else {
+    ts_src = out_by_cols ? out_by_cols->tensor_scale : out_by_rows->tensor_scale;
+  }
+  return metis_launch_quantize(x, dtype, rows, cols, ld, rounding, seed, stream_id, cols, 1, ts_src, is_amax,
+                               out_by_cols, out_by_rows, s);
+}
+
+metis_status_t metis_gemm_nvfp4(metis_handle_t h, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d,
+                                int32_t d_dtype, int64_t ldd, int32_t impl, metis_stream_t stream) {
+  if (!h || !a || !b || !d) return METIS_ERR_INVALID_ARG;
+  if (!a->codes || !b->codes || !a->scales || !b->scales || !a->tensor_scale || !b->tensor_scale) return METIS_ERR_INVALID_ARG;
+  if (a->k_len != b->k_len || a->k_len % 16) return METIS_ERR_SHAPE;
+  if (ldd < b->rows) return METIS_ERR_SHAPE;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (impl == 1) return metis_launch_gemm_check(a, b, d, d_dtype, ldd, s);
+  if (impl != 0) return METIS_ERR_INVALID_ARG;
+  return metis_launch_gemm_tc(h, a, b, d, d_dtype, ldd, s);
+}
+
+}  // extern "C"

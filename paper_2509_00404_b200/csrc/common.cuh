@@ -1,0 +1,139 @@
+// Shared device/host helpers of the Metis B200 library: context, error plumbing, Philox, NVFP4 scalar math.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/metis.h"
+
+struct metis_context {
+  int device;
+  int sm_count;
+  __nv_bfloat16* quantile_lut;   // 65536 bf16 standard-normal quantiles (Section 3.1 Gaussian test matrix)
+  uint32_t* dev_status;          // device status word (METIS_DEV_* bits)
+  void* encode_tiled;            // cuTensorMapEncodeTiled entry point, resolved at create
+};
+
+#define METIS_CUDA_TRY(expr)                         \
+  do {                                               \
+    cudaError_t e__ = (expr);                        \
+    if (e__ != cudaSuccess) return METIS_ERR_CUDA;   \
+  } while (0)
+
+#define METIS_TRY(expr)                              \
+  do {                                               \
+    metis_status_t s__ = (expr);                     \
+    if (s__ != METIS_OK) return s__;                 \
+  } while (0)
+
+static inline bool metis_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline int64_t metis_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al. 2011).  One call yields 128 bits = eight 16-bit draws.
+// Draw rule: element index e -> counter (lo32(e>>3), hi32(e>>3), stream, 0), key (lo32 seed, hi32 seed),
+// 16-bit half number e&7 of the four output words (low half first).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 metis_philox(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                              uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+__device__ __forceinline__ uint4 metis_philox_block(uint64_t block_index, uint64_t seed, uint32_t stream) {
+  return metis_philox((uint32_t)block_index, (uint32_t)(block_index >> 32), stream, 0u, (uint32_t)seed,
+                      (uint32_t)(seed >> 32));
+}
+
+__device__ __forceinline__ uint32_t metis_u16_of(const uint4& w, uint32_t h) {
+  const uint32_t word = (h >> 1) == 0 ? w.x : (h >> 1) == 1 ? w.y : (h >> 1) == 2 ? w.z : w.w;
+  return (word >> (16u * (h & 1u))) & 0xFFFFu;
+}
+
+__device__ __forceinline__ uint32_t metis_draw_u16(uint64_t e, uint64_t seed, uint32_t stream) {
+  return metis_u16_of(metis_philox_block(e >> 3, seed, stream), (uint32_t)(e & 7u));
+}
+
+// ---------------------------------------------------------------------------------------------
+// NVFP4 scalar arithmetic (Section 2.3).  Every step is a single IEEE binary32 operation with
+// round-to-nearest-even and no contraction; this order defines the format's rounding decisions.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float metis_tensor_scale(float amax) { return amax == 0.0f ? 1.0f : __fdiv_rn(amax, 2688.0f); }
+
+// smallest non-negative finite E4M3 value >= t (0 <= t <= 448); returns the byte and the value
+__device__ __forceinline__ uint32_t metis_e4m3_ceil(float t, float* value) {
+  if (!(t > 0.0f)) { *value = 0.0f; return 0u; }
+  if (t <= 0.015625f) {                       // subnormal range: multiples of 2^-9 up to 2^-6
+    const int f = (int)ceilf(__fmul_rn(t, 512.0f));
+    *value = __fmul_rn((float)f, 0.001953125f);
+    return (uint32_t)f;                       // f == 8 is the first normal number (byte 0x08)
+  }
+  uint32_t b = __float_as_uint(t);
+  b = (b + 0xFFFFFu) & 0xFFF00000u;           // keep 3 mantissa bits, round up (carry moves the exponent)
+  *value = __uint_as_float(b);
+  const uint32_t e = (b >> 23) - 127u + 7u;
+  return (e << 3) | ((b >> 20) & 7u);
+}
+
+__device__ __forceinline__ float metis_e4m3_value(uint32_t byte) {
+  const uint32_t e = (byte >> 3) & 15u, f = byte & 7u;
+  return e == 0 ? __fmul_rn((float)f, 0.001953125f) : __uint_as_float(((e + 120u) << 23) | (f << 20));
+}
+
+__device__ __forceinline__ float metis_e2m1_value(uint32_t code) {
+  const uint32_t m = code & 7u;
+  const float mag = m < 4 ? 0.5f * (float)m : (m == 4 ? 2.0f : m == 5 ? 3.0f : m == 6 ? 4.0f : 6.0f);
+  return (code & 8u) ? -mag : mag;
+}
+
+// two round-to-nearest-even E2M1 codes in one byte: lo in bits 0-3, hi in bits 4-7
+__device__ __forceinline__ uint32_t metis_e2m1x2_rne(float lo, float hi) {
+  uint32_t out;
+  asm("{ .reg .b8 t8; cvt.rn.satfinite.e2m1x2.f32 t8, %1, %2; cvt.u32.u8 %0, t8; }" : "=r"(out) : "f"(hi), "f"(lo));
+  return out;
+}
+
+// stochastic rounding of y to E2M1 with a 16-bit draw: up iff frac * 65536 > u
+__device__ __forceinline__ uint32_t metis_e2m1_sr(float y, uint32_t u16) {
+  const float a = fminf(fabsf(y), 6.0f);
+  const uint32_t sign = (__float_as_uint(y) >> 28) & 8u;
+  int lo_c = (a >= 0.5f) + (a >= 1.0f) + (a >= 1.5f) + (a >= 2.0f) + (a >= 3.0f) + (a >= 4.0f) + (a >= 6.0f);
+  if (lo_c == 7) return sign | 7u;
+  const float lo = lo_c < 4 ? 0.5f * (float)lo_c : (lo_c == 4 ? 2.0f : lo_c == 5 ? 3.0f : 4.0f);
+  const float inv_step = lo_c < 4 ? 2.0f : (lo_c == 6 ? 0.5f : 1.0f);
+  const float f = __fmul_rn(__fsub_rn(a, lo), inv_step);
+  const uint32_t up = __fmul_rn(f, 65536.0f) > (float)u16 ? 1u : 0u;
+  return sign | (uint32_t)(lo_c + up);
+}
+
+// byte offset of scale (row r, block b) in the 128x4-tiled layout; blocks_per_row = k_len/16
+__host__ __device__ __forceinline__ int64_t metis_sf_offset_tiled(int64_t r, int64_t b, int64_t blocks_per_row) {
+  return ((r >> 7) * (blocks_per_row >> 2) + (b >> 2)) * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4 + (b & 3);
+}
+__host__ __device__ __forceinline__ int64_t metis_sf_offset(int64_t r, int64_t b, int64_t blocks_per_row, int layout) {
+  return layout == METIS_SF_TILED ? metis_sf_offset_tiled(r, b, blocks_per_row) : r * blocks_per_row + b;
+}
+
+__device__ __forceinline__ float metis_ld_as_float(const void* p, int dtype, int64_t idx) {
+  return dtype == METIS_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx])
+                             : reinterpret_cast<const float*>(p)[idx];
+}
+
+// ---- internal entry points shared between translation units --------------------------------
+metis_status_t metis_launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* amax_out,
+                                 cudaStream_t s);
+metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int rounding,
+                                     uint64_t seed, uint32_t stream_id, int64_t e_stride_r, int64_t e_stride_c,
+                                     const float* tscale_src, int tscale_is_amax, const metis_nvfp4_t* by_cols,
+                                     const metis_nvfp4_t* by_rows, cudaStream_t s);
+metis_status_t metis_launch_gemm_check(const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d, int d_dtype,
+                                       int64_t ldd, cudaStream_t s);
+metis_status_t metis_launch_gemm_tc(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d,
+                                    int d_dtype, int64_t ldd, cudaStream_t s);

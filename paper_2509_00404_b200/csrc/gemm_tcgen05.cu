@@ -1,0 +1,372 @@
+// Block-scaled NVFP4 GEMM on the 5th-generation tensor cores (tcgen05) of sm_100a.
+//
+//   D[M x N] = alpha * sum_k  e2m1(A[m,k]) * ue4m3(SFA[m,k/16]) * e2m1(B[n,k]) * ue4m3(SFB[n,k/16])
+//
+// A (M x K) and B (N x K) are K-major packed FP4 (two codes per byte) with one UE4M3 scale per 16
+// elements stored in the 128 x 4 tiled layout, alpha = tensor_scale(A) * tensor_scale(B).
+// This is the product that carries "over 95 % of the training workload" (Section 3): the
+// residual x residual term of Eq. 2 / Eq. 3 / the weight gradient, and the skinny factor products.
+//
+// Structure (one CTA per SM, persistent over output tiles, warp-specialised):
+//   warp 0      producer: TMA tensor loads of the A/B code tiles (128-byte swizzle) and bulk copies of
+//               the scale atoms into a multi-stage shared-memory ring, completion on mbarriers
+//   warp 1      MMA issuer: copies the scale atoms shared memory -> tensor memory (tcgen05.cp), issues
+//               tcgen05.mma kind::mxf4nvf4 (block16 scales) accumulating FP32 in tensor memory,
+//               releases ring slots with tcgen05.commit
+//   warps 2-5   epilogue: tcgen05.ld the accumulator (one TMEM lane quarter per warp), scale by alpha,
+//               convert and store; accumulators are double-buffered so the epilogue of tile i overlaps
+//               the main loop of tile i+1
+// Every mbarrier wait is bounded; on expiry the kernel records METIS_DEV_TIMEOUT and unwinds.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 256;                  // elements per stage = 128 bytes of packed FP4 = one swizzle row
+constexpr int MMA_K = 64;                     // elements per tcgen05.mma (kind::mxf4nvf4, dense)
+constexpr int K_STEPS = BLOCK_K / MMA_K;      // 4
+constexpr int NUM_THREADS = 192;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+template <int BLOCK_N>
+struct Cfg {
+  static constexpr int STAGES = BLOCK_N == 128 ? 6 : 4;
+  static constexpr int NUM_ACC = BLOCK_N == 128 ? 2 : 1;
+  static constexpr int N_TILES_SF = BLOCK_N / 128;                 // 128-row scale tiles of B per stage
+  static constexpr int A_BYTES = BLOCK_M * BLOCK_K / 2;            // 16 KiB
+  static constexpr int B_BYTES = BLOCK_N * BLOCK_K / 2;
+  static constexpr int SFA_BYTES = K_STEPS * 512;
+  static constexpr int SFB_BYTES = N_TILES_SF * K_STEPS * 512;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
+  static constexpr int ACC_COLS = NUM_ACC * BLOCK_N;               // 256
+  static constexpr int SFA_COL = ACC_COLS;                         // 16 columns
+  static constexpr int SFB_COL = ACC_COLS + 4 * K_STEPS;           // 16 or 32 columns
+  static constexpr int TMEM_COLS = 512;
+  static constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: returns false (and records the timeout) instead of spinning forever.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* dev_status, volatile int* dead) {
+  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (i > 32) __nanosleep(64);
+    if ((i & 1023u) == 1023u && *dead) break;
+  }
+  *dead = 1;
+  atomicOr(dev_status, METIS_DEV_TIMEOUT);
+  return false;
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{ .reg .pred p; setp.ne.b32 p, %4, 0;\n"
+      "  tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p; }"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor (sm_100 format): start address [0,14) in 16-byte units, leading byte
+// offset [16,30), stride byte offset [32,46), descriptor version 1 at [46,48), swizzle mode [61,64).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t sbo_bytes, uint32_t swizzle_mode) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;
+  d |= (uint64_t)swizzle_mode << 61;
+  return d;
+}
+constexpr uint32_t SWIZZLE_NONE = 0, SWIZZLE_128B = 2;
+
+// Instruction descriptor for kind::mxf4nvf4 with UE4M3 scales: E2M1 operands (format 1) at [7,10) and
+// [10,13), both K-major, N/8 at [17,23), scale format 0 (UE4M3) at bit 23, M/16 at [24,29).
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
+  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+struct GemmArgs {
+  const uint8_t* a_sf; const uint8_t* b_sf;
+  const float* a_ts; const float* b_ts;
+  void* d; int d_dtype; int64_t ldd;
+  int M, N, K;
+  uint32_t* dev_status;
+};
+
+template <int BLOCK_N>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmArgs g) {
+  using C = Cfg<BLOCK_N>;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;              // 1024-byte alignment for the 128-byte swizzle
+  unsigned char* gen_base = smem_raw + (base - raw);
+  auto a_addr = [&](int s) { return base + (uint32_t)s * C::STAGE_BYTES; };
+  auto b_addr = [&](int s) { return a_addr(s) + C::A_BYTES; };
+  auto sfa_addr = [&](int s) { return b_addr(s) + C::B_BYTES; };
+  auto sfb_addr = [&](int s) { return sfa_addr(s) + C::SFA_BYTES; };
+  const uint32_t bar_base = base + (uint32_t)C::STAGES * C::STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + C::NUM_ACC + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + (size_t)C::STAGES * C::STAGE_BYTES + 8 * (2 * C::STAGES + 2 * C::NUM_ACC));
+  volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_m = (g.M + BLOCK_M - 1) / BLOCK_M, num_n = (g.N + BLOCK_N - 1) / BLOCK_N;
+  const int num_tiles = num_m * num_n;
+  const int num_kb = (g.K + BLOCK_K - 1) / BLOCK_K;
+  const int sf_k_atoms = g.K / MMA_K;                        // 512-byte scale atoms per 128-row tile
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < C::NUM_ACC; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    *dead = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------- producer -------------------------------
+    if (lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int mb = tile % num_m, nb = tile / num_m;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
+          const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
+          const uint32_t bytes = C::A_BYTES + C::B_BYTES + (uint32_t)atoms * 512u * (1 + C::N_TILES_SF);
+          mbar_expect_tx(full_bar(s), bytes);
+          tma_load_2d(a_addr(s), &map_a, kb * (BLOCK_K / 2), mb * BLOCK_M, full_bar(s));
+          tma_load_2d(b_addr(s), &map_b, kb * (BLOCK_K / 2), nb * BLOCK_N, full_bar(s));
+          bulk_load(sfa_addr(s), g.a_sf + ((size_t)mb * sf_k_atoms + (size_t)kb * K_STEPS) * 512, atoms * 512, full_bar(s));
+#pragma unroll
+          for (int t = 0; t < C::N_TILES_SF; ++t)
+            bulk_load(sfb_addr(s) + t * K_STEPS * 512,
+                      g.b_sf + ((size_t)(nb * C::N_TILES_SF + t) * sf_k_atoms + (size_t)kb * K_STEPS) * 512, atoms * 512,
+                      full_bar(s));
+          if (++s == C::STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer -----------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
+      int s = 0; uint32_t ph = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+        const int acc = it % C::NUM_ACC;
+        const uint32_t acc_ph = (uint32_t)(it / C::NUM_ACC) & 1u;
+        if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BLOCK_N);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
+          tc_fence_after();
+          const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
+          for (int k = 0; k < atoms; ++k) {
+            tc_cp_sf(tmem_base + C::SFA_COL + 4 * k, make_smem_desc(sfa_addr(s) + k * 512, 128, SWIZZLE_NONE));
+#pragma unroll
+            for (int t = 0; t < C::N_TILES_SF; ++t)
+              tc_cp_sf(tmem_base + C::SFB_COL + 4 * (k * C::N_TILES_SF + t),
+                       make_smem_desc(sfb_addr(s) + (t * K_STEPS + k) * 512, 128, SWIZZLE_NONE));
+          }
+          for (int k = 0; k < atoms; ++k) {
+            const uint64_t a_desc = make_smem_desc(a_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
+            const uint64_t b_desc = make_smem_desc(b_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
+            tc_mma_nvf4(d_tmem, a_desc, b_desc, idesc, tmem_base + C::SFA_COL + 4 * k,
+                        tmem_base + C::SFB_COL + 4 * k * C::N_TILES_SF, (kb | k) != 0 ? 1u : 0u);
+          }
+          tc_commit(empty_bar(s));                           // slot reusable once these MMAs have read it
+          if (++s == C::STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (ok) tc_commit(tfull_bar(acc));                   // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------- epilogue -------------------------------
+    const int quarter = warp & 3;                            // TMEM lanes 32*quarter .. +31 belong to this warp
+    const float alpha = (*g.a_ts) * (*g.b_ts);
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      const int mb = tile % num_m, nb = tile / num_m;
+      const int acc = it % C::NUM_ACC;
+      const uint32_t acc_ph = (uint32_t)(it / C::NUM_ACC) & 1u;
+      if (!mbar_wait(tfull_bar(acc), acc_ph, g.dev_status, dead)) { ok = false; break; }
+      tc_fence_after();
+      const int row = mb * BLOCK_M + quarter * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BLOCK_N; c0 += 32) {
+        uint32_t r[32];
+        tc_ld32(t_row + c0, r);
+        const int col = nb * BLOCK_N + c0;
+        if (row < g.M && col < g.N) {
+          if (g.d_dtype == METIS_FP32) {
+            float* dst = reinterpret_cast<float*>(g.d) + (size_t)row * g.ldd + col;
+            if (col + 32 <= g.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
+                                                                  __uint_as_float(r[j + 2]) * alpha, __uint_as_float(r[j + 3]) * alpha);
+            } else {
+              for (int j = 0; j < 32 && col + j < g.N; ++j) dst[j] = __uint_as_float(r[j]) * alpha;
+            }
+          } else {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(g.d) + (size_t)row * g.ldd + col;
+            if (col + 32 <= g.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                uint32_t w[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * q]) * alpha,
+                                                                 __uint_as_float(r[j + 2 * q + 1]) * alpha);
+                  w[q] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+                *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            } else {
+              for (int j = 0; j < 32 && col + j < g.N; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]) * alpha);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+    }
+  }
+
+  // ------------------------------- teardown ---------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (*dead) {
+    // a wait expired: give copies already in flight time to land before the shared memory is released
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+metis_status_t make_codes_map(metis_context* ctx, CUtensorMap* map, const metis_nvfp4_t* t, int box_rows) {
+  const cuuint64_t dims[2] = {(cuuint64_t)(t->k_len / 2), (cuuint64_t)t->rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)(t->k_len / 2)};
+  const cuuint32_t box[2] = {(cuuint32_t)(BLOCK_K / 2), (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+      map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, t->codes, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? METIS_OK : METIS_ERR_CUDA;
+}
+
+template <int BLOCK_N>
+metis_status_t launch(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d, int d_dtype,
+                      int64_t ldd, cudaStream_t s) {
+  using C = Cfg<BLOCK_N>;
+  CUtensorMap map_a, map_b;
+  METIS_TRY(make_codes_map(ctx, &map_a, a, BLOCK_M));
+  METIS_TRY(make_codes_map(ctx, &map_b, b, BLOCK_N));
+  GemmArgs g{};
+  g.a_sf = a->scales; g.b_sf = b->scales; g.a_ts = a->tensor_scale; g.b_ts = b->tensor_scale;
+  g.d = d; g.d_dtype = d_dtype; g.ldd = ldd;
+  g.M = (int)a->rows; g.N = (int)b->rows; g.K = (int)a->k_len;
+  g.dev_status = ctx->dev_status;
+  static bool attr_set = false;
+  if (!attr_set) {
+    METIS_CUDA_TRY(cudaFuncSetAttribute(gemm_nvfp4_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
+    attr_set = true;
+  }
+  const int tiles = (int)(metis_ceil_div(g.M, BLOCK_M) * metis_ceil_div(g.N, BLOCK_N));
+  const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  gemm_nvfp4_kernel<BLOCK_N><<<grid, NUM_THREADS, C::SMEM_BYTES, s>>>(map_a, map_b, g);
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
+
+}  // namespace
+
+metis_status_t metis_launch_gemm_tc(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d,
+                                    int d_dtype, int64_t ldd, cudaStream_t s) {
+  if (a->rows == 0 || b->rows == 0) return METIS_OK;
+  if (a->k_len != b->k_len || a->k_len % 64 != 0 || a->k_len <= 0) return METIS_ERR_SHAPE;
+  if (a->sf_layout != METIS_SF_TILED || b->sf_layout != METIS_SF_TILED) return METIS_ERR_INVALID_ARG;
+  if (!metis_aligned16(a->codes) || !metis_aligned16(b->codes) || !metis_aligned16(a->scales) || !metis_aligned16(b->scales))
+    return METIS_ERR_ALIGNMENT;
+  if (a->rows > INT32_MAX || b->rows > INT32_MAX || a->k_len > INT32_MAX) return METIS_ERR_SHAPE;
+  return launch<128>(ctx, a, b, d, d_dtype, ldd, s);
+}

@@ -1,0 +1,187 @@
+// Split-FP4 linear layer: forward (Eq. 2), input gradient (Eq. 3) and weight gradient (Section 3.2).
+//
+// With both operands written as  Ta = Fo_a diag(sa) Fc_a^T + Res_a  (M x K) and
+// Tb = Fo_b diag(sb) Fc_b^T + Res_b (N x K), where Fc_* are the factors lying along the contraction
+// axis and Fo_* those lying along the output axes, the product expands into
+//
+//   Ta Tb^T = Res_a Res_b^T                          main FP4 GEMM           (M x N)
+//           + (G1 + Fo_a sa P) sb Fo_b^T             G1 = Res_a Fc_b (M x kb), P = Fc_a^T Fc_b (ka x kb)
+//           + (Fo_a sa) Wt^T                         Wt = Res_b Fc_a (N x ka)
+//
+// i.e. one large and three skinny block-scaled FP4 GEMMs followed by a rank-(ka+kb) FP32 update.
+// All four quantized cross terms of the paper's expansion are kept.
+#include "common.cuh"
+
+namespace {
+
+__device__ __forceinline__ float deq_at(const uint8_t* codes, const uint8_t* sf, int layout, int64_t k_len, int64_t r,
+                                        int64_t c) {
+  const uint32_t byte = codes[r * (k_len / 2) + c / 2];
+  const uint32_t code = (c & 1) ? (byte >> 4) : (byte & 15u);
+  return metis_e2m1_value(code) * metis_e4m3_value(sf[metis_sf_offset(r, c / 16, k_len / 16, layout)]);
+}
+
+// Lcat [M][kb + ka], Rcat [N][kb + ka]
+__global__ void lowrank_prepare_kernel(int64_t M, int64_t N, int ka, int kb,
+                                       const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts,
+                                       const float* sa,
+                                       const uint8_t* fob_codes, const uint8_t* fob_sf, int fob_layout, const float* fob_ts,
+                                       const float* sb,
+                                       const float* __restrict__ g1, const float* __restrict__ wt, const float* __restrict__ pm,
+                                       float* __restrict__ lcat, float* __restrict__ rcat) {
+  const int kc = ka + kb;
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i < M) {
+    float fa[64];
+    const float tsa = ka ? *foa_ts : 0.0f;
+    for (int u = 0; u < ka; ++u) fa[u] = deq_at(foa_codes, foa_sf, foa_layout, M, u, i) * tsa * sa[u];
+    for (int t = 0; t < kb; ++t) {
+      float v = g1[i * kb + t];
+      for (int u = 0; u < ka; ++u) v = fmaf(fa[u], pm[u * kb + t], v);
+      lcat[i * kc + t] = v * sb[t];
+    }
+    for (int u = 0; u < ka; ++u) lcat[i * kc + kb + u] = fa[u];
+  }
+  if (i < N) {
+    const float tsb = kb ? *fob_ts : 0.0f;
+    for (int t = 0; t < kb; ++t) rcat[i * kc + t] = deq_at(fob_codes, fob_sf, fob_layout, N, t, i) * tsb;
+    for (int u = 0; u < ka; ++u) rcat[i * kc + kb + u] = wt[i * ka + u];
+  }
+}
+
+// out = y0 + Lcat Rcat^T, 64 x 64 tile per CTA
+__global__ void __launch_bounds__(256)
+rank_update_kernel(const float* __restrict__ y0, int64_t M, int64_t N, int kc, const float* __restrict__ lcat,
+                   const float* __restrict__ rcat, void* __restrict__ out, int out_dtype, int64_t ldo) {
+  extern __shared__ float sm[];
+  float* ls = sm;                       // [kc][64 + 4]
+  float* rs = sm + kc * 68;
+  const int tid = threadIdx.x;
+  const int64_t m0 = (int64_t)blockIdx.y * 64, n0 = (int64_t)blockIdx.x * 64;
+  for (int i = tid; i < 64 * kc; i += 256) {
+    const int r = i / kc, t = i % kc;
+    ls[t * 68 + r] = (m0 + r < M) ? lcat[(m0 + r) * kc + t] : 0.0f;
+    rs[t * 68 + r] = (n0 + r < N) ? rcat[(n0 + r) * kc + t] : 0.0f;
+  }
+  __syncthreads();
+  const int ty = tid >> 4, tx = tid & 15;
+  float acc[4][4] = {};
+  for (int t = 0; t < kc; ++t) {
+    const float4 a = *reinterpret_cast<const float4*>(ls + t * 68 + ty * 4);
+    const float4 b = *reinterpret_cast<const float4*>(rs + t * 68 + tx * 4);
+    const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t r = m0 + ty * 4 + i, c = n0 + tx * 4 + j;
+      if (r < M && c < N) {
+        const float v = y0[r * N + c] + acc[i][j];
+        if (out_dtype == METIS_BF16) reinterpret_cast<__nv_bfloat16*>(out)[r * ldo + c] = __float2bfloat16_rn(v);
+        else reinterpret_cast<float*>(out)[r * ldo + c] = v;
+      }
+    }
+}
+
+struct Side {
+  const metis_nvfp4_t* res;   // residual, K-major along the contraction axis
+  const metis_nvfp4_t* fc;    // factor along the contraction axis (k x K)
+  const metis_nvfp4_t* fo;    // factor along the output axis      (k x M or k x N)
+  const float* sigma;
+  int k;
+};
+
+size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+metis_status_t check_nvfp4(const metis_nvfp4_t* t) {
+  if (!t || !t->codes || !t->scales || !t->tensor_scale) return METIS_ERR_INVALID_ARG;
+  if (t->sf_layout != METIS_SF_TILED) return METIS_ERR_INVALID_ARG;
+  if (t->k_len % 64 || t->rows <= 0) return METIS_ERR_SHAPE;
+  return METIS_OK;
+}
+
+metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void* d, int d_dtype, int64_t ldd, void* ws,
+                          size_t ws_bytes, cudaStream_t s) {
+  METIS_TRY(check_nvfp4(a.res));
+  METIS_TRY(check_nvfp4(b.res));
+  const int64_t M = a.res->rows, N = b.res->rows, K = a.res->k_len;
+  if (b.res->k_len != K) return METIS_ERR_SHAPE;
+  const int ka = a.k, kb = b.k, kc = ka + kb;
+  if (kc == 0) return metis_launch_gemm_tc(ctx, a.res, b.res, d, d_dtype, ldd, s);
+  if (ka > 64 || kb > 64) return METIS_ERR_SHAPE;
+  if (ka) { METIS_TRY(check_nvfp4(a.fc)); METIS_TRY(check_nvfp4(a.fo)); if (a.fc->k_len != K || a.fo->k_len != M || !a.sigma) return METIS_ERR_SHAPE; }
+  if (kb) { METIS_TRY(check_nvfp4(b.fc)); METIS_TRY(check_nvfp4(b.fo)); if (b.fc->k_len != K || b.fo->k_len != N || !b.sigma) return METIS_ERR_SHAPE; }
+  unsigned char* w = reinterpret_cast<unsigned char*>(ws);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
+  float* y0 = reinterpret_cast<float*>(w + take(sizeof(float) * M * N));
+  float* g1 = reinterpret_cast<float*>(w + take(sizeof(float) * M * (kb ? kb : 1)));
+  float* wt = reinterpret_cast<float*>(w + take(sizeof(float) * N * (ka ? ka : 1)));
+  float* pm = reinterpret_cast<float*>(w + take(sizeof(float) * 64 * 64));
+  float* lcat = reinterpret_cast<float*>(w + take(sizeof(float) * M * kc));
+  float* rcat = reinterpret_cast<float*>(w + take(sizeof(float) * N * kc));
+  if (!ws || off > ws_bytes) return METIS_ERR_WORKSPACE;
+
+  METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.res, y0, METIS_FP32, N, s));
+  if (kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.fc, g1, METIS_FP32, kb, s));
+  if (ka) METIS_TRY(metis_launch_gemm_tc(ctx, b.res, a.fc, wt, METIS_FP32, ka, s));
+  if (ka && kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.fc, b.fc, pm, METIS_FP32, kb, s));
+  const int64_t mx = M > N ? M : N;
+  lowrank_prepare_kernel<<<(unsigned)metis_ceil_div(mx, 128), 128, 0, s>>>(
+      M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
+      ka ? a.fo->tensor_scale : nullptr, a.sigma, kb ? b.fo->codes : nullptr, kb ? b.fo->scales : nullptr,
+      kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, g1, wt, pm, lcat, rcat);
+  dim3 grid((unsigned)metis_ceil_div(N, 64), (unsigned)metis_ceil_div(M, 64));
+  const size_t smem = sizeof(float) * 2 * kc * 68;
+  static bool attr = false;
+  if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(rank_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 2 * 128 * 68))); attr = true; }
+  rank_update_kernel<<<grid, 256, smem, s>>>(y0, M, N, kc, lcat, rcat, d, d_dtype, ldd);
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
+
+}  // namespace
+
+size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k) {
+  const int kc = 2 * k;
+  return align256(sizeof(float) * M * N) + align256(sizeof(float) * M * (k ? k : 1)) +
+         align256(sizeof(float) * N * (k ? k : 1)) + align256(sizeof(float) * 64 * 64) +
+         align256(sizeof(float) * M * (kc ? kc : 1)) + align256(sizeof(float) * N * (kc ? kc : 1));
+}
+
+metis_status_t metis_linear_fwd(metis_handle_t h, const metis_operand_t* x, const metis_operand_t* w, void* y,
+                                int32_t y_dtype, int64_t ldy, void* ws, size_t ws_bytes, metis_stream_t stream) {
+  if (!h || !x || !w || !y) return METIS_ERR_INVALID_ARG;
+  if (x->cols != w->cols) return METIS_ERR_SHAPE;
+  // contraction over in-features: X (l x m) by columns, W_t (n x m) by columns
+  Side a{&x->res_by_cols, &x->right_q, &x->left_q, x->sigma, x->k};
+  Side b{&w->res_by_cols, &w->right_q, &w->left_q, w->sigma, w->k};
+  return split_gemm(h, a, b, y, y_dtype, ldy, ws, ws_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+metis_status_t metis_linear_bwd(metis_handle_t h, const metis_operand_t* dy, const metis_operand_t* x,
+                                const metis_operand_t* w, void* dx, int32_t dx_dtype, int64_t lddx, void* dw,
+                                int32_t dw_dtype, int64_t lddw, void* ws, size_t ws_bytes, metis_stream_t stream) {
+  if (!h || !dy) return METIS_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (dx) {
+    if (!w || dy->cols != w->rows) return METIS_ERR_SHAPE;
+    // dX (l x m) = D W_t, contraction over out-features n: D by columns, W_t by rows (stored m x n)
+    Side a{&dy->res_by_cols, &dy->right_q, &dy->left_q, dy->sigma, dy->k};
+    Side b{&w->res_by_rows, &w->left_q, &w->right_q, w->sigma, w->k};
+    METIS_TRY(split_gemm(h, a, b, dx, dx_dtype, lddx, ws, ws_bytes, s));
+  }
+  if (dw) {
+    if (!x || dy->rows != x->rows) return METIS_ERR_SHAPE;
+    // dW_t (n x m) = D^T X, contraction over tokens l: both by rows (stored n x l and m x l)
+    Side a{&dy->res_by_rows, &dy->left_q, &dy->right_q, dy->sigma, dy->k};
+    Side b{&x->res_by_rows, &x->left_q, &x->right_q, x->sigma, x->k};
+    METIS_TRY(split_gemm(h, a, b, dw, dw_dtype, lddw, ws, ws_bytes, s));
+  }
+  return METIS_OK;
+}

@@ -1,0 +1,188 @@
+// NVFP4 quantization of a 128 x 128 FP32 tile held in shared memory, in one or both block
+// orientations (Section 2.3).  Used by the stand-alone quantizer and by the fused
+// residual -> quantizer kernel of the split, so both produce identical codes for identical values.
+#pragma once
+#include "common.cuh"
+
+namespace metis_qt {
+
+constexpr int TILE = 128;
+constexpr int PITCH = 132;            // floats per shared-memory tile row (conflict-free float4 access by row)
+constexpr int THREADS = 256;
+
+struct QuantParams {
+  int64_t rows, cols;                 // source matrix extent
+  int rounding;
+  uint64_t seed;
+  uint32_t stream_id;
+  int64_t e_stride_r, e_stride_c;     // logical element index = r*e_stride_r + c*e_stride_c (keys the SR draw)
+  // outputs (either may be absent: codes == nullptr)
+  uint8_t* c_codes; uint8_t* c_scales; int c_layout;    // blocks along columns: stored rows x cols
+  uint8_t* r_codes; uint8_t* r_scales; int r_layout;    // blocks along rows:    stored cols x rows
+};
+
+struct __align__(16) Stage {
+  uint8_t codes[TILE][TILE / 2];      // 8 KiB: [stored row in tile][packed k]
+  uint8_t sf[TILE][TILE / 16];        // 1 KiB: [stored row in tile][block]
+};
+
+// Encodes one block of 16 values; returns the scale byte, writes 8 code bytes.
+__device__ __forceinline__ uint32_t encode_block(const float (&v)[16], const uint32_t (&u)[16], bool sr, float s_T,
+                                                 float six_s_T, uint32_t (&packed)[2]) {
+  float amax = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+  float t = fminf(__fdiv_rn(amax, six_s_T), 448.0f);
+  float sb;
+  const uint32_t byte = metis_e4m3_ceil(t, &sb);
+  const float r = sb == 0.0f ? 0.0f : __fdiv_rn(1.0f, __fmul_rn(sb, s_T));
+  packed[0] = packed[1] = 0u;
+  if (!sr) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const uint32_t b = metis_e2m1x2_rne(__fmul_rn(v[2 * i], r), __fmul_rn(v[2 * i + 1], r));
+      packed[i >> 2] |= b << (8 * (i & 3));
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint32_t c = metis_e2m1_sr(__fmul_rn(v[i], r), u[i]);
+      packed[i >> 3] |= c << (4 * (i & 7));
+    }
+  }
+  return byte;
+}
+
+// tile:  [TILE][PITCH] floats, rows/cols outside the matrix already zero-filled
+// rnd:   [TILE][TILE] 16-bit draws (only read when rounding == SR)
+// stage: scratch
+// All THREADS threads of the block must call this; contains __syncthreads().
+__device__ __forceinline__ void quantize_tile(const float* tile, const uint16_t* rnd, Stage* stage,
+                                              const QuantParams& p, int64_t row0, int64_t col0, float s_T) {
+  const int tid = threadIdx.x;
+  const bool sr = p.rounding == METIS_ROUND_SR;
+  const float six_s_T = __fmul_rn(6.0f, s_T);
+  const int vrows = (int)min((int64_t)TILE, p.rows - row0);
+  const int vcols = (int)min((int64_t)TILE, p.cols - col0);
+
+  if (p.c_codes != nullptr) {
+    // blocks along columns: thread -> (row = tid % 128, blocks b = tid/128 + 2*it)
+#pragma unroll 1
+    for (int it = 0; it < 4; ++it) {
+      const int r = tid & 127, b = (tid >> 7) + 2 * it;
+      float v[16];
+      uint32_t u[16];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float4 q = *reinterpret_cast<const float4*>(tile + r * PITCH + b * 16 + i * 4);
+        v[4 * i] = q.x; v[4 * i + 1] = q.y; v[4 * i + 2] = q.z; v[4 * i + 3] = q.w;
+      }
+      if (sr) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) u[i] = rnd[r * TILE + b * 16 + i];
+      }
+      uint32_t packed[2];
+      const uint32_t byte = encode_block(v, u, sr, s_T, six_s_T, packed);
+      *reinterpret_cast<uint2*>(&stage->codes[r][b * 8]) = make_uint2(packed[0], packed[1]);
+      stage->sf[r][b] = (uint8_t)byte;
+    }
+    __syncthreads();
+    // coalesced write-out
+    const int64_t kbytes = p.cols / 2;
+    for (int i = tid; i < TILE * 8; i += THREADS) {      // 8-byte units: one block of 16 codes each
+      const int r = i >> 3, seg = i & 7;
+      if (r < vrows && seg * 16 < vcols) {
+        *reinterpret_cast<uint2*>(p.c_codes + (row0 + r) * kbytes + col0 / 2 + seg * 8) =
+            *reinterpret_cast<const uint2*>(&stage->codes[r][seg * 8]);
+      }
+    }
+    const int64_t bpr = p.cols / 16;
+    for (int i = tid; i < TILE * 8; i += THREADS) {
+      int r, b;
+      if (p.c_layout == METIS_SF_TILED) {   // walk the two 512-byte atoms in storage order
+        const int atom = i >> 9, w = i & 511;
+        r = (w >> 4) + 32 * ((w >> 2) & 3);
+        b = atom * 4 + (w & 3);
+      } else {
+        r = i >> 3; b = i & 7;
+      }
+      if (b * 16 < vcols && (r < vrows || p.c_layout == METIS_SF_TILED)) {
+        const uint8_t val = r < vrows ? stage->sf[r][b] : (uint8_t)0;
+        p.c_scales[metis_sf_offset(row0 + r, col0 / 16 + b, bpr, p.c_layout)] = val;
+      }
+    }
+    __syncthreads();
+  }
+
+  if (p.r_codes != nullptr) {
+    // blocks along rows: stored row = source column.  thread -> (col = tid % 128, row-blocks b = tid/128 + 2*it)
+#pragma unroll 1
+    for (int it = 0; it < 4; ++it) {
+      const int c = tid & 127, b = (tid >> 7) + 2 * it;
+      float v[16];
+      uint32_t u[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) v[i] = tile[(b * 16 + i) * PITCH + c];
+      if (sr) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) u[i] = rnd[(b * 16 + i) * TILE + c];
+      }
+      uint32_t packed[2];
+      const uint32_t byte = encode_block(v, u, sr, s_T, six_s_T, packed);
+      *reinterpret_cast<uint2*>(&stage->codes[c][b * 8]) = make_uint2(packed[0], packed[1]);
+      stage->sf[c][b] = (uint8_t)byte;
+    }
+    __syncthreads();
+    const int64_t kbytes = p.rows / 2;
+    for (int i = tid; i < TILE * 8; i += THREADS) {
+      const int c = i >> 3, seg = i & 7;
+      if (c < vcols && seg * 16 < vrows) {
+        *reinterpret_cast<uint2*>(p.r_codes + (col0 + c) * kbytes + row0 / 2 + seg * 8) =
+            *reinterpret_cast<const uint2*>(&stage->codes[c][seg * 8]);
+      }
+    }
+    const int64_t bpr = p.rows / 16;
+    for (int i = tid; i < TILE * 8; i += THREADS) {
+      int c, b;
+      if (p.r_layout == METIS_SF_TILED) {
+        const int atom = i >> 9, w = i & 511;
+        c = (w >> 4) + 32 * ((w >> 2) & 3);
+        b = atom * 4 + (w & 3);
+      } else {
+        c = i >> 3; b = i & 7;
+      }
+      if (b * 16 < vrows && (c < vcols || p.r_layout == METIS_SF_TILED)) {
+        const uint8_t val = c < vcols ? stage->sf[c][b] : (uint8_t)0;
+        p.r_scales[metis_sf_offset(col0 + c, row0 / 16 + b, bpr, p.r_layout)] = val;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// Fills the tile's 16-bit draws.  Fast path: elements consecutive along a row share Philox counters.
+__device__ __forceinline__ void fill_draws(uint16_t* rnd, const QuantParams& p, int64_t row0, int64_t col0) {
+  const int tid = threadIdx.x;
+  if (p.e_stride_c == 1 && (p.e_stride_r & 7) == 0 && (col0 & 7) == 0) {
+    for (int i = tid; i < TILE * (TILE / 8); i += THREADS) {
+      const int r = i >> 4, g = i & 15;
+      const uint64_t e = (uint64_t)(row0 + r) * (uint64_t)p.e_stride_r + (uint64_t)(col0 + g * 8);
+      const uint4 w = metis_philox_block(e >> 3, p.seed, p.stream_id);
+      uint4 out;
+      out.x = w.x; out.y = w.y; out.z = w.z; out.w = w.w;   // halves in order: low half of word 0 first
+      *reinterpret_cast<uint4*>(rnd + r * TILE + g * 8) = out;
+    }
+  } else {
+    for (int i = tid; i < TILE * TILE; i += THREADS) {
+      const int r = i >> 7, c = i & 127;
+      const uint64_t e = (uint64_t)(row0 + r) * (uint64_t)p.e_stride_r + (uint64_t)(col0 + c) * (uint64_t)p.e_stride_c;
+      rnd[i] = (uint16_t)metis_draw_u16(e, p.seed, p.stream_id);
+    }
+  }
+}
+
+constexpr size_t smem_bytes(bool sr) {
+  return sizeof(float) * TILE * PITCH + sizeof(Stage) + (sr ? sizeof(uint16_t) * TILE * TILE : 0);
+}
+
+}  // namespace metis_qt

@@ -1,0 +1,91 @@
+"""GPU parity: the split-FP4 linear layer end to end (Eq. 2, Eq. 3, weight gradient) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import layer as olay, nvfp4 as onv, split as osp
+from paper_2509_00404_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3        # relative Frobenius error of layer outputs / gradients against the oracle's own split-FP4 result
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2509_00404_b200 import binding as B
+    h = B.Handle(0)
+    yield B, h
+    h.close()
+
+
+def _oracle_from_gpu_operand(op, k):
+    """Dequantize the library's own quantized pieces in float64 (isolates the GEMM composition from the split)."""
+    from gpu_util import nv_dequant
+    res_c = nv_dequant(op.res_by_cols) if op.res_by_cols else None
+    res_r = nv_dequant(op.res_by_rows).T if op.res_by_rows else None
+    if k == 0:
+        z = np.zeros((op.rows, op.cols))
+        return z, res_c, res_r
+    lq, rq = nv_dequant(op.left_q)[:k].T, nv_dequant(op.right_q)[:k].T
+    low = (lq * op.sigma.cpu().numpy().astype(np.float64)) @ rq.T
+    return low, res_c, res_r
+
+
+def test_small_config_forward(ctx):
+    from gpu_util import to_dev_bf16, rel_fro
+    B, h = ctx
+    c = synth.config_small()
+    xo = h.split(to_dev_bf16(c["x"]), 4, 4, sketch=B.SKETCH_FULL, seed=1)
+    wo = h.split(to_dev_bf16(c["w"]), 4, 4, sketch=B.SKETCH_FULL, seed=2)
+    y = h.linear_fwd(xo, wo)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    xq = olay.quantize_operand(c["x"], 4, 4, osp.MODE_FULL, 1)
+    wq = olay.quantize_operand(c["w"], 4, 4, osp.MODE_FULL, 2)
+    assert rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)) < TOL
+    # composition alone, on the library's own codes: tight
+    lx, rxc, _ = _oracle_from_gpu_operand(xo, 4)
+    lw, rwc, _ = _oracle_from_gpu_operand(wo, 4)
+    assert rel_fro(y.cpu().numpy(), (lx + rxc) @ (lw + rwc).T) < 2e-5
+
+
+@pytest.mark.parametrize("k", [0, 8])
+def test_forward_and_backward_medium(ctx, k):
+    from gpu_util import to_dev_bf16, rel_fro
+    B, h = ctx
+    l, m, n, p = 512, 384, 256, 8 if k else 0
+    x, _ = synth.llama_like(l, m, 1.0, 51, rank=8)
+    w, _ = synth.llama_like(n, m, 0.02, 52, rank=8)
+    d, _ = synth.llama_like(l, n, 1e-4, 53, rank=8)
+    xo = h.split(to_dev_bf16(x), k, p, sketch=B.SKETCH_SAMPLED, seed=1)
+    wo = h.split(to_dev_bf16(w), k, p, sketch=B.SKETCH_FULL, seed=2)
+    do = h.split(to_dev_bf16(d), k, p, sketch=B.SKETCH_SAMPLED, seed=3, rounding=B.ROUND_SR)
+    y = h.linear_fwd(xo, wo)
+    dx, dw = h.linear_bwd(do, xo, wo)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    xq = olay.quantize_operand(x, k, p, osp.MODE_SAMPLED, 1)
+    wq = olay.quantize_operand(w, k, p, osp.MODE_FULL, 2)
+    dq = olay.quantize_operand(d, k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
+    assert rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)) < TOL
+    assert rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)) < TOL
+    assert rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq)) < TOL
+    lx, rxc, rxr = _oracle_from_gpu_operand(xo, k)
+    lw, rwc, rwr = _oracle_from_gpu_operand(wo, k)
+    ld, rdc, rdr = _oracle_from_gpu_operand(do, k)
+    assert rel_fro(y.cpu().numpy(), (lx + rxc) @ (lw + rwc).T) < 2e-5
+    assert rel_fro(dx.cpu().numpy(), (ld + rdc) @ (lw + rwr)) < 2e-5
+    assert rel_fro(dw.cpu().numpy(), (ld + rdr).T @ (lx + rxr)) < 2e-5
+
+
+def test_bf16_output(ctx):
+    from gpu_util import to_dev_bf16, rel_fro
+    B, h = ctx
+    c = synth.config_small()
+    xo = h.split(to_dev_bf16(c["x"]), 4, 4, sketch=B.SKETCH_FULL, seed=1)
+    wo = h.split(to_dev_bf16(c["w"]), 4, 4, sketch=B.SKETCH_FULL, seed=2)
+    y32 = h.linear_fwd(xo, wo)
+    y16 = h.linear_fwd(xo, wo, out_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    assert rel_fro(y16.float().cpu().numpy(), y32.cpu().numpy()) < 4e-3

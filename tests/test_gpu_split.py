@@ -1,0 +1,101 @@
+"""GPU parity: metis_split (sketch, orthonormalisation, top-k projection, residual, quantization)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import nvfp4 as onv, split as osp, metrics
+from paper_2509_00404_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2509_00404_b200 import binding as B
+    h = B.Handle(0)
+    yield B, h
+    h.close()
+
+
+def _run(B, h, x, k, p, mode, seed, rounding=0):
+    from gpu_util import to_dev_bf16
+    op, dense = h.split(to_dev_bf16(x), k, p, sketch=mode, seed=seed, rounding=rounding, want_residual=True)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    return op, dense.cpu().numpy()
+
+
+def _check_against_oracle(B, h, x, k, p, mode, seed, rounding=0):
+    from gpu_util import nv_to_numpy, rel_fro
+    op, dense = _run(B, h, x, k, p, mode, seed, rounding)
+    sp = osp.split(x.astype(np.float64), k, p, mode, seed=seed)
+    sig = op.sigma.cpu().numpy()
+    assert np.max(np.abs(sig - sp.sigma) / sp.sigma) < 1e-3                 # top-k singular values
+    assert rel_fro(dense, sp.residual) < 1e-5                               # residual before quantization
+    left, right = op.left.cpu().numpy().T.astype(np.float64), op.right.cpu().numpy().T.astype(np.float64)
+    assert rel_fro(left, sp.left) < 1e-3 and rel_fro(right, sp.right) < 1e-3
+    # invariants that hold whatever the oracle says
+    assert np.allclose(left.T @ left, np.eye(k), atol=1e-4) and np.allclose(right.T @ right, np.eye(k), atol=1e-4)
+    assert rel_fro((left * sig) @ right.T + dense, x) < 1e-5
+    # the fused quantizer saw `dense`: the oracle's encoder on the same values must give the same bytes
+    s_src = onv.tensor_scale_from_amax(np.max(np.abs(x)))
+    for t, axis in ((op.res_by_cols, onv.AXIS_COLS), (op.res_by_rows, onv.AXIS_ROWS)):
+        c, s, ts = nv_to_numpy(t)
+        oc, os_, _ = onv.quantize(dense, axis, rounding, seed=seed, tensor_scale=s_src)
+        assert ts == s_src and np.array_equal(s, os_) and np.array_equal(c, oc)
+    # factors: quantized from the FP32 factors the library kept
+    for t, f, stream in ((op.left_q, op.left, 0x11), (op.right_q, op.right, 0x12)):
+        c, s, ts = nv_to_numpy(t)
+        oc, os_, ots = onv.quantize(f.cpu().numpy()[:k], onv.AXIS_COLS, rounding, seed=seed, stream=stream)
+        assert ts == ots and np.array_equal(s[:k], os_) and np.array_equal(c[:k], oc)
+    return op, sp
+
+
+def test_full_mode_small_config(ctx):
+    B, h = ctx
+    c = synth.config_small()
+    _check_against_oracle(B, h, c["x"], 4, 4, B.SKETCH_FULL, seed=11)
+    _check_against_oracle(B, h, c["w"], 4, 4, B.SKETCH_FULL, seed=12)
+
+
+def test_sampled_mode_and_stochastic_rounding(ctx):
+    B, h = ctx
+    x, _ = synth.llama_like(2048, 512, 1.0, 41, rank=16)
+    _check_against_oracle(B, h, x, 16, 8, B.SKETCH_SAMPLED, seed=21)
+    d, _ = synth.llama_like(1024, 384, 1e-4, 42, rank=8)
+    _check_against_oracle(B, h, d, 8, 8, B.SKETCH_SAMPLED, seed=22, rounding=1)
+
+
+def test_planted_noise_free_spectrum_is_recovered(ctx):
+    """Closed form: with no bulk and rank <= k+p the sketch captures the whole matrix, Lambda = planted values."""
+    B, h = ctx
+    x, s = synth.planted(128, 256, 8, 200.0, 20.0, 0.0, 1001)
+    op, dense = _run(B, h, x, 4, 4, B.SKETCH_FULL, seed=3)
+    s_true = np.linalg.svd(x.astype(np.float64), compute_uv=False)          # bf16 rounding moves the planted values slightly
+    assert np.max(np.abs(op.sigma.cpu().numpy() - s_true[:4]) / s_true[:4]) < 1e-5
+    x2, _ = synth.planted(2048, 256, 8, 50.0, 5.0, 0.0, 77)
+    op2, dense2 = _run(B, h, x2, 8, 4, B.SKETCH_SAMPLED, seed=9)           # rank-deficient sketch: k + p > rank
+    s2 = np.linalg.svd(x2.astype(np.float64), compute_uv=False)
+    assert np.max(np.abs(op2.sigma.cpu().numpy() - s2[:8]) / s2[:8]) < 1e-4
+    assert np.linalg.norm(dense2) < 2e-2 * np.linalg.norm(x2)               # only bf16 rounding noise is left
+
+
+def test_rank_zero_is_plain_quantization(ctx):
+    from gpu_util import to_dev_bf16, nv_to_numpy
+    B, h = ctx
+    c = synth.config_small()
+    op = h.split(to_dev_bf16(c["x"]), 0, 0, seed=5)
+    torch.cuda.synchronize()
+    for t, axis in ((op.res_by_cols, onv.AXIS_COLS), (op.res_by_rows, onv.AXIS_ROWS)):
+        cg, sg, ts = nv_to_numpy(t)
+        oc, os_, ots = onv.quantize(c["x"], axis)
+        assert ts == ots and np.array_equal(sg, os_) and np.array_equal(cg, oc)
+
+
+def test_workspace_and_shape_errors(ctx):
+    B, h = ctx
+    x = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.MetisError):
+        h.split(x, 60, 8)                      # k + p > 64
+    with pytest.raises(B.MetisError):
+        h.split(x, 6, 2)                       # k not a multiple of 4
