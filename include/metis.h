@@ -124,6 +124,9 @@ metis_status_t metis_last_device_status(metis_handle_t h, uint32_t* out, metis_s
  * matrix of the random projection is drawn through this table). */
 metis_status_t metis_debug_quantile_table(metis_handle_t h, uint16_t* host_out);
 
+/* Test / benchmark hook: kernels launched by the library in this process so far (host counter). */
+uint64_t metis_debug_launch_count(void);
+
 /* Bytes of scale storage for a stored rows x k_len NVFP4 tensor (host-only helper, no handle). */
 size_t metis_sf_bytes(int64_t rows, int64_t k_len, int32_t sf_layout);
 

@@ -25,6 +25,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "ALIGNMENT", 4: "WORKS
                 7: "NONFINITE", 8: "NUMERIC", 9: "TIMEOUT"}
 
 EXPORTED = ["metis_create", "metis_destroy", "metis_last_device_status", "metis_debug_quantile_table",
+            "metis_debug_launch_count",
             "metis_sf_bytes", "metis_workspace_bytes", "metis_default_sample_count", "metis_quantize_nvfp4",
             "metis_split", "metis_linear_fwd", "metis_linear_bwd", "metis_gemm_nvfp4"]
 
@@ -66,6 +67,8 @@ def lib():
     l.metis_destroy.argtypes = [vp]
     l.metis_last_device_status.argtypes = [vp, P(u32), vp]
     l.metis_debug_quantile_table.argtypes = [vp, vp]
+    l.metis_debug_launch_count.argtypes = []
+    l.metis_debug_launch_count.restype = u64
     l.metis_sf_bytes.argtypes = [i64, i64, i32]
     l.metis_sf_bytes.restype = sz
     l.metis_workspace_bytes.argtypes = [i32, i64, i64, i32, i32, P(sz)]
@@ -79,7 +82,7 @@ def lib():
                                    i64, vp, sz, vp]
     l.metis_gemm_nvfp4.argtypes = [vp, P(NvFp4Struct), P(NvFp4Struct), vp, i32, i64, i32, vp]
     for name in EXPORTED:
-        if name not in ("metis_sf_bytes", "metis_default_sample_count"):
+        if name not in ("metis_sf_bytes", "metis_default_sample_count", "metis_debug_launch_count"):
             getattr(l, name).restype = ctypes.c_int
     _lib = l
     return l
@@ -105,6 +108,10 @@ def _dtype_code(t):
     if t.dtype == torch.float32:
         return FP32
     raise TypeError("expected a bfloat16 or float32 tensor")
+
+
+def launch_count():
+    return int(lib().metis_debug_launch_count())
 
 
 def sf_bytes(rows, k_len, layout):
@@ -247,6 +254,21 @@ class Handle:
                                                 axes, ctypes.byref(st), _ptr(dense), _ptr(ws), ws.numel(),
                                                 _stream_ptr(stream)))
         return (op, dense) if want_residual else op
+
+    def requantize_weight(self, src, residual_bf16, out, rounding=ROUND_RNE, seed=0, stream=None):
+        """Weights held as (left, sigma, right, residual) and only re-quantized each step (Section 3.2 keeps the
+        low-rank and residual parts of a weight as separate stored tensors): three metis_quantize_nvfp4 calls."""
+        k = src.k
+        self.quantize_nvfp4(residual_bf16, BLOCKS_BOTH, rounding, seed, STREAM_RESIDUAL,
+                            out=(out.res_by_cols, out.res_by_rows), stream=stream)
+        if k:
+            self.quantize_nvfp4(src.left[:k], BLOCKS_ALONG_COLS, rounding, seed, STREAM_LEFT, out=(out.left_q, None), stream=stream)
+            self.quantize_nvfp4(src.right[:k], BLOCKS_ALONG_COLS, rounding, seed, STREAM_RIGHT, out=(out.right_q, None), stream=stream)
+            if out is not src:
+                out.left.copy_(src.left)
+                out.right.copy_(src.right)
+                out.sigma.copy_(src.sigma)
+        return out
 
     # -- metis_linear_fwd / metis_linear_bwd ---------------------------------------------------
     def linear_fwd(self, x_op, w_op, out_dtype=torch.float32, out=None, stream=None):

@@ -8,6 +8,8 @@
 size_t metis_split_ws_bytes(int64_t rows, int64_t cols, int k, int p);
 size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k);
 
+unsigned long long g_metis_launch_count = 0;
+
 namespace {
 
 // Standard normal quantile for 0 < p <= 0.5 by Newton iteration on the complementary error function,
@@ -87,6 +89,8 @@ metis_status_t metis_debug_quantile_table(metis_handle_t h, uint16_t* host_out) 
   METIS_CUDA_TRY(cudaMemcpy(host_out, h->quantile_lut, 65536 * sizeof(uint16_t), cudaMemcpyDeviceToHost));
   return METIS_OK;
 }
+
+uint64_t metis_debug_launch_count(void) { return g_metis_launch_count; }
 
 size_t metis_sf_bytes(int64_t rows, int64_t k_len, int32_t sf_layout) {
   if (rows <= 0 || k_len <= 0) return 0;

@@ -26,6 +26,10 @@ struct metis_context {
     if (s__ != METIS_OK) return s__;                 \
   } while (0)
 
+// Number of kernels the library has launched in this process (read through metis_debug_launch_count).
+extern unsigned long long g_metis_launch_count;
+#define METIS_COUNT_LAUNCH() (++g_metis_launch_count)
+
 static inline bool metis_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline int64_t metis_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 

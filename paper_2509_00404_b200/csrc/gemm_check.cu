@@ -85,7 +85,7 @@ metis_status_t metis_launch_gemm_check(const metis_nvfp4_t* a, const metis_nvfp4
   if (M == 0 || N == 0) return METIS_OK;
   dim3 grid((unsigned)metis_ceil_div(N, BN), (unsigned)metis_ceil_div(M, BM));
   gemm_check_kernel<<<grid, 256, 0, s>>>(a->codes, a->scales, a->tensor_scale, a->sf_layout, b->codes, b->scales,
-                                         b->tensor_scale, b->sf_layout, M, N, K, d, d_dtype, ldd);
+                                         b->tensor_scale, b->sf_layout, M, N, K, d, d_dtype, ldd); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }

@@ -353,7 +353,7 @@ metis_status_t launch(metis_context* ctx, const metis_nvfp4_t* a, const metis_nv
   }
   const int tiles = (int)(metis_ceil_div(g.M, BLOCK_M) * metis_ceil_div(g.N, BLOCK_N));
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-  gemm_nvfp4_kernel<BLOCK_N><<<grid, NUM_THREADS, C::SMEM_BYTES, s>>>(map_a, map_b, g);
+  gemm_nvfp4_kernel<BLOCK_N><<<grid, NUM_THREADS, C::SMEM_BYTES, s>>>(map_a, map_b, g); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }

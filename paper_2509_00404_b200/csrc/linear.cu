@@ -135,12 +135,12 @@ metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void
   lowrank_prepare_kernel<<<(unsigned)metis_ceil_div(mx, 128), 128, 0, s>>>(
       M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
       ka ? a.fo->tensor_scale : nullptr, a.sigma, kb ? b.fo->codes : nullptr, kb ? b.fo->scales : nullptr,
-      kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, g1, wt, pm, lcat, rcat);
+      kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, g1, wt, pm, lcat, rcat); METIS_COUNT_LAUNCH();
   dim3 grid((unsigned)metis_ceil_div(N, 64), (unsigned)metis_ceil_div(M, 64));
   const size_t smem = sizeof(float) * 2 * kc * 68;
   static bool attr = false;
   if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(rank_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 2 * 128 * 68))); attr = true; }
-  rank_update_kernel<<<grid, 256, smem, s>>>(y0, M, N, kc, lcat, rcat, d, d_dtype, ldd);
+  rank_update_kernel<<<grid, 256, smem, s>>>(y0, M, N, kc, lcat, rcat, d, d_dtype, ldd); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }

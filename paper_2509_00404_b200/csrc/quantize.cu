@@ -89,7 +89,7 @@ metis_status_t metis_launch_amax(const void* x, int dtype, int64_t rows, int64_t
   if (rows * cols == 0) return METIS_OK;
   const int64_t work = metis_ceil_div(rows * cols, 8 * 256);
   const int grid = (int)(work < 148 * 8 ? (work < 1 ? 1 : work) : 148 * 8);
-  amax_kernel<<<grid, 256, 0, s>>>(x, dtype, rows, cols, ld, amax_out);
+  amax_kernel<<<grid, 256, 0, s>>>(x, dtype, rows, cols, ld, amax_out); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }
@@ -115,7 +115,7 @@ metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int
   dim3 grid((unsigned)metis_ceil_div(cols, TILE), (unsigned)metis_ceil_div(rows, TILE));
   quantize_kernel<<<grid, THREADS, smem, s>>>(x, dtype, ld, p, tscale_src, tscale_is_amax,
                                               by_cols ? by_cols->tensor_scale : nullptr,
-                                              by_rows ? by_rows->tensor_scale : nullptr);
+                                              by_rows ? by_rows->tensor_scale : nullptr); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }

@@ -631,44 +631,44 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM)); attr = true; }
   }
   // (1) row sample, (2) sketch
-  sample_rows_kernel<<<(unsigned)metis_ceil_div(n_s, 256), 256, 0, s>>>(idx, (int)n_s, rows, seed, full ? 1 : 0);
+  sample_rows_kernel<<<(unsigned)metis_ceil_div(n_s, 256), 256, 0, s>>>(idx, (int)n_s, rows, seed, full ? 1 : 0); METIS_COUNT_LAUNCH();
   const int chunks = (int)metis_ceil_div(cols, SK_COLS);
   {
     const size_t smem = sizeof(float) * (SK_COLS * q + SK_ROWS * SK_COLS);
     static bool attr = false;
     if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(sketch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * (SK_COLS * MAXQ + SK_ROWS * SK_COLS)))); attr = true; }
     dim3 grid((unsigned)(n_s / SK_ROWS), (unsigned)chunks);
-    sketch_kernel<<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp);
+    sketch_kernel<<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp); METIS_COUNT_LAUNCH();
   }
-  reduce_partials_kernel<<<(unsigned)metis_ceil_div(n_s * q, 256), 256, 0, s>>>(zp, chunks, n_s * q, z);
+  reduce_partials_kernel<<<(unsigned)metis_ceil_div(n_s * q, 256), 256, 0, s>>>(zp, chunks, n_s * q, z); METIS_COUNT_LAUNCH();
   // (3) CholeskyQR2: orthonormal basis H of range(Z), in place
   for (int pass = 0; pass < 2; ++pass) {
     int64_t rpp; const int parts = gram_parts(n_s, &rpp);
-    gram_kernel<<<parts, 256, 0, s>>>(z, n_s, q, q, 1, rpp, gram);
-    cholqr_apply_kernel<<<(unsigned)metis_ceil_div(n_s, 128), 128, 0, s>>>(z, n_s, q, gram, parts, ctx->dev_status);
+    gram_kernel<<<parts, 256, 0, s>>>(z, n_s, q, q, 1, rpp, gram); METIS_COUNT_LAUNCH();
+    cholqr_apply_kernel<<<(unsigned)metis_ceil_div(n_s, 128), 128, 0, s>>>(z, n_s, q, gram, parts, ctx->dev_status); METIS_COUNT_LAUNCH();
   }
   // (4) M = H^T x[S,:], eigen-decomposition of M M^T, right basis
-  project_kernel<<<(unsigned)metis_ceil_div(cols, PJ_COLS), 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, m);
+  project_kernel<<<(unsigned)metis_ceil_div(cols, PJ_COLS), 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, m); METIS_COUNT_LAUNCH();
   {
     int64_t rpp; const int parts = gram_parts(cols, &rpp);
-    gram_kernel<<<parts, 256, 0, s>>>(m, cols, q, 1, cols, rpp, gram);
-    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram, parts, q, evals, evecs);
+    gram_kernel<<<parts, 256, 0, s>>>(m, cols, q, 1, cols, rpp, gram); METIS_COUNT_LAUNCH();
+    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram, parts, q, evals, evecs); METIS_COUNT_LAUNCH();
   }
   right_basis_kernel<<<(unsigned)metis_ceil_div(cols, 256), 256, 0, s>>>(m, cols, q, k, evals, evecs, basis,
-                                                                          full ? out->sigma : nullptr);
+                                                                          full ? out->sigma : nullptr); METIS_COUNT_LAUNCH();
   // (5) factors
   const float* res_coef; const float* res_scale; const float* res_basis;
   if (full) {
     // left = H U~_k, right = basis; residual against left * sigma * right^T
-    right_rotate_sign_kernel<<<k, 256, 0, s>>>(basis, cols, k, nullptr, out->right, sign);
+    right_rotate_sign_kernel<<<k, 256, 0, s>>>(basis, cols, k, nullptr, out->right, sign); METIS_COUNT_LAUNCH();
     left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 256), 256, 0, s>>>(z, rows, q, k, 1, q, evecs, nullptr, sign,
-                                                                           out->left, nullptr);
+                                                                           out->left, nullptr); METIS_COUNT_LAUNCH();
     res_coef = out->left; res_scale = out->sigma; res_basis = out->right;
   } else {
     const size_t smem = sizeof(float) * (CF_ROWS + k) * (CF_COLS + 1);
     static bool attr = false;
     if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * (CF_ROWS + MAXQ) * (CF_COLS + 1)))); attr = true; }
-    coeff_kernel<<<(unsigned)metis_ceil_div(rows, CF_ROWS), 256, smem, s>>>(x, rows, cols, k, basis, coef);
+    coeff_kernel<<<(unsigned)metis_ceil_div(rows, CF_ROWS), 256, smem, s>>>(x, rows, cols, k, basis, coef); METIS_COUNT_LAUNCH();
     res_coef = coef; res_scale = nullptr; res_basis = basis;
   }
   // (6) fused residual + quantizer (tensor scale from the source tensor's amax)
@@ -685,16 +685,16 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     dim3 grid((unsigned)metis_ceil_div(cols, TILE), (unsigned)metis_ceil_div(rows, TILE));
     residual_quant_kernel<<<grid, THREADS, smem, s>>>(x, k, res_coef, res_scale, res_basis, qp, amax,
                                                       want_c ? rc.tensor_scale : nullptr,
-                                                      want_r ? rr.tensor_scale : nullptr, residual_dense);
+                                                      want_r ? rr.tensor_scale : nullptr, residual_dense); METIS_COUNT_LAUNCH();
   }
   if (!full) {
     // (7) Rayleigh-Ritz on C^T C, rotate both factors, singular values
     int64_t rpp; const int parts = gram_parts(rows, &rpp);
-    gram_kernel<<<parts, 256, 0, s>>>(coef, rows, k, 1, rows, rpp, gram);
-    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram, parts, k, evals2, evecs2);
-    right_rotate_sign_kernel<<<k, 256, 0, s>>>(basis, cols, k, evecs2, out->right, sign);
+    gram_kernel<<<parts, 256, 0, s>>>(coef, rows, k, 1, rows, rpp, gram); METIS_COUNT_LAUNCH();
+    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram, parts, k, evals2, evecs2); METIS_COUNT_LAUNCH();
+    right_rotate_sign_kernel<<<k, 256, 0, s>>>(basis, cols, k, evecs2, out->right, sign); METIS_COUNT_LAUNCH();
     left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 256), 256, 0, s>>>(coef, rows, k, k, rows, 1, evecs2, evals2, sign,
-                                                                           out->left, out->sigma);
+                                                                           out->left, out->sigma); METIS_COUNT_LAUNCH();
   }
   METIS_CUDA_TRY(cudaGetLastError());
   // (8) quantize the factors (stored transposed: k x rows, k x cols; blocks along the long dimension)
