@@ -21,31 +21,40 @@ __device__ __forceinline__ float deq_at(const uint8_t* codes, const uint8_t* sf,
   return metis_e2m1_value(code) * metis_e4m3_value(sf[metis_sf_offset(r, c / 16, k_len / 16, layout)]);
 }
 
-// Lcat [M][kb + ka], Rcat [N][kb + ka]
-__global__ void lowrank_prepare_kernel(int64_t M, int64_t N, int ka, int kb,
-                                       const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts,
-                                       const float* sa,
-                                       const uint8_t* fob_codes, const uint8_t* fob_sf, int fob_layout, const float* fob_ts,
-                                       const float* sb,
-                                       const float* __restrict__ g1, const float* __restrict__ wt, const float* __restrict__ pm,
-                                       float* __restrict__ lcat, float* __restrict__ rcat) {
+// Finishes the two skinny operands of the rank-(ka+kb) update, in place.  Layout: Lcat [M][kb + ka],
+// Rcat [N][kb + ka].  On entry Lcat[:, :kb] holds G1 and Rcat[:, kb:] holds Wt (written there by the skinny
+// GEMMs).  On exit  Lcat[:, :kb] = (G1 + Fo_a sa P) sb,  Lcat[:, kb:] = Fo_a sa,  Rcat[:, :kb] = Fo_b.
+// One warp per row.
+__global__ void __launch_bounds__(256)
+lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
+                      const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts,
+                      const float* sa,
+                      const uint8_t* fob_codes, const uint8_t* fob_sf, int fob_layout, const float* fob_ts,
+                      const float* sb, const float* __restrict__ pm, float* __restrict__ lcat, float* __restrict__ rcat) {
+  __shared__ float ps[64][65];
+  __shared__ float fa[8][64];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int kc = ka + kb;
-  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  for (int o = tid; o < ka * kb; o += 256) ps[o / kb][o % kb] = pm[o];
+  __syncthreads();
+  const int64_t i = (int64_t)blockIdx.x * 8 + warp;
   if (i < M) {
-    float fa[64];
     const float tsa = ka ? *foa_ts : 0.0f;
-    for (int u = 0; u < ka; ++u) fa[u] = deq_at(foa_codes, foa_sf, foa_layout, M, u, i) * tsa * sa[u];
-    for (int t = 0; t < kb; ++t) {
-      float v = g1[i * kb + t];
-      for (int u = 0; u < ka; ++u) v = fmaf(fa[u], pm[u * kb + t], v);
+    for (int u = lane; u < ka; u += 32) {
+      const float v = deq_at(foa_codes, foa_sf, foa_layout, M, u, i) * tsa * sa[u];
+      fa[warp][u] = v;
+      lcat[i * kc + kb + u] = v;
+    }
+    __syncwarp();
+    for (int t = lane; t < kb; t += 32) {
+      float v = lcat[i * kc + t];
+      for (int u = 0; u < ka; ++u) v = fmaf(fa[warp][u], ps[u][t], v);
       lcat[i * kc + t] = v * sb[t];
     }
-    for (int u = 0; u < ka; ++u) lcat[i * kc + kb + u] = fa[u];
   }
   if (i < N) {
     const float tsb = kb ? *fob_ts : 0.0f;
-    for (int t = 0; t < kb; ++t) rcat[i * kc + t] = deq_at(fob_codes, fob_sf, fob_layout, N, t, i) * tsb;
-    for (int u = 0; u < ka; ++u) rcat[i * kc + kb + u] = wt[i * ka + u];
+    for (int t = lane; t < kb; t += 32) rcat[i * kc + t] = deq_at(fob_codes, fob_sf, fob_layout, N, t, i) * tsb;
   }
 }
 
@@ -120,22 +129,21 @@ metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
   float* y0 = reinterpret_cast<float*>(w + take(sizeof(float) * M * N));
-  float* g1 = reinterpret_cast<float*>(w + take(sizeof(float) * M * (kb ? kb : 1)));
-  float* wt = reinterpret_cast<float*>(w + take(sizeof(float) * N * (ka ? ka : 1)));
   float* pm = reinterpret_cast<float*>(w + take(sizeof(float) * 64 * 64));
   float* lcat = reinterpret_cast<float*>(w + take(sizeof(float) * M * kc));
   float* rcat = reinterpret_cast<float*>(w + take(sizeof(float) * N * kc));
   if (!ws || off > ws_bytes) return METIS_ERR_WORKSPACE;
 
   METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.res, y0, METIS_FP32, N, s));
-  if (kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.fc, g1, METIS_FP32, kb, s));
-  if (ka) METIS_TRY(metis_launch_gemm_tc(ctx, b.res, a.fc, wt, METIS_FP32, ka, s));
+  // the skinny products land directly in their slots of the concatenated operands
+  if (kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.fc, lcat, METIS_FP32, kc, s));
+  if (ka) METIS_TRY(metis_launch_gemm_tc(ctx, b.res, a.fc, rcat + kb, METIS_FP32, kc, s));
   if (ka && kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.fc, b.fc, pm, METIS_FP32, kb, s));
   const int64_t mx = M > N ? M : N;
-  lowrank_prepare_kernel<<<(unsigned)metis_ceil_div(mx, 128), 128, 0, s>>>(
+  lowrank_finish_kernel<<<(unsigned)metis_ceil_div(mx, 8), 256, 0, s>>>(
       M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
       ka ? a.fo->tensor_scale : nullptr, a.sigma, kb ? b.fo->codes : nullptr, kb ? b.fo->scales : nullptr,
-      kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, g1, wt, pm, lcat, rcat); METIS_COUNT_LAUNCH();
+      kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, pm, lcat, rcat); METIS_COUNT_LAUNCH();
   dim3 grid((unsigned)metis_ceil_div(N, 64), (unsigned)metis_ceil_div(M, 64));
   const size_t smem = sizeof(float) * 2 * kc * 68;
   static bool attr = false;
@@ -149,8 +157,7 @@ metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void
 
 size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k) {
   const int kc = 2 * k;
-  return align256(sizeof(float) * M * N) + align256(sizeof(float) * M * (k ? k : 1)) +
-         align256(sizeof(float) * N * (k ? k : 1)) + align256(sizeof(float) * 64 * 64) +
+  return align256(sizeof(float) * M * N) + align256(sizeof(float) * 64 * 64) +
          align256(sizeof(float) * M * (kc ? kc : 1)) + align256(sizeof(float) * N * (kc ? kc : 1));
 }
 

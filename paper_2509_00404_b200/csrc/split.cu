@@ -24,13 +24,14 @@ __global__ void sample_rows_kernel(int* __restrict__ idx, int n_s, int64_t rows,
 
 // ------------------------------------------------------------------------------------------------
 // Sketch partials: Zp[chunk][row][j] = sum over the chunk's 256 columns of x[idx[row], col] * Omega[col, j].
-constexpr int SK_ROWS = 16, SK_COLS = 256;
+// One CTA: 64 sampled rows x 256 columns; Omega's 256 x q slice is generated once per CTA into shared memory.
+constexpr int SK_ROWS = 64, SK_COLS = 256, SK_PITCH = SK_COLS + 4;
 __global__ void __launch_bounds__(256)
 sketch_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
               uint64_t seed, const __nv_bfloat16* __restrict__ lut, float* __restrict__ zp) {
   extern __shared__ __align__(16) unsigned char smem[];
-  float* om = reinterpret_cast<float*>(smem);                  // [SK_COLS * q]
-  float* xs = om + SK_COLS * q;                                // [SK_ROWS][SK_COLS]
+  float* om = reinterpret_cast<float*>(smem);                  // [SK_COLS][q]
+  float* xs = om + SK_COLS * MAXQ;                             // [SK_ROWS][SK_PITCH]
   const int tid = threadIdx.x;
   const int64_t col0 = (int64_t)blockIdx.y * SK_COLS;
   const int row0 = blockIdx.x * SK_ROWS;
@@ -45,17 +46,48 @@ sketch_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __re
       if (e >= e_lo && e < e_hi) om[e - e_lo] = __bfloat162float(lut[metis_u16_of(w, h)]);
     }
   }
-  for (int i = tid; i < SK_ROWS * SK_COLS; i += 256) {
-    const int r = i / SK_COLS, c = i % SK_COLS;
-    xs[i] = (row0 + r < n_s && c < ncols) ? __bfloat162float(x[(int64_t)idx[row0 + r] * cols + col0 + c]) : 0.0f;
+  for (int i = tid; i < SK_ROWS * (SK_COLS / 8); i += 256) {
+    const int r = i >> 5, g = i & 31;
+    float v[8];
+    if (row0 + r < n_s && g * 8 + 8 <= ncols) {
+      const uint4 qv = *reinterpret_cast<const uint4*>(x + (int64_t)idx[row0 + r] * cols + col0 + g * 8);
+      const uint32_t w[4] = {qv.x, qv.y, qv.z, qv.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { v[2 * j] = __uint_as_float(w[j] << 16); v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u); }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        v[j] = (row0 + r < n_s && g * 8 + j < ncols) ? __bfloat162float(x[(int64_t)idx[row0 + r] * cols + col0 + g * 8 + j]) : 0.0f;
+    }
+    *reinterpret_cast<float4*>(xs + r * SK_PITCH + g * 8) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(xs + r * SK_PITCH + g * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
   }
   __syncthreads();
-  for (int o = tid; o < SK_ROWS * q; o += 256) {
-    const int r = o / q, j = o % q;
-    float acc = 0.0f;
-    for (int t = 0; t < ncols; ++t) acc = fmaf(xs[r * SK_COLS + t], om[t * q + j], acc);
-    if (row0 + r < n_s) zp[((int64_t)blockIdx.y * n_s + row0 + r) * q + j] = acc;
+  // thread -> rows tr*4 .. +3, sketch columns tj, tj+16, tj+32, tj+48
+  const int tr = tid >> 4, tj = tid & 15;
+  float acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0f;
+  for (int t = 0; t < ncols; ++t) {
+    float xv[4], ov[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) xv[a] = xs[(tr * 4 + a) * SK_PITCH + t];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) ov[b] = (tj + 16 * b < q) ? om[t * q + tj + 16 * b] : 0.0f;
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(xv[a], ov[b], acc[a][b]);
   }
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int r = row0 + tr * 4 + a, j = tj + 16 * b;
+      if (r < n_s && j < q) zp[((int64_t)blockIdx.y * n_s + r) * q + j] = acc[a][b];
+    }
 }
 
 __global__ void reduce_partials_kernel(const float* __restrict__ zp, int n_chunks, int64_t n, float* __restrict__ z) {
@@ -108,177 +140,231 @@ gram_kernel(const float* __restrict__ v, int64_t n_rows, int n, int64_t stride_r
 }
 
 // ------------------------------------------------------------------------------------------------
-// One CholeskyQR pass: G = sum of Gram partials = L L^T (FP64, in shared memory, every CTA redundantly),
-// then z_row <- z_row L^-T for the CTA's rows.  A pivot below 1e-13 of the largest diagonal marks a
-// dependent sketch column: its output column becomes zero instead of amplified noise.
-__global__ void __launch_bounds__(128)
-cholqr_apply_kernel(float* __restrict__ z, int64_t n_rows, int q, const double* __restrict__ part, int n_parts,
-                    uint32_t* dev_status) {
+__device__ __forceinline__ double chol_rsqrt(double x) {
+  // scale into the FP32 range by an even power of two, seed with rsqrtf, two Newton steps in FP64
+  int e;
+  const double mant = frexp(x, &e);                     // x = mant * 2^e, mant in [0.5, 1)
+  const int e2 = e & ~1;
+  const double xs = ldexp(mant, e - e2);                // in [0.5, 2)
+  double y = (double)rsqrtf((float)xs);
+  y = y * (1.5 - 0.5 * xs * y * y);
+  y = y * (1.5 - 0.5 * xs * y * y);
+  return ldexp(y, -(e2 / 2));
+}
+
+// One CholeskyQR pass, step 1 (one CTA): G (one Gram partial) = L L^T in FP64; writes L (q x q, row-major,
+// upper part unused) and the reciprocal pivots.  A pivot below 1e-13 of the largest diagonal marks a
+// dependent sketch column: its reciprocal is stored as zero, so the corresponding column of H = Z L^-T
+// becomes zero instead of amplified noise.
+__global__ void __launch_bounds__(256)
+chol_kernel(const double* __restrict__ g, int q, double* __restrict__ l_out, double* __restrict__ invd_out) {
   __shared__ double L[MAXQ][MAXQ + 1];
-  __shared__ double invd[MAXQ];
   __shared__ double gmax_s;
-  const int tid = threadIdx.x;
-  for (int o = tid; o < q * q; o += 128) {
-    double s = 0.0;
-    for (int p = 0; p < n_parts; ++p) s += part[(int64_t)p * q * q + o];
-    L[o / q][o % q] = s;
-  }
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  for (int o = tid; o < q * q; o += 256) L[o / q][o % q] = g[o];
   __syncthreads();
-  if (tid == 0) {
-    double g = 0.0;
-    for (int i = 0; i < q; ++i) g = fmax(g, L[i][i]);
-    gmax_s = g;
+  if (tid < 32) {
+    double gm = 0.0;
+    for (int i = tid; i < q; i += 32) gm = fmax(gm, L[i][i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) gm = fmax(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, o));
+    if (tid == 0) gmax_s = gm;
   }
   __syncthreads();
   const double tol = 1e-13 * gmax_s;
   for (int j = 0; j < q; ++j) {
     const double d = L[j][j];
     const bool dep = !(d > tol);
+    const double inv = dep ? 0.0 : chol_rsqrt(d);
     __syncthreads();
-    if (dep) {
-      for (int i = j + tid; i < q; i += 128) L[i][j] = 0.0;
-      if (tid == 0) invd[j] = 0.0;
-    } else {
-      const double ljj = sqrt(d);
-      for (int i = j + 1 + tid; i < q; i += 128) L[i][j] /= ljj;
-      if (tid == 0) { L[j][j] = ljj; invd[j] = 1.0 / ljj; }
-    }
+    for (int i = j + 1 + tid; i < q; i += 256) L[i][j] *= inv;
+    if (tid == 0) { L[j][j] = dep ? 0.0 : d * inv; invd_out[j] = inv; }
     __syncthreads();
     if (!dep) {
-      const int m = q - j - 1;
-      for (int o = tid; o < m * m; o += 128) {
-        const int a = j + 1 + o / m, b = j + 1 + o % m;
-        if (b <= a) L[a][b] -= L[a][j] * L[b][j];
+      for (int a = j + 1 + ty; a < q; a += 16) {
+        const double laj = L[a][j];
+        for (int b = j + 1 + tx; b <= a; b += 16) L[a][b] -= laj * L[b][j];
       }
     }
     __syncthreads();
   }
-  const int64_t r = (int64_t)blockIdx.x * 128 + tid;
-  if (r < n_rows) {
-    double h[MAXQ];
-    for (int j = 0; j < q; ++j) {
-      double s = (double)z[r * q + j];
-      for (int i = 0; i < j; ++i) s -= h[i] * L[j][i];
-      h[j] = s * invd[j];
-    }
-    for (int j = 0; j < q; ++j) z[r * q + j] = (float)h[j];
+  for (int o = tid; o < q * q; o += 256) l_out[o] = L[o / q][o % q];
+}
+
+// One CholeskyQR pass, step 2: z_row <- z_row L^-T by forward substitution, one warp per row:
+// h_j = (z_j - sum_{i<j} h_i L[j][i]) / L[j][j]; lane i%32 keeps h_i, the dot product is a warp reduction.
+__global__ void __launch_bounds__(256)
+apply_chol_kernel(float* __restrict__ z, int64_t n_rows, int q, const double* __restrict__ l, const double* __restrict__ invd) {
+  __shared__ double L[MAXQ][MAXQ + 1];
+  __shared__ double inv_s[MAXQ];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int o = tid; o < q * q; o += 256) L[o / q][o % q] = l[o];
+  if (tid < q) inv_s[tid] = invd[tid];
+  __syncthreads();
+  const int64_t r = (int64_t)blockIdx.x * 8 + warp;
+  if (r >= n_rows) return;
+  double h0 = 0.0, h1 = 0.0;                         // h_lane, h_(lane+32)
+  const double z0 = lane < q ? (double)z[r * q + lane] : 0.0;
+  const double z1 = lane + 32 < q ? (double)z[r * q + lane + 32] : 0.0;
+  for (int j = 0; j < q; ++j) {
+    double part = 0.0;
+    if (lane < j) part += h0 * L[j][lane];
+    if (lane + 32 < j) part += h1 * L[j][lane + 32];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+    const double zj = __shfl_sync(0xFFFFFFFFu, j < 32 ? z0 : z1, j & 31);
+    const double hj = (zj - part) * inv_s[j];
+    if (lane == (j & 31)) { if (j < 32) h0 = hj; else h1 = hj; }
   }
-  (void)dev_status;
+  if (lane < q) z[r * q + lane] = (float)h0;
+  if (lane + 32 < q) z[r * q + lane + 32] = (float)h1;
 }
 
 // ------------------------------------------------------------------------------------------------
-// M[j][col] = sum_r H[r][j] * x[idx[r], col]     (q x cols, row j contiguous)
-constexpr int PJ_COLS = 128, PJ_ROWS = 32;
+// Projection partials: Mp[part][j][col] = sum over the part's sampled rows r of H[r][j] * x[idx[r], col]
+// (q x cols per part, row j contiguous).  Thread: two adjacent columns, every second sketch column.
+constexpr int PJ_COLS = 256, PJ_ROWS = 32;
+template <int NJ4>                                                  // float4 groups of sketch columns per thread
 __global__ void __launch_bounds__(256)
 project_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
-               const float* __restrict__ h, float* __restrict__ m) {
-  __shared__ float hs[PJ_ROWS][MAXQ];
-  const int tid = threadIdx.x, c = tid & (PJ_COLS - 1), jg = tid >> 7;       // 2 groups of factor indices
-  const int64_t col = (int64_t)blockIdx.x * PJ_COLS + c;
-  float acc[MAXQ / 2];
+               const float* __restrict__ h, int rows_per_part, float* __restrict__ mp) {
+  __shared__ __align__(16) float hs[2][PJ_ROWS][MAXQ / 2];
+  __shared__ int ids[PJ_ROWS];
+  const int tid = threadIdx.x, c2 = tid & 127, jg = tid >> 7;       // jg: sketch columns 2*j + jg
+  const int64_t col = (int64_t)blockIdx.x * PJ_COLS + c2 * 2;
+  const int r_begin = blockIdx.y * rows_per_part, r_end = min(n_s, r_begin + rows_per_part);
+  float acc0[NJ4 * 4], acc1[NJ4 * 4];
 #pragma unroll
-  for (int j = 0; j < MAXQ / 2; ++j) acc[j] = 0.0f;
-  for (int r0 = 0; r0 < n_s; r0 += PJ_ROWS) {
-    for (int i = tid; i < PJ_ROWS * q; i += 256) {
-      const int rr = i / q, jj = i % q;
-      hs[rr][jj] = (r0 + rr < n_s) ? h[(int64_t)(r0 + rr) * q + jj] : 0.0f;
+  for (int j = 0; j < NJ4 * 4; ++j) { acc0[j] = 0.0f; acc1[j] = 0.0f; }
+  for (int r0 = r_begin; r0 < r_end; r0 += PJ_ROWS) {
+    for (int i = tid; i < PJ_ROWS * MAXQ; i += 256) {
+      const int rr = i / MAXQ, jj = i % MAXQ;
+      hs[jj & 1][rr][jj >> 1] = (r0 + rr < r_end && jj < q) ? h[(int64_t)(r0 + rr) * q + jj] : 0.0f;
     }
+    if (tid < PJ_ROWS) ids[tid] = (r0 + tid < r_end) ? idx[r0 + tid] : 0;
     __syncthreads();
-    const int nr = min(PJ_ROWS, n_s - r0);
+    const int nr = min(PJ_ROWS, r_end - r0);
     for (int rr = 0; rr < nr; ++rr) {
-      const float xv = col < cols ? __bfloat162float(x[(int64_t)idx[r0 + rr] * cols + col]) : 0.0f;
+      float x0 = 0.0f, x1 = 0.0f;
+      if (col + 1 < cols) {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(x + (int64_t)ids[rr] * cols + col);
+        x0 = __uint_as_float(w << 16); x1 = __uint_as_float(w & 0xFFFF0000u);
+      } else if (col < cols) {
+        x0 = __bfloat162float(x[(int64_t)ids[rr] * cols + col]);
+      }
 #pragma unroll
-      for (int j = 0; j < MAXQ / 2; ++j)
-        if (2 * j + jg < q) acc[j] = fmaf(hs[rr][2 * j + jg], xv, acc[j]);
+      for (int j4 = 0; j4 < NJ4; ++j4) {
+        const float4 hv = *reinterpret_cast<const float4*>(&hs[jg][rr][j4 * 4]);
+        acc0[j4 * 4 + 0] = fmaf(hv.x, x0, acc0[j4 * 4 + 0]); acc1[j4 * 4 + 0] = fmaf(hv.x, x1, acc1[j4 * 4 + 0]);
+        acc0[j4 * 4 + 1] = fmaf(hv.y, x0, acc0[j4 * 4 + 1]); acc1[j4 * 4 + 1] = fmaf(hv.y, x1, acc1[j4 * 4 + 1]);
+        acc0[j4 * 4 + 2] = fmaf(hv.z, x0, acc0[j4 * 4 + 2]); acc1[j4 * 4 + 2] = fmaf(hv.z, x1, acc1[j4 * 4 + 2]);
+        acc0[j4 * 4 + 3] = fmaf(hv.w, x0, acc0[j4 * 4 + 3]); acc1[j4 * 4 + 3] = fmaf(hv.w, x1, acc1[j4 * 4 + 3]);
+      }
     }
     __syncthreads();
   }
-  if (col < cols)
+  float* dst = mp + (int64_t)blockIdx.y * q * cols;
 #pragma unroll
-    for (int j = 0; j < MAXQ / 2; ++j)
-      if (2 * j + jg < q) m[(int64_t)(2 * j + jg) * cols + col] = acc[j];
+  for (int j = 0; j < NJ4 * 4; ++j)
+    if (2 * j + jg < q) {
+      if (col < cols) dst[(int64_t)(2 * j + jg) * cols + col] = acc0[j];
+      if (col + 1 < cols) dst[(int64_t)(2 * j + jg) * cols + col + 1] = acc1[j];
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
 // Symmetric eigen-decomposition (n <= 64) by parallel-order cyclic Jacobi in FP64, one CTA.
-// Input: Gram partials.  Output: eigenvalues descending, eigenvectors as columns of vec[n][n].
-__global__ void __launch_bounds__(256)
-jacobi_eig_kernel(const double* __restrict__ part, int n_parts, int n, double* __restrict__ evals,
+// Each round pairs the indices into n/2 disjoint (p, q) couples (round-robin tournament); thread (I, J)
+// owns the 2 x 2 block (rows of couple I, columns of couple J), so one round is: rotation angles from
+// the diagonal blocks, then every thread applies J_I^T . block . J_J in registers - two barriers a round.
+// Input: Gram matrix (ld x ld, leading n x n block used).  Output: eigenvalues descending,
+// eigenvectors as columns of evecs[n][n].
+__device__ __forceinline__ void jacobi_pair(int I, int step, int np, int* p, int* q) {
+  int a, b;
+  if (I == 0) { a = 0; b = (step % (np - 1)) + 1; }
+  else { a = ((step + I) % (np - 1)) + 1; b = ((step + np - 1 - I) % (np - 1)) + 1; }
+  *p = min(a, b); *q = max(a, b);
+}
+
+// 1/sqrt(x) in FP64 from an FP32 seed and two Newton steps (x in the FP32 range; relative error ~1e-16).
+__device__ __forceinline__ double fast_rsqrt(double x) {
+  double y = (double)rsqrtf((float)x);
+  y = y * (1.5 - 0.5 * x * y * y);
+  y = y * (1.5 - 0.5 * x * y * y);
+  return y;
+}
+
+__global__ void __launch_bounds__(1024)
+jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, double* __restrict__ evals,
                   double* __restrict__ evecs) {
   extern __shared__ __align__(16) unsigned char jsm[];
   double (*A)[MAXQ + 1] = reinterpret_cast<double (*)[MAXQ + 1]>(jsm);
   double (*V)[MAXQ + 1] = reinterpret_cast<double (*)[MAXQ + 1]>(jsm + sizeof(double) * MAXQ * (MAXQ + 1));
   __shared__ double cs[MAXQ / 2][2];
-  __shared__ int pr[MAXQ / 2][2];
-  __shared__ double red[2];
+  __shared__ double red[2][32];
   __shared__ int order[MAXQ];
-  const int tid = threadIdx.x;
-  for (int o = tid; o < n * n; o += 256) {
-    double s = 0.0;
-    for (int p = 0; p < n_parts; ++p) s += part[(int64_t)p * n * n + o];
-    A[o / n][o % n] = s;
-    V[o / n][o % n] = (o / n == o % n) ? 1.0 : 0.0;
-  }
-  __syncthreads();
-  for (int o = tid; o < n * n; o += 256) {            // symmetrise (partials are symmetric up to summation order)
-    const int i = o / n, j = o % n;
-    if (i < j) { const double s = 0.5 * (A[i][j] + A[j][i]); A[i][j] = s; A[j][i] = s; }
-  }
-  __syncthreads();
+  __shared__ uint8_t pairs[MAXQ][MAXQ / 2][2];          // [round][couple] -> (p, q)
+  const int tid = threadIdx.x, nthr = blockDim.x;
   const int np = n + (n & 1), half = np / 2;
-  for (int sweep = 0; sweep < 14; ++sweep) {
-    if (tid == 0) {
-      double off = 0.0, dg = 0.0;
-      for (int i = 0; i < n; ++i) {
-        dg += A[i][i] * A[i][i];
-        for (int j = i + 1; j < n; ++j) off += A[i][j] * A[i][j];
-      }
-      red[0] = off; red[1] = dg;
+  for (int o = tid; o < np * np; o += nthr) {
+    const int i = o / np, j = o % np;
+    A[i][j] = (i < n && j < n) ? 0.5 * (g[i * ld + j] + g[j * ld + i]) : 0.0;
+    V[i][j] = (i == j) ? 1.0 : 0.0;
+  }
+  for (int o = tid; o < (np - 1) * half; o += nthr) {
+    int p, q;
+    jacobi_pair(o % half, o / half, np, &p, &q);
+    pairs[o / half][o % half][0] = (uint8_t)p; pairs[o / half][o % half][1] = (uint8_t)q;
+  }
+  __syncthreads();
+  const bool active = tid < half * half;
+  const int I = active ? tid / half : 0, J = active ? tid % half : 0;
+  for (int sweep = 0; sweep < 12; ++sweep) {
+    // convergence: off-diagonal energy against diagonal energy
+    double off = 0.0, dg = 0.0;
+    for (int o = tid; o < np * np; o += nthr) {
+      const int i = o / np, j = o % np;
+      const double v = A[i][j] * A[i][j];
+      if (i == j) dg += v; else off += v;
     }
+#pragma unroll
+    for (int sft = 16; sft > 0; sft >>= 1) { off += __shfl_xor_sync(0xFFFFFFFFu, off, sft); dg += __shfl_xor_sync(0xFFFFFFFFu, dg, sft); }
+    if ((tid & 31) == 0) { red[0][tid >> 5] = off; red[1][tid >> 5] = dg; }
     __syncthreads();
-    if (red[0] <= 1e-30 * red[1] || red[0] == 0.0) break;
+    off = 0.0; dg = 0.0;
+    for (int w = 0; w < (nthr >> 5); ++w) { off += red[0][w]; dg += red[1][w]; }
+    __syncthreads();
+    if (off <= 1e-22 * dg) break;
     for (int step = 0; step < np - 1; ++step) {
-      if (tid < half) {
-        int a, b;
-        if (tid == 0) { a = 0; b = (step % (np - 1)) + 1; }
-        else { a = ((step + tid) % (np - 1)) + 1; b = ((step + np - 1 - tid) % (np - 1)) + 1; }
-        if (a > b) { const int t = a; a = b; b = t; }
+      const int pi = pairs[step][I][0], qi = pairs[step][I][1], pj = pairs[step][J][0], qj = pairs[step][J][1];
+      if (active && I == J) {
+        // rotation angle: the tangent only needs FP32 accuracy (it steers convergence); cos/sin are then made
+        // orthonormal to FP64 accuracy, so the accumulated eigenvector matrix stays orthogonal
+        const double apq = A[pi][qi];
         double c = 1.0, s = 0.0;
-        if (b < n) {
-          const double apq = A[a][b];
-          if (fabs(apq) > 1e-300) {
-            const double theta = (A[b][b] - A[a][a]) / (2.0 * apq);
-            const double t = (theta >= 0.0 ? 1.0 : -1.0) / (fabs(theta) + sqrt(theta * theta + 1.0));
-            c = 1.0 / sqrt(t * t + 1.0);
-            s = t * c;
-          }
+        if (fabs(apq) > 1e-300) {
+          const float theta = (float)(A[qi][qi] - A[pi][pi]) / (2.0f * (float)apq);
+          const float tf = copysignf(1.0f, theta) / (fabsf(theta) + sqrtf(fmaf(theta, theta, 1.0f)));
+          const double t = (double)tf;
+          c = fast_rsqrt(t * t + 1.0);
+          s = t * c;
         }
-        pr[tid][0] = a; pr[tid][1] = b; cs[tid][0] = c; cs[tid][1] = s;
+        cs[I][0] = c; cs[I][1] = s;
       }
       __syncthreads();
-      for (int o = tid; o < half * n; o += 256) {       // rows p,q of A <- J^T A
-        const int m = o / n, col = o % n;
-        const int p = pr[m][0], q2 = pr[m][1];
-        if (q2 < n) {
-          const double c = cs[m][0], s = cs[m][1];
-          const double ap = A[p][col], aq = A[q2][col];
-          A[p][col] = c * ap - s * aq;
-          A[q2][col] = s * ap + c * aq;
-        }
-      }
-      __syncthreads();
-      for (int o = tid; o < half * n; o += 256) {       // columns p,q of A and V <- (.) J
-        const int m = o / n, row = o % n;
-        const int p = pr[m][0], q2 = pr[m][1];
-        if (q2 < n) {
-          const double c = cs[m][0], s = cs[m][1];
-          const double ap = A[row][p], aq = A[row][q2];
-          A[row][p] = c * ap - s * aq;
-          A[row][q2] = s * ap + c * aq;
-          const double vp = V[row][p], vq = V[row][q2];
-          V[row][p] = c * vp - s * vq;
-          V[row][q2] = s * vp + c * vq;
-        }
+      if (active) {
+        const double ci = cs[I][0], si = cs[I][1], cj = cs[J][0], sj = cs[J][1];
+        // block rows (pi, qi), columns (pj, qj):  B <- Ji^T B Jj,  J = [[c, s], [-s, c]]
+        const double b00 = A[pi][pj], b01 = A[pi][qj], b10 = A[qi][pj], b11 = A[qi][qj];
+        const double r00 = ci * b00 - si * b10, r01 = ci * b01 - si * b11;
+        const double r10 = si * b00 + ci * b10, r11 = si * b01 + ci * b11;
+        A[pi][pj] = cj * r00 - sj * r01; A[pi][qj] = sj * r00 + cj * r01;
+        A[qi][pj] = cj * r10 - sj * r11; A[qi][qj] = sj * r10 + cj * r11;
+        // eigenvector accumulation: rows 2I, 2I+1 (fixed), columns (pj, qj):  V <- V Jj
+        const int r0 = 2 * I, r1 = 2 * I + 1;
+        const double v00 = V[r0][pj], v01 = V[r0][qj], v10 = V[r1][pj], v11 = V[r1][qj];
+        V[r0][pj] = cj * v00 - sj * v01; V[r0][qj] = sj * v00 + cj * v01;
+        V[r1][pj] = cj * v10 - sj * v11; V[r1][qj] = sj * v10 + cj * v11;
       }
       __syncthreads();
     }
@@ -295,25 +381,25 @@ jacobi_eig_kernel(const double* __restrict__ part, int n_parts, int n, double* _
   }
   __syncthreads();
   if (tid < n) evals[tid] = A[order[tid]][order[tid]];
-  for (int o = tid; o < n * n; o += 256) evecs[o] = V[o / n][order[o % n]];
+  for (int o = tid; o < n * n; o += nthr) evecs[o] = V[o / n][order[o % n]];
 }
 
 // ------------------------------------------------------------------------------------------------
 // Right basis from the small SVD: B[j][col] = sum_i Ut[i][j] M[i][col] / s_j, s_j = sqrt(eval_j); j < k.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(64)
 right_basis_kernel(const float* __restrict__ m, int64_t cols, int q, int k, const double* __restrict__ evals,
                    const double* __restrict__ evecs, float* __restrict__ basis, float* __restrict__ sigma_out) {
   __shared__ double ut[MAXQ][MAXQ + 1];
   __shared__ double inv_s[MAXQ];
   const int tid = threadIdx.x;
-  for (int o = tid; o < q * q; o += 256) ut[o / q][o % q] = evecs[o];
+  for (int o = tid; o < q * q; o += 64) ut[o / q][o % q] = evecs[o];
   if (tid < k) {
     const double s = sqrt(fmax(evals[tid], 0.0));
     inv_s[tid] = s > 0.0 ? 1.0 / s : 0.0;
     if (blockIdx.x == 0 && sigma_out != nullptr) sigma_out[tid] = (float)s;
   }
   __syncthreads();
-  const int64_t col = (int64_t)blockIdx.x * 256 + tid;
+  const int64_t col = (int64_t)blockIdx.x * 64 + tid;
   if (col >= cols) return;
   float mv[MAXQ];
   for (int i = 0; i < q; ++i) mv[i] = m[(int64_t)i * cols + col];
@@ -325,121 +411,247 @@ right_basis_kernel(const float* __restrict__ m, int64_t cols, int q, int k, cons
 }
 
 // ------------------------------------------------------------------------------------------------
-// Broadcast of the sampled subspace to every row: Ct[j][r] = sum_col x[r, col] * B[j][col].
-constexpr int CF_ROWS = 32, CF_COLS = 128;
-__global__ void __launch_bounds__(256)
-coeff_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols, int k, const float* __restrict__ basis,
-             float* __restrict__ coef_t) {
-  extern __shared__ __align__(16) unsigned char smem[];
-  float* xs = reinterpret_cast<float*>(smem);                 // [CF_ROWS][CF_COLS + 1]
-  float* bs = xs + CF_ROWS * (CF_COLS + 1);                   // [k][CF_COLS + 1]
-  const int tid = threadIdx.x, r = tid >> 3, jg = tid & 7;
-  const int64_t row0 = (int64_t)blockIdx.x * CF_ROWS;
-  float acc[MAXQ / 8];
+// Tensor-core helpers (warp-level mma.sync m16n8k16, BF16 operands, FP32 accumulate).  FP32 operands
+// are fed as three BF16 terms (hi + lo + lo2 = 24 mantissa bits) so the products stay FP32-accurate.
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+// three-term BF16 split of a pair of floats: v = hi + lo + lo2 (each term BF16, packed as pairs)
+__device__ __forceinline__ void split3(float x, float y, uint32_t& hi, uint32_t& lo, uint32_t& lo2) {
+  const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
+  const float xr = x - __bfloat162float(xh), yr = y - __bfloat162float(yh);
+  const __nv_bfloat16 xl = __float2bfloat16_rn(xr), yl = __float2bfloat16_rn(yr);
+  const float xr2 = xr - __bfloat162float(xl), yr2 = yr - __bfloat162float(yl);
+  hi = (uint32_t)__bfloat16_as_ushort(xh) | ((uint32_t)__bfloat16_as_ushort(yh) << 16);
+  lo = (uint32_t)__bfloat16_as_ushort(xl) | ((uint32_t)__bfloat16_as_ushort(yl) << 16);
+  lo2 = pack_bf16(xr2, yr2);
+}
+
+// BF16 splits of the right basis in both operand orientations:
+//   bs[t][j][col]  (col contiguous; B operand of C = x B, contraction over col)
+//   bt[t][col][j]  (j contiguous, padded to kp; B operand of C B^T, contraction over j)
+__global__ void __launch_bounds__(128)
+basis_splits_kernel(const float* __restrict__ basis, int64_t cols, int k, int kp, __nv_bfloat16* __restrict__ bs,
+                    __nv_bfloat16* __restrict__ bt) {
+  const int64_t col = (int64_t)blockIdx.x * 128 + threadIdx.x;
+  if (col >= cols) return;
+  for (int j0 = 0; j0 < kp; j0 += 8) {
+    uint32_t w[3][4];
 #pragma unroll
-  for (int j = 0; j < MAXQ / 8; ++j) acc[j] = 0.0f;
-  for (int64_t c0 = 0; c0 < cols; c0 += CF_COLS) {
-    for (int i = tid; i < CF_ROWS * CF_COLS; i += 256) {
-      const int rr = i / CF_COLS, cc = i % CF_COLS;
-      xs[rr * (CF_COLS + 1) + cc] =
-          (row0 + rr < rows && c0 + cc < cols) ? __bfloat162float(x[(row0 + rr) * cols + c0 + cc]) : 0.0f;
+    for (int jj = 0; jj < 8; jj += 2) {
+      const float v0 = j0 + jj < k ? basis[(int64_t)(j0 + jj) * cols + col] : 0.0f;
+      const float v1 = j0 + jj + 1 < k ? basis[(int64_t)(j0 + jj + 1) * cols + col] : 0.0f;
+      split3(v0, v1, w[0][jj >> 1], w[1][jj >> 1], w[2][jj >> 1]);
     }
-    for (int i = tid; i < k * CF_COLS; i += 256) {
-      const int jj = i / CF_COLS, cc = i % CF_COLS;
-      bs[jj * (CF_COLS + 1) + cc] = (c0 + cc < cols) ? basis[(int64_t)jj * cols + c0 + cc] : 0.0f;
-    }
-    __syncthreads();
-    for (int t = 0; t < CF_COLS; ++t) {
-      const float xv = xs[r * (CF_COLS + 1) + t];
 #pragma unroll
-      for (int j = 0; j < MAXQ / 8; ++j)
-        if (j * 8 + jg < k) acc[j] = fmaf(xv, bs[(j * 8 + jg) * (CF_COLS + 1) + t], acc[j]);
+    for (int t = 0; t < 3; ++t) {
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj)
+        bs[((int64_t)t * kp + j0 + jj) * cols + col] = __ushort_as_bfloat16((unsigned short)((w[t][jj >> 1] >> (16 * (jj & 1))) & 0xFFFFu));
+      *reinterpret_cast<uint4*>(bt + ((int64_t)t * cols + col) * kp + j0) = make_uint4(w[t][0], w[t][1], w[t][2], w[t][3]);
     }
-    __syncthreads();
   }
-  if (row0 + r < rows)
+}
+
+// Broadcast of the sampled subspace to every row (Section 3.1): C[r][j] = sum_col x[r, col] * B[j][col],
+// stored row-major with kp columns (zero padded).  One CTA = 32 rows; its 8 warps split the columns and
+// their partial tiles are added in fixed order.  Fused by-products of the same pass over x: amax|x|
+// (atomic max, order independent) and the FP64 Gram partial of the CTA's rows of C (for Rayleigh-Ritz).
+template <int KP>
+__global__ void __launch_bounds__(256)
+coeff_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols, const __nv_bfloat16* __restrict__ bs,
+                 float* __restrict__ coef, float* __restrict__ amax_out, double* __restrict__ gram_part) {
+  constexpr int NT = KP / 8;
+  extern __shared__ __align__(16) unsigned char smem[];
+  float* red = reinterpret_cast<float*>(smem);                 // [8 warps][32 rows][KP]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int64_t row0 = (int64_t)blockIdx.x * 32;
+  const int ksteps = (int)(cols / 16);
+  const int ks_begin = (int)((int64_t)ksteps * warp / 8), ks_end = (int)((int64_t)ksteps * (warp + 1) / 8);
+  float acc[2][NT][4];
 #pragma unroll
-    for (int j = 0; j < MAXQ / 8; ++j)
-      if (j * 8 + jg < k) coef_t[(int64_t)(j * 8 + jg) * rows + row0 + r] = acc[j];
+  for (int m = 0; m < 2; ++m)
+#pragma unroll
+    for (int n = 0; n < NT; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[m][n][e] = 0.0f;
+  uint32_t amax2 = 0u;                                         // two running |.| maxima, BF16 pair
+  const bool v0 = row0 + g < rows, v1 = row0 + g + 8 < rows, v2 = row0 + g + 16 < rows, v3 = row0 + g + 24 < rows;
+  const __nv_bfloat16* xr0 = x + (row0 + g) * cols;
+#pragma unroll 2
+  for (int ks = ks_begin; ks < ks_end; ++ks) {
+    const int kk = ks * 16 + 2 * t;
+    uint32_t a[2][4];
+    a[0][0] = v0 ? *reinterpret_cast<const uint32_t*>(xr0 + kk) : 0u;
+    a[0][1] = v1 ? *reinterpret_cast<const uint32_t*>(xr0 + 8 * cols + kk) : 0u;
+    a[0][2] = v0 ? *reinterpret_cast<const uint32_t*>(xr0 + kk + 8) : 0u;
+    a[0][3] = v1 ? *reinterpret_cast<const uint32_t*>(xr0 + 8 * cols + kk + 8) : 0u;
+    a[1][0] = v2 ? *reinterpret_cast<const uint32_t*>(xr0 + 16 * cols + kk) : 0u;
+    a[1][1] = v3 ? *reinterpret_cast<const uint32_t*>(xr0 + 24 * cols + kk) : 0u;
+    a[1][2] = v2 ? *reinterpret_cast<const uint32_t*>(xr0 + 16 * cols + kk + 8) : 0u;
+    a[1][3] = v3 ? *reinterpret_cast<const uint32_t*>(xr0 + 24 * cols + kk + 8) : 0u;
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t ab = a[m][e] & 0x7FFF7FFFu;             // |.| of both halves; BF16 magnitudes order like integers
+        const uint32_t lo = max(ab & 0xFFFFu, amax2 & 0xFFFFu), hi = max(ab >> 16, amax2 >> 16);
+        amax2 = lo | (hi << 16);
+      }
+#pragma unroll
+    for (int sp = 0; sp < 3; ++sp) {
+      const __nv_bfloat16* bsp = bs + (int64_t)sp * KP * cols;
+#pragma unroll
+      for (int n = 0; n < NT; ++n) {
+        const __nv_bfloat16* bp = bsp + (int64_t)(n * 8 + g) * cols + kk;
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(bp), b1 = *reinterpret_cast<const uint32_t*>(bp + 8);
+        mma_bf16(acc[0][n], a[0], b0, b1);
+        mma_bf16(acc[1][n], a[1], b0, b1);
+      }
+    }
+  }
+  // per-warp partial tile -> shared memory
+#pragma unroll
+  for (int m = 0; m < 2; ++m)
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      float* r0p = red + ((warp * 32) + m * 16 + g) * KP + n * 8 + 2 * t;
+      r0p[0] = acc[m][n][0]; r0p[1] = acc[m][n][1];
+      r0p[8 * KP] = acc[m][n][2]; r0p[8 * KP + 1] = acc[m][n][3];
+    }
+  {
+    float am = fmaxf(__uint_as_float((amax2 & 0xFFFFu) << 16), __uint_as_float(amax2 & 0xFFFF0000u));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+    if (lane == 0 && amax_out) atomicMax(reinterpret_cast<unsigned int*>(amax_out), __float_as_uint(am));
+  }
+  __syncthreads();
+  float* cfin = red + 8 * 32 * KP;                             // [32][KP] final tile
+  for (int o = tid; o < 32 * KP; o += 256) {
+    float sacc = 0.0f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) sacc += red[w * 32 * KP + o];
+    cfin[o] = sacc;
+    const int64_t r = row0 + o / KP;
+    if (r < rows) coef[r * KP + (o % KP)] = sacc;
+  }
+  __syncthreads();
+  if (gram_part) {
+    for (int o = tid; o < KP * KP; o += 256) {
+      const int i = o / KP, j = o % KP;
+      double a = 0.0;
+#pragma unroll 8
+      for (int r = 0; r < 32; ++r) a += (double)cfin[r * KP + i] * (double)cfin[r * KP + j];
+      gram_part[(int64_t)blockIdx.x * KP * KP + o] = a;
+    }
+  }
+}
+
+// out[e] = sum over all partials p of in[p][e], in order (eight independent loads in flight per thread).
+__global__ void reduce_gram_kernel(const double* __restrict__ in, int n_in, int nn, double* __restrict__ out) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= nn) return;
+  double a = 0.0;
+  int p = 0;
+  for (; p + 8 <= n_in; p += 8) {
+    double v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = in[(int64_t)(p + u) * nn + e];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) a += v[u];
+  }
+  for (; p < n_in; ++p) a += in[(int64_t)p * nn + e];
+  out[e] = a;
 }
 
 // ------------------------------------------------------------------------------------------------
-// Fused residual + quantizer: R = x - sum_j coefT[j][r] * scale_j * basis[j][col] on a 128 x 128 tile,
-// then NVFP4 in one or both block orientations straight from shared memory (the residual never goes
-// to HBM unless `dense` is given).
-__global__ void __launch_bounds__(metis_qt::THREADS)
-residual_quant_kernel(const __nv_bfloat16* __restrict__ x, int k, const float* __restrict__ coef_t,
-                      const float* __restrict__ scale, const float* __restrict__ basis, metis_qt::QuantParams p,
+// Fused residual + quantizer: R = x - C B^T on a 128 x 128 tile (tensor cores, three-term BF16 splits of
+// both FP32 operands), then NVFP4 in one or both block orientations straight from shared memory (the
+// residual never goes to HBM unless `dense` is given).  coef: [rows][KP] row-major, bt: [3][cols][KP].
+template <int KP>
+__global__ void __launch_bounds__(metis_qt::THREADS, 2)
+residual_quant_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ coef,
+                      const __nv_bfloat16* __restrict__ bt, metis_qt::QuantParams p,
                       const float* __restrict__ amax_src, float* ts_out0, float* ts_out1, float* __restrict__ dense) {
   using namespace metis_qt;
   extern __shared__ __align__(16) unsigned char smem[];
   float* tile = reinterpret_cast<float*>(smem);
   Stage* stage = reinterpret_cast<Stage*>(smem + sizeof(float) * TILE * PITCH);
-  unsigned char* after = smem + sizeof(float) * TILE * PITCH + sizeof(Stage);
+  uint16_t* rnd = reinterpret_cast<uint16_t*>(smem + sizeof(float) * TILE * PITCH + sizeof(Stage));
   const bool sr = p.rounding == METIS_ROUND_SR;
-  uint16_t* rnd = reinterpret_cast<uint16_t*>(after);
-  float* cs = reinterpret_cast<float*>(after + (sr ? sizeof(uint16_t) * TILE * TILE : 0));   // [k][TILE]
-  float* bs = cs + k * TILE;                                                                 // [k][TILE]
-
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int64_t row0 = (int64_t)blockIdx.y * TILE, col0 = (int64_t)blockIdx.x * TILE;
   const float s_T = metis_tensor_scale(*amax_src);
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
     if (ts_out0) *ts_out0 = s_T;
     if (ts_out1) *ts_out1 = s_T;
   }
-  for (int i = tid; i < TILE * (TILE / 8); i += THREADS) {
-    const int r = i >> 4, g = i & 15;
-    const int64_t gr = row0 + r, gc = col0 + g * 8;
-    float v[8];
-    if (gr < p.rows && gc + 8 <= p.cols) {
-      const uint4 q = *reinterpret_cast<const uint4*>(x + gr * p.cols + gc);
-      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) { v[2 * j] = __uint_as_float(w[j] << 16); v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u); }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) v[j] = (gr < p.rows && gc + j < p.cols) ? __bfloat162float(x[gr * p.cols + gc + j]) : 0.0f;
-    }
-    *reinterpret_cast<float4*>(tile + r * PITCH + g * 8) = make_float4(v[0], v[1], v[2], v[3]);
-    *reinterpret_cast<float4*>(tile + r * PITCH + g * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
-  }
-  for (int i = tid; i < k * TILE; i += THREADS) {
-    const int j = i >> 7, t = i & 127;
-    const float sc = scale ? scale[j] : 1.0f;
-    cs[i] = (row0 + t < p.rows) ? coef_t[(int64_t)j * p.rows + row0 + t] * sc : 0.0f;
-    bs[i] = (col0 + t < p.cols) ? basis[(int64_t)j * p.cols + col0 + t] : 0.0f;
-  }
   if (sr) fill_draws(rnd, p, row0, col0);
-  __syncthreads();
-  {
-    const int r0 = (tid >> 4) * 8, c0 = (tid & 15) * 8;
-    float acc[8][8];
+  // this warp: rows row0 + 16*warp .. +15, all 128 columns
+  const int64_t ra = row0 + warp * 16 + g, rb = ra + 8;
+  const bool va = ra < p.rows, vb = rb < p.rows;
+  float acc[16][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+  for (int n = 0; n < 16; ++n)
 #pragma unroll
-      for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
-    for (int j = 0; j < k; ++j) {
-      const float4 a0 = *reinterpret_cast<const float4*>(cs + j * TILE + r0), a1 = *reinterpret_cast<const float4*>(cs + j * TILE + r0 + 4);
-      const float4 b0 = *reinterpret_cast<const float4*>(bs + j * TILE + c0), b1 = *reinterpret_cast<const float4*>(bs + j * TILE + c0 + 4);
-      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-      const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    for (int e = 0; e < 4; ++e) acc[n][e] = 0.0f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-#pragma unroll
-        for (int jj = 0; jj < 8; ++jj) acc[i][jj] = fmaf(a[i], b[jj], acc[i][jj]);
+  for (int ks = 0; ks < KP / 16; ++ks) {
+    const int kk = ks * 16 + 2 * t;
+    uint32_t ah[4], al[4], al2[4];
+    {
+      const float2 z = make_float2(0.0f, 0.0f);
+      const float2 c0 = va ? *reinterpret_cast<const float2*>(coef + ra * KP + kk) : z;
+      const float2 c1 = vb ? *reinterpret_cast<const float2*>(coef + rb * KP + kk) : z;
+      const float2 c2 = va ? *reinterpret_cast<const float2*>(coef + ra * KP + kk + 8) : z;
+      const float2 c3 = vb ? *reinterpret_cast<const float2*>(coef + rb * KP + kk + 8) : z;
+      split3(c0.x, c0.y, ah[0], al[0], al2[0]);
+      split3(c1.x, c1.y, ah[1], al[1], al2[1]);
+      split3(c2.x, c2.y, ah[2], al[2], al2[2]);
+      split3(c3.x, c3.y, ah[3], al[3], al2[3]);
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      float* t = tile + (r0 + i) * PITCH + c0;
-      float4 v0 = *reinterpret_cast<float4*>(t), v1 = *reinterpret_cast<float4*>(t + 4);
-      v0.x -= acc[i][0]; v0.y -= acc[i][1]; v0.z -= acc[i][2]; v0.w -= acc[i][3];
-      v1.x -= acc[i][4]; v1.y -= acc[i][5]; v1.z -= acc[i][6]; v1.w -= acc[i][7];
-      *reinterpret_cast<float4*>(t) = v0; *reinterpret_cast<float4*>(t + 4) = v1;
-      if (dense != nullptr && row0 + r0 + i < p.rows && col0 + c0 + 8 <= p.cols) {
-        float* d = dense + (row0 + r0 + i) * p.cols + col0 + c0;
-        *reinterpret_cast<float4*>(d) = v0; *reinterpret_cast<float4*>(d + 4) = v1;
+    for (int n = 0; n < 16; ++n) {
+      const int64_t col = col0 + n * 8 + g;
+      uint32_t bh0 = 0, bh1 = 0, bl0 = 0, bl1 = 0, bm0 = 0, bm1 = 0;
+      if (col < p.cols) {
+        const __nv_bfloat16* bp = bt + col * KP + kk;
+        bh0 = *reinterpret_cast<const uint32_t*>(bp); bh1 = *reinterpret_cast<const uint32_t*>(bp + 8);
+        bl0 = *reinterpret_cast<const uint32_t*>(bp + p.cols * KP); bl1 = *reinterpret_cast<const uint32_t*>(bp + p.cols * KP + 8);
+        bm0 = *reinterpret_cast<const uint32_t*>(bp + 2 * p.cols * KP); bm1 = *reinterpret_cast<const uint32_t*>(bp + 2 * p.cols * KP + 8);
       }
+      // smallest terms first
+      mma_bf16(acc[n], al, bl0, bl1);
+      mma_bf16(acc[n], al2, bh0, bh1);
+      mma_bf16(acc[n], ah, bm0, bm1);
+      mma_bf16(acc[n], al, bh0, bh1);
+      mma_bf16(acc[n], ah, bl0, bl1);
+      mma_bf16(acc[n], ah, bh0, bh1);
+    }
+  }
+  // R = x - acc into the shared tile (and to `dense` when asked)
+#pragma unroll
+  for (int n = 0; n < 16; ++n) {
+    const int64_t col = col0 + n * 8 + 2 * t;
+    const int lc = n * 8 + 2 * t;
+    float x00 = 0.0f, x01 = 0.0f, x10 = 0.0f, x11 = 0.0f;
+    if (col < p.cols) {
+      if (va) { const uint32_t w = *reinterpret_cast<const uint32_t*>(x + ra * p.cols + col); x00 = __uint_as_float(w << 16); x01 = __uint_as_float(w & 0xFFFF0000u); }
+      if (vb) { const uint32_t w = *reinterpret_cast<const uint32_t*>(x + rb * p.cols + col); x10 = __uint_as_float(w << 16); x11 = __uint_as_float(w & 0xFFFF0000u); }
+    }
+    const float2 r0v = make_float2(x00 - acc[n][0], x01 - acc[n][1]);
+    const float2 r1v = make_float2(x10 - acc[n][2], x11 - acc[n][3]);
+    *reinterpret_cast<float2*>(tile + (warp * 16 + g) * PITCH + lc) = (va && col < p.cols) ? r0v : make_float2(0.0f, 0.0f);
+    *reinterpret_cast<float2*>(tile + (warp * 16 + g + 8) * PITCH + lc) = (vb && col < p.cols) ? r1v : make_float2(0.0f, 0.0f);
+    if (dense != nullptr && col < p.cols) {
+      if (va) *reinterpret_cast<float2*>(dense + ra * p.cols + col) = r0v;
+      if (vb) *reinterpret_cast<float2*>(dense + rb * p.cols + col) = r1v;
     }
   }
   __syncthreads();
@@ -447,55 +659,84 @@ residual_quant_kernel(const __nv_bfloat16* __restrict__ x, int k, const float* _
 }
 
 // ------------------------------------------------------------------------------------------------
-// right[j][col] = sum_i basis[i][col] * W[i][j] (W == nullptr: identity), then the sign convention:
-// the largest-magnitude entry of each right vector (lowest index on ties) is made positive.
+// right[j][col] = sum_i basis[i][col] * W[i][j] (W == nullptr: identity).  One thread per column; each CTA
+// also records, for every j, its largest |right[j][col]| (lowest column on ties) for the sign convention.
 __global__ void __launch_bounds__(256)
-right_rotate_sign_kernel(const float* __restrict__ basis, int64_t cols, int n_in, const double* __restrict__ w,
-                         float* __restrict__ right, float* __restrict__ sign_out) {
-  __shared__ double wj[MAXQ];
-  __shared__ float best_v[256];
-  __shared__ long long best_i[256];
-  const int j = blockIdx.x, tid = threadIdx.x;
-  if (tid < n_in) wj[tid] = w ? w[tid * n_in + j] : (tid == j ? 1.0 : 0.0);
+right_rotate_kernel(const float* __restrict__ basis, int64_t cols, int k, const double* __restrict__ w,
+                    float* __restrict__ right, float* __restrict__ cand_v, int* __restrict__ cand_i) {
+  __shared__ float wsm[MAXQ][MAXQ + 1];
+  __shared__ float red_v[8][MAXQ];
+  __shared__ int red_i[8][MAXQ];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (w) for (int o = tid; o < k * k; o += 256) wsm[o / k][o % k] = (float)w[o];
   __syncthreads();
-  float bv = -1.0f, bsgn = 1.0f;
-  long long bi = 0x7FFFFFFFFFFFFFFFll;
-  for (int64_t col = tid; col < cols; col += 256) {
-    double a = 0.0;
-    if (w) { for (int i = 0; i < n_in; ++i) a += (double)basis[(int64_t)i * cols + col] * wj[i]; }
-    else a = (double)basis[(int64_t)j * cols + col];
-    const float v = (float)a;
-    right[(int64_t)j * cols + col] = v;
-    if (fabsf(v) > bv) { bv = fabsf(v); bi = col; bsgn = v < 0.0f ? -1.0f : 1.0f; }
-  }
-  best_v[tid] = bv; best_i[tid] = bi;
-  __shared__ float sgn_s[256];
-  sgn_s[tid] = bsgn;
-  __syncthreads();
-  for (int s = 128; s > 0; s >>= 1) {
-    if (tid < s) {
-      const bool take = best_v[tid + s] > best_v[tid] || (best_v[tid + s] == best_v[tid] && best_i[tid + s] < best_i[tid]);
-      if (take) { best_v[tid] = best_v[tid + s]; best_i[tid] = best_i[tid + s]; sgn_s[tid] = sgn_s[tid + s]; }
+  const int64_t col = (int64_t)blockIdx.x * 256 + tid;
+  float bv[MAXQ];
+#pragma unroll
+  for (int i = 0; i < MAXQ; ++i) bv[i] = (i < k && col < cols) ? basis[(int64_t)i * cols + col] : 0.0f;
+  for (int j = 0; j < k; ++j) {
+    float v;
+    if (w) {
+      v = 0.0f;
+#pragma unroll
+      for (int i = 0; i < MAXQ; ++i) if (i < k) v = fmaf(bv[i], wsm[i][j], v);
+    } else {
+      v = 0.0f;
+#pragma unroll
+      for (int i = 0; i < MAXQ; ++i) if (i == j) v = bv[i];
     }
-    __syncthreads();
+    if (col < cols) right[(int64_t)j * cols + col] = v;
+    float av = col < cols ? fabsf(v) : -1.0f;
+    int ai = (int)min(col, (int64_t)0x7FFFFFFF);
+#pragma unroll
+    for (int sft = 16; sft > 0; sft >>= 1) {
+      const float ov = __shfl_xor_sync(0xFFFFFFFFu, av, sft);
+      const int oi = __shfl_xor_sync(0xFFFFFFFFu, ai, sft);
+      if (ov > av || (ov == av && oi < ai)) { av = ov; ai = oi; }
+    }
+    if (lane == 0) { red_v[warp][j] = av; red_i[warp][j] = ai; }
   }
-  const float sg = sgn_s[0];
-  if (tid == 0) sign_out[j] = sg;
-  if (sg < 0.0f)
-    for (int64_t col = tid; col < cols; col += 256) right[(int64_t)j * cols + col] = -right[(int64_t)j * cols + col];
+  __syncthreads();
+  if (tid < k) {
+    float av = red_v[0][tid]; int ai = red_i[0][tid];
+    for (int wv = 1; wv < 8; ++wv)
+      if (red_v[wv][tid] > av || (red_v[wv][tid] == av && red_i[wv][tid] < ai)) { av = red_v[wv][tid]; ai = red_i[wv][tid]; }
+    cand_v[(int64_t)blockIdx.x * k + tid] = av;
+    cand_i[(int64_t)blockIdx.x * k + tid] = ai;
+  }
+}
+
+// Sign convention: the largest-magnitude entry of each right vector (lowest index on ties) is made positive.
+// grid (column chunks, k).  Every CTA re-derives the winner of its vector from the candidates.
+__global__ void __launch_bounds__(256)
+sign_fix_kernel(float* __restrict__ right, int64_t cols, int k, const float* __restrict__ cand_v,
+                const int* __restrict__ cand_i, int n_cand, float* __restrict__ sign_out) {
+  const int j = blockIdx.y;
+  float av = -1.0f; int ai = 0x7FFFFFFF;
+  for (int c = 0; c < n_cand; ++c) {
+    const float v = cand_v[(int64_t)c * k + j]; const int i = cand_i[(int64_t)c * k + j];
+    if (v > av || (v == av && i < ai)) { av = v; ai = i; }
+  }
+  const float sg = right[(int64_t)j * cols + ai] < 0.0f ? -1.0f : 1.0f;
+  __syncthreads();                                 // every thread has read the winner before anyone flips it
+  if (blockIdx.x == 0 && threadIdx.x == 0) sign_out[j] = sg;
+  const int64_t col = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (sg < 0.0f && col < cols) right[(int64_t)j * cols + col] = -right[(int64_t)j * cols + col];
 }
 
 // left[j][r] = sign_j * scale_j * sum_i coef(i, r) * W[i][j],  coef(i, r) = c[i*stride_i + r*stride_r]
 // scale_j = 1/sqrt(eval_j) when inv_sqrt_evals is given (Rayleigh-Ritz normalisation), else 1.
-// Also writes sigma_out[j] = sqrt(eval_j) when asked.
-__global__ void __launch_bounds__(256)
+// Also writes sigma_out[j] = sqrt(eval_j) when asked, and coef_rm[r][j] = left[j][r] * sigma_for_coef[j]
+// (row-major, kp columns, zero padded) when asked.
+__global__ void __launch_bounds__(64)
 left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, int64_t stride_i, int64_t stride_r,
                    const double* __restrict__ w, const double* __restrict__ evals_for_scale,
-                   const float* __restrict__ sign, float* __restrict__ left, float* __restrict__ sigma_out) {
+                   const float* __restrict__ sign, float* __restrict__ left, float* __restrict__ sigma_out,
+                   float* __restrict__ coef_rm, int kp, const float* __restrict__ sigma_for_coef) {
   __shared__ double ws[MAXQ][MAXQ + 1];
   __shared__ double scl[MAXQ];
   const int tid = threadIdx.x;
-  for (int o = tid; o < n_in * n_in; o += 256) ws[o / n_in][o % n_in] = w[o];
+  for (int o = tid; o < n_in * n_in; o += 64) ws[o / n_in][o % n_in] = w[o];
   if (tid < k) {
     double s = 1.0;
     if (evals_for_scale) {
@@ -506,20 +747,38 @@ left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, i
     scl[tid] = s * (double)sign[tid];
   }
   __syncthreads();
-  const int64_t r = (int64_t)blockIdx.x * 256 + tid;
+  const int64_t r = (int64_t)blockIdx.x * 64 + tid;
   if (r >= rows) return;
   float cv[MAXQ];
   for (int i = 0; i < n_in; ++i) cv[i] = c[i * stride_i + r * stride_r];
   for (int j = 0; j < k; ++j) {
     double a = 0.0;
     for (int i = 0; i < n_in; ++i) a += (double)cv[i] * ws[i][j];
-    left[(int64_t)j * rows + r] = (float)(a * scl[j]);
+    const float v = (float)(a * scl[j]);
+    left[(int64_t)j * rows + r] = v;
+    if (coef_rm) coef_rm[r * kp + j] = v * sigma_for_coef[j];
   }
+  if (coef_rm) for (int j = k; j < kp; ++j) coef_rm[r * kp + j] = 0.0f;
 }
 
 struct SplitWs {
-  size_t amax, idx, zp, z, gram, evals, evecs, m, basis, coef, sign, evals2, evecs2, total;
+  size_t amax, idx, zp, z, gram, gram1, linv, evals, evecs, mp, m, basis, coef, sign, cand_v, cand_i, evals2, evecs2, bs, bt,
+      gram_c, total;
 };
+
+constexpr int PJ_MAX_PARTS = 16;
+
+int project_parts(int64_t n_s, int64_t cols, int* rows_per_part) {
+  const int64_t col_chunks = metis_ceil_div(cols, PJ_COLS);
+  int64_t parts = metis_ceil_div(2 * 148, col_chunks);          // aim at two CTAs per SM
+  if (parts > PJ_MAX_PARTS) parts = PJ_MAX_PARTS;
+  if (parts > metis_ceil_div(n_s, 16)) parts = metis_ceil_div(n_s, 16);
+  if (parts < 1) parts = 1;
+  int64_t rpp = metis_ceil_div(n_s, parts);
+  rpp = metis_ceil_div(rpp, 16) * 16;
+  *rows_per_part = (int)rpp;
+  return (int)metis_ceil_div(n_s, rpp);
+}
 
 SplitWs split_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s) {
   SplitWs w{};
@@ -532,12 +791,21 @@ SplitWs split_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s) {
   w.zp = take(sizeof(float) * (size_t)chunks * n_s * q);
   w.z = take(sizeof(float) * (size_t)n_s * q);
   w.gram = take(sizeof(double) * 64 * MAXQ * MAXQ);
+  w.linv = take(sizeof(double) * (MAXQ * MAXQ + MAXQ));
+  w.gram1 = take(sizeof(double) * MAXQ * MAXQ);
   w.evals = take(sizeof(double) * MAXQ);
   w.evecs = take(sizeof(double) * MAXQ * MAXQ);
+  w.mp = take(sizeof(float) * (size_t)PJ_MAX_PARTS * q * cols);
   w.m = take(sizeof(float) * (size_t)q * cols);
   w.basis = take(sizeof(float) * (size_t)k * cols);
-  w.coef = take(sizeof(float) * (size_t)k * rows);
+  const int kp = (k + 15) / 16 * 16;
+  w.coef = take(sizeof(float) * (size_t)kp * rows);
+  w.bs = take(sizeof(__nv_bfloat16) * 3 * (size_t)kp * cols);
+  w.bt = take(sizeof(__nv_bfloat16) * 3 * (size_t)kp * cols);
+  w.gram_c = take(sizeof(double) * (size_t)metis_ceil_div(rows, 32) * kp * kp);
   w.sign = take(sizeof(float) * MAXQ);
+  w.cand_v = take(sizeof(float) * MAXQ * (size_t)metis_ceil_div(cols, 256));
+  w.cand_i = take(sizeof(int) * MAXQ * (size_t)metis_ceil_div(cols, 256));
   w.evals2 = take(sizeof(double) * MAXQ);
   w.evecs2 = take(sizeof(double) * MAXQ * MAXQ);
   w.total = off;
@@ -545,13 +813,25 @@ SplitWs split_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s) {
 }
 
 int gram_parts(int64_t n_rows, int64_t* rows_per_part) {
-  int parts = (int)metis_ceil_div(n_rows, 512);
+  int parts = (int)metis_ceil_div(n_rows, 64);
   if (parts > 64) parts = 64;
   if (parts < 1) parts = 1;
   int64_t rpp = metis_ceil_div(n_rows, parts);
   rpp = metis_ceil_div(rpp, GR_TILE) * GR_TILE;
   *rows_per_part = rpp;
   return (int)metis_ceil_div(n_rows, rpp);
+}
+
+template <int NJ4>
+void launch_project(dim3 grid, cudaStream_t s, const __nv_bfloat16* x, int64_t cols, const int* idx, int n_s, int q,
+                    const float* h, int rpp, float* mp) {
+  project_kernel<NJ4><<<grid, 256, 0, s>>>(x, cols, idx, n_s, q, h, rpp, mp); METIS_COUNT_LAUNCH();
+}
+
+int jacobi_threads(int n) {
+  const int half = (n + 1) / 2;
+  int t = (half * half + 31) / 32 * 32;
+  return t < 64 ? 64 : t;
 }
 
 }  // namespace
@@ -598,11 +878,10 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(xv);
   float* amax = reinterpret_cast<float*>(wsb + L.amax);
 
-  METIS_TRY(metis_launch_amax(x, METIS_BF16, rows, cols, cols, amax, s));
-
   metis_nvfp4_t rc = out->res_by_cols, rr = out->res_by_rows;
   rc.rows = rows; rc.k_len = cols; rr.rows = cols; rr.k_len = rows;
   if (k == 0) {
+    METIS_TRY(metis_launch_amax(x, METIS_BF16, rows, cols, cols, amax, s));
     return metis_launch_quantize(x, METIS_BF16, rows, cols, cols, rounding, seed, METIS_STREAM_RESIDUAL, cols, 1, amax,
                                  1, want_c ? &rc : nullptr, want_r ? &rr : nullptr, s);
   }
@@ -616,28 +895,50 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   float* zp = reinterpret_cast<float*>(wsb + L.zp);
   float* z = reinterpret_cast<float*>(wsb + L.z);
   double* gram = reinterpret_cast<double*>(wsb + L.gram);
+  double* linv = reinterpret_cast<double*>(wsb + L.linv);
+  double* invd = linv + MAXQ * MAXQ;
+  double* gram1 = reinterpret_cast<double*>(wsb + L.gram1);
   double* evals = reinterpret_cast<double*>(wsb + L.evals);
   double* evecs = reinterpret_cast<double*>(wsb + L.evecs);
+  float* mp = reinterpret_cast<float*>(wsb + L.mp);
   float* m = reinterpret_cast<float*>(wsb + L.m);
   float* basis = reinterpret_cast<float*>(wsb + L.basis);
   float* coef = reinterpret_cast<float*>(wsb + L.coef);
   float* sign = reinterpret_cast<float*>(wsb + L.sign);
+  float* cand_v = reinterpret_cast<float*>(wsb + L.cand_v);
+  int* cand_i = reinterpret_cast<int*>(wsb + L.cand_i);
   double* evals2 = reinterpret_cast<double*>(wsb + L.evals2);
   double* evecs2 = reinterpret_cast<double*>(wsb + L.evecs2);
+  __nv_bfloat16* bs = reinterpret_cast<__nv_bfloat16*>(wsb + L.bs);
+  __nv_bfloat16* bt = reinterpret_cast<__nv_bfloat16*>(wsb + L.bt);
+  double* gram_c = reinterpret_cast<double*>(wsb + L.gram_c);
   metis_context* ctx = h;
-
+  const int kp = (k + 15) / 16 * 16;
   {
     static bool attr = false;
-    if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM)); attr = true; }
+    if (!attr) {
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(sketch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)(sizeof(float) * (SK_COLS * MAXQ + SK_ROWS * SK_PITCH))));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 64)));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 48)));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
+      attr = true;
+    }
   }
+  // amax|x| for the residual's tensor scale: its own pass in FULL mode, fused into the broadcast pass in SAMPLED mode
+  if (full) METIS_TRY(metis_launch_amax(x, METIS_BF16, rows, cols, cols, amax, s));
+  else METIS_CUDA_TRY(cudaMemsetAsync(amax, 0, sizeof(float), s));
+
   // (1) row sample, (2) sketch
   sample_rows_kernel<<<(unsigned)metis_ceil_div(n_s, 256), 256, 0, s>>>(idx, (int)n_s, rows, seed, full ? 1 : 0); METIS_COUNT_LAUNCH();
   const int chunks = (int)metis_ceil_div(cols, SK_COLS);
   {
-    const size_t smem = sizeof(float) * (SK_COLS * q + SK_ROWS * SK_COLS);
-    static bool attr = false;
-    if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(sketch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * (SK_COLS * MAXQ + SK_ROWS * SK_COLS)))); attr = true; }
-    dim3 grid((unsigned)(n_s / SK_ROWS), (unsigned)chunks);
+    const size_t smem = sizeof(float) * (SK_COLS * MAXQ + SK_ROWS * SK_PITCH);
+    dim3 grid((unsigned)metis_ceil_div(n_s, SK_ROWS), (unsigned)chunks);
     sketch_kernel<<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp); METIS_COUNT_LAUNCH();
   }
   reduce_partials_kernel<<<(unsigned)metis_ceil_div(n_s * q, 256), 256, 0, s>>>(zp, chunks, n_s * q, z); METIS_COUNT_LAUNCH();
@@ -645,56 +946,81 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   for (int pass = 0; pass < 2; ++pass) {
     int64_t rpp; const int parts = gram_parts(n_s, &rpp);
     gram_kernel<<<parts, 256, 0, s>>>(z, n_s, q, q, 1, rpp, gram); METIS_COUNT_LAUNCH();
-    cholqr_apply_kernel<<<(unsigned)metis_ceil_div(n_s, 128), 128, 0, s>>>(z, n_s, q, gram, parts, ctx->dev_status); METIS_COUNT_LAUNCH();
+    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1); METIS_COUNT_LAUNCH();
+    chol_kernel<<<1, 256, 0, s>>>(gram1, q, linv, invd); METIS_COUNT_LAUNCH();
+    apply_chol_kernel<<<(unsigned)metis_ceil_div(n_s, 8), 256, 0, s>>>(z, n_s, q, linv, invd); METIS_COUNT_LAUNCH();
   }
   // (4) M = H^T x[S,:], eigen-decomposition of M M^T, right basis
-  project_kernel<<<(unsigned)metis_ceil_div(cols, PJ_COLS), 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, m); METIS_COUNT_LAUNCH();
+  {
+    int rpp; const int parts = project_parts(n_s, cols, &rpp);
+    dim3 grid((unsigned)metis_ceil_div(cols, PJ_COLS), (unsigned)parts);
+    const int nj4 = (q + 7) / 8;
+    switch (nj4) {
+      case 1: launch_project<1>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+      case 2: launch_project<2>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+      case 3: launch_project<3>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+      case 4: launch_project<4>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+      case 5: launch_project<5>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+      case 6: launch_project<6>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+      case 7: launch_project<7>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+      default: launch_project<8>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+    }
+    reduce_partials_kernel<<<(unsigned)metis_ceil_div((int64_t)q * cols, 256), 256, 0, s>>>(mp, parts, (int64_t)q * cols, m); METIS_COUNT_LAUNCH();
+  }
   {
     int64_t rpp; const int parts = gram_parts(cols, &rpp);
     gram_kernel<<<parts, 256, 0, s>>>(m, cols, q, 1, cols, rpp, gram); METIS_COUNT_LAUNCH();
-    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram, parts, q, evals, evecs); METIS_COUNT_LAUNCH();
+    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1); METIS_COUNT_LAUNCH();
+    jacobi_eig_kernel<<<1, jacobi_threads(q), JACOBI_SMEM, s>>>(gram1, q, q, evals, evecs); METIS_COUNT_LAUNCH();
   }
-  right_basis_kernel<<<(unsigned)metis_ceil_div(cols, 256), 256, 0, s>>>(m, cols, q, k, evals, evecs, basis,
+  right_basis_kernel<<<(unsigned)metis_ceil_div(cols, 64), 64, 0, s>>>(m, cols, q, k, evals, evecs, basis,
                                                                           full ? out->sigma : nullptr); METIS_COUNT_LAUNCH();
-  // (5) factors
-  const float* res_coef; const float* res_scale; const float* res_basis;
+  // (5) coefficients of every row in the basis, (6) fused residual + quantizer
+  const int n_cand = (int)metis_ceil_div(cols, 256);
+  const int n_cta_c = (int)metis_ceil_div(rows, 32);
   if (full) {
-    // left = H U~_k, right = basis; residual against left * sigma * right^T
-    right_rotate_sign_kernel<<<k, 256, 0, s>>>(basis, cols, k, nullptr, out->right, sign); METIS_COUNT_LAUNCH();
-    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 256), 256, 0, s>>>(z, rows, q, k, 1, q, evecs, nullptr, sign,
-                                                                           out->left, nullptr); METIS_COUNT_LAUNCH();
-    res_coef = out->left; res_scale = out->sigma; res_basis = out->right;
+    // left = H U~_k, right = basis (sign fixed); coefficients = left * sigma
+    right_rotate_kernel<<<n_cand, 256, 0, s>>>(basis, cols, k, nullptr, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
+    sign_fix_kernel<<<dim3(n_cand, k), 256, 0, s>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign); METIS_COUNT_LAUNCH();
+    basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(out->right, cols, k, kp, bs, bt); METIS_COUNT_LAUNCH();
+    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 64, 0, s>>>(z, rows, q, k, 1, q, evecs, nullptr, sign,
+                                                                           out->left, nullptr, coef, kp, out->sigma); METIS_COUNT_LAUNCH();
   } else {
-    const size_t smem = sizeof(float) * (CF_ROWS + k) * (CF_COLS + 1);
-    static bool attr = false;
-    if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * (CF_ROWS + MAXQ) * (CF_COLS + 1)))); attr = true; }
-    coeff_kernel<<<(unsigned)metis_ceil_div(rows, CF_ROWS), 256, smem, s>>>(x, rows, cols, k, basis, coef); METIS_COUNT_LAUNCH();
-    res_coef = coef; res_scale = nullptr; res_basis = basis;
+    basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(basis, cols, k, kp, bs, bt); METIS_COUNT_LAUNCH();
+    const size_t smem = sizeof(float) * 9 * 32 * kp;
+    switch (kp) {
+      case 16: coeff_mma_kernel<16><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
+      case 32: coeff_mma_kernel<32><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
+      case 48: coeff_mma_kernel<48><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
+      default: coeff_mma_kernel<64><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
+    }
+    METIS_COUNT_LAUNCH();
   }
-  // (6) fused residual + quantizer (tensor scale from the source tensor's amax)
   {
     QuantParams qp{};
     qp.rows = rows; qp.cols = cols; qp.rounding = rounding; qp.seed = seed; qp.stream_id = METIS_STREAM_RESIDUAL;
     qp.e_stride_r = cols; qp.e_stride_c = 1;
     if (want_c) { qp.c_codes = rc.codes; qp.c_scales = rc.scales; qp.c_layout = rc.sf_layout; }
     if (want_r) { qp.r_codes = rr.codes; qp.r_scales = rr.scales; qp.r_layout = rr.sf_layout; }
-    const bool sr = rounding == METIS_ROUND_SR;
-    const size_t smem = smem_bytes(sr) + sizeof(float) * 2 * k * TILE;
-    static bool attr = false;
-    if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem_bytes(true) + sizeof(float) * 2 * MAXQ * TILE))); attr = true; }
+    const size_t smem = smem_bytes(rounding == METIS_ROUND_SR);
     dim3 grid((unsigned)metis_ceil_div(cols, TILE), (unsigned)metis_ceil_div(rows, TILE));
-    residual_quant_kernel<<<grid, THREADS, smem, s>>>(x, k, res_coef, res_scale, res_basis, qp, amax,
-                                                      want_c ? rc.tensor_scale : nullptr,
-                                                      want_r ? rr.tensor_scale : nullptr, residual_dense); METIS_COUNT_LAUNCH();
+    float* t0 = want_c ? rc.tensor_scale : nullptr; float* t1 = want_r ? rr.tensor_scale : nullptr;
+    switch (kp) {
+      case 16: residual_quant_kernel<16><<<grid, THREADS, smem, s>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+      case 32: residual_quant_kernel<32><<<grid, THREADS, smem, s>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+      case 48: residual_quant_kernel<48><<<grid, THREADS, smem, s>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+      default: residual_quant_kernel<64><<<grid, THREADS, smem, s>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+    }
+    METIS_COUNT_LAUNCH();
   }
   if (!full) {
-    // (7) Rayleigh-Ritz on C^T C, rotate both factors, singular values
-    int64_t rpp; const int parts = gram_parts(rows, &rpp);
-    gram_kernel<<<parts, 256, 0, s>>>(coef, rows, k, 1, rows, rpp, gram); METIS_COUNT_LAUNCH();
-    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram, parts, k, evals2, evecs2); METIS_COUNT_LAUNCH();
-    right_rotate_sign_kernel<<<k, 256, 0, s>>>(basis, cols, k, evecs2, out->right, sign); METIS_COUNT_LAUNCH();
-    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 256), 256, 0, s>>>(coef, rows, k, k, rows, 1, evecs2, evals2, sign,
-                                                                           out->left, out->sigma); METIS_COUNT_LAUNCH();
+    // (7) Rayleigh-Ritz on C^T C (Gram partials came out of the broadcast pass), rotate both factors
+    reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 128), 128, 0, s>>>(gram_c, n_cta_c, kp * kp, gram1); METIS_COUNT_LAUNCH();
+    jacobi_eig_kernel<<<1, jacobi_threads(k), JACOBI_SMEM, s>>>(gram1, k, kp, evals2, evecs2); METIS_COUNT_LAUNCH();
+    right_rotate_kernel<<<n_cand, 256, 0, s>>>(basis, cols, k, evecs2, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
+    sign_fix_kernel<<<dim3(n_cand, k), 256, 0, s>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign); METIS_COUNT_LAUNCH();
+    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 64, 0, s>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
+                                                                           out->left, out->sigma, nullptr, 0, nullptr); METIS_COUNT_LAUNCH();
   }
   METIS_CUDA_TRY(cudaGetLastError());
   // (8) quantize the factors (stored transposed: k x rows, k x cols; blocks along the long dimension)
