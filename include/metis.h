@@ -183,6 +183,24 @@ metis_status_t metis_linear_fwd(metis_handle_t h, const metis_operand_t* x, cons
                                 void* y, int32_t y_dtype, int64_t ldy, void* ws, size_t ws_bytes,
                                 metis_stream_t stream);
 
+/* Forward layer without a caller workspace.  (No counterpart in the paper: this is an integration aid.)
+ * Same result as metis_linear_fwd, bit for bit, but the intermediates live in a METIS_STATIC_WS_BYTES array
+ * built into the library image (each GPU that loads the library carries it until the process exits).  It is
+ * meant for callers that own inputs and outputs but cannot obtain scratch memory: a process whose memory
+ * pool already holds every free byte of the device, or a plug-in that is not allowed to call an allocator.
+ * The call allocates nothing on host or device.
+ *  - Limit: layers whose metis_workspace_bytes(2, l, n, k, 0) exceeds METIS_STATIC_WS_BYTES are refused with
+ *    METIS_ERR_WORKSPACE and nothing is enqueued.
+ *  - h's device must be the current device (else METIS_ERR_INVALID_ARG).
+ *  - The first call on each device looks up the array's device address (a one-time runtime query); make that
+ *    first call during start-up, before any stream capture is begun.
+ *  - All calls on a device share the one array, which keeps whatever the last call left in it; the layer
+ *    needs no zeroed scratch, so nothing is cleared.  Two calls whose kernels overlap on the GPU (different
+ *    streams, or different threads) race on it: serialise them. */
+#define METIS_STATIC_WS_BYTES (4u << 20)
+metis_status_t metis_linear_fwd_static_ws(metis_handle_t h, const metis_operand_t* x, const metis_operand_t* w,
+                                          void* y, int32_t y_dtype, int64_t ldy, metis_stream_t stream);
+
 /* dx (l x m) = Dq Wq' (Eq. 3; needs dy->res_by_cols, w->res_by_rows) and
  * dw (n x m) = Dq''^T Xq'' (weight gradient; needs dy->res_by_rows, x->res_by_rows).
  * Either output may be NULL to skip it. */

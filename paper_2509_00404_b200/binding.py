@@ -27,7 +27,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "ALIGNMENT", 4: "WORKS
 EXPORTED = ["metis_create", "metis_destroy", "metis_last_device_status", "metis_debug_quantile_table",
             "metis_debug_launch_count",
             "metis_sf_bytes", "metis_workspace_bytes", "metis_default_sample_count", "metis_quantize_nvfp4",
-            "metis_split", "metis_linear_fwd", "metis_linear_bwd", "metis_gemm_nvfp4"]
+            "metis_split", "metis_linear_fwd", "metis_linear_fwd_static_ws", "metis_linear_bwd", "metis_gemm_nvfp4"]
 
 
 class MetisError(RuntimeError):
@@ -78,6 +78,7 @@ def lib():
                                        vp, sz, vp]
     l.metis_split.argtypes = [vp, vp, i64, i64, i32, i32, i32, i64, u64, i32, i32, P(OperandStruct), vp, vp, sz, vp]
     l.metis_linear_fwd.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp, sz, vp]
+    l.metis_linear_fwd_static_ws.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp]
     l.metis_linear_bwd.argtypes = [vp, P(OperandStruct), P(OperandStruct), P(OperandStruct), vp, i32, i64, vp, i32,
                                    i64, vp, sz, vp]
     l.metis_gemm_nvfp4.argtypes = [vp, P(NvFp4Struct), P(NvFp4Struct), vp, i32, i64, i32, vp]
@@ -279,6 +280,15 @@ class Handle:
         _check("metis_linear_fwd", lib().metis_linear_fwd(self._h, ctypes.byref(sx), ctypes.byref(sw), _ptr(y),
                                                           _dtype_code(y), y.stride(0), _ptr(ws), ws.numel(),
                                                           _stream_ptr(stream)))
+        return y
+
+    def linear_fwd_static_ws(self, x_op, w_op, out_dtype=torch.float32, out=None, stream=None):
+        """metis_linear_fwd_static_ws: forward layer for callers that cannot supply scratch memory (for example
+        because a framework pool already owns all device memory).  Allocates no workspace here either."""
+        y = out if out is not None else torch.empty((x_op.rows, w_op.rows), dtype=out_dtype, device="cuda")
+        sx, sw = x_op.struct(), w_op.struct()
+        _check("metis_linear_fwd_static_ws", lib().metis_linear_fwd_static_ws(
+            self._h, ctypes.byref(sx), ctypes.byref(sw), _ptr(y), _dtype_code(y), y.stride(0), _stream_ptr(stream)))
         return y
 
     def linear_bwd(self, dy_op, x_op, w_op, out_dtype=torch.float32, need_dx=True, need_dw=True, out=None, stream=None):
