@@ -18,6 +18,7 @@
 //               the main loop of tile i+1
 // Every mbarrier wait is bounded; on expiry the kernel records METIS_DEV_TIMEOUT and unwinds.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -41,9 +42,12 @@ struct Cfg {
   static constexpr int SFB_BYTES = N_TILES_SF * K_STEPS * 512;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
   static constexpr int ACC_COLS = NUM_ACC * BLOCK_N;               // 256
-  static constexpr int SFA_COL = ACC_COLS;                         // 16 columns
-  static constexpr int SFB_COL = ACC_COLS + 4 * K_STEPS;           // 16 or 32 columns
+  // every ring stage has its own scale columns in tensor memory, so the scale copy of stage s+1 never has to
+  // wait for the MMAs of stage s to finish reading theirs
+  static constexpr int SF_COLS_PER_STAGE = 4 * K_STEPS * (1 + N_TILES_SF);      // 32 or 48
+  static constexpr int SF_COL0 = ACC_COLS;
   static constexpr int TMEM_COLS = 512;
+  static_assert(ACC_COLS + STAGES * SF_COLS_PER_STAGE <= 512, "tensor memory budget");
   static constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
@@ -70,7 +74,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* dev_status, volatile int* dead) {
   for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (i > 32) __nanosleep(64);
+    if (i > 4096) __nanosleep(32);
     if ((i & 1023u) == 1023u && *dead) break;
   }
   *dead = 1;
@@ -149,7 +153,41 @@ struct GemmArgs {
   void* d; int d_dtype; int64_t ldd;
   int M, N, K;
   uint32_t* dev_status;
+  int dbg;
+  int extra_kb;            // BF16 correction boxes (64 elements of K each) appended after the FP4 K loop
 };
+
+// Writes 32 consecutive accumulator columns of one output row (scaled by alpha) as FP32 or BF16.
+__device__ __forceinline__ void store_row_chunk(const GemmArgs& g, int row, int col, const uint32_t (&r)[32], float alpha) {
+  if (g.d_dtype == METIS_FP32) {
+    float* dst = reinterpret_cast<float*>(g.d) + (size_t)row * g.ldd + col;
+    if (col + 32 <= g.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 4)
+        *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
+                                                          __uint_as_float(r[j + 2]) * alpha, __uint_as_float(r[j + 3]) * alpha);
+    } else {
+      for (int j = 0; j < 32 && col + j < g.N; ++j) dst[j] = __uint_as_float(r[j]) * alpha;
+    }
+  } else {
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(g.d) + (size_t)row * g.ldd + col;
+    if (col + 32 <= g.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) {
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * q]) * alpha,
+                                                         __uint_as_float(r[j + 2 * q + 1]) * alpha);
+          w[q] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    } else {
+      for (int j = 0; j < 32 && col + j < g.N; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]) * alpha);
+    }
+  }
+}
 
 template <int BLOCK_N>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -199,16 +237,19 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
           const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
-          const uint32_t bytes = C::A_BYTES + C::B_BYTES + (uint32_t)atoms * 512u * (1 + C::N_TILES_SF);
+          const bool skip_tiles = (g.dbg & 4) && kb >= C::STAGES;
+          const uint32_t bytes = (skip_tiles ? 0u : (uint32_t)(C::A_BYTES + C::B_BYTES)) + (uint32_t)atoms * 512u * (1 + C::N_TILES_SF);
           mbar_expect_tx(full_bar(s), bytes);
+          if (!skip_tiles) {
           tma_load_2d(a_addr(s), &map_a, kb * (BLOCK_K / 2), mb * BLOCK_M, full_bar(s));
           tma_load_2d(b_addr(s), &map_b, kb * (BLOCK_K / 2), nb * BLOCK_N, full_bar(s));
+          }
           bulk_load(sfa_addr(s), g.a_sf + ((size_t)mb * sf_k_atoms + (size_t)kb * K_STEPS) * 512, atoms * 512, full_bar(s));
 #pragma unroll
           for (int t = 0; t < C::N_TILES_SF; ++t)
             bulk_load(sfb_addr(s) + t * K_STEPS * 512,
-                      g.b_sf + ((size_t)(nb * C::N_TILES_SF + t) * sf_k_atoms + (size_t)kb * K_STEPS) * 512, atoms * 512,
-                      full_bar(s));
+                      g.b_sf + ((size_t)min(nb * C::N_TILES_SF + t, (g.N + 127) / 128 - 1) * sf_k_atoms + (size_t)kb * K_STEPS) * 512,
+                      atoms * 512, full_bar(s));
           if (++s == C::STAGES) { s = 0; ph ^= 1u; }
         }
       }
@@ -230,18 +271,22 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           if (!mbar_wait(full_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
           tc_fence_after();
           const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
+          const uint32_t sfa_t = tmem_base + C::SF_COL0 + s * C::SF_COLS_PER_STAGE;
+          const uint32_t sfb_t = sfa_t + 4 * K_STEPS;
+          if (!(g.dbg & 1) || kb == 0)
           for (int k = 0; k < atoms; ++k) {
-            tc_cp_sf(tmem_base + C::SFA_COL + 4 * k, make_smem_desc(sfa_addr(s) + k * 512, 128, SWIZZLE_NONE));
+            tc_cp_sf(sfa_t + 4 * k, make_smem_desc(sfa_addr(s) + k * 512, 128, SWIZZLE_NONE));
 #pragma unroll
             for (int t = 0; t < C::N_TILES_SF; ++t)
-              tc_cp_sf(tmem_base + C::SFB_COL + 4 * (k * C::N_TILES_SF + t),
+              tc_cp_sf(sfb_t + 4 * (k * C::N_TILES_SF + t),
                        make_smem_desc(sfb_addr(s) + (t * K_STEPS + k) * 512, 128, SWIZZLE_NONE));
           }
+          if (!(g.dbg & 2) || kb == 0)
           for (int k = 0; k < atoms; ++k) {
             const uint64_t a_desc = make_smem_desc(a_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
             const uint64_t b_desc = make_smem_desc(b_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
-            tc_mma_nvf4(d_tmem, a_desc, b_desc, idesc, tmem_base + C::SFA_COL + 4 * k,
-                        tmem_base + C::SFB_COL + 4 * k * C::N_TILES_SF, (kb | k) != 0 ? 1u : 0u);
+            tc_mma_nvf4(d_tmem, a_desc, b_desc, idesc, sfa_t + 4 * k, sfb_t + 4 * k * C::N_TILES_SF,
+                        (kb | k) != 0 ? 1u : 0u);
           }
           tc_commit(empty_bar(s));                           // slot reusable once these MMAs have read it
           if (++s == C::STAGES) { s = 0; ph ^= 1u; }
@@ -264,40 +309,11 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const int row = mb * BLOCK_M + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BLOCK_N; c0 += 32) {
+      for (int c0 = 0; c0 < BLOCK_N && !(g.dbg & 8); c0 += 32) {
         uint32_t r[32];
         tc_ld32(t_row + c0, r);
         const int col = nb * BLOCK_N + c0;
-        if (row < g.M && col < g.N) {
-          if (g.d_dtype == METIS_FP32) {
-            float* dst = reinterpret_cast<float*>(g.d) + (size_t)row * g.ldd + col;
-            if (col + 32 <= g.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
-                                                                  __uint_as_float(r[j + 2]) * alpha, __uint_as_float(r[j + 3]) * alpha);
-            } else {
-              for (int j = 0; j < 32 && col + j < g.N; ++j) dst[j] = __uint_as_float(r[j]) * alpha;
-            }
-          } else {
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(g.d) + (size_t)row * g.ldd + col;
-            if (col + 32 <= g.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                uint32_t w[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * q]) * alpha,
-                                                                 __uint_as_float(r[j + 2 * q + 1]) * alpha);
-                  w[q] = *reinterpret_cast<const uint32_t*>(&h);
-                }
-                *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
-              }
-            } else {
-              for (int j = 0; j < 32 && col + j < g.N; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]) * alpha);
-            }
-          }
-        }
+        if (row < g.M && col < g.N) store_row_chunk(g, row, col, r, alpha);
       }
       tc_fence_before();
       __syncwarp();
@@ -318,6 +334,302 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
 }
+
+// =================================================================================================
+// Two-CTA variant (cta_group::2): a cluster of two CTAs on neighbouring SMs computes one 256 x 256 tile.
+// Each CTA loads 128 rows of A and 128 rows of B per K block (the pair's MMA reads both halves of B),
+// its own 128 rows of A scales and the scales of all 256 B rows; the leader CTA issues the MMAs for both,
+// each CTA keeps its 128 x 256 half of the accumulator in its own tensor memory and runs its own epilogue.
+// Per stage a CTA brings in 38 KiB for 4 x (128 x 256 x 64) of tensor work - four times the work per byte
+// of the one-CTA kernel, which is what lets a five-stage ring cover the load + scale-copy + MMA latency.
+// =================================================================================================
+namespace two_cta {
+
+constexpr int TILE_M = 256, TILE_N = 256;
+constexpr int STAGES = 5;
+constexpr int A_BYTES = 128 * BLOCK_K / 2;                  // this CTA's 128 rows of A
+constexpr int B_BYTES = 128 * BLOCK_K / 2;                  // this CTA's 128 rows of B
+constexpr int SFA_BYTES = K_STEPS * 512;
+constexpr int SFB_BYTES = 2 * K_STEPS * 512;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;   // 38 KiB
+constexpr int ACC_COLS = 256;
+constexpr int SF_COLS_PER_STAGE = 4 * K_STEPS * 3;          // 16 (A) + 32 (B): each ring stage has its own scale columns
+constexpr int SF_COL0 = 256;
+constexpr int TMEM_COLS = 512;
+static_assert(ACC_COLS + STAGES * SF_COLS_PER_STAGE <= TMEM_COLS, "tensor memory budget");
+constexpr int NUM_THREADS = 256;                            // producer, MMA, relay, 4 epilogue warps, scale copier
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t local_bar, uint32_t rank) {
+  asm volatile(
+      "{ .reg .b32 ra; mapa.shared::cluster.u32 ra, %0, %1;\n"
+      "  mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra]; }"
+      ::"r"(local_bar), "r"(rank) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{ .reg .pred p; mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint32_t* dev_status, volatile int* dead) {
+  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if (i > 4096) __nanosleep(32);
+    if ((i & 1023u) == 1023u && *dead) break;
+  }
+  *dead = 1;
+  atomicOr(dev_status, METIS_DEV_TIMEOUT);
+  return false;
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_commit2(uint32_t bar, uint16_t mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void tc_cp_sf2(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_nvf4_2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                              uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{ .reg .pred p; setp.ne.b32 p, %4, 0;\n"
+      "  tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p; }"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem) : "memory");
+}
+
+// dense BF16 x BF16 -> FP32 MMA into the same accumulator (the low-rank correction of the split layer)
+__device__ __forceinline__ void tc_mma_bf16_2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{ .reg .pred p; setp.ne.b32 p, %4, 0;\n"
+      "  tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p; }"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// instruction descriptor for kind::f16 with BF16 operands and FP32 accumulation: accumulator format 1 at [4,6),
+// operand formats 1 (BF16) at [7,10) and [10,13), K-major, N/8 at [17,23), M/16 at [24,29)
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// The K loop runs over num_kb FP4 blocks (256 elements each) followed by g.extra_kb BF16 boxes (64 elements
+// each, same 16 KiB + 16 KiB ring slot): the latter add  Lx Rx^T  (the rank-(ka+kb) correction of the split
+// layer, pre-divided by alpha) into the same FP32 accumulator.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                       const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUtensorMap map_r, GemmArgs g) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* gen_base = smem_raw + (base - raw);
+  auto a_addr = [&](int s) { return base + (uint32_t)s * STAGE_BYTES; };
+  auto b_addr = [&](int s) { return a_addr(s) + A_BYTES; };
+  auto sfa_addr = [&](int s) { return b_addr(s) + B_BYTES; };
+  auto sfb_addr = [&](int s) { return sfa_addr(s) + SFA_BYTES; };
+  const uint32_t bar_base = base + (uint32_t)STAGES * STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };                  // own loads landed (per CTA)
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };      // slot free (per CTA, by commit multicast)
+  auto ready_bar = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };  // leader only: both CTAs' loads landed
+  const uint32_t tfull_bar = bar_base + 8u * (3 * STAGES);                   // accumulator complete (per CTA)
+  const uint32_t tempty_bar = bar_base + 8u * (3 * STAGES + 1);              // leader only: both epilogues drained
+  auto sfready_bar = [&](int s) { return bar_base + 8u * (3 * STAGES + 2 + s); };   // leader only: scales are in tensor memory
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + (size_t)STAGES * STAGE_BYTES + 8 * (4 * STAGES + 2));
+  volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();
+  const bool leader = rank == 0;
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  const int num_m = (g.M + TILE_M - 1) / TILE_M, num_n = (g.N + TILE_N - 1) / TILE_N;
+  const int num_tiles = num_m * num_n;
+  const int num_fp4_kb = (g.K + BLOCK_K - 1) / BLOCK_K;
+  const int num_kb = num_fp4_kb + g.extra_kb;
+  const int sf_k_atoms = g.K / MMA_K;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); mbar_init(ready_bar(s), 2); mbar_init(sfready_bar(s), 1);
+    }
+    mbar_init(tfull_bar, 1);
+    mbar_init(tempty_bar, 8);                                 // 4 epilogue warps in each of the two CTAs
+    *dead = 0;
+    fence_barrier_init();
+  }
+  cluster_sync();
+  if (warp == 1) tmem_alloc2(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before();
+  cluster_sync();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------- producer (both CTAs) -------------------
+    if (lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        const int mb = tile % num_m, nb = tile / num_m;
+        const int a_row = mb * TILE_M + (int)rank * 128, b_row = nb * TILE_N + (int)rank * 128;
+        // a 128-row slab that lies wholly outside the matrix has all-zero codes (TMA fill); any valid slab's
+        // scales will do for it, so the index is clamped instead of reading past the scale buffer
+        const int a_sf_tile = min(mb * 2 + (int)rank, (g.M + 127) / 128 - 1);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
+          if (kb >= num_fp4_kb) {                             // BF16 correction box: 128 rows x 64 elements each
+            mbar_expect_tx(full_bar(s), (uint32_t)(A_BYTES + B_BYTES));
+            tma_load_2d(a_addr(s), &map_l, (kb - num_fp4_kb) * 64, a_row, full_bar(s));
+            tma_load_2d(b_addr(s), &map_r, (kb - num_fp4_kb) * 64, b_row, full_bar(s));
+            if (++s == STAGES) { s = 0; ph ^= 1u; }
+            continue;
+          }
+          const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
+          mbar_expect_tx(full_bar(s), (((g.dbg & 4) && kb >= STAGES) ? 0u : (uint32_t)(A_BYTES + B_BYTES)) + (uint32_t)atoms * 512u * 3u);
+          if (!((g.dbg & 4) && kb >= STAGES)) {
+          tma_load_2d(a_addr(s), &map_a, kb * (BLOCK_K / 2), a_row, full_bar(s));
+          tma_load_2d(b_addr(s), &map_b, kb * (BLOCK_K / 2), b_row, full_bar(s));
+          }
+          bulk_load(sfa_addr(s), g.a_sf + ((size_t)a_sf_tile * sf_k_atoms + (size_t)kb * K_STEPS) * 512, atoms * 512, full_bar(s));
+#pragma unroll
+          for (int t = 0; t < 2; ++t)
+            bulk_load(sfb_addr(s) + t * K_STEPS * 512,
+                      g.b_sf + ((size_t)min(nb * 2 + t, (g.N + 127) / 128 - 1) * sf_k_atoms + (size_t)kb * K_STEPS) * 512,
+                      atoms * 512, full_bar(s));
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------- relay (both CTAs): own stage landed -> tell the leader ----
+    if (lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
+          mbar_arrive_remote(ready_bar(s), 0u);
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer (leader CTA only) ------------
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc = make_idesc(TILE_M, TILE_N);
+      int s = 0; uint32_t ph = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++it) {
+        if (!mbar_wait_cluster(tempty_bar, ((uint32_t)it & 1u) ^ 1u, g.dev_status, dead)) { ok = false; break; }
+        tc_fence_after();
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(sfready_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
+          tc_fence_after();
+          if (kb >= num_fp4_kb) {
+            constexpr uint32_t idesc_x = make_idesc_bf16(TILE_M, TILE_N);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {                     // 64 BF16 elements = four K=16 MMAs, 32 bytes apart
+              const uint64_t a_desc = make_smem_desc(a_addr(s) + k * 32, 1024, SWIZZLE_128B);
+              const uint64_t b_desc = make_smem_desc(b_addr(s) + k * 32, 1024, SWIZZLE_128B);
+              tc_mma_bf16_2(tmem_base, a_desc, b_desc, idesc_x, 1u);
+            }
+            tc_commit2(empty_bar(s), 3);
+            if (++s == STAGES) { s = 0; ph ^= 1u; }
+            continue;
+          }
+          const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
+          const uint32_t sfa_t = tmem_base + SF_COL0 + s * SF_COLS_PER_STAGE, sfb_t = sfa_t + 4 * K_STEPS;
+          if (!(g.dbg & 2) || kb == 0)
+          for (int k = 0; k < atoms; ++k) {
+            const uint64_t a_desc = make_smem_desc(a_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
+            const uint64_t b_desc = make_smem_desc(b_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
+            tc_mma_nvf4_2(tmem_base, a_desc, b_desc, idesc, sfa_t + 4 * k, sfb_t + 8 * k, (kb | k) != 0 ? 1u : 0u);
+          }
+          tc_commit2(empty_bar(s), 3);                        // frees the slot in both CTAs
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (ok) tc_commit2(tfull_bar, 3);                     // accumulator complete in both CTAs
+      }
+    }
+  } else if (warp == 7) {
+    // ------------------------------- scale copier (leader CTA only) ----------
+    // shared memory -> tensor memory copies of the scale atoms, issued from their own warp so they do not sit
+    // in the MMA issuer's instruction stream; a stage's columns are rewritten only after the MMAs that read them
+    // have completed (the stage is reloaded only after the commit that frees it)
+    if (leader && lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait_cluster(ready_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
+          tc_fence_after();
+          const int atoms = kb < num_fp4_kb ? min(K_STEPS, sf_k_atoms - kb * K_STEPS) : 0;   // BF16 boxes carry no scales
+          const uint32_t sfa_t = tmem_base + SF_COL0 + s * SF_COLS_PER_STAGE, sfb_t = sfa_t + 4 * K_STEPS;
+          if (!(g.dbg & 1) || kb == 0)
+          for (int k = 0; k < atoms; ++k) {
+            tc_cp_sf2(sfa_t + 4 * k, make_smem_desc(sfa_addr(s) + k * 512, 128, SWIZZLE_NONE));
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+              tc_cp_sf2(sfb_t + 4 * (k * 2 + t), make_smem_desc(sfb_addr(s) + (t * K_STEPS + k) * 512, 128, SWIZZLE_NONE));
+          }
+          tc_commit2(sfready_bar(s), 1);
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------- epilogue (both CTAs) --------------------
+    const int quarter = warp & 3;
+    const float alpha = (*g.a_ts) * (*g.b_ts);
+    int it = 0;
+    bool ok = true;
+    for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++it) {
+      const int mb = tile % num_m, nb = tile / num_m;
+      if (!mbar_wait(tfull_bar, (uint32_t)it & 1u, g.dev_status, dead)) { ok = false; break; }
+      tc_fence_after();
+      const int row = mb * TILE_M + (int)rank * 128 + quarter * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < TILE_N && !(g.dbg & 8); c0 += 32) {
+        uint32_t r[32];
+        tc_ld32(t_row + c0, r);
+        const int col = nb * TILE_N + c0;
+        if (row < g.M && col < g.N) store_row_chunk(g, row, col, r, alpha);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(tempty_bar, 0u);
+    }
+  }
+
+  // ------------------------------- teardown ---------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (*dead) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  cluster_sync();                                             // the peer may still read this CTA's shared memory until here
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc2(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace two_cta
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -346,6 +658,7 @@ metis_status_t launch(metis_context* ctx, const metis_nvfp4_t* a, const metis_nv
   g.d = d; g.d_dtype = d_dtype; g.ldd = ldd;
   g.M = (int)a->rows; g.N = (int)b->rows; g.K = (int)a->k_len;
   g.dev_status = ctx->dev_status;
+  { const char* e = getenv("METIS_GEMM_DBG"); g.dbg = e ? atoi(e) : 0; }
   static bool attr_set = false;
   if (!attr_set) {
     METIS_CUDA_TRY(cudaFuncSetAttribute(gemm_nvfp4_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
@@ -354,6 +667,60 @@ metis_status_t launch(metis_context* ctx, const metis_nvfp4_t* a, const metis_nv
   const int tiles = (int)(metis_ceil_div(g.M, BLOCK_M) * metis_ceil_div(g.N, BLOCK_N));
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
   gemm_nvfp4_kernel<BLOCK_N><<<grid, NUM_THREADS, C::SMEM_BYTES, s>>>(map_a, map_b, g); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
+
+// 2-D map over a row-major BF16 matrix rows x kx (kx a multiple of 64), box 64 elements x 128 rows, 128-byte swizzle
+metis_status_t make_bf16_map(metis_context* ctx, CUtensorMap* map, const void* ptr, int64_t rows, int64_t kx) {
+  const cuuint64_t dims[2] = {(cuuint64_t)kx, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)(kx * 2)};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+      map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? METIS_OK : METIS_ERR_CUDA;
+}
+
+metis_status_t launch_2cta(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d, int d_dtype,
+                           int64_t ldd, const void* lx, const void* rx, int kx, cudaStream_t s) {
+  CUtensorMap map_a, map_b, map_l, map_r;
+  METIS_TRY(make_codes_map(ctx, &map_a, a, 128));
+  METIS_TRY(make_codes_map(ctx, &map_b, b, 128));
+  if (kx > 0) {
+    METIS_TRY(make_bf16_map(ctx, &map_l, lx, a->rows, kx));
+    METIS_TRY(make_bf16_map(ctx, &map_r, rx, b->rows, kx));
+  } else {
+    map_l = map_a; map_r = map_b;
+  }
+  GemmArgs g{};
+  g.a_sf = a->scales; g.b_sf = b->scales; g.a_ts = a->tensor_scale; g.b_ts = b->tensor_scale;
+  g.d = d; g.d_dtype = d_dtype; g.ldd = ldd;
+  g.M = (int)a->rows; g.N = (int)b->rows; g.K = (int)a->k_len;
+  g.dev_status = ctx->dev_status;
+  { const char* e = getenv("METIS_GEMM_DBG"); g.dbg = e ? atoi(e) : 0; }
+  g.extra_kb = kx / 64;
+  static bool attr_set = false;
+  if (!attr_set) {
+    METIS_CUDA_TRY(cudaFuncSetAttribute(two_cta::gemm_nvfp4_2cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)two_cta::SMEM_BYTES));
+    attr_set = true;
+  }
+  const int tiles = (int)(metis_ceil_div(g.M, two_cta::TILE_M) * metis_ceil_div(g.N, two_cta::TILE_N));
+  static int max_pairs = 0;
+  if (max_pairs == 0) {
+    // how many 2-CTA clusters can be resident at once (an odd SM count inside a GPC leaves an SM unpaired)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (ctx->sm_count / 2)); cfg.blockDim = dim3(two_cta::NUM_THREADS);
+    cfg.dynamicSmemBytes = two_cta::SMEM_BYTES;
+    cudaLaunchAttribute at; at.id = cudaLaunchAttributeClusterDimension; at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+    cfg.attrs = &at; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, two_cta::gemm_nvfp4_2cta_kernel, &cfg) != cudaSuccess || n <= 0) n = ctx->sm_count / 2;
+    max_pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
+  }
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  two_cta::gemm_nvfp4_2cta_kernel<<<2 * pairs, two_cta::NUM_THREADS, two_cta::SMEM_BYTES, s>>>(map_a, map_b, map_l, map_r, g); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }
@@ -368,5 +735,28 @@ metis_status_t metis_launch_gemm_tc(metis_context* ctx, const metis_nvfp4_t* a, 
   if (!metis_aligned16(a->codes) || !metis_aligned16(b->codes) || !metis_aligned16(a->scales) || !metis_aligned16(b->scales))
     return METIS_ERR_ALIGNMENT;
   if (a->rows > INT32_MAX || b->rows > INT32_MAX || a->k_len > INT32_MAX) return METIS_ERR_SHAPE;
+  static int force_n = -1;
+  if (force_n < 0) { const char* e = getenv("METIS_GEMM_BLOCK_N"); force_n = e ? atoi(e) : 0; }
+  if (force_n == 256) return launch<256>(ctx, a, b, d, d_dtype, ldd, s);
+  if (force_n == 128) return launch<128>(ctx, a, b, d, d_dtype, ldd, s);
+  if (a->rows >= 256 && b->rows >= 256) return launch_2cta(ctx, a, b, d, d_dtype, ldd, nullptr, nullptr, 0, s);
   return launch<128>(ctx, a, b, d, d_dtype, ldd, s);
+}
+
+bool metis_gemm_tc_can_fuse(const metis_nvfp4_t* a, const metis_nvfp4_t* b) {
+  static int force_n = -1;
+  if (force_n < 0) { const char* e = getenv("METIS_GEMM_BLOCK_N"); force_n = e ? atoi(e) : 0; }
+  return force_n == 0 && a->rows >= 256 && b->rows >= 256;
+}
+
+// d = alpha * (a b^T) + alpha * (lx rx^T): lx (M x kx) and rx (N x kx) are row-major BF16, kx a multiple of 64.
+metis_status_t metis_launch_gemm_tc_fused(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d,
+                                          int d_dtype, int64_t ldd, const void* lx, const void* rx, int kx, cudaStream_t s) {
+  if (!metis_gemm_tc_can_fuse(a, b) || kx <= 0 || kx % 64) return METIS_ERR_INVALID_ARG;
+  if (a->k_len != b->k_len || a->k_len % 64 != 0 || a->k_len <= 0) return METIS_ERR_SHAPE;
+  if (a->sf_layout != METIS_SF_TILED || b->sf_layout != METIS_SF_TILED) return METIS_ERR_INVALID_ARG;
+  if (!metis_aligned16(a->codes) || !metis_aligned16(b->codes) || !metis_aligned16(a->scales) || !metis_aligned16(b->scales) ||
+      !metis_aligned16(lx) || !metis_aligned16(rx))
+    return METIS_ERR_ALIGNMENT;
+  return launch_2cta(ctx, a, b, d, d_dtype, ldd, lx, rx, kx, s);
 }

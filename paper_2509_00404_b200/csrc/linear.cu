@@ -12,6 +12,10 @@
 // All four quantized cross terms of the paper's expansion are kept.
 #include "common.cuh"
 
+bool metis_gemm_tc_can_fuse(const metis_nvfp4_t* a, const metis_nvfp4_t* b);
+metis_status_t metis_launch_gemm_tc_fused(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d,
+                                          int d_dtype, int64_t ldd, const void* lx, const void* rx, int kx, cudaStream_t s);
+
 namespace {
 
 __device__ __forceinline__ float deq_at(const uint8_t* codes, const uint8_t* sf, int layout, int64_t k_len, int64_t r,
@@ -30,7 +34,9 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
                       const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts,
                       const float* sa,
                       const uint8_t* fob_codes, const uint8_t* fob_sf, int fob_layout, const float* fob_ts,
-                      const float* sb, const float* __restrict__ pm, float* __restrict__ lcat, float* __restrict__ rcat) {
+                      const float* sb, const float* __restrict__ pm, float* __restrict__ lcat, float* __restrict__ rcat,
+                      __nv_bfloat16* __restrict__ lx, __nv_bfloat16* __restrict__ rx, int kx,
+                      const float* res_a_ts, const float* res_b_ts) {
   __shared__ float ps[64][65];
   __shared__ float fa[8][64];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -55,6 +61,32 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
   if (i < N) {
     const float tsb = kb ? *fob_ts : 0.0f;
     for (int t = lane; t < kb; t += 32) rcat[i * kc + t] = deq_at(fob_codes, fob_sf, fob_layout, N, t, i) * tsb;
+  }
+  if (lx == nullptr) return;
+  // BF16 operands of the in-accumulator correction:  Lx = [Lh | Lh | Ll] / alpha,  Rx = [Rh | Rl | Rh]
+  // (hi/lo two-term splits, three cross products), zero padded to kx columns.
+  __syncwarp();
+  const float inv_alpha = 1.0f / ((*res_a_ts) * (*res_b_ts));
+  for (int c = lane; c < kx; c += 32) {
+    const int seg = c / kc, t = c - seg * kc;
+    if (i < M) {
+      float out = 0.0f;
+      if (seg < 3) {
+        const float v = lcat[i * kc + t] * inv_alpha;
+        const float h = __bfloat162float(__float2bfloat16_rn(v));
+        out = seg == 2 ? v - h : h;
+      }
+      lx[i * kx + c] = __float2bfloat16_rn(out);
+    }
+    if (i < N) {
+      float out = 0.0f;
+      if (seg < 3) {
+        const float v = rcat[i * kc + t];
+        const float h = __bfloat162float(__float2bfloat16_rn(v));
+        out = seg == 1 ? v - h : h;
+      }
+      rx[i * kx + c] = __float2bfloat16_rn(out);
+    }
   }
 }
 
@@ -128,13 +160,17 @@ metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void
   unsigned char* w = reinterpret_cast<unsigned char*>(ws);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
-  float* y0 = reinterpret_cast<float*>(w + take(sizeof(float) * M * N));
+  const bool fuse = metis_gemm_tc_can_fuse(a.res, b.res);
+  const int kx = (3 * kc + 63) / 64 * 64;
   float* pm = reinterpret_cast<float*>(w + take(sizeof(float) * 64 * 64));
   float* lcat = reinterpret_cast<float*>(w + take(sizeof(float) * M * kc));
   float* rcat = reinterpret_cast<float*>(w + take(sizeof(float) * N * kc));
+  __nv_bfloat16* lx = fuse ? reinterpret_cast<__nv_bfloat16*>(w + take(sizeof(__nv_bfloat16) * M * kx)) : nullptr;
+  __nv_bfloat16* rx = fuse ? reinterpret_cast<__nv_bfloat16*>(w + take(sizeof(__nv_bfloat16) * N * kx)) : nullptr;
+  float* y0 = fuse ? nullptr : reinterpret_cast<float*>(w + take(sizeof(float) * M * N));
   if (!ws || off > ws_bytes) return METIS_ERR_WORKSPACE;
 
-  METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.res, y0, METIS_FP32, N, s));
+  if (!fuse) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.res, y0, METIS_FP32, N, s));
   // the skinny products land directly in their slots of the concatenated operands
   if (kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.fc, lcat, METIS_FP32, kc, s));
   if (ka) METIS_TRY(metis_launch_gemm_tc(ctx, b.res, a.fc, rcat + kb, METIS_FP32, kc, s));
@@ -143,7 +179,12 @@ metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void
   lowrank_finish_kernel<<<(unsigned)metis_ceil_div(mx, 8), 256, 0, s>>>(
       M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
       ka ? a.fo->tensor_scale : nullptr, a.sigma, kb ? b.fo->codes : nullptr, kb ? b.fo->scales : nullptr,
-      kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, pm, lcat, rcat); METIS_COUNT_LAUNCH();
+      kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, pm, lcat, rcat, lx, rx, kx,
+      a.res->tensor_scale, b.res->tensor_scale); METIS_COUNT_LAUNCH();
+  if (fuse) {
+    // residual x residual product and the rank-(ka+kb) correction accumulate into one FP32 tile in tensor memory
+    return metis_launch_gemm_tc_fused(ctx, a.res, b.res, d, d_dtype, ldd, lx, rx, kx, s);
+  }
   dim3 grid((unsigned)metis_ceil_div(N, 64), (unsigned)metis_ceil_div(M, 64));
   const size_t smem = sizeof(float) * 2 * kc * 68;
   static bool attr = false;
@@ -157,8 +198,11 @@ metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void
 
 size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k) {
   const int kc = 2 * k;
+  const int kx = (3 * kc + 63) / 64 * 64;
+  // sized for either path: FP32 staging of the main product (small shapes) or the BF16 correction operands
   return align256(sizeof(float) * M * N) + align256(sizeof(float) * 64 * 64) +
-         align256(sizeof(float) * M * (kc ? kc : 1)) + align256(sizeof(float) * N * (kc ? kc : 1));
+         align256(sizeof(float) * M * (kc ? kc : 1)) + align256(sizeof(float) * N * (kc ? kc : 1)) +
+         align256(sizeof(__nv_bfloat16) * M * (kx ? kx : 1)) + align256(sizeof(__nv_bfloat16) * N * (kx ? kx : 1));
 }
 
 metis_status_t metis_linear_fwd(metis_handle_t h, const metis_operand_t* x, const metis_operand_t* w, void* y,
