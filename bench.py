@@ -178,15 +178,31 @@ def main():
         wo0, w_res_dense = h.split(dev_sets[0]["w"], k, p, sketch=B.SKETCH_FULL, seed=2, want_residual=True)
         w_res_bf = w_res_dense.to(bf)
 
+    # The three operand decompositions are independent of each other, and the dY chain is independent of the
+    # forward product: they run on three streams and join by events (torch streams: plumbing only).
+    main = torch.cuda.current_stream()
+    side_w, side_d = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_start, ev_w, ev_d = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+    h_x, h_w, h_d = h, B.Handle(local_rank), B.Handle(local_rank)     # one workspace owner per stream
+
     def step(bufs, i):
-        h.split(bufs["x"], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 1, rounding=B.ROUND_RNE, out=xo)
-        if args.weights == "split":
-            h.split(bufs["w"], k, p, sketch=B.SKETCH_FULL, seed=3 * i + 2, rounding=B.ROUND_RNE, out=wo)
-        else:
-            h.requantize_weight(wo0, w_res_bf, out=wo)
-        h.linear_fwd(xo, wo, out=y)
-        h.split(bufs["dy"], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 3, rounding=B.ROUND_SR, out=do)
-        h.linear_bwd(do, xo, wo, out=(dx, dw))
+        ev_start.record(main)
+        side_w.wait_event(ev_start)
+        side_d.wait_event(ev_start)
+        with torch.cuda.stream(side_w):
+            if args.weights == "split":
+                h_w.split(bufs["w"], k, p, sketch=B.SKETCH_FULL, seed=3 * i + 2, rounding=B.ROUND_RNE, out=wo, stream=side_w)
+            else:
+                h_w.requantize_weight(wo0, w_res_bf, out=wo, stream=side_w)
+            ev_w.record(side_w)
+        with torch.cuda.stream(side_d):
+            h_d.split(bufs["dy"], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 3, rounding=B.ROUND_SR, out=do, stream=side_d)
+            ev_d.record(side_d)
+        h_x.split(bufs["x"], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 1, rounding=B.ROUND_RNE, out=xo)
+        main.wait_event(ev_w)
+        h_x.linear_fwd(xo, wo, out=y)
+        main.wait_event(ev_d)
+        h_x.linear_bwd(do, xo, wo, out=(dx, dw))
         if world > 1:
             dist.all_reduce(dw)
 
@@ -212,7 +228,7 @@ def main():
     barrier()
     ms = e0.elapsed_time(e1) / args.steps
     launches = B.launch_count() - launches0
-    status = h.device_status()
+    status = h.device_status() | h_w.device_status() | h_d.device_status()
 
     # ---- end to end: pinned host inputs in, results out, every step ---------------------------------
     stage = {key: torch.empty_like(v) for key, v in dev_sets[0].items()}

@@ -129,6 +129,19 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // Shared-memory matrix descriptor (sm_100 format): start address [0,14) in 16-byte units, leading byte
 // offset [16,30), stride byte offset [32,46), descriptor version 1 at [46,48), swizzle mode [61,64).
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t sbo_bytes, uint32_t swizzle_mode) {
@@ -167,7 +180,8 @@ __device__ __forceinline__ void store_row_chunk(const GemmArgs& g, int row, int 
         *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
                                                           __uint_as_float(r[j + 2]) * alpha, __uint_as_float(r[j + 3]) * alpha);
     } else {
-      for (int j = 0; j < 32 && col + j < g.N; ++j) dst[j] = __uint_as_float(r[j]) * alpha;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (col + j < g.N) dst[j] = __uint_as_float(r[j]) * alpha;
     }
   } else {
     __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(g.d) + (size_t)row * g.ldd + col;
@@ -184,7 +198,8 @@ __device__ __forceinline__ void store_row_chunk(const GemmArgs& g, int row, int 
         *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
       }
     } else {
-      for (int j = 0; j < 32 && col + j < g.N; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]) * alpha);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (col + j < g.N) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]) * alpha);
     }
   }
 }
@@ -357,7 +372,7 @@ constexpr int SF_COLS_PER_STAGE = 4 * K_STEPS * 3;          // 16 (A) + 32 (B): 
 constexpr int SF_COL0 = 256;
 constexpr int TMEM_COLS = 512;
 static_assert(ACC_COLS + STAGES * SF_COLS_PER_STAGE <= TMEM_COLS, "tensor memory budget");
-constexpr int NUM_THREADS = 256;                            // producer, MMA, relay, 4 epilogue warps, scale copier
+constexpr int NUM_THREADS = 384;                            // producer, MMA, relay, scale copier, 8 epilogue warps
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
 
 __device__ __forceinline__ uint32_t cluster_rank() {
@@ -466,7 +481,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); mbar_init(ready_bar(s), 2); mbar_init(sfready_bar(s), 1);
     }
     mbar_init(tfull_bar, 1);
-    mbar_init(tempty_bar, 8);                                 // 4 epilogue warps in each of the two CTAs
+    mbar_init(tempty_bar, 16);                                // 8 epilogue warps in each of the two CTAs
     *dead = 0;
     fence_barrier_init();
   }
@@ -565,7 +580,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         if (ok) tc_commit2(tfull_bar, 3);                     // accumulator complete in both CTAs
       }
     }
-  } else if (warp == 7) {
+  } else if (warp == 3) {
     // ------------------------------- scale copier (leader CTA only) ----------
     // shared memory -> tensor memory copies of the scale atoms, issued from their own warp so they do not sit
     // in the MMA issuer's instruction stream; a stage's columns are rewritten only after the MMAs that read them
@@ -591,9 +606,12 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         }
       }
     }
-  } else {
+  } else if (warp >= 4) {
     // ------------------------------- epilogue (both CTAs) --------------------
-    const int quarter = warp & 3;
+    // Eight warps: warp w drains TMEM lane quarter w % 4, column half (w - 4) / 4.  A thread pulls its 128
+    // accumulator columns into registers in one go and releases the accumulator at once, so the next tile's
+    // MMAs start while this tile is still being scaled, converted and stored.
+    const int quarter = warp & 3, half = (warp - 4) >> 2;
     const float alpha = (*g.a_ts) * (*g.b_ts);
     int it = 0;
     bool ok = true;
@@ -602,17 +620,25 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       if (!mbar_wait(tfull_bar, (uint32_t)it & 1u, g.dev_status, dead)) { ok = false; break; }
       tc_fence_after();
       const int row = mb * TILE_M + (int)rank * 128 + quarter * 32 + lane;
-      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
-#pragma unroll 1
-      for (int c0 = 0; c0 < TILE_N && !(g.dbg & 8); c0 += 32) {
-        uint32_t r[32];
-        tc_ld32(t_row + c0, r);
-        const int col = nb * TILE_N + c0;
-        if (row < g.M && col < g.N) store_row_chunk(g, row, col, r, alpha);
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 128);
+      uint32_t r[4][32];
+      if (!(g.dbg & 8)) {
+        tc_ld32_nowait(t_row, r[0]);
+        tc_ld32_nowait(t_row + 32, r[1]);
+        tc_ld32_nowait(t_row + 64, r[2]);
+        tc_ld32_nowait(t_row + 96, r[3]);
+        tc_wait_ld();
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_remote(tempty_bar, 0u);
+      if (!(g.dbg & 8)) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int col = nb * TILE_N + half * 128 + c * 32;
+          if (row < g.M && col < g.N) store_row_chunk(g, row, col, r[c], alpha);
+        }
+      }
     }
   }
 
