@@ -10,7 +10,7 @@
 namespace {
 
 constexpr int MAXQ = 64;
-constexpr size_t JACOBI_SMEM = sizeof(double) * 2 * MAXQ * (MAXQ + 1);
+constexpr size_t JACOBI_SMEM = sizeof(double) * MAXQ * (MAXQ + 1);
 
 // ------------------------------------------------------------------------------------------------
 __global__ void sample_rows_kernel(int* __restrict__ idx, int n_s, int64_t rows, uint64_t seed, int full) {
@@ -152,6 +152,8 @@ __device__ __forceinline__ double chol_rsqrt(double x) {
   return ldexp(y, -(e2 / 2));
 }
 
+__device__ __forceinline__ double fast_rsqrt_wide(double x) { return chol_rsqrt(x); }
+
 // One CholeskyQR pass, step 1 (one CTA): G (one Gram partial) = L L^T in FP64; writes L (q x q, row-major,
 // upper part unused) and the reciprocal pivots.  A pivot below 1e-13 of the largest diagonal marks a
 // dependent sketch column: its reciprocal is stored as zero, so the corresponding column of H = Z L^-T
@@ -273,12 +275,16 @@ project_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __r
 }
 
 // ------------------------------------------------------------------------------------------------
-// Symmetric eigen-decomposition (n <= 64) by parallel-order cyclic Jacobi in FP64, one CTA.
-// Each round pairs the indices into n/2 disjoint (p, q) couples (round-robin tournament); thread (I, J)
-// owns the 2 x 2 block (rows of couple I, columns of couple J), so one round is: rotation angles from
-// the diagonal blocks, then every thread applies J_I^T . block . J_J in registers - two barriers a round.
-// Input: Gram matrix (ld x ld, leading n x n block used).  Output: eigenvalues descending,
-// eigenvectors as columns of evecs[n][n].
+// Symmetric positive semi-definite eigen-decomposition (n <= 64) in FP64, one CTA.
+// G = L L^T (Cholesky, dependent columns zeroed), then one-sided (Hestenes) Jacobi on the columns of Y = L:
+// plane rotations make the columns mutually orthogonal, Y J1 J2 ... = U Sigma, so G = Y Y^T = U Sigma^2 U^T:
+// eigenvalues are the squared column norms and eigenvectors the normalised columns.  Working on the
+// Cholesky factor needs one matrix instead of two (no separate eigenvector accumulation), one barrier per
+// round, and converges in few sweeps.  Each round pairs the columns into n/2 disjoint couples (round-robin
+// tournament); a couple is handled by 8 threads that split the rows, reduce the three inner products with
+// shuffles and rotate their rows in registers.
+// Input: Gram matrix (ld x ld, leading n x n block used).  Output: eigenvalues descending, eigenvectors as
+// columns of evecs[n][n].
 __device__ __forceinline__ void jacobi_pair(int I, int step, int np, int* p, int* q) {
   int a, b;
   if (I == 0) { a = 0; b = (step % (np - 1)) + 1; }
@@ -294,94 +300,125 @@ __device__ __forceinline__ double fast_rsqrt(double x) {
   return y;
 }
 
-__global__ void __launch_bounds__(1024)
-jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, double* __restrict__ evals,
-                  double* __restrict__ evecs) {
+__global__ void __launch_bounds__(256)
+jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, double* __restrict__ evals, double* __restrict__ evecs) {
   extern __shared__ __align__(16) unsigned char jsm[];
-  double (*A)[MAXQ + 1] = reinterpret_cast<double (*)[MAXQ + 1]>(jsm);
-  double (*V)[MAXQ + 1] = reinterpret_cast<double (*)[MAXQ + 1]>(jsm + sizeof(double) * MAXQ * (MAXQ + 1));
-  __shared__ double cs[MAXQ / 2][2];
-  __shared__ double red[2][32];
+  double (*Y)[MAXQ + 1] = reinterpret_cast<double (*)[MAXQ + 1]>(jsm);
+  __shared__ double lam[MAXQ];
+  __shared__ double gmax_s;
   __shared__ int order[MAXQ];
+  __shared__ int rotated[2];
   __shared__ uint8_t pairs[MAXQ][MAXQ / 2][2];          // [round][couple] -> (p, q)
-  const int tid = threadIdx.x, nthr = blockDim.x;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const int np = n + (n & 1), half = np / 2;
-  for (int o = tid; o < np * np; o += nthr) {
+  for (int o = tid; o < np * np; o += 256) {
     const int i = o / np, j = o % np;
-    A[i][j] = (i < n && j < n) ? 0.5 * (g[i * ld + j] + g[j * ld + i]) : 0.0;
-    V[i][j] = (i == j) ? 1.0 : 0.0;
+    Y[i][j] = (i < n && j < n) ? 0.5 * (g[i * ld + j] + g[j * ld + i]) : 0.0;
   }
-  for (int o = tid; o < (np - 1) * half; o += nthr) {
+  for (int o = tid; o < (np - 1) * half; o += 256) {
     int p, q;
     jacobi_pair(o % half, o / half, np, &p, &q);
     pairs[o / half][o % half][0] = (uint8_t)p; pairs[o / half][o % half][1] = (uint8_t)q;
   }
+  if (tid == 0) { rotated[0] = 0; rotated[1] = 0; }
   __syncthreads();
-  const bool active = tid < half * half;
-  const int I = active ? tid / half : 0, J = active ? tid % half : 0;
-  for (int sweep = 0; sweep < 12; ++sweep) {
-    // convergence: off-diagonal energy against diagonal energy
-    double off = 0.0, dg = 0.0;
-    for (int o = tid; o < np * np; o += nthr) {
-      const int i = o / np, j = o % np;
-      const double v = A[i][j] * A[i][j];
-      if (i == j) dg += v; else off += v;
-    }
+  // ---- Cholesky, lower factor in place; the strict upper triangle is cleared afterwards ----
+  if (tid < 32) {
+    double gm = 0.0;
+    for (int i = tid; i < n; i += 32) gm = fmax(gm, Y[i][i]);
 #pragma unroll
-    for (int sft = 16; sft > 0; sft >>= 1) { off += __shfl_xor_sync(0xFFFFFFFFu, off, sft); dg += __shfl_xor_sync(0xFFFFFFFFu, dg, sft); }
-    if ((tid & 31) == 0) { red[0][tid >> 5] = off; red[1][tid >> 5] = dg; }
+    for (int o = 16; o > 0; o >>= 1) gm = fmax(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, o));
+    if (tid == 0) gmax_s = gm;
+  }
+  __syncthreads();
+  const double tol = 1e-14 * gmax_s;
+  for (int j = 0; j < n; ++j) {
+    const double d = Y[j][j];
+    const bool dep = !(d > tol);
+    const double inv = dep ? 0.0 : chol_rsqrt(d);
     __syncthreads();
-    off = 0.0; dg = 0.0;
-    for (int w = 0; w < (nthr >> 5); ++w) { off += red[0][w]; dg += red[1][w]; }
+    for (int i = j + 1 + tid; i < n; i += 256) Y[i][j] *= inv;
+    if (tid == 0) Y[j][j] = dep ? 0.0 : d * inv;
     __syncthreads();
-    if (off <= 1e-22 * dg) break;
-    for (int step = 0; step < np - 1; ++step) {
-      const int pi = pairs[step][I][0], qi = pairs[step][I][1], pj = pairs[step][J][0], qj = pairs[step][J][1];
-      if (active && I == J) {
-        // rotation angle: the tangent only needs FP32 accuracy (it steers convergence); cos/sin are then made
-        // orthonormal to FP64 accuracy, so the accumulated eigenvector matrix stays orthogonal
-        const double apq = A[pi][qi];
-        double c = 1.0, s = 0.0;
-        if (fabs(apq) > 1e-300) {
-          const float theta = (float)(A[qi][qi] - A[pi][pi]) / (2.0f * (float)apq);
-          const float tf = copysignf(1.0f, theta) / (fabsf(theta) + sqrtf(fmaf(theta, theta, 1.0f)));
-          const double t = (double)tf;
-          c = fast_rsqrt(t * t + 1.0);
-          s = t * c;
-        }
-        cs[I][0] = c; cs[I][1] = s;
+    if (!dep) {
+      for (int a = j + 1 + ty; a < n; a += 16) {
+        const double laj = Y[a][j];
+        for (int b = j + 1 + tx; b <= a; b += 16) Y[a][b] -= laj * Y[b][j];
       }
-      __syncthreads();
-      if (active) {
-        const double ci = cs[I][0], si = cs[I][1], cj = cs[J][0], sj = cs[J][1];
-        // block rows (pi, qi), columns (pj, qj):  B <- Ji^T B Jj,  J = [[c, s], [-s, c]]
-        const double b00 = A[pi][pj], b01 = A[pi][qj], b10 = A[qi][pj], b11 = A[qi][qj];
-        const double r00 = ci * b00 - si * b10, r01 = ci * b01 - si * b11;
-        const double r10 = si * b00 + ci * b10, r11 = si * b01 + ci * b11;
-        A[pi][pj] = cj * r00 - sj * r01; A[pi][qj] = sj * r00 + cj * r01;
-        A[qi][pj] = cj * r10 - sj * r11; A[qi][qj] = sj * r10 + cj * r11;
-        // eigenvector accumulation: rows 2I, 2I+1 (fixed), columns (pj, qj):  V <- V Jj
-        const int r0 = 2 * I, r1 = 2 * I + 1;
-        const double v00 = V[r0][pj], v01 = V[r0][qj], v10 = V[r1][pj], v11 = V[r1][qj];
-        V[r0][pj] = cj * v00 - sj * v01; V[r0][qj] = sj * v00 + cj * v01;
-        V[r1][pj] = cj * v10 - sj * v11; V[r1][qj] = sj * v10 + cj * v11;
+    }
+    __syncthreads();
+  }
+  for (int o = tid; o < np * np; o += 256) {
+    const int i = o / np, j = o % np;
+    if (j > i) Y[i][j] = 0.0;
+  }
+  __syncthreads();
+  // ---- one-sided Jacobi on the columns of Y ----
+  const int m = tid >> 3, sub = tid & 7;                // couple index, row slice
+  const bool active = m < half;
+  for (int sweep = 0; sweep < 16; ++sweep) {
+    for (int step = 0; step < np - 1; ++step) {
+      {
+        // every lane takes part in the shuffles; lanes of couples beyond n/2 carry zeros and write nothing
+        const int p = active ? pairs[step][m][0] : 0, q = active ? pairs[step][m][1] : 0;
+        double yp[MAXQ / 8], yq[MAXQ / 8];
+        double a = 0.0, b = 0.0, c = 0.0;
+#pragma unroll
+        for (int t = 0; t < MAXQ / 8; ++t) {
+          const int i = sub + 8 * t;
+          yp[t] = (active && i < np) ? Y[i][p] : 0.0;
+          yq[t] = (active && i < np) ? Y[i][q] : 0.0;
+          a += yp[t] * yp[t]; b += yq[t] * yq[t]; c += yp[t] * yq[t];
+        }
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) {
+          a += __shfl_xor_sync(0xFFFFFFFFu, a, o); b += __shfl_xor_sync(0xFFFFFFFFu, b, o); c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+        }
+        // rotate only if the two columns are not yet orthogonal to working precision
+        if (active && c * c > 1e-26 * a * b) {
+          float zeta = (float)(b - a) / (2.0f * (float)c);
+          if (!(fabsf(zeta) < 1e18f)) zeta = copysignf(1e18f, zeta);      // huge or not finite: (almost) no rotation
+          const float tf = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
+          const double t = (double)tf;
+          const double cs = fast_rsqrt(t * t + 1.0), sn = t * cs;
+#pragma unroll
+          for (int tt = 0; tt < MAXQ / 8; ++tt) {
+            const int i = sub + 8 * tt;
+            if (i < np) {
+              Y[i][p] = cs * yp[tt] - sn * yq[tt];
+              Y[i][q] = sn * yp[tt] + cs * yq[tt];
+            }
+          }
+          if (sub == 0) rotated[sweep & 1] = 1;
+        }
       }
       __syncthreads();
     }
+    const int any = rotated[sweep & 1];
+    if (tid == 0) rotated[(sweep + 1) & 1] = 0;
+    __syncthreads();
+    if (!any) break;
+  }
+  // ---- eigenvalues = squared column norms, eigenvectors = normalised columns ----
+  if (tid < n) {
+    double a = 0.0;
+    for (int i = 0; i < n; ++i) a += Y[i][tid] * Y[i][tid];
+    lam[tid] = a;
   }
   __syncthreads();
   if (tid < n) {
-    const double li = A[tid][tid];
+    const double li = lam[tid];
     int rank = 0;
-    for (int j = 0; j < n; ++j) {
-      const double lj = A[j][j];
-      rank += (lj > li) || (lj == li && j < tid);
-    }
+    for (int j = 0; j < n; ++j) rank += (lam[j] > li) || (lam[j] == li && j < tid);
     order[rank] = tid;
   }
   __syncthreads();
-  if (tid < n) evals[tid] = A[order[tid]][order[tid]];
-  for (int o = tid; o < n * n; o += nthr) evecs[o] = V[o / n][order[o % n]];
+  if (tid < n) evals[tid] = lam[order[tid]];
+  for (int o = tid; o < n * n; o += 256) {
+    const int i = o / n, j = order[o % n];
+    const double l2 = lam[j];
+    evecs[o] = l2 > 0.0 ? Y[i][j] * fast_rsqrt_wide(l2) : 0.0;
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -971,7 +1008,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     int64_t rpp; const int parts = gram_parts(cols, &rpp);
     gram_kernel<<<parts, 256, 0, s>>>(m, cols, q, 1, cols, rpp, gram); METIS_COUNT_LAUNCH();
     reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1); METIS_COUNT_LAUNCH();
-    jacobi_eig_kernel<<<1, jacobi_threads(q), JACOBI_SMEM, s>>>(gram1, q, q, evals, evecs); METIS_COUNT_LAUNCH();
+    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram1, q, q, evals, evecs); METIS_COUNT_LAUNCH();
   }
   right_basis_kernel<<<(unsigned)metis_ceil_div(cols, 64), 64, 0, s>>>(m, cols, q, k, evals, evecs, basis,
                                                                           full ? out->sigma : nullptr); METIS_COUNT_LAUNCH();
@@ -1016,7 +1053,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   if (!full) {
     // (7) Rayleigh-Ritz on C^T C (Gram partials came out of the broadcast pass), rotate both factors
     reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 128), 128, 0, s>>>(gram_c, n_cta_c, kp * kp, gram1); METIS_COUNT_LAUNCH();
-    jacobi_eig_kernel<<<1, jacobi_threads(k), JACOBI_SMEM, s>>>(gram1, k, kp, evals2, evecs2); METIS_COUNT_LAUNCH();
+    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram1, k, kp, evals2, evecs2); METIS_COUNT_LAUNCH();
     right_rotate_kernel<<<n_cand, 256, 0, s>>>(basis, cols, k, evecs2, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
     sign_fix_kernel<<<dim3(n_cand, k), 256, 0, s>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign); METIS_COUNT_LAUNCH();
     left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 64, 0, s>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
