@@ -15,9 +15,12 @@
  * General rules
  *  - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns every
  *    buffer (inputs, outputs, workspace); the library allocates device memory only inside
- *    metis_create (a 128 KiB quantile table and a status word) and frees it in metis_destroy.
+ *    metis_create (a 128 KiB quantile table and a status word; it also creates three streams and four
+ *    events there) and frees it in metis_destroy.
  *  - All work is enqueued on the caller's stream (a cudaStream_t passed as void*); calls return
- *    without synchronising.  Host-detectable errors (null or misaligned pointer, unsupported shape,
+ *    without synchronising.  Inside a call, independent sub-chains may run on streams the handle owns;
+ *    they start after the work already on the caller's stream and are joined back into it before the
+ *    call returns, so the caller sees ordinary stream order.  One handle serves one stream at a time.  Host-detectable errors (null or misaligned pointer, unsupported shape,
  *    workspace too small) are returned at once and nothing is enqueued.  Device-detected conditions
  *    (a bounded wait that expired, a Cholesky breakdown) are OR-ed into the handle's device status
  *    word, read with metis_last_device_status after the caller has synchronised the stream.

@@ -59,6 +59,15 @@ metis_status_t metis_create(metis_handle_t* out, int device) {
   if (e == cudaSuccess) e = cudaMemcpy(ctx->quantile_lut, host, 65536 * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, 256);
   free(host);
+  int prio_least = 0, prio_greatest = 0;
+  if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest);
+  for (int i = 0; i < 3 && e == cudaSuccess; ++i) {
+    // highest priority: the side streams carry the short latency-critical chains, which must not queue up
+    // behind the thousands of blocks of a big pass running on the caller's stream
+    e = cudaStreamCreateWithPriority(&ctx->side[i], cudaStreamNonBlocking, prio_greatest);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join[i], cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
   if (e != cudaSuccess) {
     cudaFree(ctx->quantile_lut); cudaFree(ctx->dev_status); free(ctx);
     return METIS_ERR_CUDA;
@@ -69,6 +78,11 @@ metis_status_t metis_create(metis_handle_t* out, int device) {
 
 metis_status_t metis_destroy(metis_handle_t h) {
   if (!h) return METIS_OK;
+  for (int i = 0; i < 3; ++i) {
+    if (h->side[i]) { cudaStreamSynchronize(h->side[i]); cudaStreamDestroy(h->side[i]); }
+    if (h->ev_join[i]) cudaEventDestroy(h->ev_join[i]);
+  }
+  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
   cudaFree(h->quantile_lut);
   cudaFree(h->dev_status);
   free(h);

@@ -12,7 +12,25 @@ struct metis_context {
   __nv_bfloat16* quantile_lut;   // 65536 bf16 standard-normal quantiles (Section 3.1 Gaussian test matrix)
   uint32_t* dev_status;          // device status word (METIS_DEV_* bits)
   void* encode_tiled;            // cuTensorMapEncodeTiled entry point, resolved at create
+  // Internal fork/join: independent sub-chains of one call run on these side streams and are joined back into
+  // the caller's stream with events before the call's last kernels (everything stays asynchronous).
+  cudaStream_t side[3];
+  cudaEvent_t ev_fork, ev_join[3];
 };
+
+// fork: side stream i starts after everything enqueued so far on `main`
+static inline metis_status_t metis_fork(metis_context* ctx, cudaStream_t main, int n_side) {
+  if (cudaEventRecord(ctx->ev_fork, main) != cudaSuccess) return METIS_ERR_CUDA;
+  for (int i = 0; i < n_side; ++i)
+    if (cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0) != cudaSuccess) return METIS_ERR_CUDA;
+  return METIS_OK;
+}
+// join: `main` continues after everything enqueued so far on side stream i
+static inline metis_status_t metis_join(metis_context* ctx, cudaStream_t main, int i) {
+  if (cudaEventRecord(ctx->ev_join[i], ctx->side[i]) != cudaSuccess) return METIS_ERR_CUDA;
+  if (cudaStreamWaitEvent(main, ctx->ev_join[i], 0) != cudaSuccess) return METIS_ERR_CUDA;
+  return METIS_OK;
+}
 
 #define METIS_CUDA_TRY(expr)                         \
   do {                                               \

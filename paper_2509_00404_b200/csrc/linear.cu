@@ -171,10 +171,14 @@ metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void
   if (!ws || off > ws_bytes) return METIS_ERR_WORKSPACE;
 
   if (!fuse) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.res, y0, METIS_FP32, N, s));
-  // the skinny products land directly in their slots of the concatenated operands
+  // the skinny products land directly in their slots of the concatenated operands; they are independent of
+  // each other and run side by side
+  METIS_TRY(metis_fork(ctx, s, 2));
   if (kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.fc, lcat, METIS_FP32, kc, s));
-  if (ka) METIS_TRY(metis_launch_gemm_tc(ctx, b.res, a.fc, rcat + kb, METIS_FP32, kc, s));
-  if (ka && kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.fc, b.fc, pm, METIS_FP32, kb, s));
+  if (ka) METIS_TRY(metis_launch_gemm_tc(ctx, b.res, a.fc, rcat + kb, METIS_FP32, kc, ctx->side[0]));
+  if (ka && kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.fc, b.fc, pm, METIS_FP32, kb, ctx->side[1]));
+  METIS_TRY(metis_join(ctx, s, 0));
+  METIS_TRY(metis_join(ctx, s, 1));
   const int64_t mx = M > N ? M : N;
   lowrank_finish_kernel<<<(unsigned)metis_ceil_div(mx, 8), 256, 0, s>>>(
       M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,

@@ -354,26 +354,36 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, double* __restric
   }
   __syncthreads();
   // ---- one-sided Jacobi on the columns of Y ----
+  // Column norms are carried along (alpha' = alpha - t*gamma, beta' = beta + t*gamma) and recomputed exactly at
+  // the start of every sweep, so a round needs a single inner product per couple.  A sweep whose largest
+  // |cos| between paired columns was below 1e-7 is the last one: convergence is quadratic, its rotations
+  // leave the columns orthogonal to ~1e-14.
   const int m = tid >> 3, sub = tid & 7;                // couple index, row slice
   const bool active = m < half;
   for (int sweep = 0; sweep < 16; ++sweep) {
+    if (tid < np) {
+      double a = 0.0;
+      for (int i = 0; i < np; ++i) a += Y[i][tid] * Y[i][tid];
+      lam[tid] = a;
+    }
+    if (tid == 0) rotated[0] = 0;                       // reused as the sweep's max cos^2 (float bits)
+    __syncthreads();
     for (int step = 0; step < np - 1; ++step) {
       {
         // every lane takes part in the shuffles; lanes of couples beyond n/2 carry zeros and write nothing
         const int p = active ? pairs[step][m][0] : 0, q = active ? pairs[step][m][1] : 0;
         double yp[MAXQ / 8], yq[MAXQ / 8];
-        double a = 0.0, b = 0.0, c = 0.0;
+        double c = 0.0;
 #pragma unroll
         for (int t = 0; t < MAXQ / 8; ++t) {
           const int i = sub + 8 * t;
           yp[t] = (active && i < np) ? Y[i][p] : 0.0;
           yq[t] = (active && i < np) ? Y[i][q] : 0.0;
-          a += yp[t] * yp[t]; b += yq[t] * yq[t]; c += yp[t] * yq[t];
+          c += yp[t] * yq[t];
         }
 #pragma unroll
-        for (int o = 4; o > 0; o >>= 1) {
-          a += __shfl_xor_sync(0xFFFFFFFFu, a, o); b += __shfl_xor_sync(0xFFFFFFFFu, b, o); c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
-        }
+        for (int o = 4; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+        const double a = lam[p], b = lam[q];
         // rotate only if the two columns are not yet orthogonal to working precision
         if (active && c * c > 1e-26 * a * b) {
           float zeta = (float)(b - a) / (2.0f * (float)c);
@@ -389,15 +399,20 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, double* __restric
               Y[i][q] = sn * yp[tt] + cs * yq[tt];
             }
           }
-          if (sub == 0) rotated[sweep & 1] = 1;
+          if (sub == 0) {
+            // exact for the applied (cs, sn): |y_p'|^2 = cs^2 a - 2 cs sn c + sn^2 b, |y_q'|^2 = sn^2 a + 2 cs sn c + cs^2 b
+            lam[p] = cs * cs * a - 2.0 * cs * sn * c + sn * sn * b;
+            lam[q] = sn * sn * a + 2.0 * cs * sn * c + cs * cs * b;
+            const float cf = (float)c, cos2 = (cf / (float)a) * (cf / (float)b);
+            atomicMax(reinterpret_cast<unsigned int*>(&rotated[0]), __float_as_uint(fminf(cos2, 1.0f)));
+          }
         }
       }
       __syncthreads();
     }
-    const int any = rotated[sweep & 1];
-    if (tid == 0) rotated[(sweep + 1) & 1] = 0;
+    const float maxcos2 = __uint_as_float((unsigned int)rotated[0]);
     __syncthreads();
-    if (!any) break;
+    if (maxcos2 < 1e-14f) break;
   }
   // ---- eigenvalues = squared column norms, eigenvectors = normalised columns ----
   if (tid < n) {
@@ -1042,32 +1057,37 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     const size_t smem = smem_bytes(rounding == METIS_ROUND_SR);
     dim3 grid((unsigned)metis_ceil_div(cols, TILE), (unsigned)metis_ceil_div(rows, TILE));
     float* t0 = want_c ? rc.tensor_scale : nullptr; float* t1 = want_r ? rr.tensor_scale : nullptr;
+    // the big residual pass and the small factor chain below are independent from here on: the factor chain
+    // goes to a (high-priority) side stream and is joined back at the end of the call
+    METIS_TRY(metis_fork(ctx, s, 1));
+    cudaStream_t sr = s;
     switch (kp) {
-      case 16: residual_quant_kernel<16><<<grid, THREADS, smem, s>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
-      case 32: residual_quant_kernel<32><<<grid, THREADS, smem, s>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
-      case 48: residual_quant_kernel<48><<<grid, THREADS, smem, s>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
-      default: residual_quant_kernel<64><<<grid, THREADS, smem, s>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+      case 16: residual_quant_kernel<16><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+      case 32: residual_quant_kernel<32><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+      case 48: residual_quant_kernel<48><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+      default: residual_quant_kernel<64><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
     }
     METIS_COUNT_LAUNCH();
   }
+  cudaStream_t sf = ctx->side[0];
   if (!full) {
     // (7) Rayleigh-Ritz on C^T C (Gram partials came out of the broadcast pass), rotate both factors
-    reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 128), 128, 0, s>>>(gram_c, n_cta_c, kp * kp, gram1); METIS_COUNT_LAUNCH();
-    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram1, k, kp, evals2, evecs2); METIS_COUNT_LAUNCH();
-    right_rotate_kernel<<<n_cand, 256, 0, s>>>(basis, cols, k, evecs2, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
-    sign_fix_kernel<<<dim3(n_cand, k), 256, 0, s>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign); METIS_COUNT_LAUNCH();
-    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 64, 0, s>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
+    reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 128), 128, 0, sf>>>(gram_c, n_cta_c, kp * kp, gram1); METIS_COUNT_LAUNCH();
+    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, sf>>>(gram1, k, kp, evals2, evecs2); METIS_COUNT_LAUNCH();
+    right_rotate_kernel<<<n_cand, 256, 0, sf>>>(basis, cols, k, evecs2, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
+    sign_fix_kernel<<<dim3(n_cand, k), 256, 0, sf>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign); METIS_COUNT_LAUNCH();
+    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 64, 0, sf>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
                                                                            out->left, out->sigma, nullptr, 0, nullptr); METIS_COUNT_LAUNCH();
   }
   METIS_CUDA_TRY(cudaGetLastError());
   // (8) quantize the factors (stored transposed: k x rows, k x cols; blocks along the long dimension)
   metis_nvfp4_t lq = out->left_q, rq = out->right_q;
   lq.rows = k; lq.k_len = rows; rq.rows = k; rq.k_len = cols;
-  METIS_TRY(metis_launch_amax(out->left, METIS_FP32, k, rows, rows, amax + 1, s));
+  METIS_TRY(metis_launch_amax(out->left, METIS_FP32, k, rows, rows, amax + 1, sf));
   METIS_TRY(metis_launch_quantize(out->left, METIS_FP32, k, rows, rows, rounding, seed, METIS_STREAM_LEFT, rows, 1,
-                                  amax + 1, 1, &lq, nullptr, s));
-  METIS_TRY(metis_launch_amax(out->right, METIS_FP32, k, cols, cols, amax + 2, s));
+                                  amax + 1, 1, &lq, nullptr, sf));
+  METIS_TRY(metis_launch_amax(out->right, METIS_FP32, k, cols, cols, amax + 2, sf));
   METIS_TRY(metis_launch_quantize(out->right, METIS_FP32, k, cols, cols, rounding, seed, METIS_STREAM_RIGHT, cols, 1,
-                                  amax + 2, 1, &rq, nullptr, s));
-  return METIS_OK;
+                                  amax + 2, 1, &rq, nullptr, sf));
+  return metis_join(ctx, s, 0);
 }
