@@ -23,73 +23,6 @@ __global__ void sample_rows_kernel(int* __restrict__ idx, int n_s, int64_t rows,
 }
 
 // ------------------------------------------------------------------------------------------------
-// Sketch partials: Zp[chunk][row][j] = sum over the chunk's 256 columns of x[idx[row], col] * Omega[col, j].
-// One CTA: 64 sampled rows x 256 columns; Omega's 256 x q slice is generated once per CTA into shared memory.
-constexpr int SK_ROWS = 64, SK_COLS = 256, SK_PITCH = SK_COLS + 4;
-__global__ void __launch_bounds__(256)
-sketch_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
-              uint64_t seed, const __nv_bfloat16* __restrict__ lut, float* __restrict__ zp) {
-  extern __shared__ __align__(16) unsigned char smem[];
-  float* om = reinterpret_cast<float*>(smem);                  // [SK_COLS][q]
-  float* xs = om + SK_COLS * MAXQ;                             // [SK_ROWS][SK_PITCH]
-  const int tid = threadIdx.x;
-  const int64_t col0 = (int64_t)blockIdx.y * SK_COLS;
-  const int row0 = blockIdx.x * SK_ROWS;
-  const int ncols = (int)min((int64_t)SK_COLS, cols - col0);
-  // Omega rows col0 .. col0+ncols: logical indices e = col*q + j form one contiguous range
-  const uint64_t e_lo = (uint64_t)col0 * q, e_hi = (uint64_t)(col0 + ncols) * q;
-  for (uint64_t blk = (e_lo >> 3) + tid; blk <= ((e_hi - 1) >> 3); blk += 256) {
-    const uint4 w = metis_philox_block(blk, seed, METIS_STREAM_OMEGA);
-#pragma unroll
-    for (uint32_t h = 0; h < 8; ++h) {
-      const uint64_t e = (blk << 3) + h;
-      if (e >= e_lo && e < e_hi) om[e - e_lo] = __bfloat162float(lut[metis_u16_of(w, h)]);
-    }
-  }
-  for (int i = tid; i < SK_ROWS * (SK_COLS / 8); i += 256) {
-    const int r = i >> 5, g = i & 31;
-    float v[8];
-    if (row0 + r < n_s && g * 8 + 8 <= ncols) {
-      const uint4 qv = *reinterpret_cast<const uint4*>(x + (int64_t)idx[row0 + r] * cols + col0 + g * 8);
-      const uint32_t w[4] = {qv.x, qv.y, qv.z, qv.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) { v[2 * j] = __uint_as_float(w[j] << 16); v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u); }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        v[j] = (row0 + r < n_s && g * 8 + j < ncols) ? __bfloat162float(x[(int64_t)idx[row0 + r] * cols + col0 + g * 8 + j]) : 0.0f;
-    }
-    *reinterpret_cast<float4*>(xs + r * SK_PITCH + g * 8) = make_float4(v[0], v[1], v[2], v[3]);
-    *reinterpret_cast<float4*>(xs + r * SK_PITCH + g * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
-  }
-  __syncthreads();
-  // thread -> rows tr*4 .. +3, sketch columns tj, tj+16, tj+32, tj+48
-  const int tr = tid >> 4, tj = tid & 15;
-  float acc[4][4];
-#pragma unroll
-  for (int a = 0; a < 4; ++a)
-#pragma unroll
-    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0f;
-  for (int t = 0; t < ncols; ++t) {
-    float xv[4], ov[4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a) xv[a] = xs[(tr * 4 + a) * SK_PITCH + t];
-#pragma unroll
-    for (int b = 0; b < 4; ++b) ov[b] = (tj + 16 * b < q) ? om[t * q + tj + 16 * b] : 0.0f;
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-      for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(xv[a], ov[b], acc[a][b]);
-  }
-#pragma unroll
-  for (int a = 0; a < 4; ++a)
-#pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int r = row0 + tr * 4 + a, j = tj + 16 * b;
-      if (r < n_s && j < q) zp[((int64_t)blockIdx.y * n_s + r) * q + j] = acc[a][b];
-    }
-}
-
 __global__ void reduce_partials_kernel(const float* __restrict__ zp, int n_chunks, int64_t n, float* __restrict__ z) {
   const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   if (i >= n) return;
@@ -711,8 +644,174 @@ residual_quant_kernel(const __nv_bfloat16* __restrict__ x, const float* __restri
 }
 
 // ------------------------------------------------------------------------------------------------
+// ------------------------------------------------------------------------------------------------
+// Tensor-core sketch: Zp[chunk][row][j] = sum over the chunk's 256 columns of x[idx[row], col] * Omega[col, j].
+// One CTA = 256 sampled rows x 256 columns; Omega's slice is generated once per CTA (Philox + quantile
+// table) straight into shared memory, transposed to [j][col] BF16 (its values are BF16 by construction, so
+// the products are exact and only the FP32 accumulation rounds).  Optionally also reduces amax|x| over the
+// rows it reads (FULL mode reads every row exactly once per column chunk).
+constexpr int SKM_ROWS = 256, SKM_COLS = 256, SKM_PITCH = SKM_COLS + 8;
+template <int NT>                                      // sketch columns / 8, rounded up
+__global__ void __launch_bounds__(256)
+sketch_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
+                  uint64_t seed, const __nv_bfloat16* __restrict__ lut, float* __restrict__ zp, float* __restrict__ amax_out) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  __nv_bfloat16* om = reinterpret_cast<__nv_bfloat16*>(smem);          // [NT*8][SKM_PITCH]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int64_t col0 = (int64_t)blockIdx.y * SKM_COLS;
+  const int row0 = blockIdx.x * SKM_ROWS + warp * 32;
+  const int ncols = (int)min((int64_t)SKM_COLS, cols - col0);
+  for (int i = tid; i < NT * 8 * SKM_PITCH; i += 256) om[i] = __float2bfloat16_rn(0.0f);
+  __syncthreads();
+  const uint64_t e_lo = (uint64_t)col0 * q, e_hi = (uint64_t)(col0 + ncols) * q;
+  for (uint64_t blk = (e_lo >> 3) + tid; blk <= ((e_hi - 1) >> 3); blk += 256) {
+    const uint4 w = metis_philox_block(blk, seed, METIS_STREAM_OMEGA);
+#pragma unroll
+    for (uint32_t h = 0; h < 8; ++h) {
+      const uint64_t e = (blk << 3) + h;
+      if (e >= e_lo && e < e_hi) {
+        const uint32_t rel = (uint32_t)(e - e_lo);
+        om[(rel % q) * SKM_PITCH + rel / q] = lut[metis_u16_of(w, h)];
+      }
+    }
+  }
+  __syncthreads();
+  float acc[2][NT][4];
+#pragma unroll
+  for (int m = 0; m < 2; ++m)
+#pragma unroll
+    for (int n = 0; n < NT; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[m][n][e] = 0.0f;
+  const bool v0 = row0 + g < n_s, v1 = row0 + g + 8 < n_s, v2 = row0 + g + 16 < n_s, v3 = row0 + g + 24 < n_s;
+  const __nv_bfloat16* p0 = x + (int64_t)(v0 ? idx[row0 + g] : 0) * cols + col0;
+  const __nv_bfloat16* p1 = x + (int64_t)(v1 ? idx[row0 + g + 8] : 0) * cols + col0;
+  const __nv_bfloat16* p2 = x + (int64_t)(v2 ? idx[row0 + g + 16] : 0) * cols + col0;
+  const __nv_bfloat16* p3 = x + (int64_t)(v3 ? idx[row0 + g + 24] : 0) * cols + col0;
+  uint32_t amax2 = 0u;
+#pragma unroll 2
+  for (int ks = 0; ks < ncols / 16; ++ks) {
+    const int kk = ks * 16 + 2 * t;
+    uint32_t a[2][4];
+    a[0][0] = v0 ? *reinterpret_cast<const uint32_t*>(p0 + kk) : 0u;
+    a[0][1] = v1 ? *reinterpret_cast<const uint32_t*>(p1 + kk) : 0u;
+    a[0][2] = v0 ? *reinterpret_cast<const uint32_t*>(p0 + kk + 8) : 0u;
+    a[0][3] = v1 ? *reinterpret_cast<const uint32_t*>(p1 + kk + 8) : 0u;
+    a[1][0] = v2 ? *reinterpret_cast<const uint32_t*>(p2 + kk) : 0u;
+    a[1][1] = v3 ? *reinterpret_cast<const uint32_t*>(p3 + kk) : 0u;
+    a[1][2] = v2 ? *reinterpret_cast<const uint32_t*>(p2 + kk + 8) : 0u;
+    a[1][3] = v3 ? *reinterpret_cast<const uint32_t*>(p3 + kk + 8) : 0u;
+    if (amax_out) {
+#pragma unroll
+      for (int m = 0; m < 2; ++m)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t ab = a[m][e] & 0x7FFF7FFFu;
+          amax2 = max(ab & 0xFFFFu, amax2 & 0xFFFFu) | (max(ab >> 16, amax2 >> 16) << 16);
+        }
+    }
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      const __nv_bfloat16* bp = om + (n * 8 + g) * SKM_PITCH + kk;
+      const uint32_t b0 = *reinterpret_cast<const uint32_t*>(bp), b1 = *reinterpret_cast<const uint32_t*>(bp + 8);
+      mma_bf16(acc[0][n], a[0], b0, b1);
+      mma_bf16(acc[1][n], a[1], b0, b1);
+    }
+  }
+  float* dst = zp + (int64_t)blockIdx.y * n_s * q;
+#pragma unroll
+  for (int m = 0; m < 2; ++m)
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      const int r = row0 + m * 16 + g, j = n * 8 + 2 * t;
+      if (r < n_s) { if (j < q) dst[(int64_t)r * q + j] = acc[m][n][0]; if (j + 1 < q) dst[(int64_t)r * q + j + 1] = acc[m][n][1]; }
+      if (r + 8 < n_s) { if (j < q) dst[(int64_t)(r + 8) * q + j] = acc[m][n][2]; if (j + 1 < q) dst[(int64_t)(r + 8) * q + j + 1] = acc[m][n][3]; }
+    }
+  if (amax_out) {
+    float am = fmaxf(__uint_as_float((amax2 & 0xFFFFu) << 16), __uint_as_float(amax2 & 0xFFFF0000u));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+    if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(amax_out), __float_as_uint(am));
+  }
+}
+
+// Tensor-core projection: Mp[part][j][col] = sum over the part's sampled rows r of H[r][j] * x[idx[r], col].
+// The contraction runs over rows of the row-major x, so x tiles are staged in shared memory and read back
+// transposed with ldmatrix; H (FP32) is fed as three BF16 terms.  CTA = 128 columns x one slab of rows.
+constexpr int PM_COLS = 128, PM_ROWS = 32, PM_XP = PM_COLS + 8, PM_HP = PM_ROWS + 8;
+template <int MT>                                      // sketch columns / 16, rounded up
+__global__ void __launch_bounds__(256)
+project_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
+                   const float* __restrict__ h, int rows_per_part, float* __restrict__ mp) {
+  __shared__ __align__(16) __nv_bfloat16 xs[PM_ROWS][PM_XP];
+  __shared__ __align__(16) __nv_bfloat16 hs[3][MT * 16][PM_HP];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int64_t col0 = (int64_t)blockIdx.x * PM_COLS;
+  const int r_begin = blockIdx.y * rows_per_part, r_end = min(n_s, r_begin + rows_per_part);
+  float acc[MT][2][4];
+#pragma unroll
+  for (int m = 0; m < MT; ++m)
+#pragma unroll
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[m][n][e] = 0.0f;
+  for (int r0 = r_begin; r0 < r_end; r0 += PM_ROWS) {
+    // stage 32 rows x 128 columns of x (16 bytes per thread-step) and the matching rows of H, split and transposed
+    for (int i = tid; i < PM_ROWS * (PM_COLS / 8); i += 256) {
+      const int rr = i >> 4, c8 = (i & 15) * 8;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (r0 + rr < r_end && col0 + c8 + 8 <= cols) v = *reinterpret_cast<const uint4*>(x + (int64_t)idx[r0 + rr] * cols + col0 + c8);
+      *reinterpret_cast<uint4*>(&xs[rr][c8]) = v;
+    }
+    for (int i = tid; i < PM_ROWS * MT * 16; i += 256) {
+      const int rr = i / (MT * 16), j = i % (MT * 16);
+      const float v = (r0 + rr < r_end && j < q) ? h[(int64_t)(r0 + rr) * q + j] : 0.0f;
+      const __nv_bfloat16 hh = __float2bfloat16_rn(v);
+      const float r1 = v - __bfloat162float(hh);
+      const __nv_bfloat16 hl = __float2bfloat16_rn(r1);
+      hs[0][j][rr] = hh; hs[1][j][rr] = hl; hs[2][j][rr] = __float2bfloat16_rn(r1 - __bfloat162float(hl));
+    }
+    __syncthreads();
+#pragma unroll
+    for (int ks = 0; ks < PM_ROWS / 16; ++ks) {
+      uint32_t b[2][2];
+#pragma unroll
+      for (int n = 0; n < 2; ++n) {
+        const uint32_t addr = (uint32_t)__cvta_generic_to_shared(&xs[ks * 16 + (lane & 15)][(warp * 2 + n) * 8]);
+        asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(b[n][0]), "=r"(b[n][1]) : "r"(addr));
+      }
+#pragma unroll
+      for (int sp = 0; sp < 3; ++sp)
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+          uint32_t a[4];
+          a[0] = *reinterpret_cast<const uint32_t*>(&hs[sp][m * 16 + g][ks * 16 + 2 * t]);
+          a[1] = *reinterpret_cast<const uint32_t*>(&hs[sp][m * 16 + g + 8][ks * 16 + 2 * t]);
+          a[2] = *reinterpret_cast<const uint32_t*>(&hs[sp][m * 16 + g][ks * 16 + 2 * t + 8]);
+          a[3] = *reinterpret_cast<const uint32_t*>(&hs[sp][m * 16 + g + 8][ks * 16 + 2 * t + 8]);
+          mma_bf16(acc[m][0], a, b[0][0], b[0][1]);
+          mma_bf16(acc[m][1], a, b[1][0], b[1][1]);
+        }
+    }
+    __syncthreads();
+  }
+  float* dst = mp + (int64_t)blockIdx.y * q * cols;
+#pragma unroll
+  for (int m = 0; m < MT; ++m)
+#pragma unroll
+    for (int n = 0; n < 2; ++n) {
+      const int j = m * 16 + g;
+      const int64_t col = col0 + (warp * 2 + n) * 8 + 2 * t;
+      if (col + 1 < cols) {
+        if (j < q) *reinterpret_cast<float2*>(dst + (int64_t)j * cols + col) = make_float2(acc[m][n][0], acc[m][n][1]);
+        if (j + 8 < q) *reinterpret_cast<float2*>(dst + (int64_t)(j + 8) * cols + col) = make_float2(acc[m][n][2], acc[m][n][3]);
+      }
+    }
+}
+
 // right[j][col] = sum_i basis[i][col] * W[i][j] (W == nullptr: identity).  One thread per column; each CTA
-// also records, for every j, its largest |right[j][col]| (lowest column on ties) for the sign convention.
+// also records, for every j, its entry of largest magnitude (signed value and column, lowest column on ties)
+// for the sign convention.
 __global__ void __launch_bounds__(256)
 right_rotate_kernel(const float* __restrict__ basis, int64_t cols, int k, const double* __restrict__ w,
                     float* __restrict__ right, float* __restrict__ cand_v, int* __restrict__ cand_i) {
@@ -738,39 +837,42 @@ right_rotate_kernel(const float* __restrict__ basis, int64_t cols, int k, const 
       for (int i = 0; i < MAXQ; ++i) if (i == j) v = bv[i];
     }
     if (col < cols) right[(int64_t)j * cols + col] = v;
-    float av = col < cols ? fabsf(v) : -1.0f;
+    float av = col < cols ? fabsf(v) : -1.0f, sv = v;            // magnitude for the contest, signed value for the verdict
     int ai = (int)min(col, (int64_t)0x7FFFFFFF);
 #pragma unroll
     for (int sft = 16; sft > 0; sft >>= 1) {
       const float ov = __shfl_xor_sync(0xFFFFFFFFu, av, sft);
+      const float os = __shfl_xor_sync(0xFFFFFFFFu, sv, sft);
       const int oi = __shfl_xor_sync(0xFFFFFFFFu, ai, sft);
-      if (ov > av || (ov == av && oi < ai)) { av = ov; ai = oi; }
+      if (ov > av || (ov == av && oi < ai)) { av = ov; ai = oi; sv = os; }
     }
-    if (lane == 0) { red_v[warp][j] = av; red_i[warp][j] = ai; }
+    if (lane == 0) { red_v[warp][j] = sv; red_i[warp][j] = ai; }
   }
   __syncthreads();
   if (tid < k) {
-    float av = red_v[0][tid]; int ai = red_i[0][tid];
-    for (int wv = 1; wv < 8; ++wv)
-      if (red_v[wv][tid] > av || (red_v[wv][tid] == av && red_i[wv][tid] < ai)) { av = red_v[wv][tid]; ai = red_i[wv][tid]; }
-    cand_v[(int64_t)blockIdx.x * k + tid] = av;
+    float sv = red_v[0][tid]; int ai = red_i[0][tid];
+    for (int wv = 1; wv < 8; ++wv) {
+      const float ov = red_v[wv][tid];
+      if (fabsf(ov) > fabsf(sv) || (fabsf(ov) == fabsf(sv) && red_i[wv][tid] < ai)) { sv = ov; ai = red_i[wv][tid]; }
+    }
+    cand_v[(int64_t)blockIdx.x * k + tid] = sv;                  // signed winner of this column chunk
     cand_i[(int64_t)blockIdx.x * k + tid] = ai;
   }
 }
 
 // Sign convention: the largest-magnitude entry of each right vector (lowest index on ties) is made positive.
-// grid (column chunks, k).  Every CTA re-derives the winner of its vector from the candidates.
+// grid (column chunks, k).  Every CTA re-derives the winner of its vector from the per-chunk candidates, whose
+// signed values were recorded before any flipping (the flips of other CTAs must not influence the verdict).
 __global__ void __launch_bounds__(256)
 sign_fix_kernel(float* __restrict__ right, int64_t cols, int k, const float* __restrict__ cand_v,
                 const int* __restrict__ cand_i, int n_cand, float* __restrict__ sign_out) {
   const int j = blockIdx.y;
-  float av = -1.0f; int ai = 0x7FFFFFFF;
+  float sv = 0.0f; int ai = 0x7FFFFFFF;
   for (int c = 0; c < n_cand; ++c) {
     const float v = cand_v[(int64_t)c * k + j]; const int i = cand_i[(int64_t)c * k + j];
-    if (v > av || (v == av && i < ai)) { av = v; ai = i; }
+    if (fabsf(v) > fabsf(sv) || (fabsf(v) == fabsf(sv) && i < ai)) { sv = v; ai = i; }
   }
-  const float sg = right[(int64_t)j * cols + ai] < 0.0f ? -1.0f : 1.0f;
-  __syncthreads();                                 // every thread has read the winner before anyone flips it
+  const float sg = sv < 0.0f ? -1.0f : 1.0f;
   if (blockIdx.x == 0 && threadIdx.x == 0) sign_out[j] = sg;
   const int64_t col = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (sg < 0.0f && col < cols) right[(int64_t)j * cols + col] = -right[(int64_t)j * cols + col];
@@ -837,7 +939,7 @@ SplitWs split_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) & ~(size_t)255; return o; };
   const int q = k + p;
-  const int64_t chunks = metis_ceil_div(cols, SK_COLS);
+  const int64_t chunks = metis_ceil_div(cols, SKM_COLS);
   w.amax = take(256);
   w.idx = take(sizeof(int) * (size_t)n_s);
   w.zp = take(sizeof(float) * (size_t)chunks * n_s * q);
@@ -970,8 +1072,6 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     static bool attr = false;
     if (!attr) {
       METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(sketch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)(sizeof(float) * (SK_COLS * MAXQ + SK_ROWS * SK_PITCH))));
       METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 64)));
       METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 48)));
       METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
@@ -981,17 +1081,28 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       attr = true;
     }
   }
-  // amax|x| for the residual's tensor scale: its own pass in FULL mode, fused into the broadcast pass in SAMPLED mode
-  if (full) METIS_TRY(metis_launch_amax(x, METIS_BF16, rows, cols, cols, amax, s));
-  else METIS_CUDA_TRY(cudaMemsetAsync(amax, 0, sizeof(float), s));
+  // amax|x| for the residual's tensor scale: fused into the sketch pass (FULL) or the broadcast pass (SAMPLED)
+  METIS_CUDA_TRY(cudaMemsetAsync(amax, 0, sizeof(float), s));
 
-  // (1) row sample, (2) sketch
+  // (1) row sample, (2) sketch (tensor cores; Omega generated per CTA into shared memory)
   sample_rows_kernel<<<(unsigned)metis_ceil_div(n_s, 256), 256, 0, s>>>(idx, (int)n_s, rows, seed, full ? 1 : 0); METIS_COUNT_LAUNCH();
-  const int chunks = (int)metis_ceil_div(cols, SK_COLS);
+  const int chunks = (int)metis_ceil_div(cols, SKM_COLS);
   {
-    const size_t smem = sizeof(float) * (SK_COLS * MAXQ + SK_ROWS * SK_PITCH);
-    dim3 grid((unsigned)metis_ceil_div(n_s, SK_ROWS), (unsigned)chunks);
-    sketch_kernel<<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp); METIS_COUNT_LAUNCH();
+    const int nt = (q + 7) / 8;
+    const size_t smem = sizeof(__nv_bfloat16) * nt * 8 * SKM_PITCH;
+    dim3 grid((unsigned)metis_ceil_div(n_s, SKM_ROWS), (unsigned)chunks);
+    float* am = full ? amax : nullptr;                  // FULL mode: amax|x| comes out of this pass
+    switch (nt) {
+      case 1: sketch_mma_kernel<1><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+      case 2: sketch_mma_kernel<2><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+      case 3: sketch_mma_kernel<3><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+      case 4: sketch_mma_kernel<4><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+      case 5: sketch_mma_kernel<5><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+      case 6: sketch_mma_kernel<6><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+      case 7: sketch_mma_kernel<7><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+      default: sketch_mma_kernel<8><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+    }
+    METIS_COUNT_LAUNCH();
   }
   reduce_partials_kernel<<<(unsigned)metis_ceil_div(n_s * q, 256), 256, 0, s>>>(zp, chunks, n_s * q, z); METIS_COUNT_LAUNCH();
   // (3) CholeskyQR2: orthonormal basis H of range(Z), in place
@@ -1004,7 +1115,22 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   }
   // (4) M = H^T x[S,:], eigen-decomposition of M M^T, right basis
   {
-    int rpp; const int parts = project_parts(n_s, cols, &rpp);
+    int rpp; int parts;
+    if (n_s >= 1024 && cols % 8 == 0) {
+      parts = (int)metis_ceil_div(n_s, 512);
+      if (parts > PJ_MAX_PARTS) parts = PJ_MAX_PARTS;
+      rpp = (int)(metis_ceil_div(metis_ceil_div(n_s, parts), PM_ROWS) * PM_ROWS);
+      parts = (int)metis_ceil_div(n_s, rpp);
+      dim3 grid((unsigned)metis_ceil_div(cols, PM_COLS), (unsigned)parts);
+      switch ((q + 15) / 16) {
+        case 1: project_mma_kernel<1><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+        case 2: project_mma_kernel<2><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+        case 3: project_mma_kernel<3><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+        default: project_mma_kernel<4><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+      }
+      METIS_COUNT_LAUNCH();
+    } else {
+    parts = project_parts(n_s, cols, &rpp);
     dim3 grid((unsigned)metis_ceil_div(cols, PJ_COLS), (unsigned)parts);
     const int nj4 = (q + 7) / 8;
     switch (nj4) {
@@ -1016,6 +1142,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       case 6: launch_project<6>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
       case 7: launch_project<7>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
       default: launch_project<8>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+    }
     }
     reduce_partials_kernel<<<(unsigned)metis_ceil_div((int64_t)q * cols, 256), 256, 0, s>>>(mp, parts, (int64_t)q * cols, m); METIS_COUNT_LAUNCH();
   }

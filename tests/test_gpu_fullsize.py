@@ -1,0 +1,45 @@
+"""GPU parity at the benchmark's full size and launch configuration (one LLaMA-3-8B q_proj-shaped layer,
+4096 tokens, 4096 -> 4096, k=32, p=8, SR on dY), checked on sampled output rows the oracle computes exactly."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import layer as olay, nvfp4 as onv, split as osp
+from paper_2509_00404_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3
+
+
+def test_qproj_layer_forward_and_backward_on_sampled_rows():
+    from gpu_util import rel_fro
+    from paper_2509_00404_b200 import binding as B
+    h = B.Handle(0)
+    try:
+        c = synth.config_qproj(seed=2000)
+        k, p = c["k"], c["p"]
+        dev = lambda a: torch.from_numpy(a).to(torch.bfloat16).cuda()
+        xo = h.split(dev(c["x"]), k, p, sketch=B.SKETCH_SAMPLED, seed=1)
+        wo = h.split(dev(c["w"]), k, p, sketch=B.SKETCH_FULL, seed=2)
+        do = h.split(dev(c["dy"]), k, p, sketch=B.SKETCH_SAMPLED, seed=3, rounding=B.ROUND_SR)
+        y = h.linear_fwd(xo, wo, out_dtype=torch.float32)
+        dx, dw = h.linear_bwd(do, xo, wo, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        assert h.device_status() == 0
+        xq = olay.quantize_operand(c["x"], k, p, osp.MODE_SAMPLED, 1)
+        wq = olay.quantize_operand(c["w"], k, p, osp.MODE_FULL, 2)
+        dq = olay.quantize_operand(c["dy"], k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
+        # top-k singular values of all three operands
+        for op, q in ((xo, xq), (wo, wq), (do, dq)):
+            sig = op.sigma.cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(sig - q.sigma) / q.sigma) < 1e-3
+        rows = np.random.default_rng(0).choice(4096, 192, replace=False)
+        xd, wd_c = xq.dense(onv.AXIS_COLS), wq.dense(onv.AXIS_COLS)
+        assert rel_fro(y.cpu().numpy()[rows], xd[rows] @ wd_c.T) < TOL
+        dd_c, wd_r = dq.dense(onv.AXIS_COLS), wq.dense(onv.AXIS_ROWS)
+        assert rel_fro(dx.cpu().numpy()[rows], dd_c[rows] @ wd_r) < TOL
+        dd_r, xd_r = dq.dense(onv.AXIS_ROWS), xq.dense(onv.AXIS_ROWS)
+        assert rel_fro(dw.cpu().numpy()[rows], dd_r[:, rows].T @ xd_r) < TOL
+    finally:
+        h.close()

@@ -31,12 +31,15 @@ def _check_against_oracle(B, h, x, k, p, mode, seed, rounding=0):
     sp = osp.split(x.astype(np.float64), k, p, mode, seed=seed)
     sig = op.sigma.cpu().numpy()
     assert np.max(np.abs(sig - sp.sigma) / sp.sigma) < 1e-3                 # top-k singular values
-    assert rel_fro(dense, sp.residual) < 1e-5                               # residual before quantization
+    # residual before quantization: the factors are FP32, so the low-rank part carries ~2^-24 relative noise, which
+    # shows up in the residual magnified by ||X|| / ||R||
+    tol_r = max(1e-6, 32 * 2.0 ** -24 * np.linalg.norm(x) / np.linalg.norm(sp.residual))
+    assert tol_r < 1e-4 and rel_fro(dense, sp.residual) < tol_r
     left, right = op.left.cpu().numpy().T.astype(np.float64), op.right.cpu().numpy().T.astype(np.float64)
     assert rel_fro(left, sp.left) < 1e-3 and rel_fro(right, sp.right) < 1e-3
     # invariants that hold whatever the oracle says
     assert np.allclose(left.T @ left, np.eye(k), atol=1e-4) and np.allclose(right.T @ right, np.eye(k), atol=1e-4)
-    assert rel_fro((left * sig) @ right.T + dense, x) < 1e-5
+    assert rel_fro((left * sig) @ right.T + dense, x) < 1e-5 * max(1.0, 0.1 * np.linalg.norm(x) / np.linalg.norm(sp.residual))
     # the fused quantizer saw `dense`: the oracle's encoder on the same values must give the same bytes
     s_src = onv.tensor_scale_from_amax(np.max(np.abs(x)))
     for t, axis in ((op.res_by_cols, onv.AXIS_COLS), (op.res_by_rows, onv.AXIS_ROWS)):
@@ -64,6 +67,13 @@ def test_sampled_mode_and_stochastic_rounding(ctx):
     _check_against_oracle(B, h, x, 16, 8, B.SKETCH_SAMPLED, seed=21)
     d, _ = synth.llama_like(1024, 384, 1e-4, 42, rank=8)
     _check_against_oracle(B, h, d, 8, 8, B.SKETCH_SAMPLED, seed=22, rounding=1)
+
+
+def test_full_mode_tall_operand_uses_the_row_split_tensor_core_path(ctx):
+    """More than 1024 rows: the sketch spans several row tiles and the projection runs on its tensor-core kernel."""
+    B, h = ctx
+    x, _ = synth.llama_like(1536, 320, 0.02, 43, rank=8)
+    _check_against_oracle(B, h, x, 8, 8, B.SKETCH_FULL, seed=31)
 
 
 def test_planted_noise_free_spectrum_is_recovered(ctx):
