@@ -29,6 +29,7 @@ L_TOKENS, D_IN, D_OUT, RANK_K, OVERSAMPLE_P = 4096, 4096, 4096, 32, 8
 WORKLOAD = "llama3-8b q_proj linear fwd+bwd, tokens 4096 (2x2048), 4096->4096, k=32 p=8, SR on dY"
 N_SETS = 3
 FP4_OVER_BF16 = 4.0           # nominal dense FP4 : bf16 tensor throughput ratio
+GEMM_DRAM_BYTES_NCU = 19.08e6 + 0.16e6   # per 4096^3 launch (profiles/gemm_nvfp4_2cta_4096x4096x4096.md)
 
 
 def measured_peaks():
@@ -55,7 +56,7 @@ class ClockSampler(threading.Thread):
     def run(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=subprocess.PIPE, text=True)
             for line in self.proc.stdout:
                 self.rows.append([c.strip() for c in line.split(",")])
         except Exception:
@@ -297,15 +298,16 @@ def main():
                 "h2d_bytes_per_step": 3 * l * m * 2, "d2h_bytes_per_step": 3 * l * m * 2, "ms_per_step": ms_e2e},
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "roofline": {"bound": "tensor", "kernel": "gemm_nvfp4_kernel<128> (4096x4096x4096 residual GEMM)",
+        "roofline": {"bound": "tensor", "kernel": "two_cta::gemm_nvfp4_2cta_kernel (4096x4096x4096 residual GEMM, bf16 out)",
                      "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak,
-                     "traffic": None, "peak_source": "bf16 burst peak (%s) x %.0f nominal FP4:bf16 ratio" % (peaks["source"], FP4_OVER_BF16),
+                     "traffic": GEMM_DRAM_BYTES_NCU, "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch, see profiles/",
+                     "algorithmic_bytes": 0.5625 * 2 * l * m + 2.0 * l * n, "peak_source": "bf16 burst peak (%s) x %.0f nominal FP4:bf16 ratio" % (peaks["source"], FP4_OVER_BF16),
                      "ms_per_launch": gemm_ms},
         "split_overhead_vs_three_plain_gemms": overhead,
         "device_status": status,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        sample = 256
+        sample = 1024
         dt, f = oracle_sample_step(sample, 4242)
         line["cpu_baseline"] = {"value": f / dt / 1e12, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle",
                                 "sample": "%d of %d tokens, full 4096x4096 weight, one pass (%.1f s)" % (sample, l, dt)}
