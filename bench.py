@@ -150,7 +150,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2509_00404_b200 import binding as B, synth
+    from paper_2509_00404_b200 import binding as B, parallel, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -204,8 +204,7 @@ def main():
         h_x.linear_fwd(xo, wo, out=y)
         main.wait_event(ev_d)
         h_x.linear_bwd(do, xo, wo, out=(dx, dw))
-        if world > 1:
-            dist.all_reduce(dw)
+        parallel.allreduce_weight_grad_(dw)          # token-sharded ranks: the one exchange of the path
 
     def barrier():
         if world > 1:
