@@ -143,6 +143,7 @@ def main():
                     help="split: W_t is split (FULL sketch) and quantized every step; requant: W_t is split once, "
                          "its stored residual and factors are re-quantized every step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying CUDA graphs")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -181,12 +182,12 @@ def main():
 
     # The three operand decompositions are independent of each other, and the dY chain is independent of the
     # forward product: they run on three streams and join by events (torch streams: plumbing only).
-    main = torch.cuda.current_stream()
     side_w, side_d = torch.cuda.Stream(), torch.cuda.Stream()
     ev_start, ev_w, ev_d = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
     h_x, h_w, h_d = h, B.Handle(local_rank), B.Handle(local_rank)     # one workspace owner per stream
 
     def step(bufs, i):
+        main = torch.cuda.current_stream()
         ev_start.record(main)
         side_w.wait_event(ev_start)
         side_d.wait_event(ev_start)
@@ -216,22 +217,61 @@ def main():
         step(dev_sets[i % N_SETS], i)
     barrier()
     assert h.device_status() == 0, "a bounded device wait expired during warm-up"
-    launches0 = B.launch_count()
+    l0 = B.launch_count()
+    step(dev_sets[0], 0)
+    barrier()
+    launches_per_step = B.launch_count() - l0
+
+    # One step is ~100 short kernels on three streams: replaying it as a CUDA graph (one per input set; the
+    # seeds are baked in, all work is re-executed) takes the host's launch cost off the critical path.
+    use_graph = world == 1 and not args.no_graph
+    stage = {key: torch.empty_like(v) for key, v in dev_sets[0].items()}
+    graphs, graph_e2e = [], None
+    if use_graph:
+        try:
+            for s_i in range(N_SETS):
+                g_ = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_):
+                    step(dev_sets[s_i], s_i)
+                graphs.append(g_)
+            graph_e2e = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph_e2e):
+                step(stage, 0)
+            # the replay must reproduce the host-launched step bit for bit (all kernels are deterministic)
+            step(dev_sets[0], 0)
+            barrier()
+            ref_out = [t.clone() for t in (y, dx, dw)]
+            graphs[0].replay()
+            barrier()
+            assert all(torch.equal(a_, b_) for a_, b_ in zip(ref_out, (y, dx, dw))), "graph replay differs from host launches"
+            del ref_out
+        except AssertionError:
+            raise
+        except Exception as exc:                     # fall back to host launches, say so in the output
+            sys.stderr.write("CUDA graph capture failed (%s); using host launches\n" % exc)
+            use_graph, graphs, graph_e2e = False, [], None
+            torch.cuda.synchronize()
+
+    def run_step(i):
+        if use_graph:
+            graphs[i % N_SETS].replay()
+        else:
+            step(dev_sets[i % N_SETS], i)
+
     sampler.start()
     time.sleep(0.3)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
     for i in range(args.steps):
-        step(dev_sets[i % N_SETS], i)
+        run_step(i)
     e1.record()
     barrier()
     ms = e0.elapsed_time(e1) / args.steps
-    launches = B.launch_count() - launches0
+    launches = launches_per_step * args.steps
     status = h.device_status() | h_w.device_status() | h_d.device_status()
 
     # ---- end to end: pinned host inputs in, results out, every step ---------------------------------
-    stage = {key: torch.empty_like(v) for key, v in dev_sets[0].items()}
     y_h, dx_h, dw_h = (torch.empty((l, n), dtype=bf).pin_memory(), torch.empty((l, m), dtype=bf).pin_memory(),
                        torch.empty((n, m), dtype=bf).pin_memory())
 
@@ -239,7 +279,10 @@ def main():
         hs = host_sets[i % N_SETS]
         for key in ("x", "w", "dy"):
             stage[key].copy_(hs[key], non_blocking=True)
-        step(stage, i)
+        if use_graph:
+            graph_e2e.replay()
+        else:
+            step(stage, i)
         y_h.copy_(y, non_blocking=True)
         dx_h.copy_(dx, non_blocking=True)
         dw_h.copy_(dw, non_blocking=True)
@@ -290,7 +333,7 @@ def main():
         "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4 (e2m1 x ue4m3, fp32 accumulate)",
         "data": "synthetic",
-        "config": {"workload": WORKLOAD, "weights": args.weights,
+        "config": {"workload": WORKLOAD, "weights": args.weights, "cuda_graph": bool(use_graph),
                    "l2": "inputs rotate over %d sets (%d MB > 126 MB L2)" % (N_SETS, N_SETS * 3 * l * m * 2 // 2 ** 20),
                    "parallelism": "dp%d (token-sharded, dW all-reduce)" % world if world > 1 else "single GPU"},
         "e2e": {"value": world * flops_step / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s",

@@ -234,7 +234,8 @@ __device__ __forceinline__ double fast_rsqrt(double x) {
 }
 
 __global__ void __launch_bounds__(256)
-jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, double* __restrict__ evals, double* __restrict__ evecs) {
+jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, double* __restrict__ evals,
+                  double* __restrict__ evecs) {
   extern __shared__ __align__(16) unsigned char jsm[];
   double (*Y)[MAXQ + 1] = reinterpret_cast<double (*)[MAXQ + 1]>(jsm);
   __shared__ double lam[MAXQ];
@@ -289,8 +290,8 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, double* __restric
   // ---- one-sided Jacobi on the columns of Y ----
   // Column norms are carried along (alpha' = alpha - t*gamma, beta' = beta + t*gamma) and recomputed exactly at
   // the start of every sweep, so a round needs a single inner product per couple.  A sweep whose largest
-  // |cos| between paired columns was below 1e-7 is the last one: convergence is quadratic, its rotations
-  // leave the columns orthogonal to ~1e-14.
+  // cos^2 between paired columns was below exit_cos2 is the last one: convergence is quadratic, so its own
+  // rotations leave the columns orthogonal to about exit_cos2 (as |cos|).
   const int m = tid >> 3, sub = tid & 7;                // couple index, row slice
   const bool active = m < half;
   for (int sweep = 0; sweep < 16; ++sweep) {
@@ -345,7 +346,7 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, double* __restric
     }
     const float maxcos2 = __uint_as_float((unsigned int)rotated[0]);
     __syncthreads();
-    if (maxcos2 < 1e-14f) break;
+    if (maxcos2 < exit_cos2) break;
   }
   // ---- eigenvalues = squared column norms, eigenvectors = normalised columns ----
   if (tid < n) {
@@ -1150,7 +1151,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     int64_t rpp; const int parts = gram_parts(cols, &rpp);
     gram_kernel<<<parts, 256, 0, s>>>(m, cols, q, 1, cols, rpp, gram); METIS_COUNT_LAUNCH();
     reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1); METIS_COUNT_LAUNCH();
-    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram1, q, q, evals, evecs); METIS_COUNT_LAUNCH();
+    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram1, q, q, 1e-8f, evals, evecs); METIS_COUNT_LAUNCH();
   }
   right_basis_kernel<<<(unsigned)metis_ceil_div(cols, 64), 64, 0, s>>>(m, cols, q, k, evals, evecs, basis,
                                                                           full ? out->sigma : nullptr); METIS_COUNT_LAUNCH();
@@ -1200,7 +1201,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   if (!full) {
     // (7) Rayleigh-Ritz on C^T C (Gram partials came out of the broadcast pass), rotate both factors
     reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 128), 128, 0, sf>>>(gram_c, n_cta_c, kp * kp, gram1); METIS_COUNT_LAUNCH();
-    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, sf>>>(gram1, k, kp, evals2, evecs2); METIS_COUNT_LAUNCH();
+    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, sf>>>(gram1, k, kp, 1e-6f, evals2, evecs2); METIS_COUNT_LAUNCH();
     right_rotate_kernel<<<n_cand, 256, 0, sf>>>(basis, cols, k, evecs2, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
     sign_fix_kernel<<<dim3(n_cand, k), 256, 0, sf>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign); METIS_COUNT_LAUNCH();
     left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 64, 0, sf>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
