@@ -37,7 +37,8 @@ __global__ void reduce_partials_kernel(const float* __restrict__ zp, int n_chunk
 constexpr int GR_TILE = 32;
 __global__ void __launch_bounds__(256)
 gram_kernel(const float* __restrict__ v, int64_t n_rows, int n, int64_t stride_row, int64_t stride_vec,
-            int64_t rows_per_part, double* __restrict__ part) {
+            int64_t rows_per_part, double* __restrict__ part, const int* __restrict__ skip) {
+  if (skip != nullptr && *skip) return;                 // second CholeskyQR pass not needed (see chol_kernel)
   __shared__ float tile[GR_TILE][MAXQ + 1];
   const int tid = threadIdx.x;
   const int64_t r_begin = (int64_t)blockIdx.x * rows_per_part;
@@ -92,9 +93,12 @@ __device__ __forceinline__ double fast_rsqrt_wide(double x) { return chol_rsqrt(
 // dependent sketch column: its reciprocal is stored as zero, so the corresponding column of H = Z L^-T
 // becomes zero instead of amplified noise.
 __global__ void __launch_bounds__(256)
-chol_kernel(const double* __restrict__ g, int q, double* __restrict__ l_out, double* __restrict__ invd_out) {
+chol_kernel(const double* __restrict__ g, int q, double* __restrict__ l_out, double* __restrict__ invd_out,
+            const int* __restrict__ skip, int* __restrict__ well_conditioned) {
+  if (skip != nullptr && *skip) return;
   __shared__ double L[MAXQ][MAXQ + 1];
   __shared__ double gmax_s;
+  __shared__ double dmin_s;
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   for (int o = tid; o < q * q; o += 256) L[o / q][o % q] = g[o];
   __syncthreads();
@@ -113,7 +117,11 @@ chol_kernel(const double* __restrict__ g, int q, double* __restrict__ l_out, dou
     const double inv = dep ? 0.0 : chol_rsqrt(d);
     __syncthreads();
     for (int i = j + 1 + tid; i < q; i += 256) L[i][j] *= inv;
-    if (tid == 0) { L[j][j] = dep ? 0.0 : d * inv; invd_out[j] = inv; }
+    if (tid == 0) {
+      L[j][j] = dep ? 0.0 : d * inv; invd_out[j] = inv;
+      if (j == 0) dmin_s = gmax_s;
+      if (!dep) dmin_s = fmin(dmin_s, d);
+    }
     __syncthreads();
     if (!dep) {
       for (int a = j + 1 + ty; a < q; a += 16) {
@@ -123,13 +131,18 @@ chol_kernel(const double* __restrict__ g, int q, double* __restrict__ l_out, dou
     }
     __syncthreads();
   }
+  // With every pivot above 1e-8 of the largest diagonal the FP64 factorisation leaves Z L^-T orthonormal to
+  // ~1e-8 already, below the FP32 rounding of its storage: the caller's second pass is then skipped.
+  if (tid == 0 && well_conditioned != nullptr) *well_conditioned = (dmin_s > 1e-8 * gmax_s) ? 1 : 0;
   for (int o = tid; o < q * q; o += 256) l_out[o] = L[o / q][o % q];
 }
 
 // One CholeskyQR pass, step 2: z_row <- z_row L^-T by forward substitution, one warp per row:
 // h_j = (z_j - sum_{i<j} h_i L[j][i]) / L[j][j]; lane i%32 keeps h_i, the dot product is a warp reduction.
 __global__ void __launch_bounds__(256)
-apply_chol_kernel(float* __restrict__ z, int64_t n_rows, int q, const double* __restrict__ l, const double* __restrict__ invd) {
+apply_chol_kernel(float* __restrict__ z, int64_t n_rows, int q, const double* __restrict__ l, const double* __restrict__ invd,
+                  const int* __restrict__ skip) {
+  if (skip != nullptr && *skip) return;
   __shared__ double L[MAXQ][MAXQ + 1];
   __shared__ double inv_s[MAXQ];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -372,27 +385,32 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
 
 // ------------------------------------------------------------------------------------------------
 // Right basis from the small SVD: B[j][col] = sum_i Ut[i][j] M[i][col] / s_j, s_j = sqrt(eval_j); j < k.
-__global__ void __launch_bounds__(64)
+// Block = 64 columns x 4 groups of output vectors; a thread keeps four accumulators in flight.
+__global__ void __launch_bounds__(256)
 right_basis_kernel(const float* __restrict__ m, int64_t cols, int q, int k, const double* __restrict__ evals,
                    const double* __restrict__ evecs, float* __restrict__ basis, float* __restrict__ sigma_out) {
   __shared__ double ut[MAXQ][MAXQ + 1];
   __shared__ double inv_s[MAXQ];
-  const int tid = threadIdx.x;
-  for (int o = tid; o < q * q; o += 64) ut[o / q][o % q] = evecs[o];
+  const int tid = threadIdx.x, cx = tid & 63, jg = tid >> 6;
+  for (int o = tid; o < q * q; o += 256) ut[o / q][o % q] = evecs[o];
   if (tid < k) {
     const double s = sqrt(fmax(evals[tid], 0.0));
     inv_s[tid] = s > 0.0 ? 1.0 / s : 0.0;
     if (blockIdx.x == 0 && sigma_out != nullptr) sigma_out[tid] = (float)s;
   }
   __syncthreads();
-  const int64_t col = (int64_t)blockIdx.x * 64 + tid;
+  const int64_t col = (int64_t)blockIdx.x * 64 + cx;
   if (col >= cols) return;
-  float mv[MAXQ];
-  for (int i = 0; i < q; ++i) mv[i] = m[(int64_t)i * cols + col];
-  for (int j = 0; j < k; ++j) {
-    double a = 0.0;
-    for (int i = 0; i < q; ++i) a += ut[i][j] * (double)mv[i];
-    basis[(int64_t)j * cols + col] = (float)(a * inv_s[j]);
+  for (int j0 = jg * 4; j0 < k; j0 += 16) {
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    for (int i = 0; i < q; ++i) {
+      const double v = (double)m[(int64_t)i * cols + col];
+      a0 += ut[i][j0] * v; a1 += ut[i][j0 + 1] * v; a2 += ut[i][j0 + 2] * v; a3 += ut[i][j0 + 3] * v;
+    }
+    basis[(int64_t)j0 * cols + col] = (float)(a0 * inv_s[j0]);
+    if (j0 + 1 < k) basis[(int64_t)(j0 + 1) * cols + col] = (float)(a1 * inv_s[j0 + 1]);
+    if (j0 + 2 < k) basis[(int64_t)(j0 + 2) * cols + col] = (float)(a2 * inv_s[j0 + 2]);
+    if (j0 + 3 < k) basis[(int64_t)(j0 + 3) * cols + col] = (float)(a3 * inv_s[j0 + 3]);
   }
 }
 
@@ -540,7 +558,9 @@ coeff_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols
 }
 
 // out[e] = sum over all partials p of in[p][e], in order (eight independent loads in flight per thread).
-__global__ void reduce_gram_kernel(const double* __restrict__ in, int n_in, int nn, double* __restrict__ out) {
+__global__ void reduce_gram_kernel(const double* __restrict__ in, int n_in, int nn, double* __restrict__ out,
+                                   const int* __restrict__ skip) {
+  if (skip != nullptr && *skip) return;
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= nn) return;
   double a = 0.0;
@@ -866,7 +886,7 @@ right_rotate_kernel(const float* __restrict__ basis, int64_t cols, int k, const 
 // signed values were recorded before any flipping (the flips of other CTAs must not influence the verdict).
 __global__ void __launch_bounds__(256)
 sign_fix_kernel(float* __restrict__ right, int64_t cols, int k, const float* __restrict__ cand_v,
-                const int* __restrict__ cand_i, int n_cand, float* __restrict__ sign_out) {
+                const int* __restrict__ cand_i, int n_cand, float* __restrict__ sign_out, float* __restrict__ amax_out) {
   const int j = blockIdx.y;
   float sv = 0.0f; int ai = 0x7FFFFFFF;
   for (int c = 0; c < n_cand; ++c) {
@@ -874,7 +894,11 @@ sign_fix_kernel(float* __restrict__ right, int64_t cols, int k, const float* __r
     if (fabsf(v) > fabsf(sv) || (fabsf(v) == fabsf(sv) && i < ai)) { sv = v; ai = i; }
   }
   const float sg = sv < 0.0f ? -1.0f : 1.0f;
-  if (blockIdx.x == 0 && threadIdx.x == 0) sign_out[j] = sg;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    sign_out[j] = sg;
+    // the winner's magnitude is the vector's amax: the factor's tensor scale needs the max over all vectors
+    if (amax_out != nullptr) atomicMax(reinterpret_cast<unsigned int*>(amax_out), __float_as_uint(fabsf(sv)));
+  }
   const int64_t col = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (sg < 0.0f && col < cols) right[(int64_t)j * cols + col] = -right[(int64_t)j * cols + col];
 }
@@ -883,15 +907,16 @@ sign_fix_kernel(float* __restrict__ right, int64_t cols, int k, const float* __r
 // scale_j = 1/sqrt(eval_j) when inv_sqrt_evals is given (Rayleigh-Ritz normalisation), else 1.
 // Also writes sigma_out[j] = sqrt(eval_j) when asked, and coef_rm[r][j] = left[j][r] * sigma_for_coef[j]
 // (row-major, kp columns, zero padded) when asked.
-__global__ void __launch_bounds__(64)
+__global__ void __launch_bounds__(256)
 left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, int64_t stride_i, int64_t stride_r,
                    const double* __restrict__ w, const double* __restrict__ evals_for_scale,
                    const float* __restrict__ sign, float* __restrict__ left, float* __restrict__ sigma_out,
-                   float* __restrict__ coef_rm, int kp, const float* __restrict__ sigma_for_coef) {
+                   float* __restrict__ coef_rm, int kp, const float* __restrict__ sigma_for_coef,
+                   float* __restrict__ amax_out) {
   __shared__ double ws[MAXQ][MAXQ + 1];
   __shared__ double scl[MAXQ];
-  const int tid = threadIdx.x;
-  for (int o = tid; o < n_in * n_in; o += 64) ws[o / n_in][o % n_in] = w[o];
+  const int tid = threadIdx.x, rx = tid & 63, jg = tid >> 6;
+  for (int o = tid; o < n_in * n_in; o += 256) ws[o / n_in][o % n_in] = w[o];
   if (tid < k) {
     double s = 1.0;
     if (evals_for_scale) {
@@ -902,18 +927,35 @@ left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, i
     scl[tid] = s * (double)sign[tid];
   }
   __syncthreads();
-  const int64_t r = (int64_t)blockIdx.x * 64 + tid;
-  if (r >= rows) return;
-  float cv[MAXQ];
-  for (int i = 0; i < n_in; ++i) cv[i] = c[i * stride_i + r * stride_r];
-  for (int j = 0; j < k; ++j) {
-    double a = 0.0;
-    for (int i = 0; i < n_in; ++i) a += (double)cv[i] * ws[i][j];
-    const float v = (float)(a * scl[j]);
-    left[(int64_t)j * rows + r] = v;
-    if (coef_rm) coef_rm[r * kp + j] = v * sigma_for_coef[j];
+  const int64_t r = (int64_t)blockIdx.x * 64 + rx;
+  float am = 0.0f;
+  if (r < rows) {
+    for (int j0 = jg * 4; j0 < kp; j0 += 16) {
+      double a[4] = {0.0, 0.0, 0.0, 0.0};
+      if (j0 < k) {
+        for (int i = 0; i < n_in; ++i) {
+          const double v = (double)c[i * stride_i + r * stride_r];
+          a[0] += v * ws[i][j0]; a[1] += v * ws[i][j0 + 1]; a[2] += v * ws[i][j0 + 2]; a[3] += v * ws[i][j0 + 3];
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int j = j0 + t;
+        if (j < k) {
+          const float v = (float)(a[t] * scl[j]);
+          left[(int64_t)j * rows + r] = v;
+          am = fmaxf(am, fabsf(v));
+          if (coef_rm) coef_rm[r * kp + j] = v * sigma_for_coef[j];
+        } else if (coef_rm && j < kp) {
+          coef_rm[r * kp + j] = 0.0f;
+        }
+      }
+    }
   }
-  if (coef_rm) for (int j = k; j < kp; ++j) coef_rm[r * kp + j] = 0.0f;
+  // amax|left| for the factor's tensor scale (order-independent atomic max on the float bits)
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+  if ((tid & 31) == 0 && amax_out != nullptr) atomicMax(reinterpret_cast<unsigned int*>(amax_out), __float_as_uint(am));
 }
 
 struct SplitWs {
@@ -1052,6 +1094,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   double* gram = reinterpret_cast<double*>(wsb + L.gram);
   double* linv = reinterpret_cast<double*>(wsb + L.linv);
   double* invd = linv + MAXQ * MAXQ;
+  int* cond_flag = reinterpret_cast<int*>(amax + 8);
   double* gram1 = reinterpret_cast<double*>(wsb + L.gram1);
   double* evals = reinterpret_cast<double*>(wsb + L.evals);
   double* evecs = reinterpret_cast<double*>(wsb + L.evecs);
@@ -1083,7 +1126,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     }
   }
   // amax|x| for the residual's tensor scale: fused into the sketch pass (FULL) or the broadcast pass (SAMPLED)
-  METIS_CUDA_TRY(cudaMemsetAsync(amax, 0, sizeof(float), s));
+  METIS_CUDA_TRY(cudaMemsetAsync(amax, 0, 64, s));       // amax slots of x, left, right and the condition flag
 
   // (1) row sample, (2) sketch (tensor cores; Omega generated per CTA into shared memory)
   sample_rows_kernel<<<(unsigned)metis_ceil_div(n_s, 256), 256, 0, s>>>(idx, (int)n_s, rows, seed, full ? 1 : 0); METIS_COUNT_LAUNCH();
@@ -1109,10 +1152,11 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   // (3) CholeskyQR2: orthonormal basis H of range(Z), in place
   for (int pass = 0; pass < 2; ++pass) {
     int64_t rpp; const int parts = gram_parts(n_s, &rpp);
-    gram_kernel<<<parts, 256, 0, s>>>(z, n_s, q, q, 1, rpp, gram); METIS_COUNT_LAUNCH();
-    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1); METIS_COUNT_LAUNCH();
-    chol_kernel<<<1, 256, 0, s>>>(gram1, q, linv, invd); METIS_COUNT_LAUNCH();
-    apply_chol_kernel<<<(unsigned)metis_ceil_div(n_s, 8), 256, 0, s>>>(z, n_s, q, linv, invd); METIS_COUNT_LAUNCH();
+    const int* skip = pass == 0 ? nullptr : cond_flag;
+    gram_kernel<<<parts, 256, 0, s>>>(z, n_s, q, q, 1, rpp, gram, skip); METIS_COUNT_LAUNCH();
+    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1, skip); METIS_COUNT_LAUNCH();
+    chol_kernel<<<1, 256, 0, s>>>(gram1, q, linv, invd, skip, pass == 0 ? cond_flag : nullptr); METIS_COUNT_LAUNCH();
+    apply_chol_kernel<<<(unsigned)metis_ceil_div(n_s, 8), 256, 0, s>>>(z, n_s, q, linv, invd, skip); METIS_COUNT_LAUNCH();
   }
   // (4) M = H^T x[S,:], eigen-decomposition of M M^T, right basis
   {
@@ -1149,11 +1193,11 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   }
   {
     int64_t rpp; const int parts = gram_parts(cols, &rpp);
-    gram_kernel<<<parts, 256, 0, s>>>(m, cols, q, 1, cols, rpp, gram); METIS_COUNT_LAUNCH();
-    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1); METIS_COUNT_LAUNCH();
+    gram_kernel<<<parts, 256, 0, s>>>(m, cols, q, 1, cols, rpp, gram, nullptr); METIS_COUNT_LAUNCH();
+    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1, nullptr); METIS_COUNT_LAUNCH();
     jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram1, q, q, 1e-8f, evals, evecs); METIS_COUNT_LAUNCH();
   }
-  right_basis_kernel<<<(unsigned)metis_ceil_div(cols, 64), 64, 0, s>>>(m, cols, q, k, evals, evecs, basis,
+  right_basis_kernel<<<(unsigned)metis_ceil_div(cols, 64), 256, 0, s>>>(m, cols, q, k, evals, evecs, basis,
                                                                           full ? out->sigma : nullptr); METIS_COUNT_LAUNCH();
   // (5) coefficients of every row in the basis, (6) fused residual + quantizer
   const int n_cand = (int)metis_ceil_div(cols, 256);
@@ -1161,10 +1205,10 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   if (full) {
     // left = H U~_k, right = basis (sign fixed); coefficients = left * sigma
     right_rotate_kernel<<<n_cand, 256, 0, s>>>(basis, cols, k, nullptr, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
-    sign_fix_kernel<<<dim3(n_cand, k), 256, 0, s>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign); METIS_COUNT_LAUNCH();
+    sign_fix_kernel<<<dim3(n_cand, k), 256, 0, s>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2); METIS_COUNT_LAUNCH();
     basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(out->right, cols, k, kp, bs, bt); METIS_COUNT_LAUNCH();
-    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 64, 0, s>>>(z, rows, q, k, 1, q, evecs, nullptr, sign,
-                                                                           out->left, nullptr, coef, kp, out->sigma); METIS_COUNT_LAUNCH();
+    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 256, 0, s>>>(z, rows, q, k, 1, q, evecs, nullptr, sign,
+                                                                            out->left, nullptr, coef, kp, out->sigma, amax + 1); METIS_COUNT_LAUNCH();
   } else {
     basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(basis, cols, k, kp, bs, bt); METIS_COUNT_LAUNCH();
     const size_t smem = sizeof(float) * 9 * 32 * kp;
@@ -1200,21 +1244,19 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   cudaStream_t sf = ctx->side[0];
   if (!full) {
     // (7) Rayleigh-Ritz on C^T C (Gram partials came out of the broadcast pass), rotate both factors
-    reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 128), 128, 0, sf>>>(gram_c, n_cta_c, kp * kp, gram1); METIS_COUNT_LAUNCH();
+    reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 128), 128, 0, sf>>>(gram_c, n_cta_c, kp * kp, gram1, nullptr); METIS_COUNT_LAUNCH();
     jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, sf>>>(gram1, k, kp, 1e-6f, evals2, evecs2); METIS_COUNT_LAUNCH();
     right_rotate_kernel<<<n_cand, 256, 0, sf>>>(basis, cols, k, evecs2, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
-    sign_fix_kernel<<<dim3(n_cand, k), 256, 0, sf>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign); METIS_COUNT_LAUNCH();
-    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 64, 0, sf>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
-                                                                           out->left, out->sigma, nullptr, 0, nullptr); METIS_COUNT_LAUNCH();
+    sign_fix_kernel<<<dim3(n_cand, k), 256, 0, sf>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2); METIS_COUNT_LAUNCH();
+    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 256, 0, sf>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
+                                                                            out->left, out->sigma, nullptr, kp, nullptr, amax + 1); METIS_COUNT_LAUNCH();
   }
   METIS_CUDA_TRY(cudaGetLastError());
   // (8) quantize the factors (stored transposed: k x rows, k x cols; blocks along the long dimension)
   metis_nvfp4_t lq = out->left_q, rq = out->right_q;
   lq.rows = k; lq.k_len = rows; rq.rows = k; rq.k_len = cols;
-  METIS_TRY(metis_launch_amax(out->left, METIS_FP32, k, rows, rows, amax + 1, sf));
   METIS_TRY(metis_launch_quantize(out->left, METIS_FP32, k, rows, rows, rounding, seed, METIS_STREAM_LEFT, rows, 1,
                                   amax + 1, 1, &lq, nullptr, sf));
-  METIS_TRY(metis_launch_amax(out->right, METIS_FP32, k, cols, cols, amax + 2, sf));
   METIS_TRY(metis_launch_quantize(out->right, METIS_FP32, k, cols, cols, rounding, seed, METIS_STREAM_RIGHT, cols, 1,
                                   amax + 2, 1, &rq, nullptr, sf));
   return metis_join(ctx, s, 0);
