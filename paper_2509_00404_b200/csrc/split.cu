@@ -246,6 +246,7 @@ __device__ __forceinline__ double fast_rsqrt(double x) {
   return y;
 }
 
+template <int R>                                        // rows per lane: ceil(n / 8)
 __global__ void __launch_bounds__(256)
 jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, double* __restrict__ evals,
                   double* __restrict__ evecs) {
@@ -301,17 +302,22 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
   }
   __syncthreads();
   // ---- one-sided Jacobi on the columns of Y ----
-  // Column norms are carried along (alpha' = alpha - t*gamma, beta' = beta + t*gamma) and recomputed exactly at
-  // the start of every sweep, so a round needs a single inner product per couple.  A sweep whose largest
-  // cos^2 between paired columns was below exit_cos2 is the last one: convergence is quadratic, so its own
-  // rotations leave the columns orthogonal to about exit_cos2 (as |cos|).
+  // FP64 is kept for what sets the accuracy of the result - the columns themselves and the orthonormality of
+  // each applied rotation - and FP32 is used for what only steers convergence: the carried column norms, the
+  // rotation angle and the convergence measure.  (FP64 instructions are the slow ones in this latency chain.)
+  // Norms are carried along and recomputed exactly at the start of every sweep, so a round needs a single
+  // inner product per couple.  A sweep whose largest cos^2 between paired columns was below exit_cos2 is the
+  // last one: convergence is quadratic, so its own rotations leave the columns orthogonal to about exit_cos2.
+  float* lamf = reinterpret_cast<float*>(lam);          // FP32 norms during the sweeps (lam is reused below)
   const int m = tid >> 3, sub = tid & 7;                // couple index, row slice
   const bool active = m < half;
   for (int sweep = 0; sweep < 16; ++sweep) {
     if (tid < np) {
-      double a = 0.0;
-      for (int i = 0; i < np; ++i) a += Y[i][tid] * Y[i][tid];
-      lam[tid] = a;
+      double a0 = 0.0, a1 = 0.0;
+      int i = 0;
+      for (; i + 1 < np; i += 2) { a0 += Y[i][tid] * Y[i][tid]; a1 += Y[i + 1][tid] * Y[i + 1][tid]; }
+      if (i < np) a0 += Y[i][tid] * Y[i][tid];
+      lamf[tid] = (float)(a0 + a1);
     }
     if (tid == 0) rotated[0] = 0;                       // reused as the sweep's max cos^2 (float bits)
     __syncthreads();
@@ -319,10 +325,10 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
       {
         // every lane takes part in the shuffles; lanes of couples beyond n/2 carry zeros and write nothing
         const int p = active ? pairs[step][m][0] : 0, q = active ? pairs[step][m][1] : 0;
-        double yp[MAXQ / 8], yq[MAXQ / 8];
+        double yp[R], yq[R];
         double c = 0.0;
 #pragma unroll
-        for (int t = 0; t < MAXQ / 8; ++t) {
+        for (int t = 0; t < R; ++t) {
           const int i = sub + 8 * t;
           yp[t] = (active && i < np) ? Y[i][p] : 0.0;
           yq[t] = (active && i < np) ? Y[i][q] : 0.0;
@@ -330,16 +336,20 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
         }
 #pragma unroll
         for (int o = 4; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
-        const double a = lam[p], b = lam[q];
+        const float a = lamf[p], b = lamf[q], cf = (float)c;
+        const float cos2 = (cf / a) * (cf / b);
         // rotate only if the two columns are not yet orthogonal to working precision
-        if (active && c * c > 1e-26 * a * b) {
-          float zeta = (float)(b - a) / (2.0f * (float)c);
+        if (active && cos2 > 1e-26f) {
+          float zeta = (b - a) / (2.0f * cf);
           if (!(fabsf(zeta) < 1e18f)) zeta = copysignf(1e18f, zeta);      // huge or not finite: (almost) no rotation
           const float tf = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
-          const double t = (double)tf;
-          const double cs = fast_rsqrt(t * t + 1.0), sn = t * cs;
+          const float c32 = rsqrtf(fmaf(tf, tf, 1.0f)), s32 = tf * c32;
+          // (c32, s32) is a unit vector to ~1e-7; one Newton step on 1/sqrt(c^2 + s^2) in FP64 makes it one to ~1e-14
+          const double cd = (double)c32, sd = (double)s32;
+          const double scale = 1.5 - 0.5 * (cd * cd + sd * sd);
+          const double cs = cd * scale, sn = sd * scale;
 #pragma unroll
-          for (int tt = 0; tt < MAXQ / 8; ++tt) {
+          for (int tt = 0; tt < R; ++tt) {
             const int i = sub + 8 * tt;
             if (i < np) {
               Y[i][p] = cs * yp[tt] - sn * yq[tt];
@@ -347,10 +357,9 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
             }
           }
           if (sub == 0) {
-            // exact for the applied (cs, sn): |y_p'|^2 = cs^2 a - 2 cs sn c + sn^2 b, |y_q'|^2 = sn^2 a + 2 cs sn c + cs^2 b
-            lam[p] = cs * cs * a - 2.0 * cs * sn * c + sn * sn * b;
-            lam[q] = sn * sn * a + 2.0 * cs * sn * c + cs * cs * b;
-            const float cf = (float)c, cos2 = (cf / (float)a) * (cf / (float)b);
+            const float tc = tf * cf;                   // |y_p'|^2 = a - t c, |y_q'|^2 = b + t c for the exact rotation
+            lamf[p] = a - tc;
+            lamf[q] = b + tc;
             atomicMax(reinterpret_cast<unsigned int*>(&rotated[0]), __float_as_uint(fminf(cos2, 1.0f)));
           }
         }
@@ -1019,6 +1028,21 @@ int gram_parts(int64_t n_rows, int64_t* rows_per_part) {
   return (int)metis_ceil_div(n_rows, rpp);
 }
 
+void launch_jacobi(cudaStream_t s, const double* g, int n, int ld, float exit_cos2, double* evals, double* evecs) {
+  const int r = (n + (n & 1) + 7) / 8;
+  switch (r) {
+    case 1: jacobi_eig_kernel<1><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+    case 2: jacobi_eig_kernel<2><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+    case 3: jacobi_eig_kernel<3><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+    case 4: jacobi_eig_kernel<4><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+    case 5: jacobi_eig_kernel<5><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+    case 6: jacobi_eig_kernel<6><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+    case 7: jacobi_eig_kernel<7><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+    default: jacobi_eig_kernel<8><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+  }
+  METIS_COUNT_LAUNCH();
+}
+
 template <int NJ4>
 void launch_project(dim3 grid, cudaStream_t s, const __nv_bfloat16* x, int64_t cols, const int* idx, int n_s, int q,
                     const float* h, int rpp, float* mp) {
@@ -1115,7 +1139,14 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   {
     static bool attr = false;
     if (!attr) {
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
       METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 64)));
       METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 48)));
       METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
@@ -1195,7 +1226,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     int64_t rpp; const int parts = gram_parts(cols, &rpp);
     gram_kernel<<<parts, 256, 0, s>>>(m, cols, q, 1, cols, rpp, gram, nullptr); METIS_COUNT_LAUNCH();
     reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1, nullptr); METIS_COUNT_LAUNCH();
-    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, s>>>(gram1, q, q, 1e-8f, evals, evecs); METIS_COUNT_LAUNCH();
+    launch_jacobi(s, gram1, q, q, 1e-8f, evals, evecs);
   }
   right_basis_kernel<<<(unsigned)metis_ceil_div(cols, 64), 256, 0, s>>>(m, cols, q, k, evals, evecs, basis,
                                                                           full ? out->sigma : nullptr); METIS_COUNT_LAUNCH();
@@ -1245,7 +1276,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   if (!full) {
     // (7) Rayleigh-Ritz on C^T C (Gram partials came out of the broadcast pass), rotate both factors
     reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 128), 128, 0, sf>>>(gram_c, n_cta_c, kp * kp, gram1, nullptr); METIS_COUNT_LAUNCH();
-    jacobi_eig_kernel<<<1, 256, JACOBI_SMEM, sf>>>(gram1, k, kp, 1e-6f, evals2, evecs2); METIS_COUNT_LAUNCH();
+    launch_jacobi(sf, gram1, k, kp, 1e-6f, evals2, evecs2);
     right_rotate_kernel<<<n_cand, 256, 0, sf>>>(basis, cols, k, evecs2, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
     sign_fix_kernel<<<dim3(n_cand, k), 256, 0, sf>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2); METIS_COUNT_LAUNCH();
     left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 256, 0, sf>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
