@@ -150,7 +150,8 @@ int64_t metis_default_sample_count(int64_t rows, int32_t q);
  * by (seed, stream_id, row*cols + col), so both orientations use the same draw).
  * tscale == METIS_TSCALE_AMAX_SELF: tensor_scale <- amax(x)/2688 (1 if x == 0), written to both
  * outputs' tensor_scale; METIS_TSCALE_GIVEN: the outputs' tensor_scale already hold the value.
- * Requires cols % 16 == 0 (by cols), rows % 16 == 0 (by rows); tiled scales need % 64.
+ * Requires cols % 16 == 0, rows % 16 == 0 when blocks along rows are asked for, tiled scales need % 64 along
+ * their block axis, and ld % 8 == 0 (BF16) or ld % 4 == 0 (FP32) so that every row starts 16-byte aligned.
  * Workspace: metis_workspace_bytes(0, ...). */
 metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dtype, int64_t rows, int64_t cols,
                                     int64_t ld, int32_t rounding, uint64_t seed, uint32_t stream_id,

@@ -122,17 +122,23 @@ __device__ __forceinline__ uint32_t metis_e2m1x2_rne(float lo, float hi) {
   return out;
 }
 
-// stochastic rounding of y to E2M1 with a 16-bit draw: up iff frac * 65536 > u
+// stochastic rounding of y to E2M1 with a 16-bit draw: up iff frac * 65536 > u, frac = (a - lo)/(hi - lo).
+// For a >= 1 the E2M1 grid has one mantissa bit per binade, so lo is the top mantissa bit of a and frac is the
+// remaining 22 bits: frac * 65536 > u  <=>  (mantissa & 0x3FFFFF) > 64 u, an exact integer comparison.
+// Below 1 the grid is {0, 0.5, 1}: uniform step 0.5, all operations exact in binary32.
 __device__ __forceinline__ uint32_t metis_e2m1_sr(float y, uint32_t u16) {
   const float a = fminf(fabsf(y), 6.0f);
   const uint32_t sign = (__float_as_uint(y) >> 28) & 8u;
-  int lo_c = (a >= 0.5f) + (a >= 1.0f) + (a >= 1.5f) + (a >= 2.0f) + (a >= 3.0f) + (a >= 4.0f) + (a >= 6.0f);
-  if (lo_c == 7) return sign | 7u;
-  const float lo = lo_c < 4 ? 0.5f * (float)lo_c : (lo_c == 4 ? 2.0f : lo_c == 5 ? 3.0f : 4.0f);
-  const float inv_step = lo_c < 4 ? 2.0f : (lo_c == 6 ? 0.5f : 1.0f);
-  const float f = __fmul_rn(__fsub_rn(a, lo), inv_step);
-  const uint32_t up = __fmul_rn(f, 65536.0f) > (float)u16 ? 1u : 0u;
-  return sign | (uint32_t)(lo_c + up);
+  const uint32_t bits = __float_as_uint(a);
+  if (bits >= 0x40C00000u) return sign | 7u;                       // a == 6 (saturated): no draw
+  if (bits >= 0x3F800000u) {                                       // 1 <= a < 6
+    const uint32_t e = (bits >> 23) - 127u, half = (bits >> 22) & 1u, frac22 = bits & 0x3FFFFFu;
+    return sign | (2u + 2u * e + half + (frac22 > (u16 << 6) ? 1u : 0u));
+  }
+  const float t2 = __fadd_rn(a, a);                                // a / 0.5, exact
+  const float fl = t2 >= 1.0f ? 1.0f : 0.0f;
+  const float fr = __fsub_rn(t2, fl);
+  return sign | ((uint32_t)fl + (__fmul_rn(fr, 65536.0f) > (float)u16 ? 1u : 0u));
 }
 
 // byte offset of scale (row r, block b) in the 128x4-tiled layout; blocks_per_row = k_len/16

@@ -40,45 +40,193 @@ __global__ void amax_kernel(const void* __restrict__ x, int dtype, int64_t rows,
   }
 }
 
-__global__ void __launch_bounds__(metis_qt::THREADS)
-quantize_kernel(const void* __restrict__ x, int dtype, int64_t ld, metis_qt::QuantParams p,
-                const float* __restrict__ tscale_src, int tscale_is_amax, float* ts_out0, float* ts_out1) {
+// Stand-alone quantizer, 128 x 128 elements per CTA.
+//  pass 1  every thread loads 16 consecutive elements of a row (32 bytes of BF16) - exactly one block along the
+//          columns - and, if that orientation is wanted, encodes it in registers and writes its 8 code bytes
+//          straight to global memory (8 threads = 64 contiguous bytes of a row); the values (BF16 or FP32) and
+//          the stochastic-rounding draws go to shared memory for pass 2
+//  pass 2  blocks along the rows: a thread reads 16 values down a column from shared memory, encodes them and
+//          stages the bytes; the transposed codes and both scale tiles are then written out coalesced
+template <typename T>   // T = __nv_bfloat16 or float: element type of the shared tile (= input type)
+__global__ void __launch_bounds__(metis_qt::THREADS, 2)
+quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, const float* __restrict__ tscale_src,
+                int tscale_is_amax, float* ts_out0, float* ts_out1) {
   using namespace metis_qt;
+  constexpr int TP = TILE + (sizeof(T) == 2 ? 2 : 1);            // tile pitch in elements (odd word stride)
   extern __shared__ __align__(16) unsigned char smem[];
-  float* tile = reinterpret_cast<float*>(smem);
-  Stage* stage = reinterpret_cast<Stage*>(smem + sizeof(float) * TILE * PITCH);
-  uint16_t* rnd = reinterpret_cast<uint16_t*>(smem + sizeof(float) * TILE * PITCH + sizeof(Stage));
+  T* tile = reinterpret_cast<T*>(smem);                                        // [TILE][TP]
+  Stage* stage = reinterpret_cast<Stage*>(smem + ((sizeof(T) * TILE * TP + 15) & ~(size_t)15));
+  uint8_t* sfc = reinterpret_cast<uint8_t*>(stage + 1);                        // [TILE][8] scales of the column blocks
+  uint16_t* rnd = reinterpret_cast<uint16_t*>(sfc + TILE * 8);                 // [TILE][TILE] draws (SR only)
 
+  const int tid = threadIdx.x;
   const int64_t row0 = (int64_t)blockIdx.y * TILE, col0 = (int64_t)blockIdx.x * TILE;
   const float s_T = tscale_is_amax ? metis_tensor_scale(*tscale_src) : *tscale_src;
-  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+  const float six_s_T = __fmul_rn(6.0f, s_T);
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
     if (ts_out0 != nullptr && ts_out0 != tscale_src) *ts_out0 = s_T;
     if (ts_out1 != nullptr && ts_out1 != tscale_src) *ts_out1 = s_T;
   }
-  const int tid = threadIdx.x;
-  // load the tile (zero fill outside the matrix), 8 elements per step
-  for (int i = tid; i < TILE * (TILE / 8); i += THREADS) {
-    const int r = i >> 4, g = i & 15;
-    const int64_t gr = row0 + r, gc = col0 + g * 8;
-    float v[8];
-    if (gr < p.rows && gc + 8 <= p.cols && dtype == METIS_BF16 && (ld & 7) == 0) {
-      const uint4 q = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(x) + gr * ld + gc);
-      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+  const bool sr = p.rounding == METIS_ROUND_SR;
+  const bool want_c = p.c_codes != nullptr, want_r = p.r_codes != nullptr;
+  const int vrows = (int)min((int64_t)TILE, p.rows - row0), vcols = (int)min((int64_t)TILE, p.cols - col0);
+  const bool fast_draws = p.e_stride_c == 1 && (p.e_stride_r & 7) == 0;
+
+  // ---- pass 1 ----
+  // all global loads of the tile are issued before the first block is encoded: 128 bytes per thread in flight
+  uint4 raw[sizeof(T) == 2 ? 8 : 1];
+  if (sizeof(T) == 2) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        v[2 * j] = __uint_as_float(w[j] << 16);
-        v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+    for (int it = 0; it < 4; ++it) {
+      const int b = tid & 7, r = (tid >> 3) + 32 * it;
+      raw[2 * it] = raw[2 * it + 1] = make_uint4(0u, 0u, 0u, 0u);
+      if (r < vrows && b * 16 < vcols) {
+        const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(x) + (row0 + r) * ld + col0 + b * 16);
+        raw[2 * it] = src[0]; raw[2 * it + 1] = src[1];
+      }
+    }
+  }
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int b = tid & 7, r = (tid >> 3) + 32 * it;
+    const int64_t gr = row0 + r, gc = col0 + b * 16;
+    const bool in = r < vrows && b * 16 < vcols;
+    float v[16];
+    uint32_t u[16];
+    if (sizeof(T) == 2) {
+      const uint4 q0 = raw[sizeof(T) == 2 ? 2 * it : 0], q1 = raw[sizeof(T) == 2 ? 2 * it + 1 : 0];
+      const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { v[2 * j] = __uint_as_float(w[j] << 16); v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u); }
+      if (want_r) {
+        uint32_t* dst = reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(tile) + r * TP + b * 16);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) dst[j] = w[j];
+      }
+    } else if (in) {
+      const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(x) + gr * ld + gc);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { const float4 q = src[j]; v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w; }
+      if (want_r) {
+        float* dst = reinterpret_cast<float*>(tile) + r * TP + b * 16;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) dst[j] = v[j];
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) v[j] = (gr < p.rows && gc + j < p.cols) ? metis_ld_as_float(x, dtype, gr * ld + gc + j) : 0.0f;
+      for (int j = 0; j < 16; ++j) v[j] = 0.0f;
+      if (want_r) {
+        T* dst = tile + r * TP + b * 16;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) dst[j] = T(0.0f);
+      }
     }
-    *reinterpret_cast<float4*>(tile + r * PITCH + g * 8) = make_float4(v[0], v[1], v[2], v[3]);
-    *reinterpret_cast<float4*>(tile + r * PITCH + g * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+    if (sr) {
+      if (fast_draws && in) {
+        const uint64_t e = (uint64_t)gr * (uint64_t)p.e_stride_r + (uint64_t)gc;
+        const uint4 w0 = metis_philox_block(e >> 3, p.seed, p.stream_id), w1 = metis_philox_block((e >> 3) + 1, p.seed, p.stream_id);
+        const uint32_t ww[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { u[2 * j] = ww[j] & 0xFFFFu; u[2 * j + 1] = ww[j] >> 16; }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          u[j] = in ? metis_draw_u16((uint64_t)gr * (uint64_t)p.e_stride_r + (uint64_t)(gc + j) * (uint64_t)p.e_stride_c, p.seed, p.stream_id) : 0u;
+      }
+      if (want_r) {
+        uint32_t* dst = reinterpret_cast<uint32_t*>(rnd + r * TILE + b * 16);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) dst[j] = u[2 * j] | (u[2 * j + 1] << 16);
+      }
+    }
+    if (want_c) {
+      uint32_t packed[2];
+      const uint32_t byte = encode_block(v, u, sr, s_T, six_s_T, packed);
+      if (in) *reinterpret_cast<uint2*>(p.c_codes + gr * (p.cols / 2) + gc / 2) = make_uint2(packed[0], packed[1]);
+      sfc[r * 8 + b] = in ? (uint8_t)byte : (uint8_t)0;
+    }
   }
-  if (p.rounding == METIS_ROUND_SR) fill_draws(rnd, p, row0, col0);
   __syncthreads();
-  quantize_tile(tile, rnd, stage, p, row0, col0, s_T);
+  // ---- pass 2 ----
+  if (want_r) {
+    if (sizeof(T) == 2) {
+      // BF16 tile: a thread takes two adjacent columns (one 32-bit shared load per row) and four of the eight
+      // row blocks, i.e. eight blocks in two rounds of four
+#pragma unroll 1
+      for (int it = 0; it < 2; ++it) {
+        const int c = (tid & 63) * 2, b = (tid >> 6) + 4 * it;
+        float v0[16], v1[16];
+        uint32_t u0[16], u1[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const uint32_t w = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const __nv_bfloat16*>(tile) + (b * 16 + i) * TP + c);
+          v0[i] = __uint_as_float(w << 16); v1[i] = __uint_as_float(w & 0xFFFF0000u);
+        }
+        if (sr) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(rnd + (b * 16 + i) * TILE + c);
+            u0[i] = w & 0xFFFFu; u1[i] = w >> 16;
+          }
+        }
+        uint32_t packed[2];
+        uint32_t byte = encode_block(v0, u0, sr, s_T, six_s_T, packed);
+        *reinterpret_cast<uint2*>(&stage->codes[c][b * 8]) = make_uint2(packed[0], packed[1]);
+        stage->sf[c][b] = (uint8_t)byte;
+        byte = encode_block(v1, u1, sr, s_T, six_s_T, packed);
+        *reinterpret_cast<uint2*>(&stage->codes[c + 1][b * 8]) = make_uint2(packed[0], packed[1]);
+        stage->sf[c + 1][b] = (uint8_t)byte;
+      }
+    } else {
+#pragma unroll 1
+    for (int it = 0; it < 4; ++it) {
+      const int c = tid & 127, b = (tid >> 7) + 2 * it;
+      float v[16];
+      uint32_t u[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) v[i] = reinterpret_cast<const float*>(tile)[(b * 16 + i) * TP + c];
+      if (sr) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) u[i] = rnd[(b * 16 + i) * TILE + c];
+      }
+      uint32_t packed[2];
+      const uint32_t byte = encode_block(v, u, sr, s_T, six_s_T, packed);
+      *reinterpret_cast<uint2*>(&stage->codes[c][b * 8]) = make_uint2(packed[0], packed[1]);
+      stage->sf[c][b] = (uint8_t)byte;
+    }
+    }
+    __syncthreads();
+    const int64_t kbytes = p.rows / 2;
+    for (int i = tid; i < TILE * 8; i += THREADS) {
+      const int c = i >> 3, seg = i & 7;
+      if (c < vcols && seg * 16 < vrows)
+        *reinterpret_cast<uint2*>(p.r_codes + (col0 + c) * kbytes + row0 / 2 + seg * 8) = *reinterpret_cast<const uint2*>(&stage->codes[c][seg * 8]);
+    }
+    const int64_t bpr = p.rows / 16;
+    for (int i = tid; i < TILE * 8; i += THREADS) {
+      int c, b;
+      if (p.r_layout == METIS_SF_TILED) { const int atom = i >> 9, w = i & 511; c = (w >> 4) + 32 * ((w >> 2) & 3); b = atom * 4 + (w & 3); }
+      else { c = i >> 3; b = i & 7; }
+      if (b * 16 < vrows && (c < vcols || p.r_layout == METIS_SF_TILED))
+        p.r_scales[metis_sf_offset(col0 + c, row0 / 16 + b, bpr, p.r_layout)] = c < vcols ? stage->sf[c][b] : (uint8_t)0;
+    }
+  }
+  if (want_c) {
+    const int64_t bpr = p.cols / 16;
+    for (int i = tid; i < TILE * 8; i += THREADS) {
+      int r, b;
+      if (p.c_layout == METIS_SF_TILED) { const int atom = i >> 9, w = i & 511; r = (w >> 4) + 32 * ((w >> 2) & 3); b = atom * 4 + (w & 3); }
+      else { r = i >> 3; b = i & 7; }
+      if (b * 16 < vcols && (r < vrows || p.c_layout == METIS_SF_TILED))
+        p.c_scales[metis_sf_offset(row0 + r, col0 / 16 + b, bpr, p.c_layout)] = r < vrows ? sfc[r * 8 + b] : (uint8_t)0;
+    }
+  }
+}
+
+template <typename T>
+constexpr size_t quantize_smem(bool sr) {
+  return ((sizeof(T) * metis_qt::TILE * (metis_qt::TILE + (sizeof(T) == 2 ? 2 : 1)) + 15) & ~(size_t)15) + sizeof(metis_qt::Stage) +
+         metis_qt::TILE * 8 + (sr ? sizeof(uint16_t) * metis_qt::TILE * metis_qt::TILE : 0);
 }
 
 }  // namespace
@@ -100,22 +248,29 @@ metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int
                                      const metis_nvfp4_t* by_rows, cudaStream_t s) {
   using namespace metis_qt;
   if (rows == 0 || cols == 0) return METIS_OK;
+  // vector loads of 16 elements per thread: the rows must start on 16-byte boundaries
+  if (cols % 16 || (dtype == METIS_BF16 ? ld % 8 : ld % 4)) return METIS_ERR_ALIGNMENT;
   QuantParams p{};
   p.rows = rows; p.cols = cols; p.rounding = rounding; p.seed = seed; p.stream_id = stream_id;
   p.e_stride_r = e_stride_r; p.e_stride_c = e_stride_c;
   if (by_cols) { p.c_codes = by_cols->codes; p.c_scales = by_cols->scales; p.c_layout = by_cols->sf_layout; }
   if (by_rows) { p.r_codes = by_rows->codes; p.r_scales = by_rows->scales; p.r_layout = by_rows->sf_layout; }
   const bool sr = rounding == METIS_ROUND_SR;
-  const size_t smem = smem_bytes(sr);
-  static bool attr_set[2] = {false, false};
-  if (!attr_set[sr]) {
-    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
-    attr_set[0] = attr_set[1] = true;
+  static bool attr_set = false;
+  if (!attr_set) {
+    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<__nv_bfloat16>(true)));
+    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<float>(true)));
+    attr_set = true;
   }
   dim3 grid((unsigned)metis_ceil_div(cols, TILE), (unsigned)metis_ceil_div(rows, TILE));
-  quantize_kernel<<<grid, THREADS, smem, s>>>(x, dtype, ld, p, tscale_src, tscale_is_amax,
-                                              by_cols ? by_cols->tensor_scale : nullptr,
-                                              by_rows ? by_rows->tensor_scale : nullptr); METIS_COUNT_LAUNCH();
+  float* t0 = by_cols ? by_cols->tensor_scale : nullptr; float* t1 = by_rows ? by_rows->tensor_scale : nullptr;
+  if (dtype == METIS_BF16)
+    quantize_kernel<__nv_bfloat16><<<grid, THREADS, quantize_smem<__nv_bfloat16>(sr), s>>>(
+        reinterpret_cast<const __nv_bfloat16*>(x), ld, p, tscale_src, tscale_is_amax, t0, t1);
+  else
+    quantize_kernel<float><<<grid, THREADS, quantize_smem<float>(sr), s>>>(reinterpret_cast<const float*>(x), ld, p, tscale_src,
+                                                                          tscale_is_amax, t0, t1);
+  METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }
