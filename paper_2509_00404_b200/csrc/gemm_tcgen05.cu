@@ -166,7 +166,6 @@ struct GemmArgs {
   void* d; int d_dtype; int64_t ldd;
   int M, N, K;
   uint32_t* dev_status;
-  int dbg;
   int extra_kb;            // BF16 correction boxes (64 elements of K each) appended after the FP4 K loop
 };
 
@@ -252,13 +251,9 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
           const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
-          const bool skip_tiles = (g.dbg & 4) && kb >= C::STAGES;
-          const uint32_t bytes = (skip_tiles ? 0u : (uint32_t)(C::A_BYTES + C::B_BYTES)) + (uint32_t)atoms * 512u * (1 + C::N_TILES_SF);
-          mbar_expect_tx(full_bar(s), bytes);
-          if (!skip_tiles) {
+          mbar_expect_tx(full_bar(s), (uint32_t)(C::A_BYTES + C::B_BYTES) + (uint32_t)atoms * 512u * (1 + C::N_TILES_SF));
           tma_load_2d(a_addr(s), &map_a, kb * (BLOCK_K / 2), mb * BLOCK_M, full_bar(s));
           tma_load_2d(b_addr(s), &map_b, kb * (BLOCK_K / 2), nb * BLOCK_N, full_bar(s));
-          }
           bulk_load(sfa_addr(s), g.a_sf + ((size_t)mb * sf_k_atoms + (size_t)kb * K_STEPS) * 512, atoms * 512, full_bar(s));
 #pragma unroll
           for (int t = 0; t < C::N_TILES_SF; ++t)
@@ -288,7 +283,6 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
           const uint32_t sfa_t = tmem_base + C::SF_COL0 + s * C::SF_COLS_PER_STAGE;
           const uint32_t sfb_t = sfa_t + 4 * K_STEPS;
-          if (!(g.dbg & 1) || kb == 0)
           for (int k = 0; k < atoms; ++k) {
             tc_cp_sf(sfa_t + 4 * k, make_smem_desc(sfa_addr(s) + k * 512, 128, SWIZZLE_NONE));
 #pragma unroll
@@ -296,7 +290,6 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
               tc_cp_sf(sfb_t + 4 * (k * C::N_TILES_SF + t),
                        make_smem_desc(sfb_addr(s) + (t * K_STEPS + k) * 512, 128, SWIZZLE_NONE));
           }
-          if (!(g.dbg & 2) || kb == 0)
           for (int k = 0; k < atoms; ++k) {
             const uint64_t a_desc = make_smem_desc(a_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
             const uint64_t b_desc = make_smem_desc(b_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
@@ -324,7 +317,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const int row = mb * BLOCK_M + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BLOCK_N && !(g.dbg & 8); c0 += 32) {
+      for (int c0 = 0; c0 < BLOCK_N; c0 += 32) {
         uint32_t r[32];
         tc_ld32(t_row + c0, r);
         const int col = nb * BLOCK_N + c0;
@@ -353,10 +346,12 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 // =================================================================================================
 // Two-CTA variant (cta_group::2): a cluster of two CTAs on neighbouring SMs computes one 256 x 256 tile.
 // Each CTA loads 128 rows of A and 128 rows of B per K block (the pair's MMA reads both halves of B),
-// its own 128 rows of A scales and the scales of all 256 B rows; the leader CTA issues the MMAs for both,
-// each CTA keeps its 128 x 256 half of the accumulator in its own tensor memory and runs its own epilogue.
-// Per stage a CTA brings in 38 KiB for 4 x (128 x 256 x 64) of tensor work - four times the work per byte
-// of the one-CTA kernel, which is what lets a five-stage ring cover the load + scale-copy + MMA latency.
+// its own 128 rows of A scales and the scales of all 256 B rows; the leader CTA issues the scale copies and
+// the MMAs for both, each CTA keeps its 128 x 256 half of the accumulator in its own tensor memory and runs
+// its own epilogue.  All loads of a stage, code tiles and scale atoms alike, are TMA tensor copies in the
+// cta_group::2 form that credit the LEADER's barrier, so a stage costs two barrier hand-offs in all
+// (slot free -> producer, data landed -> MMA issuer): the ring of five 38 KiB stages has to cover that
+// round trip, and it is this latency, not the tensor pipe, that bounds the kernel.
 // =================================================================================================
 namespace two_cta {
 
@@ -372,7 +367,7 @@ constexpr int SF_COLS_PER_STAGE = 4 * K_STEPS * 3;          // 16 (A) + 32 (B): 
 constexpr int SF_COL0 = 256;
 constexpr int TMEM_COLS = 512;
 static_assert(ACC_COLS + STAGES * SF_COLS_PER_STAGE <= TMEM_COLS, "tensor memory budget");
-constexpr int NUM_THREADS = 384;                            // producer, MMA, relay, scale copier, 8 epilogue warps
+constexpr int NUM_THREADS = 384;                            // producer, MMA issuer, two idle warps, 8 epilogue warps
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
 
 __device__ __forceinline__ uint32_t cluster_rank() {
@@ -389,6 +384,24 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t local_bar, uint32_t 
       "{ .reg .b32 ra; mapa.shared::cluster.u32 ra, %0, %1;\n"
       "  mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra]; }"
       ::"r"(local_bar), "r"(rank) : "memory");
+}
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(pred));
+  return pred != 0;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+// Tensor load into THIS CTA's shared memory whose byte count is credited to a barrier that may live in the
+// pair's other CTA (cta_group::2 form; no multicast): both CTAs of a pair report to the leader's barrier.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t cluster_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -447,6 +460,7 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int m, int n) {
 // layer, pre-divided by alpha) into the same FP32 accumulator.
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                       const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
                        const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUtensorMap map_r, GemmArgs g) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -457,13 +471,11 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   auto sfa_addr = [&](int s) { return b_addr(s) + B_BYTES; };
   auto sfb_addr = [&](int s) { return sfa_addr(s) + SFA_BYTES; };
   const uint32_t bar_base = base + (uint32_t)STAGES * STAGE_BYTES;
-  auto full_bar = [&](int s) { return bar_base + 8u * s; };                  // own loads landed (per CTA)
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };                  // leader only: both CTAs' loads landed
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };      // slot free (per CTA, by commit multicast)
-  auto ready_bar = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };  // leader only: both CTAs' loads landed
-  const uint32_t tfull_bar = bar_base + 8u * (3 * STAGES);                   // accumulator complete (per CTA)
-  const uint32_t tempty_bar = bar_base + 8u * (3 * STAGES + 1);              // leader only: both epilogues drained
-  auto sfready_bar = [&](int s) { return bar_base + 8u * (3 * STAGES + 2 + s); };   // leader only: scales are in tensor memory
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + (size_t)STAGES * STAGE_BYTES + 8 * (4 * STAGES + 2));
+  const uint32_t tfull_bar = bar_base + 8u * (2 * STAGES);                   // accumulator complete (per CTA)
+  const uint32_t tempty_bar = bar_base + 8u * (2 * STAGES + 1);              // leader only: both epilogues drained
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + (size_t)STAGES * STAGE_BYTES + 8 * (2 * STAGES + 2));
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -477,9 +489,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   const int sf_k_atoms = g.K / MMA_K;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); mbar_init(ready_bar(s), 2); mbar_init(sfready_bar(s), 1);
-    }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(tfull_bar, 1);
     mbar_init(tempty_bar, 16);                                // 8 epilogue warps in each of the two CTAs
     *dead = 0;
@@ -494,56 +504,51 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 
   if (warp == 0) {
     // ------------------------------- producer (both CTAs) -------------------
-    if (lane == 0) {
+    // The leader announces the bytes of BOTH CTAs on its barrier; the other CTA only issues its loads.  A load
+    // of the other CTA may land before the announcement: the count just goes negative for a moment, and the
+    // phase cannot complete before the leader's arrival.  Every box is delivered in full (rows or K beyond
+    // the matrix are filled with zeros), so the byte count of a stage does not depend on the position.
+    // The whole warp walks the loop so that every address stays warp-uniform; one elected lane issues.
+    {
       int s = 0; uint32_t ph = 0;
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
         const int mb = tile % num_m, nb = tile / num_m;
         const int a_row = mb * TILE_M + (int)rank * 128, b_row = nb * TILE_N + (int)rank * 128;
-        // a 128-row slab that lies wholly outside the matrix has all-zero codes (TMA fill); any valid slab's
-        // scales will do for it, so the index is clamped instead of reading past the scale buffer
+        // a 128-row slab that lies wholly outside the matrix has all-zero codes; any valid slab's scales will
+        // do for it, so the index is clamped instead of reading another tensor's bytes
         const int a_sf_tile = min(mb * 2 + (int)rank, (g.M + 127) / 128 - 1);
+        const int b_sf_tile0 = min(nb * 2, (g.N + 127) / 128 - 1), b_sf_tile1 = min(nb * 2 + 1, (g.N + 127) / 128 - 1);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
-          if (kb >= num_fp4_kb) {                             // BF16 correction box: 128 rows x 64 elements each
-            mbar_expect_tx(full_bar(s), (uint32_t)(A_BYTES + B_BYTES));
-            tma_load_2d(a_addr(s), &map_l, (kb - num_fp4_kb) * 64, a_row, full_bar(s));
-            tma_load_2d(b_addr(s), &map_r, (kb - num_fp4_kb) * 64, b_row, full_bar(s));
-            if (++s == STAGES) { s = 0; ph ^= 1u; }
-            continue;
+          if (elect_one()) {
+            const uint32_t bar = map_to_rank(full_bar(s), 0u);
+            if (kb >= num_fp4_kb) {                           // BF16 correction box: 128 rows x 64 elements each
+              if (leader) mbar_expect_tx(full_bar(s), 2u * (uint32_t)(A_BYTES + B_BYTES));
+              tma_load_2d_pair(a_addr(s), &map_l, (kb - num_fp4_kb) * 64, a_row, bar);
+              tma_load_2d_pair(b_addr(s), &map_r, (kb - num_fp4_kb) * 64, b_row, bar);
+            } else {
+              if (leader) mbar_expect_tx(full_bar(s), 2u * (uint32_t)STAGE_BYTES);
+              tma_load_2d_pair(a_addr(s), &map_a, kb * (BLOCK_K / 2), a_row, bar);
+              tma_load_2d_pair(b_addr(s), &map_b, kb * (BLOCK_K / 2), b_row, bar);
+              tma_load_2d_pair(sfa_addr(s), &map_sfa, 0, a_sf_tile * sf_k_atoms + kb * K_STEPS, bar);
+              tma_load_2d_pair(sfb_addr(s), &map_sfb, 0, b_sf_tile0 * sf_k_atoms + kb * K_STEPS, bar);
+              tma_load_2d_pair(sfb_addr(s) + K_STEPS * 512, &map_sfb, 0, b_sf_tile1 * sf_k_atoms + kb * K_STEPS, bar);
+            }
           }
-          const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
-          mbar_expect_tx(full_bar(s), (((g.dbg & 4) && kb >= STAGES) ? 0u : (uint32_t)(A_BYTES + B_BYTES)) + (uint32_t)atoms * 512u * 3u);
-          if (!((g.dbg & 4) && kb >= STAGES)) {
-          tma_load_2d(a_addr(s), &map_a, kb * (BLOCK_K / 2), a_row, full_bar(s));
-          tma_load_2d(b_addr(s), &map_b, kb * (BLOCK_K / 2), b_row, full_bar(s));
-          }
-          bulk_load(sfa_addr(s), g.a_sf + ((size_t)a_sf_tile * sf_k_atoms + (size_t)kb * K_STEPS) * 512, atoms * 512, full_bar(s));
-#pragma unroll
-          for (int t = 0; t < 2; ++t)
-            bulk_load(sfb_addr(s) + t * K_STEPS * 512,
-                      g.b_sf + ((size_t)min(nb * 2 + t, (g.N + 127) / 128 - 1) * sf_k_atoms + (size_t)kb * K_STEPS) * 512,
-                      atoms * 512, full_bar(s));
-          if (++s == STAGES) { s = 0; ph ^= 1u; }
-        }
-      }
-    }
-  } else if (warp == 2) {
-    // ------------------------------- relay (both CTAs): own stage landed -> tell the leader ----
-    if (lane == 0) {
-      int s = 0; uint32_t ph = 0;
-      bool ok = true;
-      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-        for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(full_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
-          mbar_arrive_remote(ready_bar(s), 0u);
+          __syncwarp();
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------- MMA issuer (leader CTA only) ------------
-    if (leader && lane == 0) {
+    // ------------------------------- scale copies + MMA issue (leader CTA only) ------------
+    // tcgen05.cp and tcgen05.mma issued by one thread execute in order, so the scale atoms of a stage are
+    // copied shared -> tensor memory right in front of the MMAs that read them.  Each ring stage has its own
+    // scale columns; they are rewritten only after the MMAs of the stage's previous use have completed (the
+    // stage is reloaded only after the commit that frees it).
+    if (leader) {
+      // the whole warp walks the loop (so that addresses and descriptors stay warp-uniform); one elected lane issues
       constexpr uint32_t idesc = make_idesc(TILE_M, TILE_N);
       int s = 0; uint32_t ph = 0;
       int it = 0;
@@ -552,58 +557,49 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         if (!mbar_wait_cluster(tempty_bar, ((uint32_t)it & 1u) ^ 1u, g.dev_status, dead)) { ok = false; break; }
         tc_fence_after();
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(sfready_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
+          if (!mbar_wait_cluster(full_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
           tc_fence_after();
-          if (kb >= num_fp4_kb) {
-            constexpr uint32_t idesc_x = make_idesc_bf16(TILE_M, TILE_N);
+          if (elect_one()) {
+            if (kb >= num_fp4_kb) {
+              constexpr uint32_t idesc_x = make_idesc_bf16(TILE_M, TILE_N);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {                     // 64 BF16 elements = four K=16 MMAs, 32 bytes apart
-              const uint64_t a_desc = make_smem_desc(a_addr(s) + k * 32, 1024, SWIZZLE_128B);
-              const uint64_t b_desc = make_smem_desc(b_addr(s) + k * 32, 1024, SWIZZLE_128B);
-              tc_mma_bf16_2(tmem_base, a_desc, b_desc, idesc_x, 1u);
+              for (int k = 0; k < 4; ++k) {                   // 64 BF16 elements = four K=16 MMAs, 32 bytes apart
+                const uint64_t a_desc = make_smem_desc(a_addr(s) + k * 32, 1024, SWIZZLE_128B);
+                const uint64_t b_desc = make_smem_desc(b_addr(s) + k * 32, 1024, SWIZZLE_128B);
+                tc_mma_bf16_2(tmem_base, a_desc, b_desc, idesc_x, 1u);
+              }
+            } else {
+              const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
+              const uint32_t sfa_t = tmem_base + SF_COL0 + s * SF_COLS_PER_STAGE, sfb_t = sfa_t + 4 * K_STEPS;
+              const uint64_t sfa_d = make_smem_desc(sfa_addr(s), 128, SWIZZLE_NONE), sfb_d = make_smem_desc(sfb_addr(s), 128, SWIZZLE_NONE);
+              const uint64_t a_d = make_smem_desc(a_addr(s), 1024, SWIZZLE_128B), b_d = make_smem_desc(b_addr(s), 1024, SWIZZLE_128B);
+              if (atoms == K_STEPS) {
+#pragma unroll
+                for (int k = 0; k < K_STEPS; ++k) {
+                  tc_cp_sf2(sfa_t + 4 * k, sfa_d + (uint64_t)(k * 32));
+                  tc_cp_sf2(sfb_t + 8 * k, sfb_d + (uint64_t)(k * 32));
+                  tc_cp_sf2(sfb_t + 8 * k + 4, sfb_d + (uint64_t)((K_STEPS + k) * 32));
+                }
+#pragma unroll
+                for (int k = 0; k < K_STEPS; ++k)
+                  tc_mma_nvf4_2(tmem_base, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc, sfa_t + 4 * k, sfb_t + 8 * k, (kb | k) != 0 ? 1u : 0u);
+              } else {
+                for (int k = 0; k < atoms; ++k) {
+                  tc_cp_sf2(sfa_t + 4 * k, sfa_d + (uint64_t)(k * 32));
+                  tc_cp_sf2(sfb_t + 8 * k, sfb_d + (uint64_t)(k * 32));
+                  tc_cp_sf2(sfb_t + 8 * k + 4, sfb_d + (uint64_t)((K_STEPS + k) * 32));
+                }
+                for (int k = 0; k < atoms; ++k)
+                  tc_mma_nvf4_2(tmem_base, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc, sfa_t + 4 * k, sfb_t + 8 * k, (kb | k) != 0 ? 1u : 0u);
+              }
             }
-            tc_commit2(empty_bar(s), 3);
-            if (++s == STAGES) { s = 0; ph ^= 1u; }
-            continue;
+            tc_commit2(empty_bar(s), 3);                      // frees the slot in both CTAs
           }
-          const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
-          const uint32_t sfa_t = tmem_base + SF_COL0 + s * SF_COLS_PER_STAGE, sfb_t = sfa_t + 4 * K_STEPS;
-          if (!(g.dbg & 2) || kb == 0)
-          for (int k = 0; k < atoms; ++k) {
-            const uint64_t a_desc = make_smem_desc(a_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
-            const uint64_t b_desc = make_smem_desc(b_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
-            tc_mma_nvf4_2(tmem_base, a_desc, b_desc, idesc, sfa_t + 4 * k, sfb_t + 8 * k, (kb | k) != 0 ? 1u : 0u);
-          }
-          tc_commit2(empty_bar(s), 3);                        // frees the slot in both CTAs
+          __syncwarp();
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
-        if (ok) tc_commit2(tfull_bar, 3);                     // accumulator complete in both CTAs
-      }
-    }
-  } else if (warp == 3) {
-    // ------------------------------- scale copier (leader CTA only) ----------
-    // shared memory -> tensor memory copies of the scale atoms, issued from their own warp so they do not sit
-    // in the MMA issuer's instruction stream; a stage's columns are rewritten only after the MMAs that read them
-    // have completed (the stage is reloaded only after the commit that frees it)
-    if (leader && lane == 0) {
-      int s = 0; uint32_t ph = 0;
-      bool ok = true;
-      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-        for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait_cluster(ready_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
-          tc_fence_after();
-          const int atoms = kb < num_fp4_kb ? min(K_STEPS, sf_k_atoms - kb * K_STEPS) : 0;   // BF16 boxes carry no scales
-          const uint32_t sfa_t = tmem_base + SF_COL0 + s * SF_COLS_PER_STAGE, sfb_t = sfa_t + 4 * K_STEPS;
-          if (!(g.dbg & 1) || kb == 0)
-          for (int k = 0; k < atoms; ++k) {
-            tc_cp_sf2(sfa_t + 4 * k, make_smem_desc(sfa_addr(s) + k * 512, 128, SWIZZLE_NONE));
-#pragma unroll
-            for (int t = 0; t < 2; ++t)
-              tc_cp_sf2(sfb_t + 4 * (k * 2 + t), make_smem_desc(sfb_addr(s) + (t * K_STEPS + k) * 512, 128, SWIZZLE_NONE));
-          }
-          tc_commit2(sfready_bar(s), 1);
-          if (++s == STAGES) { s = 0; ph ^= 1u; }
-        }
+        if (ok && elect_one()) tc_commit2(tfull_bar, 3);      // accumulator complete in both CTAs
+        __syncwarp();
       }
     }
   } else if (warp >= 4) {
@@ -622,22 +618,18 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       const int row = mb * TILE_M + (int)rank * 128 + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 128);
       uint32_t r[4][32];
-      if (!(g.dbg & 8)) {
-        tc_ld32_nowait(t_row, r[0]);
-        tc_ld32_nowait(t_row + 32, r[1]);
-        tc_ld32_nowait(t_row + 64, r[2]);
-        tc_ld32_nowait(t_row + 96, r[3]);
-        tc_wait_ld();
-      }
+      tc_ld32_nowait(t_row, r[0]);
+      tc_ld32_nowait(t_row + 32, r[1]);
+      tc_ld32_nowait(t_row + 64, r[2]);
+      tc_ld32_nowait(t_row + 96, r[3]);
+      tc_wait_ld();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_remote(tempty_bar, 0u);
-      if (!(g.dbg & 8)) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int col = nb * TILE_N + half * 128 + c * 32;
-          if (row < g.M && col < g.N) store_row_chunk(g, row, col, r[c], alpha);
-        }
+      for (int c = 0; c < 4; ++c) {
+        const int col = nb * TILE_N + half * 128 + c * 32;
+        if (row < g.M && col < g.N) store_row_chunk(g, row, col, r[c], alpha);
       }
     }
   }
@@ -672,6 +664,20 @@ metis_status_t make_codes_map(metis_context* ctx, CUtensorMap* map, const metis_
   return r == CUDA_SUCCESS ? METIS_OK : METIS_ERR_CUDA;
 }
 
+// 2-D map over the tiled scale bytes of one NVFP4 tensor: one row per 512-byte atom (128 rows x 4 blocks),
+// atoms of one 128-row slab consecutive along K; a box is the K_STEPS atoms of one K block.
+metis_status_t make_scales_map(metis_context* ctx, CUtensorMap* map, const metis_nvfp4_t* t) {
+  const cuuint64_t atoms = (cuuint64_t)metis_ceil_div(t->rows, 128) * (cuuint64_t)(t->k_len / MMA_K);
+  const cuuint64_t dims[2] = {128, atoms};
+  const cuuint64_t strides[1] = {512};
+  const cuuint32_t box[2] = {128, (cuuint32_t)K_STEPS};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+      map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, t->scales, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+      CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? METIS_OK : METIS_ERR_CUDA;
+}
+
 template <int BLOCK_N>
 metis_status_t launch(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d, int d_dtype,
                       int64_t ldd, cudaStream_t s) {
@@ -684,7 +690,6 @@ metis_status_t launch(metis_context* ctx, const metis_nvfp4_t* a, const metis_nv
   g.d = d; g.d_dtype = d_dtype; g.ldd = ldd;
   g.M = (int)a->rows; g.N = (int)b->rows; g.K = (int)a->k_len;
   g.dev_status = ctx->dev_status;
-  { const char* e = getenv("METIS_GEMM_DBG"); g.dbg = e ? atoi(e) : 0; }
   static bool attr_set = false;
   if (!attr_set) {
     METIS_CUDA_TRY(cudaFuncSetAttribute(gemm_nvfp4_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
@@ -711,9 +716,11 @@ metis_status_t make_bf16_map(metis_context* ctx, CUtensorMap* map, const void* p
 
 metis_status_t launch_2cta(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d, int d_dtype,
                            int64_t ldd, const void* lx, const void* rx, int kx, cudaStream_t s) {
-  CUtensorMap map_a, map_b, map_l, map_r;
+  CUtensorMap map_a, map_b, map_sfa, map_sfb, map_l, map_r;
   METIS_TRY(make_codes_map(ctx, &map_a, a, 128));
   METIS_TRY(make_codes_map(ctx, &map_b, b, 128));
+  METIS_TRY(make_scales_map(ctx, &map_sfa, a));
+  METIS_TRY(make_scales_map(ctx, &map_sfb, b));
   if (kx > 0) {
     METIS_TRY(make_bf16_map(ctx, &map_l, lx, a->rows, kx));
     METIS_TRY(make_bf16_map(ctx, &map_r, rx, b->rows, kx));
@@ -725,7 +732,6 @@ metis_status_t launch_2cta(metis_context* ctx, const metis_nvfp4_t* a, const met
   g.d = d; g.d_dtype = d_dtype; g.ldd = ldd;
   g.M = (int)a->rows; g.N = (int)b->rows; g.K = (int)a->k_len;
   g.dev_status = ctx->dev_status;
-  { const char* e = getenv("METIS_GEMM_DBG"); g.dbg = e ? atoi(e) : 0; }
   g.extra_kb = kx / 64;
   static bool attr_set = false;
   if (!attr_set) {
@@ -746,7 +752,7 @@ metis_status_t launch_2cta(metis_context* ctx, const metis_nvfp4_t* a, const met
     max_pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
   }
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  two_cta::gemm_nvfp4_2cta_kernel<<<2 * pairs, two_cta::NUM_THREADS, two_cta::SMEM_BYTES, s>>>(map_a, map_b, map_l, map_r, g); METIS_COUNT_LAUNCH();
+  two_cta::gemm_nvfp4_2cta_kernel<<<2 * pairs, two_cta::NUM_THREADS, two_cta::SMEM_BYTES, s>>>(map_a, map_b, map_sfa, map_sfb, map_l, map_r, g); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }
