@@ -207,11 +207,21 @@ metis_status_t metis_linear_fwd_static_ws(metis_handle_t h, const metis_operand_
 
 /* dx (l x m) = Dq Wq' (Eq. 3; needs dy->res_by_cols, w->res_by_rows) and
  * dw (n x m) = Dq''^T Xq'' (weight gradient; needs dy->res_by_rows, x->res_by_rows).
- * Either output may be NULL to skip it. */
+ * Either output may be NULL to skip it.
+ *
+ * Factor gradients (Section 3.2, the derivatives that follow Eq. 3), optional, each may be NULL: with the
+ * weight operand W_t = left diag(sigma) right^T + Res (left = the paper's V, n x k; right = the paper's U,
+ * m x k) and dw as just computed,
+ *   d_left  (k x n, like w->left)   = sigma_t * sum_i dw[j][i] * right_q[t][i]      (the paper's dL/dV),
+ *   d_right (k x m, like w->right)  = sigma_t * sum_j dw[j][i] * left_q[t][j]       (the paper's dL/dU),
+ *   d_sigma (k)                     = sum_ij left_q[t][j] dw[j][i] right_q[t][i]    (diagonal of dL/dS),
+ * using the dequantized NVFP4 factors and FP32 accumulation in a fixed order.  The gradient of the residual
+ * W_R is dw itself.  They need dw and w non-NULL (else METIS_ERR_INVALID_ARG) and d_sigma needs d_left;
+ * dw is read back in the type it was written in. */
 metis_status_t metis_linear_bwd(metis_handle_t h, const metis_operand_t* dy, const metis_operand_t* x,
-                                const metis_operand_t* w, void* dx, int32_t dx_dtype, int64_t lddx,
-                                void* dw, int32_t dw_dtype, int64_t lddw, void* ws, size_t ws_bytes,
-                                metis_stream_t stream);
+                                const metis_operand_t* w, void* dx, int32_t dx_dtype, int64_t lddx, void* dw,
+                                int32_t dw_dtype, int64_t lddw, float* d_left, float* d_sigma, float* d_right,
+                                void* ws, size_t ws_bytes, metis_stream_t stream);
 
 /* Plain block-scaled FP4 GEMM on already quantized tensors: d (M x N, ldd) = a b^T * (a.ts * b.ts),
  * a: M x K, b: N x K, both K-major with METIS_SF_TILED scales.  Exposed for tests and benchmarks of

@@ -80,7 +80,7 @@ def lib():
     l.metis_linear_fwd.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp, sz, vp]
     l.metis_linear_fwd_static_ws.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp]
     l.metis_linear_bwd.argtypes = [vp, P(OperandStruct), P(OperandStruct), P(OperandStruct), vp, i32, i64, vp, i32,
-                                   i64, vp, sz, vp]
+                                   i64, vp, vp, vp, vp, sz, vp]
     l.metis_gemm_nvfp4.argtypes = [vp, P(NvFp4Struct), P(NvFp4Struct), vp, i32, i64, i32, vp]
     for name in EXPORTED:
         if name not in ("metis_sf_bytes", "metis_default_sample_count", "metis_debug_launch_count"):
@@ -291,7 +291,10 @@ class Handle:
             self._h, ctypes.byref(sx), ctypes.byref(sw), _ptr(y), _dtype_code(y), y.stride(0), _stream_ptr(stream)))
         return y
 
-    def linear_bwd(self, dy_op, x_op, w_op, out_dtype=torch.float32, need_dx=True, need_dw=True, out=None, stream=None):
+    def linear_bwd(self, dy_op, x_op, w_op, out_dtype=torch.float32, need_dx=True, need_dw=True, out=None, stream=None,
+                   factor_grads=None):
+        """dx, dw of the layer.  `factor_grads`: None, or a tuple (d_left, d_sigma, d_right) of FP32 CUDA tensors
+        (k x n, k, k x m; any of them None) that receive the gradients of the weight factors."""
         l, n, m = dy_op.rows, dy_op.cols, (x_op.cols if x_op is not None else w_op.cols)
         dx = dw = None
         if out is not None:
@@ -310,6 +313,7 @@ class Handle:
             self._h, ctypes.byref(sd), ctypes.byref(sx) if sx else None, ctypes.byref(sw) if sw else None,
             _ptr(dx), _dtype_code(dx) if dx is not None else FP32, dx.stride(0) if dx is not None else 0,
             _ptr(dw), _dtype_code(dw) if dw is not None else FP32, dw.stride(0) if dw is not None else 0,
+            *(_ptr(t) for t in (factor_grads or (None, None, None))),
             _ptr(ws), ws.numel(), _stream_ptr(stream)))
         return dx, dw
 

@@ -82,6 +82,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
   return false;
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+// true in exactly one lane of a fully converged warp
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
@@ -243,13 +249,14 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
   if (warp == 0) {
     // ------------------------------- producer -------------------------------
-    if (lane == 0) {
-      int s = 0; uint32_t ph = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int mb = tile % num_m, nb = tile / num_m;
-        for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
+    // (the whole warp walks the loop so that addresses stay warp-uniform; one elected lane issues)
+    int s = 0; uint32_t ph = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      const int mb = tile % num_m, nb = tile / num_m;
+      for (int kb = 0; kb < num_kb; ++kb) {
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
+        if (elect_one()) {
           const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
           mbar_expect_tx(full_bar(s), (uint32_t)(C::A_BYTES + C::B_BYTES) + (uint32_t)atoms * 512u * (1 + C::N_TILES_SF));
           tma_load_2d(a_addr(s), &map_a, kb * (BLOCK_K / 2), mb * BLOCK_M, full_bar(s));
@@ -260,47 +267,48 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             bulk_load(sfb_addr(s) + t * K_STEPS * 512,
                       g.b_sf + ((size_t)min(nb * C::N_TILES_SF + t, (g.N + 127) / 128 - 1) * sf_k_atoms + (size_t)kb * K_STEPS) * 512,
                       atoms * 512, full_bar(s));
-          if (++s == C::STAGES) { s = 0; ph ^= 1u; }
         }
+        __syncwarp();
+        if (++s == C::STAGES) { s = 0; ph ^= 1u; }
       }
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer -----------------------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
-      int s = 0; uint32_t ph = 0;
-      int it = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
-        const int acc = it % C::NUM_ACC;
-        const uint32_t acc_ph = (uint32_t)(it / C::NUM_ACC) & 1u;
-        if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
+    constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
+    int s = 0; uint32_t ph = 0;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      const int acc = it % C::NUM_ACC;
+      const uint32_t acc_ph = (uint32_t)(it / C::NUM_ACC) & 1u;
+      if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BLOCK_N);
+      for (int kb = 0; kb < num_kb; ++kb) {
+        if (!mbar_wait(full_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BLOCK_N);
-        for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(full_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
-          tc_fence_after();
+        if (elect_one()) {
           const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
           const uint32_t sfa_t = tmem_base + C::SF_COL0 + s * C::SF_COLS_PER_STAGE;
           const uint32_t sfb_t = sfa_t + 4 * K_STEPS;
+          const uint64_t sfa_d = make_smem_desc(sfa_addr(s), 128, SWIZZLE_NONE), sfb_d = make_smem_desc(sfb_addr(s), 128, SWIZZLE_NONE);
+          const uint64_t a_d = make_smem_desc(a_addr(s), 1024, SWIZZLE_128B), b_d = make_smem_desc(b_addr(s), 1024, SWIZZLE_128B);
           for (int k = 0; k < atoms; ++k) {
-            tc_cp_sf(sfa_t + 4 * k, make_smem_desc(sfa_addr(s) + k * 512, 128, SWIZZLE_NONE));
+            tc_cp_sf(sfa_t + 4 * k, sfa_d + (uint64_t)(k * 32));
 #pragma unroll
             for (int t = 0; t < C::N_TILES_SF; ++t)
-              tc_cp_sf(sfb_t + 4 * (k * C::N_TILES_SF + t),
-                       make_smem_desc(sfb_addr(s) + (t * K_STEPS + k) * 512, 128, SWIZZLE_NONE));
+              tc_cp_sf(sfb_t + 4 * (k * C::N_TILES_SF + t), sfb_d + (uint64_t)((t * K_STEPS + k) * 32));
           }
-          for (int k = 0; k < atoms; ++k) {
-            const uint64_t a_desc = make_smem_desc(a_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
-            const uint64_t b_desc = make_smem_desc(b_addr(s) + k * (MMA_K / 2), 1024, SWIZZLE_128B);
-            tc_mma_nvf4(d_tmem, a_desc, b_desc, idesc, sfa_t + 4 * k, sfb_t + 4 * k * C::N_TILES_SF,
+          for (int k = 0; k < atoms; ++k)
+            tc_mma_nvf4(d_tmem, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc, sfa_t + 4 * k, sfb_t + 4 * k * C::N_TILES_SF,
                         (kb | k) != 0 ? 1u : 0u);
-          }
           tc_commit(empty_bar(s));                           // slot reusable once these MMAs have read it
-          if (++s == C::STAGES) { s = 0; ph ^= 1u; }
         }
-        if (ok) tc_commit(tfull_bar(acc));                   // accumulator complete
+        __syncwarp();
+        if (++s == C::STAGES) { s = 0; ph ^= 1u; }
       }
+      if (ok && elect_one()) tc_commit(tfull_bar(acc));      // accumulator complete
+      __syncwarp();
     }
   } else {
     // ------------------------------- epilogue -------------------------------
@@ -384,11 +392,6 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t local_bar, uint32_t 
       "{ .reg .b32 ra; mapa.shared::cluster.u32 ra, %0, %1;\n"
       "  mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra]; }"
       ::"r"(local_bar), "r"(rank) : "memory");
-}
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(pred));
-  return pred != 0;
 }
 // shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {

@@ -129,6 +129,138 @@ rank_update_kernel(const float* __restrict__ y0, int64_t M, int64_t N, int kc, c
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Gradients of the weight factors (Section 3.2, the derivatives listed after Eq. 3).  With the weight gradient
+// G (n x m, FP32 or BF16, as produced by the wgrad product) and a dequantized factor F stored k x len:
+//   TRANS = 0:  out[t][r] = scale_t * sum_c G[r][c] F[t][c]      (r over n, c over m:  dL/dV from U)
+//   TRANS = 1:  out[t][r] = scale_t * sum_c G[c][r] F[t][c]      (r over m, c over n:  dL/dU from V)
+// scale_t = sigma_t.  One CTA owns 32 values of r and walks c in chunks of 32; FP32 FMAs, fixed summation
+// order (deterministic).  With `other` given (the factor lying along r), the CTA also writes its partial of
+//   dsigma[t] = sum_r other[t][r] * (sum_c ...)   to ds_part[blockIdx.x][t].
+constexpr int FG_ROWS = 32, FG_CHUNK = 32;
+template <int KT, bool TRANS>                           // KT = ceil(k / 8) outputs per thread
+__global__ void __launch_bounds__(256)
+factor_grad_kernel(const void* __restrict__ gsrc, int g_dtype, int64_t ldg, int64_t n_r, int64_t n_c, int k,
+                   const uint8_t* f_codes, const uint8_t* f_sf, int f_layout, const float* f_ts,
+                   const uint8_t* o_codes, const uint8_t* o_sf, int o_layout, const float* o_ts,
+                   const float* __restrict__ sigma, float* __restrict__ out, float* __restrict__ ds_part) {
+  __shared__ float gs[FG_ROWS][FG_CHUNK + 1];
+  __shared__ __align__(16) float fs[FG_CHUNK][8 * KT + 4];
+  __shared__ float red[8][8 * KT];
+  const int tid = threadIdx.x, r = tid >> 3, tg = tid & 7;
+  const int64_t r0 = (int64_t)blockIdx.x * FG_ROWS;
+  const float fts = *f_ts;
+  float acc[KT];
+#pragma unroll
+  for (int j = 0; j < KT; ++j) acc[j] = 0.0f;
+  for (int64_t c0 = 0; c0 < n_c; c0 += FG_CHUNK) {
+    // tile of G: element (rr, cc) of this chunk
+    for (int o = tid; o < FG_ROWS * FG_CHUNK; o += 256) {
+      const int a = o >> 5, b = o & 31;                 // b runs along the contiguous axis of G
+      const int rr = TRANS ? b : a, cc = TRANS ? a : b;
+      const int64_t gr = r0 + rr, gc = c0 + cc;
+      float v = 0.0f;
+      if (gr < n_r && gc < n_c) {
+        const int64_t off = TRANS ? gc * ldg + gr : gr * ldg + gc;
+        v = g_dtype == METIS_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(gsrc)[off])
+                                  : reinterpret_cast<const float*>(gsrc)[off];
+      }
+      gs[rr][cc] = v;
+    }
+    for (int o = tid; o < FG_CHUNK * 8 * KT; o += 256) {
+      const int t = o >> 5, cc = o & 31;
+      fs[cc][t] = (t < k && c0 + cc < n_c) ? deq_at(f_codes, f_sf, f_layout, n_c, t, c0 + cc) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int cc = 0; cc < FG_CHUNK; ++cc) {
+      const float gv = gs[r][cc];
+#pragma unroll
+      for (int j = 0; j < KT; ++j) acc[j] = fmaf(gv, fs[cc][tg * KT + j], acc[j]);
+    }
+    __syncthreads();
+  }
+  const int64_t gr = r0 + r;
+#pragma unroll
+  for (int j = 0; j < KT; ++j) {
+    const int t = tg * KT + j;
+    acc[j] *= fts;
+    if (t < k && gr < n_r) out[(int64_t)t * n_r + gr] = acc[j] * sigma[t];
+  }
+  if (ds_part != nullptr) {
+    const float ots = *o_ts;
+    // sum over the CTA's 32 rows in a fixed order: 4 rows per warp by shuffles, then 8 warps through shared memory
+#pragma unroll
+    for (int j = 0; j < KT; ++j) {
+      const int t = tg * KT + j;
+      float v = (t < k && gr < n_r) ? acc[j] * deq_at(o_codes, o_sf, o_layout, n_r, t, gr) * ots : 0.0f;
+      v += __shfl_xor_sync(0xFFFFFFFFu, v, 8);
+      v += __shfl_xor_sync(0xFFFFFFFFu, v, 16);
+      if ((tid & 31) < 8) red[tid >> 5][t] = v;
+    }
+    __syncthreads();
+    if (tid < k) {
+      float v = 0.0f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) v += red[w][tid];
+      ds_part[(int64_t)blockIdx.x * k + tid] = v;
+    }
+  }
+}
+
+// dsigma[t] = sum over the partials, in order
+__global__ void factor_grad_sigma_kernel(const float* __restrict__ part, int n_part, int k, float* __restrict__ ds) {
+  const int t = threadIdx.x;
+  if (t >= k) return;
+  float v = 0.0f;
+  for (int i = 0; i < n_part; ++i) v += part[(int64_t)i * k + t];
+  ds[t] = v;
+}
+
+template <bool TRANS>
+metis_status_t launch_factor_grad(cudaStream_t s, const void* g, int g_dtype, int64_t ldg, int64_t n_r, int64_t n_c, int k,
+                                  const metis_nvfp4_t* f, const metis_nvfp4_t* o, const float* sigma, float* out, float* ds_part) {
+  const unsigned grid = (unsigned)metis_ceil_div(n_r, FG_ROWS);
+#define METIS_FG(KT) factor_grad_kernel<KT, TRANS><<<grid, 256, 0, s>>>(g, g_dtype, ldg, n_r, n_c, k, f->codes, f->scales, f->sf_layout, \
+    f->tensor_scale, o ? o->codes : nullptr, o ? o->scales : nullptr, o ? o->sf_layout : 0, o ? o->tensor_scale : nullptr, sigma, out, ds_part)
+  switch ((k + 7) / 8) {
+    case 1: METIS_FG(1); break; case 2: METIS_FG(2); break; case 3: METIS_FG(3); break; case 4: METIS_FG(4); break;
+    case 5: METIS_FG(5); break; case 6: METIS_FG(6); break; case 7: METIS_FG(7); break; case 8: METIS_FG(8); break;
+    default: return METIS_ERR_SHAPE;
+  }
+#undef METIS_FG
+  METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
+
+// d_left (k x n), d_sigma (k), d_right (k x m) of the weight operand W_t = left diag(sigma) right^T from dw (n x m).
+metis_status_t factor_grads(metis_context* ctx, const void* dw, int dw_dtype, int64_t lddw, const metis_operand_t* w,
+                            float* d_left, float* d_sigma, float* d_right, void* ws, size_t ws_bytes, cudaStream_t s) {
+  (void)ctx;
+  if (!w || w->k <= 0 || w->k > 64 || !w->sigma) return METIS_ERR_SHAPE;
+  const int64_t n = w->rows, m = w->cols;
+  const metis_nvfp4_t *lq = &w->left_q, *rq = &w->right_q;
+  if (!lq->codes || !rq->codes || lq->k_len != n || rq->k_len != m) return METIS_ERR_SHAPE;
+  const int64_t n_part = metis_ceil_div(n, FG_ROWS);
+  if (d_sigma && (!ws || ws_bytes < sizeof(float) * (size_t)n_part * w->k)) return METIS_ERR_WORKSPACE;
+  float* part = reinterpret_cast<float*>(ws);
+  // dL/dV (the paper's V = left, n x k): rows of dw against U = right; also the partials of dL/dS
+  if (d_left || d_sigma) {
+    if (!d_left) return METIS_ERR_INVALID_ARG;          // the sigma partials ride on the d_left pass
+    METIS_TRY(launch_factor_grad<false>(s, dw, dw_dtype, lddw, n, m, w->k, rq, d_sigma ? lq : nullptr, w->sigma, d_left,
+                                        d_sigma ? part : nullptr));
+    if (d_sigma) {
+      factor_grad_sigma_kernel<<<1, 64, 0, s>>>(part, (int)n_part, w->k, d_sigma); METIS_COUNT_LAUNCH();
+      METIS_CUDA_TRY(cudaGetLastError());
+    }
+  }
+  // dL/dU (the paper's U = right, m x k): columns of dw against V = left
+  if (d_right) METIS_TRY(launch_factor_grad<true>(s, dw, dw_dtype, lddw, m, n, w->k, lq, nullptr, w->sigma, d_right, nullptr));
+  return METIS_OK;
+}
+
 struct Side {
   const metis_nvfp4_t* res;   // residual, K-major along the contraction axis
   const metis_nvfp4_t* fc;    // factor along the contraction axis (k x K)
@@ -206,7 +338,8 @@ size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k) {
   // sized for either path: FP32 staging of the main product (small shapes) or the BF16 correction operands
   return align256(sizeof(float) * M * N) + align256(sizeof(float) * 64 * 64) +
          align256(sizeof(float) * M * (kc ? kc : 1)) + align256(sizeof(float) * N * (kc ? kc : 1)) +
-         align256(sizeof(__nv_bfloat16) * M * (kx ? kx : 1)) + align256(sizeof(__nv_bfloat16) * N * (kx ? kx : 1));
+         align256(sizeof(__nv_bfloat16) * M * (kx ? kx : 1)) + align256(sizeof(__nv_bfloat16) * N * (kx ? kx : 1)) +
+         align256(sizeof(float) * 64 * (size_t)metis_ceil_div(M > N ? M : N, FG_ROWS));     // partials of the sigma gradient
 }
 
 metis_status_t metis_linear_fwd(metis_handle_t h, const metis_operand_t* x, const metis_operand_t* w, void* y,
@@ -221,8 +354,10 @@ metis_status_t metis_linear_fwd(metis_handle_t h, const metis_operand_t* x, cons
 
 metis_status_t metis_linear_bwd(metis_handle_t h, const metis_operand_t* dy, const metis_operand_t* x,
                                 const metis_operand_t* w, void* dx, int32_t dx_dtype, int64_t lddx, void* dw,
-                                int32_t dw_dtype, int64_t lddw, void* ws, size_t ws_bytes, metis_stream_t stream) {
+                                int32_t dw_dtype, int64_t lddw, float* d_left, float* d_sigma, float* d_right,
+                                void* ws, size_t ws_bytes, metis_stream_t stream) {
   if (!h || !dy) return METIS_ERR_INVALID_ARG;
+  if ((d_left || d_sigma || d_right) && (!dw || !w)) return METIS_ERR_INVALID_ARG;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (dx) {
     if (!w || dy->cols != w->rows) return METIS_ERR_SHAPE;
@@ -237,6 +372,10 @@ metis_status_t metis_linear_bwd(metis_handle_t h, const metis_operand_t* dy, con
     Side a{&dy->res_by_rows, &dy->left_q, &dy->right_q, dy->sigma, dy->k};
     Side b{&x->res_by_rows, &x->left_q, &x->right_q, x->sigma, x->k};
     METIS_TRY(split_gemm(h, a, b, dw, dw_dtype, lddw, ws, ws_bytes, s));
+    if (d_left || d_sigma || d_right) {
+      if (w->rows != dy->cols || w->cols != x->cols) return METIS_ERR_SHAPE;
+      METIS_TRY(factor_grads(h, dw, dw_dtype, lddw, w, d_left, d_sigma, d_right, ws, ws_bytes, s));
+    }
   }
   return METIS_OK;
 }

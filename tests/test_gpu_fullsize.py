@@ -24,7 +24,8 @@ def test_qproj_layer_forward_and_backward_on_sampled_rows():
         wo = h.split(dev(c["w"]), k, p, sketch=B.SKETCH_FULL, seed=2)
         do = h.split(dev(c["dy"]), k, p, sketch=B.SKETCH_SAMPLED, seed=3, rounding=B.ROUND_SR)
         y = h.linear_fwd(xo, wo, out_dtype=torch.float32)
-        dx, dw = h.linear_bwd(do, xo, wo, out_dtype=torch.float32)
+        d_left, d_sigma, d_right = (torch.empty(sh, device="cuda") for sh in ((k, 4096), (k,), (k, 4096)))
+        dx, dw = h.linear_bwd(do, xo, wo, out_dtype=torch.float32, factor_grads=(d_left, d_sigma, d_right))
         torch.cuda.synchronize()
         assert h.device_status() == 0
         xq = olay.quantize_operand(c["x"], k, p, osp.MODE_SAMPLED, 1)
@@ -41,5 +42,11 @@ def test_qproj_layer_forward_and_backward_on_sampled_rows():
         assert rel_fro(dx.cpu().numpy()[rows], dd_c[rows] @ wd_r) < TOL
         dd_r, xd_r = dq.dense(onv.AXIS_ROWS), xq.dense(onv.AXIS_ROWS)
         assert rel_fro(dw.cpu().numpy()[rows], dd_r[:, rows].T @ xd_r) < TOL
+        # factor gradients of the weight operand (sampled rows of dL/dV, all of dL/dS and dL/dU) from the oracle's dW
+        dw_o = dd_r.T @ xd_r
+        du, ds, dv = olay.factor_grads(dw_o, wq)
+        assert rel_fro(d_left.cpu().numpy().T[rows], dv[rows]) < TOL
+        assert rel_fro(d_right.cpu().numpy().T, du) < TOL
+        assert rel_fro(d_sigma.cpu().numpy(), ds) < TOL
     finally:
         h.close()

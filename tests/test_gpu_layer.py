@@ -79,6 +79,54 @@ def test_forward_and_backward_medium(ctx, k):
     assert rel_fro(dw.cpu().numpy(), (ld + rdr).T @ (lx + rxr)) < 2e-5
 
 
+@pytest.mark.parametrize("dw_dtype", [torch.float32, torch.bfloat16])
+def test_factor_gradients(ctx, dw_dtype):
+    """dL/dU, dL/dS, dL/dV of the weight factors (Section 3.2) against the oracle."""
+    from gpu_util import to_dev_bf16, rel_fro, nv_dequant
+    B, h = ctx
+    l, m, n, k, p = 256, 448, 192, 12, 4
+    x, _ = synth.llama_like(l, m, 1.0, 61, rank=8)
+    w, _ = synth.llama_like(n, m, 0.02, 62, rank=8)
+    d, _ = synth.llama_like(l, n, 1e-4, 63, rank=8)
+    xo = h.split(to_dev_bf16(x), k, p, sketch=B.SKETCH_SAMPLED, seed=1)
+    wo = h.split(to_dev_bf16(w), k, p, sketch=B.SKETCH_FULL, seed=2)
+    do = h.split(to_dev_bf16(d), k, p, sketch=B.SKETCH_SAMPLED, seed=3, rounding=B.ROUND_SR)
+    d_left = torch.full((k, n), float("nan"), device="cuda")
+    d_sigma = torch.full((k,), float("nan"), device="cuda")
+    d_right = torch.full((k, m), float("nan"), device="cuda")
+    dx, dw = h.linear_bwd(do, xo, wo, out_dtype=dw_dtype, factor_grads=(d_left, d_sigma, d_right))
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    # (a) the three contractions themselves, from the library's own dw and dequantized factors, in float64
+    dwn = dw.float().cpu().numpy().astype(np.float64)
+    lq, rq = nv_dequant(wo.left_q)[:k].T, nv_dequant(wo.right_q)[:k].T            # n x k (V), m x k (U)
+    sig = wo.sigma.cpu().numpy().astype(np.float64)
+    assert rel_fro(d_left.cpu().numpy().T, (dwn @ rq) * sig) < 1e-5
+    assert rel_fro(d_right.cpu().numpy().T, (dwn.T @ lq) * sig) < 1e-5
+    assert rel_fro(d_sigma.cpu().numpy(), np.einsum("jt,ji,it->t", lq, dwn, rq)) < 1e-5
+    # (b) end to end against the oracle's own split, quantization and weight gradient
+    xq = olay.quantize_operand(x, k, p, osp.MODE_SAMPLED, 1)
+    wq = olay.quantize_operand(w, k, p, osp.MODE_FULL, 2)
+    dq = olay.quantize_operand(d, k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
+    du, ds, dv = olay.factor_grads(olay.linear_wgrad(dq, xq), wq)
+    tol = TOL if dw_dtype == torch.float32 else 3 * TOL                           # a BF16 dw carries 2^-9 per entry
+    assert rel_fro(d_right.cpu().numpy().T, du) < tol
+    assert rel_fro(d_left.cpu().numpy().T, dv) < tol
+    assert rel_fro(d_sigma.cpu().numpy(), ds) < tol
+
+
+def test_factor_gradients_need_the_weight_gradient(ctx):
+    from gpu_util import to_dev_bf16
+    B, h = ctx
+    c = synth.config_small()
+    xo = h.split(to_dev_bf16(c["x"]), 4, 4, sketch=B.SKETCH_FULL, seed=1)
+    wo = h.split(to_dev_bf16(c["w"]), 4, 4, sketch=B.SKETCH_FULL, seed=2)
+    do = h.split(torch.randn(128, 256, device="cuda").to(torch.bfloat16), 4, 4, sketch=B.SKETCH_FULL, seed=3)
+    g = torch.zeros((4, 256), device="cuda")
+    with pytest.raises(RuntimeError):
+        h.linear_bwd(do, xo, wo, need_dw=False, factor_grads=(g, None, None))
+
+
 def test_bf16_output(ctx):
     from gpu_util import to_dev_bf16, rel_fro
     B, h = ctx
