@@ -172,7 +172,9 @@ metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dty
  * scale amax(x)/2688 of the SOURCE tensor; factors with their own.  `residual_axes` selects which
  * residual orientations are produced.  `residual_dense` (optional, rows x cols FP32) receives the
  * unquantized residual the quantizer saw.  k == 0 quantizes x itself.
- * Requires rows % 16 == 0, cols % 64 == 0 (tiled scales), k + p <= 64, k % 4 == 0.
+ * Requires rows % 16 == 0, cols % 64 == 0 (tiled scales), k % 4 == 0, k <= 64 and k + p <= 72 (the
+ * orthonormalisation and the two small eigen-solvers each run in one CTA's shared memory; larger
+ * ranks are refused with METIS_ERR_SHAPE).
  * Workspace: metis_workspace_bytes(1, rows, cols, k, p). */
 metis_status_t metis_split(metis_handle_t h, const void* x, int64_t rows, int64_t cols, int32_t k, int32_t p,
                            int32_t sketch, int64_t n_sample, uint64_t seed, int32_t rounding,

@@ -91,18 +91,26 @@ def tensor_scale_from_amax(amax):
     return F32(1.0) if amax == 0 else F32(amax / F32(2688.0))
 
 
-def quantize(x, axis=AXIS_COLS, rounding=ROUND_RNE, seed=0, stream=philox.STREAM_RESIDUAL, tensor_scale=None):
+def quantize(x, axis=AXIS_COLS, rounding=ROUND_RNE, seed=0, stream=philox.STREAM_RESIDUAL, tensor_scale=None,
+             index=None):
     """Quantize a 2-D float32 array.  Returns (codes, scales, s_T) in K-major storage.
 
     codes  uint8 [R, K]     one 4-bit code per byte (pack() halves it)
     scales uint8 [R, K/16]  E4M3 bytes
     s_T    float32
     (R, K) = x.shape for AXIS_COLS and x.T.shape for AXIS_ROWS.  The stochastic-rounding draw of
-    an element is keyed by its index in x (row*cols + col) whatever the block axis.
+    an element is keyed by its index in x (row*cols + col) whatever the block axis.  `index` (uint64,
+    x's shape) replaces those keys: it lets a slice of a larger tensor be quantized with the draws its
+    elements have inside that tensor (addressing only; the arithmetic is the same).
     """
     x = np.asarray(x, dtype=F32)
     rows, cols = x.shape
-    index = np.arange(rows, dtype=np.uint64)[:, None] * np.uint64(cols) + np.arange(cols, dtype=np.uint64)[None, :]
+    if index is None:
+        index = np.arange(rows, dtype=np.uint64)[:, None] * np.uint64(cols) + np.arange(cols, dtype=np.uint64)[None, :]
+    else:
+        index = np.asarray(index, dtype=np.uint64)
+        if index.shape != x.shape:
+            raise ValueError("index must have the shape of x")
     if axis == AXIS_ROWS:
         x, index = x.T, index.T
     elif axis != AXIS_COLS:

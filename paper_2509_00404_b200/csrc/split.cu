@@ -9,7 +9,7 @@
 
 namespace {
 
-constexpr int MAXQ = 64;
+constexpr int MAXQ = 72;                               // k + p at most (k = 64 with p = 8)
 constexpr size_t JACOBI_SMEM = sizeof(double) * MAXQ * (MAXQ + 1);
 
 // ------------------------------------------------------------------------------------------------
@@ -151,21 +151,25 @@ apply_chol_kernel(float* __restrict__ z, int64_t n_rows, int q, const double* __
   __syncthreads();
   const int64_t r = (int64_t)blockIdx.x * 8 + warp;
   if (r >= n_rows) return;
-  double h0 = 0.0, h1 = 0.0;                         // h_lane, h_(lane+32)
+  static_assert(MAXQ <= 96, "three values per lane");
+  double h0 = 0.0, h1 = 0.0, h2 = 0.0;               // h_lane, h_(lane+32), h_(lane+64)
   const double z0 = lane < q ? (double)z[r * q + lane] : 0.0;
   const double z1 = lane + 32 < q ? (double)z[r * q + lane + 32] : 0.0;
+  const double z2 = lane + 64 < q ? (double)z[r * q + lane + 64] : 0.0;
   for (int j = 0; j < q; ++j) {
     double part = 0.0;
     if (lane < j) part += h0 * L[j][lane];
     if (lane + 32 < j) part += h1 * L[j][lane + 32];
+    if (lane + 64 < j) part += h2 * L[j][lane + 64];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
-    const double zj = __shfl_sync(0xFFFFFFFFu, j < 32 ? z0 : z1, j & 31);
+    const double zj = __shfl_sync(0xFFFFFFFFu, j < 32 ? z0 : (j < 64 ? z1 : z2), j & 31);
     const double hj = (zj - part) * inv_s[j];
-    if (lane == (j & 31)) { if (j < 32) h0 = hj; else h1 = hj; }
+    if (lane == (j & 31)) { if (j < 32) h0 = hj; else if (j < 64) h1 = hj; else h2 = hj; }
   }
   if (lane < q) z[r * q + lane] = (float)h0;
   if (lane + 32 < q) z[r * q + lane + 32] = (float)h1;
+  if (lane + 64 < q) z[r * q + lane + 64] = (float)h2;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -221,7 +225,7 @@ project_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __r
 }
 
 // ------------------------------------------------------------------------------------------------
-// Symmetric positive semi-definite eigen-decomposition (n <= 64) in FP64, one CTA.
+// Symmetric positive semi-definite eigen-decomposition (n <= MAXQ) in FP64, one CTA.
 // G = L L^T (Cholesky, dependent columns zeroed), then one-sided (Hestenes) Jacobi on the columns of Y = L:
 // plane rotations make the columns mutually orthogonal, Y J1 J2 ... = U Sigma, so G = Y Y^T = U Sigma^2 U^T:
 // eigenvalues are the squared column norms and eigenvectors the normalised columns.  Working on the
@@ -247,7 +251,7 @@ __device__ __forceinline__ double fast_rsqrt(double x) {
 }
 
 template <int R>                                        // rows per lane: ceil(n / 8)
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(R > 8 ? 288 : 256)    // eight lanes per couple: n = 72 needs 36 x 8 threads
 jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, double* __restrict__ evals,
                   double* __restrict__ evecs) {
   extern __shared__ __align__(16) unsigned char jsm[];
@@ -257,13 +261,14 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
   __shared__ int order[MAXQ];
   __shared__ int rotated[2];
   __shared__ uint8_t pairs[MAXQ][MAXQ / 2][2];          // [round][couple] -> (p, q)
+  constexpr int NTHR = R > 8 ? 288 : 256;
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const int np = n + (n & 1), half = np / 2;
-  for (int o = tid; o < np * np; o += 256) {
+  for (int o = tid; o < np * np; o += NTHR) {
     const int i = o / np, j = o % np;
     Y[i][j] = (i < n && j < n) ? 0.5 * (g[i * ld + j] + g[j * ld + i]) : 0.0;
   }
-  for (int o = tid; o < (np - 1) * half; o += 256) {
+  for (int o = tid; o < (np - 1) * half; o += NTHR) {
     int p, q;
     jacobi_pair(o % half, o / half, np, &p, &q);
     pairs[o / half][o % half][0] = (uint8_t)p; pairs[o / half][o % half][1] = (uint8_t)q;
@@ -285,10 +290,10 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
     const bool dep = !(d > tol);
     const double inv = dep ? 0.0 : chol_rsqrt(d);
     __syncthreads();
-    for (int i = j + 1 + tid; i < n; i += 256) Y[i][j] *= inv;
+    for (int i = j + 1 + tid; i < n; i += NTHR) Y[i][j] *= inv;
     if (tid == 0) Y[j][j] = dep ? 0.0 : d * inv;
     __syncthreads();
-    if (!dep) {
+    if (!dep && tid < 256) {                           // 16 x 16 thread grid over the trailing block
       for (int a = j + 1 + ty; a < n; a += 16) {
         const double laj = Y[a][j];
         for (int b = j + 1 + tx; b <= a; b += 16) Y[a][b] -= laj * Y[b][j];
@@ -296,7 +301,7 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
     }
     __syncthreads();
   }
-  for (int o = tid; o < np * np; o += 256) {
+  for (int o = tid; o < np * np; o += NTHR) {
     const int i = o / np, j = o % np;
     if (j > i) Y[i][j] = 0.0;
   }
@@ -385,7 +390,7 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
   }
   __syncthreads();
   if (tid < n) evals[tid] = lam[order[tid]];
-  for (int o = tid; o < n * n; o += 256) {
+  for (int o = tid; o < n * n; o += NTHR) {
     const int i = o / n, j = order[o % n];
     const double l2 = lam[j];
     evecs[o] = l2 > 0.0 ? Y[i][j] * fast_rsqrt_wide(l2) : 0.0;
@@ -1038,7 +1043,8 @@ void launch_jacobi(cudaStream_t s, const double* g, int n, int ld, float exit_co
     case 5: jacobi_eig_kernel<5><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
     case 6: jacobi_eig_kernel<6><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
     case 7: jacobi_eig_kernel<7><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
-    default: jacobi_eig_kernel<8><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+    case 8: jacobi_eig_kernel<8><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+    default: jacobi_eig_kernel<9><<<1, 288, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
   }
   METIS_COUNT_LAUNCH();
 }
@@ -1077,7 +1083,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   using namespace metis_qt;
   if (!h || !xv || !out || !ws) return METIS_ERR_INVALID_ARG;
   if (rows <= 0 || cols <= 0 || rows % 16 || cols % 16 || k < 0 || p < 0) return METIS_ERR_SHAPE;
-  if (k > 0 && (k + p > MAXQ || k % 4)) return METIS_ERR_SHAPE;
+  if (k > 0 && (k > 64 || k + p > MAXQ || k % 4)) return METIS_ERR_SHAPE;
   if (out->k != k || out->rows != rows || out->cols != cols) return METIS_ERR_INVALID_ARG;
   if (!metis_aligned16(xv) || !metis_aligned16(ws)) return METIS_ERR_ALIGNMENT;
   if (rounding != METIS_ROUND_RNE && rounding != METIS_ROUND_SR) return METIS_ERR_INVALID_ARG;
@@ -1147,6 +1153,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
       METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
       METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<9>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
       METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 64)));
       METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 48)));
       METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
@@ -1175,7 +1182,8 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       case 5: sketch_mma_kernel<5><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
       case 6: sketch_mma_kernel<6><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
       case 7: sketch_mma_kernel<7><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
-      default: sketch_mma_kernel<8><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+      case 8: sketch_mma_kernel<8><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+      default: sketch_mma_kernel<9><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
     }
     METIS_COUNT_LAUNCH();
   }
@@ -1202,7 +1210,8 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
         case 1: project_mma_kernel<1><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
         case 2: project_mma_kernel<2><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
         case 3: project_mma_kernel<3><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
-        default: project_mma_kernel<4><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+        case 4: project_mma_kernel<4><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+        default: project_mma_kernel<5><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
       }
       METIS_COUNT_LAUNCH();
     } else {
@@ -1217,7 +1226,8 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       case 5: launch_project<5>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
       case 6: launch_project<6>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
       case 7: launch_project<7>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
-      default: launch_project<8>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+      case 8: launch_project<8>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+      default: launch_project<9>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
     }
     }
     reduce_partials_kernel<<<(unsigned)metis_ceil_div((int64_t)q * cols, 256), 256, 0, s>>>(mp, parts, (int64_t)q * cols, m); METIS_COUNT_LAUNCH();

@@ -112,6 +112,10 @@ def test_workspace_and_shape_errors(ctx):
     B, h = ctx
     x = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(B.MetisError):
-        h.split(x, 60, 8)                      # k + p > 64
+        h.split(x, 68, 8)                      # k + p > 72
+    big = torch.zeros((2048, 2048), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.MetisError) as e:
+        h.split(big, 256, 8)                   # the rank-256 point of the 70B-shaped sweep is beyond the one-CTA solvers
+    assert e.value.code == 2                   # METIS_ERR_SHAPE
     with pytest.raises(B.MetisError):
         h.split(x, 6, 2)                       # k not a multiple of 4

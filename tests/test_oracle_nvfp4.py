@@ -213,3 +213,24 @@ def test_hand_worked_block():
     want = [6, -3, 2, 2, 1.5, 0.5, 0, -0.5, 0, 1, 4, -6, 4, 4, 6, 0]
     got = nvfp4.dequantize(codes, sc, s_T)[0] / 2
     assert got.tolist() == want
+
+
+def test_index_override_reproduces_slices_of_the_full_tensor():
+    """Quantizing rows (or columns) of a tensor on their own, keyed by their indices in the full tensor and with the
+    full tensor's scale, gives the same codes and scales as slicing the full result - for both roundings."""
+    rng = np.random.default_rng(7)
+    x = (rng.standard_normal((64, 96)) * 3).astype(np.float32)
+    rows, cols = np.array([3, 17, 40, 63]), np.array([0, 5, 95])
+    s_T = nvfp4.tensor_scale_from_amax(np.max(np.abs(x)))
+    for rounding in (nvfp4.ROUND_RNE, nvfp4.ROUND_SR):
+        fc = nvfp4.quantize(x, nvfp4.AXIS_COLS, rounding, seed=9, tensor_scale=s_T)
+        idx = rows[:, None].astype(np.uint64) * np.uint64(96) + np.arange(96, dtype=np.uint64)[None, :]
+        pc = nvfp4.quantize(x[rows], nvfp4.AXIS_COLS, rounding, seed=9, tensor_scale=s_T, index=idx)
+        assert np.array_equal(pc[0], fc[0][rows]) and np.array_equal(pc[1], fc[1][rows])
+        fr = nvfp4.quantize(x, nvfp4.AXIS_ROWS, rounding, seed=9, tensor_scale=s_T)
+        idx = np.arange(64, dtype=np.uint64)[:, None] * np.uint64(96) + cols[None, :].astype(np.uint64)
+        pr = nvfp4.quantize(x[:, cols], nvfp4.AXIS_ROWS, rounding, seed=9, tensor_scale=s_T, index=idx)
+        assert np.array_equal(pr[0], fr[0][cols]) and np.array_equal(pr[1], fr[1][cols])
+    # and the draws do depend on the keys
+    a = nvfp4.quantize(x[rows], nvfp4.AXIS_COLS, nvfp4.ROUND_SR, seed=9, tensor_scale=s_T)
+    assert not np.array_equal(a[0], fc[0][rows])
