@@ -88,6 +88,83 @@ __device__ __forceinline__ double chol_rsqrt(double x) {
 
 __device__ __forceinline__ double fast_rsqrt_wide(double x) { return chol_rsqrt(x); }
 
+// 1/x in FP64 for x inside the FP32 range: FP32 seed and two Newton steps; anything else takes the division
+__device__ __forceinline__ double chol_rcp(double x) {
+  if (!(x > 1e-30 && x < 1e30)) return 1.0 / x;
+  double y = (double)__frcp_rn((float)x);
+  y = y * (2.0 - x * y);
+  y = y * (2.0 - x * y);
+  return y;
+}
+
+// In-place Cholesky of the n x n lower triangle of Y (row pitch P doubles) by the whole CTA (>= 256 threads).
+// Right-looking with the column scaling deferred: step j only subtracts  Y[a][j] Y[b][j] / Y[j][j]  from the
+// trailing triangle (one barrier per column, a reciprocal instead of a square root in the serial chain); the
+// columns are divided by sqrt(pivot) together at the end.  A pivot not above `tol` marks a dependent column:
+// it takes no part in the updates and ends as a zero column with inv_out[j] = 0.
+template <int P>
+__device__ __forceinline__ void cta_cholesky(double (*Y)[P], int n, double tol, double* inv_out, double* dmin_out, int nthr) {
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  constexpr int NT = (MAXQ + 15) / 16;                  // 16 x 16 thread grid, NT x NT elements per thread
+  for (int j = 0; j < n; ++j) {
+    const double d = Y[j][j];
+    if (d > tol && tid < 256) {
+      const double rd = chol_rcp(d);
+      // operands first, then the products, then the stores: the loads of one step do not wait for its stores.
+      // `rem` is the same for every thread, so whole 16-wide groups beyond the trailing block are skipped.
+      const int rem = n - j - 1;
+      double la[NT], lb[NT], t[NT][NT];
+#pragma unroll
+      for (int u = 0; u < NT; ++u) {
+        if (16 * u < rem) {
+          const int a = j + 1 + ty + 16 * u, b = j + 1 + tx + 16 * u;
+          la[u] = a < n ? Y[a][j] * rd : 0.0;
+          lb[u] = b < n ? Y[b][j] : 0.0;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < NT; ++u)
+#pragma unroll
+        for (int v = 0; v <= u; ++v) {
+          if (16 * u < rem) {
+            const int a = j + 1 + ty + 16 * u, b = j + 1 + tx + 16 * v;
+            t[u][v] = (a < n && b <= a) ? Y[a][b] : 0.0;
+          }
+        }
+#pragma unroll
+      for (int u = 0; u < NT; ++u)
+#pragma unroll
+        for (int v = 0; v <= u; ++v) {
+          if (16 * u < rem) {
+            const int a = j + 1 + ty + 16 * u, b = j + 1 + tx + 16 * v;
+            if (a < n && b <= a) Y[a][b] = t[u][v] - la[u] * lb[v];
+          }
+        }
+    }
+    __syncthreads();
+  }
+  double dj = 0.0, inv = 0.0;
+  if (tid < n) {
+    dj = Y[tid][tid];
+    inv = dj > tol ? chol_rsqrt(dj) : 0.0;
+    inv_out[tid] = inv;
+  }
+  if (dmin_out != nullptr && tid < 32) {                // smallest accepted pivot
+    double dm = 1e300;
+    for (int i = tid; i < n; i += 32) { const double v = Y[i][i]; if (v > tol) dm = fmin(dm, v); }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dm = fmin(dm, __shfl_xor_sync(0xFFFFFFFFu, dm, o));
+    if (tid == 0) *dmin_out = dm;
+  }
+  __syncthreads();
+  for (int o = tid; o < n * n; o += nthr) {
+    const int i = o / n, j = o % n;
+    if (i > j) Y[i][j] *= inv_out[j];
+  }
+  if (tid < n) Y[tid][tid] = dj * inv;                  // sqrt(pivot), or 0 for a dependent column
+  __syncthreads();
+}
+
 // One CholeskyQR pass, step 1 (one CTA): G (one Gram partial) = L L^T in FP64; writes L (q x q, row-major,
 // upper part unused) and the reciprocal pivots.  A pivot below 1e-13 of the largest diagonal marks a
 // dependent sketch column: its reciprocal is stored as zero, so the corresponding column of H = Z L^-T
@@ -111,26 +188,9 @@ chol_kernel(const double* __restrict__ g, int q, double* __restrict__ l_out, dou
   }
   __syncthreads();
   const double tol = 1e-13 * gmax_s;
-  for (int j = 0; j < q; ++j) {
-    const double d = L[j][j];
-    const bool dep = !(d > tol);
-    const double inv = dep ? 0.0 : chol_rsqrt(d);
-    __syncthreads();
-    for (int i = j + 1 + tid; i < q; i += 256) L[i][j] *= inv;
-    if (tid == 0) {
-      L[j][j] = dep ? 0.0 : d * inv; invd_out[j] = inv;
-      if (j == 0) dmin_s = gmax_s;
-      if (!dep) dmin_s = fmin(dmin_s, d);
-    }
-    __syncthreads();
-    if (!dep) {
-      for (int a = j + 1 + ty; a < q; a += 16) {
-        const double laj = L[a][j];
-        for (int b = j + 1 + tx; b <= a; b += 16) L[a][b] -= laj * L[b][j];
-      }
-    }
-    __syncthreads();
-  }
+  __shared__ double inv_s[MAXQ];
+  cta_cholesky<MAXQ + 1>(L, q, tol, inv_s, &dmin_s, 256);
+  if (tid < q) invd_out[tid] = inv_s[tid];
   // With every pivot above 1e-8 of the largest diagonal the FP64 factorisation leaves Z L^-T orthonormal to
   // ~1e-8 already, below the FP32 rounding of its storage: the caller's second pass is then skipped.
   if (tid == 0 && well_conditioned != nullptr) *well_conditioned = (dmin_s > 1e-8 * gmax_s) ? 1 : 0;
@@ -285,22 +345,7 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
   }
   __syncthreads();
   const double tol = 1e-14 * gmax_s;
-  for (int j = 0; j < n; ++j) {
-    const double d = Y[j][j];
-    const bool dep = !(d > tol);
-    const double inv = dep ? 0.0 : chol_rsqrt(d);
-    __syncthreads();
-    for (int i = j + 1 + tid; i < n; i += NTHR) Y[i][j] *= inv;
-    if (tid == 0) Y[j][j] = dep ? 0.0 : d * inv;
-    __syncthreads();
-    if (!dep && tid < 256) {                           // 16 x 16 thread grid over the trailing block
-      for (int a = j + 1 + ty; a < n; a += 16) {
-        const double laj = Y[a][j];
-        for (int b = j + 1 + tx; b <= a; b += 16) Y[a][b] -= laj * Y[b][j];
-      }
-    }
-    __syncthreads();
-  }
+  cta_cholesky<MAXQ + 1>(Y, n, tol, lam, nullptr, NTHR);
   for (int o = tid; o < np * np; o += NTHR) {
     const int i = o / np, j = o % np;
     if (j > i) Y[i][j] = 0.0;
@@ -326,10 +371,11 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
     }
     if (tid == 0) rotated[0] = 0;                       // reused as the sweep's max cos^2 (float bits)
     __syncthreads();
+    int p = active ? pairs[0][m][0] : 0, q = active ? pairs[0][m][1] : 0;
+    float sweep_cos2 = 0.0f;                            // this couple slot's largest cos^2 of the sweep
     for (int step = 0; step < np - 1; ++step) {
       {
         // every lane takes part in the shuffles; lanes of couples beyond n/2 carry zeros and write nothing
-        const int p = active ? pairs[step][m][0] : 0, q = active ? pairs[step][m][1] : 0;
         double yp[R], yq[R];
         double c = 0.0;
 #pragma unroll
@@ -342,12 +388,16 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
 #pragma unroll
         for (int o = 4; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
         const float a = lamf[p], b = lamf[q], cf = (float)c;
-        const float cos2 = (cf / a) * (cf / b);
-        // rotate only if the two columns are not yet orthogonal to working precision
-        if (active && cos2 > 1e-26f) {
-          float zeta = (b - a) / (2.0f * cf);
-          if (!(fabsf(zeta) < 1e18f)) zeta = copysignf(1e18f, zeta);      // huge or not finite: (almost) no rotation
-          const float tf = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
+        const int pn = (active && step + 1 < np - 1) ? pairs[step + 1][m][0] : 0;      // next round's couple, fetched early
+        const int qn = (active && step + 1 < np - 1) ? pairs[step + 1][m][1] : 0;
+        // rotate only if the two columns are not yet orthogonal to working precision (cos^2 > 1e-26)
+        if (active && cf * cf > 1e-26f * (a * b)) {
+          // tan(theta) = 2c / (d + sign(d) sqrt(d^2 + 4c^2)), d = b - a: the smaller root, |theta| <= pi/4.  These
+          // FP32 quantities only steer convergence, so the fast reciprocal and reciprocal square root are enough.
+          const float d = b - a, c2 = 2.0f * cf;
+          const float h2 = fmaf(c2, c2, d * d);
+          const float hyp = h2 * rsqrtf(h2);
+          const float tf = __fdividef(d < 0.0f ? -c2 : c2, fabsf(d) + hyp);
           const float c32 = rsqrtf(fmaf(tf, tf, 1.0f)), s32 = tf * c32;
           // (c32, s32) is a unit vector to ~1e-7; one Newton step on 1/sqrt(c^2 + s^2) in FP64 makes it one to ~1e-14
           const double cd = (double)c32, sd = (double)s32;
@@ -365,12 +415,15 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
             const float tc = tf * cf;                   // |y_p'|^2 = a - t c, |y_q'|^2 = b + t c for the exact rotation
             lamf[p] = a - tc;
             lamf[q] = b + tc;
-            atomicMax(reinterpret_cast<unsigned int*>(&rotated[0]), __float_as_uint(fminf(cos2, 1.0f)));
+            sweep_cos2 = fmaxf(sweep_cos2, fminf(__fdividef(cf * cf, a * b), 1.0f));
           }
         }
+        p = pn; q = qn;
       }
       __syncthreads();
     }
+    if (sub == 0 && sweep_cos2 > 0.0f) atomicMax(reinterpret_cast<unsigned int*>(&rotated[0]), __float_as_uint(sweep_cos2));
+    __syncthreads();
     const float maxcos2 = __uint_as_float((unsigned int)rotated[0]);
     __syncthreads();
     if (maxcos2 < exit_cos2) break;
