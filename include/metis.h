@@ -138,7 +138,7 @@ size_t metis_sf_bytes(int64_t rows, int64_t k_len, int32_t sf_layout);
 metis_status_t metis_workspace_bytes(int32_t op, int64_t rows, int64_t cols, int32_t k, int32_t p, size_t* bytes);
 
 /* Number of rows the SAMPLED sketch reads for a rows-row operand with k+p sketch columns
- * (Section 3.1: "less than 1 % of sequences"; at least 4(k+p), multiple of 16). */
+ * (Section 3.1 samples under one in a hundred sequences; here at least 4(k+p) rows, a multiple of 16). */
 int64_t metis_default_sample_count(int64_t rows, int32_t q);
 
 /* ---- NVFP4 quantizer (Section 2.3; value set of Appendix C.1) ----------------------------- */

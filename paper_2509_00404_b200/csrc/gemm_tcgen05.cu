@@ -4,19 +4,17 @@
 //
 // A (M x K) and B (N x K) are K-major packed FP4 (two codes per byte) with one UE4M3 scale per 16
 // elements stored in the 128 x 4 tiled layout, alpha = tensor_scale(A) * tensor_scale(B).
-// This is the product that carries "over 95 % of the training workload" (Section 3): the
+// These matrix products are where nearly all of the training arithmetic goes (Section 3): the
 // residual x residual term of Eq. 2 / Eq. 3 / the weight gradient, and the skinny factor products.
 //
-// Structure (one CTA per SM, persistent over output tiles, warp-specialised):
-//   warp 0      producer: TMA tensor loads of the A/B code tiles (128-byte swizzle) and bulk copies of
-//               the scale atoms into a multi-stage shared-memory ring, completion on mbarriers
-//   warp 1      MMA issuer: copies the scale atoms shared memory -> tensor memory (tcgen05.cp), issues
-//               tcgen05.mma kind::mxf4nvf4 (block16 scales) accumulating FP32 in tensor memory,
-//               releases ring slots with tcgen05.commit
-//   warps 2-5   epilogue: tcgen05.ld the accumulator (one TMEM lane quarter per warp), scale by alpha,
-//               convert and store; accumulators are double-buffered so the epilogue of tile i overlaps
-//               the main loop of tile i+1
-// Every mbarrier wait is bounded; on expiry the kernel records METIS_DEV_TIMEOUT and unwinds.
+// Two kernels, both persistent over output tiles and warp-specialised (TMA producer warp, MMA issuer warp,
+// epilogue warps; shared-memory ring with mbarriers; FP32 accumulators in tensor memory):
+//   gemm_nvfp4_kernel<BLOCK_N>       one CTA per 128 x BLOCK_N tile (skinny products)
+//   two_cta::gemm_nvfp4_2cta_kernel  a CTA pair (cta_group::2) per 256 x 256 tile, optionally followed by BF16
+//                                    K boxes that add a low-rank correction into the same accumulator
+// The producer and issuer loops are walked by whole warps with one elected lane issuing, so that descriptors
+// and addresses stay in uniform registers.  Every mbarrier wait is bounded; on expiry the kernel records
+// METIS_DEV_TIMEOUT and unwinds.
 #include <cuda.h>
 #include <stdlib.h>
 
