@@ -93,6 +93,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+// shared -> global tensor store (bulk async-group completion); rows / columns beyond the tensor are clipped
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -170,6 +181,7 @@ struct GemmArgs {
   void* d; int d_dtype; int64_t ldd;
   int M, N, K;
   uint32_t* dev_status;
+  int tma_store;           // two-CTA kernel: the output goes through shared memory and tensor stores
   int extra_kb;            // BF16 correction boxes (64 elements of K each) appended after the FP4 K loop
 };
 
@@ -374,7 +386,8 @@ constexpr int SF_COL0 = 256;
 constexpr int TMEM_COLS = 512;
 static_assert(ACC_COLS + STAGES * SF_COLS_PER_STAGE <= TMEM_COLS, "tensor memory budget");
 constexpr int NUM_THREADS = 384;                            // producer, MMA issuer, two idle warps, 8 epilogue warps
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int OUT_STAGE_BYTES = 8 * 4096;                   // per epilogue warp: 32 rows x 128 bytes of converted output
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + OUT_STAGE_BYTES + 1024 + 256;
 
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
@@ -462,7 +475,8 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int m, int n) {
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                        const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
-                       const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUtensorMap map_r, GemmArgs g) {
+                       const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUtensorMap map_r,
+                       const __grid_constant__ CUtensorMap map_d, GemmArgs g) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -471,12 +485,13 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   auto b_addr = [&](int s) { return a_addr(s) + A_BYTES; };
   auto sfa_addr = [&](int s) { return b_addr(s) + B_BYTES; };
   auto sfb_addr = [&](int s) { return sfa_addr(s) + SFA_BYTES; };
-  const uint32_t bar_base = base + (uint32_t)STAGES * STAGE_BYTES;
+  const uint32_t out_base = base + (uint32_t)STAGES * STAGE_BYTES;           // 1024-byte aligned (swizzled store boxes)
+  const uint32_t bar_base = out_base + (uint32_t)OUT_STAGE_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };                  // leader only: both CTAs' loads landed
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };      // slot free (per CTA, by commit multicast)
   const uint32_t tfull_bar = bar_base + 8u * (2 * STAGES);                   // accumulator complete (per CTA)
   const uint32_t tempty_bar = bar_base + 8u * (2 * STAGES + 1);              // leader only: both epilogues drained
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + (size_t)STAGES * STAGE_BYTES + 8 * (2 * STAGES + 2));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + (size_t)STAGES * STAGE_BYTES + OUT_STAGE_BYTES + 8 * (2 * STAGES + 2));
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -485,6 +500,17 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const int num_m = (g.M + TILE_M - 1) / TILE_M, num_n = (g.N + TILE_N - 1) / TILE_N;
   const int num_tiles = num_m * num_n;
+  // Work items: whole 256 x 256 tiles, except that a last partial wave which fills at most half of the pairs is
+  // cut into 256 x 128 halves (two items per tile), so that it takes half a tile time instead of a whole one.
+  const int full_items = (num_tiles / num_pairs) * num_pairs;
+  const bool split_tail = num_tiles > full_items && 2 * (num_tiles - full_items) <= num_pairs;
+  const int num_items = split_tail ? full_items + 2 * (num_tiles - full_items) : num_tiles;
+  auto decode = [&](int item, int& mb, int& nb, int& nhalf) {      // nhalf: -1 whole tile, 0 / 1 left / right half
+    int tile = item;
+    nhalf = -1;
+    if (split_tail && item >= full_items) { tile = full_items + ((item - full_items) >> 1); nhalf = (item - full_items) & 1; }
+    mb = tile % num_m; nb = tile / num_m;
+  };
   const int num_fp4_kb = (g.K + BLOCK_K - 1) / BLOCK_K;
   const int num_kb = num_fp4_kb + g.extra_kb;
   const int sf_k_atoms = g.K / MMA_K;
@@ -513,13 +539,17 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     {
       int s = 0; uint32_t ph = 0;
       bool ok = true;
-      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-        const int mb = tile % num_m, nb = tile / num_m;
-        const int a_row = mb * TILE_M + (int)rank * 128, b_row = nb * TILE_N + (int)rank * 128;
+      for (int item = pair; item < num_items && ok; item += num_pairs) {
+        int mb, nb, nhalf;
+        decode(item, mb, nb, nhalf);
+        // a half item multiplies 128 columns: each CTA supplies 64 rows of B, the first 64 of the same 128-row
+        // box (the box and byte count of a stage stay what they are), and one scale slab serves both CTAs
+        const int a_row = mb * TILE_M + (int)rank * 128;
+        const int b_row = nhalf < 0 ? nb * TILE_N + (int)rank * 128 : nb * TILE_N + nhalf * 128 + (int)rank * 64;
         // a 128-row slab that lies wholly outside the matrix has all-zero codes; any valid slab's scales will
         // do for it, so the index is clamped instead of reading another tensor's bytes
         const int a_sf_tile = min(mb * 2 + (int)rank, (g.M + 127) / 128 - 1);
-        const int b_sf_tile0 = min(nb * 2, (g.N + 127) / 128 - 1), b_sf_tile1 = min(nb * 2 + 1, (g.N + 127) / 128 - 1);
+        const int b_sf_tile0 = min(nb * 2 + max(nhalf, 0), (g.N + 127) / 128 - 1), b_sf_tile1 = min(nb * 2 + 1, (g.N + 127) / 128 - 1);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
           if (elect_one()) {
@@ -554,7 +584,10 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       int s = 0; uint32_t ph = 0;
       int it = 0;
       bool ok = true;
-      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++it) {
+      for (int item = pair; item < num_items && ok; item += num_pairs, ++it) {
+        const bool narrow = split_tail && item >= full_items;
+        const uint32_t idesc_i = narrow ? make_idesc(TILE_M, TILE_N / 2) : idesc;
+        const uint32_t idesc_xi = narrow ? make_idesc_bf16(TILE_M, TILE_N / 2) : make_idesc_bf16(TILE_M, TILE_N);
         if (!mbar_wait_cluster(tempty_bar, ((uint32_t)it & 1u) ^ 1u, g.dev_status, dead)) { ok = false; break; }
         tc_fence_after();
         for (int kb = 0; kb < num_kb; ++kb) {
@@ -562,12 +595,11 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
           tc_fence_after();
           if (elect_one()) {
             if (kb >= num_fp4_kb) {
-              constexpr uint32_t idesc_x = make_idesc_bf16(TILE_M, TILE_N);
 #pragma unroll
               for (int k = 0; k < 4; ++k) {                   // 64 BF16 elements = four K=16 MMAs, 32 bytes apart
                 const uint64_t a_desc = make_smem_desc(a_addr(s) + k * 32, 1024, SWIZZLE_128B);
                 const uint64_t b_desc = make_smem_desc(b_addr(s) + k * 32, 1024, SWIZZLE_128B);
-                tc_mma_bf16_2(tmem_base, a_desc, b_desc, idesc_x, 1u);
+                tc_mma_bf16_2(tmem_base, a_desc, b_desc, idesc_xi, 1u);
               }
             } else {
               const int atoms = min(K_STEPS, sf_k_atoms - kb * K_STEPS);
@@ -579,19 +611,19 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 for (int k = 0; k < K_STEPS; ++k) {
                   tc_cp_sf2(sfa_t + 4 * k, sfa_d + (uint64_t)(k * 32));
                   tc_cp_sf2(sfb_t + 8 * k, sfb_d + (uint64_t)(k * 32));
-                  tc_cp_sf2(sfb_t + 8 * k + 4, sfb_d + (uint64_t)((K_STEPS + k) * 32));
+                  if (!narrow) tc_cp_sf2(sfb_t + 8 * k + 4, sfb_d + (uint64_t)((K_STEPS + k) * 32));
                 }
 #pragma unroll
                 for (int k = 0; k < K_STEPS; ++k)
-                  tc_mma_nvf4_2(tmem_base, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc, sfa_t + 4 * k, sfb_t + 8 * k, (kb | k) != 0 ? 1u : 0u);
+                  tc_mma_nvf4_2(tmem_base, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc_i, sfa_t + 4 * k, sfb_t + 8 * k, (kb | k) != 0 ? 1u : 0u);
               } else {
                 for (int k = 0; k < atoms; ++k) {
                   tc_cp_sf2(sfa_t + 4 * k, sfa_d + (uint64_t)(k * 32));
                   tc_cp_sf2(sfb_t + 8 * k, sfb_d + (uint64_t)(k * 32));
-                  tc_cp_sf2(sfb_t + 8 * k + 4, sfb_d + (uint64_t)((K_STEPS + k) * 32));
+                  if (!narrow) tc_cp_sf2(sfb_t + 8 * k + 4, sfb_d + (uint64_t)((K_STEPS + k) * 32));
                 }
                 for (int k = 0; k < atoms; ++k)
-                  tc_mma_nvf4_2(tmem_base, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc, sfa_t + 4 * k, sfb_t + 8 * k, (kb | k) != 0 ? 1u : 0u);
+                  tc_mma_nvf4_2(tmem_base, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc_i, sfa_t + 4 * k, sfb_t + 8 * k, (kb | k) != 0 ? 1u : 0u);
               }
             }
             tc_commit2(empty_bar(s), 3);                      // frees the slot in both CTAs
@@ -612,27 +644,92 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const float alpha = (*g.a_ts) * (*g.b_ts);
     int it = 0;
     bool ok = true;
-    for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++it) {
-      const int mb = tile % num_m, nb = tile / num_m;
+    for (int item = pair; item < num_items && ok; item += num_pairs, ++it) {
+      int mb, nb, nhalf;
+      decode(item, mb, nb, nhalf);
       if (!mbar_wait(tfull_bar, (uint32_t)it & 1u, g.dev_status, dead)) { ok = false; break; }
       tc_fence_after();
       const int row = mb * TILE_M + (int)rank * 128 + quarter * 32 + lane;
-      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 128);
       uint32_t r[4][32];
-      tc_ld32_nowait(t_row, r[0]);
-      tc_ld32_nowait(t_row + 32, r[1]);
-      tc_ld32_nowait(t_row + 64, r[2]);
-      tc_ld32_nowait(t_row + 96, r[3]);
+      if (nhalf < 0) {
+        const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 128);
+        tc_ld32_nowait(t_row, r[0]);
+        tc_ld32_nowait(t_row + 32, r[1]);
+        tc_ld32_nowait(t_row + 64, r[2]);
+        tc_ld32_nowait(t_row + 96, r[3]);
+      } else {                                                // 128 accumulator columns: 64 per warp
+        const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 64);
+        tc_ld32_nowait(t_row, r[0]);
+        tc_ld32_nowait(t_row + 32, r[1]);
+      }
       tc_wait_ld();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_remote(tempty_bar, 0u);
+      const int ncols_w = nhalf < 0 ? 128 : 64;                                   // columns this warp writes
+      const int col_w = nb * TILE_N + (nhalf < 0 ? half * 128 : nhalf * 128 + half * 64);
+      if (g.tma_store) {
+        // Each lane converts its row into a 128-byte line of the warp's staging box (16-byte chunks XOR-swizzled
+        // by the row, the layout of a 128-byte-swizzled tensor store), then one lane stores the 32-row box.
+        // The box is reused as soon as the previous store has finished READING it.
+        const uint32_t obuf = out_base + (uint32_t)(warp - 4) * 4096u + (uint32_t)lane * 128u;
+        const int row_w = mb * TILE_M + (int)rank * 128 + quarter * 32;
+        const uint32_t sw = (uint32_t)(lane & 7);
+        if (g.d_dtype == METIS_BF16) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int col = nb * TILE_N + half * 128 + c * 32;
-        if (row < g.M && col < g.N) store_row_chunk(g, row, col, r[c], alpha);
+          for (int st = 0; st < 2; ++st) {
+            if (st * 64 < ncols_w) {
+              if (lane == 0) bulk_wait_read_all();
+              __syncwarp();
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                uint32_t w[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const int e = (j & 3) * 8 + 2 * q;
+                  const __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(r[2 * st + (j >> 2)][e]) * alpha,
+                                                                  __uint_as_float(r[2 * st + (j >> 2)][e + 1]) * alpha);
+                  w[q] = *reinterpret_cast<const uint32_t*>(&hh);
+                }
+                st_shared_v4(obuf + (((uint32_t)j ^ sw) << 4), w[0], w[1], w[2], w[3]);
+              }
+              fence_proxy_async();
+              __syncwarp();
+              if (lane == 0 && row_w < g.M && col_w + st * 64 < g.N) {
+                tma_store_2d(&map_d, obuf, col_w + st * 64, row_w);
+                bulk_commit();
+              }
+            }
+          }
+        } else {
+#pragma unroll
+          for (int st = 0; st < 4; ++st) {
+            if (st * 32 < ncols_w) {
+              if (lane == 0) bulk_wait_read_all();
+              __syncwarp();
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                st_shared_v4(obuf + (((uint32_t)j ^ sw) << 4),
+                             __float_as_uint(__uint_as_float(r[st][4 * j]) * alpha), __float_as_uint(__uint_as_float(r[st][4 * j + 1]) * alpha),
+                             __float_as_uint(__uint_as_float(r[st][4 * j + 2]) * alpha), __float_as_uint(__uint_as_float(r[st][4 * j + 3]) * alpha));
+              fence_proxy_async();
+              __syncwarp();
+              if (lane == 0 && row_w < g.M && col_w + st * 32 < g.N) {
+                tma_store_2d(&map_d, obuf, col_w + st * 32, row_w);
+                bulk_commit();
+              }
+            }
+          }
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int col = col_w + c * 32;
+          if (c * 32 < ncols_w && row < g.M && col < g.N) store_row_chunk(g, row, col, r[c], alpha);
+        }
       }
     }
+    if (lane == 0) bulk_wait_all();                           // the staging boxes must outlive their stores
   }
 
   // ------------------------------- teardown ---------------------------------
@@ -715,9 +812,22 @@ metis_status_t make_bf16_map(metis_context* ctx, CUtensorMap* map, const void* p
   return r == CUDA_SUCCESS ? METIS_OK : METIS_ERR_CUDA;
 }
 
+// 2-D map over the output (row-major, leading dimension ldd): box = 32 rows x 128 bytes, 128-byte swizzle
+metis_status_t make_out_map(metis_context* ctx, CUtensorMap* map, void* d, int d_dtype, int64_t rows, int64_t cols, int64_t ldd) {
+  const cuuint64_t es = d_dtype == METIS_BF16 ? 2 : 4;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ldd * es};
+  const cuuint32_t box[2] = {(cuuint32_t)(128 / es), 32};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+      map, d_dtype == METIS_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, d, dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? METIS_OK : METIS_ERR_CUDA;
+}
+
 metis_status_t launch_2cta(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d, int d_dtype,
                            int64_t ldd, const void* lx, const void* rx, int kx, cudaStream_t s) {
-  CUtensorMap map_a, map_b, map_sfa, map_sfb, map_l, map_r;
+  CUtensorMap map_a, map_b, map_sfa, map_sfb, map_l, map_r, map_d;
   METIS_TRY(make_codes_map(ctx, &map_a, a, 128));
   METIS_TRY(make_codes_map(ctx, &map_b, b, 128));
   METIS_TRY(make_scales_map(ctx, &map_sfa, a));
@@ -734,6 +844,10 @@ metis_status_t launch_2cta(metis_context* ctx, const metis_nvfp4_t* a, const met
   g.M = (int)a->rows; g.N = (int)b->rows; g.K = (int)a->k_len;
   g.dev_status = ctx->dev_status;
   g.extra_kb = kx / 64;
+  // tensor stores need a 16-byte aligned base and row pitch; anything else takes the direct stores
+  g.tma_store = metis_aligned16(d) && ((ldd * (d_dtype == METIS_BF16 ? 2 : 4)) % 16 == 0) ? 1 : 0;
+  if (g.tma_store) METIS_TRY(make_out_map(ctx, &map_d, d, d_dtype, a->rows, b->rows, ldd));
+  else map_d = map_a;
   static bool attr_set = false;
   if (!attr_set) {
     METIS_CUDA_TRY(cudaFuncSetAttribute(two_cta::gemm_nvfp4_2cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)two_cta::SMEM_BYTES));
@@ -753,7 +867,7 @@ metis_status_t launch_2cta(metis_context* ctx, const metis_nvfp4_t* a, const met
     max_pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
   }
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  two_cta::gemm_nvfp4_2cta_kernel<<<2 * pairs, two_cta::NUM_THREADS, two_cta::SMEM_BYTES, s>>>(map_a, map_b, map_sfa, map_sfb, map_l, map_r, g); METIS_COUNT_LAUNCH();
+  two_cta::gemm_nvfp4_2cta_kernel<<<2 * pairs, two_cta::NUM_THREADS, two_cta::SMEM_BYTES, s>>>(map_a, map_b, map_sfa, map_sfb, map_l, map_r, map_d, g); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }

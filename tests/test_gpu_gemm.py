@@ -51,6 +51,14 @@ def test_bf16_output_and_many_tiles(ctx):
     assert _case(B, h, 2048, 1536, 512, seed=5, impl=0) < TOL
 
 
+def test_last_partial_wave_is_cut_into_half_tiles(ctx):
+    B, h = ctx
+    # 9 x 9 tiles of 256 x 256 on 74 CTA pairs: one whole wave, then 7 tiles as 14 half-tile items; the last
+    # column of tiles is ragged (192 wide), so one right half lies partly outside the matrix
+    assert _case(B, h, 2304, 2240, 512, seed=6, impl=0) < TOL
+    assert _case(B, h, 2200, 2304, 320, seed=7, impl=0, out_dtype=torch.bfloat16) < 3e-3
+
+
 def test_tensor_scales_multiply_the_result(ctx):
     B, h = ctx
     assert _case(B, h, 128, 128, 128, seed=9, impl=0, scale=1e-4) < TOL
