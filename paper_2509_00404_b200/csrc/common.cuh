@@ -161,6 +161,10 @@ metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int
                                      uint64_t seed, uint32_t stream_id, int64_t e_stride_r, int64_t e_stride_c,
                                      const float* tscale_src, int tscale_is_amax, const metis_nvfp4_t* by_cols,
                                      const metis_nvfp4_t* by_rows, cudaStream_t s);
+int metis_coeff_slices(int64_t rows, int64_t cols, int* chunks_per_slice);
+bool metis_coeff_tc_usable(const void* x, const void* bs, int64_t cols, int kp);
+metis_status_t metis_launch_coeff_tc(metis_context* ctx, const void* x, int64_t rows, int64_t cols, const void* bs, int kp,
+                                     float* part, float* amax, cudaStream_t s);
 metis_status_t metis_launch_gemm_check(const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d, int d_dtype,
                                        int64_t ldd, cudaStream_t s);
 metis_status_t metis_launch_gemm_tc(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d,

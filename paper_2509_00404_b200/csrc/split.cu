@@ -643,6 +643,36 @@ __global__ void reduce_gram_kernel(const double* __restrict__ in, int n_in, int 
   out[e] = a;
 }
 
+// Sums the column slices of the tensor-core broadcast pass in a fixed order: coef[r][j] = sum_s part[s][r][j],
+// and writes the FP64 Gram partial of the CTA's 32 rows of C (for Rayleigh-Ritz).
+template <int KP>
+__global__ void __launch_bounds__(256)
+coef_finish_kernel(const float* __restrict__ part, int slices, int64_t rows, float* __restrict__ coef,
+                   double* __restrict__ gram_part) {
+  __shared__ float cfin[32 * KP];
+  const int tid = threadIdx.x;
+  const int64_t row0 = (int64_t)blockIdx.x * 32;
+  for (int o = tid; o < 32 * KP; o += 256) {
+    const int64_t r = row0 + o / KP;
+    float v = 0.0f;
+    if (r < rows) {
+      for (int s = 0; s < slices; ++s) v += part[((int64_t)s * rows + r) * KP + (o % KP)];
+      coef[r * KP + (o % KP)] = v;
+    }
+    cfin[o] = v;
+  }
+  __syncthreads();
+  if (gram_part) {
+    for (int o = tid; o < KP * KP; o += 256) {
+      const int i = o / KP, j = o % KP;
+      double a = 0.0;
+#pragma unroll 8
+      for (int r = 0; r < 32; ++r) a += (double)cfin[r * KP + i] * (double)cfin[r * KP + j];
+      gram_part[(int64_t)blockIdx.x * KP * KP + o] = a;
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Fused residual + quantizer: R = x - C B^T on a 128 x 128 tile (tensor cores, three-term BF16 splits of
 // both FP32 operands), then NVFP4 in one or both block orientations straight from shared memory (the
@@ -1027,7 +1057,7 @@ left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, i
 
 struct SplitWs {
   size_t amax, idx, zp, z, gram, gram1, linv, evals, evecs, mp, m, basis, coef, sign, cand_v, cand_i, evals2, evecs2, bs, bt,
-      gram_c, total;
+      gram_c, part, total;
 };
 
 constexpr int PJ_MAX_PARTS = 16;
@@ -1064,6 +1094,7 @@ SplitWs split_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s) {
   w.basis = take(sizeof(float) * (size_t)k * cols);
   const int kp = (k + 15) / 16 * 16;
   w.coef = take(sizeof(float) * (size_t)kp * rows);
+  w.part = take(sizeof(float) * (size_t)metis_coeff_slices(rows, cols, nullptr) * kp * rows);
   w.bs = take(sizeof(__nv_bfloat16) * 3 * (size_t)kp * cols);
   w.bt = take(sizeof(__nv_bfloat16) * 3 * (size_t)kp * cols);
   w.gram_c = take(sizeof(double) * (size_t)metis_ceil_div(rows, 32) * kp * kp);
@@ -1193,6 +1224,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   __nv_bfloat16* bs = reinterpret_cast<__nv_bfloat16*>(wsb + L.bs);
   __nv_bfloat16* bt = reinterpret_cast<__nv_bfloat16*>(wsb + L.bt);
   double* gram_c = reinterpret_cast<double*>(wsb + L.gram_c);
+  float* part = reinterpret_cast<float*>(wsb + L.part);
   metis_context* ctx = h;
   const int kp = (k + 15) / 16 * 16;
   {
@@ -1305,12 +1337,24 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
                                                                             out->left, nullptr, coef, kp, out->sigma, amax + 1); METIS_COUNT_LAUNCH();
   } else {
     basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(basis, cols, k, kp, bs, bt); METIS_COUNT_LAUNCH();
-    const size_t smem = sizeof(float) * 9 * 32 * kp;
-    switch (kp) {
-      case 16: coeff_mma_kernel<16><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
-      case 32: coeff_mma_kernel<32><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
-      case 48: coeff_mma_kernel<48><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
-      default: coeff_mma_kernel<64><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
+    if (metis_coeff_tc_usable(x, bs, cols, kp)) {
+      // tensor-core pass over x (column slices), then the slices are summed and the Gram partials formed
+      METIS_TRY(metis_launch_coeff_tc(ctx, x, rows, cols, bs, kp, part, amax, s));
+      const int slices = metis_coeff_slices(rows, cols, nullptr);
+      switch (kp) {
+        case 16: coef_finish_kernel<16><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c); break;
+        case 32: coef_finish_kernel<32><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c); break;
+        case 48: coef_finish_kernel<48><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c); break;
+        default: coef_finish_kernel<64><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c); break;
+      }
+    } else {
+      const size_t smem = sizeof(float) * 9 * 32 * kp;
+      switch (kp) {
+        case 16: coeff_mma_kernel<16><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
+        case 32: coeff_mma_kernel<32><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
+        case 48: coeff_mma_kernel<48><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
+        default: coeff_mma_kernel<64><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
+      }
     }
     METIS_COUNT_LAUNCH();
   }
