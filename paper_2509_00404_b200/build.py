@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libmetis_b200.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm_check.cu", "gemm_tcgen05.cu", "split.cu", "coeff_tc.cu", "linear.cu", "static_ws.cu"]
+SOURCES = ["api.cu", "quantize.cu", "gemm_check.cu", "gemm_tcgen05.cu", "split.cu", "coeff_tc.cu", "residual_tc.cu", "linear.cu", "static_ws.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
          "--fmad=true", "-Xptxas", "-v"]
 

@@ -172,17 +172,6 @@ coeff_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
   }
 }
 
-metis_status_t make_map_bf16(metis_context* ctx, CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows) {
-  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
-      map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? METIS_OK : METIS_ERR_CUDA;
-}
-
 template <int NB>
 metis_status_t launch(const CUtensorMap& mx, const CUtensorMap& mb, const CoeffArgs& g, dim3 grid, cudaStream_t s) {
   constexpr size_t smem = (size_t)STAGES * (A_BYTES + NB * BK * 2) + 1024 + 128;
@@ -218,8 +207,8 @@ bool metis_coeff_tc_usable(const void* x, const void* bs, int64_t cols, int kp) 
 metis_status_t metis_launch_coeff_tc(metis_context* ctx, const void* x, int64_t rows, int64_t cols, const void* bs, int kp,
                                      float* part, float* amax, cudaStream_t s) {
   CUtensorMap mx, mb;
-  METIS_TRY(make_map_bf16(ctx, &mx, x, rows, cols, BM));
-  METIS_TRY(make_map_bf16(ctx, &mb, bs, 3 * (int64_t)kp, cols, 3 * kp));
+  METIS_TRY(make_map_bf16(ctx, &mx, x, rows, cols, cols, BM));
+  METIS_TRY(make_map_bf16(ctx, &mb, bs, 3 * (int64_t)kp, cols, cols, 3 * kp));
   CoeffArgs g{};
   g.part = part; g.amax = amax; g.rows = rows; g.kp = kp;
   g.num_chunks = (int)metis_ceil_div(cols, BK);

@@ -1,0 +1,361 @@
+// Fused residual + NVFP4 quantizer of the split (Section 3.2: the residual is taken against the unquantized
+// factors and quantized on its own):
+//
+//   R = x - C B^T          on 128 x 128 tiles, never written to HBM in high precision (unless `dense` is asked for)
+//
+// C (rows x k) and B (cols x k) are FP32; their product runs on the tcgen05 tensor cores with FP32 accuracy by
+// feeding three-term BF16 splits: the six significant cross products are laid side by side along K,
+//   A6[r] = [Ch | Ch | Cl | Ch | Cl2 | Cl],   B6[c] = [Bh | Bl | Bh | Bl2 | Bh | Bl]      (K = 6*kp, padded to 64s)
+// so one chain of `tcgen05.mma.kind::f16` (M = 128, N = 128) accumulates all of them in tensor memory.
+//
+// Persistent CTAs, warp-specialised: a TMA producer streams A6 / B6 in 64-wide K chunks through a three-slot
+// ring and the x tile into a double buffer; one warp issues the MMAs into a double-buffered accumulator; eight
+// epilogue warps turn accumulator and x into NVFP4.  An epilogue thread owns one row and 64 of its columns:
+// it subtracts in registers and encodes the blocks that run along the columns straight from registers.  For
+// the blocks that run along the rows the warp transposes its 32 x 32 patch through a private piece of shared
+// memory (a warp's 32 rows hold whole 16-row blocks), so the epilogue has no CTA-wide barrier at all.
+// Every mbarrier wait is bounded; on expiry the kernel records METIS_DEV_TIMEOUT and unwinds.
+#include <cuda.h>
+
+#include "quant_tile.cuh"
+#include "tc_ptx.cuh"
+
+namespace {
+
+using namespace metis_tc;
+using metis_qt::QuantParams;
+using metis_qt::encode_block;
+
+constexpr int TM = 128, TN = 128, BK = 64;
+constexpr int RING = 3;
+constexpr int SLOT_BYTES = 2 * TM * BK * 2;               // A6 chunk + B6 chunk, 16 KiB each
+constexpr int X_BYTES = TM * TN * 2;                      // two 64-column boxes of 16 KiB
+constexpr int PATCH_F = 32 * 33;                          // floats per warp patch
+constexpr int PATCH_U = 32 * 34;                          // 16-bit draws per warp patch
+constexpr int NUM_THREADS = 320;                          // producer, MMA issuer, 8 epilogue warps
+constexpr size_t SMEM_BYTES = (size_t)RING * SLOT_BYTES + 2 * X_BYTES + 8 * (PATCH_F * 4 + PATCH_U * 2) + 1024 + 256;
+
+struct ResidArgs {
+  QuantParams p;
+  const float* amax_src;
+  float* ts_out0; float* ts_out1;
+  float* dense;
+  int k_chunks;             // 64-wide K chunks of A6 / B6
+  uint32_t* dev_status;
+};
+
+// splits of eight consecutive FP32 values into BF16 hi / lo / lo2, packed two per word
+__device__ __forceinline__ void split3x8(const float (&v)[8], uint4& h, uint4& l, uint4& l2) {
+  uint32_t hh[4], ll[4], mm[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float x = v[2 * i], y = v[2 * i + 1];
+    const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
+    const float xr = x - __bfloat162float(xh), yr = y - __bfloat162float(yh);
+    const __nv_bfloat16 xl = __float2bfloat16_rn(xr), yl = __float2bfloat16_rn(yr);
+    const __nv_bfloat16 xm = __float2bfloat16_rn(xr - __bfloat162float(xl)), ym = __float2bfloat16_rn(yr - __bfloat162float(yl));
+    hh[i] = (uint32_t)__bfloat16_as_ushort(xh) | ((uint32_t)__bfloat16_as_ushort(yh) << 16);
+    ll[i] = (uint32_t)__bfloat16_as_ushort(xl) | ((uint32_t)__bfloat16_as_ushort(yl) << 16);
+    mm[i] = (uint32_t)__bfloat16_as_ushort(xm) | ((uint32_t)__bfloat16_as_ushort(ym) << 16);
+  }
+  h = make_uint4(hh[0], hh[1], hh[2], hh[3]); l = make_uint4(ll[0], ll[1], ll[2], ll[3]); l2 = make_uint4(mm[0], mm[1], mm[2], mm[3]);
+}
+
+// out[i][6*kp padded to kx] for vector i: pattern A = [h|h|l|h|l2|l] (coefficients), pattern B = [h|l|h|l2|h|l] (basis).
+// src element (i, j): src[i*stride_i + j*stride_j], j < k (zero beyond).  One thread per (i, group of 8 j).
+__global__ void __launch_bounds__(256)
+splits6_kernel(const float* __restrict__ src, int64_t n, int k, int kp, int kx, int64_t stride_i, int64_t stride_j, int pattern_b,
+               __nv_bfloat16* __restrict__ out) {
+  const int groups = kx / 8;
+  const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= n * groups) return;
+  const int64_t i = idx / groups;
+  const int gq = (int)(idx % groups);
+  uint4* dst = reinterpret_cast<uint4*>(out + i * kx) + gq;
+  const int term = (gq * 8) / kp, j0 = (gq * 8) % kp;      // which of the six blocks, where inside it
+  if (term >= 6) { *dst = make_uint4(0u, 0u, 0u, 0u); return; }
+  float v[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) v[e] = (j0 + e < k) ? src[i * stride_i + (int64_t)(j0 + e) * stride_j] : 0.0f;
+  uint4 h, l, l2;
+  split3x8(v, h, l, l2);
+  // term:        0  1  2  3   4   5
+  // pattern A:   h  h  l  h   l2  l
+  // pattern B:   h  l  h  l2  h   l
+  const int sel_a[6] = {0, 0, 1, 0, 2, 1}, sel_b[6] = {0, 1, 0, 2, 0, 1};
+  const int sel = pattern_b ? sel_b[term] : sel_a[term];
+  *dst = sel == 0 ? h : (sel == 1 ? l : l2);
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_a,
+                   const __grid_constant__ CUtensorMap map_b, ResidArgs g) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* gen_base = smem_raw + (base - raw);
+  auto a_addr = [&](int s) { return base + (uint32_t)s * SLOT_BYTES; };
+  auto b_addr = [&](int s) { return a_addr(s) + TM * BK * 2; };
+  auto x_addr = [&](int xb) { return base + (uint32_t)RING * SLOT_BYTES + (uint32_t)xb * X_BYTES; };
+  const size_t patch_off = (size_t)RING * SLOT_BYTES + 2 * X_BYTES;
+  const uint32_t bar_base = base + (uint32_t)(patch_off + 8 * (PATCH_F * 4 + PATCH_U * 2));
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (RING + s); };
+  auto xfull_bar = [&](int xb) { return bar_base + 8u * (2 * RING + xb); };
+  auto xempty_bar = [&](int xb) { return bar_base + 8u * (2 * RING + 2 + xb); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * RING + 4 + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * RING + 6 + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + patch_off + 8 * (PATCH_F * 4 + PATCH_U * 2) + 8 * (2 * RING + 8));
+  volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const QuantParams& p = g.p;
+  const int n_ct = (int)((p.cols + TN - 1) / TN), n_rt = (int)((p.rows + TM - 1) / TM);
+  const int num_tiles = n_ct * n_rt;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < RING; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(xfull_bar(b), 1); mbar_init(xempty_bar(b), 8);
+      mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8);
+    }
+    *dead = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 256);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------- producer -------------------------------
+    int s = 0; uint32_t ph = 0;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      const int row0 = (tile / n_ct) * TM, col0 = (tile % n_ct) * TN;
+      const int xb = it & 1;
+      if (!mbar_wait(xempty_bar(xb), (((uint32_t)it >> 1) & 1u) ^ 1u, g.dev_status, dead)) { ok = false; break; }
+      if (elect_one()) {
+        mbar_expect_tx(xfull_bar(xb), (uint32_t)X_BYTES);
+        tma_load_2d(x_addr(xb), &map_x, col0, row0, xfull_bar(xb));
+        tma_load_2d(x_addr(xb) + X_BYTES / 2, &map_x, col0 + 64, row0, xfull_bar(xb));
+      }
+      __syncwarp();
+      for (int ck = 0; ck < g.k_chunks; ++ck) {
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, g.dev_status, dead)) { ok = false; break; }
+        if (elect_one()) {
+          mbar_expect_tx(full_bar(s), (uint32_t)SLOT_BYTES);
+          tma_load_2d(a_addr(s), &map_a, ck * BK, row0, full_bar(s));
+          tma_load_2d(b_addr(s), &map_b, ck * BK, col0, full_bar(s));
+        }
+        __syncwarp();
+        if (++s == RING) { s = 0; ph ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer -----------------------------
+    constexpr uint32_t idesc = make_idesc_bf16(TM, TN);
+    int s = 0; uint32_t ph = 0;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      const int acc = it & 1;
+      if (!mbar_wait(tempty_bar(acc), (((uint32_t)it >> 1) & 1u) ^ 1u, g.dev_status, dead)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TN);
+      for (int ck = 0; ck < g.k_chunks; ++ck) {
+        if (!mbar_wait(full_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
+        tc_fence_after();
+        if (elect_one()) {
+          const uint64_t a_d = make_smem_desc(a_addr(s), 1024, SWIZZLE_128B), b_d = make_smem_desc(b_addr(s), 1024, SWIZZLE_128B);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)
+            tc_mma_bf16(d_tmem, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc, (ck | k) != 0 ? 1u : 0u);
+          tc_commit(empty_bar(s));
+        }
+        __syncwarp();
+        if (++s == RING) { s = 0; ph ^= 1u; }
+      }
+      if (ok && elect_one()) tc_commit(tfull_bar(acc));
+      __syncwarp();
+    }
+  } else {
+    // ------------------------------- epilogue -------------------------------
+    const int ew = warp - 2;                                // 0..7
+    const int quarter = warp & 3, half = ew >> 2;           // TMEM lane quarter (fixed by the warp id), column half
+    float* patch = reinterpret_cast<float*>(gen_base + patch_off) + ew * PATCH_F;
+    uint16_t* upatch = reinterpret_cast<uint16_t*>(gen_base + patch_off + 8 * PATCH_F * 4) + ew * PATCH_U;
+    const bool sr = p.rounding == METIS_ROUND_SR;
+    const float s_T = metis_tensor_scale(*g.amax_src);
+    const float six_s_T = __fmul_rn(6.0f, s_T);
+    if (blockIdx.x == 0 && threadIdx.x == 64) {
+      if (g.ts_out0) *g.ts_out0 = s_T;
+      if (g.ts_out1) *g.ts_out1 = s_T;
+    }
+    const int64_t c_kbytes = p.cols / 2, r_kbytes = p.rows / 2, c_bpr = p.cols / 16, r_bpr = p.rows / 16;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      const int row0 = (tile / n_ct) * TM, col0 = (tile % n_ct) * TN;
+      const int acc = it & 1, xb = it & 1;
+      const uint32_t par = ((uint32_t)it >> 1) & 1u;
+      if (!mbar_wait(xfull_bar(xb), par, g.dev_status, dead)) { ok = false; break; }
+      if (!mbar_wait(tfull_bar(acc), par, g.dev_status, dead)) { ok = false; break; }
+      tc_fence_after();
+      const int64_t row = (int64_t)row0 + quarter * 32 + lane;              // this thread's row
+      const bool row_ok = row < p.rows;
+      const int64_t slab_row0 = (int64_t)row0 + quarter * 32;               // first row of the warp's 32
+      const uint32_t xrow = x_addr(xb) + (uint32_t)half * (X_BYTES / 2) + (uint32_t)(quarter * 32 + lane) * 128u;
+      const uint32_t sw = (uint32_t)((quarter * 32 + lane) & 7);
+#pragma unroll 1
+      for (int cc = 0; cc < 2; ++cc) {
+        const int64_t c0 = (int64_t)col0 + half * 64 + cc * 32;             // first of this step's 32 columns
+        uint32_t a[32];
+        tc_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * TN + half * 64 + cc * 32), a);
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint32_t w0, w1, w2, w3;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
+                       : "r"(xrow + ((((uint32_t)(4 * cc + j)) ^ sw) << 4)));
+          const uint32_t ws[4] = {w0, w1, w2, w3};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            v[8 * j + 2 * e] = __uint_as_float(ws[e] << 16) - __uint_as_float(a[8 * j + 2 * e]);
+            v[8 * j + 2 * e + 1] = __uint_as_float(ws[e] & 0xFFFF0000u) - __uint_as_float(a[8 * j + 2 * e + 1]);
+          }
+        }
+        if (cc == 1) {
+          // accumulator and x tile fully read: hand both back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) { mbar_arrive(tempty_bar(acc)); mbar_arrive(xempty_bar(xb)); }
+        }
+        const bool step_ok = c0 < p.cols;                                    // false: the whole step lies outside the matrix
+        const bool blk1_ok = c0 + 16 < p.cols;
+        uint32_t u[32];
+        if (sr) {
+          const uint64_t e0 = (uint64_t)row * (uint64_t)p.e_stride_r + (uint64_t)c0;      // multiple of 8
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const uint4 w = metis_philox_block((e0 >> 3) + q4, p.seed, p.stream_id);
+#pragma unroll
+            for (uint32_t hh = 0; hh < 8; ++hh) u[8 * q4 + hh] = metis_u16_of(w, hh);
+          }
+        }
+        if (g.dense != nullptr && row_ok && step_ok) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (c0 + 4 * j < p.cols)
+              *reinterpret_cast<float4*>(g.dense + row * p.cols + c0 + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        }
+        if (p.c_codes != nullptr && step_ok) {
+          // blocks along the columns: two blocks of this row, from registers
+          float v0[16], v1[16];
+          uint32_t u0[16], u1[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { v0[i] = v[i]; v1[i] = v[16 + i]; u0[i] = sr ? u[i] : 0u; u1[i] = sr ? u[16 + i] : 0u; }
+          uint32_t pk0[2], pk1[2];
+          const uint32_t sb0 = encode_block(v0, u0, sr, s_T, six_s_T, pk0);
+          const uint32_t sb1 = encode_block(v1, u1, sr, s_T, six_s_T, pk1);
+          if (row_ok) {
+            uint8_t* cp = p.c_codes + row * c_kbytes + c0 / 2;
+            if (blk1_ok) *reinterpret_cast<uint4*>(cp) = make_uint4(pk0[0], pk0[1], pk1[0], pk1[1]);
+            else *reinterpret_cast<uint2*>(cp) = make_uint2(pk0[0], pk0[1]);
+          }
+          if (row_ok || p.c_layout == METIS_SF_TILED) {                     // padded rows of a 128-row slab get zero scales
+            const int64_t o = metis_sf_offset(row, c0 / 16, c_bpr, p.c_layout);
+            p.c_scales[o] = row_ok ? (uint8_t)sb0 : (uint8_t)0;
+            if (blk1_ok) p.c_scales[o + 1] = row_ok ? (uint8_t)sb1 : (uint8_t)0;
+          }
+        }
+        if (p.r_codes != nullptr && (step_ok || p.r_layout == METIS_SF_TILED)) {
+          // blocks along the rows: transpose the warp's 32 x 32 patch, lane = column
+#pragma unroll
+          for (int i = 0; i < 32; ++i) patch[lane * 33 + i] = v[i];
+          if (sr) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) upatch[lane * 34 + i] = (uint16_t)u[i];
+          }
+          __syncwarp();
+          const int64_t col = c0 + lane;
+          const bool col_ok = col < p.cols;
+          float t0[16], t1[16];
+          uint32_t d0[16], d1[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            t0[i] = patch[i * 33 + lane]; t1[i] = patch[(16 + i) * 33 + lane];
+            d0[i] = sr ? (uint32_t)upatch[i * 34 + lane] : 0u; d1[i] = sr ? (uint32_t)upatch[(16 + i) * 34 + lane] : 0u;
+          }
+          uint32_t pk0[2], pk1[2];
+          const uint32_t sb0 = encode_block(t0, d0, sr, s_T, six_s_T, pk0);
+          const uint32_t sb1 = encode_block(t1, d1, sr, s_T, six_s_T, pk1);
+          const bool rb0_ok = slab_row0 < p.rows, rb1_ok = slab_row0 + 16 < p.rows;
+          if (col_ok && rb0_ok) {
+            uint8_t* cp = p.r_codes + col * r_kbytes + slab_row0 / 2;
+            if (rb1_ok) *reinterpret_cast<uint4*>(cp) = make_uint4(pk0[0], pk0[1], pk1[0], pk1[1]);
+            else *reinterpret_cast<uint2*>(cp) = make_uint2(pk0[0], pk0[1]);
+          }
+          if (rb0_ok && (col_ok || p.r_layout == METIS_SF_TILED)) {         // padded columns of a 128-slab get zero scales
+            const int64_t o = metis_sf_offset(col, slab_row0 / 16, r_bpr, p.r_layout);
+            p.r_scales[o] = col_ok ? (uint8_t)sb0 : (uint8_t)0;
+            if (rb1_ok) p.r_scales[o + 1] = col_ok ? (uint8_t)sb1 : (uint8_t)0;
+          }
+          __syncwarp();
+        }
+      }
+    }
+  }
+
+  // ------------------------------- teardown ---------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (*dead) {
+    // a wait expired: give copies already in flight time to land before the shared memory is released
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 256);
+  }
+}
+
+}  // namespace
+
+int metis_residual_kx(int kp) { return (6 * kp + 63) / 64 * 64; }
+
+bool metis_residual_tc_usable(const void* x, int64_t cols) { return metis_aligned16(x) && cols % 8 == 0; }
+
+// a6: [rows][kx], b6: [cols][kx] BF16 scratch (kx = metis_residual_kx(kp)); coef: [rows][kp] FP32; basis: [k][cols] FP32.
+metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const float* coef, const float* basis, int k, int kp,
+                                        const metis_qt::QuantParams& qp, const float* amax_src, float* ts_out0, float* ts_out1,
+                                        float* dense, void* a6, void* b6, cudaStream_t s) {
+  const int kx = metis_residual_kx(kp);
+  const int64_t rows = qp.rows, cols = qp.cols;
+  splits6_kernel<<<(unsigned)metis_ceil_div(rows * (kx / 8), 256), 256, 0, s>>>(coef, rows, k, kp, kx, kp, 1, 0,
+                                                                                reinterpret_cast<__nv_bfloat16*>(a6)); METIS_COUNT_LAUNCH();
+  splits6_kernel<<<(unsigned)metis_ceil_div(cols * (kx / 8), 256), 256, 0, s>>>(basis, cols, k, kp, kx, 1, cols, 1,
+                                                                                reinterpret_cast<__nv_bfloat16*>(b6)); METIS_COUNT_LAUNCH();
+  CUtensorMap mx, ma, mb;
+  METIS_TRY(make_map_bf16(ctx, &mx, x, rows, cols, cols, TM));
+  METIS_TRY(make_map_bf16(ctx, &ma, a6, rows, kx, kx, TM));
+  METIS_TRY(make_map_bf16(ctx, &mb, b6, cols, kx, kx, TN));
+  ResidArgs g{};
+  g.p = qp; g.amax_src = amax_src; g.ts_out0 = ts_out0; g.ts_out1 = ts_out1; g.dense = dense;
+  g.k_chunks = kx / BK;
+  g.dev_status = ctx->dev_status;
+  static bool attr = false;
+  if (!attr) {
+    METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    attr = true;
+  }
+  const int64_t tiles = metis_ceil_div(rows, TM) * metis_ceil_div(cols, TN);
+  const int grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);
+  residual_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(mx, ma, mb, g); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}

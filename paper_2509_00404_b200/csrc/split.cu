@@ -7,6 +7,10 @@
 //   with the NVFP4 quantizer in both block orientations -> factor rotation, sign fix, factor quantization.
 #include "quant_tile.cuh"
 
+metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const float* coef, const float* basis, int k, int kp,
+                                        const metis_qt::QuantParams& qp, const float* amax_src, float* ts_out0, float* ts_out1,
+                                        float* dense, void* a6, void* b6, cudaStream_t s);
+
 namespace {
 
 constexpr int MAXQ = 72;                               // k + p at most (k = 64 with p = 8)
@@ -1057,7 +1061,7 @@ left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, i
 
 struct SplitWs {
   size_t amax, idx, zp, z, gram, gram1, linv, evals, evecs, mp, m, basis, coef, sign, cand_v, cand_i, evals2, evecs2, bs, bt,
-      gram_c, part, total;
+      gram_c, part, a6, b6, total;
 };
 
 constexpr int PJ_MAX_PARTS = 16;
@@ -1095,6 +1099,8 @@ SplitWs split_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s) {
   const int kp = (k + 15) / 16 * 16;
   w.coef = take(sizeof(float) * (size_t)kp * rows);
   w.part = take(sizeof(float) * (size_t)metis_coeff_slices(rows, cols, nullptr) * kp * rows);
+  w.a6 = take(sizeof(__nv_bfloat16) * (size_t)metis_residual_kx(kp) * rows);
+  w.b6 = take(sizeof(__nv_bfloat16) * (size_t)metis_residual_kx(kp) * cols);
   w.bs = take(sizeof(__nv_bfloat16) * 3 * (size_t)kp * cols);
   w.bt = take(sizeof(__nv_bfloat16) * 3 * (size_t)kp * cols);
   w.gram_c = take(sizeof(double) * (size_t)metis_ceil_div(rows, 32) * kp * kp);
@@ -1225,6 +1231,8 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   __nv_bfloat16* bt = reinterpret_cast<__nv_bfloat16*>(wsb + L.bt);
   double* gram_c = reinterpret_cast<double*>(wsb + L.gram_c);
   float* part = reinterpret_cast<float*>(wsb + L.part);
+  void* a6 = wsb + L.a6;
+  void* b6 = wsb + L.b6;
   metis_context* ctx = h;
   const int kp = (k + 15) / 16 * 16;
   {
@@ -1371,13 +1379,17 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     // goes to a (high-priority) side stream and is joined back at the end of the call
     METIS_TRY(metis_fork(ctx, s, 1));
     cudaStream_t sr = s;
-    switch (kp) {
-      case 16: residual_quant_kernel<16><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
-      case 32: residual_quant_kernel<32><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
-      case 48: residual_quant_kernel<48><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
-      default: residual_quant_kernel<64><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+    if (metis_residual_tc_usable(x, cols)) {
+      METIS_TRY(metis_launch_residual_tc(ctx, x, coef, full ? out->right : basis, k, kp, qp, amax, t0, t1, residual_dense, a6, b6, sr));
+    } else {
+      switch (kp) {
+        case 16: residual_quant_kernel<16><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+        case 32: residual_quant_kernel<32><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+        case 48: residual_quant_kernel<48><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+        default: residual_quant_kernel<64><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+      }
+      METIS_COUNT_LAUNCH();
     }
-    METIS_COUNT_LAUNCH();
   }
   cudaStream_t sf = ctx->side[0];
   if (!full) {
