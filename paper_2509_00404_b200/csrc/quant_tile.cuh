@@ -29,9 +29,11 @@ struct __align__(16) Stage {
 // Encodes one block of 16 values; returns the scale byte, writes 8 code bytes.
 __device__ __forceinline__ uint32_t encode_block(const float (&v)[16], const uint32_t (&u)[16], bool sr, float s_T,
                                                  float six_s_T, uint32_t (&packed)[2]) {
-  float amax = 0.0f;
+  // maximum by a tree: four dependent steps instead of sixteen
+  float m8[8];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+  for (int i = 0; i < 8; ++i) m8[i] = fmaxf(fabsf(v[i]), fabsf(v[i + 8]));
+  const float amax = fmaxf(fmaxf(fmaxf(m8[0], m8[4]), fmaxf(m8[1], m8[5])), fmaxf(fmaxf(m8[2], m8[6]), fmaxf(m8[3], m8[7])));
   float t = fminf(__fdiv_rn(amax, six_s_T), 448.0f);
   float sb;
   const uint32_t byte = metis_e4m3_ceil(t, &sb);
