@@ -316,6 +316,24 @@ def main():
     gemm_ms = g0.elapsed_time(g1) / (3 * reps)
     # plain (k = 0) layer time for the overhead figure: three GEMMs only
     overhead = ms / (3 * gemm_ms) - 1.0
+
+    # ---- split + quantize of each operand alone (algorithmic bytes: 2 B read + 2 x 0.5625 B written per element) ----
+    def alone(fn, reps=10):
+        fn(0)
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for r_ in range(reps):
+            fn(r_)
+        a1.record()
+        torch.cuda.synchronize()
+        return a0.elapsed_time(a1) / reps
+    ms_sx = alone(lambda i: h_x.split(dev_sets[i % N_SETS]["x"], k, p, sketch=B.SKETCH_SAMPLED, seed=i + 1, out=xo))
+    ms_sw = alone(lambda i: h_x.split(dev_sets[i % N_SETS]["w"], k, p, sketch=B.SKETCH_FULL, seed=i + 2, out=wo))
+    ms_sd = alone(lambda i: h_x.split(dev_sets[i % N_SETS]["dy"], k, p, sketch=B.SKETCH_SAMPLED, seed=i + 3, rounding=B.ROUND_SR, out=do))
+    qc, qr = B.NvFp4(l, m), B.NvFp4(m, l)
+    ms_q = alone(lambda i: h_x.quantize_nvfp4(dev_sets[i % N_SETS]["x"], B.BLOCKS_BOTH, B.ROUND_RNE, seed=1, tensor_scale=1.0, out=(qc, qr)))
+    split_gbs = lambda elems, t_ms: 3.125 * elems / (t_ms * 1e-3) / 1e9
     clocks = sampler.stop()
 
     times = torch.tensor([ms, ms_e2e], dtype=torch.float64, device="cuda")
@@ -346,6 +364,12 @@ def main():
                      "algorithmic_bytes": 0.5625 * 2 * l * m + 2.0 * l * n, "peak_source": "bf16 burst peak (%s) x %.0f nominal FP4:bf16 ratio" % (peaks["source"], FP4_OVER_BF16),
                      "ms_per_launch": gemm_ms},
         "split_overhead_vs_three_plain_gemms": overhead,
+        "split_quantize": {"unit": "GB/s of algorithmic bytes (3.125 B per element, both block orientations)",
+                           "hbm_peak_gbs": peaks["hbm_gbs"],
+                           "x_sampled": {"ms": ms_sx, "gbs": split_gbs(l * m, ms_sx)},
+                           "w_full": {"ms": ms_sw, "gbs": split_gbs(n * m, ms_sw)},
+                           "dy_sampled_sr": {"ms": ms_sd, "gbs": split_gbs(l * n, ms_sd)},
+                           "plain_quantizer_rne_given_scale": {"ms": ms_q, "gbs": split_gbs(l * m, ms_q), "frac_of_hbm": split_gbs(l * m, ms_q) / peaks["hbm_gbs"]}},
         "device_status": status,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -117,8 +117,8 @@ metis_status_t metis_workspace_bytes(int32_t op, int64_t rows, int64_t cols, int
   switch (op) {
     case 0: *bytes = 256; return METIS_OK;
     case 1: *bytes = metis_split_ws_bytes(rows, cols, k, p); return METIS_OK;
-    case 2:
-    case 3: *bytes = metis_linear_ws_bytes(rows, cols, k); return METIS_OK;
+    case 2: *bytes = metis_linear_ws_bytes(rows, cols, k); return METIS_OK;
+    case 3: *bytes = 2 * metis_linear_ws_bytes(rows, cols, k); return METIS_OK;    // two products' intermediates side by side
     default: return METIS_ERR_INVALID_ARG;
   }
 }

@@ -278,56 +278,95 @@ metis_status_t check_nvfp4(const metis_nvfp4_t* t) {
   return METIS_OK;
 }
 
-metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void* d, int d_dtype, int64_t ldd, void* ws,
-                          size_t ws_bytes, cudaStream_t s) {
+// Where the intermediates of one product live inside the caller's workspace.
+struct Plan {
+  int64_t M, N, K;
+  int ka, kb, kc, kx;
+  bool fuse;
+  float *pm, *lcat, *rcat, *y0;
+  __nv_bfloat16 *lx, *rx;
+  size_t bytes;
+};
+
+metis_status_t make_plan(const Side& a, const Side& b, void* ws, size_t ws_bytes, Plan* pl) {
   METIS_TRY(check_nvfp4(a.res));
   METIS_TRY(check_nvfp4(b.res));
-  const int64_t M = a.res->rows, N = b.res->rows, K = a.res->k_len;
-  if (b.res->k_len != K) return METIS_ERR_SHAPE;
-  const int ka = a.k, kb = b.k, kc = ka + kb;
-  if (kc == 0) return metis_launch_gemm_tc(ctx, a.res, b.res, d, d_dtype, ldd, s);
+  pl->M = a.res->rows; pl->N = b.res->rows; pl->K = a.res->k_len;
+  if (b.res->k_len != pl->K) return METIS_ERR_SHAPE;
+  pl->ka = a.k; pl->kb = b.k; pl->kc = a.k + b.k; pl->bytes = 0;
+  if (pl->kc == 0) return METIS_OK;
+  const int64_t M = pl->M, N = pl->N, K = pl->K;
+  const int ka = a.k, kb = b.k, kc = pl->kc;
   if (ka > 64 || kb > 64) return METIS_ERR_SHAPE;
   if (ka) { METIS_TRY(check_nvfp4(a.fc)); METIS_TRY(check_nvfp4(a.fo)); if (a.fc->k_len != K || a.fo->k_len != M || !a.sigma) return METIS_ERR_SHAPE; }
   if (kb) { METIS_TRY(check_nvfp4(b.fc)); METIS_TRY(check_nvfp4(b.fo)); if (b.fc->k_len != K || b.fo->k_len != N || !b.sigma) return METIS_ERR_SHAPE; }
   unsigned char* w = reinterpret_cast<unsigned char*>(ws);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
-  const bool fuse = metis_gemm_tc_can_fuse(a.res, b.res);
-  const int kx = (3 * kc + 63) / 64 * 64;
-  float* pm = reinterpret_cast<float*>(w + take(sizeof(float) * 64 * 64));
-  float* lcat = reinterpret_cast<float*>(w + take(sizeof(float) * M * kc));
-  float* rcat = reinterpret_cast<float*>(w + take(sizeof(float) * N * kc));
-  __nv_bfloat16* lx = fuse ? reinterpret_cast<__nv_bfloat16*>(w + take(sizeof(__nv_bfloat16) * M * kx)) : nullptr;
-  __nv_bfloat16* rx = fuse ? reinterpret_cast<__nv_bfloat16*>(w + take(sizeof(__nv_bfloat16) * N * kx)) : nullptr;
-  float* y0 = fuse ? nullptr : reinterpret_cast<float*>(w + take(sizeof(float) * M * N));
+  pl->fuse = metis_gemm_tc_can_fuse(a.res, b.res);
+  pl->kx = (3 * kc + 63) / 64 * 64;
+  const size_t o_pm = take(sizeof(float) * 64 * 64), o_l = take(sizeof(float) * M * kc), o_r = take(sizeof(float) * N * kc);
+  const size_t o_lx = pl->fuse ? take(sizeof(__nv_bfloat16) * M * pl->kx) : 0, o_rx = pl->fuse ? take(sizeof(__nv_bfloat16) * N * pl->kx) : 0;
+  const size_t o_y0 = pl->fuse ? 0 : take(sizeof(float) * M * N);
+  pl->bytes = off;
   if (!ws || off > ws_bytes) return METIS_ERR_WORKSPACE;
+  pl->pm = reinterpret_cast<float*>(w + o_pm); pl->lcat = reinterpret_cast<float*>(w + o_l); pl->rcat = reinterpret_cast<float*>(w + o_r);
+  pl->lx = pl->fuse ? reinterpret_cast<__nv_bfloat16*>(w + o_lx) : nullptr;
+  pl->rx = pl->fuse ? reinterpret_cast<__nv_bfloat16*>(w + o_rx) : nullptr;
+  pl->y0 = pl->fuse ? nullptr : reinterpret_cast<float*>(w + o_y0);
+  return METIS_OK;
+}
 
-  if (!fuse) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.res, y0, METIS_FP32, N, s));
-  // the skinny products land directly in their slots of the concatenated operands; they are independent of
-  // each other and run side by side
-  METIS_TRY(metis_fork(ctx, s, 2));
-  if (kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.fc, lcat, METIS_FP32, kc, s));
-  if (ka) METIS_TRY(metis_launch_gemm_tc(ctx, b.res, a.fc, rcat + kb, METIS_FP32, kc, ctx->side[0]));
-  if (ka && kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.fc, b.fc, pm, METIS_FP32, kb, ctx->side[1]));
-  METIS_TRY(metis_join(ctx, s, 0));
-  METIS_TRY(metis_join(ctx, s, 1));
+// Everything of a product that comes before its large GEMM: the three skinny products (straight into their
+// slots of the concatenated operands) and the finishing kernel.  `side_by_side`: the skinny products run on
+// the handle's streams 0 and 1 beside `s`; otherwise one after the other on `s`.
+metis_status_t split_gemm_prologue(metis_context* ctx, const Side& a, const Side& b, const Plan& pl, bool side_by_side,
+                                   cudaStream_t s) {
+  if (pl.kc == 0) return METIS_OK;
+  const int64_t M = pl.M, N = pl.N;
+  const int ka = pl.ka, kb = pl.kb, kc = pl.kc;
+  if (!pl.fuse) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.res, pl.y0, METIS_FP32, N, s));
+  cudaStream_t s1 = side_by_side ? ctx->side[0] : s, s2 = side_by_side ? ctx->side[1] : s;
+  if (side_by_side) METIS_TRY(metis_fork(ctx, s, 2));
+  if (kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.fc, pl.lcat, METIS_FP32, kc, s));
+  if (ka) METIS_TRY(metis_launch_gemm_tc(ctx, b.res, a.fc, pl.rcat + kb, METIS_FP32, kc, s1));
+  if (ka && kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.fc, b.fc, pl.pm, METIS_FP32, kb, s2));
+  if (side_by_side) {
+    METIS_TRY(metis_join(ctx, s, 0));
+    METIS_TRY(metis_join(ctx, s, 1));
+  }
   const int64_t mx = M > N ? M : N;
   lowrank_finish_kernel<<<(unsigned)metis_ceil_div(mx, 8), 256, 0, s>>>(
       M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
       ka ? a.fo->tensor_scale : nullptr, a.sigma, kb ? b.fo->codes : nullptr, kb ? b.fo->scales : nullptr,
-      kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, pm, lcat, rcat, lx, rx, kx,
+      kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, pl.pm, pl.lcat, pl.rcat, pl.lx, pl.rx, pl.kx,
       a.res->tensor_scale, b.res->tensor_scale); METIS_COUNT_LAUNCH();
-  if (fuse) {
-    // residual x residual product and the rank-(ka+kb) correction accumulate into one FP32 tile in tensor memory
-    return metis_launch_gemm_tc_fused(ctx, a.res, b.res, d, d_dtype, ldd, lx, rx, kx, s);
-  }
-  dim3 grid((unsigned)metis_ceil_div(N, 64), (unsigned)metis_ceil_div(M, 64));
-  const size_t smem = sizeof(float) * 2 * kc * 68;
-  static bool attr = false;
-  if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(rank_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 2 * 128 * 68))); attr = true; }
-  rank_update_kernel<<<grid, 256, smem, s>>>(y0, M, N, kc, lcat, rcat, d, d_dtype, ldd); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
+}
+
+metis_status_t split_gemm_main(metis_context* ctx, const Side& a, const Side& b, const Plan& pl, void* d, int d_dtype, int64_t ldd,
+                               cudaStream_t s) {
+  if (pl.kc == 0) return metis_launch_gemm_tc(ctx, a.res, b.res, d, d_dtype, ldd, s);
+  if (pl.fuse) {
+    // residual x residual product and the rank-(ka+kb) correction accumulate into one FP32 tile in tensor memory
+    return metis_launch_gemm_tc_fused(ctx, a.res, b.res, d, d_dtype, ldd, pl.lx, pl.rx, pl.kx, s);
+  }
+  dim3 grid((unsigned)metis_ceil_div(pl.N, 64), (unsigned)metis_ceil_div(pl.M, 64));
+  const size_t smem = sizeof(float) * 2 * pl.kc * 68;
+  static bool attr = false;
+  if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(rank_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 2 * 128 * 68))); attr = true; }
+  rank_update_kernel<<<grid, 256, smem, s>>>(pl.y0, pl.M, pl.N, pl.kc, pl.lcat, pl.rcat, d, d_dtype, ldd); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
+
+metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void* d, int d_dtype, int64_t ldd, void* ws,
+                          size_t ws_bytes, cudaStream_t s) {
+  Plan pl;
+  METIS_TRY(make_plan(a, b, ws, ws_bytes, &pl));
+  METIS_TRY(split_gemm_prologue(ctx, a, b, pl, true, s));
+  return split_gemm_main(ctx, a, b, pl, d, d_dtype, ldd, s);
 }
 
 }  // namespace
@@ -359,23 +398,43 @@ metis_status_t metis_linear_bwd(metis_handle_t h, const metis_operand_t* dy, con
   if (!h || !dy) return METIS_ERR_INVALID_ARG;
   if ((d_left || d_sigma || d_right) && (!dw || !w)) return METIS_ERR_INVALID_ARG;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  if (dx) {
-    if (!w || dy->cols != w->rows) return METIS_ERR_SHAPE;
-    // dX (l x m) = D W_t, contraction over out-features n: D by columns, W_t by rows (stored m x n)
-    Side a{&dy->res_by_cols, &dy->right_q, &dy->left_q, dy->sigma, dy->k};
-    Side b{&w->res_by_rows, &w->left_q, &w->right_q, w->sigma, w->k};
-    METIS_TRY(split_gemm(h, a, b, dx, dx_dtype, lddx, ws, ws_bytes, s));
-  }
-  if (dw) {
-    if (!x || dy->rows != x->rows) return METIS_ERR_SHAPE;
-    // dW_t (n x m) = D^T X, contraction over tokens l: both by rows (stored n x l and m x l)
-    Side a{&dy->res_by_rows, &dy->left_q, &dy->right_q, dy->sigma, dy->k};
-    Side b{&x->res_by_rows, &x->left_q, &x->right_q, x->sigma, x->k};
-    METIS_TRY(split_gemm(h, a, b, dw, dw_dtype, lddw, ws, ws_bytes, s));
-    if (d_left || d_sigma || d_right) {
-      if (w->rows != dy->cols || w->cols != x->cols) return METIS_ERR_SHAPE;
-      METIS_TRY(factor_grads(h, dw, dw_dtype, lddw, w, d_left, d_sigma, d_right, ws, ws_bytes, s));
+  if (dx && (!w || dy->cols != w->rows)) return METIS_ERR_SHAPE;
+  if (dw && (!x || dy->rows != x->rows)) return METIS_ERR_SHAPE;
+  // dX (l x m) = D W_t, contraction over out-features n: D by columns, W_t by rows (stored m x n)
+  Side da{&dy->res_by_cols, &dy->right_q, &dy->left_q, dy->sigma, dy->k};
+  Side db = w ? Side{&w->res_by_rows, &w->left_q, &w->right_q, w->sigma, w->k} : Side{};
+  // dW_t (n x m) = D^T X, contraction over tokens l: both by rows (stored n x l and m x l)
+  Side wa{&dy->res_by_rows, &dy->left_q, &dy->right_q, dy->sigma, dy->k};
+  Side wb = x ? Side{&x->res_by_rows, &x->left_q, &x->right_q, x->sigma, x->k} : Side{};
+  if (dx && dw) {
+    // Both products: with room for two sets of intermediates, everything that precedes the weight gradient's
+    // large GEMM runs on a side stream underneath the input gradient.
+    Plan pd, pw;
+    METIS_TRY(make_plan(da, db, ws, ws_bytes, &pd));
+    const size_t off = pd.bytes;
+    const metis_status_t st = make_plan(wa, wb, ws ? reinterpret_cast<unsigned char*>(ws) + off : nullptr,
+                                        ws_bytes > off ? ws_bytes - off : 0, &pw);
+    if (st == METIS_OK) {
+      METIS_TRY(metis_fork(h, s, 3));
+      METIS_TRY(split_gemm_prologue(h, wa, wb, pw, false, h->side[2]));
+      METIS_TRY(split_gemm_prologue(h, da, db, pd, true, s));
+      METIS_TRY(split_gemm_main(h, da, db, pd, dx, dx_dtype, lddx, s));
+      METIS_TRY(metis_join(h, s, 2));
+      METIS_TRY(split_gemm_main(h, wa, wb, pw, dw, dw_dtype, lddw, s));
+    } else if (st == METIS_ERR_WORKSPACE) {
+      METIS_TRY(split_gemm(h, da, db, dx, dx_dtype, lddx, ws, ws_bytes, s));
+      METIS_TRY(split_gemm(h, wa, wb, dw, dw_dtype, lddw, ws, ws_bytes, s));
+    } else {
+      return st;
     }
+  } else if (dx) {
+    METIS_TRY(split_gemm(h, da, db, dx, dx_dtype, lddx, ws, ws_bytes, s));
+  } else if (dw) {
+    METIS_TRY(split_gemm(h, wa, wb, dw, dw_dtype, lddw, ws, ws_bytes, s));
+  }
+  if (dw && (d_left || d_sigma || d_right)) {
+    if (w->rows != dy->cols || w->cols != x->cols) return METIS_ERR_SHAPE;
+    METIS_TRY(factor_grads(h, dw, dw_dtype, lddw, w, d_left, d_sigma, d_right, ws, ws_bytes, s));
   }
   return METIS_OK;
 }
