@@ -242,6 +242,53 @@ metis_status_t metis_launch_amax(const void* x, int dtype, int64_t rows, int64_t
   return METIS_OK;
 }
 
+
+// Few long rows (the transposed split factors: k x len FP32, blocks along the contiguous dimension only): one
+// thread per block of 16, no tiles, no shared memory.  Threads beyond `rows` inside the last 128-row slab of the
+// tiled scale layout write zero scale bytes.
+__global__ void __launch_bounds__(256)
+quantize_rowblocks_kernel(const float* __restrict__ x, int64_t ld, metis_qt::QuantParams p, const float* __restrict__ tscale_src,
+                          int tscale_is_amax, float* ts_out) {
+  const int64_t bpr = p.cols / 16;
+  const int64_t rows_pad = p.c_layout == METIS_SF_TILED ? (p.rows + 127) / 128 * 128 : p.rows;
+  const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= rows_pad * bpr) return;
+  const int64_t r = idx / bpr, b = idx % bpr;
+  if (r >= p.rows) { p.c_scales[metis_sf_offset(r, b, bpr, p.c_layout)] = 0; return; }
+  const float s_T = tscale_is_amax ? metis_tensor_scale(*tscale_src) : *tscale_src;
+  if (idx == 0 && ts_out != nullptr) *ts_out = s_T;
+  const bool sr = p.rounding == METIS_ROUND_SR;
+  float v[16];
+  uint32_t u[16];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float4 q = *reinterpret_cast<const float4*>(x + r * ld + b * 16 + i * 4);
+    v[4 * i] = q.x; v[4 * i + 1] = q.y; v[4 * i + 2] = q.z; v[4 * i + 3] = q.w;
+  }
+  if (sr) {
+    if (p.e_stride_c == 1 && (p.e_stride_r & 7) == 0) {
+      const uint64_t e0 = (uint64_t)r * (uint64_t)p.e_stride_r + (uint64_t)b * 16u;
+#pragma unroll
+      for (int h2 = 0; h2 < 2; ++h2) {
+        const uint4 w = metis_philox_block((e0 >> 3) + h2, p.seed, p.stream_id);
+#pragma unroll
+        for (uint32_t hh = 0; hh < 8; ++hh) u[8 * h2 + hh] = metis_u16_of(w, hh);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        u[i] = metis_draw_u16((uint64_t)r * (uint64_t)p.e_stride_r + (uint64_t)(b * 16 + i) * (uint64_t)p.e_stride_c, p.seed, p.stream_id);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) u[i] = 0u;
+  }
+  uint32_t packed[2];
+  const uint32_t byte = metis_qt::encode_block(v, u, sr, s_T, __fmul_rn(6.0f, s_T), packed);
+  *reinterpret_cast<uint2*>(p.c_codes + r * (p.cols / 2) + b * 8) = make_uint2(packed[0], packed[1]);
+  p.c_scales[metis_sf_offset(r, b, bpr, p.c_layout)] = (uint8_t)byte;
+}
+
 metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int rounding,
                                      uint64_t seed, uint32_t stream_id, int64_t e_stride_r, int64_t e_stride_c,
                                      const float* tscale_src, int tscale_is_amax, const metis_nvfp4_t* by_cols,
@@ -255,6 +302,13 @@ metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int
   p.e_stride_r = e_stride_r; p.e_stride_c = e_stride_c;
   if (by_cols) { p.c_codes = by_cols->codes; p.c_scales = by_cols->scales; p.c_layout = by_cols->sf_layout; }
   if (by_rows) { p.r_codes = by_rows->codes; p.r_scales = by_rows->scales; p.r_layout = by_rows->sf_layout; }
+  if (dtype == METIS_FP32 && by_cols && !by_rows && rows <= 64) {
+    const int64_t rows_pad = p.c_layout == METIS_SF_TILED ? (rows + 127) / 128 * 128 : rows;
+    quantize_rowblocks_kernel<<<(unsigned)metis_ceil_div(rows_pad * (cols / 16), 256), 256, 0, s>>>(
+        reinterpret_cast<const float*>(x), ld, p, tscale_src, tscale_is_amax, by_cols->tensor_scale); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(cudaGetLastError());
+    return METIS_OK;
+  }
   const bool sr = rounding == METIS_ROUND_SR;
   static bool attr_set = false;
   if (!attr_set) {
