@@ -29,7 +29,7 @@ L_TOKENS, D_IN, D_OUT, RANK_K, OVERSAMPLE_P = 4096, 4096, 4096, 32, 8
 WORKLOAD = "llama3-8b q_proj linear fwd+bwd, tokens 4096 (2x2048), 4096->4096, k=32 p=8, SR on dY"
 N_SETS = 3
 FP4_OVER_BF16 = 4.0           # nominal dense FP4 : bf16 tensor throughput ratio
-GEMM_DRAM_BYTES_NCU = 19.08e6 + 0.16e6   # per 4096^3 launch (profiles/gemm_nvfp4_2cta_4096x4096x4096.md)
+GEMM_DRAM_BYTES_NCU = 22.09e6 + 0.60e6   # per 4096^3 launch (profiles/gemm_nvfp4_2cta_4096x4096x4096.md)
 
 
 def measured_peaks():
