@@ -628,23 +628,30 @@ coeff_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols
   }
 }
 
-// out[e] = sum over all partials p of in[p][e], in order (eight independent loads in flight per thread).
-__global__ void reduce_gram_kernel(const double* __restrict__ in, int n_in, int nn, double* __restrict__ out,
-                                   const int* __restrict__ skip) {
+// out[e] = sum over all partials p of in[p][e].  A CTA of four warps owns 32 elements; warp s adds every fourth
+// partial (eight loads in flight), the four sums are added in a fixed order: the result does not depend on timing.
+__global__ void __launch_bounds__(128)
+reduce_gram_kernel(const double* __restrict__ in, int n_in, int nn, double* __restrict__ out,
+                   const int* __restrict__ skip) {
   if (skip != nullptr && *skip) return;
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= nn) return;
+  __shared__ double part[4][32];
+  const int lane = threadIdx.x & 31, sl = threadIdx.x >> 5;
+  const int e = blockIdx.x * 32 + lane;
   double a = 0.0;
-  int p = 0;
-  for (; p + 8 <= n_in; p += 8) {
-    double v[8];
+  if (e < nn) {
+    int p = sl;
+    for (; p + 28 < n_in; p += 32) {
+      double v[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) v[u] = in[(int64_t)(p + u) * nn + e];
+      for (int u = 0; u < 8; ++u) v[u] = in[(int64_t)(p + 4 * u) * nn + e];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) a += v[u];
+      for (int u = 0; u < 8; ++u) a += v[u];
+    }
+    for (; p < n_in; p += 4) a += in[(int64_t)p * nn + e];
   }
-  for (; p < n_in; ++p) a += in[(int64_t)p * nn + e];
-  out[e] = a;
+  part[sl][lane] = a;
+  __syncthreads();
+  if (sl == 0 && e < nn) out[e] = ((part[0][lane] + part[1][lane]) + part[2][lane]) + part[3][lane];
 }
 
 // Sums the column slices of the tensor-core broadcast pass in a fixed order: coef[r][j] = sum_s part[s][r][j],
@@ -944,10 +951,12 @@ right_rotate_kernel(const float* __restrict__ basis, int64_t cols, int k, const 
   if (w) for (int o = tid; o < k * k; o += 256) wsm[o / k][o % k] = (float)w[o];
   __syncthreads();
   const int64_t col = (int64_t)blockIdx.x * 256 + tid;
+  // blockIdx.y owns the output vectors j = 8*blockIdx.y .. +7 (a CTA per 256 columns alone leaves most SMs idle)
+  const int j_begin = blockIdx.y * 8, j_end = min(k, j_begin + 8);
   float bv[MAXQ];
 #pragma unroll
   for (int i = 0; i < MAXQ; ++i) bv[i] = (i < k && col < cols) ? basis[(int64_t)i * cols + col] : 0.0f;
-  for (int j = 0; j < k; ++j) {
+  for (int j = j_begin; j < j_end; ++j) {
     float v;
     if (w) {
       v = 0.0f;
@@ -971,7 +980,7 @@ right_rotate_kernel(const float* __restrict__ basis, int64_t cols, int k, const 
     if (lane == 0) { red_v[warp][j] = sv; red_i[warp][j] = ai; }
   }
   __syncthreads();
-  if (tid < k) {
+  if (tid >= j_begin && tid < j_end) {
     float sv = red_v[0][tid]; int ai = red_i[0][tid];
     for (int wv = 1; wv < 8; ++wv) {
       const float ov = red_v[wv][tid];
@@ -1023,7 +1032,7 @@ left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, i
     if (evals_for_scale) {
       const double lam = sqrt(fmax(evals_for_scale[tid], 0.0));
       s = lam > 0.0 ? 1.0 / lam : 0.0;
-      if (blockIdx.x == 0 && sigma_out) sigma_out[tid] = (float)lam;
+      if (blockIdx.x == 0 && blockIdx.y == 0 && sigma_out) sigma_out[tid] = (float)lam;
     }
     scl[tid] = s * (double)sign[tid];
   }
@@ -1031,9 +1040,10 @@ left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, i
   const int64_t r = (int64_t)blockIdx.x * 64 + rx;
   float am = 0.0f;
   if (r < rows) {
-    for (int j0 = jg * 4; j0 < kp; j0 += 16) {
+    for (int j0 = jg * 4 + 16 * blockIdx.y; j0 < kp; j0 += 16 * gridDim.y) {   // blockIdx.y: every gridDim.y-th group of 16 outputs
       double a[4] = {0.0, 0.0, 0.0, 0.0};
       if (j0 < k) {
+#pragma unroll 4
         for (int i = 0; i < n_in; ++i) {
           const double v = (double)c[i * stride_i + r * stride_r];
           a[0] += v * ws[i][j0]; a[1] += v * ws[i][j0 + 1]; a[2] += v * ws[i][j0 + 2]; a[3] += v * ws[i][j0 + 3];
@@ -1286,7 +1296,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     int64_t rpp; const int parts = gram_parts(n_s, &rpp);
     const int* skip = pass == 0 ? nullptr : cond_flag;
     gram_kernel<<<parts, 256, 0, s>>>(z, n_s, q, q, 1, rpp, gram, skip); METIS_COUNT_LAUNCH();
-    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1, skip); METIS_COUNT_LAUNCH();
+    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 32), 128, 0, s>>>(gram, parts, q * q, gram1, skip); METIS_COUNT_LAUNCH();
     chol_kernel<<<1, 256, 0, s>>>(gram1, q, linv, invd, skip, pass == 0 ? cond_flag : nullptr); METIS_COUNT_LAUNCH();
     apply_chol_kernel<<<(unsigned)metis_ceil_div(n_s, 8), 256, 0, s>>>(z, n_s, q, linv, invd, skip); METIS_COUNT_LAUNCH();
   }
@@ -1328,7 +1338,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   {
     int64_t rpp; const int parts = gram_parts(cols, &rpp);
     gram_kernel<<<parts, 256, 0, s>>>(m, cols, q, 1, cols, rpp, gram, nullptr); METIS_COUNT_LAUNCH();
-    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 128), 128, 0, s>>>(gram, parts, q * q, gram1, nullptr); METIS_COUNT_LAUNCH();
+    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 32), 128, 0, s>>>(gram, parts, q * q, gram1, nullptr); METIS_COUNT_LAUNCH();
     launch_jacobi(s, gram1, q, q, 1e-8f, evals, evecs);
   }
   right_basis_kernel<<<(unsigned)metis_ceil_div(cols, 64), 256, 0, s>>>(m, cols, q, k, evals, evecs, basis,
@@ -1338,10 +1348,10 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   const int n_cta_c = (int)metis_ceil_div(rows, 32);
   if (full) {
     // left = H U~_k, right = basis (sign fixed); coefficients = left * sigma
-    right_rotate_kernel<<<n_cand, 256, 0, s>>>(basis, cols, k, nullptr, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
+    right_rotate_kernel<<<dim3(n_cand, (k + 7) / 8), 256, 0, s>>>(basis, cols, k, nullptr, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
     sign_fix_kernel<<<dim3(n_cand, k), 256, 0, s>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2); METIS_COUNT_LAUNCH();
     basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(out->right, cols, k, kp, bs, bt); METIS_COUNT_LAUNCH();
-    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 256, 0, s>>>(z, rows, q, k, 1, q, evecs, nullptr, sign,
+    left_rotate_kernel<<<dim3((unsigned)metis_ceil_div(rows, 64), (unsigned)((kp + 15) / 16)), 256, 0, s>>>(z, rows, q, k, 1, q, evecs, nullptr, sign,
                                                                             out->left, nullptr, coef, kp, out->sigma, amax + 1); METIS_COUNT_LAUNCH();
   } else {
     basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(basis, cols, k, kp, bs, bt); METIS_COUNT_LAUNCH();
@@ -1394,11 +1404,11 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   cudaStream_t sf = ctx->side[0];
   if (!full) {
     // (7) Rayleigh-Ritz on C^T C (Gram partials came out of the broadcast pass), rotate both factors
-    reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 128), 128, 0, sf>>>(gram_c, n_cta_c, kp * kp, gram1, nullptr); METIS_COUNT_LAUNCH();
+    reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 32), 128, 0, sf>>>(gram_c, n_cta_c, kp * kp, gram1, nullptr); METIS_COUNT_LAUNCH();
     launch_jacobi(sf, gram1, k, kp, 1e-6f, evals2, evecs2);
-    right_rotate_kernel<<<n_cand, 256, 0, sf>>>(basis, cols, k, evecs2, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
+    right_rotate_kernel<<<dim3(n_cand, (k + 7) / 8), 256, 0, sf>>>(basis, cols, k, evecs2, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
     sign_fix_kernel<<<dim3(n_cand, k), 256, 0, sf>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2); METIS_COUNT_LAUNCH();
-    left_rotate_kernel<<<(unsigned)metis_ceil_div(rows, 64), 256, 0, sf>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
+    left_rotate_kernel<<<dim3((unsigned)metis_ceil_div(rows, 64), (unsigned)((kp + 15) / 16)), 256, 0, sf>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
                                                                             out->left, out->sigma, nullptr, kp, nullptr, amax + 1); METIS_COUNT_LAUNCH();
   }
   METIS_CUDA_TRY(cudaGetLastError());
