@@ -154,6 +154,24 @@ __device__ __forceinline__ float metis_ld_as_float(const void* p, int dtype, int
                              : reinterpret_cast<const float*>(p)[idx];
 }
 
+// splits of eight consecutive FP32 values into BF16 hi / lo / lo2, packed two per word
+__device__ __forceinline__ void metis_split3x8(const float (&v)[8], uint4& h, uint4& l, uint4& l2) {
+  uint32_t hh[4], ll[4], mm[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float x = v[2 * i], y = v[2 * i + 1];
+    const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
+    const float xr = x - __bfloat162float(xh), yr = y - __bfloat162float(yh);
+    const __nv_bfloat16 xl = __float2bfloat16_rn(xr), yl = __float2bfloat16_rn(yr);
+    const __nv_bfloat16 xm = __float2bfloat16_rn(xr - __bfloat162float(xl)), ym = __float2bfloat16_rn(yr - __bfloat162float(yl));
+    hh[i] = (uint32_t)__bfloat16_as_ushort(xh) | ((uint32_t)__bfloat16_as_ushort(yh) << 16);
+    ll[i] = (uint32_t)__bfloat16_as_ushort(xl) | ((uint32_t)__bfloat16_as_ushort(yl) << 16);
+    mm[i] = (uint32_t)__bfloat16_as_ushort(xm) | ((uint32_t)__bfloat16_as_ushort(ym) << 16);
+  }
+  h = make_uint4(hh[0], hh[1], hh[2], hh[3]); l = make_uint4(ll[0], ll[1], ll[2], ll[3]); l2 = make_uint4(mm[0], mm[1], mm[2], mm[3]);
+}
+
+
 // ---- internal entry points shared between translation units --------------------------------
 metis_status_t metis_launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* amax_out,
                                  cudaStream_t s);

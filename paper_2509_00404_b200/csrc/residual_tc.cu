@@ -44,23 +44,6 @@ struct ResidArgs {
   uint32_t* dev_status;
 };
 
-// splits of eight consecutive FP32 values into BF16 hi / lo / lo2, packed two per word
-__device__ __forceinline__ void split3x8(const float (&v)[8], uint4& h, uint4& l, uint4& l2) {
-  uint32_t hh[4], ll[4], mm[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float x = v[2 * i], y = v[2 * i + 1];
-    const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
-    const float xr = x - __bfloat162float(xh), yr = y - __bfloat162float(yh);
-    const __nv_bfloat16 xl = __float2bfloat16_rn(xr), yl = __float2bfloat16_rn(yr);
-    const __nv_bfloat16 xm = __float2bfloat16_rn(xr - __bfloat162float(xl)), ym = __float2bfloat16_rn(yr - __bfloat162float(yl));
-    hh[i] = (uint32_t)__bfloat16_as_ushort(xh) | ((uint32_t)__bfloat16_as_ushort(yh) << 16);
-    ll[i] = (uint32_t)__bfloat16_as_ushort(xl) | ((uint32_t)__bfloat16_as_ushort(yl) << 16);
-    mm[i] = (uint32_t)__bfloat16_as_ushort(xm) | ((uint32_t)__bfloat16_as_ushort(ym) << 16);
-  }
-  h = make_uint4(hh[0], hh[1], hh[2], hh[3]); l = make_uint4(ll[0], ll[1], ll[2], ll[3]); l2 = make_uint4(mm[0], mm[1], mm[2], mm[3]);
-}
-
 // out[i][6*kp padded to kx] for vector i: pattern A = [h|h|l|h|l2|l] (coefficients), pattern B = [h|l|h|l2|h|l] (basis).
 // src element (i, j): src[i*stride_i + j*stride_j], j < k (zero beyond).  One thread per (i, group of 8 j).
 __global__ void __launch_bounds__(256)
@@ -78,7 +61,7 @@ splits6_kernel(const float* __restrict__ src, int64_t n, int k, int kp, int kx, 
 #pragma unroll
   for (int e = 0; e < 8; ++e) v[e] = (j0 + e < k) ? src[i * stride_i + (int64_t)(j0 + e) * stride_j] : 0.0f;
   uint4 h, l, l2;
-  split3x8(v, h, l, l2);
+  metis_split3x8(v, h, l, l2);
   // term:        0  1  2  3   4   5
   // pattern A:   h  h  l  h   l2  l
   // pattern B:   h  l  h  l2  h   l
@@ -330,16 +313,18 @@ int metis_residual_kx(int kp) { return (6 * kp + 63) / 64 * 64; }
 
 bool metis_residual_tc_usable(const void* x, int64_t cols) { return metis_aligned16(x) && cols % 8 == 0; }
 
-// a6: [rows][kx], b6: [cols][kx] BF16 scratch (kx = metis_residual_kx(kp)); coef: [rows][kp] FP32; basis: [k][cols] FP32.
-metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const float* coef, const float* basis, int k, int kp,
+// a6: [rows][kx] = per row [Ch|Ch|Cl|Ch|Cl2|Cl], b6: [cols][kx] = per column [Bh|Bl|Bh|Bl2|Bh|Bl] (BF16,
+// kx = metis_residual_kx(kp)).  b6 is filled by the caller; a6 too unless `coef` ([rows][kp] FP32) is given,
+// in which case it is written here first.
+metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const float* coef, int k, int kp,
                                         const metis_qt::QuantParams& qp, const float* amax_src, float* ts_out0, float* ts_out1,
                                         float* dense, void* a6, void* b6, cudaStream_t s) {
   const int kx = metis_residual_kx(kp);
   const int64_t rows = qp.rows, cols = qp.cols;
-  splits6_kernel<<<(unsigned)metis_ceil_div(rows * (kx / 8), 256), 256, 0, s>>>(coef, rows, k, kp, kx, kp, 1, 0,
-                                                                                reinterpret_cast<__nv_bfloat16*>(a6)); METIS_COUNT_LAUNCH();
-  splits6_kernel<<<(unsigned)metis_ceil_div(cols * (kx / 8), 256), 256, 0, s>>>(basis, cols, k, kp, kx, 1, cols, 1,
-                                                                                reinterpret_cast<__nv_bfloat16*>(b6)); METIS_COUNT_LAUNCH();
+  if (coef != nullptr) {
+    splits6_kernel<<<(unsigned)metis_ceil_div(rows * (kx / 8), 256), 256, 0, s>>>(coef, rows, k, kp, kx, kp, 1, 0,
+                                                                                  reinterpret_cast<__nv_bfloat16*>(a6)); METIS_COUNT_LAUNCH();
+  }
   CUtensorMap mx, ma, mb;
   METIS_TRY(make_map_bf16(ctx, &mx, x, rows, cols, cols, TM));
   METIS_TRY(make_map_bf16(ctx, &ma, a6, rows, kx, kx, TM));

@@ -7,7 +7,7 @@
 //   with the NVFP4 quantizer in both block orientations -> factor rotation, sign fix, factor quantization.
 #include "quant_tile.cuh"
 
-metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const float* coef, const float* basis, int k, int kp,
+metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const float* coef, int k, int kp,
                                         const metis_qt::QuantParams& qp, const float* amax_src, float* ts_out0, float* ts_out1,
                                         float* dense, void* a6, void* b6, cudaStream_t s);
 
@@ -513,9 +513,12 @@ __device__ __forceinline__ void split3(float x, float y, uint32_t& hi, uint32_t&
 //   bt[t][col][j]  (j contiguous, padded to kp; B operand of C B^T, contraction over j)
 __global__ void __launch_bounds__(128)
 basis_splits_kernel(const float* __restrict__ basis, int64_t cols, int k, int kp, __nv_bfloat16* __restrict__ bs,
-                    __nv_bfloat16* __restrict__ bt) {
+                    __nv_bfloat16* __restrict__ bt, __nv_bfloat16* __restrict__ b6, int kx) {
   const int64_t col = (int64_t)blockIdx.x * 128 + threadIdx.x;
   if (col >= cols) return;
+  // b6 (optional): [cols][kx], per column the six K blocks [Bh | Bl | Bh | Bl2 | Bh | Bl] of the residual product
+  if (b6 != nullptr)
+    for (int z = 6 * kp; z < kx; z += 8) *reinterpret_cast<uint4*>(b6 + col * kx + z) = make_uint4(0u, 0u, 0u, 0u);
   for (int j0 = 0; j0 < kp; j0 += 8) {
     uint32_t w[3][4];
 #pragma unroll
@@ -530,6 +533,12 @@ basis_splits_kernel(const float* __restrict__ basis, int64_t cols, int k, int kp
       for (int jj = 0; jj < 8; ++jj)
         bs[((int64_t)t * kp + j0 + jj) * cols + col] = __ushort_as_bfloat16((unsigned short)((w[t][jj >> 1] >> (16 * (jj & 1))) & 0xFFFFu));
       *reinterpret_cast<uint4*>(bt + ((int64_t)t * cols + col) * kp + j0) = make_uint4(w[t][0], w[t][1], w[t][2], w[t][3]);
+    }
+    if (b6 != nullptr) {
+      const int sel[6] = {0, 1, 0, 2, 0, 1};
+#pragma unroll
+      for (int term = 0; term < 6; ++term)
+        *reinterpret_cast<uint4*>(b6 + col * kx + term * kp + j0) = make_uint4(w[sel[term]][0], w[sel[term]][1], w[sel[term]][2], w[sel[term]][3]);
     }
   }
 }
@@ -659,7 +668,7 @@ reduce_gram_kernel(const double* __restrict__ in, int n_in, int nn, double* __re
 template <int KP>
 __global__ void __launch_bounds__(256)
 coef_finish_kernel(const float* __restrict__ part, int slices, int64_t rows, float* __restrict__ coef,
-                   double* __restrict__ gram_part) {
+                   double* __restrict__ gram_part, __nv_bfloat16* __restrict__ a6, int kx) {
   __shared__ float cfin[32 * KP];
   const int tid = threadIdx.x;
   const int64_t row0 = (int64_t)blockIdx.x * 32;
@@ -673,6 +682,24 @@ coef_finish_kernel(const float* __restrict__ part, int slices, int64_t rows, flo
     cfin[o] = v;
   }
   __syncthreads();
+  if (a6 != nullptr) {
+    // a6: [rows][kx], per row the six K blocks [Ch | Ch | Cl | Ch | Cl2 | Cl] of the residual product (zero padded)
+    for (int o = tid; o < 32 * (KP / 8); o += 256) {
+      const int rr = o / (KP / 8), j0 = (o % (KP / 8)) * 8;
+      const int64_t r = row0 + rr;
+      if (r >= rows) continue;
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = cfin[rr * KP + j0 + e];
+      uint4 h, l, l2;
+      metis_split3x8(v, h, l, l2);
+      __nv_bfloat16* dst = a6 + r * kx + j0;
+      *reinterpret_cast<uint4*>(dst) = h; *reinterpret_cast<uint4*>(dst + KP) = h; *reinterpret_cast<uint4*>(dst + 2 * KP) = l;
+      *reinterpret_cast<uint4*>(dst + 3 * KP) = h; *reinterpret_cast<uint4*>(dst + 4 * KP) = l2; *reinterpret_cast<uint4*>(dst + 5 * KP) = l;
+      if (j0 == 0)
+        for (int z = 6 * KP; z < kx; z += 8) *reinterpret_cast<uint4*>(a6 + r * kx + z) = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
   if (gram_part) {
     for (int o = tid; o < KP * KP; o += 256) {
       const int i = o / KP, j = o % KP;
@@ -1243,6 +1270,12 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   float* part = reinterpret_cast<float*>(wsb + L.part);
   void* a6 = wsb + L.a6;
   void* b6 = wsb + L.b6;
+  // the residual kernel's K-concatenated BF16 operands are written by the kernels that produce coefficients and basis
+  const bool resid_tc = metis_residual_tc_usable(x, cols);
+  const int kx6 = metis_residual_kx((k + 15) / 16 * 16);
+  __nv_bfloat16* a6p = resid_tc ? reinterpret_cast<__nv_bfloat16*>(a6) : nullptr;
+  __nv_bfloat16* b6p = resid_tc ? reinterpret_cast<__nv_bfloat16*>(b6) : nullptr;
+  bool a6_ready = false;
   metis_context* ctx = h;
   const int kp = (k + 15) / 16 * 16;
   {
@@ -1350,20 +1383,21 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     // left = H U~_k, right = basis (sign fixed); coefficients = left * sigma
     right_rotate_kernel<<<dim3(n_cand, (k + 7) / 8), 256, 0, s>>>(basis, cols, k, nullptr, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
     sign_fix_kernel<<<dim3(n_cand, k), 256, 0, s>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2); METIS_COUNT_LAUNCH();
-    basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(out->right, cols, k, kp, bs, bt); METIS_COUNT_LAUNCH();
+    basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(out->right, cols, k, kp, bs, bt, b6p, kx6); METIS_COUNT_LAUNCH();
     left_rotate_kernel<<<dim3((unsigned)metis_ceil_div(rows, 64), (unsigned)((kp + 15) / 16)), 256, 0, s>>>(z, rows, q, k, 1, q, evecs, nullptr, sign,
                                                                             out->left, nullptr, coef, kp, out->sigma, amax + 1); METIS_COUNT_LAUNCH();
   } else {
-    basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(basis, cols, k, kp, bs, bt); METIS_COUNT_LAUNCH();
+    basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(basis, cols, k, kp, bs, bt, b6p, kx6); METIS_COUNT_LAUNCH();
     if (metis_coeff_tc_usable(x, bs, cols, kp)) {
       // tensor-core pass over x (column slices), then the slices are summed and the Gram partials formed
       METIS_TRY(metis_launch_coeff_tc(ctx, x, rows, cols, bs, kp, part, amax, s));
+      a6_ready = resid_tc;
       const int slices = metis_coeff_slices(rows, cols, nullptr);
       switch (kp) {
-        case 16: coef_finish_kernel<16><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c); break;
-        case 32: coef_finish_kernel<32><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c); break;
-        case 48: coef_finish_kernel<48><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c); break;
-        default: coef_finish_kernel<64><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c); break;
+        case 16: coef_finish_kernel<16><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c, a6p, kx6); break;
+        case 32: coef_finish_kernel<32><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c, a6p, kx6); break;
+        case 48: coef_finish_kernel<48><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c, a6p, kx6); break;
+        default: coef_finish_kernel<64><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c, a6p, kx6); break;
       }
     } else {
       const size_t smem = sizeof(float) * 9 * 32 * kp;
@@ -1389,8 +1423,8 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     // goes to a (high-priority) side stream and is joined back at the end of the call
     METIS_TRY(metis_fork(ctx, s, 1));
     cudaStream_t sr = s;
-    if (metis_residual_tc_usable(x, cols)) {
-      METIS_TRY(metis_launch_residual_tc(ctx, x, coef, full ? out->right : basis, k, kp, qp, amax, t0, t1, residual_dense, a6, b6, sr));
+    if (resid_tc) {
+      METIS_TRY(metis_launch_residual_tc(ctx, x, a6_ready ? nullptr : coef, k, kp, qp, amax, t0, t1, residual_dense, a6, b6, sr));
     } else {
       switch (kp) {
         case 16: residual_quant_kernel<16><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
