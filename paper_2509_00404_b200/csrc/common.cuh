@@ -122,23 +122,21 @@ __device__ __forceinline__ uint32_t metis_e2m1x2_rne(float lo, float hi) {
   return out;
 }
 
-// stochastic rounding of y to E2M1 with a 16-bit draw: up iff frac * 65536 > u, frac = (a - lo)/(hi - lo).
-// For a >= 1 the E2M1 grid has one mantissa bit per binade, so lo is the top mantissa bit of a and frac is the
-// remaining 22 bits: frac * 65536 > u  <=>  (mantissa & 0x3FFFFF) > 64 u, an exact integer comparison.
-// Below 1 the grid is {0, 0.5, 1}: uniform step 0.5, all operations exact in binary32.
+// stochastic rounding of y to E2M1 with a 16-bit draw: up iff frac * 65536 > u, frac = (a - lo)/(hi - lo), a = min(|y|, 6).
+// E2M1 is a tiny float format: one mantissa bit per binade from 1 upwards, and below 1 the grid {0, 0.5, 1} has the
+// spacing of the binade [1, 2).  So for a >= 1 the lower neighbour is the top mantissa bit of a and frac is the other
+// 22 bits, and a < 1 is mapped onto [1, 2] by adding 1 (rounded UP, so that bits lost in the addition still count as
+// "frac > 0"; a carry into the next grid point is the round-up it stands for).  Then
+//   frac * 65536 > u  <=>  (mantissa & 0x3FFFFF) > 64 u,
+// an exact integer comparison, and the code is  offset + 2 * exponent + top bit + up.  No branches.
 __device__ __forceinline__ uint32_t metis_e2m1_sr(float y, uint32_t u16) {
   const float a = fminf(fabsf(y), 6.0f);
   const uint32_t sign = (__float_as_uint(y) >> 28) & 8u;
-  const uint32_t bits = __float_as_uint(a);
-  if (bits >= 0x40C00000u) return sign | 7u;                       // a == 6 (saturated): no draw
-  if (bits >= 0x3F800000u) {                                       // 1 <= a < 6
-    const uint32_t e = (bits >> 23) - 127u, half = (bits >> 22) & 1u, frac22 = bits & 0x3FFFFFu;
-    return sign | (2u + 2u * e + half + (frac22 > (u16 << 6) ? 1u : 0u));
-  }
-  const float t2 = __fadd_rn(a, a);                                // a / 0.5, exact
-  const float fl = t2 >= 1.0f ? 1.0f : 0.0f;
-  const float fr = __fsub_rn(t2, fl);
-  return sign | ((uint32_t)fl + (__fmul_rn(fr, 65536.0f) > (float)u16 ? 1u : 0u));
+  const bool small = a < 1.0f;
+  const uint32_t bits = __float_as_uint(small ? __fadd_ru(a, 1.0f) : a);
+  const uint32_t g = ((bits >> 22) & 0x1FFu) - 254u;               // 2 * exponent + top mantissa bit (0 at 1.0)
+  const uint32_t up = (bits & 0x3FFFFFu) > (u16 << 6) ? 1u : 0u;
+  return sign | ((small ? 0u : 2u) + g + up);
 }
 
 // byte offset of scale (row r, block b) in the 128x4-tiled layout; blocks_per_row = k_len/16
