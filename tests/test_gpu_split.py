@@ -96,6 +96,36 @@ def test_planted_noise_free_spectrum_is_recovered(ctx):
     assert np.linalg.norm(dense2) < 2e-2 * np.linalg.norm(x2)               # only bf16 rounding noise is left
 
 
+@pytest.mark.parametrize("shape", [(320, 448), (192, 320), (448, 192)])
+def test_ragged_tiles_sampled_and_full(ctx, shape):
+    """Rows and columns that are multiples of 64 (the tiled scale layout) but not of the 128-wide tiles: partial TMA boxes, partial
+    accumulator tiles, half-valid 32-row slabs and 32-column steps in the fused residual quantizer."""
+    B, h = ctx
+    rows, cols = shape
+    x, _ = synth.llama_like(rows, cols, 1.0, 500 + rows, rank=8)
+    _check_against_oracle(B, h, x, 8, 4, B.SKETCH_SAMPLED, seed=31)
+    _check_against_oracle(B, h, x, 8, 4, B.SKETCH_SAMPLED, seed=32, rounding=1)
+    _check_against_oracle(B, h, x, 8, 4, B.SKETCH_FULL, seed=33)
+
+
+def test_all_zero_operand_is_degenerate_but_clean(ctx):
+    """x = 0: every pivot of the orthonormalisation is dependent, every eigenvalue zero.  The library must return
+    zero factors, a zero residual (signs kept, scale bytes 0) and status OK - no NaN anywhere."""
+    from gpu_util import nv_to_numpy
+    B, h = ctx
+    x = torch.zeros((256, 320), dtype=torch.bfloat16, device="cuda")
+    for mode in (B.SKETCH_SAMPLED, B.SKETCH_FULL):
+        op, dense = h.split(x, 8, 4, sketch=mode, seed=5, want_residual=True)
+        torch.cuda.synchronize()
+        assert h.device_status() == 0
+        assert torch.count_nonzero(dense) == 0
+        for t in (op.left, op.right, op.sigma):
+            assert torch.isfinite(t).all() and torch.count_nonzero(t[:8]) == 0
+        for t in (op.res_by_cols, op.res_by_rows, op.left_q, op.right_q):
+            c, s, ts = nv_to_numpy(t)
+            assert np.count_nonzero(c & 7) == 0 and np.count_nonzero(s) == 0 and np.isfinite(ts)
+
+
 def test_rank_zero_is_plain_quantization(ctx):
     from gpu_util import to_dev_bf16, nv_to_numpy
     B, h = ctx
