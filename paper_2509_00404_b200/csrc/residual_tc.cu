@@ -339,7 +339,12 @@ metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const
     attr = true;
   }
   const int64_t tiles = metis_ceil_div(rows, TM) * metis_ceil_div(cols, TN);
-  const int grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);
+  // A persistent CTA fills its SM (216 KB of shared memory).  A few SMs are left free so that the small kernels
+  // of the factor chain, which run beside this pass on another stream, and those of other operands' chains do
+  // not have to wait for the whole pass to end.
+  constexpr int reserve = 16;
+  const int usable = ctx->sm_count > 2 * reserve ? ctx->sm_count - reserve : ctx->sm_count;
+  const int grid = (int)(tiles < usable ? tiles : usable);
   residual_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(mx, ma, mb, g); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
