@@ -127,6 +127,10 @@ metis_status_t metis_last_device_status(metis_handle_t h, uint32_t* out, metis_s
  * matrix of the random projection is drawn through this table). */
 metis_status_t metis_debug_quantile_table(metis_handle_t h, uint16_t* host_out);
 
+/* Benchmark hook: enqueues a one-thread kernel that writes the GPU's nanosecond timer (%globaltimer) to
+ * *device_slot when `stream` reaches it; usable inside a stream capture, where events cannot be timed. */
+metis_status_t metis_debug_timestamp(metis_handle_t h, uint64_t* device_slot, metis_stream_t stream);
+
 /* Test / benchmark hook: kernels launched by the library in this process so far (host counter). */
 uint64_t metis_debug_launch_count(void);
 

@@ -123,6 +123,21 @@ metis_status_t metis_workspace_bytes(int32_t op, int64_t rows, int64_t cols, int
   }
 }
 
+namespace {
+__global__ void timestamp_kernel(unsigned long long* slot) {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  *slot = t;
+}
+}  // namespace
+
+metis_status_t metis_debug_timestamp(metis_handle_t h, uint64_t* device_slot, metis_stream_t stream) {
+  if (!h || !device_slot) return METIS_ERR_INVALID_ARG;
+  timestamp_kernel<<<1, 1, 0, reinterpret_cast<cudaStream_t>(stream)>>>(reinterpret_cast<unsigned long long*>(device_slot));
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
+
 metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dtype, int64_t rows, int64_t cols,
                                     int64_t ld, int32_t rounding, uint64_t seed, uint32_t stream_id, int32_t tscale,
                                     metis_nvfp4_t* out_by_cols, metis_nvfp4_t* out_by_rows, void* ws, size_t ws_bytes,
