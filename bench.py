@@ -186,8 +186,12 @@ def main():
     ev_start, ev_w, ev_d = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
     h_x, h_w, h_d = h, B.Handle(local_rank), B.Handle(local_rank)     # one workspace owner per stream
 
-    def step(bufs, i):
+    stamps = torch.zeros(8, dtype=torch.int64, device="cuda")
+
+    def step(bufs, i, stamp=False):
         main = torch.cuda.current_stream()
+        if stamp:
+            h_x.timestamp(stamps[0:1], main)
         ev_start.record(main)
         side_w.wait_event(ev_start)
         side_d.wait_event(ev_start)
@@ -196,15 +200,25 @@ def main():
                 h_w.split(bufs["w"], k, p, sketch=B.SKETCH_FULL, seed=3 * i + 2, rounding=B.ROUND_RNE, out=wo, stream=side_w)
             else:
                 h_w.requantize_weight(wo0, w_res_bf, out=wo, stream=side_w)
+            if stamp:
+                h_w.timestamp(stamps[2:3], side_w)
             ev_w.record(side_w)
         with torch.cuda.stream(side_d):
             h_d.split(bufs["dy"], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 3, rounding=B.ROUND_SR, out=do, stream=side_d)
+            if stamp:
+                h_d.timestamp(stamps[3:4], side_d)
             ev_d.record(side_d)
         h_x.split(bufs["x"], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 1, rounding=B.ROUND_RNE, out=xo)
+        if stamp:
+            h_x.timestamp(stamps[1:2], main)
         main.wait_event(ev_w)
         h_x.linear_fwd(xo, wo, out=y)
+        if stamp:
+            h_x.timestamp(stamps[4:5], main)
         main.wait_event(ev_d)
         h_x.linear_bwd(do, xo, wo, out=(dx, dw))
+        if stamp:
+            h_x.timestamp(stamps[5:6], main)
         parallel.allreduce_weight_grad_(dw)          # token-sharded ranks: the one exchange of the path
 
     def barrier():
@@ -334,6 +348,31 @@ def main():
     qc, qr = B.NvFp4(l, m), B.NvFp4(m, l)
     ms_q = alone(lambda i: h_x.quantize_nvfp4(dev_sets[i % N_SETS]["x"], B.BLOCKS_BOTH, B.ROUND_RNE, seed=1, tensor_scale=1.0, out=(qc, qr)))
     split_gbs = lambda elems, t_ms: 3.125 * elems / (t_ms * 1e-3) / 1e9
+
+    # ---- where the step's time goes: GPU timer stamps at the end of each phase (their own graph, not the timed one) ----
+    timeline = None
+    try:
+        if use_graph:
+            g_t = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_t):
+                step(dev_sets[0], 0, stamp=True)
+            run_t = g_t.replay
+        else:
+            run_t = lambda: step(dev_sets[0], 0, stamp=True)
+        acc_t = [0.0] * 6
+        for _ in range(2):
+            run_t()
+        torch.cuda.synchronize()
+        for _ in range(10):
+            run_t()
+            torch.cuda.synchronize()
+            t_ = stamps.cpu().tolist()
+            for j_ in range(6):
+                acc_t[j_] += (t_[j_] - t_[0]) / 1e6 / 10
+        timeline = {"unit": "ms after the step's start (one input set, ten replays)", "x_split_done": acc_t[1], "w_split_done": acc_t[2],
+                    "dy_split_done": acc_t[3], "forward_done": acc_t[4], "backward_done": acc_t[5]}
+    except Exception as exc:
+        sys.stderr.write("timeline not measured (%s)\n" % exc)
     clocks = sampler.stop()
 
     times = torch.tensor([ms, ms_e2e], dtype=torch.float64, device="cuda")
@@ -364,6 +403,7 @@ def main():
                      "algorithmic_bytes": 0.5625 * 2 * l * m + 2.0 * l * n, "peak_source": "bf16 burst peak (%s) x %.0f nominal FP4:bf16 ratio" % (peaks["source"], FP4_OVER_BF16),
                      "ms_per_launch": gemm_ms},
         "split_overhead_vs_three_plain_gemms": overhead,
+        "timeline": timeline,
         "split_quantize": {"unit": "GB/s of algorithmic bytes (3.125 B per element, both block orientations)",
                            "hbm_peak_gbs": peaks["hbm_gbs"],
                            "x_sampled": {"ms": ms_sx, "gbs": split_gbs(l * m, ms_sx)},
