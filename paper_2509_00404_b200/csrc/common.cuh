@@ -32,6 +32,23 @@ static inline metis_status_t metis_join(metis_context* ctx, cudaStream_t main, i
   return METIS_OK;
 }
 
+// Programmatic dependent launch: a kernel launched with this helper may be scheduled while the kernel before it
+// in the stream is still draining; it must call metis_pdl_wait() before it touches global memory (the wait
+// returns when the preceding kernel has completed and its writes are visible).  Saves the launch gap between
+// the many short dependent kernels of a decomposition.
+__device__ __forceinline__ void metis_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t metis_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 #define METIS_CUDA_TRY(expr)                         \
   do {                                               \
     cudaError_t e__ = (expr);                        \

@@ -18,6 +18,7 @@ constexpr size_t JACOBI_SMEM = sizeof(double) * MAXQ * (MAXQ + 1);
 
 // ------------------------------------------------------------------------------------------------
 __global__ void sample_rows_kernel(int* __restrict__ idx, int n_s, int64_t rows, uint64_t seed, int full) {
+  metis_pdl_wait();
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= n_s) return;
   if (full) { idx[j] = j; return; }
@@ -28,6 +29,7 @@ __global__ void sample_rows_kernel(int* __restrict__ idx, int n_s, int64_t rows,
 
 // ------------------------------------------------------------------------------------------------
 __global__ void reduce_partials_kernel(const float* __restrict__ zp, int n_chunks, int64_t n, float* __restrict__ z) {
+  metis_pdl_wait();
   const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   if (i >= n) return;
   float acc = 0.0f;
@@ -42,6 +44,7 @@ constexpr int GR_TILE = 32;
 __global__ void __launch_bounds__(256)
 gram_kernel(const float* __restrict__ v, int64_t n_rows, int n, int64_t stride_row, int64_t stride_vec,
             int64_t rows_per_part, double* __restrict__ part, const int* __restrict__ skip) {
+  metis_pdl_wait();
   if (skip != nullptr && *skip) return;                 // second CholeskyQR pass not needed (see chol_kernel)
   __shared__ float tile[GR_TILE][MAXQ + 1];
   const int tid = threadIdx.x;
@@ -176,6 +179,7 @@ __device__ __forceinline__ void cta_cholesky(double (*Y)[P], int n, double tol, 
 __global__ void __launch_bounds__(256)
 chol_kernel(const double* __restrict__ g, int q, double* __restrict__ l_out, double* __restrict__ invd_out,
             const int* __restrict__ skip, int* __restrict__ well_conditioned) {
+  metis_pdl_wait();
   if (skip != nullptr && *skip) return;
   __shared__ double L[MAXQ][MAXQ + 1];
   __shared__ double gmax_s;
@@ -206,6 +210,7 @@ chol_kernel(const double* __restrict__ g, int q, double* __restrict__ l_out, dou
 __global__ void __launch_bounds__(256)
 apply_chol_kernel(float* __restrict__ z, int64_t n_rows, int q, const double* __restrict__ l, const double* __restrict__ invd,
                   const int* __restrict__ skip) {
+  metis_pdl_wait();
   if (skip != nullptr && *skip) return;
   __shared__ double L[MAXQ][MAXQ + 1];
   __shared__ double inv_s[MAXQ];
@@ -244,6 +249,7 @@ template <int NJ4>                                                  // float4 gr
 __global__ void __launch_bounds__(256)
 project_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
                const float* __restrict__ h, int rows_per_part, float* __restrict__ mp) {
+  metis_pdl_wait();
   __shared__ __align__(16) float hs[2][PJ_ROWS][MAXQ / 2];
   __shared__ int ids[PJ_ROWS];
   const int tid = threadIdx.x, c2 = tid & 127, jg = tid >> 7;       // jg: sketch columns 2*j + jg
@@ -318,6 +324,7 @@ template <int R>                                        // rows per lane: ceil(n
 __global__ void __launch_bounds__(R > 8 ? 288 : 256)    // eight lanes per couple: n = 72 needs 36 x 8 threads
 jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, double* __restrict__ evals,
                   double* __restrict__ evecs) {
+  metis_pdl_wait();
   extern __shared__ __align__(16) unsigned char jsm[];
   double (*Y)[MAXQ + 1] = reinterpret_cast<double (*)[MAXQ + 1]>(jsm);
   __shared__ double lam[MAXQ];
@@ -460,6 +467,7 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
 __global__ void __launch_bounds__(256)
 right_basis_kernel(const float* __restrict__ m, int64_t cols, int q, int k, const double* __restrict__ evals,
                    const double* __restrict__ evecs, float* __restrict__ basis, float* __restrict__ sigma_out) {
+  metis_pdl_wait();
   __shared__ double ut[MAXQ][MAXQ + 1];
   __shared__ double inv_s[MAXQ];
   const int tid = threadIdx.x, cx = tid & 63, jg = tid >> 6;
@@ -514,6 +522,7 @@ __device__ __forceinline__ void split3(float x, float y, uint32_t& hi, uint32_t&
 __global__ void __launch_bounds__(128)
 basis_splits_kernel(const float* __restrict__ basis, int64_t cols, int k, int kp, __nv_bfloat16* __restrict__ bs,
                     __nv_bfloat16* __restrict__ bt, __nv_bfloat16* __restrict__ b6, int kx) {
+  metis_pdl_wait();
   const int64_t col = (int64_t)blockIdx.x * 128 + threadIdx.x;
   if (col >= cols) return;
   // b6 (optional): [cols][kx], per column the six K blocks [Bh | Bl | Bh | Bl2 | Bh | Bl] of the residual product
@@ -551,6 +560,7 @@ template <int KP>
 __global__ void __launch_bounds__(256)
 coeff_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols, const __nv_bfloat16* __restrict__ bs,
                  float* __restrict__ coef, float* __restrict__ amax_out, double* __restrict__ gram_part) {
+  metis_pdl_wait();
   constexpr int NT = KP / 8;
   extern __shared__ __align__(16) unsigned char smem[];
   float* red = reinterpret_cast<float*>(smem);                 // [8 warps][32 rows][KP]
@@ -642,6 +652,7 @@ coeff_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols
 __global__ void __launch_bounds__(128)
 reduce_gram_kernel(const double* __restrict__ in, int n_in, int nn, double* __restrict__ out,
                    const int* __restrict__ skip) {
+  metis_pdl_wait();
   if (skip != nullptr && *skip) return;
   __shared__ double part[4][32];
   const int lane = threadIdx.x & 31, sl = threadIdx.x >> 5;
@@ -669,6 +680,7 @@ template <int KP>
 __global__ void __launch_bounds__(256)
 coef_finish_kernel(const float* __restrict__ part, int slices, int64_t rows, float* __restrict__ coef,
                    double* __restrict__ gram_part, __nv_bfloat16* __restrict__ a6, int kx) {
+  metis_pdl_wait();
   __shared__ float cfin[32 * KP];
   const int tid = threadIdx.x;
   const int64_t row0 = (int64_t)blockIdx.x * 32;
@@ -720,6 +732,7 @@ __global__ void __launch_bounds__(metis_qt::THREADS, 2)
 residual_quant_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ coef,
                       const __nv_bfloat16* __restrict__ bt, metis_qt::QuantParams p,
                       const float* __restrict__ amax_src, float* ts_out0, float* ts_out1, float* __restrict__ dense) {
+  metis_pdl_wait();
   using namespace metis_qt;
   extern __shared__ __align__(16) unsigned char smem[];
   float* tile = reinterpret_cast<float*>(smem);
@@ -811,6 +824,7 @@ template <int NT>                                      // sketch columns / 8, ro
 __global__ void __launch_bounds__(256)
 sketch_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
                   uint64_t seed, const __nv_bfloat16* __restrict__ lut, float* __restrict__ zp, float* __restrict__ amax_out) {
+  metis_pdl_wait();
   extern __shared__ __align__(16) unsigned char smem[];
   __nv_bfloat16* om = reinterpret_cast<__nv_bfloat16*>(smem);          // [NT*8][SKM_PITCH]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
@@ -899,6 +913,7 @@ template <int MT>                                      // sketch columns / 16, r
 __global__ void __launch_bounds__(256)
 project_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
                    const float* __restrict__ h, int rows_per_part, float* __restrict__ mp) {
+  metis_pdl_wait();
   __shared__ __align__(16) __nv_bfloat16 xs[PM_ROWS][PM_XP];
   __shared__ __align__(16) __nv_bfloat16 hs[3][MT * 16][PM_HP];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
@@ -971,6 +986,7 @@ project_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int*
 __global__ void __launch_bounds__(256)
 right_rotate_kernel(const float* __restrict__ basis, int64_t cols, int k, const double* __restrict__ w,
                     float* __restrict__ right, float* __restrict__ cand_v, int* __restrict__ cand_i) {
+  metis_pdl_wait();
   __shared__ float wsm[MAXQ][MAXQ + 1];
   __shared__ float red_v[8][MAXQ];
   __shared__ int red_i[8][MAXQ];
@@ -1024,6 +1040,7 @@ right_rotate_kernel(const float* __restrict__ basis, int64_t cols, int k, const 
 __global__ void __launch_bounds__(256)
 sign_fix_kernel(float* __restrict__ right, int64_t cols, int k, const float* __restrict__ cand_v,
                 const int* __restrict__ cand_i, int n_cand, float* __restrict__ sign_out, float* __restrict__ amax_out) {
+  metis_pdl_wait();
   const int j = blockIdx.y;
   float sv = 0.0f; int ai = 0x7FFFFFFF;
   for (int c = 0; c < n_cand; ++c) {
@@ -1050,6 +1067,7 @@ left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, i
                    const float* __restrict__ sign, float* __restrict__ left, float* __restrict__ sigma_out,
                    float* __restrict__ coef_rm, int kp, const float* __restrict__ sigma_for_coef,
                    float* __restrict__ amax_out) {
+  metis_pdl_wait();
   __shared__ double ws[MAXQ][MAXQ + 1];
   __shared__ double scl[MAXQ];
   const int tid = threadIdx.x, rx = tid & 63, jg = tid >> 6;
@@ -1163,15 +1181,15 @@ int gram_parts(int64_t n_rows, int64_t* rows_per_part) {
 void launch_jacobi(cudaStream_t s, const double* g, int n, int ld, float exit_cos2, double* evals, double* evecs) {
   const int r = (n + (n & 1) + 7) / 8;
   switch (r) {
-    case 1: jacobi_eig_kernel<1><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
-    case 2: jacobi_eig_kernel<2><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
-    case 3: jacobi_eig_kernel<3><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
-    case 4: jacobi_eig_kernel<4><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
-    case 5: jacobi_eig_kernel<5><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
-    case 6: jacobi_eig_kernel<6><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
-    case 7: jacobi_eig_kernel<7><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
-    case 8: jacobi_eig_kernel<8><<<1, 256, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
-    default: jacobi_eig_kernel<9><<<1, 288, JACOBI_SMEM, s>>>(g, n, ld, exit_cos2, evals, evecs); break;
+    case 1: (void)(metis_launch_pdl((jacobi_eig_kernel<1>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    case 2: (void)(metis_launch_pdl((jacobi_eig_kernel<2>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    case 3: (void)(metis_launch_pdl((jacobi_eig_kernel<3>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    case 4: (void)(metis_launch_pdl((jacobi_eig_kernel<4>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    case 5: (void)(metis_launch_pdl((jacobi_eig_kernel<5>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    case 6: (void)(metis_launch_pdl((jacobi_eig_kernel<6>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    case 7: (void)(metis_launch_pdl((jacobi_eig_kernel<7>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    case 8: (void)(metis_launch_pdl((jacobi_eig_kernel<8>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    default: (void)(metis_launch_pdl((jacobi_eig_kernel<9>), dim3(1), dim3(288), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
   }
   METIS_COUNT_LAUNCH();
 }
@@ -1179,7 +1197,7 @@ void launch_jacobi(cudaStream_t s, const double* g, int n, int ld, float exit_co
 template <int NJ4>
 void launch_project(dim3 grid, cudaStream_t s, const __nv_bfloat16* x, int64_t cols, const int* idx, int n_s, int q,
                     const float* h, int rpp, float* mp) {
-  project_kernel<NJ4><<<grid, 256, 0, s>>>(x, cols, idx, n_s, q, h, rpp, mp); METIS_COUNT_LAUNCH();
+  (void)(metis_launch_pdl((project_kernel<NJ4>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, n_s, q, h, rpp, mp)); METIS_COUNT_LAUNCH();
 }
 
 int jacobi_threads(int n) {
@@ -1303,7 +1321,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   METIS_CUDA_TRY(cudaMemsetAsync(amax, 0, 64, s));       // amax slots of x, left, right and the condition flag
 
   // (1) row sample, (2) sketch (tensor cores; Omega generated per CTA into shared memory)
-  sample_rows_kernel<<<(unsigned)metis_ceil_div(n_s, 256), 256, 0, s>>>(idx, (int)n_s, rows, seed, full ? 1 : 0); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(metis_launch_pdl((sample_rows_kernel), dim3((unsigned)metis_ceil_div(n_s, 256)), dim3(256), (size_t)(0), s, idx, (int)n_s, rows, seed, full ? 1 : 0)); METIS_COUNT_LAUNCH();
   const int chunks = (int)metis_ceil_div(cols, SKM_COLS);
   {
     const int nt = (q + 7) / 8;
@@ -1311,27 +1329,27 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     dim3 grid((unsigned)metis_ceil_div(n_s, SKM_ROWS), (unsigned)chunks);
     float* am = full ? amax : nullptr;                  // FULL mode: amax|x| comes out of this pass
     switch (nt) {
-      case 1: sketch_mma_kernel<1><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
-      case 2: sketch_mma_kernel<2><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
-      case 3: sketch_mma_kernel<3><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
-      case 4: sketch_mma_kernel<4><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
-      case 5: sketch_mma_kernel<5><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
-      case 6: sketch_mma_kernel<6><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
-      case 7: sketch_mma_kernel<7><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
-      case 8: sketch_mma_kernel<8><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
-      default: sketch_mma_kernel<9><<<grid, 256, smem, s>>>(x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am); break;
+      case 1: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<1>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
+      case 2: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<2>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
+      case 3: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<3>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
+      case 4: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<4>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
+      case 5: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<5>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
+      case 6: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<6>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
+      case 7: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<7>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
+      case 8: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<8>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
+      default: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<9>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
     }
     METIS_COUNT_LAUNCH();
   }
-  reduce_partials_kernel<<<(unsigned)metis_ceil_div(n_s * q, 256), 256, 0, s>>>(zp, chunks, n_s * q, z); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(metis_launch_pdl((reduce_partials_kernel), dim3((unsigned)metis_ceil_div(n_s * q, 256)), dim3(256), (size_t)(0), s, zp, chunks, n_s * q, z)); METIS_COUNT_LAUNCH();
   // (3) CholeskyQR2: orthonormal basis H of range(Z), in place
   for (int pass = 0; pass < 2; ++pass) {
     int64_t rpp; const int parts = gram_parts(n_s, &rpp);
     const int* skip = pass == 0 ? nullptr : cond_flag;
-    gram_kernel<<<parts, 256, 0, s>>>(z, n_s, q, q, 1, rpp, gram, skip); METIS_COUNT_LAUNCH();
-    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 32), 128, 0, s>>>(gram, parts, q * q, gram1, skip); METIS_COUNT_LAUNCH();
-    chol_kernel<<<1, 256, 0, s>>>(gram1, q, linv, invd, skip, pass == 0 ? cond_flag : nullptr); METIS_COUNT_LAUNCH();
-    apply_chol_kernel<<<(unsigned)metis_ceil_div(n_s, 8), 256, 0, s>>>(z, n_s, q, linv, invd, skip); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((gram_kernel), dim3(parts), dim3(256), (size_t)(0), s, z, n_s, q, q, 1, rpp, gram, skip)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((reduce_gram_kernel), dim3((unsigned)metis_ceil_div(q * q, 32)), dim3(128), (size_t)(0), s, gram, parts, q * q, gram1, skip)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((chol_kernel), dim3(1), dim3(256), (size_t)(0), s, gram1, q, linv, invd, skip, pass == 0 ? cond_flag : nullptr)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((apply_chol_kernel), dim3((unsigned)metis_ceil_div(n_s, 8)), dim3(256), (size_t)(0), s, z, n_s, q, linv, invd, skip)); METIS_COUNT_LAUNCH();
   }
   // (4) M = H^T x[S,:], eigen-decomposition of M M^T, right basis
   {
@@ -1343,11 +1361,11 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       parts = (int)metis_ceil_div(n_s, rpp);
       dim3 grid((unsigned)metis_ceil_div(cols, PM_COLS), (unsigned)parts);
       switch ((q + 15) / 16) {
-        case 1: project_mma_kernel<1><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
-        case 2: project_mma_kernel<2><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
-        case 3: project_mma_kernel<3><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
-        case 4: project_mma_kernel<4><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
-        default: project_mma_kernel<5><<<grid, 256, 0, s>>>(x, cols, idx, (int)n_s, q, z, rpp, mp); break;
+        case 1: METIS_CUDA_TRY(metis_launch_pdl((project_mma_kernel<1>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, (int)n_s, q, z, rpp, mp)); break;
+        case 2: METIS_CUDA_TRY(metis_launch_pdl((project_mma_kernel<2>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, (int)n_s, q, z, rpp, mp)); break;
+        case 3: METIS_CUDA_TRY(metis_launch_pdl((project_mma_kernel<3>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, (int)n_s, q, z, rpp, mp)); break;
+        case 4: METIS_CUDA_TRY(metis_launch_pdl((project_mma_kernel<4>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, (int)n_s, q, z, rpp, mp)); break;
+        default: METIS_CUDA_TRY(metis_launch_pdl((project_mma_kernel<5>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, (int)n_s, q, z, rpp, mp)); break;
       }
       METIS_COUNT_LAUNCH();
     } else {
@@ -1366,46 +1384,46 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       default: launch_project<9>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
     }
     }
-    reduce_partials_kernel<<<(unsigned)metis_ceil_div((int64_t)q * cols, 256), 256, 0, s>>>(mp, parts, (int64_t)q * cols, m); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((reduce_partials_kernel), dim3((unsigned)metis_ceil_div((int64_t)q * cols, 256)), dim3(256), (size_t)(0), s, mp, parts, (int64_t)q * cols, m)); METIS_COUNT_LAUNCH();
   }
   {
     int64_t rpp; const int parts = gram_parts(cols, &rpp);
-    gram_kernel<<<parts, 256, 0, s>>>(m, cols, q, 1, cols, rpp, gram, nullptr); METIS_COUNT_LAUNCH();
-    reduce_gram_kernel<<<(unsigned)metis_ceil_div(q * q, 32), 128, 0, s>>>(gram, parts, q * q, gram1, nullptr); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((gram_kernel), dim3(parts), dim3(256), (size_t)(0), s, m, cols, q, 1, cols, rpp, gram, nullptr)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((reduce_gram_kernel), dim3((unsigned)metis_ceil_div(q * q, 32)), dim3(128), (size_t)(0), s, gram, parts, q * q, gram1, nullptr)); METIS_COUNT_LAUNCH();
     launch_jacobi(s, gram1, q, q, 1e-8f, evals, evecs);
   }
-  right_basis_kernel<<<(unsigned)metis_ceil_div(cols, 64), 256, 0, s>>>(m, cols, q, k, evals, evecs, basis,
-                                                                          full ? out->sigma : nullptr); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(metis_launch_pdl((right_basis_kernel), dim3((unsigned)metis_ceil_div(cols, 64)), dim3(256), (size_t)(0), s, m, cols, q, k, evals, evecs, basis,
+                                                                          full ? out->sigma : nullptr)); METIS_COUNT_LAUNCH();
   // (5) coefficients of every row in the basis, (6) fused residual + quantizer
   const int n_cand = (int)metis_ceil_div(cols, 256);
   const int n_cta_c = (int)metis_ceil_div(rows, 32);
   if (full) {
     // left = H U~_k, right = basis (sign fixed); coefficients = left * sigma
-    right_rotate_kernel<<<dim3(n_cand, (k + 7) / 8), 256, 0, s>>>(basis, cols, k, nullptr, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
-    sign_fix_kernel<<<dim3(n_cand, k), 256, 0, s>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2); METIS_COUNT_LAUNCH();
-    basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(out->right, cols, k, kp, bs, bt, b6p, kx6); METIS_COUNT_LAUNCH();
-    left_rotate_kernel<<<dim3((unsigned)metis_ceil_div(rows, 64), (unsigned)((kp + 15) / 16)), 256, 0, s>>>(z, rows, q, k, 1, q, evecs, nullptr, sign,
-                                                                            out->left, nullptr, coef, kp, out->sigma, amax + 1); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((right_rotate_kernel), dim3(dim3(n_cand, (k + 7) / 8)), dim3(256), (size_t)(0), s, basis, cols, k, nullptr, out->right, cand_v, cand_i)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((sign_fix_kernel), dim3(dim3(n_cand, k)), dim3(256), (size_t)(0), s, out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((basis_splits_kernel), dim3((unsigned)metis_ceil_div(cols, 128)), dim3(128), (size_t)(0), s, out->right, cols, k, kp, bs, bt, b6p, kx6)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((left_rotate_kernel), dim3(dim3((unsigned)metis_ceil_div(rows, 64), (unsigned)((kp + 15) / 16))), dim3(256), (size_t)(0), s, z, rows, q, k, 1, q, evecs, nullptr, sign,
+                                                                            out->left, nullptr, coef, kp, out->sigma, amax + 1)); METIS_COUNT_LAUNCH();
   } else {
-    basis_splits_kernel<<<(unsigned)metis_ceil_div(cols, 128), 128, 0, s>>>(basis, cols, k, kp, bs, bt, b6p, kx6); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((basis_splits_kernel), dim3((unsigned)metis_ceil_div(cols, 128)), dim3(128), (size_t)(0), s, basis, cols, k, kp, bs, bt, b6p, kx6)); METIS_COUNT_LAUNCH();
     if (metis_coeff_tc_usable(x, bs, cols, kp)) {
       // tensor-core pass over x (column slices), then the slices are summed and the Gram partials formed
       METIS_TRY(metis_launch_coeff_tc(ctx, x, rows, cols, bs, kp, part, amax, s));
       a6_ready = resid_tc;
       const int slices = metis_coeff_slices(rows, cols, nullptr);
       switch (kp) {
-        case 16: coef_finish_kernel<16><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c, a6p, kx6); break;
-        case 32: coef_finish_kernel<32><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c, a6p, kx6); break;
-        case 48: coef_finish_kernel<48><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c, a6p, kx6); break;
-        default: coef_finish_kernel<64><<<n_cta_c, 256, 0, s>>>(part, slices, rows, coef, gram_c, a6p, kx6); break;
+        case 16: METIS_CUDA_TRY(metis_launch_pdl((coef_finish_kernel<16>), dim3(n_cta_c), dim3(256), (size_t)(0), s, part, slices, rows, coef, gram_c, a6p, kx6)); break;
+        case 32: METIS_CUDA_TRY(metis_launch_pdl((coef_finish_kernel<32>), dim3(n_cta_c), dim3(256), (size_t)(0), s, part, slices, rows, coef, gram_c, a6p, kx6)); break;
+        case 48: METIS_CUDA_TRY(metis_launch_pdl((coef_finish_kernel<48>), dim3(n_cta_c), dim3(256), (size_t)(0), s, part, slices, rows, coef, gram_c, a6p, kx6)); break;
+        default: METIS_CUDA_TRY(metis_launch_pdl((coef_finish_kernel<64>), dim3(n_cta_c), dim3(256), (size_t)(0), s, part, slices, rows, coef, gram_c, a6p, kx6)); break;
       }
     } else {
       const size_t smem = sizeof(float) * 9 * 32 * kp;
       switch (kp) {
-        case 16: coeff_mma_kernel<16><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
-        case 32: coeff_mma_kernel<32><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
-        case 48: coeff_mma_kernel<48><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
-        default: coeff_mma_kernel<64><<<n_cta_c, 256, smem, s>>>(x, rows, cols, bs, coef, amax, gram_c); break;
+        case 16: METIS_CUDA_TRY(metis_launch_pdl((coeff_mma_kernel<16>), dim3(n_cta_c), dim3(256), (size_t)(smem), s, x, rows, cols, bs, coef, amax, gram_c)); break;
+        case 32: METIS_CUDA_TRY(metis_launch_pdl((coeff_mma_kernel<32>), dim3(n_cta_c), dim3(256), (size_t)(smem), s, x, rows, cols, bs, coef, amax, gram_c)); break;
+        case 48: METIS_CUDA_TRY(metis_launch_pdl((coeff_mma_kernel<48>), dim3(n_cta_c), dim3(256), (size_t)(smem), s, x, rows, cols, bs, coef, amax, gram_c)); break;
+        default: METIS_CUDA_TRY(metis_launch_pdl((coeff_mma_kernel<64>), dim3(n_cta_c), dim3(256), (size_t)(smem), s, x, rows, cols, bs, coef, amax, gram_c)); break;
       }
     }
     METIS_COUNT_LAUNCH();
@@ -1427,10 +1445,10 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       METIS_TRY(metis_launch_residual_tc(ctx, x, a6_ready ? nullptr : coef, k, kp, qp, amax, t0, t1, residual_dense, a6, b6, sr));
     } else {
       switch (kp) {
-        case 16: residual_quant_kernel<16><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
-        case 32: residual_quant_kernel<32><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
-        case 48: residual_quant_kernel<48><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
-        default: residual_quant_kernel<64><<<grid, THREADS, smem, sr>>>(x, coef, bt, qp, amax, t0, t1, residual_dense); break;
+        case 16: METIS_CUDA_TRY(metis_launch_pdl((residual_quant_kernel<16>), dim3(grid), dim3(THREADS), (size_t)(smem), sr, x, coef, bt, qp, amax, t0, t1, residual_dense)); break;
+        case 32: METIS_CUDA_TRY(metis_launch_pdl((residual_quant_kernel<32>), dim3(grid), dim3(THREADS), (size_t)(smem), sr, x, coef, bt, qp, amax, t0, t1, residual_dense)); break;
+        case 48: METIS_CUDA_TRY(metis_launch_pdl((residual_quant_kernel<48>), dim3(grid), dim3(THREADS), (size_t)(smem), sr, x, coef, bt, qp, amax, t0, t1, residual_dense)); break;
+        default: METIS_CUDA_TRY(metis_launch_pdl((residual_quant_kernel<64>), dim3(grid), dim3(THREADS), (size_t)(smem), sr, x, coef, bt, qp, amax, t0, t1, residual_dense)); break;
       }
       METIS_COUNT_LAUNCH();
     }
@@ -1438,12 +1456,12 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   cudaStream_t sf = ctx->side[0];
   if (!full) {
     // (7) Rayleigh-Ritz on C^T C (Gram partials came out of the broadcast pass), rotate both factors
-    reduce_gram_kernel<<<(unsigned)metis_ceil_div(kp * kp, 32), 128, 0, sf>>>(gram_c, n_cta_c, kp * kp, gram1, nullptr); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((reduce_gram_kernel), dim3((unsigned)metis_ceil_div(kp * kp, 32)), dim3(128), (size_t)(0), sf, gram_c, n_cta_c, kp * kp, gram1, nullptr)); METIS_COUNT_LAUNCH();
     launch_jacobi(sf, gram1, k, kp, 1e-6f, evals2, evecs2);
-    right_rotate_kernel<<<dim3(n_cand, (k + 7) / 8), 256, 0, sf>>>(basis, cols, k, evecs2, out->right, cand_v, cand_i); METIS_COUNT_LAUNCH();
-    sign_fix_kernel<<<dim3(n_cand, k), 256, 0, sf>>>(out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2); METIS_COUNT_LAUNCH();
-    left_rotate_kernel<<<dim3((unsigned)metis_ceil_div(rows, 64), (unsigned)((kp + 15) / 16)), 256, 0, sf>>>(coef, rows, k, k, 1, kp, evecs2, evals2, sign,
-                                                                            out->left, out->sigma, nullptr, kp, nullptr, amax + 1); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((right_rotate_kernel), dim3(dim3(n_cand, (k + 7) / 8)), dim3(256), (size_t)(0), sf, basis, cols, k, evecs2, out->right, cand_v, cand_i)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((sign_fix_kernel), dim3(dim3(n_cand, k)), dim3(256), (size_t)(0), sf, out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((left_rotate_kernel), dim3(dim3((unsigned)metis_ceil_div(rows, 64), (unsigned)((kp + 15) / 16))), dim3(256), (size_t)(0), sf, coef, rows, k, k, 1, kp, evecs2, evals2, sign,
+                                                                            out->left, out->sigma, nullptr, kp, nullptr, amax + 1)); METIS_COUNT_LAUNCH();
   }
   METIS_CUDA_TRY(cudaGetLastError());
   // (8) quantize the factors (stored transposed: k x rows, k x cols; blocks along the long dimension)
