@@ -127,6 +127,33 @@ def test_factor_gradients_need_the_weight_gradient(ctx):
         h.linear_bwd(do, xo, wo, need_dw=False, factor_grads=(g, None, None))
 
 
+@pytest.mark.parametrize("kp", [(12, 4), (24, 8), (40, 0), (48, 8), (64, 8)])
+def test_rank_and_oversampling_range(ctx, kp):
+    """Ranks that are not multiples of 16 (padded coefficient blocks), no oversampling, and the largest rank."""
+    from gpu_util import to_dev_bf16, rel_fro
+    B, h = ctx
+    k, p = kp
+    l, m, n = 512, 768, 640
+    x, _ = synth.llama_like(l, m, 1.0, 91, rank=max(k, 8))
+    w, _ = synth.llama_like(n, m, 0.02, 92, rank=max(k, 8))
+    d, _ = synth.llama_like(l, n, 1e-4, 93, rank=max(k, 8))
+    xo = h.split(to_dev_bf16(x), k, p, sketch=B.SKETCH_SAMPLED, seed=1)
+    wo = h.split(to_dev_bf16(w), k, p, sketch=B.SKETCH_FULL, seed=2)
+    do = h.split(to_dev_bf16(d), k, p, sketch=B.SKETCH_SAMPLED, seed=3, rounding=B.ROUND_SR)
+    y = h.linear_fwd(xo, wo)
+    dx, dw = h.linear_bwd(do, xo, wo)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    xq = olay.quantize_operand(x, k, p, osp.MODE_SAMPLED, 1)
+    wq = olay.quantize_operand(w, k, p, osp.MODE_FULL, 2)
+    dq = olay.quantize_operand(d, k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
+    for op, q in ((xo, xq), (wo, wq), (do, dq)):
+        assert np.max(np.abs(op.sigma.cpu().numpy()[:k] - q.sigma) / q.sigma) < 1e-3
+    assert rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)) < TOL
+    assert rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)) < TOL
+    assert rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq)) < TOL
+
+
 def test_ragged_layer_through_the_two_cta_gemm(ctx):
     """l, m, n above 256 but not multiples of the 256-wide GEMM tiles: ragged tiles in every product, the fused
     low-rank correction boxes, tensor stores clipped at the matrix edge."""
