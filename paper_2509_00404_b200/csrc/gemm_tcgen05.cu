@@ -16,7 +16,6 @@
 // and addresses stay in uniform registers.  Every mbarrier wait is bounded; on expiry the kernel records
 // METIS_DEV_TIMEOUT and unwinds.
 #include <cuda.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -757,18 +756,12 @@ metis_status_t metis_launch_gemm_tc(metis_context* ctx, const metis_nvfp4_t* a, 
   if (!metis_aligned16(a->codes) || !metis_aligned16(b->codes) || !metis_aligned16(a->scales) || !metis_aligned16(b->scales))
     return METIS_ERR_ALIGNMENT;
   if (a->rows > INT32_MAX || b->rows > INT32_MAX || a->k_len > INT32_MAX) return METIS_ERR_SHAPE;
-  static int force_n = -1;
-  if (force_n < 0) { const char* e = getenv("METIS_GEMM_BLOCK_N"); force_n = e ? atoi(e) : 0; }
-  if (force_n == 256) return launch<256>(ctx, a, b, d, d_dtype, ldd, s);
-  if (force_n == 128) return launch<128>(ctx, a, b, d, d_dtype, ldd, s);
   if (a->rows >= 256 && b->rows >= 256) return launch_2cta(ctx, a, b, d, d_dtype, ldd, nullptr, nullptr, 0, s);
   return launch<128>(ctx, a, b, d, d_dtype, ldd, s);
 }
 
 bool metis_gemm_tc_can_fuse(const metis_nvfp4_t* a, const metis_nvfp4_t* b) {
-  static int force_n = -1;
-  if (force_n < 0) { const char* e = getenv("METIS_GEMM_BLOCK_N"); force_n = e ? atoi(e) : 0; }
-  return force_n == 0 && a->rows >= 256 && b->rows >= 256;
+  return a->rows >= 256 && b->rows >= 256;
 }
 
 // d = alpha * (a b^T) + alpha * (lx rx^T): lx (M x kx) and rx (N x kx) are row-major BF16, kx a multiple of 64.
