@@ -37,6 +37,9 @@ static inline metis_status_t metis_join(metis_context* ctx, cudaStream_t main, i
 // returns when the preceding kernel has completed and its writes are visible).  Saves the launch gap between
 // the many short dependent kernels of a decomposition.
 __device__ __forceinline__ void metis_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream (if it was launched with the helper below) be scheduled as soon as SMs have
+// room, before this kernel has finished; it still waits for this kernel's completion in its own metis_pdl_wait().
+__device__ __forceinline__ void metis_pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>
 static inline cudaError_t metis_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {

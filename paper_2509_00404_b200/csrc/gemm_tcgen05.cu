@@ -105,6 +105,7 @@ template <int BLOCK_N>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmArgs g) {
   using C = Cfg<BLOCK_N>;
+  metis_pdl_trigger();
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;              // 1024-byte alignment for the 128-byte swizzle
@@ -138,6 +139,8 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above touched only this CTA's shared and tensor memory: it may overlap the previous kernel's tail
+  metis_pdl_wait();
 
   if (warp == 0) {
     // ------------------------------- producer -------------------------------
@@ -354,6 +357,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                        const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
                        const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUtensorMap map_r,
                        const __grid_constant__ CUtensorMap map_d, GemmArgs g) {
+  metis_pdl_trigger();
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -405,6 +409,8 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   cluster_sync();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above touched only this CTA's shared and tensor memory: it may overlap the previous kernel's tail
+  metis_pdl_wait();
 
   if (warp == 0) {
     // ------------------------------- producer (both CTAs) -------------------
@@ -669,8 +675,7 @@ metis_status_t launch(metis_context* ctx, const metis_nvfp4_t* a, const metis_nv
   }
   const int tiles = (int)(metis_ceil_div(g.M, BLOCK_M) * metis_ceil_div(g.N, BLOCK_N));
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-  gemm_nvfp4_kernel<BLOCK_N><<<grid, NUM_THREADS, C::SMEM_BYTES, s>>>(map_a, map_b, g); METIS_COUNT_LAUNCH();
-  METIS_CUDA_TRY(cudaGetLastError());
+  METIS_CUDA_TRY(metis_launch_pdl(gemm_nvfp4_kernel<BLOCK_N>, dim3(grid), dim3(NUM_THREADS), C::SMEM_BYTES, s, map_a, map_b, g)); METIS_COUNT_LAUNCH();
   return METIS_OK;
 }
 
@@ -741,8 +746,8 @@ metis_status_t launch_2cta(metis_context* ctx, const metis_nvfp4_t* a, const met
     max_pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
   }
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  two_cta::gemm_nvfp4_2cta_kernel<<<2 * pairs, two_cta::NUM_THREADS, two_cta::SMEM_BYTES, s>>>(map_a, map_b, map_sfa, map_sfb, map_l, map_r, map_d, g); METIS_COUNT_LAUNCH();
-  METIS_CUDA_TRY(cudaGetLastError());
+  METIS_CUDA_TRY(metis_launch_pdl(two_cta::gemm_nvfp4_2cta_kernel, dim3(2 * pairs), dim3(two_cta::NUM_THREADS), two_cta::SMEM_BYTES, s,
+                                  map_a, map_b, map_sfa, map_sfb, map_l, map_r, map_d, g)); METIS_COUNT_LAUNCH();
   return METIS_OK;
 }
 

@@ -39,6 +39,8 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
                       const float* res_a_ts, const float* res_b_ts) {
   __shared__ float ps[64][65];
   __shared__ float fa[8][64];
+  metis_pdl_wait();
+  metis_pdl_trigger();                                      // the large GEMM behind this kernel sets itself up meanwhile
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int kc = ka + kb;
   for (int o = tid; o < ka * kb; o += 256) ps[o / kb][o % kb] = pm[o];
@@ -336,11 +338,11 @@ metis_status_t split_gemm_prologue(metis_context* ctx, const Side& a, const Side
     METIS_TRY(metis_join(ctx, s, 1));
   }
   const int64_t mx = M > N ? M : N;
-  lowrank_finish_kernel<<<(unsigned)metis_ceil_div(mx, 8), 256, 0, s>>>(
+  METIS_CUDA_TRY(metis_launch_pdl(lowrank_finish_kernel, dim3((unsigned)metis_ceil_div(mx, 8)), dim3(256), 0, s,
       M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
       ka ? a.fo->tensor_scale : nullptr, a.sigma, kb ? b.fo->codes : nullptr, kb ? b.fo->scales : nullptr,
       kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, pl.pm, pl.lcat, pl.rcat, pl.lx, pl.rx, pl.kx,
-      a.res->tensor_scale, b.res->tensor_scale); METIS_COUNT_LAUNCH();
+      a.res->tensor_scale, b.res->tensor_scale)); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }
