@@ -908,17 +908,45 @@ sketch_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* 
 // Tensor-core projection: Mp[part][j][col] = sum over the part's sampled rows r of H[r][j] * x[idx[r], col].
 // The contraction runs over rows of the row-major x, so x tiles are staged in shared memory and read back
 // transposed with ldmatrix; H (FP32) is fed as three BF16 terms.  CTA = 128 columns x one slab of rows.
-constexpr int PM_COLS = 128, PM_ROWS = 32, PM_XP = PM_COLS + 8, PM_HP = PM_ROWS + 8;
+// ------------------------------------------------------------------------------------------------
+// Projection M = H^T x over many rows (every row in FULL mode), software-pipelined: the CTA owns 128 columns and
+// a slab of rows, and walks the slab in chunks of 64 rows through a three-stage cp.async ring (x rows gathered
+// by idx, the three BF16 terms of H pre-split and transposed by h_splits_kernel), so the loads of chunk c + 2
+// overlap the MMAs of chunk c.  Same partial layout as project_kernel: Mp[part][j][col].
+constexpr int PP_COLS = 128, PP_K = 64, PP_STAGES = 3, PP_XP = PP_COLS + 8, PP_HP = PP_K + 8;
+
+// hsp[sp][j][r] (r contiguous, ldh >= rows rounded up to 64, zero padded): three-term BF16 split of H[r][j]
+__global__ void __launch_bounds__(256)
+h_splits_kernel(const float* __restrict__ h, int n_s, int q, int jp, int ldh, __nv_bfloat16* __restrict__ hsp) {
+  metis_pdl_wait();
+  const int r = blockIdx.x * 256 + threadIdx.x, j = blockIdx.y;
+  if (r >= ldh) return;
+  const float v = (r < n_s && j < q) ? h[(int64_t)r * q + j] : 0.0f;
+  const __nv_bfloat16 hh = __float2bfloat16_rn(v);
+  const float r1 = v - __bfloat162float(hh);
+  const __nv_bfloat16 hl = __float2bfloat16_rn(r1);
+  hsp[((int64_t)0 * jp + j) * ldh + r] = hh;
+  hsp[((int64_t)1 * jp + j) * ldh + r] = hl;
+  hsp[((int64_t)2 * jp + j) * ldh + r] = __float2bfloat16_rn(r1 - __bfloat162float(hl));
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+  const int bytes = valid ? 16 : 0;                      // 0: the 16 destination bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+
 template <int MT>                                      // sketch columns / 16, rounded up
 __global__ void __launch_bounds__(256)
-project_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
-                   const float* __restrict__ h, int rows_per_part, float* __restrict__ mp) {
+project_pipe_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
+                    const __nv_bfloat16* __restrict__ hsp, int ldh, int rows_per_part, float* __restrict__ mp) {
   metis_pdl_wait();
-  __shared__ __align__(16) __nv_bfloat16 xs[PM_ROWS][PM_XP];
-  __shared__ __align__(16) __nv_bfloat16 hs[3][MT * 16][PM_HP];
+  extern __shared__ __align__(16) unsigned char psm[];
+  constexpr int XS_BYTES = PP_K * PP_XP * 2, HS_BYTES = 3 * MT * 16 * PP_HP * 2, STAGE = XS_BYTES + HS_BYTES;
+  const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(psm);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int64_t col0 = (int64_t)blockIdx.x * PM_COLS;
+  const int64_t col0 = (int64_t)blockIdx.x * PP_COLS;
   const int r_begin = blockIdx.y * rows_per_part, r_end = min(n_s, r_begin + rows_per_part);
+  const int n_chunks = (r_end - r_begin + PP_K - 1) / PP_K;
   float acc[MT][2][4];
 #pragma unroll
   for (int m = 0; m < MT; ++m)
@@ -926,29 +954,40 @@ project_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int*
     for (int n = 0; n < 2; ++n)
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[m][n][e] = 0.0f;
-  for (int r0 = r_begin; r0 < r_end; r0 += PM_ROWS) {
-    // stage 32 rows x 128 columns of x (16 bytes per thread-step) and the matching rows of H, split and transposed
-    for (int i = tid; i < PM_ROWS * (PM_COLS / 8); i += 256) {
+
+  auto load_chunk = [&](int c) {
+    const int st = c % PP_STAGES;
+    const int r0 = r_begin + c * PP_K;
+    const uint32_t xs = sbase + (uint32_t)st * STAGE, hs = xs + XS_BYTES;
+    for (int i = tid; i < PP_K * (PP_COLS / 8); i += 256) {
       const int rr = i >> 4, c8 = (i & 15) * 8;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (r0 + rr < r_end && col0 + c8 + 8 <= cols) v = *reinterpret_cast<const uint4*>(x + (int64_t)idx[r0 + rr] * cols + col0 + c8);
-      *reinterpret_cast<uint4*>(&xs[rr][c8]) = v;
+      const bool ok = r0 + rr < r_end && col0 + c8 + 8 <= cols;
+      const __nv_bfloat16* src = ok ? x + (int64_t)idx[r0 + rr] * cols + col0 + c8 : x;
+      cp_async16(xs + (uint32_t)(rr * PP_XP + c8) * 2u, src, ok);
     }
-    for (int i = tid; i < PM_ROWS * MT * 16; i += 256) {
-      const int rr = i / (MT * 16), j = i % (MT * 16);
-      const float v = (r0 + rr < r_end && j < q) ? h[(int64_t)(r0 + rr) * q + j] : 0.0f;
-      const __nv_bfloat16 hh = __float2bfloat16_rn(v);
-      const float r1 = v - __bfloat162float(hh);
-      const __nv_bfloat16 hl = __float2bfloat16_rn(r1);
-      hs[0][j][rr] = hh; hs[1][j][rr] = hl; hs[2][j][rr] = __float2bfloat16_rn(r1 - __bfloat162float(hl));
+    for (int i = tid; i < 3 * MT * 16 * (PP_K / 8); i += 256) {
+      const int row = i >> 3, k8 = (i & 7) * 8;          // row = sp * MT*16 + j
+      cp_async16(hs + (uint32_t)(row * PP_HP + k8) * 2u, hsp + (int64_t)row * ldh + r0 + k8, true);
     }
-    __syncthreads();
+  };
+
+  for (int c = 0; c < PP_STAGES - 1; ++c) {
+    if (c < n_chunks) load_chunk(c);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  for (int c = 0; c < n_chunks; ++c) {
+    asm volatile("cp.async.wait_group %0;" ::"n"(PP_STAGES - 2) : "memory");
+    __syncthreads();                                     // chunk c has landed; everyone is done with chunk c - 1
+    if (c + PP_STAGES - 1 < n_chunks) load_chunk(c + PP_STAGES - 1);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    const int st = c % PP_STAGES;
+    const uint32_t xs = sbase + (uint32_t)st * STAGE, hs = xs + XS_BYTES;
 #pragma unroll
-    for (int ks = 0; ks < PM_ROWS / 16; ++ks) {
+    for (int ks = 0; ks < PP_K / 16; ++ks) {
       uint32_t b[2][2];
 #pragma unroll
       for (int n = 0; n < 2; ++n) {
-        const uint32_t addr = (uint32_t)__cvta_generic_to_shared(&xs[ks * 16 + (lane & 15)][(warp * 2 + n) * 8]);
+        const uint32_t addr = xs + (uint32_t)((ks * 16 + (lane & 15)) * PP_XP + (warp * 2 + n) * 8) * 2u;
         asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(b[n][0]), "=r"(b[n][1]) : "r"(addr));
       }
 #pragma unroll
@@ -956,15 +995,13 @@ project_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int*
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
           uint32_t a[4];
-          a[0] = *reinterpret_cast<const uint32_t*>(&hs[sp][m * 16 + g][ks * 16 + 2 * t]);
-          a[1] = *reinterpret_cast<const uint32_t*>(&hs[sp][m * 16 + g + 8][ks * 16 + 2 * t]);
-          a[2] = *reinterpret_cast<const uint32_t*>(&hs[sp][m * 16 + g][ks * 16 + 2 * t + 8]);
-          a[3] = *reinterpret_cast<const uint32_t*>(&hs[sp][m * 16 + g + 8][ks * 16 + 2 * t + 8]);
+          const uint32_t addr = hs + (uint32_t)(((sp * MT + m) * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PP_HP + ks * 16 + (lane >> 4) * 8) * 2u;
+          asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(addr));
           mma_bf16(acc[m][0], a, b[0][0], b[0][1]);
           mma_bf16(acc[m][1], a, b[1][0], b[1][1]);
         }
     }
-    __syncthreads();
   }
   float* dst = mp + (int64_t)blockIdx.y * q * cols;
 #pragma unroll
@@ -979,6 +1016,7 @@ project_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int*
       }
     }
 }
+
 
 // right[j][col] = sum_i basis[i][col] * W[i][j] (W == nullptr: identity).  One thread per column; each CTA
 // also records, for every j, its entry of largest magnitude (signed value and column, lowest column on ties)
@@ -1116,7 +1154,7 @@ left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, i
 
 struct SplitWs {
   size_t amax, idx, zp, z, gram, gram1, linv, evals, evecs, mp, m, basis, coef, sign, cand_v, cand_i, evals2, evecs2, bs, bt,
-      gram_c, part, a6, b6, total;
+      gram_c, part, a6, b6, hsp, total;
 };
 
 constexpr int PJ_MAX_PARTS = 16;
@@ -1156,6 +1194,7 @@ SplitWs split_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s) {
   w.part = take(sizeof(float) * (size_t)metis_coeff_slices(rows, cols, nullptr) * kp * rows);
   w.a6 = take(sizeof(__nv_bfloat16) * (size_t)metis_residual_kx(kp) * rows);
   w.b6 = take(sizeof(__nv_bfloat16) * (size_t)metis_residual_kx(kp) * cols);
+  w.hsp = take(n_s >= 1024 ? sizeof(__nv_bfloat16) * 3 * (size_t)((q + 15) / 16 * 16) * (size_t)((n_s + 63) / 64 * 64) : 0);
   w.bs = take(sizeof(__nv_bfloat16) * 3 * (size_t)kp * cols);
   w.bt = take(sizeof(__nv_bfloat16) * 3 * (size_t)kp * cols);
   w.gram_c = take(sizeof(double) * (size_t)metis_ceil_div(rows, 32) * kp * kp);
@@ -1286,6 +1325,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   __nv_bfloat16* bt = reinterpret_cast<__nv_bfloat16*>(wsb + L.bt);
   double* gram_c = reinterpret_cast<double*>(wsb + L.gram_c);
   float* part = reinterpret_cast<float*>(wsb + L.part);
+  __nv_bfloat16* hsp = reinterpret_cast<__nv_bfloat16*>(wsb + L.hsp);
   void* a6 = wsb + L.a6;
   void* b6 = wsb + L.b6;
   // the residual kernel's K-concatenated BF16 operands are written by the kernels that produce coefficients and basis
@@ -1357,16 +1397,22 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     if (n_s >= 1024 && cols % 8 == 0) {
       parts = (int)metis_ceil_div(n_s, 512);
       if (parts > PJ_MAX_PARTS) parts = PJ_MAX_PARTS;
-      rpp = (int)(metis_ceil_div(metis_ceil_div(n_s, parts), PM_ROWS) * PM_ROWS);
+      rpp = (int)(metis_ceil_div(metis_ceil_div(n_s, parts), PP_K) * PP_K);
       parts = (int)metis_ceil_div(n_s, rpp);
-      dim3 grid((unsigned)metis_ceil_div(cols, PM_COLS), (unsigned)parts);
-      switch ((q + 15) / 16) {
-        case 1: METIS_CUDA_TRY(metis_launch_pdl((project_mma_kernel<1>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, (int)n_s, q, z, rpp, mp)); break;
-        case 2: METIS_CUDA_TRY(metis_launch_pdl((project_mma_kernel<2>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, (int)n_s, q, z, rpp, mp)); break;
-        case 3: METIS_CUDA_TRY(metis_launch_pdl((project_mma_kernel<3>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, (int)n_s, q, z, rpp, mp)); break;
-        case 4: METIS_CUDA_TRY(metis_launch_pdl((project_mma_kernel<4>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, (int)n_s, q, z, rpp, mp)); break;
-        default: METIS_CUDA_TRY(metis_launch_pdl((project_mma_kernel<5>), dim3(grid), dim3(256), (size_t)(0), s, x, cols, idx, (int)n_s, q, z, rpp, mp)); break;
+      const int mt = (q + 15) / 16, jp = mt * 16, ldh = (int)((n_s + 63) / 64 * 64);
+      METIS_CUDA_TRY(metis_launch_pdl(h_splits_kernel, dim3((unsigned)metis_ceil_div(ldh, 256), (unsigned)jp), dim3(256), (size_t)0, s, z, (int)n_s, q, jp, ldh, hsp)); METIS_COUNT_LAUNCH();
+      dim3 grid((unsigned)metis_ceil_div(cols, PP_COLS), (unsigned)parts);
+      const size_t psmem = (size_t)PP_STAGES * (PP_K * PP_XP * 2 + 3 * jp * PP_HP * 2);
+#define METIS_PP(MTV) { static bool at_ = false; if (!at_) { METIS_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<MTV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psmem)); at_ = true; } \
+        METIS_CUDA_TRY(metis_launch_pdl((project_pipe_kernel<MTV>), grid, dim3(256), psmem, s, x, cols, idx, (int)n_s, q, hsp, ldh, rpp, mp)); }
+      switch (mt) {
+        case 1: METIS_PP(1); break;
+        case 2: METIS_PP(2); break;
+        case 3: METIS_PP(3); break;
+        case 4: METIS_PP(4); break;
+        default: METIS_PP(5); break;
       }
+#undef METIS_PP
       METIS_COUNT_LAUNCH();
     } else {
     parts = project_parts(n_s, cols, &rpp);
