@@ -41,42 +41,70 @@ __global__ void reduce_partials_kernel(const float* __restrict__ zp, int n_chunk
 // Gram partials in FP64: part[p][i][j] = sum over the p-th slab of rows r of v(r,i) v(r,j),
 // v(r,i) = V[r*stride_row + i*stride_vec].
 constexpr int GR_TILE = 32;
+constexpr int GR_PITCH = MAXQ + 2;                      // doubles per tile row: even, so that 4-wide groups stay 16-byte aligned
+constexpr int GR_NB = (MAXQ + 3) / 4;                   // 4 x 4 output blocks per dimension
 __global__ void __launch_bounds__(256)
 gram_kernel(const float* __restrict__ v, int64_t n_rows, int n, int64_t stride_row, int64_t stride_vec,
             int64_t rows_per_part, double* __restrict__ part, const int* __restrict__ skip) {
   metis_pdl_wait();
   if (skip != nullptr && *skip) return;                 // second CholeskyQR pass not needed (see chol_kernel)
-  __shared__ float tile[GR_TILE][MAXQ + 1];
+  // The tile is converted to FP64 once when it is staged (FP32 -> FP64 conversions are a slow-rate instruction).
+  // A thread owns 4 x 4 blocks of the output: eight shared-memory loads feed sixteen multiply-adds, which keeps
+  // the kernel off the shared-memory pipe that bounds a one-output-per-thread formulation.
+  __shared__ __align__(16) double tile[GR_TILE][GR_PITCH];
   const int tid = threadIdx.x;
   const int64_t r_begin = (int64_t)blockIdx.x * rows_per_part;
   const int64_t r_end = min(n_rows, r_begin + rows_per_part);
-  double acc[(MAXQ * MAXQ + 255) / 256];
+  const int nb = (n + 3) / 4, n_blocks = nb * nb;
+  constexpr int BPT = (GR_NB * GR_NB + 255) / 256;      // blocks per thread at the largest n
+  double acc[BPT][4][4];
 #pragma unroll
-  for (int e = 0; e < (MAXQ * MAXQ + 255) / 256; ++e) acc[e] = 0.0;
+  for (int b = 0; b < BPT; ++b)
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[b][i][j] = 0.0;
+  for (int i = tid; i < GR_TILE * (GR_PITCH - n); i += 256) {                    // columns n .. pitch-1 stay zero
+    const int rr = i / (GR_PITCH - n), ii = n + i % (GR_PITCH - n);
+    tile[rr][ii] = 0.0;
+  }
   for (int64_t r0 = r_begin; r0 < r_end; r0 += GR_TILE) {
     for (int i = tid; i < GR_TILE * n; i += 256) {
       int rr, ii;
       if (stride_row == 1) { rr = i % GR_TILE; ii = i / GR_TILE; } else { ii = i % n; rr = i / n; }
-      tile[rr][ii] = (r0 + rr < r_end) ? v[(r0 + rr) * stride_row + ii * stride_vec] : 0.0f;
+      tile[rr][ii] = (r0 + rr < r_end) ? (double)v[(r0 + rr) * stride_row + ii * stride_vec] : 0.0;
     }
     __syncthreads();
 #pragma unroll
-    for (int e = 0; e < (MAXQ * MAXQ + 255) / 256; ++e) {
-      const int o = tid + e * 256;
-      if (o < n * n) {
-        const int i = o / n, j = o % n;
-        double a = acc[e];
-#pragma unroll 8
-        for (int rr = 0; rr < GR_TILE; ++rr) a += (double)tile[rr][i] * (double)tile[rr][j];
-        acc[e] = a;
+    for (int b = 0; b < BPT; ++b) {
+      const int o = tid + b * 256;
+      if (o < n_blocks) {
+        const int bi = o / nb, bj = o % nb;
+#pragma unroll 4
+        for (int rr = 0; rr < GR_TILE; ++rr) {
+          const double2 a01 = *reinterpret_cast<const double2*>(&tile[rr][4 * bi]), a23 = *reinterpret_cast<const double2*>(&tile[rr][4 * bi + 2]);
+          const double2 b01 = *reinterpret_cast<const double2*>(&tile[rr][4 * bj]), b23 = *reinterpret_cast<const double2*>(&tile[rr][4 * bj + 2]);
+          const double av[4] = {a01.x, a01.y, a23.x, a23.y}, bv[4] = {b01.x, b01.y, b23.x, b23.y};
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[b][i][j] += av[i] * bv[j];
+        }
       }
     }
     __syncthreads();
   }
 #pragma unroll
-  for (int e = 0; e < (MAXQ * MAXQ + 255) / 256; ++e) {
-    const int o = tid + e * 256;
-    if (o < n * n) part[(int64_t)blockIdx.x * n * n + o] = acc[e];
+  for (int b = 0; b < BPT; ++b) {
+    const int o = tid + b * 256;
+    if (o < n_blocks) {
+      const int bi = o / nb, bj = o % nb;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (4 * bi + i < n && 4 * bj + j < n) part[(int64_t)blockIdx.x * n * n + (4 * bi + i) * n + 4 * bj + j] = acc[b][i][j];
+    }
   }
 }
 
@@ -713,11 +741,14 @@ coef_finish_kernel(const float* __restrict__ part, int slices, int64_t rows, flo
     }
   }
   if (gram_part) {
+    __shared__ double cd[32 * KP];                      // converted once: FP32 -> FP64 is a slow-rate instruction
+    for (int o = tid; o < 32 * KP; o += 256) cd[o] = (double)cfin[o];
+    __syncthreads();
     for (int o = tid; o < KP * KP; o += 256) {
       const int i = o / KP, j = o % KP;
       double a = 0.0;
 #pragma unroll 8
-      for (int r = 0; r < 32; ++r) a += (double)cfin[r * KP + i] * (double)cfin[r * KP + j];
+      for (int r = 0; r < 32; ++r) a += cd[r * KP + i] * cd[r * KP + j];
       gram_part[(int64_t)blockIdx.x * KP * KP + o] = a;
     }
   }
