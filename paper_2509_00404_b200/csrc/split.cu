@@ -854,14 +854,15 @@ constexpr int SKM_ROWS = 256, SKM_COLS = 256, SKM_PITCH = SKM_COLS + 8;
 template <int NT>                                      // sketch columns / 8, rounded up
 __global__ void __launch_bounds__(256)
 sketch_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __restrict__ idx, int n_s, int q,
-                  uint64_t seed, const __nv_bfloat16* __restrict__ lut, float* __restrict__ zp, float* __restrict__ amax_out) {
+                  uint64_t seed, const __nv_bfloat16* __restrict__ lut, float* __restrict__ zp, float* __restrict__ amax_out,
+                  int ccols) {
   metis_pdl_wait();
   extern __shared__ __align__(16) unsigned char smem[];
   __nv_bfloat16* om = reinterpret_cast<__nv_bfloat16*>(smem);          // [NT*8][SKM_PITCH]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int64_t col0 = (int64_t)blockIdx.y * SKM_COLS;
+  const int64_t col0 = (int64_t)blockIdx.y * ccols;        // ccols <= SKM_COLS columns per CTA
   const int row0 = blockIdx.x * SKM_ROWS + warp * 32;
-  const int ncols = (int)min((int64_t)SKM_COLS, cols - col0);
+  const int ncols = (int)min((int64_t)ccols, cols - col0);
   for (int i = tid; i < NT * 8 * SKM_PITCH; i += 256) om[i] = __float2bfloat16_rn(0.0f);
   __syncthreads();
   const uint64_t e_lo = (uint64_t)col0 * q, e_hi = (uint64_t)(col0 + ncols) * q;
@@ -1183,6 +1184,10 @@ left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, i
   if ((tid & 31) == 0 && amax_out != nullptr) atomicMax(reinterpret_cast<unsigned int*>(amax_out), __float_as_uint(am));
 }
 
+// Columns per sketch CTA: a sampled sketch has few rows, so narrow chunks are what gives it enough CTAs; a full
+// sketch has one CTA per 256 rows already and wide chunks keep the partial buffer small.
+int sketch_chunk_cols(int64_t n_s) { return n_s <= 512 ? 64 : SKM_COLS; }
+
 struct SplitWs {
   size_t amax, idx, zp, z, gram, gram1, linv, evals, evecs, mp, m, basis, coef, sign, cand_v, cand_i, evals2, evecs2, bs, bt,
       gram_c, part, a6, b6, hsp, total;
@@ -1207,7 +1212,7 @@ SplitWs split_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) & ~(size_t)255; return o; };
   const int q = k + p;
-  const int64_t chunks = metis_ceil_div(cols, SKM_COLS);
+  const int64_t chunks = metis_ceil_div(cols, sketch_chunk_cols(n_s));
   w.amax = take(256);
   w.idx = take(sizeof(int) * (size_t)n_s);
   w.zp = take(sizeof(float) * (size_t)chunks * n_s * q);
@@ -1287,8 +1292,11 @@ int64_t metis_default_sample_count(int64_t rows, int32_t q) {
 }
 
 size_t metis_split_ws_bytes(int64_t rows, int64_t cols, int k, int p) {
-  // sized for the FULL sketch (n_s = rows), which bounds the SAMPLED one
-  return split_ws_layout(rows, cols, k, p, rows).total;
+  // Every buffer grows with the sample count except the sketch partials, whose chunk width steps from 64 to 256
+  // columns above 512 sampled rows: the FULL sketch (n_s = rows) and a 512-row sample bound every other case.
+  const size_t full = split_ws_layout(rows, cols, k, p, rows).total;
+  const size_t narrow = split_ws_layout(rows, cols, k, p, rows < 512 ? rows : 512).total;
+  return full > narrow ? full : narrow;
 }
 
 metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64_t cols, int32_t k, int32_t p,
@@ -1393,22 +1401,23 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
 
   // (1) row sample, (2) sketch (tensor cores; Omega generated per CTA into shared memory)
   METIS_CUDA_TRY(metis_launch_pdl((sample_rows_kernel), dim3((unsigned)metis_ceil_div(n_s, 256)), dim3(256), (size_t)(0), s, idx, (int)n_s, rows, seed, full ? 1 : 0)); METIS_COUNT_LAUNCH();
-  const int chunks = (int)metis_ceil_div(cols, SKM_COLS);
+  const int ccols = sketch_chunk_cols(n_s);
+  const int chunks = (int)metis_ceil_div(cols, ccols);
   {
     const int nt = (q + 7) / 8;
     const size_t smem = sizeof(__nv_bfloat16) * nt * 8 * SKM_PITCH;
     dim3 grid((unsigned)metis_ceil_div(n_s, SKM_ROWS), (unsigned)chunks);
     float* am = full ? amax : nullptr;                  // FULL mode: amax|x| comes out of this pass
     switch (nt) {
-      case 1: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<1>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
-      case 2: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<2>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
-      case 3: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<3>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
-      case 4: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<4>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
-      case 5: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<5>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
-      case 6: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<6>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
-      case 7: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<7>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
-      case 8: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<8>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
-      default: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<9>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am)); break;
+      case 1: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<1>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am, ccols)); break;
+      case 2: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<2>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am, ccols)); break;
+      case 3: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<3>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am, ccols)); break;
+      case 4: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<4>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am, ccols)); break;
+      case 5: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<5>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am, ccols)); break;
+      case 6: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<6>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am, ccols)); break;
+      case 7: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<7>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am, ccols)); break;
+      case 8: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<8>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am, ccols)); break;
+      default: METIS_CUDA_TRY(metis_launch_pdl((sketch_mma_kernel<9>), dim3(grid), dim3(256), (size_t)(smem), s, x, cols, idx, (int)n_s, q, seed, ctx->quantile_lut, zp, am, ccols)); break;
     }
     METIS_COUNT_LAUNCH();
   }
