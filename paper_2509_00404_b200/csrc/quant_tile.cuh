@@ -55,6 +55,54 @@ __device__ __forceinline__ uint32_t encode_block(const float (&v)[16], const uin
   return byte;
 }
 
+// The element multiplier r = 1 / (E4M3(byte) * s_T) depends only on the block's scale byte and the tensor scale, so a
+// kernel can evaluate the defined operations once per byte and look the result up per block (0 for byte 0).
+constexpr int R_TABLE = 128;
+__device__ __forceinline__ void fill_r_table(float* tab, float s_T, int tid, int nthreads) {
+  for (int b = tid; b < R_TABLE; b += nthreads)
+    tab[b] = (b == 0 || b == 127) ? 0.0f : __fdiv_rn(1.0f, __fmul_rn(metis_e4m3_value((uint32_t)b), s_T));
+}
+
+// four round-to-nearest-even code bytes (eight values) packed into one word
+__device__ __forceinline__ uint32_t e2m1x8_rne(float a0, float a1, float a2, float a3, float a4, float a5, float a6, float a7) {
+  uint32_t w;
+  asm("{ .reg .b8 t0, t1, t2, t3;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 t2, %6, %5;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 t3, %8, %7;\n"
+      "mov.b32 %0, {t0, t1, t2, t3}; }"
+      : "=r"(w) : "f"(a0), "f"(a1), "f"(a2), "f"(a3), "f"(a4), "f"(a5), "f"(a6), "f"(a7));
+  return w;
+}
+
+// encode_block with the multiplier looked up in a table filled by fill_r_table (same bytes as encode_block)
+__device__ __forceinline__ uint32_t encode_block_tab(const float (&v)[16], const uint32_t (&u)[16], bool sr, float six_s_T,
+                                                     const float* r_tab, uint32_t (&packed)[2]) {
+  float m8[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) m8[i] = fmaxf(fabsf(v[i]), fabsf(v[i + 8]));
+  const float amax = fmaxf(fmaxf(fmaxf(m8[0], m8[4]), fmaxf(m8[1], m8[5])), fmaxf(fmaxf(m8[2], m8[6]), fmaxf(m8[3], m8[7])));
+  const float t = fminf(__fdiv_rn(amax, six_s_T), 448.0f);
+  float sb_unused;
+  const uint32_t byte = metis_e4m3_ceil(t, &sb_unused);
+  const float r = r_tab[byte];
+  if (!sr) {
+    packed[0] = e2m1x8_rne(__fmul_rn(v[0], r), __fmul_rn(v[1], r), __fmul_rn(v[2], r), __fmul_rn(v[3], r),
+                           __fmul_rn(v[4], r), __fmul_rn(v[5], r), __fmul_rn(v[6], r), __fmul_rn(v[7], r));
+    packed[1] = e2m1x8_rne(__fmul_rn(v[8], r), __fmul_rn(v[9], r), __fmul_rn(v[10], r), __fmul_rn(v[11], r),
+                           __fmul_rn(v[12], r), __fmul_rn(v[13], r), __fmul_rn(v[14], r), __fmul_rn(v[15], r));
+  } else {
+    packed[0] = packed[1] = 0u;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint32_t c = metis_e2m1_sr(__fmul_rn(v[i], r), u[i]);
+      packed[i >> 3] |= c << (4 * (i & 7));
+    }
+  }
+  return byte;
+}
+
 // tile:  [TILE][PITCH] floats, rows/cols outside the matrix already zero-filled
 // rnd:   [TILE][TILE] 16-bit draws (only read when rounding == SR)
 // stage: scratch

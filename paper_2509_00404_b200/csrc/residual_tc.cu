@@ -24,16 +24,17 @@ namespace {
 
 using namespace metis_tc;
 using metis_qt::QuantParams;
-using metis_qt::encode_block;
+using metis_qt::encode_block_tab;
 
 constexpr int TM = 128, TN = 128, BK = 64;
 constexpr int RING = 3;
 constexpr int SLOT_BYTES = 2 * TM * BK * 2;               // A6 chunk + B6 chunk, 16 KiB each
 constexpr int X_BYTES = TM * TN * 2;                      // two 64-column boxes of 16 KiB
-constexpr int PATCH_F = 32 * 33;                          // floats per warp patch
-constexpr int PATCH_U = 32 * 34;                          // 16-bit draws per warp patch
-constexpr int NUM_THREADS = 320;                          // producer, MMA issuer, 8 epilogue warps
-constexpr size_t SMEM_BYTES = (size_t)RING * SLOT_BYTES + 2 * X_BYTES + 8 * (PATCH_F * 4 + PATCH_U * 2) + 1024 + 256;
+constexpr int N_EW = 16;                                  // epilogue warps: four TMEM lane quarters x four column quarters
+constexpr int PATCH_F = 32 * 17;                          // floats per warp patch (32 rows x 16 columns, odd pitch)
+constexpr int PATCH_U = 32 * 18;                          // 16-bit draws per warp patch
+constexpr int NUM_THREADS = 64 + 32 * N_EW;               // producer, MMA issuer, epilogue warps
+constexpr size_t SMEM_BYTES = (size_t)RING * SLOT_BYTES + 2 * X_BYTES + N_EW * (PATCH_F * 4 + PATCH_U * 2) + 1024 + 256 + metis_qt::R_TABLE * 4;
 
 struct ResidArgs {
   QuantParams p;
@@ -70,6 +71,10 @@ splits6_kernel(const float* __restrict__ src, int64_t n, int k, int kp, int kx, 
   *dst = sel == 0 ? h : (sel == 1 ? l : l2);
 }
 
+// SR: stochastic rounding (compile-time, so the round-to-nearest kernel carries no draws).  FAST: the matrix is a whole
+// number of 128 x 128 tiles, both scale layouts are the tiled one and no dense residual is asked for, so every
+// bounds test and layout switch of the epilogue folds away.
+template <bool SR, bool FAST>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_a,
                    const __grid_constant__ CUtensorMap map_b, ResidArgs g) {
@@ -81,15 +86,16 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
   auto b_addr = [&](int s) { return a_addr(s) + TM * BK * 2; };
   auto x_addr = [&](int xb) { return base + (uint32_t)RING * SLOT_BYTES + (uint32_t)xb * X_BYTES; };
   const size_t patch_off = (size_t)RING * SLOT_BYTES + 2 * X_BYTES;
-  const uint32_t bar_base = base + (uint32_t)(patch_off + 8 * (PATCH_F * 4 + PATCH_U * 2));
+  const uint32_t bar_base = base + (uint32_t)(patch_off + N_EW * (PATCH_F * 4 + PATCH_U * 2));
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (RING + s); };
   auto xfull_bar = [&](int xb) { return bar_base + 8u * (2 * RING + xb); };
   auto xempty_bar = [&](int xb) { return bar_base + 8u * (2 * RING + 2 + xb); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * RING + 4 + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * RING + 6 + a); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + patch_off + 8 * (PATCH_F * 4 + PATCH_U * 2) + 8 * (2 * RING + 8));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + patch_off + N_EW * (PATCH_F * 4 + PATCH_U * 2) + 8 * (2 * RING + 8));
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* r_tab = reinterpret_cast<float*>(gen_base + patch_off + N_EW * (PATCH_F * 4 + PATCH_U * 2) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const QuantParams& p = g.p;
@@ -99,8 +105,8 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
   if (threadIdx.x == 0) {
     for (int s = 0; s < RING; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(xfull_bar(b), 1); mbar_init(xempty_bar(b), 8);
-      mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8);
+      mbar_init(xfull_bar(b), 1); mbar_init(xempty_bar(b), N_EW);
+      mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), N_EW);
     }
     *dead = 0;
     fence_barrier_init();
@@ -167,13 +173,16 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     }
   } else {
     // ------------------------------- epilogue -------------------------------
-    const int ew = warp - 2;                                // 0..7
-    const int quarter = warp & 3, half = ew >> 2;           // TMEM lane quarter (fixed by the warp id), column half
+    const int ew = warp - 2;                                // 0..15
+    const int quarter = warp & 3, colq = ew >> 2;           // TMEM lane quarter (fixed by the warp id), column quarter
     float* patch = reinterpret_cast<float*>(gen_base + patch_off) + ew * PATCH_F;
-    uint16_t* upatch = reinterpret_cast<uint16_t*>(gen_base + patch_off + 8 * PATCH_F * 4) + ew * PATCH_U;
-    const bool sr = p.rounding == METIS_ROUND_SR;
+    uint16_t* upatch = reinterpret_cast<uint16_t*>(gen_base + patch_off + N_EW * PATCH_F * 4) + ew * PATCH_U;
+    constexpr bool sr = SR;
+    const int c_layout = FAST ? (int)METIS_SF_TILED : p.c_layout, r_layout = FAST ? (int)METIS_SF_TILED : p.r_layout;
     const float s_T = metis_tensor_scale(*g.amax_src);
     const float six_s_T = __fmul_rn(6.0f, s_T);
+    metis_qt::fill_r_table(r_tab, s_T, (int)threadIdx.x - 64, 32 * N_EW);
+    asm volatile("bar.sync 1, %0;" ::"n"(32 * N_EW) : "memory");       // the epilogue warps only
     if (blockIdx.x == 0 && threadIdx.x == 64) {
       if (g.ts_out0) *g.ts_out0 = s_T;
       if (g.ts_out1) *g.ts_out1 = s_T;
@@ -189,21 +198,21 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
       if (!mbar_wait(tfull_bar(acc), par, g.dev_status, dead)) { ok = false; break; }
       tc_fence_after();
       const int64_t row = (int64_t)row0 + quarter * 32 + lane;              // this thread's row
-      const bool row_ok = row < p.rows;
+      const bool row_ok = FAST || row < p.rows;
       const int64_t slab_row0 = (int64_t)row0 + quarter * 32;               // first row of the warp's 32
-      const uint32_t xrow = x_addr(xb) + (uint32_t)half * (X_BYTES / 2) + (uint32_t)(quarter * 32 + lane) * 128u;
+      const int64_t c0 = (int64_t)col0 + colq * 32;                         // first of this warp's 32 columns
+      // x tile: two 64-column boxes of 128-byte rows, 16-byte chunks XOR-swizzled by the row
+      const uint32_t xrow = x_addr(xb) + (uint32_t)(colq >> 1) * (X_BYTES / 2) + (uint32_t)(quarter * 32 + lane) * 128u;
       const uint32_t sw = (uint32_t)((quarter * 32 + lane) & 7);
-#pragma unroll 1
-      for (int cc = 0; cc < 2; ++cc) {
-        const int64_t c0 = (int64_t)col0 + half * 64 + cc * 32;             // first of this step's 32 columns
+      float v[32];
+      {
         uint32_t a[32];
-        tc_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * TN + half * 64 + cc * 32), a);
-        float v[32];
+        tc_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * TN + colq * 32), a);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           uint32_t w0, w1, w2, w3;
           asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
-                       : "r"(xrow + ((((uint32_t)(4 * cc + j)) ^ sw) << 4)));
+                       : "r"(xrow + ((((uint32_t)(4 * (colq & 1) + j)) ^ sw) << 4)));
           const uint32_t ws[4] = {w0, w1, w2, w3};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
@@ -211,82 +220,81 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             v[8 * j + 2 * e + 1] = __uint_as_float(ws[e] & 0xFFFF0000u) - __uint_as_float(a[8 * j + 2 * e + 1]);
           }
         }
-        if (cc == 1) {
-          // accumulator and x tile fully read: hand both back
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) { mbar_arrive(tempty_bar(acc)); mbar_arrive(xempty_bar(xb)); }
+      }
+      // accumulator and x tile read: hand both back
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(tempty_bar(acc)); mbar_arrive(xempty_bar(xb)); }
+      const bool step_ok = FAST || c0 < p.cols;                                      // false: the warp's columns lie outside the matrix
+      const bool blk1_ok = FAST || c0 + 16 < p.cols;
+      uint32_t u[32];
+      if (sr) {
+        const uint64_t e0 = (uint64_t)row * (uint64_t)p.e_stride_r + (uint64_t)c0;        // multiple of 8
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const uint4 w = metis_philox_block((e0 >> 3) + q4, p.seed, p.stream_id);
+#pragma unroll
+          for (uint32_t hh = 0; hh < 8; ++hh) u[8 * q4 + hh] = metis_u16_of(w, hh);
         }
-        const bool step_ok = c0 < p.cols;                                    // false: the whole step lies outside the matrix
-        const bool blk1_ok = c0 + 16 < p.cols;
-        uint32_t u[32];
-        if (sr) {
-          const uint64_t e0 = (uint64_t)row * (uint64_t)p.e_stride_r + (uint64_t)c0;      // multiple of 8
+      }
+      if (!FAST && g.dense != nullptr && row_ok && step_ok) {
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            const uint4 w = metis_philox_block((e0 >> 3) + q4, p.seed, p.stream_id);
+        for (int j = 0; j < 8; ++j)
+          if (c0 + 4 * j < p.cols)
+            *reinterpret_cast<float4*>(g.dense + row * p.cols + c0 + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+      }
+      if (p.c_codes != nullptr && step_ok) {
+        // blocks along the columns: two blocks of this row, from registers
+        float v0[16], v1[16];
+        uint32_t u0[16], u1[16];
 #pragma unroll
-            for (uint32_t hh = 0; hh < 8; ++hh) u[8 * q4 + hh] = metis_u16_of(w, hh);
-          }
+        for (int i = 0; i < 16; ++i) { v0[i] = v[i]; v1[i] = v[16 + i]; u0[i] = sr ? u[i] : 0u; u1[i] = sr ? u[16 + i] : 0u; }
+        uint32_t pk0[2], pk1[2];
+        const uint32_t sb0 = encode_block_tab(v0, u0, sr, six_s_T, r_tab, pk0);
+        const uint32_t sb1 = encode_block_tab(v1, u1, sr, six_s_T, r_tab, pk1);
+        if (row_ok) {
+          uint8_t* cp = p.c_codes + row * c_kbytes + c0 / 2;
+          if (blk1_ok) *reinterpret_cast<uint4*>(cp) = make_uint4(pk0[0], pk0[1], pk1[0], pk1[1]);
+          else *reinterpret_cast<uint2*>(cp) = make_uint2(pk0[0], pk0[1]);
         }
-        if (g.dense != nullptr && row_ok && step_ok) {
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            if (c0 + 4 * j < p.cols)
-              *reinterpret_cast<float4*>(g.dense + row * p.cols + c0 + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-        }
-        if (p.c_codes != nullptr && step_ok) {
-          // blocks along the columns: two blocks of this row, from registers
-          float v0[16], v1[16];
-          uint32_t u0[16], u1[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) { v0[i] = v[i]; v1[i] = v[16 + i]; u0[i] = sr ? u[i] : 0u; u1[i] = sr ? u[16 + i] : 0u; }
-          uint32_t pk0[2], pk1[2];
-          const uint32_t sb0 = encode_block(v0, u0, sr, s_T, six_s_T, pk0);
-          const uint32_t sb1 = encode_block(v1, u1, sr, s_T, six_s_T, pk1);
-          if (row_ok) {
-            uint8_t* cp = p.c_codes + row * c_kbytes + c0 / 2;
-            if (blk1_ok) *reinterpret_cast<uint4*>(cp) = make_uint4(pk0[0], pk0[1], pk1[0], pk1[1]);
-            else *reinterpret_cast<uint2*>(cp) = make_uint2(pk0[0], pk0[1]);
-          }
-          if (row_ok || p.c_layout == METIS_SF_TILED) {                     // padded rows of a 128-row slab get zero scales
-            const int64_t o = metis_sf_offset(row, c0 / 16, c_bpr, p.c_layout);
+        if (row_ok || c_layout == METIS_SF_TILED) {                         // padded rows of a 128-row slab get zero scales
+          const int64_t o = metis_sf_offset(row, c0 / 16, c_bpr, c_layout);
+          if (FAST) {
+            *reinterpret_cast<uint16_t*>(p.c_scales + o) = (uint16_t)(sb0 | (sb1 << 8));   // c0 / 16 is even: an aligned pair
+          } else {
             p.c_scales[o] = row_ok ? (uint8_t)sb0 : (uint8_t)0;
             if (blk1_ok) p.c_scales[o + 1] = row_ok ? (uint8_t)sb1 : (uint8_t)0;
           }
         }
-        if (p.r_codes != nullptr && (step_ok || p.r_layout == METIS_SF_TILED)) {
-          // blocks along the rows: transpose the warp's 32 x 32 patch, lane = column
+      }
+      if (p.r_codes != nullptr && (step_ok || r_layout == METIS_SF_TILED)) {
+        // blocks along the rows: the warp transposes its 32 x 32 values 16 columns at a time through its patch;
+        // in each half lane l encodes the block of column l % 16, rows 16 * (l / 16) .. +15
+        const int cb = lane & 15, rb = lane >> 4;
+        const bool rb_ok = FAST || slab_row0 + 16 * rb < p.rows;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) patch[lane * 33 + i] = v[i];
+        for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) patch[lane * 17 + i] = v[16 * hf + i];
           if (sr) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) upatch[lane * 34 + i] = (uint16_t)u[i];
+            for (int i = 0; i < 16; ++i) upatch[lane * 18 + i] = (uint16_t)u[16 * hf + i];
           }
           __syncwarp();
-          const int64_t col = c0 + lane;
-          const bool col_ok = col < p.cols;
-          float t0[16], t1[16];
-          uint32_t d0[16], d1[16];
+          const int64_t col = c0 + 16 * hf + cb;
+          const bool col_ok = FAST || col < p.cols;
+          float t[16];
+          uint32_t d[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            t0[i] = patch[i * 33 + lane]; t1[i] = patch[(16 + i) * 33 + lane];
-            d0[i] = sr ? (uint32_t)upatch[i * 34 + lane] : 0u; d1[i] = sr ? (uint32_t)upatch[(16 + i) * 34 + lane] : 0u;
+            t[i] = patch[(16 * rb + i) * 17 + cb];
+            d[i] = sr ? (uint32_t)upatch[(16 * rb + i) * 18 + cb] : 0u;
           }
-          uint32_t pk0[2], pk1[2];
-          const uint32_t sb0 = encode_block(t0, d0, sr, s_T, six_s_T, pk0);
-          const uint32_t sb1 = encode_block(t1, d1, sr, s_T, six_s_T, pk1);
-          const bool rb0_ok = slab_row0 < p.rows, rb1_ok = slab_row0 + 16 < p.rows;
-          if (col_ok && rb0_ok) {
-            uint8_t* cp = p.r_codes + col * r_kbytes + slab_row0 / 2;
-            if (rb1_ok) *reinterpret_cast<uint4*>(cp) = make_uint4(pk0[0], pk0[1], pk1[0], pk1[1]);
-            else *reinterpret_cast<uint2*>(cp) = make_uint2(pk0[0], pk0[1]);
-          }
-          if (rb0_ok && (col_ok || p.r_layout == METIS_SF_TILED)) {         // padded columns of a 128-slab get zero scales
-            const int64_t o = metis_sf_offset(col, slab_row0 / 16, r_bpr, p.r_layout);
-            p.r_scales[o] = col_ok ? (uint8_t)sb0 : (uint8_t)0;
-            if (rb1_ok) p.r_scales[o + 1] = col_ok ? (uint8_t)sb1 : (uint8_t)0;
-          }
+          uint32_t pk[2];
+          const uint32_t sb = encode_block_tab(t, d, sr, six_s_T, r_tab, pk);
+          if (col_ok && rb_ok) *reinterpret_cast<uint2*>(p.r_codes + col * r_kbytes + (slab_row0 + 16 * rb) / 2) = make_uint2(pk[0], pk[1]);
+          if (rb_ok && (col_ok || r_layout == METIS_SF_TILED))               // padded columns of a 128-slab get zero scales
+            p.r_scales[metis_sf_offset(col, slab_row0 / 16 + rb, r_bpr, r_layout)] = col_ok ? (uint8_t)sb : (uint8_t)0;
           __syncwarp();
         }
       }
@@ -335,9 +343,16 @@ metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const
   g.dev_status = ctx->dev_status;
   static bool attr = false;
   if (!attr) {
-    METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
     attr = true;
   }
+  const bool fast = rows % TM == 0 && cols % TN == 0 && dense == nullptr &&
+                    (qp.c_codes == nullptr || (qp.c_layout == METIS_SF_TILED && reinterpret_cast<uintptr_t>(qp.c_scales) % 2 == 0)) &&
+                    (qp.r_codes == nullptr || qp.r_layout == METIS_SF_TILED);
+  const bool sr = qp.rounding == METIS_ROUND_SR;
   const int64_t tiles = metis_ceil_div(rows, TM) * metis_ceil_div(cols, TN);
   // A persistent CTA fills its SM (216 KB of shared memory).  A few SMs are left free so that the small kernels
   // of the factor chain, which run beside this pass on another stream, and those of other operands' chains do
@@ -345,7 +360,14 @@ metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const
   constexpr int reserve = 16;
   const int usable = ctx->sm_count > 2 * reserve ? ctx->sm_count - reserve : ctx->sm_count;
   const int grid = (int)(tiles < usable ? tiles : usable);
-  residual_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(mx, ma, mb, g); METIS_COUNT_LAUNCH();
+  if (sr) {
+    if (fast) residual_tc_kernel<true, true><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(mx, ma, mb, g);
+    else residual_tc_kernel<true, false><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(mx, ma, mb, g);
+  } else {
+    if (fast) residual_tc_kernel<false, true><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(mx, ma, mb, g);
+    else residual_tc_kernel<false, false><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(mx, ma, mb, g);
+  }
+  METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }
