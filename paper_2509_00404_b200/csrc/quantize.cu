@@ -47,7 +47,7 @@ __global__ void amax_kernel(const void* __restrict__ x, int dtype, int64_t rows,
 //          the stochastic-rounding draws go to shared memory for pass 2
 //  pass 2  blocks along the rows: a thread reads 16 values down a column from shared memory, encodes them and
 //          stages the bytes; the transposed codes and both scale tiles are then written out coalesced
-template <typename T>   // T = __nv_bfloat16 or float: element type of the shared tile (= input type)
+template <typename T, bool SR>   // T = __nv_bfloat16 or float: element type of the shared tile (= input type)
 __global__ void __launch_bounds__(metis_qt::THREADS, 3)
 quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, const float* __restrict__ tscale_src,
                 int tscale_is_amax, float* ts_out0, float* ts_out1) {
@@ -57,7 +57,8 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
   T* tile = reinterpret_cast<T*>(smem);                                        // [TILE][TP]
   Stage* stage = reinterpret_cast<Stage*>(smem + ((sizeof(T) * TILE * TP + 15) & ~(size_t)15));
   uint8_t* sfc = reinterpret_cast<uint8_t*>(stage + 1);                        // [TILE][8] scales of the column blocks
-  uint16_t* rnd = reinterpret_cast<uint16_t*>(sfc + TILE * 8);                 // [TILE][TILE] draws (SR only)
+  float* r_tab = reinterpret_cast<float*>(sfc + TILE * 8);                     // multiplier per scale byte
+  uint16_t* rnd = reinterpret_cast<uint16_t*>(r_tab + R_TABLE);                // [TILE][TILE] draws (SR only)
 
   const int tid = threadIdx.x;
   const int64_t row0 = (int64_t)blockIdx.y * TILE, col0 = (int64_t)blockIdx.x * TILE;
@@ -67,7 +68,8 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
     if (ts_out0 != nullptr && ts_out0 != tscale_src) *ts_out0 = s_T;
     if (ts_out1 != nullptr && ts_out1 != tscale_src) *ts_out1 = s_T;
   }
-  const bool sr = p.rounding == METIS_ROUND_SR;
+  constexpr bool sr = SR;
+  fill_r_table(r_tab, s_T, tid, THREADS);
   const bool want_c = p.c_codes != nullptr, want_r = p.r_codes != nullptr;
   const int vrows = (int)min((int64_t)TILE, p.rows - row0), vcols = (int)min((int64_t)TILE, p.cols - col0);
   const bool fast_draws = p.e_stride_c == 1 && (p.e_stride_r & 7) == 0;
@@ -86,6 +88,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
       }
     }
   }
+  __syncthreads();                                         // multiplier table complete (the tile loads are in flight)
 #pragma unroll
   for (int it = 0; it < 4; ++it) {
     const int b = tid & 7, r = (tid >> 3) + 32 * it;
@@ -141,7 +144,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
     }
     if (want_c) {
       uint32_t packed[2];
-      const uint32_t byte = encode_block(v, u, sr, s_T, six_s_T, packed);
+      const uint32_t byte = encode_block_tab(v, u, sr, six_s_T, r_tab, packed);
       if (in) *reinterpret_cast<uint2*>(p.c_codes + gr * (p.cols / 2) + gc / 2) = make_uint2(packed[0], packed[1]);
       sfc[r * 8 + b] = in ? (uint8_t)byte : (uint8_t)0;
     }
@@ -170,10 +173,10 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
           }
         }
         uint32_t packed[2];
-        uint32_t byte = encode_block(v0, u0, sr, s_T, six_s_T, packed);
+        uint32_t byte = encode_block_tab(v0, u0, sr, six_s_T, r_tab, packed);
         *reinterpret_cast<uint2*>(&stage->codes[c][b * 8]) = make_uint2(packed[0], packed[1]);
         stage->sf[c][b] = (uint8_t)byte;
-        byte = encode_block(v1, u1, sr, s_T, six_s_T, packed);
+        byte = encode_block_tab(v1, u1, sr, six_s_T, r_tab, packed);
         *reinterpret_cast<uint2*>(&stage->codes[c + 1][b * 8]) = make_uint2(packed[0], packed[1]);
         stage->sf[c + 1][b] = (uint8_t)byte;
       }
@@ -190,7 +193,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
         for (int i = 0; i < 16; ++i) u[i] = rnd[(b * 16 + i) * TILE + c];
       }
       uint32_t packed[2];
-      const uint32_t byte = encode_block(v, u, sr, s_T, six_s_T, packed);
+      const uint32_t byte = encode_block_tab(v, u, sr, six_s_T, r_tab, packed);
       *reinterpret_cast<uint2*>(&stage->codes[c][b * 8]) = make_uint2(packed[0], packed[1]);
       stage->sf[c][b] = (uint8_t)byte;
     }
@@ -226,7 +229,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
 template <typename T>
 constexpr size_t quantize_smem(bool sr) {
   return ((sizeof(T) * metis_qt::TILE * (metis_qt::TILE + (sizeof(T) == 2 ? 2 : 1)) + 15) & ~(size_t)15) + sizeof(metis_qt::Stage) +
-         metis_qt::TILE * 8 + (sr ? sizeof(uint16_t) * metis_qt::TILE * metis_qt::TILE : 0);
+         metis_qt::TILE * 8 + sizeof(float) * metis_qt::R_TABLE + (sr ? sizeof(uint16_t) * metis_qt::TILE * metis_qt::TILE : 0);
 }
 
 }  // namespace
@@ -312,18 +315,23 @@ metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int
   const bool sr = rounding == METIS_ROUND_SR;
   static bool attr_set = false;
   if (!attr_set) {
-    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<__nv_bfloat16>(true)));
-    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<float>(true)));
+    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<__nv_bfloat16>(true)));
+    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<float>(true)));
+    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<__nv_bfloat16>(false)));
+    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<float>(false)));
     attr_set = true;
   }
   dim3 grid((unsigned)metis_ceil_div(cols, TILE), (unsigned)metis_ceil_div(rows, TILE));
   float* t0 = by_cols ? by_cols->tensor_scale : nullptr; float* t1 = by_rows ? by_rows->tensor_scale : nullptr;
-  if (dtype == METIS_BF16)
-    quantize_kernel<__nv_bfloat16><<<grid, THREADS, quantize_smem<__nv_bfloat16>(sr), s>>>(
-        reinterpret_cast<const __nv_bfloat16*>(x), ld, p, tscale_src, tscale_is_amax, t0, t1);
-  else
-    quantize_kernel<float><<<grid, THREADS, quantize_smem<float>(sr), s>>>(reinterpret_cast<const float*>(x), ld, p, tscale_src,
-                                                                          tscale_is_amax, t0, t1);
+  if (dtype == METIS_BF16) {
+    const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(x);
+    if (sr) quantize_kernel<__nv_bfloat16, true><<<grid, THREADS, quantize_smem<__nv_bfloat16>(true), s>>>(xb, ld, p, tscale_src, tscale_is_amax, t0, t1);
+    else quantize_kernel<__nv_bfloat16, false><<<grid, THREADS, quantize_smem<__nv_bfloat16>(false), s>>>(xb, ld, p, tscale_src, tscale_is_amax, t0, t1);
+  } else {
+    const float* xf = reinterpret_cast<const float*>(x);
+    if (sr) quantize_kernel<float, true><<<grid, THREADS, quantize_smem<float>(true), s>>>(xf, ld, p, tscale_src, tscale_is_amax, t0, t1);
+    else quantize_kernel<float, false><<<grid, THREADS, quantize_smem<float>(false), s>>>(xf, ld, p, tscale_src, tscale_is_amax, t0, t1);
+  }
   METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
