@@ -123,61 +123,78 @@ __device__ __forceinline__ double chol_rsqrt(double x) {
 
 __device__ __forceinline__ double fast_rsqrt_wide(double x) { return chol_rsqrt(x); }
 
-// 1/x in FP64 for x inside the FP32 range: FP32 seed and two Newton steps; anything else takes the division
+// 1/x in FP64: the hardware's 20-bit FP64 reciprocal seed and three Newton steps
 __device__ __forceinline__ double chol_rcp(double x) {
-  if (!(x > 1e-30 && x < 1e30)) return 1.0 / x;
-  double y = (double)__frcp_rn((float)x);
+  double y;
+  asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+  y = y * (2.0 - x * y);
   y = y * (2.0 - x * y);
   y = y * (2.0 - x * y);
   return y;
 }
 
-// In-place Cholesky of the n x n lower triangle of Y (row pitch P doubles) by the whole CTA (>= 256 threads).
+// In-place Cholesky of the n x n lower triangle of Y (row pitch P doubles) by the first 256 threads of the CTA.
 // Right-looking with the column scaling deferred: step j only subtracts  Y[a][j] Y[b][j] / Y[j][j]  from the
 // trailing triangle (one barrier per column, a reciprocal instead of a square root in the serial chain); the
-// columns are divided by sqrt(pivot) together at the end.  A pivot not above `tol` marks a dependent column:
-// it takes no part in the updates and ends as a zero column with inv_out[j] = 0.
+// columns are divided by sqrt(pivot) together at the end.  The matrix lives in registers for the whole
+// factorisation - thread (ty, tx) of a 16 x 16 grid keeps the elements (ty + 16u, tx + 16v) - and a step reads
+// only column j and the reciprocal of its pivot, which their owners publish through shared memory before the
+// barrier of the step before; the step itself has no data-dependent branch.  A pivot not above `tol` marks a
+// dependent column: its reciprocal is published as zero, so it takes no part in the updates, and it ends as a
+// zero column with inv_out[j] = 0.
 template <int P>
 __device__ __forceinline__ void cta_cholesky(double (*Y)[P], int n, double tol, double* inv_out, double* dmin_out, int nthr) {
-  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
-  constexpr int NT = (MAXQ + 15) / 16;                  // 16 x 16 thread grid, NT x NT elements per thread
+  constexpr int NB = (MAXQ + 15) / 16;
+  __shared__ double colbuf[2][16 * NB];
+  __shared__ double rd_s[2];
+  const int tid = threadIdx.x, ty = (tid >> 4) & 15, tx = tid & 15;
+  const bool worker = tid < 256;
+  double r[NB][NB];
+#pragma unroll
+  for (int u = 0; u < NB; ++u)
+#pragma unroll
+    for (int v = 0; v <= u; ++v) {
+      const int a = ty + 16 * u, b = tx + 16 * v;
+      r[u][v] = (worker && a < n && b <= a) ? Y[a][b] : 0.0;
+    }
+  if (worker && tx == 0) {
+#pragma unroll
+    for (int u = 0; u < NB; ++u) colbuf[0][ty + 16 * u] = r[u][0];
+  }
+  if (tid == 0) { const double d0 = r[0][0]; rd_s[0] = d0 > tol ? chol_rcp(d0) : 0.0; }
+  __syncthreads();
   for (int j = 0; j < n; ++j) {
-    const double d = Y[j][j];
-    if (d > tol && tid < 256) {
-      const double rd = chol_rcp(d);
-      // operands first, then the products, then the stores: the loads of one step do not wait for its stores.
-      // `rem` is the same for every thread, so whole 16-wide groups beyond the trailing block are skipped.
-      const int rem = n - j - 1;
-      double la[NT], lb[NT], t[NT][NT];
+    if (worker) {
+      const double* cb = colbuf[j & 1];
+      const double rd = rd_s[j & 1];                    // 0 for a dependent column: the step is a no-op
+      const int jn = j + 1;
+      double la[NB], lb[NB];
 #pragma unroll
-      for (int u = 0; u < NT; ++u) {
-        if (16 * u < rem) {
-          const int a = j + 1 + ty + 16 * u, b = j + 1 + tx + 16 * u;
-          la[u] = a < n ? Y[a][j] * rd : 0.0;
-          lb[u] = b < n ? Y[b][j] : 0.0;
-        }
-      }
+      for (int u = 0; u < NB; ++u)
+        if (16 * u < n) { la[u] = cb[ty + 16 * u] * rd; lb[u] = cb[tx + 16 * u]; }
 #pragma unroll
-      for (int u = 0; u < NT; ++u)
+      for (int u = 0; u < NB; ++u)
 #pragma unroll
-        for (int v = 0; v <= u; ++v) {
-          if (16 * u < rem) {
-            const int a = j + 1 + ty + 16 * u, b = j + 1 + tx + 16 * v;
-            t[u][v] = (a < n && b <= a) ? Y[a][b] : 0.0;
+        for (int v = 0; v <= u; ++v)
+          if (16 * u < n) {
+            const int a = ty + 16 * u, b = tx + 16 * v;
+            if (a > j && b > j && b <= a) r[u][v] -= la[u] * lb[v];
+            if (b == jn) colbuf[jn & 1][a] = r[u][v];
+            if (b == jn && a == jn) { const double dn = r[u][v]; rd_s[jn & 1] = dn > tol ? chol_rcp(dn) : 0.0; }
           }
-        }
-#pragma unroll
-      for (int u = 0; u < NT; ++u)
-#pragma unroll
-        for (int v = 0; v <= u; ++v) {
-          if (16 * u < rem) {
-            const int a = j + 1 + ty + 16 * u, b = j + 1 + tx + 16 * v;
-            if (a < n && b <= a) Y[a][b] = t[u][v] - la[u] * lb[v];
-          }
-        }
     }
     __syncthreads();
   }
+  if (worker) {
+#pragma unroll
+    for (int u = 0; u < NB; ++u)
+#pragma unroll
+      for (int v = 0; v <= u; ++v) {
+        const int a = ty + 16 * u, b = tx + 16 * v;
+        if (a < n && b <= a) Y[a][b] = r[u][v];
+      }
+  }
+  __syncthreads();
   double dj = 0.0, inv = 0.0;
   if (tid < n) {
     dj = Y[tid][tid];
