@@ -28,6 +28,7 @@ struct CoeffArgs {
   float* amax;              // running amax|x| as the bits of a non-negative float (may be NULL)
   int64_t rows;
   int kp, num_chunks, chunks_per_slice;
+  int raw;                  // 1: write all 3 * kp accumulator columns as they are, part[slices][rows][3 * kp]
   uint32_t* dev_status;
 };
 
@@ -138,8 +139,22 @@ coeff_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
       const int quarter = warp & 3;                         // TMEM lanes 32*quarter .. +31 belong to this warp
       const int64_t row = (int64_t)row0 + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      if (g.raw) {
+        float* dst = g.part + ((int64_t)blockIdx.y * g.rows + row) * NB;
+        for (int jb = 0; jb < NB; jb += 16) {
+          uint32_t r0[16];
+          tc_ld16(t_row + (uint32_t)jb, r0);
+          tc_wait_ld();
+          if (row < g.rows) {
+#pragma unroll
+            for (int e = 0; e < 16; e += 4)
+              *reinterpret_cast<float4*>(dst + jb + e) = make_float4(__uint_as_float(r0[e]), __uint_as_float(r0[e + 1]),
+                                                                     __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]));
+          }
+        }
+      }
       float* dst = g.part + ((int64_t)blockIdx.y * g.rows + row) * g.kp;
-      for (int jb = 0; jb < g.kp; jb += 16) {
+      for (int jb = 0; jb < (g.raw ? 0 : g.kp); jb += 16) {
         uint32_t r0[16], r1[16], r2[16];
         tc_ld16(t_row + (uint32_t)jb, r0);
         tc_ld16(t_row + (uint32_t)(g.kp + jb), r1);
@@ -204,13 +219,15 @@ bool metis_coeff_tc_usable(const void* x, const void* bs, int64_t cols, int kp) 
 }
 
 // part: [metis_coeff_slices(rows, cols, ..)][rows][kp] FP32; bs: [3][kp][cols] BF16 (three-term split of the basis).
+// raw = 1: the operand is a single (3 * kp) x cols BF16 matrix and the accumulator columns are written unsummed,
+// part[slice][rows][3 * kp] (the sketch Z = X Omega of a full-mode split).
 metis_status_t metis_launch_coeff_tc(metis_context* ctx, const void* x, int64_t rows, int64_t cols, const void* bs, int kp,
-                                     float* part, float* amax, cudaStream_t s) {
+                                     float* part, float* amax, int raw, cudaStream_t s) {
   CUtensorMap mx, mb;
   METIS_TRY(make_map_bf16(ctx, &mx, x, rows, cols, cols, BM));
   METIS_TRY(make_map_bf16(ctx, &mb, bs, 3 * (int64_t)kp, cols, cols, 3 * kp));
   CoeffArgs g{};
-  g.part = part; g.amax = amax; g.rows = rows; g.kp = kp;
+  g.part = part; g.amax = amax; g.rows = rows; g.kp = kp; g.raw = raw;
   g.num_chunks = (int)metis_ceil_div(cols, BK);
   const int slices = metis_coeff_slices(rows, cols, &g.chunks_per_slice);
   g.dev_status = ctx->dev_status;

@@ -954,6 +954,41 @@ sketch_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* 
   }
 }
 
+// Full-mode sketch on the tcgen05 path: Omega is written once, transposed and zero-padded to nb rows
+// (omt[j][col], BF16: its values are BF16 by construction), and Z = X Omega runs on the same kernel as the
+// coefficient pass.  One thread per Philox block of eight consecutive elements e = col * q + j.
+__global__ void __launch_bounds__(256)
+omega_rows_kernel(int64_t cols, int q, int nb, uint64_t seed, const __nv_bfloat16* __restrict__ lut, __nv_bfloat16* __restrict__ omt) {
+  metis_pdl_wait();
+  const uint64_t total = (uint64_t)cols * (uint64_t)q;
+  const uint64_t blk = (uint64_t)blockIdx.x * 256 + threadIdx.x;
+  if (blk < (total + 7) / 8) {
+    const uint4 w = metis_philox_block(blk, seed, METIS_STREAM_OMEGA);
+#pragma unroll
+    for (uint32_t h = 0; h < 8; ++h) {
+      const uint64_t e = (blk << 3) + h;
+      if (e < total) omt[(e % q) * cols + e / q] = lut[metis_u16_of(w, h)];
+    }
+  }
+  // rows q .. nb-1 are zero
+  const int64_t pad = (int64_t)(nb - q) * cols;
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < pad; i += (int64_t)gridDim.x * 256)
+    omt[(int64_t)q * cols + i] = __float2bfloat16_rn(0.0f);
+}
+
+// z[r][j] = sum over slices s of part[s][r][j], j < q (part rows are nb wide); fixed order
+__global__ void __launch_bounds__(256)
+reduce_sketch_kernel(const float* __restrict__ part, int slices, int64_t rows, int nb, int q, float* __restrict__ z) {
+  metis_pdl_wait();
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= rows * q) return;
+  const int64_t r = i / q;
+  const int j = (int)(i % q);
+  float acc = 0.0f;
+  for (int s = 0; s < slices; ++s) acc += part[((int64_t)s * rows + r) * nb + j];
+  z[i] = acc;
+}
+
 // Tensor-core projection: Mp[part][j][col] = sum over the part's sampled rows r of H[r][j] * x[idx[r], col].
 // The contraction runs over rows of the row-major x, so x tiles are staged in shared memory and read back
 // transposed with ldmatrix; H (FP32) is fed as three BF16 terms.  CTA = 128 columns x one slab of rows.
@@ -1203,10 +1238,13 @@ left_rotate_kernel(const float* __restrict__ c, int64_t rows, int n_in, int k, i
 
 // Columns per sketch CTA: a sampled sketch has few rows, so narrow chunks are what gives it enough CTAs; a full
 // sketch has one CTA per 256 rows already and wide chunks keep the partial buffer small.
+// accumulator columns of the tensor-core sketch: k + p rounded up to what the coefficient kernel is built for
+int sketch_tc_cols(int q) { return q <= 48 ? 48 : 96; }
+
 int sketch_chunk_cols(int64_t n_s) { return n_s <= 512 ? 64 : SKM_COLS; }
 
 struct SplitWs {
-  size_t amax, idx, zp, z, gram, gram1, linv, evals, evecs, mp, m, basis, coef, sign, cand_v, cand_i, evals2, evecs2, bs, bt,
+  size_t amax, idx, zp, omt, z, gram, gram1, linv, evals, evecs, mp, m, basis, coef, sign, cand_v, cand_i, evals2, evecs2, bs, bt,
       gram_c, part, a6, b6, hsp, total;
 };
 
@@ -1232,7 +1270,11 @@ SplitWs split_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s) {
   const int64_t chunks = metis_ceil_div(cols, sketch_chunk_cols(n_s));
   w.amax = take(256);
   w.idx = take(sizeof(int) * (size_t)n_s);
-  w.zp = take(sizeof(float) * (size_t)chunks * n_s * q);
+  // the full-mode tensor-core sketch writes slices x rows x nb partials into the same buffer
+  const int nb_sk = sketch_tc_cols(q);
+  const size_t zp_mma = (size_t)chunks * n_s * q, zp_tc = (size_t)metis_coeff_slices(rows, cols, nullptr) * rows * nb_sk;
+  w.zp = take(sizeof(float) * (zp_mma > zp_tc ? zp_mma : zp_tc));
+  w.omt = take(sizeof(__nv_bfloat16) * (size_t)nb_sk * cols);
   w.z = take(sizeof(float) * (size_t)n_s * q);
   w.gram = take(sizeof(double) * 64 * MAXQ * MAXQ);
   w.linv = take(sizeof(double) * (MAXQ * MAXQ + MAXQ));
@@ -1420,7 +1462,16 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   METIS_CUDA_TRY(metis_launch_pdl((sample_rows_kernel), dim3((unsigned)metis_ceil_div(n_s, 256)), dim3(256), (size_t)(0), s, idx, (int)n_s, rows, seed, full ? 1 : 0)); METIS_COUNT_LAUNCH();
   const int ccols = sketch_chunk_cols(n_s);
   const int chunks = (int)metis_ceil_div(cols, ccols);
-  {
+  __nv_bfloat16* omt = reinterpret_cast<__nv_bfloat16*>(wsb + L.omt);
+  const int nb_sk = sketch_tc_cols(q);
+  const bool sketch_tc = full && q <= 96 && metis_coeff_tc_usable(x, omt, cols, nb_sk / 3);
+  if (sketch_tc) {
+    const uint64_t blocks = ((uint64_t)cols * q + 7) / 8;
+    METIS_CUDA_TRY(metis_launch_pdl((omega_rows_kernel), dim3((unsigned)metis_ceil_div((int64_t)blocks, 256)), dim3(256), (size_t)(0), s, cols, q, nb_sk, seed, ctx->quantile_lut, omt)); METIS_COUNT_LAUNCH();
+    METIS_TRY(metis_launch_coeff_tc(ctx, x, rows, cols, omt, nb_sk / 3, zp, amax, 1, s));
+    const int slices = metis_coeff_slices(rows, cols, nullptr);
+    METIS_CUDA_TRY(metis_launch_pdl((reduce_sketch_kernel), dim3((unsigned)metis_ceil_div(rows * q, 256)), dim3(256), (size_t)(0), s, zp, slices, rows, nb_sk, q, z)); METIS_COUNT_LAUNCH();
+  } else {
     const int nt = (q + 7) / 8;
     const size_t smem = sizeof(__nv_bfloat16) * nt * 8 * SKM_PITCH;
     dim3 grid((unsigned)metis_ceil_div(n_s, SKM_ROWS), (unsigned)chunks);
@@ -1438,7 +1489,9 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     }
     METIS_COUNT_LAUNCH();
   }
-  METIS_CUDA_TRY(metis_launch_pdl((reduce_partials_kernel), dim3((unsigned)metis_ceil_div(n_s * q, 256)), dim3(256), (size_t)(0), s, zp, chunks, n_s * q, z)); METIS_COUNT_LAUNCH();
+  if (!sketch_tc) {
+    METIS_CUDA_TRY(metis_launch_pdl((reduce_partials_kernel), dim3((unsigned)metis_ceil_div(n_s * q, 256)), dim3(256), (size_t)(0), s, zp, chunks, n_s * q, z)); METIS_COUNT_LAUNCH();
+  }
   // (3) CholeskyQR2: orthonormal basis H of range(Z), in place
   for (int pass = 0; pass < 2; ++pass) {
     int64_t rpp; const int parts = gram_parts(n_s, &rpp);
@@ -1511,7 +1564,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     METIS_CUDA_TRY(metis_launch_pdl((basis_splits_kernel), dim3((unsigned)metis_ceil_div(cols, 128)), dim3(128), (size_t)(0), s, basis, cols, k, kp, bs, bt, b6p, kx6)); METIS_COUNT_LAUNCH();
     if (metis_coeff_tc_usable(x, bs, cols, kp)) {
       // tensor-core pass over x (column slices), then the slices are summed and the Gram partials formed
-      METIS_TRY(metis_launch_coeff_tc(ctx, x, rows, cols, bs, kp, part, amax, s));
+      METIS_TRY(metis_launch_coeff_tc(ctx, x, rows, cols, bs, kp, part, amax, 0, s));
       a6_ready = resid_tc;
       const int slices = metis_coeff_slices(rows, cols, nullptr);
       switch (kp) {

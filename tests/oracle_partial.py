@@ -23,6 +23,7 @@ class PartialOperand:
             lq = onv.quantize(np.ascontiguousarray(sp.left.T).astype(np.float32), onv.AXIS_COLS, rounding, seed, philox.STREAM_LEFT)
             rq = onv.quantize(np.ascontiguousarray(sp.right.T).astype(np.float32), onv.AXIS_COLS, rounding, seed, philox.STREAM_RIGHT)
             self.left_q, self.right_q = onv.dequantize(*lq).T, onv.dequantize(*rq).T
+            self.raw = {"left": lq, "right": rq}
         else:
             self.sigma = np.zeros(0)
             self.res = x32

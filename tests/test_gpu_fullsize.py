@@ -13,7 +13,7 @@ TOL = 2e-3
 
 
 def test_qproj_layer_forward_and_backward_on_sampled_rows():
-    from gpu_util import rel_fro
+    from gpu_util import rel_fro, flip_allowance
     from paper_2509_00404_b200 import binding as B
     h = B.Handle(0)
     try:
@@ -36,17 +36,18 @@ def test_qproj_layer_forward_and_backward_on_sampled_rows():
             sig = op.sigma.cpu().numpy().astype(np.float64)
             assert np.max(np.abs(sig - q.sigma) / q.sigma) < 1e-3
         rows = np.random.default_rng(0).choice(4096, 192, replace=False)
+        tol = TOL + flip_allowance([(xo, xq), (wo, wq), (do, dq)])
         xd, wd_c = xq.dense(onv.AXIS_COLS), wq.dense(onv.AXIS_COLS)
-        assert rel_fro(y.cpu().numpy()[rows], xd[rows] @ wd_c.T) < TOL
+        assert rel_fro(y.cpu().numpy()[rows], xd[rows] @ wd_c.T) < tol
         dd_c, wd_r = dq.dense(onv.AXIS_COLS), wq.dense(onv.AXIS_ROWS)
-        assert rel_fro(dx.cpu().numpy()[rows], dd_c[rows] @ wd_r) < TOL
+        assert rel_fro(dx.cpu().numpy()[rows], dd_c[rows] @ wd_r) < tol
         dd_r, xd_r = dq.dense(onv.AXIS_ROWS), xq.dense(onv.AXIS_ROWS)
-        assert rel_fro(dw.cpu().numpy()[rows], dd_r[:, rows].T @ xd_r) < TOL
+        assert rel_fro(dw.cpu().numpy()[rows], dd_r[:, rows].T @ xd_r) < tol
         # factor gradients of the weight operand (sampled rows of dL/dV, all of dL/dS and dL/dU) from the oracle's dW
         dw_o = dd_r.T @ xd_r
         du, ds, dv = olay.factor_grads(dw_o, wq)
-        assert rel_fro(d_left.cpu().numpy().T[rows], dv[rows]) < TOL
-        assert rel_fro(d_right.cpu().numpy().T, du) < TOL
-        assert rel_fro(d_sigma.cpu().numpy(), ds) < TOL
+        assert rel_fro(d_left.cpu().numpy().T[rows], dv[rows]) < tol
+        assert rel_fro(d_right.cpu().numpy().T, du) < tol
+        assert rel_fro(d_sigma.cpu().numpy(), ds) < tol
     finally:
         h.close()
