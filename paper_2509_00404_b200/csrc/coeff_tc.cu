@@ -29,6 +29,7 @@ struct CoeffArgs {
   int64_t rows;
   int kp, num_chunks, chunks_per_slice;
   int raw;                  // 1: write all 3 * kp accumulator columns as they are, part[slices][rows][3 * kp]
+  int a_mn;                 // 1: the A operand is x transposed (M runs along the columns of x, K along its rows)
   uint32_t* dev_status;
 };
 
@@ -76,7 +77,12 @@ coeff_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
       if (!mbar_wait(empty_bar(s), ph ^ 1u, g.dev_status, dead)) break;
       if (elect_one()) {
         mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES);
-        tma_load_2d(a_addr(s), &map_x, c * BK, row0, full_bar(s));
+        if (g.a_mn) {                                       // two boxes of 64 columns x 64 rows: MN-major A
+          tma_load_2d(a_addr(s), &map_x, row0, c * BK, full_bar(s));
+          tma_load_2d(a_addr(s) + A_BYTES / 2, &map_x, row0 + 64, c * BK, full_bar(s));
+        } else {
+          tma_load_2d(a_addr(s), &map_x, c * BK, row0, full_bar(s));
+        }
         tma_load_2d(b_addr(s), &map_b, c * BK, 0, full_bar(s));
       }
       __syncwarp();
@@ -84,17 +90,22 @@ coeff_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer -----------------------------
-    constexpr uint32_t idesc = make_idesc_bf16(BM, NB);
+    constexpr uint32_t idesc_k = make_idesc_bf16(BM, NB), idesc_mn = make_idesc_bf16_a_mn(BM, NB);
+    const uint32_t idesc = g.a_mn ? idesc_mn : idesc_k;
     int s = 0; uint32_t ph = 0;
     bool ok = true;
     for (int c = c_begin; c < c_end; ++c) {
       if (!mbar_wait(full_bar(s), ph, g.dev_status, dead)) { ok = false; break; }
       tc_fence_after();
       if (elect_one()) {
-        const uint64_t a_d = make_smem_desc(a_addr(s), 1024, SWIZZLE_128B), b_d = make_smem_desc(b_addr(s), 1024, SWIZZLE_128B);
+        const uint64_t b_d = make_smem_desc(b_addr(s), 1024, SWIZZLE_128B);
+        // K-major A: 16 elements = 32 bytes per step inside the 128-byte rows.  MN-major A: a step is 16 K-rows of
+        // 128 bytes (two atoms of 8 rows, 1024 bytes apart); the second 64 columns are the second box, 8 KiB on.
+        const uint64_t a_d = g.a_mn ? make_smem_desc_mn(a_addr(s), A_BYTES / 2, 1024, SWIZZLE_128B) : make_smem_desc(a_addr(s), 1024, SWIZZLE_128B);
+        const uint64_t a_step = g.a_mn ? (uint64_t)(16 * 128 / 16) : 2ull;
 #pragma unroll
-        for (int k = 0; k < BK / 16; ++k)                   // 16 BF16 elements = 32 bytes per step
-          tc_mma_bf16(tmem_base, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc, (c > c_begin || k > 0) ? 1u : 0u);
+        for (int k = 0; k < BK / 16; ++k)
+          tc_mma_bf16(tmem_base, a_d + (uint64_t)k * a_step, b_d + (uint64_t)(k * 2), idesc, (c > c_begin || k > 0) ? 1u : 0u);
         tc_commit(empty_bar(s));
       }
       __syncwarp();
@@ -221,13 +232,43 @@ bool metis_coeff_tc_usable(const void* x, const void* bs, int64_t cols, int kp) 
 // part: [metis_coeff_slices(rows, cols, ..)][rows][kp] FP32; bs: [3][kp][cols] BF16 (three-term split of the basis).
 // raw = 1: the operand is a single (3 * kp) x cols BF16 matrix and the accumulator columns are written unsummed,
 // part[slice][rows][3 * kp] (the sketch Z = X Omega of a full-mode split).
+// Projection of a full-mode split on the same kernel: part[slice][col][jp] = sum over the slice's rows r of
+// x[r][col] * H[r][j], i.e. M^T = x^T H with x as an MN-major A operand (M runs along the columns of x).
+// hsp: [3][jp][ldh] BF16 (three-term split of H, transposed, ldh >= rows rounded up to 64, zero padded).
+bool metis_project_tc_usable(const void* x, const void* hsp, int64_t cols, int jp) {
+  return metis_aligned16(x) && metis_aligned16(hsp) && cols % 8 == 0 && (jp == 16 || jp == 32 || jp == 48 || jp == 64 || jp == 80);
+}
+
+int metis_project_slices(int64_t rows, int64_t cols) { return metis_coeff_slices(cols, rows, nullptr); }
+
+metis_status_t metis_launch_project_tc(metis_context* ctx, const void* x, int64_t rows, int64_t cols, const void* hsp, int jp,
+                                       int64_t ldh, float* part, cudaStream_t s) {
+  CUtensorMap mx, mb;
+  METIS_TRY(make_map_bf16(ctx, &mx, x, rows, cols, cols, BK));
+  METIS_TRY(make_map_bf16(ctx, &mb, hsp, 3 * (int64_t)jp, ldh, ldh, 3 * jp));
+  CoeffArgs g{};
+  g.part = part; g.amax = nullptr; g.rows = cols; g.kp = jp; g.raw = 0; g.a_mn = 1;
+  g.num_chunks = (int)metis_ceil_div(rows, BK);
+  const int slices = metis_coeff_slices(cols, rows, &g.chunks_per_slice);
+  g.dev_status = ctx->dev_status;
+  dim3 grid((unsigned)metis_ceil_div(cols, BM), (unsigned)slices);
+  switch (jp) {
+    case 16: return launch<48>(mx, mb, g, grid, s);
+    case 32: return launch<96>(mx, mb, g, grid, s);
+    case 48: return launch<144>(mx, mb, g, grid, s);
+    case 64: return launch<192>(mx, mb, g, grid, s);
+    case 80: return launch<240>(mx, mb, g, grid, s);
+    default: return METIS_ERR_SHAPE;
+  }
+}
+
 metis_status_t metis_launch_coeff_tc(metis_context* ctx, const void* x, int64_t rows, int64_t cols, const void* bs, int kp,
                                      float* part, float* amax, int raw, cudaStream_t s) {
   CUtensorMap mx, mb;
   METIS_TRY(make_map_bf16(ctx, &mx, x, rows, cols, cols, BM));
   METIS_TRY(make_map_bf16(ctx, &mb, bs, 3 * (int64_t)kp, cols, cols, 3 * kp));
   CoeffArgs g{};
-  g.part = part; g.amax = amax; g.rows = rows; g.kp = kp; g.raw = raw;
+  g.part = part; g.amax = amax; g.rows = rows; g.kp = kp; g.raw = raw; g.a_mn = 0;
   g.num_chunks = (int)metis_ceil_div(cols, BK);
   const int slices = metis_coeff_slices(rows, cols, &g.chunks_per_slice);
   g.dev_status = ctx->dev_status;

@@ -976,6 +976,24 @@ omega_rows_kernel(int64_t cols, int q, int nb, uint64_t seed, const __nv_bfloat1
     omt[(int64_t)q * cols + i] = __float2bfloat16_rn(0.0f);
 }
 
+// m[j][col] = sum over slices s of part[s][col][j], j < q (the tensor-core projection writes M transposed, jp wide)
+__global__ void __launch_bounds__(256)
+reduce_proj_kernel(const float* __restrict__ part, int slices, int64_t cols, int jp, int q, float* __restrict__ m) {
+  metis_pdl_wait();
+  __shared__ float t[32][33];
+  const int64_t c0 = (int64_t)blockIdx.x * 32;
+  const int j0 = blockIdx.y * 32, tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int r = ty; r < 32; r += 8) {                     // r: column of x inside the tile, tx: sketch index
+    float acc = 0.0f;
+    if (c0 + r < cols && j0 + tx < q)
+      for (int s = 0; s < slices; ++s) acc += part[((int64_t)s * cols + c0 + r) * jp + j0 + tx];
+    t[r][tx] = acc;
+  }
+  __syncthreads();
+  for (int r = ty; r < 32; r += 8)                        // r: sketch index, tx: column
+    if (j0 + r < q && c0 + tx < cols) m[(int64_t)(j0 + r) * cols + c0 + tx] = t[tx][r];
+}
+
 // z[r][j] = sum over slices s of part[s][r][j], j < q (part rows are nb wide); fixed order
 __global__ void __launch_bounds__(256)
 reduce_sketch_kernel(const float* __restrict__ part, int slices, int64_t rows, int nb, int q, float* __restrict__ z) {
@@ -1281,7 +1299,10 @@ SplitWs split_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s) {
   w.gram1 = take(sizeof(double) * MAXQ * MAXQ);
   w.evals = take(sizeof(double) * MAXQ);
   w.evecs = take(sizeof(double) * MAXQ * MAXQ);
-  w.mp = take(sizeof(float) * (size_t)PJ_MAX_PARTS * q * cols);
+  {
+    const size_t per_col_mma = (size_t)PJ_MAX_PARTS * q, per_col_tc = (size_t)8 * ((q + 15) / 16 * 16);   // tensor-core projection: <= 8 slices x jp
+    w.mp = take(sizeof(float) * (per_col_mma > per_col_tc ? per_col_mma : per_col_tc) * cols);
+  }
   w.m = take(sizeof(float) * (size_t)q * cols);
   w.basis = take(sizeof(float) * (size_t)k * cols);
   const int kp = (k + 15) / 16 * 16;
@@ -1504,6 +1525,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   // (4) M = H^T x[S,:], eigen-decomposition of M M^T, right basis
   {
     int rpp; int parts;
+    bool project_tc = false;
     if (n_s >= 1024 && cols % 8 == 0) {
       parts = (int)metis_ceil_div(n_s, 512);
       if (parts > PJ_MAX_PARTS) parts = PJ_MAX_PARTS;
@@ -1511,6 +1533,13 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       parts = (int)metis_ceil_div(n_s, rpp);
       const int mt = (q + 15) / 16, jp = mt * 16, ldh = (int)((n_s + 63) / 64 * 64);
       METIS_CUDA_TRY(metis_launch_pdl(h_splits_kernel, dim3((unsigned)metis_ceil_div(ldh, 256), (unsigned)jp), dim3(256), (size_t)0, s, z, (int)n_s, q, jp, ldh, hsp)); METIS_COUNT_LAUNCH();
+      project_tc = full && metis_project_tc_usable(x, hsp, cols, jp);
+      if (project_tc) {
+        // every row, in order: M^T = x^T H on the tcgen05 kernel of the broadcast pass (x as an MN-major operand)
+        METIS_TRY(metis_launch_project_tc(ctx, x, rows, cols, hsp, jp, ldh, mp, s));
+        dim3 rgrid((unsigned)metis_ceil_div(cols, 32), (unsigned)metis_ceil_div(q, 32));
+        METIS_CUDA_TRY(metis_launch_pdl((reduce_proj_kernel), rgrid, dim3(256), (size_t)(0), s, mp, metis_project_slices(rows, cols), cols, jp, q, m)); METIS_COUNT_LAUNCH();
+      } else {
       dim3 grid((unsigned)metis_ceil_div(cols, PP_COLS), (unsigned)parts);
       const size_t psmem = (size_t)PP_STAGES * (PP_K * PP_XP * 2 + 3 * jp * PP_HP * 2);
 #define METIS_PP(MTV) { static bool at_ = false; if (!at_) { METIS_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<MTV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psmem)); at_ = true; } \
@@ -1524,6 +1553,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       }
 #undef METIS_PP
       METIS_COUNT_LAUNCH();
+      }
     } else {
     parts = project_parts(n_s, cols, &rpp);
     dim3 grid((unsigned)metis_ceil_div(cols, PJ_COLS), (unsigned)parts);
@@ -1540,7 +1570,9 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       default: launch_project<9>(grid, s, x, cols, idx, (int)n_s, q, z, rpp, mp); break;
     }
     }
-    METIS_CUDA_TRY(metis_launch_pdl((reduce_partials_kernel), dim3((unsigned)metis_ceil_div((int64_t)q * cols, 256)), dim3(256), (size_t)(0), s, mp, parts, (int64_t)q * cols, m)); METIS_COUNT_LAUNCH();
+    if (!project_tc) {
+      METIS_CUDA_TRY(metis_launch_pdl((reduce_partials_kernel), dim3((unsigned)metis_ceil_div((int64_t)q * cols, 256)), dim3(256), (size_t)(0), s, mp, parts, (int64_t)q * cols, m)); METIS_COUNT_LAUNCH();
+    }
   }
   {
     int64_t rpp; const int parts = gram_parts(cols, &rpp);

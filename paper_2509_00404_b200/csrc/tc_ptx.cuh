@@ -128,6 +128,12 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t sbo_
   return d;
 }
 constexpr uint32_t SWIZZLE_NONE = 0, SWIZZLE_128B = 2;
+// descriptor of an MN-major operand (the M or N index is the contiguous one in shared memory), 128-byte swizzle:
+// 64 contiguous MN elements x 8 K-rows of 128 bytes form an atom; lbo = bytes between atoms along MN,
+// sbo = bytes between atoms along K
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swizzle_mode) {
+  return make_smem_desc(saddr, sbo_bytes, swizzle_mode) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
 
 // tcgen05.ld of 16 consecutive 32-bit columns of this warp's 32 lanes
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -151,6 +157,9 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
 __host__ __device__ constexpr uint32_t make_idesc_bf16(int m, int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
+
+// the same with an MN-major A operand (bit 15)
+__host__ __device__ constexpr uint32_t make_idesc_bf16_a_mn(int m, int n) { return make_idesc_bf16(m, n) | (1u << 15); }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
