@@ -172,7 +172,8 @@ metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dty
  *                                 right basis B, then C = x B for all rows, Rayleigh-Ritz on C^T C,
  *                                 residual x - C B^T.
  * Omega (cols x (k+p)) is generated on the fly from Philox (seed, METIS_STREAM_OMEGA) through the
- * quantile table; it never exists in global memory.  The residual is quantized with the tensor
+ * quantile table (per thread block in shared memory for sampled sketches, once per call into the
+ * workspace for full ones); it is never an input or an output.  The residual is quantized with the tensor
  * scale amax(x)/2688 of the SOURCE tensor; factors with their own.  `residual_axes` selects which
  * residual orientations are produced.  `residual_dense` (optional, rows x cols FP32) receives the
  * unquantized residual the quantizer saw.  k == 0 quantizes x itself.
