@@ -76,8 +76,29 @@ __device__ __forceinline__ uint32_t e2m1x8_rne(float a0, float a1, float a2, flo
   return w;
 }
 
-// encode_block with the multiplier looked up in a table filled by fill_r_table (same bytes as encode_block)
-__device__ __forceinline__ uint32_t encode_block_tab(const float (&v)[16], const uint32_t (&u)[16], bool sr, float six_s_T,
+// Eight stochastically rounded codes in one word; thr[i] = draw_i << 16.  The same decision as metis_e2m1_sr,
+// arranged for the instruction mix of the SM (integer logic and compares issue at half the FP32 / IMAD rate):
+//   b = max(a, RU(a/2 + 1/2)) maps a < 1 onto [1/2, 1] (the E2M1 grid {0, 1/2, 1} becomes {1/2, 3/4, 1}: one
+//       mantissa bit per binade like the values from 1 up) and leaves a >= 1 alone, without a select;
+//   up = (bits(b) << 10) > thr compares the 22 mantissa bits below the grid bit with the draw, no masks;
+//   the magnitude code is (bits(b) >> 22) - 252 + up; the eight "- 252" are taken off the packed word at once;
+//   the sign nibbles are gathered with one funnel shift per element and masked once per word.
+__device__ __forceinline__ uint32_t e2m1x8_sr(const float (&y)[8], const uint32_t (&thr)[8]) {
+  uint32_t mag = 0u, sgn = 0u;
+#pragma unroll
+  for (int i = 7; i >= 0; --i) {
+    const float a = fminf(fabsf(y[i]), 6.0f);
+    const uint32_t bits = __float_as_uint(fmaxf(a, __fmaf_ru(a, 0.5f, 0.5f)));
+    const uint32_t t = (bits >> 22) + (((bits << 10) > thr[i]) ? 1u : 0u);
+    mag = mag * 16u + t;                                   // modulo 2^32: the excess of 252 per nibble is removed below
+    sgn = __funnelshift_l(__float_as_uint(y[i]), sgn, 4);  // top nibble of y (sign and three exponent bits) shifted in
+  }
+  return (mag - 252u * 0x11111111u) | (sgn & 0x88888888u);
+}
+
+// encode_block with the multiplier looked up in a table filled by fill_r_table (same bytes as encode_block).
+// thr[i] = draw_i << 16 (only read with stochastic rounding).
+__device__ __forceinline__ uint32_t encode_block_tab(const float (&v)[16], const uint32_t (&thr)[16], bool sr, float six_s_T,
                                                      const float* r_tab, uint32_t (&packed)[2]) {
   float m8[8];
 #pragma unroll
@@ -93,12 +114,12 @@ __device__ __forceinline__ uint32_t encode_block_tab(const float (&v)[16], const
     packed[1] = e2m1x8_rne(__fmul_rn(v[8], r), __fmul_rn(v[9], r), __fmul_rn(v[10], r), __fmul_rn(v[11], r),
                            __fmul_rn(v[12], r), __fmul_rn(v[13], r), __fmul_rn(v[14], r), __fmul_rn(v[15], r));
   } else {
-    packed[0] = packed[1] = 0u;
+    float y0[8], y1[8];
+    uint32_t t0[8], t1[8];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const uint32_t c = metis_e2m1_sr(__fmul_rn(v[i], r), u[i]);
-      packed[i >> 3] |= c << (4 * (i & 7));
-    }
+    for (int i = 0; i < 8; ++i) { y0[i] = __fmul_rn(v[i], r); y1[i] = __fmul_rn(v[8 + i], r); t0[i] = thr[i]; t1[i] = thr[8 + i]; }
+    packed[0] = e2m1x8_sr(y0, t0);
+    packed[1] = e2m1x8_sr(y1, t1);
   }
   return byte;
 }

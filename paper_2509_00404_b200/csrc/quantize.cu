@@ -130,16 +130,16 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
         const uint4 w0 = metis_philox_block(e >> 3, p.seed, p.stream_id), w1 = metis_philox_block((e >> 3) + 1, p.seed, p.stream_id);
         const uint32_t ww[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { u[2 * j] = ww[j] & 0xFFFFu; u[2 * j + 1] = ww[j] >> 16; }
+        for (int j = 0; j < 8; ++j) { u[2 * j] = ww[j] << 16; u[2 * j + 1] = ww[j] & 0xFFFF0000u; }   // thresholds: draw << 16
       } else {
 #pragma unroll
         for (int j = 0; j < 16; ++j)
-          u[j] = in ? metis_draw_u16((uint64_t)gr * (uint64_t)p.e_stride_r + (uint64_t)(gc + j) * (uint64_t)p.e_stride_c, p.seed, p.stream_id) : 0u;
+          u[j] = in ? metis_draw_u16((uint64_t)gr * (uint64_t)p.e_stride_r + (uint64_t)(gc + j) * (uint64_t)p.e_stride_c, p.seed, p.stream_id) << 16 : 0u;
       }
       if (want_r) {
         uint32_t* dst = reinterpret_cast<uint32_t*>(rnd + r * TILE + b * 16);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) dst[j] = u[2 * j] | (u[2 * j + 1] << 16);
+        for (int j = 0; j < 8; ++j) dst[j] = (u[2 * j] >> 16) | u[2 * j + 1];
       }
     }
     if (want_c) {
@@ -169,7 +169,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const uint32_t w = *reinterpret_cast<const uint32_t*>(rnd + (b * 16 + i) * TILE + c);
-            u0[i] = w & 0xFFFFu; u1[i] = w >> 16;
+            u0[i] = w << 16; u1[i] = w & 0xFFFF0000u;
           }
         }
         uint32_t packed[2];
@@ -190,7 +190,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
       for (int i = 0; i < 16; ++i) v[i] = reinterpret_cast<const float*>(tile)[(b * 16 + i) * TP + c];
       if (sr) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) u[i] = rnd[(b * 16 + i) * TILE + c];
+        for (int i = 0; i < 16; ++i) u[i] = (uint32_t)rnd[(b * 16 + i) * TILE + c] << 16;
       }
       uint32_t packed[2];
       const uint32_t byte = encode_block_tab(v, u, sr, six_s_T, r_tab, packed);

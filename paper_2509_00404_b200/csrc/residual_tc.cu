@@ -233,8 +233,9 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 #pragma unroll
         for (int q4 = 0; q4 < 4; ++q4) {
           const uint4 w = metis_philox_block((e0 >> 3) + q4, p.seed, p.stream_id);
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-          for (uint32_t hh = 0; hh < 8; ++hh) u[8 * q4 + hh] = metis_u16_of(w, hh);
+          for (int j = 0; j < 4; ++j) { u[8 * q4 + 2 * j] = ww[j] << 16; u[8 * q4 + 2 * j + 1] = ww[j] & 0xFFFF0000u; }   // thresholds: draw << 16
         }
       }
       if (!FAST && g.dense != nullptr && row_ok && step_ok) {
@@ -278,7 +279,7 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
           for (int i = 0; i < 16; ++i) patch[lane * 17 + i] = v[16 * hf + i];
           if (sr) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) upatch[lane * 18 + i] = (uint16_t)u[16 * hf + i];
+            for (int i = 0; i < 16; ++i) upatch[lane * 18 + i] = (uint16_t)(u[16 * hf + i] >> 16);
           }
           __syncwarp();
           const int64_t col = c0 + 16 * hf + cb;
@@ -288,7 +289,7 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             t[i] = patch[(16 * rb + i) * 17 + cb];
-            d[i] = sr ? (uint32_t)upatch[(16 * rb + i) * 18 + cb] : 0u;
+            d[i] = sr ? (uint32_t)upatch[(16 * rb + i) * 18 + cb] << 16 : 0u;
           }
           uint32_t pk[2];
           const uint32_t sb = encode_block_tab(t, d, sr, six_s_T, r_tab, pk);
@@ -357,7 +358,9 @@ metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const
   // A persistent CTA fills its SM (216 KB of shared memory).  A few SMs are left free so that the small kernels
   // of the factor chain, which run beside this pass on another stream, and those of other operands' chains do
   // not have to wait for the whole pass to end.
-  constexpr int reserve = 16;
+  // A large operand's pass is long against those chains and throughput-bound: it leaves only a few SMs (with
+  // none free the factor chain, which runs beside it, would simply be appended to it).
+  const int reserve = tiles <= 4096 ? 16 : 4;
   const int usable = ctx->sm_count > 2 * reserve ? ctx->sm_count - reserve : ctx->sm_count;
   const int grid = (int)(tiles < usable ? tiles : usable);
   if (sr) {
