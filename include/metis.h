@@ -66,7 +66,8 @@ typedef enum {
 
 /* bits of the device status word */
 #define METIS_DEV_TIMEOUT 1u     /* a bounded wait inside a kernel expired                      */
-#define METIS_DEV_NUMERIC 2u     /* Cholesky breakdown / non-positive pivot in the orthonormaliser */
+#define METIS_DEV_NUMERIC 2u     /* the small eigen-decomposition of a split produced a non-finite value */
+#define METIS_DEV_NONFINITE 4u   /* the operand of a split or of an amax-scaled quantization holds a NaN or an infinity */
 
 typedef enum { METIS_BF16 = 0, METIS_FP32 = 1 } metis_dtype_t;
 typedef enum { METIS_ROUND_RNE = 0, METIS_ROUND_SR = 1 } metis_round_t;

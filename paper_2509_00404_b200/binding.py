@@ -19,7 +19,7 @@ TSCALE_AMAX_SELF, TSCALE_GIVEN = 0, 1
 SKETCH_FULL, SKETCH_SAMPLED = 0, 1
 SF_LINEAR, SF_TILED = 0, 1
 STREAM_RESIDUAL, STREAM_LEFT, STREAM_RIGHT = 0x10, 0x11, 0x12
-DEV_TIMEOUT, DEV_NUMERIC = 1, 2
+DEV_TIMEOUT, DEV_NUMERIC, DEV_NONFINITE = 1, 2, 4
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "ALIGNMENT", 4: "WORKSPACE", 5: "ARCH", 6: "CUDA",
                 7: "NONFINITE", 8: "NUMERIC", 9: "TIMEOUT"}

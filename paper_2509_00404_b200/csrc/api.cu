@@ -168,6 +168,7 @@ metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dty
     if (!ws || ws_bytes < 256) return METIS_ERR_WORKSPACE;
     float* amax = static_cast<float*>(ws);
     METIS_TRY(metis_launch_amax(x, dtype, rows, cols, ld, amax, s));
+    METIS_TRY(metis_launch_amax_check(h, amax, s));
     ts_src = amax;
     is_amax = 1;
   } else {

@@ -140,10 +140,11 @@ coeff_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
       if (++s == STAGES) { s = 0; ph ^= 1u; }
     }
     if (g.amax != nullptr) {
-      float am = fmaxf(__uint_as_float((amax2 & 0xFFFFu) << 16), __uint_as_float(amax2 & 0xFFFF0000u));
+      // as ordered bit patterns all the way (a NaN ranks above infinity and must survive: fmaxf would drop it)
+      uint32_t am = max((amax2 & 0xFFFFu) << 16, amax2 & 0xFFFF0000u);
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
-      if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(g.amax), __float_as_uint(am));
+      for (int o = 16; o > 0; o >>= 1) am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+      if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(g.amax), am);
     }
     if (ok && c_end > c_begin && mbar_wait(tfull_bar, 0u, g.dev_status, dead)) {
       tc_fence_after();

@@ -5,7 +5,9 @@ namespace {
 
 __global__ void amax_kernel(const void* __restrict__ x, int dtype, int64_t rows, int64_t cols, int64_t ld,
                             float* __restrict__ out) {
-  float m = 0.0f;
+  // |x| as a bit pattern: non-negative floats order like their bit patterns, infinity above every number and a
+  // NaN above infinity, so a non-finite element survives the reduction (fmaxf would drop a NaN)
+  uint32_t m = 0u;
   const int64_t n8 = cols / 8;
   if (dtype == METIS_BF16 && (cols & 7) == 0 && (ld & 7) == 0) {
     const int64_t total = rows * n8;
@@ -15,28 +17,27 @@ __global__ void amax_kernel(const void* __restrict__ x, int dtype, int64_t rows,
       const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        m = fmaxf(m, fabsf(__uint_as_float(w[j] << 16)));
-        m = fmaxf(m, fabsf(__uint_as_float(w[j] & 0xFFFF0000u)));
+        m = max(m, (w[j] << 16) & 0x7FFFFFFFu);
+        m = max(m, w[j] & 0x7FFF0000u);
       }
     }
   } else {
     const int64_t total = rows * cols;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
       const int64_t r = i / cols, c = i - r * cols;
-      m = fmaxf(m, fabsf(metis_ld_as_float(x, dtype, r * ld + c)));
+      m = max(m, __float_as_uint(metis_ld_as_float(x, dtype, r * ld + c)) & 0x7FFFFFFFu);
     }
   }
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-  __shared__ float wmax[32];
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  __shared__ uint32_t wmax[32];
   if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = m;
   __syncthreads();
   if (threadIdx.x < 32) {
-    m = threadIdx.x < (blockDim.x >> 5) ? wmax[threadIdx.x] : 0.0f;
+    m = threadIdx.x < (blockDim.x >> 5) ? wmax[threadIdx.x] : 0u;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-    // non-negative floats order like their bit patterns
-    if (threadIdx.x == 0) atomicMax(reinterpret_cast<unsigned int*>(out), __float_as_uint(m));
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if (threadIdx.x == 0) atomicMax(reinterpret_cast<unsigned int*>(out), m);
   }
 }
 

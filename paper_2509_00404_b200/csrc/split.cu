@@ -28,6 +28,17 @@ __global__ void sample_rows_kernel(int* __restrict__ idx, int n_s, int64_t rows,
 }
 
 // ------------------------------------------------------------------------------------------------
+// Device-detected conditions of a split: amax|x| not finite (a NaN or an infinity in the operand: amax is kept as
+// an ordered bit pattern, so a NaN ranks above every number), a non-finite eigenvalue.  One warp.
+__global__ void split_status_kernel(const float* __restrict__ amax, const double* __restrict__ evals, int k, uint32_t* dev_status) {
+  metis_pdl_wait();
+  uint32_t bits = 0u;
+  if (threadIdx.x == 0 && !(fabsf(*amax) <= 3.0e38f)) bits |= METIS_DEV_NONFINITE;
+  for (int j = threadIdx.x; j < k; j += 32)
+    if (!(fabs(evals[j]) <= 1.0e300)) bits |= METIS_DEV_NUMERIC;
+  if (bits) atomicOr(dev_status, bits);
+}
+
 __global__ void reduce_partials_kernel(const float* __restrict__ zp, int n_chunks, int64_t n, float* __restrict__ z) {
   metis_pdl_wait();
   const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
@@ -489,6 +500,7 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
     double a = 0.0;
     for (int i = 0; i < n; ++i) a += Y[i][tid] * Y[i][tid];
     lam[tid] = a;
+    order[tid] = tid;                                   // stays a valid index if NaNs make the ranks below collide
   }
   __syncthreads();
   if (tid < n) {
@@ -665,10 +677,10 @@ coeff_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols
       r0p[8 * KP] = acc[m][n][2]; r0p[8 * KP + 1] = acc[m][n][3];
     }
   {
-    float am = fmaxf(__uint_as_float((amax2 & 0xFFFFu) << 16), __uint_as_float(amax2 & 0xFFFF0000u));
+    uint32_t am = max((amax2 & 0xFFFFu) << 16, amax2 & 0xFFFF0000u);      // ordered bit patterns: a NaN survives
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
-    if (lane == 0 && amax_out) atomicMax(reinterpret_cast<unsigned int*>(amax_out), __float_as_uint(am));
+    for (int o = 16; o > 0; o >>= 1) am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+    if (lane == 0 && amax_out) atomicMax(reinterpret_cast<unsigned int*>(amax_out), am);
   }
   __syncthreads();
   float* cfin = red + 8 * 32 * KP;                             // [32][KP] final tile
@@ -947,10 +959,10 @@ sketch_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* 
       if (r + 8 < n_s) { if (j < q) dst[(int64_t)(r + 8) * q + j] = acc[m][n][2]; if (j + 1 < q) dst[(int64_t)(r + 8) * q + j + 1] = acc[m][n][3]; }
     }
   if (amax_out) {
-    float am = fmaxf(__uint_as_float((amax2 & 0xFFFFu) << 16), __uint_as_float(amax2 & 0xFFFF0000u));
+    uint32_t am = max((amax2 & 0xFFFFu) << 16, amax2 & 0xFFFF0000u);      // ordered bit patterns: a NaN survives
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
-    if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(amax_out), __float_as_uint(am));
+    for (int o = 16; o > 0; o >>= 1) am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+    if (lane == 0) atomicMax(reinterpret_cast<unsigned int*>(amax_out), am);
   }
 }
 
@@ -1371,6 +1383,13 @@ int64_t metis_default_sample_count(int64_t rows, int32_t q) {
   return want < rows ? want : rows;
 }
 
+// flags METIS_DEV_NONFINITE when *amax (the amax of a tensor about to be quantized) is not a finite number
+metis_status_t metis_launch_amax_check(metis_context* ctx, const float* amax, cudaStream_t s) {
+  METIS_CUDA_TRY(metis_launch_pdl((split_status_kernel), dim3(1), dim3(32), (size_t)(0), s, amax, (const double*)nullptr, 0, ctx->dev_status));
+  METIS_COUNT_LAUNCH();
+  return METIS_OK;
+}
+
 size_t metis_split_ws_bytes(int64_t rows, int64_t cols, int k, int p) {
   // Every buffer grows with the sample count except the sketch partials, whose chunk width steps from 64 to 256
   // columns above 512 sampled rows: the FULL sketch (n_s = rows) and a 512-row sample bound every other case.
@@ -1412,8 +1431,10 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   rc.rows = rows; rc.k_len = cols; rr.rows = cols; rr.k_len = rows;
   if (k == 0) {
     METIS_TRY(metis_launch_amax(x, METIS_BF16, rows, cols, cols, amax, s));
-    return metis_launch_quantize(x, METIS_BF16, rows, cols, cols, rounding, seed, METIS_STREAM_RESIDUAL, cols, 1, amax,
-                                 1, want_c ? &rc : nullptr, want_r ? &rr : nullptr, s);
+    METIS_TRY(metis_launch_quantize(x, METIS_BF16, rows, cols, cols, rounding, seed, METIS_STREAM_RESIDUAL, cols, 1, amax,
+                                    1, want_c ? &rc : nullptr, want_r ? &rr : nullptr, s));
+    METIS_CUDA_TRY(metis_launch_pdl((split_status_kernel), dim3(1), dim3(32), (size_t)(0), s, amax, (const double*)nullptr, 0, h->dev_status)); METIS_COUNT_LAUNCH();
+    return METIS_OK;
   }
   if (!out->left || !out->sigma || !out->right || !out->left_q.codes || !out->right_q.codes || !out->left_q.scales ||
       !out->right_q.scales || !out->left_q.tensor_scale || !out->right_q.tensor_scale)
@@ -1640,6 +1661,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       }
       METIS_COUNT_LAUNCH();
     }
+    METIS_CUDA_TRY(metis_launch_pdl((split_status_kernel), dim3(1), dim3(32), (size_t)(0), sr, amax, evals, k, ctx->dev_status)); METIS_COUNT_LAUNCH();
   }
   cudaStream_t sf = ctx->side[0];
   if (!full) {

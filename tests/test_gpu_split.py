@@ -149,3 +149,30 @@ def test_workspace_and_shape_errors(ctx):
     assert e.value.code == 2                   # METIS_ERR_SHAPE
     with pytest.raises(B.MetisError):
         h.split(x, 6, 2)                       # k not a multiple of 4
+
+
+@pytest.mark.parametrize("bad", [float("nan"), float("inf"), -float("inf")])
+def test_non_finite_operand_is_reported_in_the_device_status(bad):
+    """A NaN or an infinity anywhere in the operand sets METIS_DEV_NONFINITE (sampled and full sketch, plain
+    quantization, the amax-scaled stand-alone quantizer); a clean operand on the same handle leaves the word alone."""
+    from paper_2509_00404_b200 import binding as B
+    x, _ = synth.llama_like(256, 512, 1.0, 77, rank=8)
+    xd = torch.from_numpy(x).to(torch.bfloat16).cuda()
+    dirty = xd.clone()
+    dirty[131, 257] = bad
+    for kind in ("sampled", "full", "plain", "quantize"):
+        h = B.Handle(0)
+        try:
+            run = {"sampled": lambda t: h.split(t, 8, 8, sketch=B.SKETCH_SAMPLED, seed=5),
+                   "full": lambda t: h.split(t, 8, 8, sketch=B.SKETCH_FULL, seed=5),
+                   "plain": lambda t: h.split(t, 0, 0, seed=5),
+                   "quantize": lambda t: h.quantize_nvfp4(t, B.BLOCKS_BOTH, B.ROUND_RNE)}[kind]
+            run(xd)
+            torch.cuda.synchronize()
+            assert h.device_status() == 0, kind
+            run(dirty)
+            torch.cuda.synchronize()
+            assert h.device_status() & B.DEV_NONFINITE, kind
+            assert not (h.device_status() & B.DEV_TIMEOUT), kind
+        finally:
+            h.close()
