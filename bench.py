@@ -188,7 +188,8 @@ def main():
 
     stamps = torch.zeros(8, dtype=torch.int64, device="cuda")
 
-    def step(bufs, i, stamp=False):
+    def step(bufs, i, stamp=False, outs=None):
+        y_, dx_, dw_ = outs if outs is not None else (y, dx, dw)
         main = torch.cuda.current_stream()
         if stamp:
             h_x.timestamp(stamps[0:1], main)
@@ -212,14 +213,14 @@ def main():
         if stamp:
             h_x.timestamp(stamps[1:2], main)
         main.wait_event(ev_w)
-        h_x.linear_fwd(xo, wo, out=y)
+        h_x.linear_fwd(xo, wo, out=y_)
         if stamp:
             h_x.timestamp(stamps[4:5], main)
         main.wait_event(ev_d)
-        h_x.linear_bwd(do, xo, wo, out=(dx, dw))
+        h_x.linear_bwd(do, xo, wo, out=(dx_, dw_))
         if stamp:
             h_x.timestamp(stamps[5:6], main)
-        parallel.allreduce_weight_grad_(dw)          # token-sharded ranks: the one exchange of the path
+        parallel.allreduce_weight_grad_(dw_)         # token-sharded ranks: the one exchange of the path
 
     def barrier():
         if world > 1:
@@ -239,7 +240,9 @@ def main():
     # One step is ~100 short kernels on three streams: replaying it as a CUDA graph (one per input set; the
     # seeds are baked in, all work is re-executed) takes the host's launch cost off the critical path.
     use_graph = world == 1 and not args.no_graph
-    stage = {key: torch.empty_like(v) for key, v in dev_sets[0].items()}
+    # end-to-end run: two staging sets (inputs and outputs), so that the copies of neighbouring steps overlap the compute
+    stages = [{key: torch.empty_like(v) for key, v in dev_sets[0].items()} for _ in range(2)]
+    out_sets = [(y, dx, dw), tuple(torch.empty_like(t) for t in (y, dx, dw))]
     graphs, graph_e2e = [], None
     if use_graph:
         try:
@@ -248,9 +251,12 @@ def main():
                 with torch.cuda.graph(g_):
                     step(dev_sets[s_i], s_i)
                 graphs.append(g_)
-            graph_e2e = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph_e2e):
-                step(stage, 0)
+            graph_e2e = []
+            for b_ in range(2):
+                g_ = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_):
+                    step(stages[b_], 0, outs=out_sets[b_])
+                graph_e2e.append(g_)
             # the replay must reproduce the host-launched step bit for bit (all kernels are deterministic)
             step(dev_sets[0], 0)
             barrier()
@@ -289,26 +295,44 @@ def main():
     y_h, dx_h, dw_h = (torch.empty((l, n), dtype=bf).pin_memory(), torch.empty((l, m), dtype=bf).pin_memory(),
                        torch.empty((n, m), dtype=bf).pin_memory())
 
-    def e2e_step(i):
-        hs = host_sets[i % N_SETS]
-        for key in ("x", "w", "dy"):
-            stage[key].copy_(hs[key], non_blocking=True)
-        if use_graph:
-            graph_e2e.replay()
-        else:
-            step(stage, i)
-        y_h.copy_(y, non_blocking=True)
-        dx_h.copy_(dx, non_blocking=True)
-        dw_h.copy_(dw, non_blocking=True)
+    # Step i uses staging set i % 2: its inputs go up on one copy stream while step i - 1 computes, its results come
+    # down on another while step i + 1 computes (PCIe is full duplex).  Every step still copies all of its inputs
+    # from pinned host memory and all of its results back.
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in, ev_comp, ev_out = ([torch.cuda.Event() for _ in range(2)] for _ in range(3))
 
-    for i in range(2):
+    def e2e_step(i):
+        b_ = i & 1
+        hs = host_sets[i % N_SETS]
+        comp = torch.cuda.current_stream()
+        s_in.wait_event(ev_comp[b_])                   # the compute of step i - 2 has read this staging set
+        with torch.cuda.stream(s_in):
+            for key in ("x", "w", "dy"):
+                stages[b_][key].copy_(hs[key], non_blocking=True)
+            ev_in[b_].record(s_in)
+        comp.wait_event(ev_in[b_])
+        comp.wait_event(ev_out[b_])                    # the results of step i - 2 have left this output set
+        if use_graph:
+            graph_e2e[b_].replay()
+        else:
+            step(stages[b_], i, outs=out_sets[b_])
+        ev_comp[b_].record(comp)
+        s_out.wait_event(ev_comp[b_])
+        with torch.cuda.stream(s_out):
+            for host_t, dev_t in zip((y_h, dx_h, dw_h), out_sets[b_]):
+                host_t.copy_(dev_t, non_blocking=True)
+            ev_out[b_].record(s_out)
+
+    for i in range(4):
         e2e_step(i)
     barrier()
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n_e2e = max(3, min(args.steps, 10))
+    n_e2e = max(4, min(args.steps, 10))
     e2.record()
     for i in range(n_e2e):
         e2e_step(i)
+    for b_ in range(2):
+        torch.cuda.current_stream().wait_event(ev_out[b_])
     e3.record()
     barrier()
     ms_e2e = e2.elapsed_time(e3) / n_e2e
@@ -394,7 +418,8 @@ def main():
                    "l2": "inputs rotate over %d sets (%d MB > 126 MB L2)" % (N_SETS, N_SETS * 3 * l * m * 2 // 2 ** 20),
                    "parallelism": "dp%d (token-sharded, dW all-reduce)" % world if world > 1 else "single GPU"},
         "e2e": {"value": world * flops_step / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s",
-                "h2d_bytes_per_step": 3 * l * m * 2, "d2h_bytes_per_step": 3 * l * m * 2, "ms_per_step": ms_e2e},
+                "h2d_bytes_per_step": 3 * l * m * 2, "d2h_bytes_per_step": 3 * l * m * 2, "ms_per_step": ms_e2e,
+                "overlap": "two staging sets: the copies of step i+1 / i-1 run on their own streams beside the compute of step i"},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"bound": "tensor", "kernel": "two_cta::gemm_nvfp4_2cta_kernel (4096x4096x4096 residual GEMM, bf16 out)",
