@@ -357,12 +357,29 @@ def main():
 
     # ---- split + quantize of each operand alone (algorithmic bytes: 2 B read + 2 x 0.5625 B written per element) ----
     def alone(fn, reps=10):
+        """Mean device time of fn over `reps` calls; the calls are replayed as one CUDA graph where that is possible,
+        so that a single short kernel is not timed by the host's launch rate."""
         fn(0)
         torch.cuda.synchronize()
+        graph = None
+        if use_graph:
+            try:
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph):
+                    for r_ in range(reps):
+                        fn(r_)
+                graph.replay()
+                torch.cuda.synchronize()
+            except Exception:
+                graph = None
+                torch.cuda.synchronize()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a0.record()
-        for r_ in range(reps):
-            fn(r_)
+        if graph is not None:
+            graph.replay()
+        else:
+            for r_ in range(reps):
+                fn(r_)
         a1.record()
         torch.cuda.synchronize()
         return a0.elapsed_time(a1) / reps

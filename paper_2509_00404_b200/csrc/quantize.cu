@@ -49,7 +49,7 @@ __global__ void amax_kernel(const void* __restrict__ x, int dtype, int64_t rows,
 //  pass 2  blocks along the rows: a thread reads 16 values down a column from shared memory, encodes them and
 //          stages the bytes; the transposed codes and both scale tiles are then written out coalesced
 template <typename T, bool SR>   // T = __nv_bfloat16 or float: element type of the shared tile (= input type)
-__global__ void __launch_bounds__(metis_qt::THREADS, 3)
+__global__ void __launch_bounds__(metis_qt::THREADS, SR ? 3 : 4)
 quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, const float* __restrict__ tscale_src,
                 int tscale_is_amax, float* ts_out0, float* ts_out1) {
   using namespace metis_qt;
