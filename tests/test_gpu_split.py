@@ -76,6 +76,17 @@ def test_full_mode_tall_operand_uses_the_row_split_tensor_core_path(ctx):
     _check_against_oracle(B, h, x, 8, 8, B.SKETCH_FULL, seed=31)
 
 
+@pytest.mark.parametrize("shape_kp", [((1088, 448), 8, 8), ((2112, 192), 24, 8), ((1024, 1088), 40, 8)])
+def test_full_mode_ragged_shapes_on_the_tensor_core_sketch_and_projection(ctx, shape_kp):
+    """Full sketches of operands whose rows are not a multiple of 128 and whose columns are not a multiple of 128:
+    clipped TMA boxes in both roles of x (K-major for the sketch, MN-major for the projection), every width of the
+    projection's accumulator (k + p = 16, 32, 48), rows split over several slices."""
+    B, h = ctx
+    (rows, cols), k, p = shape_kp
+    x, _ = synth.llama_like(rows, cols, 0.5, 47, rank=max(k, 8))
+    _check_against_oracle(B, h, x, k, p, B.SKETCH_FULL, seed=33)
+
+
 def test_planted_noise_free_spectrum_is_recovered(ctx):
     """Closed form: with no bulk and rank <= k+p the sketch captures the whole matrix and Lambda is the planted
     spectrum.  The library only takes bfloat16 input, whose rounding adds a full-rank perturbation of relative size
