@@ -357,7 +357,7 @@ project_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __r
 // eigenvalues are the squared column norms and eigenvectors the normalised columns.  Working on the
 // Cholesky factor needs one matrix instead of two (no separate eigenvector accumulation), one barrier per
 // round, and converges in few sweeps.  Each round pairs the columns into n/2 disjoint couples (round-robin
-// tournament); a couple is handled by 8 threads that split the rows, reduce the three inner products with
+// tournament); a couple is handled by LANES threads that split the rows, reduce the inner product with
 // shuffles and rotate their rows in registers.
 // Input: Gram matrix (ld x ld, leading n x n block used).  Output: eigenvalues descending, eigenvectors as
 // columns of evecs[n][n].
@@ -376,8 +376,8 @@ __device__ __forceinline__ double fast_rsqrt(double x) {
   return y;
 }
 
-template <int R>                                        // rows per lane: ceil(n / 8)
-__global__ void __launch_bounds__(R > 8 ? 288 : 256)    // eight lanes per couple: n = 72 needs 36 x 8 threads
+template <int R, int LANES>                             // lanes per couple (8 or 16), rows per lane: ceil(n / LANES)
+__global__ void __launch_bounds__(LANES == 8 ? (R > 8 ? 288 : 256) : (128 * R > 256 ? 128 * R : 256))
 jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, double* __restrict__ evals,
                   double* __restrict__ evecs) {
   metis_pdl_wait();
@@ -388,8 +388,8 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
   __shared__ int order[MAXQ];
   __shared__ int rotated[2];
   __shared__ uint8_t pairs[MAXQ][MAXQ / 2][2];          // [round][couple] -> (p, q)
-  constexpr int NTHR = R > 8 ? 288 : 256;
-  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  constexpr int NTHR = LANES == 8 ? (R > 8 ? 288 : 256) : (128 * R > 256 ? 128 * R : 256);
+  const int tid = threadIdx.x;
   const int np = n + (n & 1), half = np / 2;
   for (int o = tid; o < np * np; o += NTHR) {
     const int i = o / np, j = o % np;
@@ -426,7 +426,7 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
   // inner product per couple.  A sweep whose largest cos^2 between paired columns was below exit_cos2 is the
   // last one: convergence is quadratic, so its own rotations leave the columns orthogonal to about exit_cos2.
   float* lamf = reinterpret_cast<float*>(lam);          // FP32 norms during the sweeps (lam is reused below)
-  const int m = tid >> 3, sub = tid & 7;                // couple index, row slice
+  const int m = tid / LANES, sub = tid % LANES;         // couple index, row slice
   const bool active = m < half;
   for (int sweep = 0; sweep < 16; ++sweep) {
     if (tid < np) {
@@ -447,13 +447,13 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
         double c = 0.0;
 #pragma unroll
         for (int t = 0; t < R; ++t) {
-          const int i = sub + 8 * t;
+          const int i = sub + LANES * t;
           yp[t] = (active && i < np) ? Y[i][p] : 0.0;
           yq[t] = (active && i < np) ? Y[i][q] : 0.0;
           c += yp[t] * yq[t];
         }
 #pragma unroll
-        for (int o = 4; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+        for (int o = LANES / 2; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
         const float a = lamf[p], b = lamf[q], cf = (float)c;
         const int pn = (active && step + 1 < np - 1) ? pairs[step + 1][m][0] : 0;      // next round's couple, fetched early
         const int qn = (active && step + 1 < np - 1) ? pairs[step + 1][m][1] : 0;
@@ -472,7 +472,7 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
           const double cs = cd * scale, sn = sd * scale;
 #pragma unroll
           for (int tt = 0; tt < R; ++tt) {
-            const int i = sub + 8 * tt;
+            const int i = sub + LANES * tt;
             if (i < np) {
               Y[i][p] = cs * yp[tt] - sn * yq[tt];
               Y[i][q] = sn * yp[tt] + cs * yq[tt];
@@ -1346,17 +1346,15 @@ int gram_parts(int64_t n_rows, int64_t* rows_per_part) {
 }
 
 void launch_jacobi(cudaStream_t s, const double* g, int n, int ld, float exit_cos2, double* evals, double* evecs) {
-  const int r = (n + (n & 1) + 7) / 8;
-  switch (r) {
-    case 1: (void)(metis_launch_pdl((jacobi_eig_kernel<1>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
-    case 2: (void)(metis_launch_pdl((jacobi_eig_kernel<2>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
-    case 3: (void)(metis_launch_pdl((jacobi_eig_kernel<3>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
-    case 4: (void)(metis_launch_pdl((jacobi_eig_kernel<4>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
-    case 5: (void)(metis_launch_pdl((jacobi_eig_kernel<5>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
-    case 6: (void)(metis_launch_pdl((jacobi_eig_kernel<6>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
-    case 7: (void)(metis_launch_pdl((jacobi_eig_kernel<7>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
-    case 8: (void)(metis_launch_pdl((jacobi_eig_kernel<8>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
-    default: (void)(metis_launch_pdl((jacobi_eig_kernel<9>), dim3(1), dim3(288), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+  // sixteen lanes per couple: 8 lanes (longer per-thread instruction streams) and 32 lanes (five shuffle stages, up
+  // to 1024 threads at the barrier) both measured slower
+  const int np = n + (n & 1);
+  switch ((np + 15) / 16) {
+    case 1: (void)(metis_launch_pdl((jacobi_eig_kernel<1, 16>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    case 2: (void)(metis_launch_pdl((jacobi_eig_kernel<2, 16>), dim3(1), dim3(256), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    case 3: (void)(metis_launch_pdl((jacobi_eig_kernel<3, 16>), dim3(1), dim3(384), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    case 4: (void)(metis_launch_pdl((jacobi_eig_kernel<4, 16>), dim3(1), dim3(512), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
+    default: (void)(metis_launch_pdl((jacobi_eig_kernel<5, 16>), dim3(1), dim3(640), (size_t)(JACOBI_SMEM), s, g, n, ld, exit_cos2, evals, evecs)); break;
   }
   METIS_COUNT_LAUNCH();
 }
@@ -1479,15 +1477,11 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   {
     static bool attr = false;
     if (!attr) {
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<9>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<1, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<2, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<3, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<5, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
       METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 64)));
       METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 48)));
       METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
