@@ -44,7 +44,15 @@ __global__ void reduce_partials_kernel(const float* __restrict__ zp, int n_chunk
   const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   if (i >= n) return;
   float acc = 0.0f;
-  for (int c = 0; c < n_chunks; ++c) acc += zp[(int64_t)c * n + i];     // fixed order: reproducible
+  int c = 0;
+  for (; c + 8 <= n_chunks; c += 8) {                                    // eight loads in flight; fixed order: reproducible
+    float t[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) t[u] = zp[(int64_t)(c + u) * n + i];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc += t[u];
+  }
+  for (; c < n_chunks; ++c) acc += zp[(int64_t)c * n + i];
   z[i] = acc;
 }
 
@@ -261,8 +269,9 @@ chol_kernel(const double* __restrict__ g, int q, double* __restrict__ l_out, dou
   for (int o = tid; o < q * q; o += 256) l_out[o] = L[o / q][o % q];
 }
 
-// One CholeskyQR pass, step 2: z_row <- z_row L^-T by forward substitution, one warp per row:
-// h_j = (z_j - sum_{i<j} h_i L[j][i]) / L[j][j]; lane i%32 keeps h_i, the dot product is a warp reduction.
+// One CholeskyQR pass, step 2: z_row <- z_row L^-T by forward substitution, one warp per row, column-oriented:
+// lane i%32 keeps z_i; step j broadcasts h_j = z_j / L[j][j] from its owner and every lane subtracts h_j L[i][j]
+// from its own later entries, so a step is one shuffle and one multiply-add deep (no reduction across lanes).
 __global__ void __launch_bounds__(256)
 apply_chol_kernel(float* __restrict__ z, int64_t n_rows, int q, const double* __restrict__ l, const double* __restrict__ invd,
                   const int* __restrict__ skip) {
@@ -277,24 +286,23 @@ apply_chol_kernel(float* __restrict__ z, int64_t n_rows, int q, const double* __
   const int64_t r = (int64_t)blockIdx.x * 8 + warp;
   if (r >= n_rows) return;
   static_assert(MAXQ <= 96, "three values per lane");
-  double h0 = 0.0, h1 = 0.0, h2 = 0.0;               // h_lane, h_(lane+32), h_(lane+64)
-  const double z0 = lane < q ? (double)z[r * q + lane] : 0.0;
-  const double z1 = lane + 32 < q ? (double)z[r * q + lane + 32] : 0.0;
-  const double z2 = lane + 64 < q ? (double)z[r * q + lane + 64] : 0.0;
+  double z0 = lane < q ? (double)z[r * q + lane] : 0.0;               // entries lane, lane + 32, lane + 64
+  double z1 = lane + 32 < q ? (double)z[r * q + lane + 32] : 0.0;
+  double z2 = lane + 64 < q ? (double)z[r * q + lane + 64] : 0.0;
   for (int j = 0; j < q; ++j) {
-    double part = 0.0;
-    if (lane < j) part += h0 * L[j][lane];
-    if (lane + 32 < j) part += h1 * L[j][lane + 32];
-    if (lane + 64 < j) part += h2 * L[j][lane + 64];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+    const double lj0 = lane < q ? L[lane][j] : 0.0;                    // column j of L (zero above the diagonal is not
+    const double lj1 = lane + 32 < q ? L[lane + 32][j] : 0.0;          // stored: masked by the index tests below)
+    const double lj2 = lane + 64 < q ? L[lane + 64][j] : 0.0;
     const double zj = __shfl_sync(0xFFFFFFFFu, j < 32 ? z0 : (j < 64 ? z1 : z2), j & 31);
-    const double hj = (zj - part) * inv_s[j];
-    if (lane == (j & 31)) { if (j < 32) h0 = hj; else if (j < 64) h1 = hj; else h2 = hj; }
+    const double hj = zj * inv_s[j];
+    if (lane == (j & 31)) { if (j < 32) z0 = hj; else if (j < 64) z1 = hj; else z2 = hj; }
+    if (lane > j) z0 -= hj * lj0;
+    if (lane + 32 > j) z1 -= hj * lj1;
+    if (lane + 64 > j) z2 -= hj * lj2;
   }
-  if (lane < q) z[r * q + lane] = (float)h0;
-  if (lane + 32 < q) z[r * q + lane + 32] = (float)h1;
-  if (lane + 64 < q) z[r * q + lane + 64] = (float)h2;
+  if (lane < q) z[r * q + lane] = (float)z0;
+  if (lane + 32 < q) z[r * q + lane + 32] = (float)z1;
+  if (lane + 64 < q) z[r * q + lane + 64] = (float)z2;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -322,14 +330,20 @@ project_kernel(const __nv_bfloat16* __restrict__ x, int64_t cols, const int* __r
     if (tid < PJ_ROWS) ids[tid] = (r0 + tid < r_end) ? idx[r0 + tid] : 0;
     __syncthreads();
     const int nr = min(PJ_ROWS, r_end - r0);
-    for (int rr = 0; rr < nr; ++rr) {
-      float x0 = 0.0f, x1 = 0.0f;
-      if (col + 1 < cols) {
-        const uint32_t w = *reinterpret_cast<const uint32_t*>(x + (int64_t)ids[rr] * cols + col);
-        x0 = __uint_as_float(w << 16); x1 = __uint_as_float(w & 0xFFFF0000u);
-      } else if (col < cols) {
-        x0 = __bfloat162float(x[(int64_t)ids[rr] * cols + col]);
+    // the tile's x values first, all loads in flight (inside the loop below each was an L2 round trip per row)
+    uint32_t xw[PJ_ROWS];
+#pragma unroll
+    for (int rr = 0; rr < PJ_ROWS; ++rr) {
+      xw[rr] = 0u;
+      if (rr < nr) {
+        if (col + 1 < cols) xw[rr] = *reinterpret_cast<const uint32_t*>(x + (int64_t)ids[rr] * cols + col);
+        else if (col < cols) xw[rr] = (uint32_t)__bfloat16_as_ushort(x[(int64_t)ids[rr] * cols + col]);
       }
+    }
+#pragma unroll
+    for (int rr = 0; rr < PJ_ROWS; ++rr) {
+      if (rr >= nr) break;
+      const float x0 = __uint_as_float(xw[rr] << 16), x1 = __uint_as_float(xw[rr] & 0xFFFF0000u);
 #pragma unroll
       for (int j4 = 0; j4 < NJ4; ++j4) {
         const float4 hv = *reinterpret_cast<const float4*>(&hs[jg][rr][j4 * 4]);
@@ -521,26 +535,35 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
 // ------------------------------------------------------------------------------------------------
 // Right basis from the small SVD: B[j][col] = sum_i Ut[i][j] M[i][col] / s_j, s_j = sqrt(eval_j); j < k.
 // Block = 64 columns x 4 groups of output vectors; a thread keeps four accumulators in flight.
+constexpr int RB_COLS = 32;
 __global__ void __launch_bounds__(256)
 right_basis_kernel(const float* __restrict__ m, int64_t cols, int q, int k, const double* __restrict__ evals,
                    const double* __restrict__ evecs, float* __restrict__ basis, float* __restrict__ sigma_out) {
   metis_pdl_wait();
-  __shared__ double ut[MAXQ][MAXQ + 1];
-  __shared__ double inv_s[MAXQ];
-  const int tid = threadIdx.x, cx = tid & 63, jg = tid >> 6;
-  for (int o = tid; o < q * q; o += 256) ut[o / q][o % q] = evecs[o];
+  // 32 columns per CTA; the CTA's slice of M is staged in shared memory first, so that all of its loads are in
+  // flight at once (read inside the accumulation loop they were one L2 round trip per term)
+  __shared__ double ut[MAXQ][64 + 1];                   // eigenvectors, the k <= 64 wanted columns
+  __shared__ double inv_s[64];
+  __shared__ float ms[MAXQ][RB_COLS];
+  const int tid = threadIdx.x, cx = tid & (RB_COLS - 1), jg = tid / RB_COLS;      // 8 groups of output vectors
+  const int64_t col0 = (int64_t)blockIdx.x * RB_COLS;
+  for (int o = tid; o < q * RB_COLS; o += 256) {
+    const int i = o / RB_COLS, c = o % RB_COLS;
+    ms[i][c] = col0 + c < cols ? m[(int64_t)i * cols + col0 + c] : 0.0f;
+  }
+  for (int o = tid; o < q * k; o += 256) ut[o / k][o % k] = evecs[(o / k) * q + o % k];
   if (tid < k) {
     const double s = sqrt(fmax(evals[tid], 0.0));
     inv_s[tid] = s > 0.0 ? 1.0 / s : 0.0;
     if (blockIdx.x == 0 && sigma_out != nullptr) sigma_out[tid] = (float)s;
   }
   __syncthreads();
-  const int64_t col = (int64_t)blockIdx.x * 64 + cx;
+  const int64_t col = col0 + cx;
   if (col >= cols) return;
-  for (int j0 = jg * 4; j0 < k; j0 += 16) {
+  for (int j0 = jg * 4; j0 < k; j0 += 32) {
     double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
     for (int i = 0; i < q; ++i) {
-      const double v = (double)m[(int64_t)i * cols + col];
+      const double v = (double)ms[i][cx];
       a0 += ut[i][j0] * v; a1 += ut[i][j0 + 1] * v; a2 += ut[i][j0 + 2] * v; a3 += ut[i][j0 + 3] * v;
     }
     basis[(int64_t)j0 * cols + col] = (float)(a0 * inv_s[j0]);
@@ -583,9 +606,10 @@ basis_splits_kernel(const float* __restrict__ basis, int64_t cols, int k, int kp
   const int64_t col = (int64_t)blockIdx.x * 128 + threadIdx.x;
   if (col >= cols) return;
   // b6 (optional): [cols][kx], per column the six K blocks [Bh | Bl | Bh | Bl2 | Bh | Bl] of the residual product
-  if (b6 != nullptr)
+  if (b6 != nullptr && blockIdx.y == 0)
     for (int z = 6 * kp; z < kx; z += 8) *reinterpret_cast<uint4*>(b6 + col * kx + z) = make_uint4(0u, 0u, 0u, 0u);
-  for (int j0 = 0; j0 < kp; j0 += 8) {
+  {
+    const int j0 = blockIdx.y * 8;                        // grid.y = kp / 8: one group of eight vectors per thread
     uint32_t w[3][4];
 #pragma unroll
     for (int jj = 0; jj < 8; jj += 2) {
@@ -745,7 +769,11 @@ coef_finish_kernel(const float* __restrict__ part, int slices, int64_t rows, flo
     const int64_t r = row0 + o / KP;
     float v = 0.0f;
     if (r < rows) {
-      for (int s = 0; s < slices; ++s) v += part[((int64_t)s * rows + r) * KP + (o % KP)];
+      float t[8];                                          // at most eight slices; all loads in flight, fixed order of the sum
+#pragma unroll
+      for (int s = 0; s < 8; ++s) t[s] = s < slices ? part[((int64_t)s * rows + r) * KP + (o % KP)] : 0.0f;
+#pragma unroll
+      for (int s = 0; s < 8; ++s) v += t[s];
       coef[r * KP + (o % KP)] = v;
     }
     cfin[o] = v;
@@ -997,8 +1025,13 @@ reduce_proj_kernel(const float* __restrict__ part, int slices, int64_t cols, int
   const int j0 = blockIdx.y * 32, tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   for (int r = ty; r < 32; r += 8) {                     // r: column of x inside the tile, tx: sketch index
     float acc = 0.0f;
-    if (c0 + r < cols && j0 + tx < q)
-      for (int s = 0; s < slices; ++s) acc += part[((int64_t)s * cols + c0 + r) * jp + j0 + tx];
+    if (c0 + r < cols && j0 + tx < q) {
+      float v[8];                                           // at most eight slices
+#pragma unroll
+      for (int s = 0; s < 8; ++s) v[s] = s < slices ? part[((int64_t)s * cols + c0 + r) * jp + j0 + tx] : 0.0f;
+#pragma unroll
+      for (int s = 0; s < 8; ++s) acc += v[s];
+    }
     t[r][tx] = acc;
   }
   __syncthreads();
@@ -1014,8 +1047,11 @@ reduce_sketch_kernel(const float* __restrict__ part, int slices, int64_t rows, i
   if (i >= rows * q) return;
   const int64_t r = i / q;
   const int j = (int)(i % q);
-  float acc = 0.0f;
-  for (int s = 0; s < slices; ++s) acc += part[((int64_t)s * rows + r) * nb + j];
+  float t[8], acc = 0.0f;                                 // at most eight slices
+#pragma unroll
+  for (int s = 0; s < 8; ++s) t[s] = s < slices ? part[((int64_t)s * rows + r) * nb + j] : 0.0f;
+#pragma unroll
+  for (int s = 0; s < 8; ++s) acc += t[s];
   z[i] = acc;
 }
 
@@ -1595,7 +1631,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     METIS_CUDA_TRY(metis_launch_pdl((reduce_gram_kernel), dim3((unsigned)metis_ceil_div(q * q, 32)), dim3(128), (size_t)(0), s, gram, parts, q * q, gram1, nullptr)); METIS_COUNT_LAUNCH();
     launch_jacobi(s, gram1, q, q, 1e-8f, evals, evecs);
   }
-  METIS_CUDA_TRY(metis_launch_pdl((right_basis_kernel), dim3((unsigned)metis_ceil_div(cols, 64)), dim3(256), (size_t)(0), s, m, cols, q, k, evals, evecs, basis,
+  METIS_CUDA_TRY(metis_launch_pdl((right_basis_kernel), dim3((unsigned)metis_ceil_div(cols, RB_COLS)), dim3(256), (size_t)(0), s, m, cols, q, k, evals, evecs, basis,
                                                                           full ? out->sigma : nullptr)); METIS_COUNT_LAUNCH();
   // (5) coefficients of every row in the basis, (6) fused residual + quantizer
   const int n_cand = (int)metis_ceil_div(cols, 256);
@@ -1604,11 +1640,11 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     // left = H U~_k, right = basis (sign fixed); coefficients = left * sigma
     METIS_CUDA_TRY(metis_launch_pdl((right_rotate_kernel), dim3(dim3(n_cand, (k + 7) / 8)), dim3(256), (size_t)(0), s, basis, cols, k, nullptr, out->right, cand_v, cand_i)); METIS_COUNT_LAUNCH();
     METIS_CUDA_TRY(metis_launch_pdl((sign_fix_kernel), dim3(dim3(n_cand, k)), dim3(256), (size_t)(0), s, out->right, cols, k, cand_v, cand_i, n_cand, sign, amax + 2)); METIS_COUNT_LAUNCH();
-    METIS_CUDA_TRY(metis_launch_pdl((basis_splits_kernel), dim3((unsigned)metis_ceil_div(cols, 128)), dim3(128), (size_t)(0), s, out->right, cols, k, kp, bs, bt, b6p, kx6)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((basis_splits_kernel), dim3((unsigned)metis_ceil_div(cols, 128), (unsigned)(kp / 8)), dim3(128), (size_t)(0), s, out->right, cols, k, kp, bs, bt, b6p, kx6)); METIS_COUNT_LAUNCH();
     METIS_CUDA_TRY(metis_launch_pdl((left_rotate_kernel), dim3(dim3((unsigned)metis_ceil_div(rows, 64), (unsigned)((kp + 15) / 16))), dim3(256), (size_t)(0), s, z, rows, q, k, 1, q, evecs, nullptr, sign,
                                                                             out->left, nullptr, coef, kp, out->sigma, amax + 1)); METIS_COUNT_LAUNCH();
   } else {
-    METIS_CUDA_TRY(metis_launch_pdl((basis_splits_kernel), dim3((unsigned)metis_ceil_div(cols, 128)), dim3(128), (size_t)(0), s, basis, cols, k, kp, bs, bt, b6p, kx6)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((basis_splits_kernel), dim3((unsigned)metis_ceil_div(cols, 128), (unsigned)(kp / 8)), dim3(128), (size_t)(0), s, basis, cols, k, kp, bs, bt, b6p, kx6)); METIS_COUNT_LAUNCH();
     if (metis_coeff_tc_usable(x, bs, cols, kp)) {
       // tensor-core pass over x (column slices), then the slices are summed and the Gram partials formed
       METIS_TRY(metis_launch_coeff_tc(ctx, x, rows, cols, bs, kp, part, amax, 0, s));
