@@ -182,27 +182,36 @@ __device__ __forceinline__ void cta_cholesky(double (*Y)[P], int n, double tol, 
   }
   if (tid == 0) { const double d0 = r[0][0]; rd_s[0] = d0 > tol ? chol_rcp(d0) : 0.0; }
   __syncthreads();
-  for (int j = 0; j < n; ++j) {
-    if (worker) {
-      const double* cb = colbuf[j & 1];
-      const double rd = rd_s[j & 1];                    // 0 for a dependent column: the step is a no-op
-      const int jn = j + 1;
-      double la[NB], lb[NB];
+  // Steps in phases of sixteen: during phase w (columns 16w .. 16w+15) only the register blocks u, v >= w still
+  // change, so the unrolled block loops shrink from phase to phase (an instruction stream a thread does not run
+  // costs nothing; one it runs predicated-off still costs its issue slots).
 #pragma unroll
-      for (int u = 0; u < NB; ++u)
-        if (16 * u < n) { la[u] = cb[ty + 16 * u] * rd; lb[u] = cb[tx + 16 * u]; }
+  for (int w = 0; w < NB; ++w) {
+    if (16 * w < n) {
+      const int j_end = min(n, 16 * w + 16);
+      for (int j = 16 * w; j < j_end; ++j) {
+        if (worker) {
+          const double* cb = colbuf[j & 1];
+          const double rd = rd_s[j & 1];                // 0 for a dependent column: the step is a no-op
+          const int jn = j + 1;
+          double la[NB], lb[NB];
 #pragma unroll
-      for (int u = 0; u < NB; ++u)
+          for (int u = w; u < NB; ++u)
+            if (16 * u < n) { la[u] = cb[ty + 16 * u] * rd; lb[u] = cb[tx + 16 * u]; }
 #pragma unroll
-        for (int v = 0; v <= u; ++v)
-          if (16 * u < n) {
-            const int a = ty + 16 * u, b = tx + 16 * v;
-            if (a > j && b > j && b <= a) r[u][v] -= la[u] * lb[v];
-            if (b == jn) colbuf[jn & 1][a] = r[u][v];
-            if (b == jn && a == jn) { const double dn = r[u][v]; rd_s[jn & 1] = dn > tol ? chol_rcp(dn) : 0.0; }
-          }
+          for (int u = w; u < NB; ++u)
+#pragma unroll
+            for (int v = w; v <= u; ++v)
+              if (16 * u < n) {
+                const int a = ty + 16 * u, b = tx + 16 * v;
+                if (a > j && b > j && b <= a) r[u][v] -= la[u] * lb[v];
+                if (b == jn) colbuf[jn & 1][a] = r[u][v];
+                if (b == jn && a == jn) { const double dn = r[u][v]; rd_s[jn & 1] = dn > tol ? chol_rcp(dn) : 0.0; }
+              }
+        }
+        __syncthreads();
+      }
     }
-    __syncthreads();
   }
   if (worker) {
 #pragma unroll
