@@ -76,6 +76,11 @@ gram_kernel(const float* __restrict__ v, int64_t n_rows, int n, int64_t stride_r
   const int64_t r_end = min(n_rows, r_begin + rows_per_part);
   const int nb = (n + 3) / 4, n_blocks = nb * nb;
   constexpr int BPT = (GR_NB * GR_NB + 255) / 256;      // blocks per thread at the largest n
+  // With at most 128 output blocks (n <= 44) two threads share a block, each taking half of the tile's rows; their
+  // partial sums are added once at the end (second half first into shared memory: a fixed order).
+  const bool halved = 2 * n_blocks <= 256;
+  const int half = halved ? tid / n_blocks : 0;         // 0 or 1 (threads beyond 2 * n_blocks idle)
+  const int rr_begin = halved ? half * (GR_TILE / 2) : 0, rr_end = halved ? rr_begin + GR_TILE / 2 : GR_TILE;
   double acc[BPT][4][4];
 #pragma unroll
   for (int b = 0; b < BPT; ++b)
@@ -96,11 +101,11 @@ gram_kernel(const float* __restrict__ v, int64_t n_rows, int n, int64_t stride_r
     __syncthreads();
 #pragma unroll
     for (int b = 0; b < BPT; ++b) {
-      const int o = tid + b * 256;
-      if (o < n_blocks) {
+      const int o = halved ? tid - half * n_blocks : tid + b * 256;
+      if (o < n_blocks && half < 2 && (!halved || b == 0)) {
         const int bi = o / nb, bj = o % nb;
 #pragma unroll 4
-        for (int rr = 0; rr < GR_TILE; ++rr) {
+        for (int rr = rr_begin; rr < rr_end; ++rr) {
           const double2 a01 = *reinterpret_cast<const double2*>(&tile[rr][4 * bi]), a23 = *reinterpret_cast<const double2*>(&tile[rr][4 * bi + 2]);
           const double2 b01 = *reinterpret_cast<const double2*>(&tile[rr][4 * bj]), b23 = *reinterpret_cast<const double2*>(&tile[rr][4 * bj + 2]);
           const double av[4] = {a01.x, a01.y, a23.x, a23.y}, bv[4] = {b01.x, b01.y, b23.x, b23.y};
@@ -113,10 +118,27 @@ gram_kernel(const float* __restrict__ v, int64_t n_rows, int n, int64_t stride_r
     }
     __syncthreads();
   }
+  if (halved) {
+    double* scratch = &tile[0][0];                      // the tile is free now: GR_TILE * GR_PITCH >= 16 * 128 doubles
+    const int o = tid - half * n_blocks;
+    if (half == 1 && o < n_blocks) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) scratch[o * 16 + i * 4 + j] = acc[0][i][j];
+    }
+    __syncthreads();
+    if (half == 0 && o < n_blocks) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[0][i][j] += scratch[o * 16 + i * 4 + j];
+    }
+  }
 #pragma unroll
   for (int b = 0; b < BPT; ++b) {
-    const int o = tid + b * 256;
-    if (o < n_blocks) {
+    const int o = halved ? tid : tid + b * 256;
+    if (o < n_blocks && (!halved || b == 0)) {
       const int bi = o / nb, bj = o % nb;
 #pragma unroll
       for (int i = 0; i < 4; ++i)
@@ -484,11 +506,15 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
         if (active && cf * cf > 1e-26f * (a * b)) {
           // tan(theta) = 2c / (d + sign(d) sqrt(d^2 + 4c^2)), d = b - a: the smaller root, |theta| <= pi/4.  These
           // FP32 quantities only steer convergence, so the fast reciprocal and reciprocal square root are enough.
+          // with cos(2 theta) = |d| / hyp and sin(2 theta) = +-2c / hyp:  cos^2(theta) = (1 + cos 2theta) / 2,
+          // sin(theta) = sin(2 theta) / (2 cos theta): two reciprocal square roots, no division
           const float d = b - a, c2 = 2.0f * cf;
           const float h2 = fmaf(c2, c2, d * d);
-          const float hyp = h2 * rsqrtf(h2);
-          const float tf = __fdividef(d < 0.0f ? -c2 : c2, fabsf(d) + hyp);
-          const float c32 = rsqrtf(fmaf(tf, tf, 1.0f)), s32 = tf * c32;
+          const float rh = rsqrtf(h2);
+          const float cc = fmaf(0.5f * fabsf(d), rh, 0.5f);
+          const float rs = rsqrtf(cc);
+          const float c32 = cc * rs, s32 = (d < 0.0f ? -c2 : c2) * (0.5f * rh) * rs;
+          const float tf = s32 * rs;                      // tan(theta), for the carried norms
           // (c32, s32) is a unit vector to ~1e-7; one Newton step on 1/sqrt(c^2 + s^2) in FP64 makes it one to ~1e-14
           const double cd = (double)c32, sd = (double)s32;
           const double scale = 1.5 - 0.5 * (cd * cd + sd * sd);
