@@ -183,7 +183,7 @@ def main():
     # The three operand decompositions are independent of each other, and the dY chain is independent of the
     # forward product: they run on three streams and join by events (torch streams: plumbing only).
     side_w, side_d = torch.cuda.Stream(), torch.cuda.Stream()
-    ev_start, ev_w, ev_d = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+    ev_start, ev_w, ev_d, ev_x, ev_b = (torch.cuda.Event() for _ in range(5))
     h_x, h_w, h_d = h, B.Handle(local_rank), B.Handle(local_rank)     # one workspace owner per stream
 
     stamps = torch.zeros(8, dtype=torch.int64, device="cuda")
@@ -210,17 +210,24 @@ def main():
                 h_d.timestamp(stamps[3:4], side_d)
             ev_d.record(side_d)
         h_x.split(bufs["x"], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 1, rounding=B.ROUND_RNE, out=xo)
+        ev_x.record(main)
         if stamp:
             h_x.timestamp(stamps[1:2], main)
         main.wait_event(ev_w)
         h_x.linear_fwd(xo, wo, out=y_)
         if stamp:
             h_x.timestamp(stamps[4:5], main)
-        main.wait_event(ev_d)
-        h_x.linear_bwd(do, xo, wo, out=(dx_, dw_))
-        if stamp:
-            h_x.timestamp(stamps[5:6], main)
-        parallel.allreduce_weight_grad_(dw_)         # token-sharded ranks: the one exchange of the path
+        # The backward products need dY, X and W but not the forward product: they follow the dY decomposition on its
+        # stream (in the forward's stream they would queue behind its GEMM, prologue included).
+        side_d.wait_event(ev_x)
+        side_d.wait_event(ev_w)
+        with torch.cuda.stream(side_d):
+            h_d.linear_bwd(do, xo, wo, out=(dx_, dw_), stream=side_d)
+            if stamp:
+                h_d.timestamp(stamps[5:6], side_d)
+            parallel.allreduce_weight_grad_(dw_)     # token-sharded ranks: the one exchange of the path
+            ev_b.record(side_d)
+        main.wait_event(ev_b)
 
     def barrier():
         if world > 1:
