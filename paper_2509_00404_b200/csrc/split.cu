@@ -936,12 +936,12 @@ residual_quant_kernel(const __nv_bfloat16* __restrict__ x, const float* __restri
 }
 
 // ------------------------------------------------------------------------------------------------
-// ------------------------------------------------------------------------------------------------
-// Tensor-core sketch: Zp[chunk][row][j] = sum over the chunk's 256 columns of x[idx[row], col] * Omega[col, j].
-// One CTA = 256 sampled rows x 256 columns; Omega's slice is generated once per CTA (Philox + quantile
-// table) straight into shared memory, transposed to [j][col] BF16 (its values are BF16 by construction, so
-// the products are exact and only the FP32 accumulation rounds).  Optionally also reduces amax|x| over the
-// rows it reads (FULL mode reads every row exactly once per column chunk).
+// Sketch of gathered rows (mma.sync): Zp[chunk][row][j] = sum over the chunk's columns of x[idx[row], col] * Omega[col, j].
+// One CTA = 256 sampled rows x one column chunk (`ccols` = 64 or 256 columns, see sketch_chunk_cols); Omega's slice
+// is generated once per CTA (Philox + quantile table) straight into shared memory, transposed to [j][col] BF16 (its
+// values are BF16 by construction, so the products are exact and only the FP32 accumulation rounds).  Optionally also
+// reduces amax|x| over the rows it reads.  A full sketch of an aligned operand does not come here: it runs on the
+// tcgen05 kernel of the broadcast pass (omega_rows_kernel + metis_launch_coeff_tc in its raw mode).
 constexpr int SKM_ROWS = 256, SKM_COLS = 256, SKM_PITCH = SKM_COLS + 8;
 template <int NT>                                      // sketch columns / 8, rounded up
 __global__ void __launch_bounds__(256)
