@@ -358,9 +358,11 @@ metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const
   // A persistent CTA fills its SM (216 KB of shared memory).  A few SMs are left free so that the small kernels
   // of the factor chain, which run beside this pass on another stream, and those of other operands' chains do
   // not have to wait for the whole pass to end.
-  // A large operand's pass is long against those chains and throughput-bound: it leaves only a few SMs (with
-  // none free the factor chain, which runs beside it, would simply be appended to it).
-  const int reserve = tiles <= 4096 ? 16 : 4;
+  // The smaller the operand, the more of the step is those chains: up to 1024 tiles (4096 x 4096) the pass leaves
+  // 40 SMs (measured best of 0 ... 100 on the three-operand layer step), up to 4096 tiles 16.  A large operand's
+  // pass is long against the chains and throughput-bound: it leaves only a few SMs (with none free the factor
+  // chain, which runs beside it, would simply be appended to it).
+  const int reserve = tiles <= 1024 ? 40 : (tiles <= 4096 ? 16 : 4);
   const int usable = ctx->sm_count > 2 * reserve ? ctx->sm_count - reserve : ctx->sm_count;
   const int grid = (int)(tiles < usable ? tiles : usable);
   if (sr) {
