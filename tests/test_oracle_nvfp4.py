@@ -13,11 +13,24 @@ import pytest
 from oracle import nvfp4, philox
 
 F32 = np.float32
-PAPER_SET = [0, 0.5, 1, 1.5, 2, 3, 4, 6]          # Appendix C.1: +-{0,0.5,1,1.5,2,3,4,6}
 
 
-def test_value_set_is_the_papers():
+def _golden(name):
+    """Values the paper prints (tests/golden/nvfp4_format.txt, each line with its citation)."""
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "nvfp4_format.txt")
+    for line in open(path):
+        if line.startswith(name + ":"):
+            return [float(t) for t in line.split(":", 1)[1].split()]
+    raise KeyError(name)
+
+
+PAPER_SET = _golden("e2m1_magnitudes")             # Appendix C.1: +-{0,0.5,1,1.5,2,3,4,6}
+
+
+def test_value_set_and_block_size_are_the_papers():
     assert nvfp4.E2M1_GRID.tolist() == PAPER_SET
+    assert nvfp4.BLOCK == int(_golden("block_size")[0])
 
 
 def test_all_16_codes_roundtrip():
