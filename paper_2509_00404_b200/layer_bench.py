@@ -8,7 +8,8 @@ Besides the step it times, each alone: the decomposition of every operand (algor
 of the same layer without any split (the denominator of the split overhead).  Inputs are planted-spectrum
 matrices generated on the device (rank-r spike, top singular value 100x the bulk edge, 10:1 span, Gaussian
 bulk); they are regenerated from the seed, never read from disk.  Timing: CUDA events on the launching stream,
-inputs rotate over enough sets to exceed the L2, host launches (no graph).
+inputs rotate over enough sets to exceed the L2; the step (about 100 kernels on three streams) is replayed as one
+CUDA graph per input set unless --no-graph is given, so that the host's launch rate does not bound the smaller layers.
 """
 import argparse
 import json
@@ -54,6 +55,7 @@ def main():
     ap.add_argument("--rank", type=int, default=32, help="planted rank of the synthetic inputs")
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--no-graph", action="store_true", help="time host launches instead of CUDA graph replays")
     a = ap.parse_args()
     l, m, n, k, p = a.tokens, a.d_in, a.d_out, a.k, a.p
     bf = torch.bfloat16
@@ -73,6 +75,8 @@ def main():
     def split_w(i, st=None): h_w.split(sets[i % n_sets]["w"], k, p, sketch=B.SKETCH_FULL, seed=3 * i + 2, out=wo, stream=st)
     def split_d(i, st=None): h_d.split(sets[i % n_sets]["dy"], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 3, rounding=B.ROUND_SR, out=do, stream=st)
 
+    ev_x, ev_b = torch.cuda.Event(), torch.cuda.Event()
+
     def step(i):
         main_s = torch.cuda.current_stream()
         ev0.record(main_s)
@@ -85,16 +89,35 @@ def main():
             split_d(i, side_d)
             ev_d.record(side_d)
         split_x(i)
+        ev_x.record(main_s)
         main_s.wait_event(ev_w)
         h_x.linear_fwd(xo, wo, out=y)
-        main_s.wait_event(ev_d)
-        h_x.linear_bwd(do, xo, wo, out=(dx, dw))
+        # the backward products need dY, X and W but not the forward product: they follow dY's decomposition on its stream
+        side_d.wait_event(ev_x)
+        side_d.wait_event(ev_w)
+        with torch.cuda.stream(side_d):
+            h_d.linear_bwd(do, xo, wo, out=(dx, dw), stream=side_d)
+            ev_b.record(side_d)
+        main_s.wait_event(ev_b)
 
     for i in range(a.warmup):
         step(i)
     torch.cuda.synchronize()
     status = h_x.device_status() | h_w.device_status() | h_d.device_status()
-    ms_step = timed(step, a.steps)
+    graphs = []
+    if not a.no_graph:
+        try:
+            for s_i in range(n_sets):
+                g_ = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_):
+                    step(s_i)
+                graphs.append(g_)
+            graphs[0].replay()
+            torch.cuda.synchronize()
+        except Exception:
+            graphs = []
+            torch.cuda.synchronize()
+    ms_step = timed((lambda i: graphs[i % n_sets].replay()) if graphs else step, a.steps)
     ms_sx, ms_sw, ms_sd = timed(split_x, a.steps), timed(split_w, a.steps), timed(split_d, a.steps)
 
     # plain NVFP4 layer (k = 0): the three GEMMs alone, and the plain quantizer on X (both orientations)
@@ -118,7 +141,7 @@ def main():
         "split_ms": {"x_sampled": ms_sx, "w_full": ms_sw, "dy_sampled_sr": ms_sd},
         "split_gbs": {"x_sampled": gb(l * m, ms_sx), "w_full": gb(n * m, ms_sw), "dy_sampled_sr": gb(l * n, ms_sd)},
         "quantizer_both_orientations_gbs": gb(l * m, ms_q),
-        "input_sets": n_sets, "device_status": int(status),
+        "input_sets": n_sets, "cuda_graph": bool(graphs), "device_status": int(status),
     }
     print(json.dumps(line))
 
