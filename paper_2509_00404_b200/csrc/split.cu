@@ -431,7 +431,6 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
   __shared__ double lam[MAXQ];
   __shared__ double gmax_s;
   __shared__ int order[MAXQ];
-  __shared__ int rotated[2];
   __shared__ uint8_t pairs[MAXQ][MAXQ / 2][2];          // [round][couple] -> (p, q)
   constexpr int NTHR = LANES == 8 ? (R > 8 ? 288 : 256) : (128 * R > 256 ? 128 * R : 256);
   const int tid = threadIdx.x;
@@ -445,7 +444,6 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
     jacobi_pair(o % half, o / half, np, &p, &q);
     pairs[o / half][o % half][0] = (uint8_t)p; pairs[o / half][o % half][1] = (uint8_t)q;
   }
-  if (tid == 0) { rotated[0] = 0; rotated[1] = 0; }
   __syncthreads();
   // ---- Cholesky, lower factor in place; the strict upper triangle is cleared afterwards ----
   if (tid < 32) {
@@ -473,6 +471,7 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
   float* lamf = reinterpret_cast<float*>(lam);          // FP32 norms during the sweeps (lam is reused below)
   const int m = tid / LANES, sub = tid % LANES;         // couple index, row slice
   const bool active = m < half;
+  const int mc = min(m, MAXQ / 2 - 1);                  // table column of this couple slot (idle slots beyond the table share the last)
   for (int sweep = 0; sweep < 16; ++sweep) {
     if (tid < np) {
       double a0 = 0.0, a1 = 0.0;
@@ -481,10 +480,9 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
       if (i < np) a0 += Y[i][tid] * Y[i][tid];
       lamf[tid] = (float)(a0 + a1);
     }
-    if (tid == 0) rotated[0] = 0;                       // reused as the sweep's max cos^2 (float bits)
     __syncthreads();
     int p = active ? pairs[0][m][0] : 0, q = active ? pairs[0][m][1] : 0;
-    float sweep_cos2 = 0.0f;                            // this couple slot's largest cos^2 of the sweep
+    bool above = false;                                 // some couple of this slot had cos^2 above exit_cos2 in this sweep
     for (int step = 0; step < np - 1; ++step) {
       {
         // every lane takes part in the shuffles; lanes of couples beyond n/2 carry zeros and write nothing
@@ -500,8 +498,9 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
 #pragma unroll
         for (int o = LANES / 2; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
         const float a = lamf[p], b = lamf[q], cf = (float)c;
-        const int pn = (active && step + 1 < np - 1) ? pairs[step + 1][m][0] : 0;      // next round's couple, fetched early
-        const int qn = (active && step + 1 < np - 1) ? pairs[step + 1][m][1] : 0;
+        // next round's couple, fetched early (after the last round, and for idle couple slots, the table entry is
+        // unused filler: it is inside the array and never used as an index)
+        const int pn = pairs[step + 1][mc][0], qn = pairs[step + 1][mc][1];
         // rotate only if the two columns are not yet orthogonal to working precision (cos^2 > 1e-26)
         if (active && cf * cf > 1e-26f * (a * b)) {
           // tan(theta) = 2c / (d + sign(d) sqrt(d^2 + 4c^2)), d = b - a: the smaller root, |theta| <= pi/4.  These
@@ -527,22 +526,18 @@ jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, 
               Y[i][q] = sn * yp[tt] + cs * yq[tt];
             }
           }
-          if (sub == 0) {
-            const float tc = tf * cf;                   // |y_p'|^2 = a - t c, |y_q'|^2 = b + t c for the exact rotation
-            lamf[p] = a - tc;
-            lamf[q] = b + tc;
-            sweep_cos2 = fmaxf(sweep_cos2, fminf(__fdividef(cf * cf, a * b), 1.0f));
-          }
+          // |y_p'|^2 = a - t c, |y_q'|^2 = b + t c for the exact rotation.  Every lane of the couple holds the same
+          // numbers and stores them (one value per address): no lane-dependent branch inside the round.
+          const float tc = tf * cf;
+          lamf[p] = a - tc;
+          lamf[q] = b + tc;
+          above |= cf * cf > exit_cos2 * (a * b);
         }
         p = pn; q = qn;
       }
       __syncthreads();
     }
-    if (sub == 0 && sweep_cos2 > 0.0f) atomicMax(reinterpret_cast<unsigned int*>(&rotated[0]), __float_as_uint(sweep_cos2));
-    __syncthreads();
-    const float maxcos2 = __uint_as_float((unsigned int)rotated[0]);
-    __syncthreads();
-    if (maxcos2 < exit_cos2) break;
+    if (!__syncthreads_or(above ? 1 : 0)) break;        // no couple above the threshold: this was the last sweep
   }
   // ---- eigenvalues = squared column norms, eigenvectors = normalised columns ----
   if (tid < n) {
