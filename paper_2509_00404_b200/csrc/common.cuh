@@ -201,6 +201,9 @@ int metis_coeff_slices(int64_t rows, int64_t cols, int* chunks_per_slice);
 bool metis_coeff_tc_usable(const void* x, const void* bs, int64_t cols, int kp);
 metis_status_t metis_launch_coeff_tc(metis_context* ctx, const void* x, int64_t rows, int64_t cols, const void* bs, int kp,
                                      float* part, float* amax, int raw, cudaStream_t s);
+metis_status_t metis_launch_quantize_factors(const float* left, int64_t rows, const float* right, int64_t cols, int k, int rounding,
+                                             uint64_t seed, const float* amax_left, const float* amax_right,
+                                             const metis_nvfp4_t* lq, const metis_nvfp4_t* rq, cudaStream_t s);
 metis_status_t metis_launch_amax_check(metis_context* ctx, const float* amax, cudaStream_t s);
 bool metis_project_tc_usable(const void* x, const void* hsp, int64_t cols, int jp);
 int metis_project_slices(int64_t rows, int64_t cols);

@@ -250,9 +250,8 @@ metis_status_t metis_launch_amax(const void* x, int dtype, int64_t rows, int64_t
 // Few long rows (the transposed split factors: k x len FP32, blocks along the contiguous dimension only): one
 // thread per block of 16, no tiles, no shared memory.  Threads beyond `rows` inside the last 128-row slab of the
 // tiled scale layout write zero scale bytes.
-__global__ void __launch_bounds__(256)
-quantize_rowblocks_kernel(const float* __restrict__ x, int64_t ld, metis_qt::QuantParams p, const float* __restrict__ tscale_src,
-                          int tscale_is_amax, float* ts_out) {
+__device__ __forceinline__ void rowblocks_body(const float* __restrict__ x, int64_t ld, const metis_qt::QuantParams& p,
+                                               const float* __restrict__ tscale_src, int tscale_is_amax, float* ts_out) {
   const int64_t bpr = p.cols / 16;
   const int64_t rows_pad = p.c_layout == METIS_SF_TILED ? (p.rows + 127) / 128 * 128 : p.rows;
   const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
@@ -291,6 +290,20 @@ quantize_rowblocks_kernel(const float* __restrict__ x, int64_t ld, metis_qt::Qua
   const uint32_t byte = metis_qt::encode_block(v, u, sr, s_T, __fmul_rn(6.0f, s_T), packed);
   *reinterpret_cast<uint2*>(p.c_codes + r * (p.cols / 2) + b * 8) = make_uint2(packed[0], packed[1]);
   p.c_scales[metis_sf_offset(r, b, bpr, p.c_layout)] = (uint8_t)byte;
+}
+
+__global__ void __launch_bounds__(256)
+quantize_rowblocks_kernel(const float* __restrict__ x, int64_t ld, metis_qt::QuantParams p, const float* __restrict__ tscale_src,
+                          int tscale_is_amax, float* ts_out) {
+  rowblocks_body(x, ld, p, tscale_src, tscale_is_amax, ts_out);
+}
+
+// two factor tensors in one launch (blockIdx.y selects): the left and right factors of a decomposition
+struct RowblocksJob { const float* x; int64_t ld; metis_qt::QuantParams p; const float* tscale_src; float* ts_out; };
+__global__ void __launch_bounds__(256)
+quantize_rowblocks_pair_kernel(RowblocksJob a, RowblocksJob b) {
+  const RowblocksJob& j = blockIdx.y == 0 ? a : b;
+  rowblocks_body(j.x, j.ld, j.p, j.tscale_src, 1, j.ts_out);
 }
 
 metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int rounding,
@@ -334,6 +347,28 @@ metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int
     else quantize_kernel<float, false><<<grid, THREADS, quantize_smem<float>(false), s>>>(xf, ld, p, tscale_src, tscale_is_amax, t0, t1);
   }
   METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
+
+// The two FP32 factor tensors of a decomposition (k x rows and k x cols, k <= 64, blocks along the long dimension,
+// tensor scale from each tensor's own amax) in one launch.
+metis_status_t metis_launch_quantize_factors(const float* left, int64_t rows, const float* right, int64_t cols, int k, int rounding,
+                                             uint64_t seed, const float* amax_left, const float* amax_right,
+                                             const metis_nvfp4_t* lq, const metis_nvfp4_t* rq, cudaStream_t s) {
+  using namespace metis_qt;
+  if (k <= 0 || k > 64 || rows % 16 || cols % 16) return METIS_ERR_SHAPE;
+  RowblocksJob a{}, b{};
+  a.x = left; a.ld = rows; a.tscale_src = amax_left; a.ts_out = lq->tensor_scale;
+  a.p.rows = k; a.p.cols = rows; a.p.rounding = rounding; a.p.seed = seed; a.p.stream_id = METIS_STREAM_LEFT;
+  a.p.e_stride_r = rows; a.p.e_stride_c = 1; a.p.c_codes = lq->codes; a.p.c_scales = lq->scales; a.p.c_layout = lq->sf_layout;
+  b.x = right; b.ld = cols; b.tscale_src = amax_right; b.ts_out = rq->tensor_scale;
+  b.p.rows = k; b.p.cols = cols; b.p.rounding = rounding; b.p.seed = seed; b.p.stream_id = METIS_STREAM_RIGHT;
+  b.p.e_stride_r = cols; b.p.e_stride_c = 1; b.p.c_codes = rq->codes; b.p.c_scales = rq->scales; b.p.c_layout = rq->sf_layout;
+  const int64_t pad_a = a.p.c_layout == METIS_SF_TILED ? (k + 127) / 128 * 128 : k, pad_b = b.p.c_layout == METIS_SF_TILED ? (k + 127) / 128 * 128 : k;
+  const int64_t work_a = pad_a * (rows / 16), work_b = pad_b * (cols / 16);
+  const unsigned gx = (unsigned)metis_ceil_div(work_a > work_b ? work_a : work_b, 256);
+  quantize_rowblocks_pair_kernel<<<dim3(gx, 2), 256, 0, s>>>(a, b); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }

@@ -1737,9 +1737,6 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   // (8) quantize the factors (stored transposed: k x rows, k x cols; blocks along the long dimension)
   metis_nvfp4_t lq = out->left_q, rq = out->right_q;
   lq.rows = k; lq.k_len = rows; rq.rows = k; rq.k_len = cols;
-  METIS_TRY(metis_launch_quantize(out->left, METIS_FP32, k, rows, rows, rounding, seed, METIS_STREAM_LEFT, rows, 1,
-                                  amax + 1, 1, &lq, nullptr, sf));
-  METIS_TRY(metis_launch_quantize(out->right, METIS_FP32, k, cols, cols, rounding, seed, METIS_STREAM_RIGHT, cols, 1,
-                                  amax + 2, 1, &rq, nullptr, sf));
+  METIS_TRY(metis_launch_quantize_factors(out->left, rows, out->right, cols, k, rounding, seed, amax + 1, amax + 2, &lq, &rq, sf));
   return metis_join(ctx, s, 0);
 }
