@@ -300,6 +300,87 @@ chol_kernel(const double* __restrict__ g, int q, double* __restrict__ l_out, dou
   for (int o = tid; o < q * q; o += 256) l_out[o] = L[o / q][o % q];
 }
 
+// One CholeskyQR pass, steps 0 and 1 in one CTA, for a sketch short enough to sit in shared memory as FP64 (the
+// row-sampled case: a few hundred rows): G = Z^T Z and its Cholesky factor without a trip through global memory.
+// The Gram phase computes the lower 4 x 4 blocks only; S threads (adjacent lanes) share a block, each taking
+// every S-th row, and add their partial sums with shuffles in a fixed order.
+constexpr int GC_THREADS = 512;
+constexpr size_t GC_MAX_SMEM = 144 * 1024;              // beside ~45 KiB of static shared memory
+__host__ __device__ inline int gram_chol_pitch(int q) { return 4 * ((q + 3) / 4) + 2; }
+__host__ inline size_t gram_chol_smem(int64_t n_s, int q) { return (size_t)n_s * gram_chol_pitch(q) * sizeof(double); }
+__global__ void __launch_bounds__(GC_THREADS, 1)
+gram_chol_kernel(const float* __restrict__ z, int n_s, int q, double* __restrict__ l_out, double* __restrict__ invd_out,
+                 const int* __restrict__ skip, int* __restrict__ well_conditioned) {
+  metis_pdl_wait();
+  if (skip != nullptr && *skip) return;
+  extern __shared__ __align__(16) double zs[];
+  __shared__ double L[MAXQ][MAXQ + 1];
+  __shared__ double gmax_s;
+  __shared__ double dmin_s;
+  __shared__ double inv_s[MAXQ];
+  const int tid = threadIdx.x;
+  const int nb = (q + 3) / 4, zp = gram_chol_pitch(q);
+  for (int o = tid; o < n_s * zp; o += GC_THREADS) {
+    const int r = o / zp, c = o - r * zp;
+    zs[o] = c < q ? (double)z[(int64_t)r * q + c] : 0.0;
+  }
+  const int blocks = nb * (nb + 1) / 2;
+  int S = 1;
+  while (2 * S * blocks <= GC_THREADS && S < 32) S *= 2;
+  const int o = tid / S, part = tid - o * S;
+  int bi = 0;
+  while ((bi + 1) * (bi + 2) / 2 <= o) ++bi;
+  const int bj = o - bi * (bi + 1) / 2;
+  const bool active = o < blocks;
+  double acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+  __syncthreads();
+  if (active) {
+    const double* pa = zs + 4 * bi;
+    const double* pb = zs + 4 * bj;
+#pragma unroll 2
+    for (int rr = part; rr < n_s; rr += S) {
+      const double2 a01 = *reinterpret_cast<const double2*>(pa + rr * zp), a23 = *reinterpret_cast<const double2*>(pa + rr * zp + 2);
+      const double2 b01 = *reinterpret_cast<const double2*>(pb + rr * zp), b23 = *reinterpret_cast<const double2*>(pb + rr * zp + 2);
+      const double av[4] = {a01.x, a01.y, a23.x, a23.y}, bv[4] = {b01.x, b01.y, b23.x, b23.y};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] += av[i] * bv[j];
+    }
+  }
+  for (int off = S >> 1; off > 0; off >>= 1) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] += __shfl_xor_sync(0xFFFFFFFFu, acc[i][j], off);
+  }
+  if (active && part == 0) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (4 * bi + i < q && 4 * bj + j < q) L[4 * bi + i][4 * bj + j] = acc[i][j];
+  }
+  __syncthreads();
+  if (tid < 32) {
+    double gm = 0.0;
+    for (int i = tid; i < q; i += 32) gm = fmax(gm, L[i][i]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) gm = fmax(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, off));
+    if (tid == 0) gmax_s = gm;
+  }
+  __syncthreads();
+  const double tol = 1e-13 * gmax_s;
+  cta_cholesky<MAXQ + 1>(L, q, tol, inv_s, &dmin_s, GC_THREADS);
+  if (tid < q) invd_out[tid] = inv_s[tid];
+  if (tid == 0 && well_conditioned != nullptr) *well_conditioned = (dmin_s > 1e-8 * gmax_s) ? 1 : 0;
+  for (int e = tid; e < q * q; e += GC_THREADS) l_out[e] = L[e / q][e % q];
+}
+
 // One CholeskyQR pass, step 2: z_row <- z_row L^-T by forward substitution, one warp per row, column-oriented:
 // lane i%32 keeps z_i; step j broadcasts h_j = z_j / L[j][j] from its owner and every lane subtracts h_j L[i][j]
 // from its own later entries, so a step is one shuffle and one multiply-add deep (no reduction across lanes).
@@ -422,7 +503,7 @@ __device__ __forceinline__ double fast_rsqrt(double x) {
 }
 
 template <int R, int LANES>                             // lanes per couple (8 or 16), rows per lane: ceil(n / LANES)
-__global__ void __launch_bounds__(LANES == 8 ? (R > 8 ? 288 : 256) : (128 * R > 256 ? 128 * R : 256))
+__global__ void __launch_bounds__(LANES == 8 ? (R > 8 ? 288 : 256) : (128 * R > 256 ? 128 * R : 256), 1)
 jacobi_eig_kernel(const double* __restrict__ g, int n, int ld, float exit_cos2, double* __restrict__ evals,
                   double* __restrict__ evecs) {
   metis_pdl_wait();
@@ -1598,9 +1679,16 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   for (int pass = 0; pass < 2; ++pass) {
     int64_t rpp; const int parts = gram_parts(n_s, &rpp);
     const int* skip = pass == 0 ? nullptr : cond_flag;
+    if (gram_chol_smem(n_s, q) <= GC_MAX_SMEM) {
+      // a short sketch: Gram matrix and factorisation in one CTA
+      static bool at_ = false;
+      if (!at_) { METIS_CUDA_TRY(cudaFuncSetAttribute(gram_chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GC_MAX_SMEM)); at_ = true; }
+      METIS_CUDA_TRY(metis_launch_pdl((gram_chol_kernel), dim3(1), dim3(GC_THREADS), gram_chol_smem(n_s, q), s, z, (int)n_s, q, linv, invd, skip, pass == 0 ? cond_flag : nullptr)); METIS_COUNT_LAUNCH();
+    } else {
     METIS_CUDA_TRY(metis_launch_pdl((gram_kernel), dim3(parts), dim3(256), (size_t)(0), s, z, n_s, q, q, 1, rpp, gram, skip)); METIS_COUNT_LAUNCH();
     METIS_CUDA_TRY(metis_launch_pdl((reduce_gram_kernel), dim3((unsigned)metis_ceil_div(q * q, 32)), dim3(128), (size_t)(0), s, gram, parts, q * q, gram1, skip)); METIS_COUNT_LAUNCH();
     METIS_CUDA_TRY(metis_launch_pdl((chol_kernel), dim3(1), dim3(256), (size_t)(0), s, gram1, q, linv, invd, skip, pass == 0 ? cond_flag : nullptr)); METIS_COUNT_LAUNCH();
+    }
     METIS_CUDA_TRY(metis_launch_pdl((apply_chol_kernel), dim3((unsigned)metis_ceil_div(n_s, 8)), dim3(256), (size_t)(0), s, z, n_s, q, linv, invd, skip)); METIS_COUNT_LAUNCH();
   }
   // (4) M = H^T x[S,:], eigen-decomposition of M M^T, right basis
