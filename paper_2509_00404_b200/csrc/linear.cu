@@ -28,7 +28,12 @@ __device__ __forceinline__ float deq_at(const uint8_t* codes, const uint8_t* sf,
 // Finishes the two skinny operands of the rank-(ka+kb) update, in place.  Layout: Lcat [M][kb + ka],
 // Rcat [N][kb + ka].  On entry Lcat[:, :kb] holds G1 and Rcat[:, kb:] holds Wt (written there by the skinny
 // GEMMs).  On exit  Lcat[:, :kb] = (G1 + Fo_a sa P) sb,  Lcat[:, kb:] = Fo_a sa,  Rcat[:, :kb] = Fo_b.
-// One warp per row.
+// One warp per row.  Every global load of a row is issued before the first value is used (the loads are one
+// round trip instead of a chain of them), and the finished rows stay in shared memory for the BF16 pass.
+__device__ __forceinline__ float deq_of(uint32_t byte, uint32_t sf_byte, int64_t c) {
+  const uint32_t code = (c & 1) ? (byte >> 4) : (byte & 15u);
+  return metis_e2m1_value(code) * metis_e4m3_value((uint8_t)sf_byte);
+}
 __global__ void __launch_bounds__(256)
 lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
                       const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts,
@@ -39,42 +44,86 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
                       const float* res_a_ts, const float* res_b_ts) {
   __shared__ float ps[64][65];
   __shared__ float fa[8][64];
+  __shared__ float lrow[8][128];
+  __shared__ float rrow[8][128];
   metis_pdl_wait();
   metis_pdl_trigger();                                      // the large GEMM behind this kernel sets itself up meanwhile
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int kc = ka + kb;
+  const int64_t i = (int64_t)blockIdx.x * 8 + warp;
+  // ---- loads (ka, kb <= 64: two values per lane and operand) ----
+  uint32_t a_byte[2] = {0u, 0u}, a_sfb[2] = {0u, 0u}, b_byte[2] = {0u, 0u}, b_sfb[2] = {0u, 0u};
+  float sa_v[2] = {0.0f, 0.0f}, sb_v[2] = {0.0f, 0.0f}, g1[2] = {0.0f, 0.0f}, wt[2] = {0.0f, 0.0f};
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int u = lane + 32 * j;
+    if (u < ka) {
+      sa_v[j] = sa[u];
+      if (i < M) {
+        a_byte[j] = foa_codes[(int64_t)u * (M / 2) + i / 2];
+        a_sfb[j] = foa_sf[metis_sf_offset(u, i / 16, M / 16, foa_layout)];
+      }
+      if (i < N) wt[j] = rcat[i * kc + kb + u];
+    }
+    if (u < kb) {
+      sb_v[j] = sb[u];
+      if (i < M) g1[j] = lcat[i * kc + u];
+      if (i < N) {
+        b_byte[j] = fob_codes[(int64_t)u * (N / 2) + i / 2];
+        b_sfb[j] = fob_sf[metis_sf_offset(u, i / 16, N / 16, fob_layout)];
+      }
+    }
+  }
+  const float tsa = ka ? *foa_ts : 0.0f, tsb = kb ? *fob_ts : 0.0f;
+  const float inv_alpha = lx != nullptr ? 1.0f / ((*res_a_ts) * (*res_b_ts)) : 0.0f;
   for (int o = tid; o < ka * kb; o += 256) ps[o / kb][o % kb] = pm[o];
   __syncthreads();
-  const int64_t i = (int64_t)blockIdx.x * 8 + warp;
   if (i < M) {
-    const float tsa = ka ? *foa_ts : 0.0f;
-    for (int u = lane; u < ka; u += 32) {
-      const float v = deq_at(foa_codes, foa_sf, foa_layout, M, u, i) * tsa * sa[u];
-      fa[warp][u] = v;
-      lcat[i * kc + kb + u] = v;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int u = lane + 32 * j;
+      if (u < ka) {
+        const float v = deq_of(a_byte[j], a_sfb[j], i) * tsa * sa_v[j];
+        fa[warp][u] = v;
+        lrow[warp][kb + u] = v;
+        lcat[i * kc + kb + u] = v;
+      }
     }
     __syncwarp();
-    for (int t = lane; t < kb; t += 32) {
-      float v = lcat[i * kc + t];
-      for (int u = 0; u < ka; ++u) v = fmaf(fa[warp][u], ps[u][t], v);
-      lcat[i * kc + t] = v * sb[t];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int t = lane + 32 * j;
+      if (t < kb) {
+        float v = g1[j];
+        for (int u = 0; u < ka; ++u) v = fmaf(fa[warp][u], ps[u][t], v);
+        v *= sb_v[j];
+        lrow[warp][t] = v;
+        lcat[i * kc + t] = v;
+      }
     }
   }
   if (i < N) {
-    const float tsb = kb ? *fob_ts : 0.0f;
-    for (int t = lane; t < kb; t += 32) rcat[i * kc + t] = deq_at(fob_codes, fob_sf, fob_layout, N, t, i) * tsb;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int t = lane + 32 * j;
+      if (t < kb) {
+        const float v = deq_of(b_byte[j], b_sfb[j], i) * tsb;
+        rrow[warp][t] = v;
+        rcat[i * kc + t] = v;
+      }
+      if (t < ka) rrow[warp][kb + t] = wt[j];
+    }
   }
   if (lx == nullptr) return;
   // BF16 operands of the in-accumulator correction:  Lx = [Lh | Lh | Ll] / alpha,  Rx = [Rh | Rl | Rh]
   // (hi/lo two-term splits, three cross products), zero padded to kx columns.
   __syncwarp();
-  const float inv_alpha = 1.0f / ((*res_a_ts) * (*res_b_ts));
   for (int c = lane; c < kx; c += 32) {
     const int seg = c / kc, t = c - seg * kc;
     if (i < M) {
       float out = 0.0f;
       if (seg < 3) {
-        const float v = lcat[i * kc + t] * inv_alpha;
+        const float v = lrow[warp][t] * inv_alpha;
         const float h = __bfloat162float(__float2bfloat16_rn(v));
         out = seg == 2 ? v - h : h;
       }
@@ -83,7 +132,7 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
     if (i < N) {
       float out = 0.0f;
       if (seg < 3) {
-        const float v = rcat[i * kc + t];
+        const float v = rrow[warp][t];
         const float h = __bfloat162float(__float2bfloat16_rn(v));
         out = seg == 1 ? v - h : h;
       }
