@@ -61,7 +61,7 @@ metis_status_t metis_create(metis_handle_t* out, int device) {
   free(host);
   int prio_least = 0, prio_greatest = 0;
   if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest);
-  for (int i = 0; i < 3 && e == cudaSuccess; ++i) {
+  for (int i = 0; i < METIS_N_SIDE && e == cudaSuccess; ++i) {
     // highest priority: the side streams carry the short latency-critical chains, which must not queue up
     // behind the thousands of blocks of a big pass running on the caller's stream
     e = cudaStreamCreateWithPriority(&ctx->side[i], cudaStreamNonBlocking, prio_greatest);
@@ -78,7 +78,7 @@ metis_status_t metis_create(metis_handle_t* out, int device) {
 
 metis_status_t metis_destroy(metis_handle_t h) {
   if (!h) return METIS_OK;
-  for (int i = 0; i < 3; ++i) {
+  for (int i = 0; i < METIS_N_SIDE; ++i) {
     if (h->side[i]) { cudaStreamSynchronize(h->side[i]); cudaStreamDestroy(h->side[i]); }
     if (h->ev_join[i]) cudaEventDestroy(h->ev_join[i]);
   }

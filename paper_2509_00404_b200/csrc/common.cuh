@@ -6,6 +6,7 @@
 
 #include "../../include/metis.h"
 
+constexpr int METIS_N_SIDE = 5;                        // side streams per handle (the backward pass uses all five)
 struct metis_context {
   int device;
   int sm_count;
@@ -14,8 +15,8 @@ struct metis_context {
   void* encode_tiled;            // cuTensorMapEncodeTiled entry point, resolved at create
   // Internal fork/join: independent sub-chains of one call run on these side streams and are joined back into
   // the caller's stream with events before the call's last kernels (everything stays asynchronous).
-  cudaStream_t side[3];
-  cudaEvent_t ev_fork, ev_join[3];
+  cudaStream_t side[METIS_N_SIDE];
+  cudaEvent_t ev_fork, ev_join[METIS_N_SIDE];
 };
 
 // fork: side stream i starts after everything enqueued so far on `main`

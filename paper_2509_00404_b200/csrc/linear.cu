@@ -369,23 +369,20 @@ metis_status_t make_plan(const Side& a, const Side& b, void* ws, size_t ws_bytes
 }
 
 // Everything of a product that comes before its large GEMM: the three skinny products (straight into their
-// slots of the concatenated operands) and the finishing kernel.  `side_by_side`: the skinny products run on
-// the handle's streams 0 and 1 beside `s`; otherwise one after the other on `s`.
-metis_status_t split_gemm_prologue(metis_context* ctx, const Side& a, const Side& b, const Plan& pl, bool side_by_side,
+// slots of the concatenated operands) and the finishing kernel.  The skinny products run on the handle's side
+// streams `side0` and `side0 + 1` beside `s` (the caller has made those streams wait for `s`'s past already).
+metis_status_t split_gemm_prologue(metis_context* ctx, const Side& a, const Side& b, const Plan& pl, int side0,
                                    cudaStream_t s) {
   if (pl.kc == 0) return METIS_OK;
   const int64_t M = pl.M, N = pl.N;
   const int ka = pl.ka, kb = pl.kb, kc = pl.kc;
   if (!pl.fuse) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.res, pl.y0, METIS_FP32, N, s));
-  cudaStream_t s1 = side_by_side ? ctx->side[0] : s, s2 = side_by_side ? ctx->side[1] : s;
-  if (side_by_side) METIS_TRY(metis_fork(ctx, s, 2));
+  cudaStream_t s1 = ctx->side[side0], s2 = ctx->side[side0 + 1];
   if (kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.res, b.fc, pl.lcat, METIS_FP32, kc, s));
   if (ka) METIS_TRY(metis_launch_gemm_tc(ctx, b.res, a.fc, pl.rcat + kb, METIS_FP32, kc, s1));
   if (ka && kb) METIS_TRY(metis_launch_gemm_tc(ctx, a.fc, b.fc, pl.pm, METIS_FP32, kb, s2));
-  if (side_by_side) {
-    METIS_TRY(metis_join(ctx, s, 0));
-    METIS_TRY(metis_join(ctx, s, 1));
-  }
+  METIS_TRY(metis_join(ctx, s, side0));
+  METIS_TRY(metis_join(ctx, s, side0 + 1));
   const int64_t mx = M > N ? M : N;
   METIS_CUDA_TRY(metis_launch_pdl(lowrank_finish_kernel, dim3((unsigned)metis_ceil_div(mx, 8)), dim3(256), 0, s,
       M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
@@ -416,7 +413,8 @@ metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void
                           size_t ws_bytes, cudaStream_t s) {
   Plan pl;
   METIS_TRY(make_plan(a, b, ws, ws_bytes, &pl));
-  METIS_TRY(split_gemm_prologue(ctx, a, b, pl, true, s));
+  METIS_TRY(metis_fork(ctx, s, 2));
+  METIS_TRY(split_gemm_prologue(ctx, a, b, pl, 0, s));
   return split_gemm_main(ctx, a, b, pl, d, d_dtype, ldd, s);
 }
 
@@ -466,9 +464,10 @@ metis_status_t metis_linear_bwd(metis_handle_t h, const metis_operand_t* dy, con
     const metis_status_t st = make_plan(wa, wb, ws ? reinterpret_cast<unsigned char*>(ws) + off : nullptr,
                                         ws_bytes > off ? ws_bytes - off : 0, &pw);
     if (st == METIS_OK) {
-      METIS_TRY(metis_fork(h, s, 3));
-      METIS_TRY(split_gemm_prologue(h, wa, wb, pw, false, h->side[2]));
-      METIS_TRY(split_gemm_prologue(h, da, db, pd, true, s));
+      // all six skinny products at once (a large GEMM, once resident, leaves no SM to a kernel that comes later)
+      METIS_TRY(metis_fork(h, s, METIS_N_SIDE));
+      METIS_TRY(split_gemm_prologue(h, wa, wb, pw, 3, h->side[2]));
+      METIS_TRY(split_gemm_prologue(h, da, db, pd, 0, s));
       METIS_TRY(split_gemm_main(h, da, db, pd, dx, dx_dtype, lddx, s));
       METIS_TRY(metis_join(h, s, 2));
       METIS_TRY(split_gemm_main(h, wa, wb, pw, dw, dw_dtype, lddw, s));
