@@ -188,6 +188,19 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           const uint32_t sfb_t = sfa_t + 4 * K_STEPS;
           const uint64_t sfa_d = make_smem_desc(sfa_addr(s), 128, SWIZZLE_NONE), sfb_d = make_smem_desc(sfb_addr(s), 128, SWIZZLE_NONE);
           const uint64_t a_d = make_smem_desc(a_addr(s), 1024, SWIZZLE_128B), b_d = make_smem_desc(b_addr(s), 1024, SWIZZLE_128B);
+          if (atoms == K_STEPS) {
+#pragma unroll
+            for (int k = 0; k < K_STEPS; ++k) {
+              tc_cp_sf(sfa_t + 4 * k, sfa_d + (uint64_t)(k * 32));
+#pragma unroll
+              for (int t = 0; t < C::N_TILES_SF; ++t)
+                tc_cp_sf(sfb_t + 4 * (k * C::N_TILES_SF + t), sfb_d + (uint64_t)((t * K_STEPS + k) * 32));
+            }
+#pragma unroll
+            for (int k = 0; k < K_STEPS; ++k)
+              tc_mma_nvf4(d_tmem, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc, sfa_t + 4 * k, sfb_t + 4 * k * C::N_TILES_SF,
+                          (kb | k) != 0 ? 1u : 0u);
+          } else {
           for (int k = 0; k < atoms; ++k) {
             tc_cp_sf(sfa_t + 4 * k, sfa_d + (uint64_t)(k * 32));
 #pragma unroll
@@ -197,6 +210,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           for (int k = 0; k < atoms; ++k)
             tc_mma_nvf4(d_tmem, a_d + (uint64_t)(k * 2), b_d + (uint64_t)(k * 2), idesc, sfa_t + 4 * k, sfb_t + 4 * k * C::N_TILES_SF,
                         (kb | k) != 0 ? 1u : 0u);
+          }
           tc_commit(empty_bar(s));                           // slot reusable once these MMAs have read it
         }
         __syncwarp();
