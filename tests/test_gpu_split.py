@@ -137,6 +137,43 @@ def test_all_zero_operand_is_degenerate_but_clean(ctx):
             assert np.count_nonzero(c & 7) == 0 and np.count_nonzero(s) == 0 and np.isfinite(ts)
 
 
+@pytest.mark.parametrize("mode_name", ["sampled", "full"])
+def test_rank_deficient_operand(ctx, mode_name):
+    """An operand of exact rank 3 (small integers: no BF16 rounding) split with k = 8: the sketch has dependent columns
+    and five of the eight singular values are zero.  What is unique must match - the three non-zero singular values
+    (against a library SVD and the oracle), the projector onto their right singular vectors, a residual that is
+    zero - and the rest must be clean: finite everywhere, zero factors for the zero values, status OK."""
+    from gpu_util import to_dev_bf16
+    B, h = ctx
+    mode = B.SKETCH_SAMPLED if mode_name == "sampled" else B.SKETCH_FULL
+    rng = np.random.default_rng(77)
+    rows, cols, r, k, p = 640, 384, 3, 8, 4
+    u = rng.integers(-2, 3, size=(rows, r)).astype(np.float64)
+    v = rng.integers(-2, 3, size=(cols, r)).astype(np.float64)
+    x = u @ v.T                                                   # integers of magnitude <= 12: exact in BF16
+    op, dense = h.split(to_dev_bf16(x), k, p, sketch=mode, seed=9, want_residual=True)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    sig = op.sigma.cpu().numpy().astype(np.float64)
+    left, right = op.left.cpu().numpy().astype(np.float64), op.right.cpu().numpy().astype(np.float64)
+    dense = dense.cpu().numpy().astype(np.float64)
+    assert np.isfinite(sig).all() and np.isfinite(left).all() and np.isfinite(right).all() and np.isfinite(dense).all()
+    s_true = np.linalg.svd(x, compute_uv=False)[:r]
+    assert np.max(np.abs(sig[:r] - s_true) / s_true) < 1e-4
+    sp = osp.split(x, k, p, osp.MODE_SAMPLED if mode_name == "sampled" else osp.MODE_FULL, seed=9)
+    assert np.max(np.abs(sp.sigma[:r] - s_true) / s_true) < 1e-8
+    assert np.max(np.abs(sig[r:k])) < 1e-3 * s_true[0]
+    # projector onto the top right singular vectors (unique although the vectors of equal values are not)
+    vt = np.linalg.svd(x, full_matrices=False)[2][:r]
+    pr = right[:r].T @ right[:r]
+    assert np.linalg.norm(pr - vt.T @ vt) < 1e-4
+    # everything is in the low-rank part: reconstruction from the first three factors, residual at rounding level
+    recon = (left[:r].T * sig[:r]) @ right[:r]
+    assert np.linalg.norm(recon - x) < 1e-5 * np.linalg.norm(x)
+    assert np.linalg.norm(dense) < 1e-5 * np.linalg.norm(x)
+    assert np.linalg.norm((left[:k].T * sig[:k]) @ right[:k] + dense - x) < 1e-5 * np.linalg.norm(x)
+
+
 def test_rank_zero_is_plain_quantization(ctx):
     from gpu_util import to_dev_bf16, nv_to_numpy
     B, h = ctx
