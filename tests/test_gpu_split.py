@@ -174,6 +174,35 @@ def test_rank_deficient_operand(ctx, mode_name):
     assert np.linalg.norm((left[:k].T * sig[:k]) @ right[:k] + dense - x) < 1e-5 * np.linalg.norm(x)
 
 
+@pytest.mark.parametrize("mode_name", ["sampled", "full"])
+def test_repeated_singular_values_inside_the_top_k(ctx, mode_name):
+    """Four equal singular values, then distinct ones, over a Gaussian bulk, k = 8: the singular vectors of the equal
+    values are any basis of their 4-dimensional space, so only that space is compared (projector), together with the
+    singular values, the projector of the whole rank-8 part and the residual, which do not depend on the choice."""
+    from gpu_util import rel_fro
+    B, h = ctx
+    mode, omode = (B.SKETCH_SAMPLED, osp.MODE_SAMPLED) if mode_name == "sampled" else (B.SKETCH_FULL, osp.MODE_FULL)
+    rng = np.random.default_rng(31)
+    rows, cols, k, p = 1024, 512, 8, 8
+    u, _ = np.linalg.qr(rng.standard_normal((rows, k)))
+    v, _ = np.linalg.qr(rng.standard_normal((cols, k)))
+    sv = np.array([400.0, 400.0, 400.0, 400.0, 300.0, 250.0, 200.0, 150.0])
+    x = synth.to_bf16_values((u * sv) @ v.T + 0.05 * rng.standard_normal((rows, cols))).astype(np.float64)
+    op, dense = _run(B, h, x, k, p, mode, seed=4)
+    sp = osp.split(x, k, p, omode, seed=4)
+    sig = op.sigma.cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(sig - sp.sigma) / sp.sigma) < 1e-3
+    right = op.right.cpu().numpy().astype(np.float64)[:k].T
+    left = op.left.cpu().numpy().astype(np.float64)[:k].T
+    for cols_ in (slice(0, 4), slice(0, k)):
+        assert np.linalg.norm(right[:, cols_] @ right[:, cols_].T - sp.right[:, cols_] @ sp.right[:, cols_].T) < 2e-3
+        assert np.linalg.norm(left[:, cols_] @ left[:, cols_].T - sp.left[:, cols_] @ sp.left[:, cols_].T) < 2e-3
+    assert np.allclose(right.T @ right, np.eye(k), atol=1e-4) and np.allclose(left.T @ left, np.eye(k), atol=1e-4)
+    tol_r = max(1e-6, 32 * 2.0 ** -24 * np.linalg.norm(x) / np.linalg.norm(sp.residual))
+    assert rel_fro(dense, sp.residual) < tol_r
+    assert rel_fro((left * sig) @ right.T + dense, x) < 1e-5
+
+
 def test_rank_zero_is_plain_quantization(ctx):
     from gpu_util import to_dev_bf16, nv_to_numpy
     B, h = ctx
