@@ -15,7 +15,7 @@
  * General rules
  *  - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns every
  *    buffer (inputs, outputs, workspace); the library allocates device memory only inside
- *    metis_create (a 128 KiB quantile table and a status word; it also creates three streams and four
+ *    metis_create (a 128 KiB quantile table and a status word; it also creates five streams and six
  *    events there) and frees it in metis_destroy.
  *  - All work is enqueued on the caller's stream (a cudaStream_t passed as void*); calls return
  *    without synchronising.  Inside a call, independent sub-chains may run on streams the handle owns;

@@ -8,7 +8,7 @@ Besides the step it times, each alone: the decomposition of every operand (algor
 of the same layer without any split (the denominator of the split overhead).  Inputs are planted-spectrum
 matrices generated on the device (rank-r spike, top singular value 100x the bulk edge, 10:1 span, Gaussian
 bulk); they are regenerated from the seed, never read from disk.  Timing: CUDA events on the launching stream,
-inputs rotate over enough sets to exceed the L2; the step (about 100 kernels on three streams) is replayed as one
+inputs rotate over enough sets to exceed the L2; the step (about 90 kernels on three streams) is replayed as one
 CUDA graph per input set unless --no-graph is given, so that the host's launch rate does not bound the smaller layers.
 """
 import argparse
