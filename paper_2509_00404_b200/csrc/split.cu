@@ -308,17 +308,21 @@ constexpr int GC_THREADS = 512;
 constexpr size_t GC_MAX_SMEM = 144 * 1024;              // beside ~45 KiB of static shared memory
 __host__ __device__ inline int gram_chol_pitch(int q) { return 4 * ((q + 3) / 4) + 2; }
 __host__ inline size_t gram_chol_smem(int64_t n_s, int q) { return (size_t)n_s * gram_chol_pitch(q) * sizeof(double); }
+// Well-conditioned sketch (every pivot above 1e-8 of the largest diagonal: Z L^-T is orthonormal to ~1e-8 already):
+// the kernel writes L and the reciprocal pivots and clears *applied; apply_chol_kernel, on many CTAs, does the
+// triangular solves.  Otherwise (rare) the whole CholeskyQR2 runs here on the FP64 copy - solve, second Gram
+// matrix, second factor, second solve - H is written over z and *applied is set, which makes the apply kernel
+// behind this one return at once.
 __global__ void __launch_bounds__(GC_THREADS, 1)
-gram_chol_kernel(const float* __restrict__ z, int n_s, int q, double* __restrict__ l_out, double* __restrict__ invd_out,
-                 const int* __restrict__ skip, int* __restrict__ well_conditioned) {
+gram_chol_kernel(float* __restrict__ z, int n_s, int q, double* __restrict__ l_out, double* __restrict__ invd_out,
+                 int* __restrict__ applied) {
   metis_pdl_wait();
-  if (skip != nullptr && *skip) return;
   extern __shared__ __align__(16) double zs[];
   __shared__ double L[MAXQ][MAXQ + 1];
   __shared__ double gmax_s;
   __shared__ double dmin_s;
   __shared__ double inv_s[MAXQ];
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nb = (q + 3) / 4, zp = gram_chol_pitch(q);
   for (int o = tid; o < n_s * zp; o += GC_THREADS) {
     const int r = o / zp, c = o - r * zp;
@@ -332,53 +336,82 @@ gram_chol_kernel(const float* __restrict__ z, int n_s, int q, double* __restrict
   while ((bi + 1) * (bi + 2) / 2 <= o) ++bi;
   const int bj = o - bi * (bi + 1) / 2;
   const bool active = o < blocks;
-  double acc[4][4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+  bool solved_here = false;
   __syncthreads();
-  if (active) {
-    const double* pa = zs + 4 * bi;
-    const double* pb = zs + 4 * bj;
+  for (int pass = 0; pass < 2; ++pass) {
+    double acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+    if (active) {
+      const double* pa = zs + 4 * bi;
+      const double* pb = zs + 4 * bj;
 #pragma unroll 2
-    for (int rr = part; rr < n_s; rr += S) {
-      const double2 a01 = *reinterpret_cast<const double2*>(pa + rr * zp), a23 = *reinterpret_cast<const double2*>(pa + rr * zp + 2);
-      const double2 b01 = *reinterpret_cast<const double2*>(pb + rr * zp), b23 = *reinterpret_cast<const double2*>(pb + rr * zp + 2);
-      const double av[4] = {a01.x, a01.y, a23.x, a23.y}, bv[4] = {b01.x, b01.y, b23.x, b23.y};
+      for (int rr = part; rr < n_s; rr += S) {
+        const double2 a01 = *reinterpret_cast<const double2*>(pa + rr * zp), a23 = *reinterpret_cast<const double2*>(pa + rr * zp + 2);
+        const double2 b01 = *reinterpret_cast<const double2*>(pb + rr * zp), b23 = *reinterpret_cast<const double2*>(pb + rr * zp + 2);
+        const double av[4] = {a01.x, a01.y, a23.x, a23.y}, bv[4] = {b01.x, b01.y, b23.x, b23.y};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] += av[i] * bv[j];
+      }
+    }
+    for (int off = S >> 1; off > 0; off >>= 1) {
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] += av[i] * bv[j];
+        for (int j = 0; j < 4; ++j) acc[i][j] += __shfl_xor_sync(0xFFFFFFFFu, acc[i][j], off);
     }
+    if (active && part == 0) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (4 * bi + i < q && 4 * bj + j < q) L[4 * bi + i][4 * bj + j] = acc[i][j];
+    }
+    __syncthreads();
+    if (tid < 32) {
+      double gm = 0.0;
+      for (int i = tid; i < q; i += 32) gm = fmax(gm, L[i][i]);
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) gm = fmax(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, off));
+      if (tid == 0) gmax_s = gm;
+    }
+    __syncthreads();
+    const double tol = 1e-13 * gmax_s;
+    cta_cholesky<MAXQ + 1>(L, q, tol, inv_s, &dmin_s, GC_THREADS);
+    if (pass == 0 && dmin_s > 1e-8 * gmax_s) break;
+    // z_row <- z_row L^-T in shared memory, one warp per row (the recurrence of apply_chol_kernel)
+    solved_here = true;
+    for (int r = warp; r < n_s; r += GC_THREADS / 32) {
+      double* zr = zs + r * zp;
+      double z0 = lane < q ? zr[lane] : 0.0, z1 = lane + 32 < q ? zr[lane + 32] : 0.0, z2 = lane + 64 < q ? zr[lane + 64] : 0.0;
+      for (int j = 0; j < q; ++j) {
+        const double lj0 = lane < q ? L[lane][j] : 0.0;
+        const double lj1 = lane + 32 < q ? L[lane + 32][j] : 0.0;
+        const double lj2 = lane + 64 < q ? L[lane + 64][j] : 0.0;
+        const double zj = __shfl_sync(0xFFFFFFFFu, j < 32 ? z0 : (j < 64 ? z1 : z2), j & 31);
+        const double hj = zj * inv_s[j];
+        if (lane == (j & 31)) { if (j < 32) z0 = hj; else if (j < 64) z1 = hj; else z2 = hj; }
+        if (lane > j) z0 -= hj * lj0;
+        if (lane + 32 > j) z1 -= hj * lj1;
+        if (lane + 64 > j) z2 -= hj * lj2;
+      }
+      if (lane < q) zr[lane] = z0;
+      if (lane + 32 < q) zr[lane + 32] = z1;
+      if (lane + 64 < q) zr[lane + 64] = z2;
+    }
+    __syncthreads();
   }
-  for (int off = S >> 1; off > 0; off >>= 1) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) acc[i][j] += __shfl_xor_sync(0xFFFFFFFFu, acc[i][j], off);
+  if (tid == 0) *applied = solved_here ? 1 : 0;
+  if (solved_here) {
+    for (int e = tid; e < n_s * q; e += GC_THREADS) z[e] = (float)zs[(e / q) * zp + e % q];
+  } else {
+    if (tid < q) invd_out[tid] = inv_s[tid];
+    for (int e = tid; e < q * q; e += GC_THREADS) l_out[e] = L[e / q][e % q];
   }
-  if (active && part == 0) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-        if (4 * bi + i < q && 4 * bj + j < q) L[4 * bi + i][4 * bj + j] = acc[i][j];
-  }
-  __syncthreads();
-  if (tid < 32) {
-    double gm = 0.0;
-    for (int i = tid; i < q; i += 32) gm = fmax(gm, L[i][i]);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) gm = fmax(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, off));
-    if (tid == 0) gmax_s = gm;
-  }
-  __syncthreads();
-  const double tol = 1e-13 * gmax_s;
-  cta_cholesky<MAXQ + 1>(L, q, tol, inv_s, &dmin_s, GC_THREADS);
-  if (tid < q) invd_out[tid] = inv_s[tid];
-  if (tid == 0 && well_conditioned != nullptr) *well_conditioned = (dmin_s > 1e-8 * gmax_s) ? 1 : 0;
-  for (int e = tid; e < q * q; e += GC_THREADS) l_out[e] = L[e / q][e % q];
 }
 
 // One CholeskyQR pass, step 2: z_row <- z_row L^-T by forward substitution, one warp per row, column-oriented:
@@ -1676,20 +1709,22 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     METIS_CUDA_TRY(metis_launch_pdl((reduce_partials_kernel), dim3((unsigned)metis_ceil_div(n_s * q, 256)), dim3(256), (size_t)(0), s, zp, chunks, n_s * q, z)); METIS_COUNT_LAUNCH();
   }
   // (3) CholeskyQR2: orthonormal basis H of range(Z), in place
+  if (gram_chol_smem(n_s, q) <= GC_MAX_SMEM) {
+    // a short sketch: Gram matrix and factorisation in one CTA; the triangular solves on many CTAs unless the sketch
+    // was ill-conditioned, in which case the first kernel has done both passes itself and the second returns at once
+    static bool at_ = false;
+    if (!at_) { METIS_CUDA_TRY(cudaFuncSetAttribute(gram_chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GC_MAX_SMEM)); at_ = true; }
+    METIS_CUDA_TRY(metis_launch_pdl((gram_chol_kernel), dim3(1), dim3(GC_THREADS), gram_chol_smem(n_s, q), s, z, (int)n_s, q, linv, invd, cond_flag)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((apply_chol_kernel), dim3((unsigned)metis_ceil_div(n_s, 8)), dim3(256), (size_t)(0), s, z, n_s, q, linv, invd, (const int*)cond_flag)); METIS_COUNT_LAUNCH();
+  } else {
   for (int pass = 0; pass < 2; ++pass) {
     int64_t rpp; const int parts = gram_parts(n_s, &rpp);
     const int* skip = pass == 0 ? nullptr : cond_flag;
-    if (gram_chol_smem(n_s, q) <= GC_MAX_SMEM) {
-      // a short sketch: Gram matrix and factorisation in one CTA
-      static bool at_ = false;
-      if (!at_) { METIS_CUDA_TRY(cudaFuncSetAttribute(gram_chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GC_MAX_SMEM)); at_ = true; }
-      METIS_CUDA_TRY(metis_launch_pdl((gram_chol_kernel), dim3(1), dim3(GC_THREADS), gram_chol_smem(n_s, q), s, z, (int)n_s, q, linv, invd, skip, pass == 0 ? cond_flag : nullptr)); METIS_COUNT_LAUNCH();
-    } else {
     METIS_CUDA_TRY(metis_launch_pdl((gram_kernel), dim3(parts), dim3(256), (size_t)(0), s, z, n_s, q, q, 1, rpp, gram, skip)); METIS_COUNT_LAUNCH();
     METIS_CUDA_TRY(metis_launch_pdl((reduce_gram_kernel), dim3((unsigned)metis_ceil_div(q * q, 32)), dim3(128), (size_t)(0), s, gram, parts, q * q, gram1, skip)); METIS_COUNT_LAUNCH();
     METIS_CUDA_TRY(metis_launch_pdl((chol_kernel), dim3(1), dim3(256), (size_t)(0), s, gram1, q, linv, invd, skip, pass == 0 ? cond_flag : nullptr)); METIS_COUNT_LAUNCH();
-    }
     METIS_CUDA_TRY(metis_launch_pdl((apply_chol_kernel), dim3((unsigned)metis_ceil_div(n_s, 8)), dim3(256), (size_t)(0), s, z, n_s, q, linv, invd, skip)); METIS_COUNT_LAUNCH();
+  }
   }
   // (4) M = H^T x[S,:], eigen-decomposition of M M^T, right basis
   {

@@ -203,6 +203,45 @@ def test_repeated_singular_values_inside_the_top_k(ctx, mode_name):
     assert rel_fro((left * sig) @ right.T + dense, x) < 1e-5
 
 
+@pytest.mark.parametrize("mode_name", ["sampled", "full"])
+def test_ill_conditioned_sketch_needs_the_second_orthonormalisation_pass(ctx, mode_name):
+    """Block-diagonal operand of exact small-integer entries: a rank-4 block with singular values near 500 and a
+    full-rank block scaled by 2^-16 (singular values near 7e-4).  The sketch columns beyond the fourth differ from
+    combinations of the first four only at the 1e-6 level, so the Gram matrix has pivots near 1e-10 of its largest
+    (1.1e-10 ... 4.6e-10, computed from the oracle's sketch for this seed): neither dependent (below 1e-13) nor
+    well-conditioned (above 1e-8), the case the second CholeskyQR pass exists for.  Checked against a
+    library SVD and the oracle: top singular values, their right projector, orthonormal factors, exact split."""
+    from gpu_util import to_dev_bf16
+    B, h = ctx
+    mode, omode = (B.SKETCH_SAMPLED, osp.MODE_SAMPLED) if mode_name == "sampled" else (B.SKETCH_FULL, osp.MODE_FULL)
+    rng = np.random.default_rng(123)
+    rows, cols, r, k, p = 640, 384, 4, 4, 4
+    x = np.zeros((rows, cols))
+    x[: rows // 2, : cols // 2] = rng.integers(-2, 3, size=(rows // 2, r)) @ rng.integers(-2, 3, size=(r, cols // 2))
+    x[rows // 2 :, cols // 2 :] = rng.integers(-2, 3, size=(rows // 2, cols // 2)) * 2.0 ** -16
+    assert np.array_equal(synth.to_bf16_values(x), x)
+    op, dense = h.split(to_dev_bf16(x), k, p, sketch=mode, seed=6, want_residual=True)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    sig = op.sigma.cpu().numpy().astype(np.float64)[:k]
+    left = op.left.cpu().numpy().astype(np.float64)[:k].T
+    right = op.right.cpu().numpy().astype(np.float64)[:k].T
+    dense = dense.cpu().numpy().astype(np.float64)
+    uu, ss, vt = np.linalg.svd(x, full_matrices=False)
+    assert ss[3] / ss[4] > 1e4
+    assert np.max(np.abs(sig - ss[:k]) / ss[:k]) < 1e-5
+    sp = osp.split(x, k, p, omode, seed=6)
+    assert np.max(np.abs(sp.sigma - ss[:k]) / ss[:k]) < 1e-7
+    # the orthonormal basis is stored in FP32: entries of the small block's rows, exactly zero in the true vectors,
+    # come out at the 1e-5 level (FP32 rounding of columns that are 1e6 times smaller than the first ones)
+    assert np.linalg.norm(right @ right.T - vt[:k].T @ vt[:k]) < 1e-3
+    assert np.linalg.norm(left @ left.T - uu[:, :k] @ uu[:, :k].T) < 1e-3
+    assert np.allclose(left.T @ left, np.eye(k), atol=1e-4) and np.allclose(right.T @ right, np.eye(k), atol=1e-4)
+    assert np.linalg.norm((left * sig) @ right.T + dense - x) < 1e-6 * np.linalg.norm(x)
+    # the residual is the small block (plus FP32 rounding of the large one)
+    assert np.linalg.norm(dense - sp.residual) < 1e-6 * np.linalg.norm(x)
+
+
 def test_rank_zero_is_plain_quantization(ctx):
     from gpu_util import to_dev_bf16, nv_to_numpy
     B, h = ctx
