@@ -16,7 +16,7 @@
  *  - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns every
  *    buffer (inputs, outputs, workspace); the library allocates device memory only inside
  *    metis_create (a 128 KiB quantile table and a status word; it also creates five streams and six
- *    events there) and frees it in metis_destroy.
+ *    events there and sets the per-device kernel attributes) and frees it in metis_destroy.
  *  - All work is enqueued on the caller's stream (a cudaStream_t passed as void*); calls return
  *    without synchronising.  Inside a call, independent sub-chains may run on streams the handle owns;
  *    they start after the work already on the caller's stream and are joined back into it before the
@@ -132,7 +132,15 @@ metis_status_t metis_debug_quantile_table(metis_handle_t h, uint16_t* host_out);
  * *device_slot when `stream` reaches it; usable inside a stream capture, where events cannot be timed. */
 metis_status_t metis_debug_timestamp(metis_handle_t h, uint64_t* device_slot, metis_stream_t stream);
 
-/* Test / benchmark hook: kernels launched by the library in this process so far (host counter). */
+/* Failure-detection hook (the library's kernels bound every wait on an mbarrier and report an expired one through
+ * METIS_DEV_TIMEOUT instead of hanging): enqueues a two-warp kernel whose first warp waits at most `polls`
+ * (1 .. 2^20) polls on a barrier that is never completed, and whose second warp waits on another one until it
+ * sees the first warp's give-up flag.  Afterwards the status word holds METIS_DEV_TIMEOUT and device_seen[0..1]
+ * (device, two words) hold, per warp, bit 0 = "my wait expired", bit 1 = "the give-up flag was set".  The kernel
+ * returns normally; the context stays usable. */
+metis_status_t metis_debug_wait_timeout(metis_handle_t h, uint32_t polls, uint32_t* device_seen, metis_stream_t stream);
+
+/* Test / benchmark hook: kernels launched by the library in this process so far (host counter, atomic). */
 uint64_t metis_debug_launch_count(void);
 
 /* Bytes of scale storage for a stored rows x k_len NVFP4 tensor (host-only helper, no handle). */
@@ -201,8 +209,10 @@ metis_status_t metis_linear_fwd(metis_handle_t h, const metis_operand_t* x, cons
  * meant for callers that own inputs and outputs but cannot obtain scratch memory: a process whose memory
  * pool already holds every free byte of the device, or a plug-in that is not allowed to call an allocator.
  * The call allocates nothing on host or device.
- *  - Limit: layers whose metis_workspace_bytes(2, l, n, k, 0) exceeds METIS_STATIC_WS_BYTES are refused with
- *    METIS_ERR_WORKSPACE and nothing is enqueued.
+ *  - Limit: the layer's intermediates must fit METIS_STATIC_WS_BYTES, else METIS_ERR_WORKSPACE is returned and
+ *    nothing is enqueued.  With k = k_x + k_w they are 4 (l + n) k bytes of FP32 skinny operands plus, when l and
+ *    n are both at least 256, 2 (l + n) roundup64(3 k) bytes of BF16 correction operands, or else (a smaller
+ *    layer) 4 l n bytes of FP32 staging for the main product; plain NVFP4 operands (k = 0) need nothing.
  *  - h's device must be the current device (else METIS_ERR_INVALID_ARG).
  *  - The first call on each device looks up the array's device address (a one-time runtime query); make that
  *    first call during start-up, before any stream capture is begun.

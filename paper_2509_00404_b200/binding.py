@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "ALIGNMENT", 4: "WORKS
                 7: "NONFINITE", 8: "NUMERIC", 9: "TIMEOUT"}
 
 EXPORTED = ["metis_create", "metis_destroy", "metis_last_device_status", "metis_debug_quantile_table",
-            "metis_debug_launch_count", "metis_debug_timestamp",
+            "metis_debug_launch_count", "metis_debug_timestamp", "metis_debug_wait_timeout",
             "metis_sf_bytes", "metis_workspace_bytes", "metis_default_sample_count", "metis_quantize_nvfp4",
             "metis_split", "metis_linear_fwd", "metis_linear_fwd_static_ws", "metis_linear_bwd", "metis_gemm_nvfp4"]
 
@@ -69,6 +69,7 @@ def lib():
     l.metis_debug_quantile_table.argtypes = [vp, vp]
     l.metis_debug_launch_count.argtypes = []
     l.metis_debug_timestamp.argtypes = [vp, vp, vp]
+    l.metis_debug_wait_timeout.argtypes = [vp, u32, vp, vp]
     l.metis_debug_launch_count.restype = u64
     l.metis_sf_bytes.argtypes = [i64, i64, i32]
     l.metis_sf_bytes.restype = sz
@@ -321,6 +322,12 @@ class Handle:
     def timestamp(self, slot, stream=None):
         """Enqueues a kernel that writes the GPU nanosecond timer into the int64 CUDA tensor element `slot`."""
         _check("metis_debug_timestamp", lib().metis_debug_timestamp(self._h, _ptr(slot), _stream_ptr(stream)))
+
+    def wait_timeout(self, polls=256, stream=None):
+        """metis_debug_wait_timeout: runs the bounded-wait hook; returns the two per-warp words as a CUDA int32 tensor."""
+        seen = torch.zeros(2, dtype=torch.int32, device="cuda")
+        _check("metis_debug_wait_timeout", lib().metis_debug_wait_timeout(self._h, polls, _ptr(seen), _stream_ptr(stream)))
+        return seen
 
     # -- metis_gemm_nvfp4 ----------------------------------------------------------------------
     def gemm_nvfp4(self, a, b, out_dtype=torch.float32, impl=0, out=None, stream=None):

@@ -3,12 +3,15 @@
 #include <math.h>
 #include <stdlib.h>
 
-#include "common.cuh"
+#include <atomic>
+
+#include "tc_ptx.cuh"
 
 size_t metis_split_ws_bytes(int64_t rows, int64_t cols, int k, int p);
 size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k);
 
-unsigned long long g_metis_launch_count = 0;
+static std::atomic<unsigned long long> g_metis_launch_count{0};
+void metis_count_launch() { g_metis_launch_count.fetch_add(1, std::memory_order_relaxed); }
 
 namespace {
 
@@ -68,9 +71,17 @@ metis_status_t metis_create(metis_handle_t* out, int device) {
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join[i], cudaEventDisableTiming);
   }
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
-  if (e != cudaSuccess) {
-    cudaFree(ctx->quantile_lut); cudaFree(ctx->dev_status); free(ctx);
-    return METIS_ERR_CUDA;
+  metis_status_t st = e == cudaSuccess ? METIS_OK : METIS_ERR_CUDA;
+  // kernel attributes of this device (the device is current here)
+  if (st == METIS_OK) st = metis_quantize_set_attrs();
+  if (st == METIS_OK) st = metis_gemm_set_attrs(ctx);
+  if (st == METIS_OK) st = metis_split_set_attrs();
+  if (st == METIS_OK) st = metis_coeff_set_attrs();
+  if (st == METIS_OK) st = metis_residual_set_attrs();
+  if (st == METIS_OK) st = metis_linear_set_attrs();
+  if (st != METIS_OK) {
+    metis_destroy(ctx);                                // releases whatever was created so far
+    return st;
   }
   *out = ctx;
   return METIS_OK;
@@ -104,7 +115,7 @@ metis_status_t metis_debug_quantile_table(metis_handle_t h, uint16_t* host_out) 
   return METIS_OK;
 }
 
-uint64_t metis_debug_launch_count(void) { return g_metis_launch_count; }
+uint64_t metis_debug_launch_count(void) { return g_metis_launch_count.load(std::memory_order_relaxed); }
 
 size_t metis_sf_bytes(int64_t rows, int64_t k_len, int32_t sf_layout) {
   if (rows <= 0 || k_len <= 0) return 0;
@@ -130,6 +141,34 @@ __global__ void timestamp_kernel(unsigned long long* slot) {
   *slot = t;
 }
 }  // namespace
+
+namespace {
+// Failure-detection hook: the producer / consumer skeleton of the tensor-core kernels with nothing in flight.
+// Warp 0 waits (bounded) on a "data landed" barrier that nobody will ever arrive at; warp 1 waits on a second one
+// and must notice the shared `dead` flag; everybody then meets at the CTA barrier and returns.  No TMA, no MMA, no
+// tensor memory: the only thing exercised is the give-up path of the bounded wait and the status word.
+__global__ void __launch_bounds__(64) wait_timeout_kernel(uint32_t* dev_status, uint32_t polls, uint32_t* seen) {
+  __shared__ __align__(8) uint64_t bars[2];
+  __shared__ int dead;
+  using namespace metis_tc;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) { mbar_init(smem_u32(&bars[0]), 1); mbar_init(smem_u32(&bars[1]), 1); dead = 0; fence_barrier_init(); }
+  __syncthreads();
+  bool ok = true;
+  if (lane == 0) ok = mbar_wait_n(smem_u32(&bars[warp]), 0, dev_status, &dead, warp == 0 ? polls : 16u * polls + 4096u);
+  __syncwarp();
+  __syncthreads();
+  if (lane == 0) seen[warp] = (ok ? 0u : 1u) | (dead ? 2u : 0u);
+}
+}  // namespace
+
+metis_status_t metis_debug_wait_timeout(metis_handle_t h, uint32_t polls, uint32_t* device_seen, metis_stream_t stream) {
+  if (!h || !device_seen || polls == 0 || polls > (1u << 20)) return METIS_ERR_INVALID_ARG;
+  wait_timeout_kernel<<<1, 64, 0, reinterpret_cast<cudaStream_t>(stream)>>>(h->dev_status, polls, device_seen);
+  METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
 
 metis_status_t metis_debug_timestamp(metis_handle_t h, uint64_t* device_slot, metis_stream_t stream) {
   if (!h || !device_slot) return METIS_ERR_INVALID_ARG;

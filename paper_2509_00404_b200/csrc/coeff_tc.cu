@@ -200,19 +200,25 @@ coeff_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 }
 
 template <int NB>
+constexpr size_t coeff_smem() { return (size_t)STAGES * (A_BYTES + NB * BK * 2) + 1024 + 128; }
+template <int NB>
+cudaError_t set_attr() { return cudaFuncSetAttribute(coeff_tc_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)coeff_smem<NB>()); }
+
+template <int NB>
 metis_status_t launch(const CUtensorMap& mx, const CUtensorMap& mb, const CoeffArgs& g, dim3 grid, cudaStream_t s) {
-  constexpr size_t smem = (size_t)STAGES * (A_BYTES + NB * BK * 2) + 1024 + 128;
-  static bool attr = false;
-  if (!attr) {
-    METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_tc_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr = true;
-  }
+  constexpr size_t smem = coeff_smem<NB>();
   coeff_tc_kernel<NB><<<grid, NUM_THREADS, smem, s>>>(mx, mb, g); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }
 
 }  // namespace
+
+metis_status_t metis_coeff_set_attrs() {
+  METIS_CUDA_TRY(set_attr<48>()); METIS_CUDA_TRY(set_attr<96>()); METIS_CUDA_TRY(set_attr<144>());
+  METIS_CUDA_TRY(set_attr<192>()); METIS_CUDA_TRY(set_attr<240>());
+  return METIS_OK;
+}
 
 // number of column slices (grid.y) and 64-column chunks per slice: about one CTA per SM, at most 8 slices
 int metis_coeff_slices(int64_t rows, int64_t cols, int* chunks_per_slice) {

@@ -17,7 +17,18 @@ struct metis_context {
   // the caller's stream with events before the call's last kernels (everything stays asynchronous).
   cudaStream_t side[METIS_N_SIDE];
   cudaEvent_t ev_fork, ev_join[METIS_N_SIDE];
+  int max_pairs;                 // two-CTA clusters of the large GEMM that this device keeps resident at once
 };
+
+// Per-device kernel attributes (dynamic shared memory above 48 KiB).  Function attributes belong to the device
+// that is current when they are set, so metis_create sets them for the handle's device, once per handle; no
+// launch helper keeps a process-wide "already set" flag.
+metis_status_t metis_quantize_set_attrs();
+metis_status_t metis_gemm_set_attrs(metis_context* ctx);
+metis_status_t metis_split_set_attrs();
+metis_status_t metis_coeff_set_attrs();
+metis_status_t metis_residual_set_attrs();
+metis_status_t metis_linear_set_attrs();
 
 // fork: side stream i starts after everything enqueued so far on `main`
 static inline metis_status_t metis_fork(metis_context* ctx, cudaStream_t main, int n_side) {
@@ -66,8 +77,9 @@ static inline cudaError_t metis_launch_pdl(void (*kernel)(KArgs...), dim3 grid, 
   } while (0)
 
 // Number of kernels the library has launched in this process (read through metis_debug_launch_count).
-extern unsigned long long g_metis_launch_count;
-#define METIS_COUNT_LAUNCH() (++g_metis_launch_count)
+// Process-wide and atomic: handles on several devices or threads may launch at the same time.
+void metis_count_launch();
+#define METIS_COUNT_LAUNCH() metis_count_launch()
 
 static inline bool metis_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline int64_t metis_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }

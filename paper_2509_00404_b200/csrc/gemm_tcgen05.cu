@@ -682,11 +682,6 @@ metis_status_t launch(metis_context* ctx, const metis_nvfp4_t* a, const metis_nv
   g.d = d; g.d_dtype = d_dtype; g.ldd = ldd;
   g.M = (int)a->rows; g.N = (int)b->rows; g.K = (int)a->k_len;
   g.dev_status = ctx->dev_status;
-  static bool attr_set = false;
-  if (!attr_set) {
-    METIS_CUDA_TRY(cudaFuncSetAttribute(gemm_nvfp4_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
-    attr_set = true;
-  }
   const int tiles = (int)(metis_ceil_div(g.M, BLOCK_M) * metis_ceil_div(g.N, BLOCK_N));
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
   METIS_CUDA_TRY(metis_launch_pdl(gemm_nvfp4_kernel<BLOCK_N>, dim3(grid), dim3(NUM_THREADS), C::SMEM_BYTES, s, map_a, map_b, g)); METIS_COUNT_LAUNCH();
@@ -741,24 +736,8 @@ metis_status_t launch_2cta(metis_context* ctx, const metis_nvfp4_t* a, const met
   g.tma_store = metis_aligned16(d) && ((ldd * (d_dtype == METIS_BF16 ? 2 : 4)) % 16 == 0) ? 1 : 0;
   if (g.tma_store) METIS_TRY(make_out_map(ctx, &map_d, d, d_dtype, a->rows, b->rows, ldd));
   else map_d = map_a;
-  static bool attr_set = false;
-  if (!attr_set) {
-    METIS_CUDA_TRY(cudaFuncSetAttribute(two_cta::gemm_nvfp4_2cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)two_cta::SMEM_BYTES));
-    attr_set = true;
-  }
   const int tiles = (int)(metis_ceil_div(g.M, two_cta::TILE_M) * metis_ceil_div(g.N, two_cta::TILE_N));
-  static int max_pairs = 0;
-  if (max_pairs == 0) {
-    // how many 2-CTA clusters can be resident at once (an odd SM count inside a GPC leaves an SM unpaired)
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * (ctx->sm_count / 2)); cfg.blockDim = dim3(two_cta::NUM_THREADS);
-    cfg.dynamicSmemBytes = two_cta::SMEM_BYTES;
-    cudaLaunchAttribute at; at.id = cudaLaunchAttributeClusterDimension; at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
-    cfg.attrs = &at; cfg.numAttrs = 1;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, two_cta::gemm_nvfp4_2cta_kernel, &cfg) != cudaSuccess || n <= 0) n = ctx->sm_count / 2;
-    max_pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
-  }
+  const int max_pairs = ctx->max_pairs;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
   METIS_CUDA_TRY(metis_launch_pdl(two_cta::gemm_nvfp4_2cta_kernel, dim3(2 * pairs), dim3(two_cta::NUM_THREADS), two_cta::SMEM_BYTES, s,
                                   map_a, map_b, map_sfa, map_sfb, map_l, map_r, map_d, g)); METIS_COUNT_LAUNCH();
@@ -766,6 +745,21 @@ metis_status_t launch_2cta(metis_context* ctx, const metis_nvfp4_t* a, const met
 }
 
 }  // namespace
+
+metis_status_t metis_gemm_set_attrs(metis_context* ctx) {
+  METIS_CUDA_TRY(cudaFuncSetAttribute(gemm_nvfp4_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<128>::SMEM_BYTES));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(two_cta::gemm_nvfp4_2cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)two_cta::SMEM_BYTES));
+  // how many 2-CTA clusters can be resident at once (an odd SM count inside a GPC leaves an SM unpaired)
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * (ctx->sm_count / 2)); cfg.blockDim = dim3(two_cta::NUM_THREADS);
+  cfg.dynamicSmemBytes = two_cta::SMEM_BYTES;
+  cudaLaunchAttribute at; at.id = cudaLaunchAttributeClusterDimension; at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+  cfg.attrs = &at; cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, two_cta::gemm_nvfp4_2cta_kernel, &cfg) != cudaSuccess || n <= 0) { n = ctx->sm_count / 2; (void)cudaGetLastError(); }
+  ctx->max_pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
+  return METIS_OK;
+}
 
 metis_status_t metis_launch_gemm_tc(metis_context* ctx, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d,
                                     int d_dtype, int64_t ldd, cudaStream_t s) {

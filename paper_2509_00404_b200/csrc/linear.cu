@@ -286,6 +286,16 @@ metis_status_t launch_factor_grad(cudaStream_t s, const void* g, int g_dtype, in
   return METIS_OK;
 }
 
+// the host-side checks of factor_grads, callable before anything is enqueued
+metis_status_t factor_grads_check(const metis_operand_t* w, const float* d_left, const float* d_sigma, const void* ws, size_t ws_bytes) {
+  if (!w || w->k <= 0 || w->k > 64 || !w->sigma) return METIS_ERR_SHAPE;
+  const metis_nvfp4_t *lq = &w->left_q, *rq = &w->right_q;
+  if (!lq->codes || !rq->codes || lq->k_len != w->rows || rq->k_len != w->cols) return METIS_ERR_SHAPE;
+  if (d_sigma && !d_left) return METIS_ERR_INVALID_ARG;          // the sigma partials ride on the d_left pass
+  if (d_sigma && (!ws || ws_bytes < sizeof(float) * (size_t)metis_ceil_div(w->rows, FG_ROWS) * w->k)) return METIS_ERR_WORKSPACE;
+  return METIS_OK;
+}
+
 // d_left (k x n), d_sigma (k), d_right (k x m) of the weight operand W_t = left diag(sigma) right^T from dw (n x m).
 metis_status_t factor_grads(metis_context* ctx, const void* dw, int dw_dtype, int64_t lddw, const metis_operand_t* w,
                             float* d_left, float* d_sigma, float* d_right, void* ws, size_t ws_bytes, cudaStream_t s) {
@@ -402,8 +412,6 @@ metis_status_t split_gemm_main(metis_context* ctx, const Side& a, const Side& b,
   }
   dim3 grid((unsigned)metis_ceil_div(pl.N, 64), (unsigned)metis_ceil_div(pl.M, 64));
   const size_t smem = sizeof(float) * 2 * pl.kc * 68;
-  static bool attr = false;
-  if (!attr) { METIS_CUDA_TRY(cudaFuncSetAttribute(rank_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 2 * 128 * 68))); attr = true; }
   rank_update_kernel<<<grid, 256, smem, s>>>(pl.y0, pl.M, pl.N, pl.kc, pl.lcat, pl.rcat, d, d_dtype, ldd); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
@@ -420,6 +428,11 @@ metis_status_t split_gemm(metis_context* ctx, const Side& a, const Side& b, void
 
 }  // namespace
 
+metis_status_t metis_linear_set_attrs() {
+  METIS_CUDA_TRY(cudaFuncSetAttribute(rank_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 2 * 128 * 68)));
+  return METIS_OK;
+}
+
 size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k) {
   const int kc = 2 * k;
   const int kx = (3 * kc + 63) / 64 * 64;
@@ -433,7 +446,8 @@ size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k) {
 metis_status_t metis_linear_fwd(metis_handle_t h, const metis_operand_t* x, const metis_operand_t* w, void* y,
                                 int32_t y_dtype, int64_t ldy, void* ws, size_t ws_bytes, metis_stream_t stream) {
   if (!h || !x || !w || !y) return METIS_ERR_INVALID_ARG;
-  if (x->cols != w->cols) return METIS_ERR_SHAPE;
+  if (y_dtype != METIS_BF16 && y_dtype != METIS_FP32) return METIS_ERR_INVALID_ARG;
+  if (x->cols != w->cols || ldy < w->rows) return METIS_ERR_SHAPE;
   // contraction over in-features: X (l x m) by columns, W_t (n x m) by columns
   Side a{&x->res_by_cols, &x->right_q, &x->left_q, x->sigma, x->k};
   Side b{&w->res_by_cols, &w->right_q, &w->left_q, w->sigma, w->k};
@@ -447,8 +461,17 @@ metis_status_t metis_linear_bwd(metis_handle_t h, const metis_operand_t* dy, con
   if (!h || !dy) return METIS_ERR_INVALID_ARG;
   if ((d_left || d_sigma || d_right) && (!dw || !w)) return METIS_ERR_INVALID_ARG;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  // every host-detectable error is reported before anything is enqueued
   if (dx && (!w || dy->cols != w->rows)) return METIS_ERR_SHAPE;
   if (dw && (!x || dy->rows != x->rows)) return METIS_ERR_SHAPE;
+  if (dx && ((dx_dtype != METIS_BF16 && dx_dtype != METIS_FP32))) return METIS_ERR_INVALID_ARG;
+  if (dw && ((dw_dtype != METIS_BF16 && dw_dtype != METIS_FP32))) return METIS_ERR_INVALID_ARG;
+  if (dx && lddx < w->cols) return METIS_ERR_SHAPE;
+  if (dw && lddw < x->cols) return METIS_ERR_SHAPE;
+  if (dw && (d_left || d_sigma || d_right)) {
+    if (w->rows != dy->cols || w->cols != x->cols) return METIS_ERR_SHAPE;
+    METIS_TRY(factor_grads_check(w, d_left, d_sigma, ws, ws_bytes));
+  }
   // dX (l x m) = D W_t, contraction over out-features n: D by columns, W_t by rows (stored m x n)
   Side da{&dy->res_by_cols, &dy->right_q, &dy->left_q, dy->sigma, dy->k};
   Side db = w ? Side{&w->res_by_rows, &w->left_q, &w->right_q, w->sigma, w->k} : Side{};
@@ -482,9 +505,7 @@ metis_status_t metis_linear_bwd(metis_handle_t h, const metis_operand_t* dy, con
   } else if (dw) {
     METIS_TRY(split_gemm(h, wa, wb, dw, dw_dtype, lddw, ws, ws_bytes, s));
   }
-  if (dw && (d_left || d_sigma || d_right)) {
-    if (w->rows != dy->cols || w->cols != x->cols) return METIS_ERR_SHAPE;
+  if (dw && (d_left || d_sigma || d_right))
     METIS_TRY(factor_grads(h, dw, dw_dtype, lddw, w, d_left, d_sigma, d_right, ws, ws_bytes, s));
-  }
   return METIS_OK;
 }

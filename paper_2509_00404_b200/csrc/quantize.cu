@@ -235,6 +235,15 @@ constexpr size_t quantize_smem(bool sr) {
 
 }  // namespace
 
+metis_status_t metis_quantize_set_attrs() {
+  using namespace metis_qt;
+  METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<__nv_bfloat16>(true)));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<float>(true)));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<__nv_bfloat16>(false)));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<float>(false)));
+  return METIS_OK;
+}
+
 metis_status_t metis_launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* amax_out,
                                  cudaStream_t s) {
   METIS_CUDA_TRY(cudaMemsetAsync(amax_out, 0, sizeof(float), s));
@@ -327,14 +336,6 @@ metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int
     return METIS_OK;
   }
   const bool sr = rounding == METIS_ROUND_SR;
-  static bool attr_set = false;
-  if (!attr_set) {
-    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<__nv_bfloat16>(true)));
-    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<float>(true)));
-    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<__nv_bfloat16>(false)));
-    METIS_CUDA_TRY(cudaFuncSetAttribute(quantize_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem<float>(false)));
-    attr_set = true;
-  }
   dim3 grid((unsigned)metis_ceil_div(cols, TILE), (unsigned)metis_ceil_div(rows, TILE));
   float* t0 = by_cols ? by_cols->tensor_scale : nullptr; float* t1 = by_rows ? by_rows->tensor_scale : nullptr;
   if (dtype == METIS_BF16) {

@@ -325,6 +325,14 @@ bool metis_residual_tc_usable(const void* x, int64_t cols) { return metis_aligne
 // a6: [rows][kx] = per row [Ch|Ch|Cl|Ch|Cl2|Cl], b6: [cols][kx] = per column [Bh|Bl|Bh|Bl2|Bh|Bl] (BF16,
 // kx = metis_residual_kx(kp)).  b6 is filled by the caller; a6 too unless `coef` ([rows][kp] FP32) is given,
 // in which case it is written here first.
+metis_status_t metis_residual_set_attrs() {
+  METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+  return METIS_OK;
+}
+
 metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const float* coef, int k, int kp,
                                         const metis_qt::QuantParams& qp, const float* amax_src, float* ts_out0, float* ts_out1,
                                         float* dense, void* a6, void* b6, cudaStream_t s) {
@@ -342,14 +350,6 @@ metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const
   g.p = qp; g.amax_src = amax_src; g.ts_out0 = ts_out0; g.ts_out1 = ts_out1; g.dense = dense;
   g.k_chunks = kx / BK;
   g.dev_status = ctx->dev_status;
-  static bool attr = false;
-  if (!attr) {
-    METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-    METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-    METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-    METIS_CUDA_TRY(cudaFuncSetAttribute(residual_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-    attr = true;
-  }
   const bool fast = rows % TM == 0 && cols % TN == 0 && dense == nullptr &&
                     (qp.c_codes == nullptr || (qp.c_layout == METIS_SF_TILED && reinterpret_cast<uintptr_t>(qp.c_scales) % 2 == 0)) &&
                     (qp.r_codes == nullptr || qp.r_layout == METIS_SF_TILED);

@@ -1561,6 +1561,27 @@ int64_t metis_default_sample_count(int64_t rows, int32_t q) {
   return want < rows ? want : rows;
 }
 
+metis_status_t metis_split_set_attrs() {
+  using namespace metis_qt;
+  METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<1, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<2, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<3, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<5, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 64)));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 48)));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(gram_chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GC_MAX_SMEM));
+#define METIS_PP_ATTR(MTV) METIS_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<MTV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+      (int)((size_t)PP_STAGES * (PP_K * PP_XP * 2 + 3 * (MTV) * 16 * PP_HP * 2))))
+  METIS_PP_ATTR(1); METIS_PP_ATTR(2); METIS_PP_ATTR(3); METIS_PP_ATTR(4); METIS_PP_ATTR(5);
+#undef METIS_PP_ATTR
+  return METIS_OK;
+}
+
 // flags METIS_DEV_NONFINITE when *amax (the amax of a tensor about to be quantized) is not a finite number
 metis_status_t metis_launch_amax_check(metis_context* ctx, const float* amax, cudaStream_t s) {
   METIS_CUDA_TRY(metis_launch_pdl((split_status_kernel), dim3(1), dim3(32), (size_t)(0), s, amax, (const double*)nullptr, 0, ctx->dev_status));
@@ -1654,23 +1675,6 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   bool a6_ready = false;
   metis_context* ctx = h;
   const int kp = (k + 15) / 16 * 16;
-  {
-    static bool attr = false;
-    if (!attr) {
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<1, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<2, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<3, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(jacobi_eig_kernel<5, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)JACOBI_SMEM));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 64)));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(coeff_mma_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * 9 * 32 * 48)));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
-      METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
-      attr = true;
-    }
-  }
   // amax|x| for the residual's tensor scale: fused into the sketch pass (FULL) or the broadcast pass (SAMPLED)
   METIS_CUDA_TRY(cudaMemsetAsync(amax, 0, 64, s));       // amax slots of x, left, right and the condition flag
 
@@ -1712,8 +1716,6 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   if (gram_chol_smem(n_s, q) <= GC_MAX_SMEM) {
     // a short sketch: Gram matrix and factorisation in one CTA; the triangular solves on many CTAs unless the sketch
     // was ill-conditioned, in which case the first kernel has done both passes itself and the second returns at once
-    static bool at_ = false;
-    if (!at_) { METIS_CUDA_TRY(cudaFuncSetAttribute(gram_chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GC_MAX_SMEM)); at_ = true; }
     METIS_CUDA_TRY(metis_launch_pdl((gram_chol_kernel), dim3(1), dim3(GC_THREADS), gram_chol_smem(n_s, q), s, z, (int)n_s, q, linv, invd, cond_flag)); METIS_COUNT_LAUNCH();
     METIS_CUDA_TRY(metis_launch_pdl((apply_chol_kernel), dim3((unsigned)metis_ceil_div(n_s, 8)), dim3(256), (size_t)(0), s, z, n_s, q, linv, invd, (const int*)cond_flag)); METIS_COUNT_LAUNCH();
   } else {
@@ -1746,7 +1748,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       } else {
       dim3 grid((unsigned)metis_ceil_div(cols, PP_COLS), (unsigned)parts);
       const size_t psmem = (size_t)PP_STAGES * (PP_K * PP_XP * 2 + 3 * jp * PP_HP * 2);
-#define METIS_PP(MTV) { static bool at_ = false; if (!at_) { METIS_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<MTV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psmem)); at_ = true; } \
+#define METIS_PP(MTV) { \
         METIS_CUDA_TRY(metis_launch_pdl((project_pipe_kernel<MTV>), grid, dim3(256), psmem, s, x, cols, idx, (int)n_s, q, hsp, ldh, rpp, mp)); }
       switch (mt) {
         case 1: METIS_PP(1); break;

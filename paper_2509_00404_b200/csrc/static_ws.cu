@@ -36,20 +36,17 @@ metis_status_t static_ws_address(int device, void** out) {
 
 }  // namespace
 
-size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k);
-
 extern "C" metis_status_t metis_linear_fwd_static_ws(metis_handle_t h, const metis_operand_t* x, const metis_operand_t* w,
                                                      void* y, int32_t y_dtype, int64_t ldy, metis_stream_t stream) {
   if (!h || !x || !w || !y) return METIS_ERR_INVALID_ARG;
   int current = -1;
   if (cudaGetDevice(&current) != cudaSuccess) return METIS_ERR_CUDA;
   if (current != h->device) return METIS_ERR_INVALID_ARG;          // the handle's device must be the current one
-  const int k = x->k > w->k ? x->k : w->k;
-  const size_t need = (x->k == 0 && w->k == 0) ? 0 : metis_linear_ws_bytes(x->rows, w->rows, k);
-  if (need > STATIC_WS_BYTES) return METIS_ERR_WORKSPACE;          // layer too large for the built-in array
   void* ws = nullptr;
   METIS_TRY(static_ws_address(current, &ws));
   // Nothing in the array has to start at zero: every intermediate the layer reads back is written earlier in
-  // the same call, so the previous call's contents are simply overwritten.
+  // the same call, so the previous call's contents are simply overwritten.  metis_linear_fwd lays its
+  // intermediates out inside the bytes it is given and refuses, before it enqueues anything, a layer whose
+  // intermediates do not fit (METIS_ERR_WORKSPACE); argument and shape errors are reported as usual.
   return metis_linear_fwd(h, x, w, y, y_dtype, ldy, ws, STATIC_WS_BYTES, stream);
 }

@@ -28,9 +28,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: returns false (and records the timeout) instead of spinning forever.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* dev_status, volatile int* dead) {
-  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+// Bounded wait: returns false (and records the timeout) instead of spinning forever.  `limit` = polls before
+// giving up; `dead` is the CTA's shared "somebody gave up" flag, which every waiting role checks now and then so
+// that one expired wait unwinds all of them.
+__device__ __forceinline__ bool mbar_wait_n(uint32_t bar, uint32_t parity, uint32_t* dev_status, volatile int* dead, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (i > 4096) __nanosleep(32);
     if ((i & 1023u) == 1023u && *dead) break;
@@ -38,6 +40,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
   *dead = 1;
   atomicOr(dev_status, METIS_DEV_TIMEOUT);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* dev_status, volatile int* dead) {
+  return mbar_wait_n(bar, parity, dev_status, dead, WAIT_LIMIT);
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 // true in exactly one lane of a fully converged warp

@@ -24,3 +24,20 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionfinish(session, exitstatus):
+    """Writes the audit table of the end-to-end comparisons (tests/gpu_util.check_e2e) to $METIS_PARITY_LOG."""
+    path = os.environ.get("METIS_PARITY_LOG")
+    try:
+        import gpu_util
+    except Exception:
+        return
+    if not path or not gpu_util.E2E_RECORDS:
+        return
+    with open(path, "w") as f:
+        f.write("# case | errors | allowance added to 2e-3 | differing factor blocks / all | plain 2e-3 held\n")
+        for r in gpu_util.E2E_RECORDS:
+            f.write("%s | %s | %.2e | %d/%d | %s\n" % (r["case"], " ".join("%s=%.3e" % kv for kv in r["errors"].items()),
+                                                     r["allowance"], r["differing_blocks"], r["factor_blocks"],
+                                                     "yes" if r["plain_tolerance_held"] else "no"))

@@ -44,6 +44,16 @@ def test_check_kernel_matches_exact_product(ctx, shape):
     assert _case(B, h, *shape, seed=1 + sum(shape), impl=1) < TOL
 
 
+@pytest.mark.parametrize("shape", [(256, 256, 14336), (256, 256, 16384), (128, 256, 16384)])
+def test_longest_contractions_of_the_workloads(ctx, shape):
+    """K = 14336 (FFN down-projection) and K = 16384 (weight gradient at 16384 tokens): the longest FP32 accumulations
+    in tensor memory that the workload list contains, through the two-CTA kernel and the one-CTA kernel."""
+    B, h = ctx
+    err = _case(B, h, *shape, seed=sum(shape), impl=0)
+    print("GEMM on identical codes %dx%dx%d: relative Frobenius error %.3e" % (*shape, err))
+    assert err < TOL
+
+
 def test_bf16_output_and_many_tiles(ctx):
     B, h = ctx
     # more tiles than SMs: exercises the persistent loop, both accumulator buffers and the barrier phase wrap

@@ -19,9 +19,9 @@ def ctx():
     h.close()
 
 
-def _flip_allowance(*pairs):
-    from gpu_util import flip_allowance
-    return flip_allowance(pairs)
+def _check_e2e(case, errors, *pairs, base_tol=TOL):
+    from gpu_util import check_e2e
+    return check_e2e(case, errors, pairs, base_tol)
 
 
 def _oracle_from_gpu_operand(op, k):
@@ -48,7 +48,7 @@ def test_small_config_forward(ctx):
     assert h.device_status() == 0
     xq = olay.quantize_operand(c["x"], 4, 4, osp.MODE_FULL, 1)
     wq = olay.quantize_operand(c["w"], 4, 4, osp.MODE_FULL, 2)
-    assert rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)) < TOL + _flip_allowance((xo, xq), (wo, wq))
+    _check_e2e("small_config_forward_128tok_256to256_k4", {"y": rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq))}, (xo, xq), (wo, wq))
     # composition alone, on the library's own codes: tight
     lx, rxc, _ = _oracle_from_gpu_operand(xo, 4)
     lw, rwc, _ = _oracle_from_gpu_operand(wo, 4)
@@ -73,16 +73,40 @@ def test_forward_and_backward_medium(ctx, k):
     xq = olay.quantize_operand(x, k, p, osp.MODE_SAMPLED, 1)
     wq = olay.quantize_operand(w, k, p, osp.MODE_FULL, 2)
     dq = olay.quantize_operand(d, k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
-    tol = TOL + _flip_allowance((xo, xq), (wo, wq), (do, dq))
-    assert rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)) < tol
-    assert rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)) < tol
-    assert rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq)) < tol
+    _check_e2e("medium_512tok_384to256_k%d" % k,
+               {"y": rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)), "dx": rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)),
+                "dw": rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq))}, (xo, xq), (wo, wq), (do, dq))
     lx, rxc, rxr = _oracle_from_gpu_operand(xo, k)
     lw, rwc, rwr = _oracle_from_gpu_operand(wo, k)
     ld, rdc, rdr = _oracle_from_gpu_operand(do, k)
     assert rel_fro(y.cpu().numpy(), (lx + rxc) @ (lw + rwc).T) < 2e-5
     assert rel_fro(dx.cpu().numpy(), (ld + rdc) @ (lw + rwr)) < 2e-5
     assert rel_fro(dw.cpu().numpy(), (ld + rdr).T @ (lx + rxr)) < 2e-5
+
+
+@pytest.mark.parametrize("k", [0, 8])
+def test_layer_on_the_oracles_own_bytes(ctx, k):
+    """No discontinuity in the way: the ORACLE's codes, scale bytes, tensor scales and singular values are uploaded
+    into the library's operands, so both sides multiply exactly the same quantized tensors.  Eq. 2, Eq. 3 and the
+    weight gradient must then agree with the oracle's float64 evaluation to FP32-accumulation accuracy, with no
+    allowance of any kind."""
+    from gpu_util import rel_fro, operand_from_oracle
+    B, h = ctx
+    l, m, n, p = 512, 384, 256, 8 if k else 0
+    x, _ = synth.llama_like(l, m, 1.0, 51, rank=8)
+    w, _ = synth.llama_like(n, m, 0.02, 52, rank=8)
+    d, _ = synth.llama_like(l, n, 1e-4, 53, rank=8)
+    xq = olay.quantize_operand(x, k, p, osp.MODE_SAMPLED, 1)
+    wq = olay.quantize_operand(w, k, p, osp.MODE_FULL, 2)
+    dq = olay.quantize_operand(d, k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
+    xo, wo, do = (operand_from_oracle(B, q) for q in (xq, wq, dq))
+    y = h.linear_fwd(xo, wo)
+    dx, dw = h.linear_bwd(do, xo, wo)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    assert rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)) < 2e-5
+    assert rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)) < 2e-5
+    assert rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq)) < 2e-5
 
 
 @pytest.mark.parametrize("dw_dtype", [torch.float32, torch.bfloat16])
@@ -115,11 +139,10 @@ def test_factor_gradients(ctx, dw_dtype):
     wq = olay.quantize_operand(w, k, p, osp.MODE_FULL, 2)
     dq = olay.quantize_operand(d, k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
     du, ds, dv = olay.factor_grads(olay.linear_wgrad(dq, xq), wq)
-    tol = TOL if dw_dtype == torch.float32 else 3 * TOL                           # a BF16 dw carries 2^-9 per entry
-    tol += _flip_allowance((xo, xq), (wo, wq), (do, dq))
-    assert rel_fro(d_right.cpu().numpy().T, du) < tol
-    assert rel_fro(d_left.cpu().numpy().T, dv) < tol
-    assert rel_fro(d_sigma.cpu().numpy(), ds) < tol
+    base = TOL if dw_dtype == torch.float32 else 3 * TOL                          # a BF16 dw carries 2^-9 per entry
+    _check_e2e("factor_gradients_256tok_448to192_k12_dw_%s" % ("fp32" if dw_dtype == torch.float32 else "bf16"),
+               {"dU": rel_fro(d_right.cpu().numpy().T, du), "dV": rel_fro(d_left.cpu().numpy().T, dv),
+                "dS": rel_fro(d_sigma.cpu().numpy(), ds)}, (xo, xq), (wo, wq), (do, dq), base_tol=base)
 
 
 def test_factor_gradients_need_the_weight_gradient(ctx):
@@ -156,10 +179,9 @@ def test_rank_and_oversampling_range(ctx, kp):
     dq = olay.quantize_operand(d, k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
     for op, q in ((xo, xq), (wo, wq), (do, dq)):
         assert np.max(np.abs(op.sigma.cpu().numpy()[:k] - q.sigma) / q.sigma) < 1e-3
-    tol = TOL + _flip_allowance((xo, xq), (wo, wq), (do, dq))
-    assert rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)) < tol
-    assert rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)) < tol
-    assert rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq)) < tol
+    _check_e2e("rank_range_512tok_768to640_k%d_p%d" % (k, p),
+               {"y": rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)), "dx": rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)),
+                "dw": rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq))}, (xo, xq), (wo, wq), (do, dq))
 
 
 def test_ragged_layer_through_the_two_cta_gemm(ctx):
@@ -187,10 +209,9 @@ def test_ragged_layer_through_the_two_cta_gemm(ctx):
     xq = olay.quantize_operand(x, k, p, osp.MODE_SAMPLED, 1)
     wq = olay.quantize_operand(w, k, p, osp.MODE_FULL, 2)
     dq = olay.quantize_operand(d, k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
-    tol = TOL + _flip_allowance((xo, xq), (wo, wq), (do, dq))
-    assert rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)) < tol
-    assert rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)) < tol
-    assert rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq)) < tol
+    _check_e2e("ragged_320tok_448to320_k8",
+               {"y": rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)), "dx": rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)),
+                "dw": rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq))}, (xo, xq), (wo, wq), (do, dq))
 
 
 def test_bf16_output(ctx):

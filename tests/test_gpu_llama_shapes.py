@@ -32,7 +32,7 @@ CASES = [
 
 @pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
 def test_layer_on_sampled_outputs(case):
-    from gpu_util import rel_fro, nv_to_numpy, flip_allowance
+    from gpu_util import rel_fro, nv_to_numpy, check_e2e
     from paper_2509_00404_b200 import binding as B
     _, l, m, n, k, p, rank, whole = case
     x, _ = synth.llama_like(l, m, 1.0, 3000, rank=rank)
@@ -63,7 +63,7 @@ def test_layer_on_sampled_outputs(case):
     dq = PartialOperand(d, k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
     for s_gpu, q in zip(sig, (xq, wq, dq)):
         assert np.max(np.abs(s_gpu - q.sigma) / q.sigma) < 1e-3
-    tol = TOL + (flip_allowance(list(zip(factors, (xq, wq, dq)))) if k else 0.0)
-    assert rel_fro(y_s, xq.dense_by_cols(rl) @ wq.dense_by_cols(rn).T) < tol
-    assert rel_fro(dx_s, dq.dense_by_cols(rl) @ wq.dense_by_rows(cm)) < tol
-    assert rel_fro(dw_s, dq.dense_by_rows(rn).T @ xq.dense_by_rows(cm)) < tol
+    check_e2e(case[0], {"y": rel_fro(y_s, xq.dense_by_cols(rl) @ wq.dense_by_cols(rn).T),
+                        "dx": rel_fro(dx_s, dq.dense_by_cols(rl) @ wq.dense_by_rows(cm)),
+                        "dw": rel_fro(dw_s, dq.dense_by_rows(rn).T @ xq.dense_by_rows(cm))},
+              list(zip(factors, (xq, wq, dq))) if k else [], TOL)

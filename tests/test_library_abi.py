@@ -63,3 +63,16 @@ def test_tiled_scale_layout_helper_matches_the_header_formula():
     lin = t.linear_scales().numpy()
     want = (np.arange(rows)[:, None] * 7 + np.arange(nb)[None, :] * 3) % 251
     assert np.array_equal(lin, want)
+
+
+def test_launch_helpers_keep_no_process_wide_state():
+    """Kernel attributes and occupancy figures belong to a device; a `static` flag or counter inside a launch helper
+    would be shared by every device and thread of the process.  They live in the context (set in metis_create)."""
+    csrc = os.path.join(ROOT, "paper_2509_00404_b200", "csrc")
+    bad = []
+    for name in sorted(os.listdir(csrc)):
+        text = open(os.path.join(csrc, name)).read()
+        for i, line in enumerate(text.splitlines(), 1):
+            if re.match(r"\s+static\s+(bool|int|unsigned|size_t|long)\b", line) and "(" not in line.split("=")[0]:
+                bad.append("%s:%d: %s" % (name, i, line.strip()))
+    assert not bad, bad

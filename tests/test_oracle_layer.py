@@ -58,20 +58,83 @@ def test_dgrad_equals_the_four_terms_of_eq3_and_wgrad_its_two():
     assert np.allclose(layer.linear_wgrad(dq, xq), two.T, rtol=1e-12, atol=1e-12)
 
 
-def test_exactly_representable_inputs_give_the_exact_product():
-    rng = np.random.default_rng(0)
+def _representable(rng, rows, cols):
+    """Values that NVFP4 with an own-amax tensor scale stores without error: E2M1 grid values times a power-of-two
+    block scale, a +-6 in every block (so the block scale amax_b/(6 s_T) is that power of two exactly), and one
+    element 6 * 448 so that the tensor scale amax/2688 is exactly 1."""
     grid = np.array([0, .5, 1, 1.5, 2, 3, 4, 6])
-    def rep(rows, cols):
-        m = rng.choice(grid, (rows, cols)) * rng.choice([-1.0, 1.0], (rows, cols))
-        m[:, ::16] = 6.0                                        # every block has amax 6 -> block scale 2^e exactly
-        return (m * 2.0 ** rng.integers(-2, 3, (rows, 1))).astype(F32)
-    x, w = rep(32, 64), rep(48, 64)
-    s_t = F32(2.0 ** -4)
-    cx = nvfp4.quantize(x, tensor_scale=s_t)
-    cw = nvfp4.quantize(w, tensor_scale=s_t)
-    assert np.array_equal(nvfp4.dequantize(*cx), x) and np.array_equal(nvfp4.dequantize(*cw), w)
+    m = rng.choice(grid, (rows, cols)) * rng.choice([-1.0, 1.0], (rows, cols))
+    m[:, ::16] = 6.0 * rng.choice([-1.0, 1.0], (rows, cols // 16))
+    e = rng.integers(-6, 9, (rows, cols // 16))                    # block scales 2^-6 .. 2^8: normal E4M3 numbers
+    m = m * np.repeat(2.0 ** e, 16, axis=1)
+    m[0, :16] = m[0, :16] / 2.0 ** e[0, 0] * 448.0                 # first block: scale 448, its 6 becomes amax = 2688
+    return m.astype(F32)
+
+
+def test_exactly_representable_inputs_give_the_exact_product():
+    """Representable inputs, plain NVFP4 (k = 0): every piece is stored without error, so Eq. 2, Eq. 3 and the weight
+    gradient of the layer must equal the exact float64 products of the inputs - not merely be close to them."""
+    rng = np.random.default_rng(0)
+    x, w, d = _representable(rng, 32, 64), _representable(rng, 48, 64), _representable(rng, 32, 48)
     xq = layer.quantize_operand(x, 0, 0, split.MODE_FULL, 0)
-    assert np.allclose(xq.res_by_cols, x, rtol=2e-2)            # own-amax tensor scale: close, not exact
+    wq = layer.quantize_operand(w, 0, 0, split.MODE_FULL, 0)
+    dq = layer.quantize_operand(d, 0, 0, split.MODE_FULL, 0)
+    for q, t in ((xq, x), (wq, w), (dq, d)):
+        assert q.raw["res_by_cols"][2] == F32(1.0)
+        assert np.array_equal(q.res_by_cols, t.astype(np.float64))
+    x64, w64, d64 = (t.astype(np.float64) for t in (x, w, d))
+    assert np.array_equal(layer.linear_fwd(xq, wq), x64 @ w64.T)
+    # the products that contract over rows use blocks along the rows: the transpose of a representable matrix is
+    # representable in that orientation
+    xr, dr, wr = _representable(rng, 64, 32).T.copy(), _representable(rng, 48, 32).T.copy(), _representable(rng, 64, 48).T.copy()
+    xrq = layer.quantize_operand(xr, 0, 0, split.MODE_FULL, 0)
+    drq = layer.quantize_operand(dr, 0, 0, split.MODE_FULL, 0)
+    wrq = layer.quantize_operand(wr, 0, 0, split.MODE_FULL, 0)
+    for q, t in ((xrq, xr), (drq, dr), (wrq, wr)):
+        assert np.array_equal(q.res_by_rows, t.astype(np.float64))
+    assert np.array_equal(layer.linear_wgrad(drq, xrq), dr.astype(np.float64).T @ xr.astype(np.float64))
+    assert np.array_equal(layer.linear_dgrad(dq, wrq), d64 @ wr.astype(np.float64))
+
+
+def test_representable_low_rank_inputs_give_the_exact_product_with_a_split():
+    """k > 0: a rank-2 operand whose singular vectors have entries +-1/8 (scaled Hadamard columns) is split into
+    factors that NVFP4 stores without error (every block is +-1/8 throughout: code 6 under scale 448), the residual
+    is zero to rounding, and the split-FP4 forward product equals the exact product to float32-scale accuracy."""
+    h2 = np.array([[1.0, 1.0], [1.0, -1.0]])
+    had = h2
+    for _ in range(5):
+        had = np.kron(had, h2)                                      # 64 x 64 Hadamard matrix
+    u, v = had[:, [3, 17]] / 8.0, had[:, [5, 40]] / 8.0             # orthonormal columns with entries +-1/8
+    x = ((u * np.array([8.0, 2.0])) @ v.T).astype(F32)              # entries in {+-1/8 +- 1/32}: exact in bf16
+    w = ((had[:, [9, 33]] / 8.0 * np.array([4.0, 1.0])) @ (had[:, [5, 21]] / 8.0).T).astype(F32)
+    xq = layer.quantize_operand(x, 2, 0, split.MODE_FULL, 3)
+    wq = layer.quantize_operand(w, 2, 0, split.MODE_FULL, 4)
+    assert np.allclose(xq.sigma, [8.0, 2.0], rtol=1e-12) and np.allclose(wq.sigma, [4.0, 1.0], rtol=1e-12)
+    assert np.allclose(np.abs(xq.left_q), 0.125, rtol=1e-6) and np.allclose(np.abs(xq.right_q), 0.125, rtol=1e-6)
+    assert np.abs(xq.res_by_cols).max() < 1e-12
+    want = x.astype(np.float64) @ w.astype(np.float64).T
+    got = layer.linear_fwd(xq, wq)
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) < 1e-6
+
+
+def test_metrics_on_cases_with_known_answers():
+    """subspace_alignment: identical bases 1, orthogonal bases 0, one shared direction of two 1/2.
+    spectral_fidelity on diagonal matrices: singular values are the diagonal, vectors the unit vectors."""
+    e = np.eye(6)
+    assert np.isclose(metrics.subspace_alignment(e[:, :2], e[:, :2]), 1.0)
+    assert np.isclose(metrics.subspace_alignment(e[:, :2], e[:, 2:4]), 0.0)
+    assert np.isclose(metrics.subspace_alignment(e[:, :2], e[:, 1:3]), 0.5)
+    rot = np.array([[np.cos(0.3), -np.sin(0.3)], [np.sin(0.3), np.cos(0.3)]])
+    assert np.isclose(metrics.subspace_alignment(e[:, :2], e[:, :2] @ rot), 1.0)      # a basis change inside the span
+    ref = np.diag([5.0, 3.0, 2.0, 1.0])
+    rs, cos = metrics.spectral_fidelity(ref, ref)
+    assert np.allclose(rs, 0.0) and np.allclose(cos, 1.0)
+    rs, cos = metrics.spectral_fidelity(ref, np.diag([5.5, 2.7, 2.0, 1.0]))
+    assert np.allclose(rs, [0.1, 0.1, 0.0, 0.0]) and np.allclose(cos, 1.0)
+    swapped = ref[[1, 0, 2, 3]]                                      # rows 0 and 1 exchanged: left vectors e2, e1, e3, e4
+    rs, cos = metrics.spectral_fidelity(ref, swapped)
+    assert np.allclose(rs, 0.0) and np.allclose(cos, [0.0, 0.0, 1.0, 1.0])
+    assert np.isclose(metrics.rel_fro(np.array([3.0, 4.0]), np.array([0.0, 4.0])), 0.75)
 
 
 def test_residual_uses_the_source_tensor_scale_and_unquantized_factors():
