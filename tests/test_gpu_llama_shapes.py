@@ -16,7 +16,7 @@ from paper_2509_00404_b200 import synth
 pytestmark = pytest.mark.gpu
 
 TOL = 2e-3
-N_SAMPLE = 64
+N_SAMPLE = 256        # sampled rows and columns per output: a 64 x 64 sample is dominated by whichever re-rounded factor block it happens to contain
 
 CASES = [
     # id, tokens, in, out, k, p, planted rank, compare the whole output
