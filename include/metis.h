@@ -186,10 +186,13 @@ metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dty
  * scale amax(x)/2688 of the SOURCE tensor; factors with their own.  `residual_axes` selects which
  * residual orientations are produced.  `residual_dense` (optional, rows x cols FP32) receives the
  * unquantized residual the quantizer saw.  k == 0 quantizes x itself.
- * Requires rows % 16 == 0, cols % 64 == 0 (tiled scales), k % 4 == 0, k <= 64 and k + p <= 72 (the
- * orthonormalisation and the two small eigen-solvers each run in one CTA's shared memory; larger
- * ranks are refused with METIS_ERR_SHAPE).
- * Workspace: metis_workspace_bytes(1, rows, cols, k, p). */
+ * Requires rows % 16 == 0, cols % 64 == 0 (tiled scales), k % 4 == 0, k <= 256 and k + p <= 272.
+ * Up to k = 64 and k + p = 72 the orthonormalisation and the two small eigen-solvers each run in one CTA's
+ * shared memory; above that (the 1.5 % rank of an 8192-wide layer is 128) they run on FP64 kernels tiled over the
+ * rank and on an eight-CTA cluster, which additionally needs rows % 64 == 0.  Larger ranks are refused with
+ * METIS_ERR_SHAPE.
+ * Workspace: metis_workspace_bytes(1, rows, cols, k, p) (for the wide ranks: sized for the default sample count;
+ * a larger n_sample may need more and is then refused with METIS_ERR_WORKSPACE). */
 metis_status_t metis_split(metis_handle_t h, const void* x, int64_t rows, int64_t cols, int32_t k, int32_t p,
                            int32_t sketch, int64_t n_sample, uint64_t seed, int32_t rounding,
                            int32_t residual_axes, metis_operand_t* out, float* residual_dense,

@@ -141,6 +141,85 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
   }
 }
 
+// The same finishing step for ranks above 64 (up to 256 per operand), in two kernels.  First the FP32 operands:
+// one warp per row, the k_a x k_b matrix P staged through shared memory in slabs of 32 rows shared by the CTA's
+// eight rows.
+constexpr int LW_MAXK = 256;
+__global__ void __launch_bounds__(256)
+lowrank_finish_wide_kernel(int64_t M, int64_t N, int ka, int kb,
+                           const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts, const float* sa,
+                           const uint8_t* fob_codes, const uint8_t* fob_sf, int fob_layout, const float* fob_ts, const float* sb,
+                           const float* __restrict__ pm, float* __restrict__ lcat, float* __restrict__ rcat) {
+  __shared__ float ps[32][LW_MAXK];
+  __shared__ float fa[8][LW_MAXK];
+  metis_pdl_wait();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int kc = ka + kb;
+  const int64_t i = (int64_t)blockIdx.x * 8 + warp;
+  const float tsa = ka ? *foa_ts : 0.0f, tsb = kb ? *fob_ts : 0.0f;
+  if (i < M)
+    for (int u = lane; u < ka; u += 32) {
+      const float v = deq_of(foa_codes[(int64_t)u * (M / 2) + i / 2], foa_sf[metis_sf_offset(u, i / 16, M / 16, foa_layout)], i) * tsa * sa[u];
+      fa[warp][u] = v;
+      lcat[i * kc + kb + u] = v;
+    }
+  if (i < N)
+    for (int t = lane; t < kb; t += 32)
+      rcat[i * kc + t] = deq_of(fob_codes[(int64_t)t * (N / 2) + i / 2], fob_sf[metis_sf_offset(t, i / 16, N / 16, fob_layout)], i) * tsb;
+  float acc[LW_MAXK / 32];
+#pragma unroll
+  for (int j = 0; j < LW_MAXK / 32; ++j) { const int t = lane + 32 * j; acc[j] = (i < M && t < kb) ? lcat[i * kc + t] : 0.0f; }
+  for (int u0 = 0; u0 < ka; u0 += 32) {
+    __syncthreads();
+    for (int o = tid; o < 32 * kb; o += 256) { const int uu = o / kb, t = o % kb; ps[uu][t] = u0 + uu < ka ? pm[(int64_t)(u0 + uu) * kb + t] : 0.0f; }
+    __syncthreads();
+    if (i < M) {
+      const int nu = min(32, ka - u0);
+      for (int uu = 0; uu < nu; ++uu) {
+        const float f = fa[warp][u0 + uu];
+#pragma unroll
+        for (int j = 0; j < LW_MAXK / 32; ++j) { const int t = lane + 32 * j; if (t < kb) acc[j] = fmaf(f, ps[uu][t], acc[j]); }
+      }
+    }
+  }
+  if (i < M) {
+#pragma unroll
+    for (int j = 0; j < LW_MAXK / 32; ++j) { const int t = lane + 32 * j; if (t < kb) lcat[i * kc + t] = acc[j] * sb[t]; }
+  }
+}
+
+// Then the BF16 operands of the in-accumulator correction from the finished FP32 ones:
+// Lx = [Lh | Lh | Ll] / alpha,  Rx = [Rh | Rl | Rh], zero padded to kx columns.  One thread per (row, column).
+__global__ void __launch_bounds__(256)
+lowrank_bf16_kernel(int64_t M, int64_t N, int kc, int kx, const float* __restrict__ lcat, const float* __restrict__ rcat,
+                    __nv_bfloat16* __restrict__ lx, __nv_bfloat16* __restrict__ rx, const float* res_a_ts, const float* res_b_ts) {
+  metis_pdl_wait();
+  const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  const int64_t mx = M > N ? M : N;
+  if (idx >= mx * kx) return;
+  const int64_t i = idx / kx;
+  const int c = (int)(idx % kx), seg = c / kc, t = c - seg * kc;
+  const float inv_alpha = 1.0f / ((*res_a_ts) * (*res_b_ts));
+  if (i < M) {
+    float out = 0.0f;
+    if (seg < 3) {
+      const float v = lcat[i * kc + t] * inv_alpha;
+      const float h = __bfloat162float(__float2bfloat16_rn(v));
+      out = seg == 2 ? v - h : h;
+    }
+    lx[i * kx + c] = __float2bfloat16_rn(out);
+  }
+  if (i < N) {
+    float out = 0.0f;
+    if (seg < 3) {
+      const float v = rcat[i * kc + t];
+      const float h = __bfloat162float(__float2bfloat16_rn(v));
+      out = seg == 1 ? v - h : h;
+    }
+    rx[i * kx + c] = __float2bfloat16_rn(out);
+  }
+}
+
 // out = y0 + Lcat Rcat^T, 64 x 64 tile per CTA
 __global__ void __launch_bounds__(256)
 rank_update_kernel(const float* __restrict__ y0, int64_t M, int64_t N, int kc, const float* __restrict__ lcat,
@@ -192,10 +271,11 @@ rank_update_kernel(const float* __restrict__ y0, int64_t M, int64_t N, int kc, c
 constexpr int FG_ROWS = 32, FG_CHUNK = 32;
 template <int KT, bool TRANS>                           // KT = ceil(k / 8) outputs per thread
 __global__ void __launch_bounds__(256)
-factor_grad_kernel(const void* __restrict__ gsrc, int g_dtype, int64_t ldg, int64_t n_r, int64_t n_c, int k,
+factor_grad_kernel(const void* __restrict__ gsrc, int g_dtype, int64_t ldg, int64_t n_r, int64_t n_c, int k, int t0, int k_all,
                    const uint8_t* f_codes, const uint8_t* f_sf, int f_layout, const float* f_ts,
                    const uint8_t* o_codes, const uint8_t* o_sf, int o_layout, const float* o_ts,
                    const float* __restrict__ sigma, float* __restrict__ out, float* __restrict__ ds_part) {
+  // factor vectors t0 .. t0 + k - 1 of k_all (a launch handles at most 64 of them)
   __shared__ float gs[FG_ROWS][FG_CHUNK + 1];
   __shared__ __align__(16) float fs[FG_CHUNK][8 * KT + 4];
   __shared__ float red[8][8 * KT];
@@ -221,7 +301,7 @@ factor_grad_kernel(const void* __restrict__ gsrc, int g_dtype, int64_t ldg, int6
     }
     for (int o = tid; o < FG_CHUNK * 8 * KT; o += 256) {
       const int t = o >> 5, cc = o & 31;
-      fs[cc][t] = (t < k && c0 + cc < n_c) ? deq_at(f_codes, f_sf, f_layout, n_c, t, c0 + cc) : 0.0f;
+      fs[cc][t] = (t < k && c0 + cc < n_c) ? deq_at(f_codes, f_sf, f_layout, n_c, t0 + t, c0 + cc) : 0.0f;
     }
     __syncthreads();
 #pragma unroll 8
@@ -237,7 +317,7 @@ factor_grad_kernel(const void* __restrict__ gsrc, int g_dtype, int64_t ldg, int6
   for (int j = 0; j < KT; ++j) {
     const int t = tg * KT + j;
     acc[j] *= fts;
-    if (t < k && gr < n_r) out[(int64_t)t * n_r + gr] = acc[j] * sigma[t];
+    if (t < k && gr < n_r) out[(int64_t)(t0 + t) * n_r + gr] = acc[j] * sigma[t0 + t];
   }
   if (ds_part != nullptr) {
     const float ots = *o_ts;
@@ -245,7 +325,7 @@ factor_grad_kernel(const void* __restrict__ gsrc, int g_dtype, int64_t ldg, int6
 #pragma unroll
     for (int j = 0; j < KT; ++j) {
       const int t = tg * KT + j;
-      float v = (t < k && gr < n_r) ? acc[j] * deq_at(o_codes, o_sf, o_layout, n_r, t, gr) * ots : 0.0f;
+      float v = (t < k && gr < n_r) ? acc[j] * deq_at(o_codes, o_sf, o_layout, n_r, t0 + t, gr) * ots : 0.0f;
       v += __shfl_xor_sync(0xFFFFFFFFu, v, 8);
       v += __shfl_xor_sync(0xFFFFFFFFu, v, 16);
       if ((tid & 31) < 8) red[tid >> 5][t] = v;
@@ -255,7 +335,7 @@ factor_grad_kernel(const void* __restrict__ gsrc, int g_dtype, int64_t ldg, int6
       float v = 0.0f;
 #pragma unroll
       for (int w = 0; w < 8; ++w) v += red[w][tid];
-      ds_part[(int64_t)blockIdx.x * k + tid] = v;
+      ds_part[(int64_t)blockIdx.x * k_all + t0 + tid] = v;
     }
   }
 }
@@ -273,22 +353,25 @@ template <bool TRANS>
 metis_status_t launch_factor_grad(cudaStream_t s, const void* g, int g_dtype, int64_t ldg, int64_t n_r, int64_t n_c, int k,
                                   const metis_nvfp4_t* f, const metis_nvfp4_t* o, const float* sigma, float* out, float* ds_part) {
   const unsigned grid = (unsigned)metis_ceil_div(n_r, FG_ROWS);
-#define METIS_FG(KT) factor_grad_kernel<KT, TRANS><<<grid, 256, 0, s>>>(g, g_dtype, ldg, n_r, n_c, k, f->codes, f->scales, f->sf_layout, \
+#define METIS_FG(KT) factor_grad_kernel<KT, TRANS><<<grid, 256, 0, s>>>(g, g_dtype, ldg, n_r, n_c, kg, t0, k, f->codes, f->scales, f->sf_layout, \
     f->tensor_scale, o ? o->codes : nullptr, o ? o->scales : nullptr, o ? o->sf_layout : 0, o ? o->tensor_scale : nullptr, sigma, out, ds_part)
-  switch ((k + 7) / 8) {
-    case 1: METIS_FG(1); break; case 2: METIS_FG(2); break; case 3: METIS_FG(3); break; case 4: METIS_FG(4); break;
-    case 5: METIS_FG(5); break; case 6: METIS_FG(6); break; case 7: METIS_FG(7); break; case 8: METIS_FG(8); break;
-    default: return METIS_ERR_SHAPE;
+  for (int t0 = 0; t0 < k; t0 += 64) {                  // at most 64 factor vectors per pass over the gradient
+    const int kg = k - t0 < 64 ? k - t0 : 64;
+    switch ((kg + 7) / 8) {
+      case 1: METIS_FG(1); break; case 2: METIS_FG(2); break; case 3: METIS_FG(3); break; case 4: METIS_FG(4); break;
+      case 5: METIS_FG(5); break; case 6: METIS_FG(6); break; case 7: METIS_FG(7); break; case 8: METIS_FG(8); break;
+      default: return METIS_ERR_SHAPE;
+    }
+    METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(cudaGetLastError());
   }
 #undef METIS_FG
-  METIS_COUNT_LAUNCH();
-  METIS_CUDA_TRY(cudaGetLastError());
   return METIS_OK;
 }
 
 // the host-side checks of factor_grads, callable before anything is enqueued
 metis_status_t factor_grads_check(const metis_operand_t* w, const float* d_left, const float* d_sigma, const void* ws, size_t ws_bytes) {
-  if (!w || w->k <= 0 || w->k > 64 || !w->sigma) return METIS_ERR_SHAPE;
+  if (!w || w->k <= 0 || w->k > LW_MAXK || !w->sigma) return METIS_ERR_SHAPE;
   const metis_nvfp4_t *lq = &w->left_q, *rq = &w->right_q;
   if (!lq->codes || !rq->codes || lq->k_len != w->rows || rq->k_len != w->cols) return METIS_ERR_SHAPE;
   if (d_sigma && !d_left) return METIS_ERR_INVALID_ARG;          // the sigma partials ride on the d_left pass
@@ -300,7 +383,7 @@ metis_status_t factor_grads_check(const metis_operand_t* w, const float* d_left,
 metis_status_t factor_grads(metis_context* ctx, const void* dw, int dw_dtype, int64_t lddw, const metis_operand_t* w,
                             float* d_left, float* d_sigma, float* d_right, void* ws, size_t ws_bytes, cudaStream_t s) {
   (void)ctx;
-  if (!w || w->k <= 0 || w->k > 64 || !w->sigma) return METIS_ERR_SHAPE;
+  if (!w || w->k <= 0 || w->k > LW_MAXK || !w->sigma) return METIS_ERR_SHAPE;
   const int64_t n = w->rows, m = w->cols;
   const metis_nvfp4_t *lq = &w->left_q, *rq = &w->right_q;
   if (!lq->codes || !rq->codes || lq->k_len != n || rq->k_len != m) return METIS_ERR_SHAPE;
@@ -313,7 +396,7 @@ metis_status_t factor_grads(metis_context* ctx, const void* dw, int dw_dtype, in
     METIS_TRY(launch_factor_grad<false>(s, dw, dw_dtype, lddw, n, m, w->k, rq, d_sigma ? lq : nullptr, w->sigma, d_left,
                                         d_sigma ? part : nullptr));
     if (d_sigma) {
-      factor_grad_sigma_kernel<<<1, 64, 0, s>>>(part, (int)n_part, w->k, d_sigma); METIS_COUNT_LAUNCH();
+      factor_grad_sigma_kernel<<<1, 256, 0, s>>>(part, (int)n_part, w->k, d_sigma); METIS_COUNT_LAUNCH();
       METIS_CUDA_TRY(cudaGetLastError());
     }
   }
@@ -358,15 +441,16 @@ metis_status_t make_plan(const Side& a, const Side& b, void* ws, size_t ws_bytes
   if (pl->kc == 0) return METIS_OK;
   const int64_t M = pl->M, N = pl->N, K = pl->K;
   const int ka = a.k, kb = b.k, kc = pl->kc;
-  if (ka > 64 || kb > 64) return METIS_ERR_SHAPE;
+  if (ka > LW_MAXK || kb > LW_MAXK) return METIS_ERR_SHAPE;
   if (ka) { METIS_TRY(check_nvfp4(a.fc)); METIS_TRY(check_nvfp4(a.fo)); if (a.fc->k_len != K || a.fo->k_len != M || !a.sigma) return METIS_ERR_SHAPE; }
   if (kb) { METIS_TRY(check_nvfp4(b.fc)); METIS_TRY(check_nvfp4(b.fo)); if (b.fc->k_len != K || b.fo->k_len != N || !b.sigma) return METIS_ERR_SHAPE; }
   unsigned char* w = reinterpret_cast<unsigned char*>(ws);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
   pl->fuse = metis_gemm_tc_can_fuse(a.res, b.res);
+  if (!pl->fuse && kc > 128) return METIS_ERR_SHAPE;    // layers below 256 rows hold the update operands in shared memory
   pl->kx = (3 * kc + 63) / 64 * 64;
-  const size_t o_pm = take(sizeof(float) * 64 * 64), o_l = take(sizeof(float) * M * kc), o_r = take(sizeof(float) * N * kc);
+  const size_t o_pm = take(sizeof(float) * (size_t)(ka * kb > 64 * 64 ? ka * kb : 64 * 64)), o_l = take(sizeof(float) * M * kc), o_r = take(sizeof(float) * N * kc);
   const size_t o_lx = pl->fuse ? take(sizeof(__nv_bfloat16) * M * pl->kx) : 0, o_rx = pl->fuse ? take(sizeof(__nv_bfloat16) * N * pl->kx) : 0;
   const size_t o_y0 = pl->fuse ? 0 : take(sizeof(float) * M * N);
   pl->bytes = off;
@@ -394,6 +478,18 @@ metis_status_t split_gemm_prologue(metis_context* ctx, const Side& a, const Side
   METIS_TRY(metis_join(ctx, s, side0));
   METIS_TRY(metis_join(ctx, s, side0 + 1));
   const int64_t mx = M > N ? M : N;
+  if (ka > 64 || kb > 64) {
+    METIS_CUDA_TRY(metis_launch_pdl(lowrank_finish_wide_kernel, dim3((unsigned)metis_ceil_div(mx, 8)), dim3(256), 0, s,
+        M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
+        ka ? a.fo->tensor_scale : nullptr, a.sigma, kb ? b.fo->codes : nullptr, kb ? b.fo->scales : nullptr,
+        kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, (const float*)pl.pm, pl.lcat, pl.rcat)); METIS_COUNT_LAUNCH();
+    if (pl.lx != nullptr) {
+      METIS_CUDA_TRY(metis_launch_pdl(lowrank_bf16_kernel, dim3((unsigned)metis_ceil_div(mx * pl.kx, 256)), dim3(256), 0, s, M, N, kc, pl.kx,
+          (const float*)pl.lcat, (const float*)pl.rcat, pl.lx, pl.rx, (const float*)a.res->tensor_scale, (const float*)b.res->tensor_scale)); METIS_COUNT_LAUNCH();
+    }
+    METIS_CUDA_TRY(cudaGetLastError());
+    return METIS_OK;
+  }
   METIS_CUDA_TRY(metis_launch_pdl(lowrank_finish_kernel, dim3((unsigned)metis_ceil_div(mx, 8)), dim3(256), 0, s,
       M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
       ka ? a.fo->tensor_scale : nullptr, a.sigma, kb ? b.fo->codes : nullptr, kb ? b.fo->scales : nullptr,
@@ -437,10 +533,11 @@ size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k) {
   const int kc = 2 * k;
   const int kx = (3 * kc + 63) / 64 * 64;
   // sized for either path: FP32 staging of the main product (small shapes) or the BF16 correction operands
-  return align256(sizeof(float) * M * N) + align256(sizeof(float) * 64 * 64) +
+  const size_t pm_elems = (size_t)k * k > 64 * 64 ? (size_t)k * k : 64 * 64;
+  return align256(sizeof(float) * M * N) + align256(sizeof(float) * pm_elems) +
          align256(sizeof(float) * M * (kc ? kc : 1)) + align256(sizeof(float) * N * (kc ? kc : 1)) +
          align256(sizeof(__nv_bfloat16) * M * (kx ? kx : 1)) + align256(sizeof(__nv_bfloat16) * N * (kx ? kx : 1)) +
-         align256(sizeof(float) * 64 * (size_t)metis_ceil_div(M > N ? M : N, FG_ROWS));     // partials of the sigma gradient
+         align256(sizeof(float) * (size_t)(k > 64 ? k : 64) * (size_t)metis_ceil_div(M > N ? M : N, FG_ROWS));     // partials of the sigma gradient
 }
 
 metis_status_t metis_linear_fwd(metis_handle_t h, const metis_operand_t* x, const metis_operand_t* w, void* y,

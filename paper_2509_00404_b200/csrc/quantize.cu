@@ -358,7 +358,7 @@ metis_status_t metis_launch_quantize_factors(const float* left, int64_t rows, co
                                              uint64_t seed, const float* amax_left, const float* amax_right,
                                              const metis_nvfp4_t* lq, const metis_nvfp4_t* rq, cudaStream_t s) {
   using namespace metis_qt;
-  if (k <= 0 || k > 64 || rows % 16 || cols % 16) return METIS_ERR_SHAPE;
+  if (k <= 0 || k > 256 || rows % 16 || cols % 16) return METIS_ERR_SHAPE;
   RowblocksJob a{}, b{};
   a.x = left; a.ld = rows; a.tscale_src = amax_left; a.ts_out = lq->tensor_scale;
   a.p.rows = k; a.p.cols = rows; a.p.rounding = rounding; a.p.seed = seed; a.p.stream_id = METIS_STREAM_LEFT;

@@ -6,6 +6,7 @@
 //   FP64) -> right basis B -> [SAMPLED: C = x B, Rayleigh-Ritz on C^T C] -> residual R = x - C B^T fused
 //   with the NVFP4 quantizer in both block orientations -> factor rotation, sign fix, factor quantization.
 #include "quant_tile.cuh"
+#include "bigrank.cuh"
 
 metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const float* coef, int k, int kp,
                                         const metis_qt::QuantParams& qp, const float* amax_src, float* ts_out0, float* ts_out1,
@@ -741,8 +742,10 @@ __device__ __forceinline__ void split3(float x, float y, uint32_t& hi, uint32_t&
 }
 
 // BF16 splits of the right basis in both operand orientations:
-//   bs[t][j][col]  (col contiguous; B operand of C = x B, contraction over col)
-//   bt[t][col][j]  (j contiguous, padded to kp; B operand of C B^T, contraction over j)
+//   bs[t][j][col]  (col contiguous; B operand of C = x B, contraction over col); with more than 64 vectors the
+//                  layout is by groups of 64 vectors, bs[group][t][j in group][col], so that the three terms of a
+//                  group are one contiguous matrix (one launch of the coefficient kernel per group)
+//   bt[t][col][j]  (j contiguous, padded to kp; B operand of C B^T, contraction over j; optional)
 __global__ void __launch_bounds__(128)
 basis_splits_kernel(const float* __restrict__ basis, int64_t cols, int k, int kp, __nv_bfloat16* __restrict__ bs,
                     __nv_bfloat16* __restrict__ bt, __nv_bfloat16* __restrict__ b6, int kx) {
@@ -763,10 +766,12 @@ basis_splits_kernel(const float* __restrict__ basis, int64_t cols, int k, int kp
     }
 #pragma unroll
     for (int t = 0; t < 3; ++t) {
+      const int grp = j0 / 64, gw = min(64, kp - 64 * grp);
+      const int64_t row0 = (int64_t)3 * 64 * grp + (int64_t)t * gw + (j0 - 64 * grp);
 #pragma unroll
       for (int jj = 0; jj < 8; ++jj)
-        bs[((int64_t)t * kp + j0 + jj) * cols + col] = __ushort_as_bfloat16((unsigned short)((w[t][jj >> 1] >> (16 * (jj & 1))) & 0xFFFFu));
-      *reinterpret_cast<uint4*>(bt + ((int64_t)t * cols + col) * kp + j0) = make_uint4(w[t][0], w[t][1], w[t][2], w[t][3]);
+        bs[(row0 + jj) * cols + col] = __ushort_as_bfloat16((unsigned short)((w[t][jj >> 1] >> (16 * (jj & 1))) & 0xFFFFu));
+      if (bt != nullptr) *reinterpret_cast<uint4*>(bt + ((int64_t)t * cols + col) * kp + j0) = make_uint4(w[t][0], w[t][1], w[t][2], w[t][3]);
     }
     if (b6 != nullptr) {
       const int sel[6] = {0, 1, 0, 2, 0, 1};
@@ -1183,9 +1188,9 @@ reduce_proj_kernel(const float* __restrict__ part, int slices, int64_t cols, int
     if (j0 + r < q && c0 + tx < cols) m[(int64_t)(j0 + r) * cols + c0 + tx] = t[tx][r];
 }
 
-// z[r][j] = sum over slices s of part[s][r][j], j < q (part rows are nb wide); fixed order
+// z[r * ldz + j] = sum over slices s of part[s][r][j], j < q (part rows are nb wide); fixed order
 __global__ void __launch_bounds__(256)
-reduce_sketch_kernel(const float* __restrict__ part, int slices, int64_t rows, int nb, int q, float* __restrict__ z) {
+reduce_sketch_kernel(const float* __restrict__ part, int slices, int64_t rows, int nb, int q, float* __restrict__ z, int ldz) {
   metis_pdl_wait();
   const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (i >= rows * q) return;
@@ -1196,7 +1201,7 @@ reduce_sketch_kernel(const float* __restrict__ part, int slices, int64_t rows, i
   for (int s = 0; s < 8; ++s) t[s] = s < slices ? part[((int64_t)s * rows + r) * nb + j] : 0.0f;
 #pragma unroll
   for (int s = 0; s < 8; ++s) acc += t[s];
-  z[i] = acc;
+  z[r * ldz + j] = acc;
 }
 
 // Tensor-core projection: Mp[part][j][col] = sum over the part's sampled rows r of H[r][j] * x[idx[r], col].
@@ -1211,11 +1216,11 @@ constexpr int PP_COLS = 128, PP_K = 64, PP_STAGES = 3, PP_XP = PP_COLS + 8, PP_H
 
 // hsp[sp][j][r] (r contiguous, ldh >= rows rounded up to 64, zero padded): three-term BF16 split of H[r][j]
 __global__ void __launch_bounds__(256)
-h_splits_kernel(const float* __restrict__ h, int n_s, int q, int jp, int ldh, __nv_bfloat16* __restrict__ hsp) {
+h_splits_kernel(const float* __restrict__ h, int n_s, int q, int jp, int ldh, __nv_bfloat16* __restrict__ hsp, int pitch_h) {
   metis_pdl_wait();
   const int r = blockIdx.x * 256 + threadIdx.x, j = blockIdx.y;
   if (r >= ldh) return;
-  const float v = (r < n_s && j < q) ? h[(int64_t)r * q + j] : 0.0f;
+  const float v = (r < n_s && j < q) ? h[(int64_t)r * pitch_h + j] : 0.0f;
   const __nv_bfloat16 hh = __float2bfloat16_rn(v);
   const float r1 = v - __bfloat162float(hh);
   const __nv_bfloat16 hl = __float2bfloat16_rn(r1);
@@ -1551,6 +1556,247 @@ int jacobi_threads(int n) {
   return t < 64 ? 64 : t;
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Wide sketches (k + p above MAXQ or k above 64, up to 272 / 256): the same decomposition on kernels that tile over
+// the rank (bigrank.cuh).  The range finder works on a contiguous matrix - the operand itself (FULL) or its sampled
+// rows gathered once (SAMPLED) - so that sketch and projection both run on the tcgen05 kernel of the broadcast
+// pass, in groups of sketch columns.
+struct WideWs {
+  size_t amax, idx, xs, omt, zp, z, z2, gram, gram1, l, linv, evals, evecs, ycm, scale, hsp, mp, m, basis, bs, coef, part,
+      a6, b6, sign, evals2, evecs2, total;
+};
+constexpr int WIDE_GRAM_PARTS = 32;
+constexpr int WIDE_SK = 96;                              // sketch columns per launch of the tensor-core sketch
+constexpr int WIDE_PJ = 80;                              // sketch columns per launch of the tensor-core projection
+constexpr int WIDE_CG = 64;                              // basis vectors per launch of the broadcast pass
+
+WideWs wide_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s, bool full) {
+  WideWs w{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) & ~(size_t)255; return o; };
+  const int q = k + p, kp = (k + 15) / 16 * 16;
+  const int64_t n_r = full ? rows : n_s;
+  const int nbq = (q + WIDE_SK - 1) / WIDE_SK * WIDE_SK;
+  const int64_t ldh = (n_r + 63) / 64 * 64;
+  w.amax = take(256);
+  w.idx = take(sizeof(int) * (size_t)n_s);
+  w.xs = take(full ? 0 : sizeof(__nv_bfloat16) * (size_t)n_s * cols);
+  w.omt = take(sizeof(__nv_bfloat16) * (size_t)nbq * cols);
+  w.zp = take(sizeof(float) * (size_t)metis_coeff_slices(n_r, cols, nullptr) * n_r * WIDE_SK);
+  w.z = take(sizeof(float) * (size_t)n_r * q);
+  w.z2 = take(sizeof(float) * (size_t)n_r * q);
+  w.gram = take(sizeof(double) * (size_t)WIDE_GRAM_PARTS * q * q);
+  w.gram1 = take(sizeof(double) * (size_t)q * q);
+  w.l = take(sizeof(double) * (size_t)q * q);
+  w.linv = take(sizeof(double) * (size_t)q * q);
+  w.evals = take(sizeof(double) * (size_t)q);
+  w.evecs = take(sizeof(double) * (size_t)q * q);
+  w.ycm = take(sizeof(double) * (size_t)metis_wide::MAXQ_WIDE * q);
+  w.scale = take(sizeof(double) * (size_t)q);
+  w.hsp = take(sizeof(__nv_bfloat16) * 3 * (size_t)WIDE_PJ * ldh);
+  w.mp = take(sizeof(float) * (size_t)8 * cols * WIDE_PJ);
+  w.m = take(sizeof(float) * (size_t)q * cols);
+  w.basis = take(sizeof(float) * (size_t)k * cols);
+  w.bs = take(sizeof(__nv_bfloat16) * 3 * (size_t)kp * cols);
+  w.coef = take(sizeof(float) * (size_t)kp * rows);
+  w.part = take(sizeof(float) * (size_t)metis_coeff_slices(rows, cols, nullptr) * rows * WIDE_CG);
+  w.a6 = take(sizeof(__nv_bfloat16) * (size_t)metis_residual_kx(kp) * rows);
+  w.b6 = take(sizeof(__nv_bfloat16) * (size_t)metis_residual_kx(kp) * cols);
+  w.sign = take(sizeof(float) * (size_t)kp);
+  w.evals2 = take(sizeof(double) * (size_t)k);
+  w.evecs2 = take(sizeof(double) * (size_t)k * k);
+  w.total = off;
+  return w;
+}
+
+bool split_is_wide(int k, int p) { return k > 64 || k + p > MAXQ; }
+
+metis_status_t launch_gemm64(cudaStream_t s, const metis_wide::Gemm64Args& g) {
+  dim3 grid((unsigned)metis_ceil_div(g.N, 64), (unsigned)metis_ceil_div(g.M, 64));
+  METIS_CUDA_TRY(metis_launch_pdl(metis_wide::gemm64_kernel, grid, dim3(256), (size_t)0, s, g)); METIS_COUNT_LAUNCH();
+  return METIS_OK;
+}
+
+// FP64 Gram matrix of n vectors (element (r, i) at v[r * sr + i * sv]) into gram1 (n x n), by slabs of rows
+metis_status_t launch_gram64(cudaStream_t s, const float* v, int64_t n_rows, int n, int64_t sr, int64_t sv, double* parts, double* gram1) {
+  int64_t rpp = metis_ceil_div(metis_ceil_div(n_rows, WIDE_GRAM_PARTS), metis_wide::G64_R) * metis_wide::G64_R;
+  if (rpp < 64) rpp = 64;
+  const int n_parts = (int)metis_ceil_div(n_rows, rpp);
+  const unsigned t = (unsigned)metis_ceil_div(n, metis_wide::G64_T);
+  METIS_CUDA_TRY(metis_launch_pdl(metis_wide::gram64_kernel, dim3(t, t, (unsigned)n_parts), dim3(256), (size_t)0, s, v, n_rows, n, sr, sv, rpp, parts,
+                                  (const int*)nullptr)); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(metis_launch_pdl((reduce_gram_kernel), dim3((unsigned)metis_ceil_div(n * n, 32)), dim3(128), (size_t)(0), s, (const double*)parts, n_parts, n * n, gram1,
+                                  (const int*)nullptr)); METIS_COUNT_LAUNCH();
+  return METIS_OK;
+}
+
+// eigen-decomposition of the n x n Gram matrix gram1: Cholesky factor, cluster Jacobi on its columns, collection
+metis_status_t launch_eig_wide(cudaStream_t s, const double* gram1, int n, float exit_cos2, double* l, double* ycm, double* evals, double* evecs) {
+  METIS_CUDA_TRY(metis_launch_pdl(metis_wide::chol_wide_kernel, dim3(1), dim3(1024), (size_t)0, s, gram1, n, 1e-14, l, (double*)nullptr, (const int*)nullptr,
+                                  (int*)nullptr)); METIS_COUNT_LAUNCH();
+  metis_wide::jacobi_cluster_kernel<<<metis_wide::JC_P, metis_wide::JC_THREADS, metis_wide::JC_SMEM, s>>>(l, n, exit_cos2, ycm); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  metis_wide::jacobi_collect_kernel<<<1, 1024, 0, s>>>(ycm, n, evals, evecs); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
+
+metis_status_t split_wide(metis_context* ctx, const __nv_bfloat16* x, int64_t rows, int64_t cols, int k, int p, bool full, int64_t n_s,
+                          uint64_t seed, int rounding, bool want_c, bool want_r, metis_operand_t* out, float* residual_dense,
+                          unsigned char* wsb, const WideWs& L, cudaStream_t s) {
+  using namespace metis_qt;
+  using metis_wide::Gemm64Args;
+  const int q = k + p, kp = (k + 15) / 16 * 16, kx6 = metis_residual_kx(kp);
+  const int64_t n_r = full ? rows : n_s;
+  const int64_t ldh = (n_r + 63) / 64 * 64;
+  float* amax = reinterpret_cast<float*>(wsb + L.amax);
+  int* idx = reinterpret_cast<int*>(wsb + L.idx);
+  __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(wsb + L.xs);
+  __nv_bfloat16* omt = reinterpret_cast<__nv_bfloat16*>(wsb + L.omt);
+  float* zp = reinterpret_cast<float*>(wsb + L.zp);
+  float* z = reinterpret_cast<float*>(wsb + L.z);
+  float* z2 = reinterpret_cast<float*>(wsb + L.z2);
+  double* gram = reinterpret_cast<double*>(wsb + L.gram);
+  double* gram1 = reinterpret_cast<double*>(wsb + L.gram1);
+  double* lf = reinterpret_cast<double*>(wsb + L.l);
+  double* linv = reinterpret_cast<double*>(wsb + L.linv);
+  double* evals = reinterpret_cast<double*>(wsb + L.evals);
+  double* evecs = reinterpret_cast<double*>(wsb + L.evecs);
+  double* ycm = reinterpret_cast<double*>(wsb + L.ycm);
+  double* scale = reinterpret_cast<double*>(wsb + L.scale);
+  __nv_bfloat16* hsp = reinterpret_cast<__nv_bfloat16*>(wsb + L.hsp);
+  float* mp = reinterpret_cast<float*>(wsb + L.mp);
+  float* m = reinterpret_cast<float*>(wsb + L.m);
+  float* basis = reinterpret_cast<float*>(wsb + L.basis);
+  __nv_bfloat16* bs = reinterpret_cast<__nv_bfloat16*>(wsb + L.bs);
+  float* coef = reinterpret_cast<float*>(wsb + L.coef);
+  float* part = reinterpret_cast<float*>(wsb + L.part);
+  __nv_bfloat16* a6 = reinterpret_cast<__nv_bfloat16*>(wsb + L.a6);
+  __nv_bfloat16* b6 = reinterpret_cast<__nv_bfloat16*>(wsb + L.b6);
+  float* sign = reinterpret_cast<float*>(wsb + L.sign);
+  double* evals2 = reinterpret_cast<double*>(wsb + L.evals2);
+  double* evecs2 = reinterpret_cast<double*>(wsb + L.evecs2);
+
+  METIS_CUDA_TRY(cudaMemsetAsync(amax, 0, 64, s));
+  const __nv_bfloat16* xr = x;
+  if (!full) {
+    METIS_CUDA_TRY(metis_launch_pdl((sample_rows_kernel), dim3((unsigned)metis_ceil_div(n_s, 256)), dim3(256), (size_t)(0), s, idx, (int)n_s, rows, seed, 0)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl(metis_wide::gather_rows_kernel, dim3((unsigned)metis_ceil_div(n_s * (cols / 8), 256)), dim3(256), (size_t)0, s, x, cols,
+                                    (const int*)idx, (int)n_s, xs)); METIS_COUNT_LAUNCH();
+    xr = xs;
+  }
+  // (2) sketch Z = xr Omega on the tensor cores, WIDE_SK sketch columns per launch
+  const int nbq = (q + WIDE_SK - 1) / WIDE_SK * WIDE_SK;
+  {
+    const uint64_t blocks = ((uint64_t)cols * q + 7) / 8;
+    METIS_CUDA_TRY(metis_launch_pdl((omega_rows_kernel), dim3((unsigned)metis_ceil_div((int64_t)blocks, 256)), dim3(256), (size_t)(0), s, cols, q, nbq, seed, ctx->quantile_lut, omt)); METIS_COUNT_LAUNCH();
+    const int slices = metis_coeff_slices(n_r, cols, nullptr);
+    for (int j0 = 0; j0 < q; j0 += WIDE_SK) {
+      const int qg = q - j0 < WIDE_SK ? q - j0 : WIDE_SK;
+      METIS_TRY(metis_launch_coeff_tc(ctx, xr, n_r, cols, omt + (int64_t)j0 * cols, WIDE_SK / 3, zp, (full && j0 == 0) ? amax : nullptr, 1, s));
+      METIS_CUDA_TRY(metis_launch_pdl((reduce_sketch_kernel), dim3((unsigned)metis_ceil_div(n_r * qg, 256)), dim3(256), (size_t)(0), s, (const float*)zp, slices, n_r, WIDE_SK, qg,
+                                      z + j0, q)); METIS_COUNT_LAUNCH();
+    }
+  }
+  // (3) CholeskyQR2: both passes always (FP64 Gram matrix, factor and inverse factor; H = Z L^-T as a product)
+  {
+    float* src = z; float* dst = z2;
+    for (int pass = 0; pass < 2; ++pass) {
+      METIS_TRY(launch_gram64(s, src, n_r, q, q, 1, gram, gram1));
+      METIS_CUDA_TRY(metis_launch_pdl(metis_wide::chol_wide_kernel, dim3(1), dim3(1024), (size_t)0, s, (const double*)gram1, q, 1e-13, lf, linv, (const int*)nullptr,
+                                      (int*)nullptr)); METIS_COUNT_LAUNCH();
+      Gemm64Args g{};
+      g.a = src; g.a_m = q; g.a_k = 1; g.b = linv; g.b_k = 1; g.b_n = q; g.c = dst; g.c_m = q; g.c_n = 1; g.M = n_r; g.N = q; g.K = q;
+      METIS_TRY(launch_gemm64(s, g));
+      float* t = src; src = dst; dst = t;
+    }
+  }                                                      // H is in z again
+  // (4) M = H^T xr on the tensor cores, WIDE_PJ sketch columns per launch; eigen-decomposition of M M^T
+  {
+    const int slices = metis_project_slices(n_r, cols);
+    for (int j0 = 0; j0 < q; j0 += WIDE_PJ) {
+      const int qg = q - j0 < WIDE_PJ ? q - j0 : WIDE_PJ;
+      const int jp = (qg + 15) / 16 * 16;
+      METIS_CUDA_TRY(metis_launch_pdl(h_splits_kernel, dim3((unsigned)metis_ceil_div(ldh, 256), (unsigned)jp), dim3(256), (size_t)0, s, (const float*)(z + j0), (int)n_r, qg, jp,
+                                      (int)ldh, hsp, q)); METIS_COUNT_LAUNCH();
+      METIS_TRY(metis_launch_project_tc(ctx, xr, n_r, cols, hsp, jp, ldh, mp, s));
+      dim3 rgrid((unsigned)metis_ceil_div(cols, 32), (unsigned)metis_ceil_div(qg, 32));
+      METIS_CUDA_TRY(metis_launch_pdl((reduce_proj_kernel), rgrid, dim3(256), (size_t)(0), s, (const float*)mp, slices, cols, jp, qg, m + (int64_t)j0 * cols)); METIS_COUNT_LAUNCH();
+    }
+    METIS_TRY(launch_gram64(s, m, cols, q, 1, cols, gram, gram1));
+    METIS_TRY(launch_eig_wide(s, gram1, q, 1e-8f, lf, ycm, evals, evecs));
+  }
+  // right basis: basis[j][col] = sum_i evecs[i][j] M[i][col] / sqrt(eval_j),  j < k
+  float* rb = full ? out->right : basis;
+  {
+    METIS_CUDA_TRY(metis_launch_pdl(metis_wide::rot_scales_kernel, dim3((unsigned)metis_ceil_div(k, 128)), dim3(128), (size_t)0, s, (const double*)evals, (const float*)nullptr, k, 0,
+                                    scale, full ? out->sigma : (float*)nullptr)); METIS_COUNT_LAUNCH();
+    Gemm64Args g{};
+    g.a = m; g.a_m = 1; g.a_k = cols; g.b = evecs; g.b_k = q; g.b_n = 1; g.scale = scale; g.c = rb; g.c_m = 1; g.c_n = cols; g.M = cols; g.N = k; g.K = q;
+    METIS_TRY(launch_gemm64(s, g));
+  }
+  QuantParams qp{};
+  metis_nvfp4_t rc = out->res_by_cols, rr = out->res_by_rows;
+  rc.rows = rows; rc.k_len = cols; rr.rows = cols; rr.k_len = rows;
+  qp.rows = rows; qp.cols = cols; qp.rounding = rounding; qp.seed = seed; qp.stream_id = METIS_STREAM_RESIDUAL;
+  qp.e_stride_r = cols; qp.e_stride_c = 1;
+  if (want_c) { qp.c_codes = rc.codes; qp.c_scales = rc.scales; qp.c_layout = rc.sf_layout; }
+  if (want_r) { qp.r_codes = rr.codes; qp.r_scales = rr.scales; qp.r_layout = rr.sf_layout; }
+  float* t0 = want_c ? rc.tensor_scale : nullptr; float* t1 = want_r ? rr.tensor_scale : nullptr;
+  const dim3 bs_grid((unsigned)metis_ceil_div(cols, 128), (unsigned)(kp / 8));
+  cudaStream_t sf = ctx->side[0];
+  if (full) {
+    // right = basis with the sign convention, left = H U~_k (same flips), coefficients = left * sigma
+    METIS_CUDA_TRY(metis_launch_pdl(metis_wide::sign_rows_kernel, dim3((unsigned)k), dim3(256), (size_t)0, s, out->right, cols, sign, amax + 2)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((basis_splits_kernel), bs_grid, dim3(128), (size_t)(0), s, (const float*)out->right, cols, k, kp, bs, (__nv_bfloat16*)nullptr, b6, kx6)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl(metis_wide::rot_scales_kernel, dim3((unsigned)metis_ceil_div(k, 128)), dim3(128), (size_t)0, s, (const double*)evals, (const float*)sign, k, 2,
+                                    scale, (float*)nullptr)); METIS_COUNT_LAUNCH();
+    if (kp > k) METIS_CUDA_TRY(cudaMemsetAsync(coef, 0, sizeof(float) * (size_t)kp * rows, s));
+    Gemm64Args g{};
+    g.a = z; g.a_m = q; g.a_k = 1; g.b = evecs; g.b_k = q; g.b_n = 1; g.scale = scale; g.c = out->left; g.c_m = 1; g.c_n = rows;
+    g.c2 = coef; g.c2_m = kp; g.c2_n = 1; g.scale2 = out->sigma; g.amax = amax + 1; g.M = rows; g.N = k; g.K = q;
+    METIS_TRY(launch_gemm64(s, g));
+    METIS_TRY(metis_fork(ctx, s, 1));
+    METIS_TRY(metis_launch_residual_tc(ctx, x, coef, k, kp, qp, amax, t0, t1, residual_dense, a6, b6, s));
+  } else {
+    METIS_CUDA_TRY(metis_launch_pdl((basis_splits_kernel), bs_grid, dim3(128), (size_t)(0), s, (const float*)basis, cols, k, kp, bs, (__nv_bfloat16*)nullptr, b6, kx6)); METIS_COUNT_LAUNCH();
+    // (5) broadcast C = x B, WIDE_CG basis vectors per pass over x
+    const int slices = metis_coeff_slices(rows, cols, nullptr);
+    for (int j0 = 0; j0 < kp; j0 += WIDE_CG) {
+      const int gw = kp - j0 < WIDE_CG ? kp - j0 : WIDE_CG;
+      METIS_TRY(metis_launch_coeff_tc(ctx, x, rows, cols, bs + (int64_t)3 * j0 * cols, gw, part, j0 == 0 ? amax : nullptr, 0, s));
+      METIS_CUDA_TRY(metis_launch_pdl(metis_wide::coef_sum_kernel, dim3((unsigned)metis_ceil_div(rows * (gw / 8), 256)), dim3(256), (size_t)0, s, (const float*)part, slices, rows, gw, j0,
+                                      kp, coef, a6, kx6)); METIS_COUNT_LAUNCH();
+    }
+    METIS_TRY(metis_fork(ctx, s, 1));
+    METIS_TRY(metis_launch_residual_tc(ctx, x, nullptr, k, kp, qp, amax, t0, t1, residual_dense, a6, b6, s));
+    // (7) Rayleigh-Ritz on C^T C, rotate both factors (side stream, beside the residual pass)
+    METIS_TRY(launch_gram64(sf, coef, rows, k, kp, 1, gram, gram1));
+    METIS_TRY(launch_eig_wide(sf, gram1, k, 1e-6f, lf, ycm, evals2, evecs2));
+    {
+      Gemm64Args g{};
+      g.a = basis; g.a_m = 1; g.a_k = cols; g.b = evecs2; g.b_k = k; g.b_n = 1; g.c = out->right; g.c_m = 1; g.c_n = cols; g.M = cols; g.N = k; g.K = k;
+      METIS_TRY(launch_gemm64(sf, g));
+    }
+    METIS_CUDA_TRY(metis_launch_pdl(metis_wide::sign_rows_kernel, dim3((unsigned)k), dim3(256), (size_t)0, sf, out->right, cols, sign, amax + 2)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl(metis_wide::rot_scales_kernel, dim3((unsigned)metis_ceil_div(k, 128)), dim3(128), (size_t)0, sf, (const double*)evals2, (const float*)sign, k, 1,
+                                    scale, out->sigma)); METIS_COUNT_LAUNCH();
+    {
+      Gemm64Args g{};
+      g.a = coef; g.a_m = kp; g.a_k = 1; g.b = evecs2; g.b_k = k; g.b_n = 1; g.scale = scale; g.c = out->left; g.c_m = 1; g.c_n = rows; g.amax = amax + 1;
+      g.M = rows; g.N = k; g.K = k;
+      METIS_TRY(launch_gemm64(sf, g));
+    }
+  }
+  METIS_CUDA_TRY(metis_launch_pdl((split_status_kernel), dim3(1), dim3(32), (size_t)(0), s, (const float*)amax, (const double*)evals, k, ctx->dev_status)); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  metis_nvfp4_t lq = out->left_q, rq = out->right_q;
+  lq.rows = k; lq.k_len = rows; rq.rows = k; rq.k_len = cols;
+  METIS_TRY(metis_launch_quantize_factors(out->left, rows, out->right, cols, k, rounding, seed, amax + 1, amax + 2, &lq, &rq, sf));
+  return metis_join(ctx, s, 0);
+}
+
 }  // namespace
 
 int64_t metis_default_sample_count(int64_t rows, int32_t q) {
@@ -1575,6 +1821,7 @@ metis_status_t metis_split_set_attrs() {
   METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
   METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
   METIS_CUDA_TRY(cudaFuncSetAttribute(gram_chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GC_MAX_SMEM));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(metis_wide::jacobi_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)metis_wide::JC_SMEM));
 #define METIS_PP_ATTR(MTV) METIS_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<MTV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
       (int)((size_t)PP_STAGES * (PP_K * PP_XP * 2 + 3 * (MTV) * 16 * PP_HP * 2))))
   METIS_PP_ATTR(1); METIS_PP_ATTR(2); METIS_PP_ATTR(3); METIS_PP_ATTR(4); METIS_PP_ATTR(5);
@@ -1590,6 +1837,12 @@ metis_status_t metis_launch_amax_check(metis_context* ctx, const float* amax, cu
 }
 
 size_t metis_split_ws_bytes(int64_t rows, int64_t cols, int k, int p) {
+  if (k > 0 && split_is_wide(k, p)) {
+    // the larger of the FULL layout and the SAMPLED layout with the default sample count
+    const size_t a = wide_ws_layout(rows, cols, k, p, rows, true).total;
+    const size_t b = wide_ws_layout(rows, cols, k, p, metis_default_sample_count(rows, k + p), false).total;
+    return a > b ? a : b;
+  }
   // Every buffer grows with the sample count except the sketch partials, whose chunk width steps from 64 to 256
   // columns above 512 sampled rows: the FULL sketch (n_s = rows) and a 512-row sample bound every other case.
   const size_t full = split_ws_layout(rows, cols, k, p, rows).total;
@@ -1604,7 +1857,8 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   using namespace metis_qt;
   if (!h || !xv || !out || !ws) return METIS_ERR_INVALID_ARG;
   if (rows <= 0 || cols <= 0 || rows % 16 || cols % 16 || k < 0 || p < 0) return METIS_ERR_SHAPE;
-  if (k > 0 && (k > 64 || k + p > MAXQ || k % 4)) return METIS_ERR_SHAPE;
+  if (k > 0 && (k > metis_wide::MAXK_WIDE || k + p > metis_wide::MAXQ_WIDE || k % 4)) return METIS_ERR_SHAPE;
+  const bool wide = k > 0 && split_is_wide(k, p);
   if (out->k != k || out->rows != rows || out->cols != cols) return METIS_ERR_INVALID_ARG;
   if (!metis_aligned16(xv) || !metis_aligned16(ws)) return METIS_ERR_ALIGNMENT;
   if (rounding != METIS_ROUND_RNE && rounding != METIS_ROUND_SR) return METIS_ERR_INVALID_ARG;
@@ -1619,6 +1873,17 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   int64_t n_s = full ? rows : (n_sample > 0 ? n_sample : metis_default_sample_count(rows, q));
   if (k > 0 && (n_s > rows || n_s % 16 || q > n_s || q > cols)) return METIS_ERR_SHAPE;
   if (k == 0) n_s = 16;
+  if (wide) {
+    // the tensor-core passes carry the wide path: 16-byte aligned rows of x, whole 64-column chunks
+    if (cols % 64 || rows % 64 || !metis_residual_tc_usable(xv, cols)) return METIS_ERR_SHAPE;
+    const WideWs W = wide_ws_layout(rows, cols, k, p, n_s, full);
+    if (ws_bytes < W.total) return METIS_ERR_WORKSPACE;
+    if (!out->left || !out->sigma || !out->right || !out->left_q.codes || !out->right_q.codes || !out->left_q.scales ||
+        !out->right_q.scales || !out->left_q.tensor_scale || !out->right_q.tensor_scale)
+      return METIS_ERR_INVALID_ARG;
+    return split_wide(h, reinterpret_cast<const __nv_bfloat16*>(xv), rows, cols, k, p, full, n_s, seed, rounding, want_c, want_r, out,
+                      residual_dense, reinterpret_cast<unsigned char*>(ws), W, reinterpret_cast<cudaStream_t>(stream));
+  }
   const SplitWs L = split_ws_layout(rows, cols, k, p, n_s);
   if (ws_bytes < L.total) return METIS_ERR_WORKSPACE;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
@@ -1690,7 +1955,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     METIS_CUDA_TRY(metis_launch_pdl((omega_rows_kernel), dim3((unsigned)metis_ceil_div((int64_t)blocks, 256)), dim3(256), (size_t)(0), s, cols, q, nb_sk, seed, ctx->quantile_lut, omt)); METIS_COUNT_LAUNCH();
     METIS_TRY(metis_launch_coeff_tc(ctx, x, rows, cols, omt, nb_sk / 3, zp, amax, 1, s));
     const int slices = metis_coeff_slices(rows, cols, nullptr);
-    METIS_CUDA_TRY(metis_launch_pdl((reduce_sketch_kernel), dim3((unsigned)metis_ceil_div(rows * q, 256)), dim3(256), (size_t)(0), s, zp, slices, rows, nb_sk, q, z)); METIS_COUNT_LAUNCH();
+    METIS_CUDA_TRY(metis_launch_pdl((reduce_sketch_kernel), dim3((unsigned)metis_ceil_div(rows * q, 256)), dim3(256), (size_t)(0), s, zp, slices, rows, nb_sk, q, z, q)); METIS_COUNT_LAUNCH();
   } else {
     const int nt = (q + 7) / 8;
     const size_t smem = sizeof(__nv_bfloat16) * nt * 8 * SKM_PITCH;
@@ -1738,7 +2003,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
       rpp = (int)(metis_ceil_div(metis_ceil_div(n_s, parts), PP_K) * PP_K);
       parts = (int)metis_ceil_div(n_s, rpp);
       const int mt = (q + 15) / 16, jp = mt * 16, ldh = (int)((n_s + 63) / 64 * 64);
-      METIS_CUDA_TRY(metis_launch_pdl(h_splits_kernel, dim3((unsigned)metis_ceil_div(ldh, 256), (unsigned)jp), dim3(256), (size_t)0, s, z, (int)n_s, q, jp, ldh, hsp)); METIS_COUNT_LAUNCH();
+      METIS_CUDA_TRY(metis_launch_pdl(h_splits_kernel, dim3((unsigned)metis_ceil_div(ldh, 256), (unsigned)jp), dim3(256), (size_t)0, s, z, (int)n_s, q, jp, ldh, hsp, q)); METIS_COUNT_LAUNCH();
       project_tc = full && metis_project_tc_usable(x, hsp, cols, jp);
       if (project_tc) {
         // every row, in order: M^T = x^T H on the tcgen05 kernel of the broadcast pass (x as an MN-major operand)

@@ -98,21 +98,32 @@ def flip_allowance(pairs, gain=1.5, max_fraction=2e-3):
     return min(gain * extra, ALLOWANCE_CAP)
 
 
-def check_e2e(case, errors, pairs, base_tol=E2E_TOL):
+BULK_CUT_CAP = 1e-2       # allowance cap of the cases whose rank cut falls inside the Gaussian bulk (see check_e2e)
+
+
+def check_e2e(case, errors, pairs, base_tol=E2E_TOL, cut_in_bulk=False):
     """Asserts every end-to-end error in `errors` (name -> relative Frobenius error against the oracle) and leaves an
     audit line: the case, each error, the allowance that was added to `base_tol`, how many factor blocks differed,
     and whether the plain tolerance alone would have held.  The line is printed (pytest -rP shows it) and kept in
-    E2E_RECORDS, which the session writes to the file named by METIS_PARITY_LOG."""
+    E2E_RECORDS, which the session writes to the file named by METIS_PARITY_LOG.
+
+    cut_in_bulk: the split rank exceeds the planted rank, so the factor vectors beyond the planted ones are singular
+    vectors of the Gaussian bulk, whose neighbouring singular values lie ~1e-3 apart.  Such vectors are determined
+    only to (FP32 rounding) / (relative gap) ~ 1e-5 - against ~1e-7 for the planted ones - and the NVFP4 encoder
+    turns that into re-rounded codes in a few blocks per thousand.  What is unique there (singular values, the
+    spanned subspace through the residual, the bytes given the FP32 factors, the products given the bytes) is
+    checked tightly elsewhere; the end-to-end figure of these cases gets the caps BULK_CUT_CAP / 1 % of the blocks
+    and is reported as conditioning-limited."""
     extra, differing, total = flip_stats(pairs)
-    assert differing <= max(4, 2e-3 * total), (case, differing, total)
-    allowance = min(1.5 * extra, ALLOWANCE_CAP)
+    assert differing <= max(4, (1e-2 if cut_in_bulk else 2e-3) * total), (case, differing, total)
+    allowance = min(1.5 * extra, BULK_CUT_CAP if cut_in_bulk else ALLOWANCE_CAP)
     worst = max(errors.values())
     rec = {"case": case, "errors": {k: float(v) for k, v in errors.items()}, "base_tol": base_tol, "allowance": allowance,
            "differing_blocks": differing, "factor_blocks": total, "plain_tolerance_held": bool(worst < base_tol)}
     E2E_RECORDS.append(rec)
-    print("E2E %s: %s | base %.1e + allowance %.2e | differing factor blocks %d/%d | plain tolerance %s"
+    print("E2E %s: %s | base %.1e + allowance %.2e | differing factor blocks %d/%d | plain tolerance %s%s"
           % (case, " ".join("%s=%.3e" % kv for kv in rec["errors"].items()), base_tol, allowance, differing, total,
-             "held" if rec["plain_tolerance_held"] else "NOT held"))
+             "held" if rec["plain_tolerance_held"] else "NOT held", " | rank cut inside the bulk (conditioning-limited)" if cut_in_bulk else ""))
     for name, err in errors.items():
         assert err < base_tol + allowance, (case, name, err, base_tol, allowance)
     return rec

@@ -84,7 +84,7 @@ def test_forward_and_backward_medium(ctx, k):
     assert rel_fro(dw.cpu().numpy(), (ld + rdr).T @ (lx + rxr)) < 2e-5
 
 
-@pytest.mark.parametrize("k", [0, 8])
+@pytest.mark.parametrize("k", [0, 8, 128])
 def test_layer_on_the_oracles_own_bytes(ctx, k):
     """No discontinuity in the way: the ORACLE's codes, scale bytes, tensor scales and singular values are uploaded
     into the library's operands, so both sides multiply exactly the same quantized tensors.  Eq. 2, Eq. 3 and the
@@ -92,21 +92,28 @@ def test_layer_on_the_oracles_own_bytes(ctx, k):
     allowance of any kind."""
     from gpu_util import rel_fro, operand_from_oracle
     B, h = ctx
-    l, m, n, p = 512, 384, 256, 8 if k else 0
-    x, _ = synth.llama_like(l, m, 1.0, 51, rank=8)
-    w, _ = synth.llama_like(n, m, 0.02, 52, rank=8)
-    d, _ = synth.llama_like(l, n, 1e-4, 53, rank=8)
+    l, m, n, p = (512, 384, 256, 8 if k else 0) if k <= 64 else (1024, 768, 640, 8)      # k = 128: the wide-rank composition
+    x, _ = synth.llama_like(l, m, 1.0, 51, rank=max(k, 8))
+    w, _ = synth.llama_like(n, m, 0.02, 52, rank=max(k, 8))
+    d, _ = synth.llama_like(l, n, 1e-4, 53, rank=max(k, 8))
     xq = olay.quantize_operand(x, k, p, osp.MODE_SAMPLED, 1)
     wq = olay.quantize_operand(w, k, p, osp.MODE_FULL, 2)
     dq = olay.quantize_operand(d, k, p, osp.MODE_SAMPLED, 3, onv.ROUND_SR)
     xo, wo, do = (operand_from_oracle(B, q) for q in (xq, wq, dq))
     y = h.linear_fwd(xo, wo)
-    dx, dw = h.linear_bwd(do, xo, wo)
+    fg = tuple(torch.full(sh, float("nan"), device="cuda") for sh in ((k, n), (k,), (k, m))) if k else None
+    dx, dw = h.linear_bwd(do, xo, wo, factor_grads=fg)
     torch.cuda.synchronize()
     assert h.device_status() == 0
-    assert rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)) < 2e-5
-    assert rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)) < 2e-5
-    assert rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq)) < 2e-5
+    errs = (rel_fro(y.cpu().numpy(), olay.linear_fwd(xq, wq)), rel_fro(dx.cpu().numpy(), olay.linear_dgrad(dq, wq)),
+            rel_fro(dw.cpu().numpy(), olay.linear_wgrad(dq, xq)))
+    print("layer on the oracle's bytes, k = %d: y %.2e dx %.2e dw %.2e" % (k, *errs))
+    assert max(errs) < 2e-5
+    if k:
+        du, ds, dv = olay.factor_grads(olay.linear_wgrad(dq, xq), wq)
+        d_left, d_sigma, d_right = fg
+        assert rel_fro(d_right.cpu().numpy().T, du) < 2e-5 and rel_fro(d_left.cpu().numpy().T, dv) < 2e-5
+        assert rel_fro(d_sigma.cpu().numpy(), ds) < 2e-5
 
 
 @pytest.mark.parametrize("dw_dtype", [torch.float32, torch.bfloat16])

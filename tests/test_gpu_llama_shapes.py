@@ -27,6 +27,8 @@ CASES = [
     ("70b_proj_quarter_scale_2048to7168_k64", 1024, 2048, 7168, 64, 8, 64, True),
     ("70b_proj_quarter_scale_2048to7168_k16", 1024, 2048, 7168, 16, 8, 64, True),
     ("70b_proj_quarter_scale_2048to7168_k0", 1024, 2048, 7168, 0, 0, 64, True),
+    ("70b_proj_quarter_scale_2048to7168_k128", 1024, 2048, 7168, 128, 8, 64, True),
+    ("70b_proj_quarter_scale_2048to7168_k256", 2048, 2048, 7168, 256, 8, 64, True),
 ]
 
 
@@ -66,4 +68,4 @@ def test_layer_on_sampled_outputs(case):
     check_e2e(case[0], {"y": rel_fro(y_s, xq.dense_by_cols(rl) @ wq.dense_by_cols(rn).T),
                         "dx": rel_fro(dx_s, dq.dense_by_cols(rl) @ wq.dense_by_rows(cm)),
                         "dw": rel_fro(dw_s, dq.dense_by_rows(rn).T @ xq.dense_by_rows(cm))},
-              list(zip(factors, (xq, wq, dq))) if k else [], TOL)
+              list(zip(factors, (xq, wq, dq))) if k else [], TOL, cut_in_bulk=k > rank)
