@@ -198,6 +198,20 @@ metis_status_t metis_split(metis_handle_t h, const void* x, int64_t rows, int64_
                            int32_t residual_axes, metis_operand_t* out, float* residual_dense,
                            void* ws, size_t ws_bytes, metis_stream_t stream);
 
+/* Re-quantization of a stored operand (Section 3.2: a weight is kept as separately stored U, S, V and W_R, which the
+ * optimizer updates; per step only their NVFP4 forms are refreshed - no decomposition).  `op` holds the stored FP32
+ * factors (op->left k x rows, op->right k x cols, op->sigma; read, never written) and receives left_q, right_q
+ * (own amax/2688 tensor scales, draws of METIS_STREAM_LEFT / _RIGHT) and the residual orientations selected by
+ * `residual_axes`, quantized from `residual` (rows x cols, leading dimension ld_res elements, BF16 or FP32) with
+ * draws of METIS_STREAM_RESIDUAL.  res_tscale == METIS_TSCALE_AMAX_SELF: the residual's tensor scale is
+ * amax(residual)/2688 (there is no source tensor to take it from); METIS_TSCALE_GIVEN: the requested outputs'
+ * tensor_scale already hold the value (e.g. the one the initial split produced).  k == 0: residual only.
+ * Five launches (three amax reductions, one kernel for both residual orientations, one for both factors).
+ * Workspace: 256 bytes. */
+metis_status_t metis_requantize_operand(metis_handle_t h, const void* residual, int32_t res_dtype, int64_t ld_res,
+                                        int32_t rounding, uint64_t seed, int32_t residual_axes, int32_t res_tscale,
+                                        metis_operand_t* op, void* ws, size_t ws_bytes, metis_stream_t stream);
+
 /* ---- linear layer (Eq. 2, Eq. 3, weight gradient) ----------------------------------------- */
 
 /* y (l x n, ldy) = Xq Wq^T, Eq. 2.  x: l x m operand with res_by_cols; w: W_t, n x m operand with

@@ -76,6 +76,30 @@ def quantize_operand(x, k, p, mode, seed, rounding=nvfp4.ROUND_RNE):
     return QOperand(k, left_q, sp.sigma, right_q, res_c, res_r, sp, raw)
 
 
+def requantize_operand(left, sigma, right, residual, rounding=nvfp4.ROUND_RNE, seed=0, residual_scale=None):
+    """NVFP4 forms of an operand that is HELD as separately stored pieces (Section 3.2 keeps a weight as U, S, V and
+    W_R, which training updates; per step they are only quantized again, never decomposed again).
+
+    left (rows x k), right (cols x k), residual (rows x cols) are the stored float32 values.  Every piece is
+    quantized on its own: the factors exactly as quantize_operand does it, the residual in both block orientations
+    with its OWN amax/2688 as tensor scale (there is no source tensor here) unless residual_scale is given."""
+    res32 = np.asarray(residual, dtype=np.float32)
+    k = int(np.asarray(sigma).shape[0])
+    rc = nvfp4.quantize(res32, nvfp4.AXIS_COLS, rounding, seed, philox.STREAM_RESIDUAL, tensor_scale=residual_scale)
+    rr = nvfp4.quantize(res32, nvfp4.AXIS_ROWS, rounding, seed, philox.STREAM_RESIDUAL, tensor_scale=residual_scale)
+    raw = {"res_by_cols": rc, "res_by_rows": rr}
+    if k:
+        lq = nvfp4.quantize(np.ascontiguousarray(np.asarray(left, dtype=np.float32).T), nvfp4.AXIS_COLS, rounding, seed, philox.STREAM_LEFT)
+        rq = nvfp4.quantize(np.ascontiguousarray(np.asarray(right, dtype=np.float32).T), nvfp4.AXIS_COLS, rounding, seed, philox.STREAM_RIGHT)
+        raw["left"], raw["right"] = lq, rq
+        left_q, right_q = nvfp4.dequantize(*lq).T, nvfp4.dequantize(*rq).T
+    else:
+        left_q, right_q = np.zeros((res32.shape[0], 0)), np.zeros((res32.shape[1], 0))
+    sp = split_mod.Split(np.asarray(left, dtype=np.float64), np.asarray(sigma, dtype=np.float64), np.asarray(right, dtype=np.float64),
+                         res32.astype(np.float64))
+    return QOperand(k, left_q, np.asarray(sigma, dtype=np.float64), right_q, nvfp4.dequantize(*rc), nvfp4.dequantize(*rr).T, sp, raw)
+
+
 def linear_fwd(xq, wq):
     """Eq. 2: Y^ = Xq Wq^T, both residuals quantized along the in-feature axis."""
     return xq.dense(nvfp4.AXIS_COLS) @ wq.dense(nvfp4.AXIS_COLS).T

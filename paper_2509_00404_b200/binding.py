@@ -27,7 +27,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "ALIGNMENT", 4: "WORKS
 EXPORTED = ["metis_create", "metis_destroy", "metis_last_device_status", "metis_debug_quantile_table",
             "metis_debug_launch_count", "metis_debug_timestamp", "metis_debug_wait_timeout",
             "metis_sf_bytes", "metis_workspace_bytes", "metis_default_sample_count", "metis_quantize_nvfp4",
-            "metis_split", "metis_linear_fwd", "metis_linear_fwd_static_ws", "metis_linear_bwd", "metis_gemm_nvfp4"]
+            "metis_split", "metis_requantize_operand", "metis_linear_fwd", "metis_linear_fwd_static_ws", "metis_linear_bwd", "metis_gemm_nvfp4"]
 
 
 class MetisError(RuntimeError):
@@ -79,6 +79,7 @@ def lib():
     l.metis_quantize_nvfp4.argtypes = [vp, vp, i32, i64, i64, i64, i32, u64, u32, i32, P(NvFp4Struct), P(NvFp4Struct),
                                        vp, sz, vp]
     l.metis_split.argtypes = [vp, vp, i64, i64, i32, i32, i32, i64, u64, i32, i32, P(OperandStruct), vp, vp, sz, vp]
+    l.metis_requantize_operand.argtypes = [vp, vp, i32, i64, i32, u64, i32, i32, P(OperandStruct), vp, sz, vp]
     l.metis_linear_fwd.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp, sz, vp]
     l.metis_linear_fwd_static_ws.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp]
     l.metis_linear_bwd.argtypes = [vp, P(OperandStruct), P(OperandStruct), P(OperandStruct), vp, i32, i64, vp, i32,
@@ -258,20 +259,21 @@ class Handle:
                                                 _stream_ptr(stream)))
         return (op, dense) if want_residual else op
 
-    def requantize_weight(self, src, residual_bf16, out, rounding=ROUND_RNE, seed=0, stream=None):
-        """Weights held as (left, sigma, right, residual) and only re-quantized each step (Section 3.2 keeps the
-        low-rank and residual parts of a weight as separate stored tensors): three metis_quantize_nvfp4 calls."""
-        k = src.k
-        self.quantize_nvfp4(residual_bf16, BLOCKS_BOTH, rounding, seed, STREAM_RESIDUAL,
-                            out=(out.res_by_cols, out.res_by_rows), stream=stream)
-        if k:
-            self.quantize_nvfp4(src.left[:k], BLOCKS_ALONG_COLS, rounding, seed, STREAM_LEFT, out=(out.left_q, None), stream=stream)
-            self.quantize_nvfp4(src.right[:k], BLOCKS_ALONG_COLS, rounding, seed, STREAM_RIGHT, out=(out.right_q, None), stream=stream)
-            if out is not src:
-                out.left.copy_(src.left)
-                out.right.copy_(src.right)
-                out.sigma.copy_(src.sigma)
-        return out
+    def requantize_operand(self, op, residual, rounding=ROUND_RNE, seed=0, axes=BLOCKS_BOTH, given_scale=None, stream=None):
+        """metis_requantize_operand: refreshes the NVFP4 members of `op` from its stored FP32 factors and the stored
+        `residual` (rows x cols, float32 or bfloat16).  given_scale: tensor scale of the residual (None = its own amax/2688)."""
+        mode = TSCALE_AMAX_SELF
+        if given_scale is not None:
+            mode = TSCALE_GIVEN
+            for o in (op.res_by_cols, op.res_by_rows):
+                if o is not None:
+                    o.tensor_scale.fill_(float(given_scale))
+        ws = self.workspace(256)
+        st = op.struct()
+        _check("metis_requantize_operand", lib().metis_requantize_operand(
+            self._h, _ptr(residual), _dtype_code(residual), residual.stride(0), rounding, seed, axes, mode, ctypes.byref(st),
+            _ptr(ws), ws.numel(), _stream_ptr(stream)))
+        return op
 
     # -- metis_linear_fwd / metis_linear_bwd ---------------------------------------------------
     def linear_fwd(self, x_op, w_op, out_dtype=torch.float32, out=None, stream=None):

@@ -217,6 +217,52 @@ metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dty
                                out_by_cols, out_by_rows, s);
 }
 
+metis_status_t metis_requantize_operand(metis_handle_t h, const void* residual, int32_t res_dtype, int64_t ld_res,
+                                        int32_t rounding, uint64_t seed, int32_t residual_axes, int32_t res_tscale,
+                                        metis_operand_t* op, void* ws, size_t ws_bytes, metis_stream_t stream) {
+  if (!h || !residual || !op) return METIS_ERR_INVALID_ARG;
+  if (res_dtype != METIS_BF16 && res_dtype != METIS_FP32) return METIS_ERR_INVALID_ARG;
+  if (rounding != METIS_ROUND_RNE && rounding != METIS_ROUND_SR) return METIS_ERR_INVALID_ARG;
+  if (res_tscale != METIS_TSCALE_AMAX_SELF && res_tscale != METIS_TSCALE_GIVEN) return METIS_ERR_INVALID_ARG;
+  const int64_t rows = op->rows, cols = op->cols;
+  const int k = op->k;
+  if (rows <= 0 || cols <= 0 || rows % 16 || cols % 16 || k < 0 || k > 256 || ld_res < cols) return METIS_ERR_SHAPE;
+  if (!metis_aligned16(residual)) return METIS_ERR_ALIGNMENT;
+  const bool want_c = (residual_axes & METIS_BLOCKS_ALONG_COLS) != 0, want_r = (residual_axes & METIS_BLOCKS_ALONG_ROWS) != 0;
+  if (!want_c && !want_r) return METIS_ERR_INVALID_ARG;
+  metis_nvfp4_t rc = op->res_by_cols, rr = op->res_by_rows;
+  rc.rows = rows; rc.k_len = cols; rr.rows = cols; rr.k_len = rows;
+  if (want_c && (!rc.codes || !rc.scales || !rc.tensor_scale || (rc.sf_layout == METIS_SF_TILED && cols % 64))) return METIS_ERR_INVALID_ARG;
+  if (want_r && (!rr.codes || !rr.scales || !rr.tensor_scale || (rr.sf_layout == METIS_SF_TILED && rows % 64))) return METIS_ERR_INVALID_ARG;
+  metis_nvfp4_t lq = op->left_q, rq = op->right_q;
+  if (k > 0) {
+    if (!op->left || !op->right || !op->sigma || !lq.codes || !lq.scales || !lq.tensor_scale || !rq.codes || !rq.scales || !rq.tensor_scale)
+      return METIS_ERR_INVALID_ARG;
+    if ((lq.sf_layout == METIS_SF_TILED && rows % 64) || (rq.sf_layout == METIS_SF_TILED && cols % 64)) return METIS_ERR_SHAPE;
+    lq.rows = k; lq.k_len = rows; rq.rows = k; rq.k_len = cols;
+  }
+  if (!ws || ws_bytes < 256 || !metis_aligned16(ws)) return METIS_ERR_WORKSPACE;
+  float* amax = static_cast<float*>(ws);                 // [0] residual, [1] left, [2] right
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const float* ts_src;
+  int is_amax = 0;
+  if (res_tscale == METIS_TSCALE_AMAX_SELF) {
+    METIS_TRY(metis_launch_amax(residual, res_dtype, rows, cols, ld_res, amax, s));
+    METIS_TRY(metis_launch_amax_check(h, amax, s));
+    ts_src = amax; is_amax = 1;
+  } else {
+    ts_src = want_c ? rc.tensor_scale : rr.tensor_scale;
+  }
+  METIS_TRY(metis_launch_quantize(residual, res_dtype, rows, cols, ld_res, rounding, seed, METIS_STREAM_RESIDUAL, cols, 1, ts_src, is_amax,
+                                  want_c ? &rc : nullptr, want_r ? &rr : nullptr, s));
+  if (k > 0) {
+    METIS_TRY(metis_launch_amax(op->left, METIS_FP32, k, rows, rows, amax + 1, s));
+    METIS_TRY(metis_launch_amax(op->right, METIS_FP32, k, cols, cols, amax + 2, s));
+    METIS_TRY(metis_launch_quantize_factors(op->left, rows, op->right, cols, k, rounding, seed, amax + 1, amax + 2, &lq, &rq, s));
+  }
+  return METIS_OK;
+}
+
 metis_status_t metis_gemm_nvfp4(metis_handle_t h, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d,
                                 int32_t d_dtype, int64_t ldd, int32_t impl, metis_stream_t stream) {
   if (!h || !a || !b || !d) return METIS_ERR_INVALID_ARG;

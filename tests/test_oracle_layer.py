@@ -194,3 +194,26 @@ def test_stochastic_rounding_config_runs_and_differs_from_rne():
     assert not np.array_equal(dq.res_by_cols, dq2.res_by_cols)
     ref = dq.split.residual
     assert metrics.rel_fro(dq.res_by_cols, ref) < 0.25
+
+
+def test_requantizing_the_stored_pieces_of_a_split_reproduces_the_split_operand():
+    """The persistent-operand route against the pinned one: the pieces that quantize_operand produced, stored in
+    float32 and quantized again with the residual's original tensor scale, give the same bytes piece by piece; with
+    the residual's own amax as scale (the stored-weight default) the residual changes scale but still covers every
+    block, and the factors are untouched."""
+    c, _, xq, _, _ = _ops()
+    sp = xq.split
+    s_src = nvfp4.tensor_scale_from_amax(np.max(np.abs(c["x"])))
+    res32 = sp.residual.astype(F32)
+    again = layer.requantize_operand(sp.left.astype(F32), sp.sigma, sp.right.astype(F32), res32, residual_scale=s_src)
+    for name in ("res_by_cols", "res_by_rows", "left", "right"):
+        for a, b in zip(again.raw[name], xq.raw[name]):
+            assert np.array_equal(a, b), name
+    assert np.array_equal(again.dense(nvfp4.AXIS_COLS), xq.dense(nvfp4.AXIS_COLS))
+    own = layer.requantize_operand(sp.left.astype(F32), sp.sigma, sp.right.astype(F32), res32)
+    assert own.raw["res_by_cols"][2] == nvfp4.tensor_scale_from_amax(np.max(np.abs(res32))) < s_src
+    assert np.array_equal(own.raw["left"][0], xq.raw["left"][0])
+    # own scale: the residual's largest element sits on code 6 of a scale-448 block and is reproduced to rounding
+    i, j = np.unravel_index(np.argmax(np.abs(res32)), res32.shape)
+    assert np.isclose(own.res_by_cols[i, j], res32[i, j], rtol=1e-6)
+    assert metrics.rel_fro(own.res_by_cols, res32) <= metrics.rel_fro(xq.res_by_cols, res32) * 1.05
