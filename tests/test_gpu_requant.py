@@ -31,6 +31,8 @@ def test_requantized_operand_matches_the_oracle_byte_for_byte(ctx, case):
     n, m, k, p, rounding = case
     w, _ = synth.llama_like(n, m, 0.02, 300 + k, rank=max(k, 8))
     wo, dense = h.split(to_dev_bf16(w), k, p, sketch=B.SKETCH_FULL, seed=2, rounding=rounding, want_residual=True)
+    if k == 0:
+        dense = to_dev_bf16(w).float()                   # a plain operand has no residual of its own: the tensor itself
     torch.cuda.synchronize()
     s_src = onv.tensor_scale_from_amax(np.max(np.abs(w)))
     first = {name: _bytes(getattr(wo, name)) for name in ("res_by_cols", "res_by_rows", "left_q", "right_q")}
