@@ -50,7 +50,22 @@ def llama_like(rows, cols, sigma, seed, rank=32):
     return planted(rows, cols, rank, s_top, s_top / 10.0, sigma, seed)
 
 
-# BASELINE configuration 0 (small, forward only) and 1 (one LLaMA-3-8B q_proj-shaped layer)
+def planted_device(rows, cols, rank, sigma, seed, device="cuda"):
+    """The llama_like recipe generated on the device with torch's seeded generator (benchmark-size matrices, where
+    the host generator would take minutes); returns a bfloat16 tensor.  Same structure, different random stream."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    u, _ = torch.linalg.qr(torch.randn((rows, rank), generator=g, device=device))
+    v, _ = torch.linalg.qr(torch.randn((cols, rank), generator=g, device=device))
+    s_top = 100.0 * sigma * (math.sqrt(rows) + math.sqrt(cols))
+    s = torch.logspace(math.log10(s_top), math.log10(s_top / 10.0), rank, device=device)
+    m = (u * s) @ v.T
+    m += sigma * torch.randn((rows, cols), generator=g, device=device)
+    return m.to(torch.bfloat16)
+
+
+# the small forward-only workload (128 tokens, 256 -> 256) and one LLaMA-3-8B q_proj-shaped layer
 def config_small(seed=1001):
     x, sx = planted(128, 256, 8, 200.0, 20.0, 1.0, seed)
     w, sw = planted(256, 256, 8, 200.0, 20.0, 1.0, seed + 1)
