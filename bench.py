@@ -188,8 +188,12 @@ class Workload:
     def __init__(self, name, spec, B, synth, handles, streams, weights_mode, world, rank, dw_sets=1):
         import torch
         self.torch, self.B, self.name, self.spec = torch, B, name, spec
-        self.h_x, self.h_w, self.h_d = handles
-        self.side_w, self.side_d = streams
+        # handles / streams: one for the activations and the forward products (the caller's current stream), N_SIDE
+        # for the weights and N_SIDE for the output gradients and the backward products (layer j uses side j % N_SIDE,
+        # so that the latency-bound start of one layer's decomposition runs beside the previous layer's big kernels)
+        self.h_x, self.h_ws, self.h_ds = handles
+        self.side_ws, self.side_ds = streams
+        self.h_w, self.h_d = self.h_ws[0], self.h_ds[0]
         self.l, self.k, self.p = spec["tokens"], spec["k"], spec["p"]
         self.layers = spec["layers"]
         self.weights_mode = weights_mode
@@ -223,7 +227,7 @@ class Workload:
         self.ev_start = torch.cuda.Event()
         self.ev_x = {g: torch.cuda.Event() for g in self.x_in}
         self.ev_w = [torch.cuda.Event() for _ in self.layers]
-        self.ev_b = torch.cuda.Event()
+        self.ev_b = [torch.cuda.Event() for _ in self.side_ds]
         self.flops = sum(6.0 * l * ly["d_in"] * ly["d_out"] for ly in self.layers)
         self.elements = {"x": sum(l * t.shape[1] for t in self.x_in.values()), "w": sum(t.numel() for t in self.w_in),
                          "dy": sum(t.numel() for t in self.d_in)}
@@ -239,15 +243,17 @@ class Workload:
         y, dx, dw = outs if outs is not None else (self.y, self.dx, self.dw_sets[dw_set])
         main = torch.cuda.current_stream()
         self.ev_start.record(main)
-        self.side_w.wait_event(self.ev_start)
-        self.side_d.wait_event(self.ev_start)
-        with torch.cuda.stream(self.side_w):
-            for j in range(len(self.layers)):
+        n_w, n_d = len(self.side_ws), len(self.side_ds)
+        for st in self.side_ws + self.side_ds:
+            st.wait_event(self.ev_start)
+        for j in range(len(self.layers)):
+            sw, hw = self.side_ws[j % n_w], self.h_ws[j % n_w]
+            with torch.cuda.stream(sw):
                 if self.w_stored is not None:
-                    self.h_w.requantize_operand(self.wo[j], self.w_stored[j], seed=3 * i + 2, stream=self.side_w)
+                    hw.requantize_operand(self.wo[j], self.w_stored[j], seed=3 * i + 2, stream=sw)
                 else:
-                    self.h_w.split(w_in[j], k, p, sketch=B.SKETCH_FULL, seed=3 * i + 2, rounding=B.ROUND_RNE, out=self.wo[j], stream=self.side_w)
-                self.ev_w[j].record(self.side_w)
+                    hw.split(w_in[j], k, p, sketch=B.SKETCH_FULL, seed=3 * i + 2, rounding=B.ROUND_RNE, out=self.wo[j], stream=sw)
+                self.ev_w[j].record(sw)
         done_x = set()
         for j, ly in enumerate(self.layers):
             g = ly["x"]
@@ -259,13 +265,15 @@ class Workload:
             self.h_x.linear_fwd(self.xo[g], self.wo[j], out=y[j])
             # the backward products need dY, X and W but not the forward product: they follow the dY decomposition on
             # its stream
-            with torch.cuda.stream(self.side_d):
-                self.h_d.split(d_in[j], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 3, rounding=B.ROUND_SR, out=self.do[j], stream=self.side_d)
-                self.side_d.wait_event(self.ev_x[g])
-                self.side_d.wait_event(self.ev_w[j])
-                self.h_d.linear_bwd(self.do[j], self.xo[g], self.wo[j], out=(dx[j], dw[j]), stream=self.side_d)
-        self.ev_b.record(self.side_d)
-        main.wait_event(self.ev_b)
+            sd, hd = self.side_ds[j % n_d], self.h_ds[j % n_d]
+            with torch.cuda.stream(sd):
+                hd.split(d_in[j], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 3, rounding=B.ROUND_SR, out=self.do[j], stream=sd)
+                sd.wait_event(self.ev_x[g])
+                sd.wait_event(self.ev_w[j])
+                hd.linear_bwd(self.do[j], self.xo[g], self.wo[j], out=(dx[j], dw[j]), stream=sd)
+        for ev, sd in zip(self.ev_b, self.side_ds):
+            ev.record(sd)
+            main.wait_event(ev)
 
     def gemm_pairs(self):
         out = []
@@ -299,6 +307,7 @@ def main():
     ap.add_argument("--workloads", default="all", help="comma-separated workload names (default: all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying CUDA graphs")
+    ap.add_argument("--side-streams", type=int, default=2, help="streams (and library handles) per operand kind for the weight and gradient decompositions")
     ap.add_argument("--sustain-seconds", type=float, default=1.0, help="length of the sustained timing loop of every workload")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -320,8 +329,10 @@ def main():
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    handles = (B.Handle(local_rank), B.Handle(local_rank), B.Handle(local_rank))     # one workspace owner per stream
-    streams = (torch.cuda.Stream(), torch.cuda.Stream())
+    n_side = max(1, args.side_streams)
+    handles = (B.Handle(local_rank), [B.Handle(local_rank) for _ in range(n_side)], [B.Handle(local_rank) for _ in range(n_side)])   # one workspace owner per stream
+    streams = ([torch.cuda.Stream() for _ in range(n_side)], [torch.cuda.Stream() for _ in range(n_side)])
+    all_handles = [handles[0]] + handles[1] + handles[2]
     comm_stream = torch.cuda.Stream()
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -355,7 +366,7 @@ def main():
             wl.step(i)
         barrier()
         status = 0
-        for h in handles:
+        for h in all_handles:
             status |= h.device_status()
         assert status == 0, "device status %d after warm-up of %s" % (status, name)
         l0 = B.launch_count()
@@ -452,7 +463,7 @@ def main():
         t_s1 = time.time()
         ms_sus = e0.elapsed_time(e1) / n_sus
         clocks_sus = sampler.summary(t_s0, t_s1)
-        for h in handles:
+        for h in all_handles:
             status |= h.device_status()
         ms, ms_sus = max_over_ranks([ms, ms_sus])
 
@@ -495,7 +506,7 @@ def main():
             "sustained": {"steps": n_sus, "ms_per_step": ms_sus, "effective_tflops": world * wl.flops / (ms_sus * 1e-3) / 1e12,
                           "clocks": clocks_sus, "ms_x_median_mhz": (ms_sus * clocks_sus["sm_mhz"]) if clocks_sus["sm_mhz"] else None},
             "clocks": clocks_timed, "launches_per_step": int(launches_per_step), "cuda_graph": bool(use_graph),
-            "input_sets": n_sets, "input_bytes_per_step": int(wl.input_bytes),
+            "input_sets": n_sets, "side_streams_per_kind": n_side, "input_bytes_per_step": int(wl.input_bytes),
             "plain_fp4_gemms": {"ms": ms_gemm, "tflops": wl.flops / (ms_gemm * 1e-3) / 1e12, "frac_of_fp4_peak": wl.flops / (ms_gemm * 1e-3) / 1e12 / fp4_peak},
             "split_overhead_vs_plain_gemms": ms / ms_gemm - 1.0,
             "largest_gemm": {"shape_mnk": [int(big[0].rows), int(big[1].rows), int(big[0].k_len)], "ms": ms_big,
