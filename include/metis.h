@@ -82,6 +82,7 @@ typedef enum { METIS_SF_LINEAR = 0, METIS_SF_TILED = 1 } metis_sf_layout_t;
 #define METIS_STREAM_RIGHT    0x12u
 #define METIS_STREAM_OMEGA    0x100u
 #define METIS_STREAM_SAMPLING 0x200u
+#define METIS_STREAM_SIGNS    0x300u
 
 typedef struct {
   uint8_t* codes;          /* rows * k_len / 2 bytes, K-major, 16-byte aligned                        */
@@ -170,6 +171,18 @@ metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dty
                                     int64_t ld, int32_t rounding, uint64_t seed, uint32_t stream_id,
                                     int32_t tscale, metis_nvfp4_t* out_by_cols, metis_nvfp4_t* out_by_rows,
                                     void* ws, size_t ws_bytes, metis_stream_t stream);
+
+/* Comparison recipe of Section 4 (the paper sets Metis against "a random Hadamard transform alongside SR"): every
+ * block of 16 consecutive elements of a row is rotated, y = H16 (s * x) / 4 with H16 the Sylvester Hadamard matrix
+ * and s random signs per column (bit 15 of the Philox draw of the column index, stream METIS_STREAM_SIGNS, so two
+ * operands quantized with the same seed share them and (x H D)(w H D)^T = x w^T), then quantized like
+ * metis_quantize_nvfp4 with blocks along the columns and tensor_scale = amax(y)/2688.  The transform is four
+ * butterfly stages in binary32 (distance 1, 2, 4, 8) and one multiplication by 1/4.  x: rows x cols (ld), BF16 or
+ * FP32, cols % 16 == 0 (% 64 for tiled scales).  Workspace: 256 bytes.  A same-box comparator for the spectral
+ * fidelity figures; not part of the split-FP4 layer. */
+metis_status_t metis_quantize_rht_nvfp4(metis_handle_t h, const void* x, int32_t dtype, int64_t rows, int64_t cols,
+                                        int64_t ld, int32_t rounding, uint64_t seed, uint32_t stream_id,
+                                        metis_nvfp4_t* out, void* ws, size_t ws_bytes, metis_stream_t stream);
 
 /* ---- split (Sections 3.1, 3.2) ------------------------------------------------------------ */
 

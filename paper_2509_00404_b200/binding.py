@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "ALIGNMENT", 4: "WORKS
 
 EXPORTED = ["metis_create", "metis_destroy", "metis_last_device_status", "metis_debug_quantile_table",
             "metis_debug_launch_count", "metis_debug_timestamp", "metis_debug_wait_timeout",
-            "metis_sf_bytes", "metis_workspace_bytes", "metis_default_sample_count", "metis_quantize_nvfp4",
+            "metis_sf_bytes", "metis_workspace_bytes", "metis_default_sample_count", "metis_quantize_nvfp4", "metis_quantize_rht_nvfp4",
             "metis_split", "metis_requantize_operand", "metis_linear_fwd", "metis_linear_fwd_static_ws", "metis_linear_bwd", "metis_gemm_nvfp4"]
 
 
@@ -78,6 +78,7 @@ def lib():
     l.metis_default_sample_count.restype = i64
     l.metis_quantize_nvfp4.argtypes = [vp, vp, i32, i64, i64, i64, i32, u64, u32, i32, P(NvFp4Struct), P(NvFp4Struct),
                                        vp, sz, vp]
+    l.metis_quantize_rht_nvfp4.argtypes = [vp, vp, i32, i64, i64, i64, i32, u64, u32, P(NvFp4Struct), vp, sz, vp]
     l.metis_split.argtypes = [vp, vp, i64, i64, i32, i32, i32, i64, u64, i32, i32, P(OperandStruct), vp, vp, sz, vp]
     l.metis_requantize_operand.argtypes = [vp, vp, i32, i64, i32, u64, i32, i32, P(OperandStruct), vp, sz, vp]
     l.metis_linear_fwd.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp, sz, vp]
@@ -244,6 +245,18 @@ class Handle:
             self._h, _ptr(x), _dtype_code(x), rows, cols, x.stride(0), rounding, seed, stream_id, mode,
             ctypes.byref(sc) if bc else None, ctypes.byref(sr) if br else None, _ptr(ws), ws.numel(), _stream_ptr(stream)))
         return bc, br
+
+    def quantize_rht_nvfp4(self, x, rounding=ROUND_SR, seed=0, stream_id=STREAM_RESIDUAL, layout=SF_TILED, out=None, stream=None):
+        """metis_quantize_rht_nvfp4: random Hadamard transform of every 16-block along the columns, then NVFP4 (the
+        comparison recipe).  Returns the NvFp4 object."""
+        rows, cols = x.shape
+        t = out if out is not None else NvFp4(rows, cols, layout)
+        st = t.struct()
+        ws = self.workspace(256)
+        _check("metis_quantize_rht_nvfp4", lib().metis_quantize_rht_nvfp4(
+            self._h, _ptr(x), _dtype_code(x), rows, cols, x.stride(0), rounding, seed, stream_id, ctypes.byref(st), _ptr(ws), ws.numel(),
+            _stream_ptr(stream)))
+        return t
 
     # -- metis_split ---------------------------------------------------------------------------
     def split(self, x, k, p, sketch=SKETCH_SAMPLED, n_sample=0, seed=0, rounding=ROUND_RNE, axes=BLOCKS_BOTH,

@@ -217,6 +217,21 @@ metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dty
                                out_by_cols, out_by_rows, s);
 }
 
+metis_status_t metis_quantize_rht_nvfp4(metis_handle_t h, const void* x, int32_t dtype, int64_t rows, int64_t cols, int64_t ld,
+                                        int32_t rounding, uint64_t seed, uint32_t stream_id, metis_nvfp4_t* out, void* ws,
+                                        size_t ws_bytes, metis_stream_t stream) {
+  if (!h || !x || !out || !out->codes || !out->scales || !out->tensor_scale) return METIS_ERR_INVALID_ARG;
+  if (dtype != METIS_BF16 && dtype != METIS_FP32) return METIS_ERR_INVALID_ARG;
+  if (rounding != METIS_ROUND_RNE && rounding != METIS_ROUND_SR) return METIS_ERR_INVALID_ARG;
+  if (out->sf_layout != METIS_SF_TILED && out->sf_layout != METIS_SF_LINEAR) return METIS_ERR_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || ld < cols || cols % 16 || (out->sf_layout == METIS_SF_TILED && cols % 64)) return METIS_ERR_SHAPE;
+  if (!metis_aligned16(out->codes)) return METIS_ERR_ALIGNMENT;
+  if (!ws || ws_bytes < 256) return METIS_ERR_WORKSPACE;
+  out->rows = rows; out->k_len = cols;
+  return metis_launch_quantize_rht(h, x, dtype, rows, cols, ld, rounding, seed, stream_id, out, static_cast<float*>(ws),
+                                   reinterpret_cast<cudaStream_t>(stream));
+}
+
 metis_status_t metis_requantize_operand(metis_handle_t h, const void* residual, int32_t res_dtype, int64_t ld_res,
                                         int32_t rounding, uint64_t seed, int32_t residual_axes, int32_t res_tscale,
                                         metis_operand_t* op, void* ws, size_t ws_bytes, metis_stream_t stream) {

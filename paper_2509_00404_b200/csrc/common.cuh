@@ -218,6 +218,8 @@ metis_status_t metis_launch_quantize_factors(const float* left, int64_t rows, co
                                              uint64_t seed, const float* amax_left, const float* amax_right,
                                              const metis_nvfp4_t* lq, const metis_nvfp4_t* rq, cudaStream_t s);
 metis_status_t metis_launch_amax_check(metis_context* ctx, const float* amax, cudaStream_t s);
+metis_status_t metis_launch_quantize_rht(metis_context* ctx, const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int rounding, uint64_t seed,
+                                         uint32_t stream_id, const metis_nvfp4_t* out, float* amax_ws, cudaStream_t s);
 bool metis_project_tc_usable(const void* x, const void* hsp, int64_t cols, int jp);
 int metis_project_slices(int64_t rows, int64_t cols);
 metis_status_t metis_launch_project_tc(metis_context* ctx, const void* x, int64_t rows, int64_t cols, const void* hsp, int jp,

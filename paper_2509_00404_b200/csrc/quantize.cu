@@ -307,6 +307,91 @@ quantize_rowblocks_kernel(const float* __restrict__ x, int64_t ld, metis_qt::Qua
   rowblocks_body(x, ld, p, tscale_src, tscale_is_amax, ts_out);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Comparison recipe of Section 4: random Hadamard transform of every 16-block along the columns, then NVFP4.
+// y = H16 (s * x) / 4, four butterfly stages in binary32 (distance 1, 2, 4, 8; (a, b) -> (a + b, a - b)), signs
+// s from bit 15 of the Philox draw of the column index (stream METIS_STREAM_SIGNS).
+__device__ __forceinline__ void rht_block(const void* __restrict__ x, int dtype, int64_t ld, int64_t r, int64_t b, uint64_t seed, float (&v)[16]) {
+  const uint4 w0 = metis_philox_block((uint64_t)b * 2, seed, METIS_STREAM_SIGNS), w1 = metis_philox_block((uint64_t)b * 2 + 1, seed, METIS_STREAM_SIGNS);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float xv = metis_ld_as_float(x, dtype, r * ld + b * 16 + i);
+    const uint32_t u = metis_u16_of(i < 8 ? w0 : w1, (uint32_t)(i & 7));
+    v[i] = (u & 0x8000u) ? -xv : xv;
+  }
+#pragma unroll
+  for (int h = 1; h < 16; h <<= 1) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+      if ((i & h) == 0) { const float a = v[i], c = v[i + h]; v[i] = __fadd_rn(a, c); v[i + h] = __fsub_rn(a, c); }
+  }
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(v[i], 0.25f);
+}
+
+__global__ void __launch_bounds__(256)
+rht_amax_kernel(const void* __restrict__ x, int dtype, int64_t rows, int64_t cols, int64_t ld, uint64_t seed, float* __restrict__ amax_out) {
+  const int64_t bpr = cols / 16;
+  const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  uint32_t m = 0u;
+  if (idx < rows * bpr) {
+    float v[16];
+    rht_block(x, dtype, ld, idx / bpr, idx % bpr, seed, v);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) m = max(m, __float_as_uint(v[i]) & 0x7FFFFFFFu);      // ordered bit patterns: a NaN survives
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  if ((threadIdx.x & 31) == 0 && m) atomicMax(reinterpret_cast<unsigned int*>(amax_out), m);
+}
+
+__global__ void __launch_bounds__(256)
+rht_quantize_kernel(const void* __restrict__ x, int dtype, int64_t ld, metis_qt::QuantParams p, const float* __restrict__ amax, float* ts_out) {
+  const int64_t bpr = p.cols / 16;
+  const int64_t rows_pad = p.c_layout == METIS_SF_TILED ? (p.rows + 127) / 128 * 128 : p.rows;
+  const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= rows_pad * bpr) return;
+  const int64_t r = idx / bpr, b = idx % bpr;
+  if (r >= p.rows) { p.c_scales[metis_sf_offset(r, b, bpr, p.c_layout)] = 0; return; }
+  const float s_T = metis_tensor_scale(*amax);
+  if (idx == 0) *ts_out = s_T;
+  const bool sr = p.rounding == METIS_ROUND_SR;
+  float v[16];
+  uint32_t u[16];
+  rht_block(x, dtype, ld, r, b, p.seed, v);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) u[i] = 0u;
+  if (sr) {
+    const uint64_t e0 = (uint64_t)r * (uint64_t)p.cols + (uint64_t)b * 16u;
+#pragma unroll
+    for (int h2 = 0; h2 < 2; ++h2) {
+      const uint4 w = metis_philox_block((e0 >> 3) + h2, p.seed, p.stream_id);
+#pragma unroll
+      for (uint32_t hh = 0; hh < 8; ++hh) u[8 * h2 + hh] = metis_u16_of(w, hh);
+    }
+  }
+  uint32_t packed[2];
+  const uint32_t byte = metis_qt::encode_block(v, u, sr, s_T, __fmul_rn(6.0f, s_T), packed);
+  *reinterpret_cast<uint2*>(p.c_codes + r * (p.cols / 2) + b * 8) = make_uint2(packed[0], packed[1]);
+  p.c_scales[metis_sf_offset(r, b, bpr, p.c_layout)] = (uint8_t)byte;
+}
+
+metis_status_t metis_launch_quantize_rht(metis_context* ctx, const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int rounding, uint64_t seed,
+                                         uint32_t stream_id, const metis_nvfp4_t* out, float* amax_ws, cudaStream_t s) {
+  using namespace metis_qt;
+  QuantParams p{};
+  p.rows = rows; p.cols = cols; p.rounding = rounding; p.seed = seed; p.stream_id = stream_id; p.e_stride_r = cols; p.e_stride_c = 1;
+  p.c_codes = out->codes; p.c_scales = out->scales; p.c_layout = out->sf_layout;
+  METIS_CUDA_TRY(cudaMemsetAsync(amax_ws, 0, sizeof(float), s));
+  const int64_t bpr = cols / 16;
+  rht_amax_kernel<<<(unsigned)metis_ceil_div(rows * bpr, 256), 256, 0, s>>>(x, dtype, rows, cols, ld, seed, amax_ws); METIS_COUNT_LAUNCH();
+  METIS_TRY(metis_launch_amax_check(ctx, amax_ws, s));
+  const int64_t rows_pad = p.c_layout == METIS_SF_TILED ? (rows + 127) / 128 * 128 : rows;
+  rht_quantize_kernel<<<(unsigned)metis_ceil_div(rows_pad * bpr, 256), 256, 0, s>>>(x, dtype, ld, p, amax_ws, out->tensor_scale); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
+
 // two factor tensors in one launch (blockIdx.y selects): the left and right factors of a decomposition
 struct RowblocksJob { const float* x; int64_t ld; metis_qt::QuantParams p; const float* tscale_src; float* ts_out; };
 __global__ void __launch_bounds__(256)

@@ -103,3 +103,31 @@ def test_quantile_table_matches_oracle(ctx):
     B, h = ctx
     ref = gauss.quantile_level(np.arange(65536))
     assert np.array_equal(h.quantile_table(), (ref.view(np.uint32) >> 16).astype(np.uint16))
+
+
+@pytest.mark.parametrize("case", [(128, 256, 1, "bf16"), (200, 192, 0, "fp32"), (1024, 4096, 1, "bf16")], ids=lambda c: "%dx%d_%s_%s" % (c[0], c[1], "sr" if c[2] else "rne", c[3]))
+def test_random_hadamard_recipe_matches_the_oracle_byte_for_byte(case):
+    """The comparison recipe of Section 4 (random Hadamard transform of every 16-block, then NVFP4 with stochastic
+    rounding): codes, scale bytes and tensor scale against the oracle, and the product-preserving property on the
+    GPU's own bytes."""
+    from oracle import hadamard as ohad
+    from gpu_util import nv_to_numpy
+    from paper_2509_00404_b200 import binding as B, synth
+    rows, cols, rounding, dt = case
+    x, _ = synth.llama_like(rows, cols, 1.0, 900 + rows, rank=8)
+    if dt == "fp32":
+        x = (x * np.float32(1.2345)).astype(np.float32)
+    xd = torch.from_numpy(x).cuda() if dt == "fp32" else torch.from_numpy(x).to(torch.bfloat16).cuda()
+    h = B.Handle(0)
+    try:
+        layout = B.SF_TILED if cols % 64 == 0 else B.SF_LINEAR
+        t = h.quantize_rht_nvfp4(xd, rounding=rounding, seed=17, layout=layout)
+        torch.cuda.synchronize()
+        assert h.device_status() == 0
+        c, s, ts = nv_to_numpy(t)
+        oc, os_, ots = ohad.quantize_rht(x, rounding, seed=17)
+        assert ts == ots and np.array_equal(s, os_) and np.array_equal(c, oc)
+        back = ohad.rht_inverse(onv.dequantize(c, s, ts), 17)
+        assert np.linalg.norm(back - x) / np.linalg.norm(x) < 0.2
+    finally:
+        h.close()
