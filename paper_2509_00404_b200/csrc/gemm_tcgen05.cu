@@ -273,6 +273,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 namespace two_cta {
 
 constexpr int TILE_M = 256, TILE_N = 256;
+constexpr int RASTER_M = 8;                                 // row tiles per raster group (see the tile order in the kernel)
 constexpr int STAGES = 5;
 constexpr int A_BYTES = 128 * BLOCK_K / 2;                  // this CTA's 128 rows of A
 constexpr int B_BYTES = 128 * BLOCK_K / 2;                  // this CTA's 128 rows of B
@@ -404,7 +405,16 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     int tile = item;
     nhalf = -1;
     if (split_tail && item >= full_items) { tile = full_items + ((item - full_items) >> 1); nhalf = (item - full_items) & 1; }
-    mb = tile % num_m; nb = tile / num_m;
+    // Tile order: groups of RASTER_M row tiles, inside a group the row tile runs fastest and the column tile sweeps
+    // the whole width.  The pairs that run at the same time then cover RASTER_M x ~9 tiles: the group's A strips stay
+    // in L2 for the whole sweep and every B strip is used by RASTER_M tiles back to back.  (With the row tile
+    // running fastest over ALL rows, a wave touched every A strip once, and at long contractions - 2 MB per strip,
+    // more than the L2 in all - each sweep of the columns read A from DRAM again: 2 GB instead of 165 MB at
+    // 16384 x 4096 x 14336.)
+    const int per_group = RASTER_M * num_n;
+    const int grp = tile / per_group, within = tile - grp * per_group;
+    const int first_m = grp * RASTER_M, gsz = min(RASTER_M, num_m - first_m);
+    mb = first_m + within % gsz; nb = within / gsz;
   };
   const int num_fp4_kb = (g.K + BLOCK_K - 1) / BLOCK_K;
   const int num_kb = num_fp4_kb + g.extra_kb;
@@ -539,6 +549,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     // MMAs start while this tile is still being scaled, converted and stored.
     const int quarter = warp & 3, half = (warp - 4) >> 2;
     const float alpha = (*g.a_ts) * (*g.b_ts);
+    const uint64_t out_policy = l2_policy_evict_first();
     int it = 0;
     bool ok = true;
     for (int item = pair; item < num_items && ok; item += num_pairs, ++it) {
@@ -593,7 +604,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
               fence_proxy_async();
               __syncwarp();
               if (lane == 0 && row_w < g.M && col_w + st * 64 < g.N) {
-                tma_store_2d(&map_d, obuf, col_w + st * 64, row_w);
+                tma_store_2d_hint(&map_d, obuf, col_w + st * 64, row_w, out_policy);
                 bulk_commit();
               }
             }
@@ -612,7 +623,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
               fence_proxy_async();
               __syncwarp();
               if (lane == 0 && row_w < g.M && col_w + st * 32 < g.N) {
-                tma_store_2d(&map_d, obuf, col_w + st * 32, row_w);
+                tma_store_2d_hint(&map_d, obuf, col_w + st * 32, row_w, out_policy);
                 bulk_commit();
               }
             }
