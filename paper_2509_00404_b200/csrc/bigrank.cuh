@@ -3,9 +3,11 @@
 // (Section 3.1: thin QR of the sketch, small SVD of the projected operand), as kernels that tile over the rank:
 //
 //   gram64_kernel            G = V^T V in FP64, 64 x 64 output tiles over slabs of rows (partials, summed in order)
-//   chol_wide_kernel         Cholesky factor of a q x q Gram matrix and its triangular inverse, one CTA, matrix in L2
-//   gemm64_kernel            C = A B with FP32 A, FP64 B and FP64 accumulation, arbitrary strides (triangular solve
-//                            H = Z L^-T as a product, right basis, factor rotations)
+//   chol_wide_kernel         blocked Cholesky factor of a q x q Gram matrix (panels of 32 columns in shared memory,
+//                            the matrix in L2) and the inverses of its diagonal blocks, one CTA
+//   trsm_wide_kernel         H = Z L^-T by blocked forward substitution (32 rows of Z per CTA)
+//   gemm64_kernel            C = A B with FP32 A, FP64 B and FP64 accumulation, arbitrary strides (right basis,
+//                            factor rotations)
 //   jacobi_cluster_kernel    one-sided Jacobi eigen-solver on a cluster of eight CTAs: the columns live in the
 //                            cluster's distributed shared memory, column blocks travel between CTAs by DSMEM stores
 //   jacobi_collect_kernel    eigenvalues (descending) and normalised eigenvectors from the rotated columns
@@ -74,83 +76,160 @@ gram64_kernel(const float* __restrict__ v, int64_t n_rows, int n, int64_t sr, in
 }
 
 // ------------------------------------------------------------------------------------------------
-// Cholesky factor of the n x n Gram matrix g (n <= MAXQ_WIDE) and, when asked, its inverse, one CTA of 1024 threads.
-// The matrix does not fit one CTA's shared memory in FP64, so it stays in global memory (it is L2-resident: half a
-// megabyte) and the CTA works column by column, left-looking: column j is the Gram column minus the contributions
-// of the columns before it, four lanes per row sharing the inner product.  A pivot not above tol_rel * (largest
-// diagonal entry) marks a dependent sketch column: its column of L and its row and column of L^-1 are zero.
-//   l_out    n x n row-major lower factor (strict upper part zero)
-//   linv_out n x n row-major L^-1 (lower), or NULL
+// Cholesky factor of the n x n Gram matrix g (n <= MAXQ_WIDE), one CTA of 1024 threads, blocked by panels of
+// CW_NB columns (left-looking): a panel is the Gram panel minus the product of the finished columns of its rows
+// with those of its own CW_NB rows - staged through shared memory in chunks of CW_NB columns, so the finished
+// part of L is read once per panel - and is then factorised inside shared memory.  The matrix itself (half a
+// megabyte in FP64) stays in global memory.  A pivot not above tol_rel * (largest diagonal entry) marks a
+// dependent sketch column: its column of L and its row and column of the diagonal-block inverse are zero.
+//   l_out     n x n row-major lower factor (strict upper part zero)
+//   dinv_out  (optional) inverses of the CW_NB x CW_NB diagonal blocks of L, [panel][CW_NB][CW_NB] row-major lower:
+//             what the triangular solve H = Z L^-T needs besides L itself (trsm_wide_kernel)
 //   well_conditioned  (optional) 1 when every pivot is above 1e-8 of the largest diagonal entry
+constexpr int CW_NB = 32, CW_P = CW_NB + 1;
+constexpr size_t CW_SMEM = sizeof(double) * ((size_t)2 * MAXQ_WIDE * CW_P + CW_NB * CW_P + MAXQ_WIDE);
 __global__ void __launch_bounds__(1024, 1)
-chol_wide_kernel(const double* __restrict__ g, int n, double tol_rel, double* l_out, double* linv_out,
+chol_wide_kernel(const double* __restrict__ g, int n, double tol_rel, double* l_out, double* dinv_out,
                  const int* __restrict__ skip, int* __restrict__ well_conditioned) {
   metis_pdl_wait();
   if (skip != nullptr && *skip) return;
-  __shared__ double rowj[MAXQ_WIDE];                    // row j of L (entries before the diagonal)
-  __shared__ double vbuf[MAXQ_WIDE];                    // column j before scaling
-  __shared__ double rinv[MAXQ_WIDE];                    // 1 / L[j][j], or 0 for a dependent column
+  extern __shared__ __align__(16) unsigned char cw_sm[];
+  double (*P)[CW_P] = reinterpret_cast<double (*)[CW_P]>(cw_sm);                                   // the panel, rows j0 .. n-1
+  double (*As)[CW_P] = reinterpret_cast<double (*)[CW_P]>(cw_sm + sizeof(double) * MAXQ_WIDE * CW_P);    // a chunk of finished columns of those rows
+  double (*Dv)[CW_P] = reinterpret_cast<double (*)[CW_P]>(cw_sm + sizeof(double) * 2 * MAXQ_WIDE * CW_P);
+  double* rinv = reinterpret_cast<double*>(cw_sm + sizeof(double) * (2 * MAXQ_WIDE * CW_P + CW_NB * CW_P));
   __shared__ double red[32];
   __shared__ double gmax_s, dmin_s;
-  const int tid = threadIdx.x, lane4 = tid & 3, rgrp = tid >> 2;      // 256 row slots of four lanes
-  for (int o = tid; o < n * n; o += 1024) {
-    const int i = o / n, j = o % n;
-    l_out[o] = j <= i ? 0.5 * (g[(int64_t)i * n + j] + g[(int64_t)j * n + i]) : 0.0;
-  }
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  for (int o = tid; o < n * n; o += 1024) l_out[o] = 0.0;
   double gm = 0.0;
   for (int i = tid; i < n; i += 1024) gm = fmax(gm, g[(int64_t)i * n + i]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) gm = fmax(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, o));
-  if ((tid & 31) == 0) red[tid >> 5] = gm;
+  if (lane == 0) red[warp] = gm;
   __syncthreads();
   if (tid == 0) { double m = 0.0; for (int w = 0; w < 32; ++w) m = fmax(m, red[w]); gmax_s = m; dmin_s = 1e300; }
   __syncthreads();
   const double tol = tol_rel * gmax_s;
-  for (int j = 0; j < n; ++j) {
-    for (int k = tid; k < j; k += 1024) rowj[k] = l_out[(int64_t)j * n + k];
-    __syncthreads();
-    for (int i = j + rgrp; i < n; i += 256) {
-      const double* li = l_out + (int64_t)i * n;
-      double s0 = 0.0, s1 = 0.0;
-      int k = lane4;
-      for (; k + 4 < j; k += 8) { s0 += li[k] * rowj[k]; s1 += li[k + 4] * rowj[k + 4]; }
-      if (k < j) s0 += li[k] * rowj[k];
-      double s = s0 + s1;
-      // the four lanes of a row run this loop together; other rows of the warp may already have left it
-      const unsigned grp_mask = 0xFu << ((tid & 31) & ~3);
-      s += __shfl_xor_sync(grp_mask, s, 1);
-      s += __shfl_xor_sync(grp_mask, s, 2);
-      if (lane4 == 0) vbuf[i] = li[j] - s;
+  const int tr = warp, tc = lane;                           // thread: panel column tc, rows tr + 32 m
+  constexpr int RM = (MAXQ_WIDE + 31) / 32;
+  for (int j0 = 0; j0 < n; j0 += CW_NB) {
+    const int w = min(CW_NB, n - j0), nr = n - j0;
+    for (int o = tid; o < nr * CW_NB; o += 1024) {
+      const int i = o / CW_NB, c = o % CW_NB;
+      P[i][c] = c < w ? 0.5 * (g[(int64_t)(j0 + i) * n + j0 + c] + g[(int64_t)(j0 + c) * n + j0 + i]) : 0.0;
+    }
+    double acc[RM];
+#pragma unroll
+    for (int m = 0; m < RM; ++m) acc[m] = 0.0;
+    for (int k0 = 0; k0 < j0; k0 += CW_NB) {
+      __syncthreads();
+      for (int o = tid; o < nr * CW_NB; o += 1024) { const int i = o / CW_NB, kk = o % CW_NB; As[i][kk] = l_out[(int64_t)(j0 + i) * n + k0 + kk]; }
+      __syncthreads();
+      if (tc < w) {
+#pragma unroll 4
+        for (int kk = 0; kk < CW_NB; ++kk) {
+          const double b = As[tc][kk];                      // rows j0 .. j0 + w - 1 of L are the first rows of the chunk
+#pragma unroll
+          for (int m = 0; m < RM; ++m) if (tr + 32 * m < nr) acc[m] += As[tr + 32 * m][kk] * b;
+        }
+      }
     }
     __syncthreads();
-    const double d = vbuf[j];
-    const double r = d > tol ? 1.0 / sqrt(d) : 0.0;
-    for (int i = j + tid; i < n; i += 1024) l_out[(int64_t)i * n + j] = i == j ? d * r : vbuf[i] * r;
-    if (tid == 0) { rinv[j] = r; if (d > tol) dmin_s = fmin(dmin_s, d); }
+    if (tc < w) {
+#pragma unroll
+      for (int m = 0; m < RM; ++m) if (tr + 32 * m < nr) P[tr + 32 * m][tc] -= acc[m];
+    }
+    __syncthreads();
+    for (int c = 0; c < w; ++c) {
+      const double d = P[c][c];
+      const double r = d > tol ? 1.0 / sqrt(d) : 0.0;
+      __syncthreads();                                     // everybody has read the pivot
+      for (int i = c + tid; i < nr; i += 1024) P[i][c] = i == c ? d * r : P[i][c] * r;
+      if (tid == 0) { rinv[j0 + c] = r; if (d > tol) dmin_s = fmin(dmin_s, d); }
+      __syncthreads();
+      const int rest = w - c - 1;
+      for (int o = tid; o < (nr - c - 1) * rest; o += 1024) {
+        const int i = c + 1 + o / rest, cp = c + 1 + o % rest;
+        if (i >= cp) P[i][cp] -= P[i][c] * P[cp][c];
+      }
+      __syncthreads();                                     // the next pivot is final
+    }
+    for (int o = tid; o < nr * w; o += 1024) {
+      const int i = o / w, c = o % w;
+      if (i >= c) l_out[(int64_t)(j0 + i) * n + j0 + c] = P[i][c];
+    }
+    if (dinv_out != nullptr) {
+      // inverse of the diagonal block, one lane per column: X[j][j] = 1 / L[j][j], X[i][j] = -X[i][i] sum_{k=j}^{i-1} L[i][k] X[k][j]
+      if (warp == 0) {
+        for (int i = 0; i < CW_NB; ++i) Dv[i][lane] = 0.0;
+        if (lane < w) {
+          Dv[lane][lane] = rinv[j0 + lane];
+          for (int i = lane + 1; i < w; ++i) {
+            double sacc = 0.0;
+            for (int k = lane; k < i; ++k) sacc += P[i][k] * Dv[k][lane];
+            Dv[i][lane] = -rinv[j0 + i] * sacc;
+          }
+        }
+      }
+      __syncthreads();
+      for (int o = tid; o < CW_NB * CW_NB; o += 1024) dinv_out[(int64_t)(j0 / CW_NB) * CW_NB * CW_NB + o] = Dv[o / CW_NB][o % CW_NB];
+    }
     __syncthreads();
   }
   if (tid == 0 && well_conditioned != nullptr) *well_conditioned = (dmin_s > 1e-8 * gmax_s) ? 1 : 0;
-  if (linv_out == nullptr) return;
-  // L^-1 row by row: X[i][i] = 1/L[i][i], X[i][j] = -X[i][i] * sum_{k=j}^{i-1} L[i][k] X[k][j]   (j < i)
-  for (int o = tid; o < n * n; o += 1024) linv_out[o] = 0.0;
-  __syncthreads();
-  const int jj = tid & 255, sl = tid >> 8;              // column slot, one of four slices of the k range
-  __shared__ double psum[4][MAXQ_WIDE];
-  for (int i = 0; i < n; ++i) {
-    for (int k = tid; k < i; k += 1024) rowj[k] = l_out[(int64_t)i * n + k];
-    __syncthreads();
-    for (int j = jj; j < i; j += 256) {
-      double s0 = 0.0, s1 = 0.0;
-      int k = j + sl;
-      for (; k + 4 < i; k += 8) { s0 += rowj[k] * linv_out[(int64_t)k * n + j]; s1 += rowj[k + 4] * linv_out[(int64_t)(k + 4) * n + j]; }
-      if (k < i) s0 += rowj[k] * linv_out[(int64_t)k * n + j];
-      psum[sl][j] = s0 + s1;
+}
+
+// H = Z L^-T by blocked forward substitution, in place: for panel J of CW_NB columns
+//   h_J = (z_J - sum_{K < J} h_K L[J][K]^T) Dinv_J^T.
+// A CTA owns 32 rows of Z and keeps their finished part of H in shared memory (FP64); L is read in CW_NB x CW_NB
+// chunks.  l, dinv: outputs of chol_wide_kernel.  FP32 in, FP64 arithmetic, FP32 out.
+constexpr int TW_ROWS = 32, TW_HP = MAXQ_WIDE + 1;
+constexpr size_t TW_SMEM = sizeof(double) * ((size_t)TW_ROWS * TW_HP + 3 * CW_NB * CW_P);
+__global__ void __launch_bounds__(256)
+trsm_wide_kernel(float* __restrict__ z, int64_t n_rows, int n, const double* __restrict__ l, const double* __restrict__ dinv) {
+  metis_pdl_wait();
+  extern __shared__ __align__(16) unsigned char tw_sm[];
+  double (*Hs)[TW_HP] = reinterpret_cast<double (*)[TW_HP]>(tw_sm);
+  double (*Ls)[CW_P] = reinterpret_cast<double (*)[CW_P]>(tw_sm + sizeof(double) * TW_ROWS * TW_HP);
+  double (*Ds)[CW_P] = Ls + CW_NB;
+  double (*Ts)[CW_P] = Ls + 2 * CW_NB;
+  const int tid = threadIdx.x, tr = tid >> 5, tc = tid & 31;       // rows tr + 8 m, column tc of the panel
+  const int64_t r0 = (int64_t)blockIdx.x * TW_ROWS;
+  for (int j0 = 0; j0 < n; j0 += CW_NB) {
+    const int w = min(CW_NB, n - j0);
+    double acc[4];
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+      const int64_t r = r0 + tr + 8 * m;
+      acc[m] = (r < n_rows && tc < w) ? (double)z[r * n + j0 + tc] : 0.0;
+    }
+    for (int k0 = 0; k0 < j0; k0 += CW_NB) {
+      __syncthreads();
+      for (int o = tid; o < CW_NB * CW_NB; o += 256) { const int c = o / CW_NB, kk = o % CW_NB; Ls[c][kk] = c < w ? l[(int64_t)(j0 + c) * n + k0 + kk] : 0.0; }
+      __syncthreads();
+#pragma unroll 8
+      for (int kk = 0; kk < CW_NB; ++kk) {
+        const double lv = Ls[tc][kk];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) acc[m] -= Hs[tr + 8 * m][k0 + kk] * lv;
+      }
     }
     __syncthreads();
-    const double ri = rinv[i];
-    for (int j = tid; j <= i; j += 1024)
-      linv_out[(int64_t)i * n + j] = j == i ? ri : -ri * (((psum[0][j] + psum[1][j]) + psum[2][j]) + psum[3][j]);
+    for (int o = tid; o < CW_NB * CW_NB; o += 256) Ds[o / CW_NB][o % CW_NB] = dinv[(int64_t)(j0 / CW_NB) * CW_NB * CW_NB + o];
+#pragma unroll
+    for (int m = 0; m < 4; ++m) Ts[tr + 8 * m][tc] = acc[m];
     __syncthreads();
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+      double sacc = 0.0;
+      for (int cp = 0; cp <= tc; ++cp) sacc += Ts[tr + 8 * m][cp] * Ds[tc][cp];
+      const int64_t r = r0 + tr + 8 * m;
+      if (tc < w) {
+        Hs[tr + 8 * m][j0 + tc] = sacc;
+        if (r < n_rows) z[r * n + j0 + tc] = (float)sacc;
+      }
+    }
   }
 }
 
@@ -264,6 +343,22 @@ __device__ __forceinline__ void jc_pair(int I, int step, int np, int* p, int* q)
   *p = min(a, b); *q = max(a, b);
 }
 
+// Rotation that makes two columns with squared norms a, b and inner product c orthogonal: the smaller root of
+// tan(2 theta) = 2c / (b - a), |theta| <= pi / 4.  The FP32 quantities only steer convergence (fast reciprocal square
+// roots); (cs, sn) is made a unit vector to ~1e-14 by one Newton step in FP64; tf = tan(theta) updates the carried norms.
+__device__ __forceinline__ void jc_rotation(float a, float b, float cf, double& cs, double& sn, float& tf) {
+  const float d = b - a, c2 = 2.0f * cf;
+  const float h2 = fmaf(c2, c2, d * d);
+  const float rh = rsqrtf(h2);
+  const float cc = fmaf(0.5f * fabsf(d), rh, 0.5f);
+  const float rs = rsqrtf(cc);
+  const float c32 = cc * rs, s32 = (d < 0.0f ? -c2 : c2) * (0.5f * rh) * rs;
+  tf = s32 * rs;
+  const double cd = (double)c32, sd = (double)s32;
+  const double scale = 1.5 - 0.5 * (cd * cd + sd * sd);
+  cs = cd * scale; sn = sd * scale;
+}
+
 __global__ void __cluster_dims__(JC_P, 1, 1) __launch_bounds__(JC_THREADS, 1)
 jacobi_cluster_kernel(const double* __restrict__ l, int n, float exit_cos2, double* __restrict__ ycm) {
   metis_pdl_wait();
@@ -298,45 +393,71 @@ jacobi_cluster_kernel(const double* __restrict__ l, int n, float exit_cos2, doub
         if (lane == 0) nrm[sc / JC_W][sc % JC_W] = (float)a;
       }
       __syncthreads();
-      const int rounds = orr == 0 ? 2 * JC_W - 1 : JC_W;
-      for (int r = 0; r < rounds; ++r) {
-        int ps, pc, qs, qc;
-        if (orr == 0) {
+      if (orr == 0) {
+        // every pair among the CTA's 2 * JC_W columns: round-robin tournament, both columns of a couple through shared memory
+        for (int r = 0; r < 2 * JC_W - 1; ++r) {
           int p, q;
           jc_pair(warp, r, 2 * JC_W, &p, &q);
-          ps = p / JC_W; pc = p % JC_W; qs = q / JC_W; qc = q % JC_W;
-        } else {
-          ps = 0; pc = warp; qs = 1; qc = (warp + r) % JC_W;
-        }
-        double* yp_s = col_ptr(cur, ps, pc);
-        double* yq_s = col_ptr(cur, qs, qc);
-        double yp[JC_RL], yq[JC_RL];
-        double c = 0.0;
+          const int ps = p / JC_W, pc = p % JC_W, qs = q / JC_W, qc = q % JC_W;
+          double* yp_s = col_ptr(cur, ps, pc);
+          double* yq_s = col_ptr(cur, qs, qc);
+          double yp[JC_RL], yq[JC_RL];
+          double c = 0.0;
 #pragma unroll
-        for (int t = 0; t < JC_RL; ++t) { yp[t] = yp_s[lane + 32 * t]; yq[t] = yq_s[lane + 32 * t]; c += yp[t] * yq[t]; }
+          for (int t = 0; t < JC_RL; ++t) { yp[t] = yp_s[lane + 32 * t]; yq[t] = yq_s[lane + 32 * t]; c += yp[t] * yq[t]; }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
-        const float a = nrm[ps][pc], b = nrm[qs][qc], cf = (float)c;
-        if (cf * cf > 1e-26f * (a * b)) {
-          const float d = b - a, c2 = 2.0f * cf;
-          const float h2 = fmaf(c2, c2, d * d);
-          const float rh = rsqrtf(h2);
-          const float cc = fmaf(0.5f * fabsf(d), rh, 0.5f);
-          const float rs = rsqrtf(cc);
-          const float c32 = cc * rs, s32 = (d < 0.0f ? -c2 : c2) * (0.5f * rh) * rs;
-          const float tf = s32 * rs;
-          const double cd = (double)c32, sd = (double)s32;
-          const double scale = 1.5 - 0.5 * (cd * cd + sd * sd);
-          const double cs = cd * scale, sn = sd * scale;
+          for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+          const float a = nrm[ps][pc], b = nrm[qs][qc], cf = (float)c;
+          if (cf * cf > 1e-26f * (a * b)) {
+            double cs, sn; float tf;
+            jc_rotation(a, b, cf, cs, sn, tf);
 #pragma unroll
-          for (int t = 0; t < JC_RL; ++t) {
-            yp_s[lane + 32 * t] = cs * yp[t] - sn * yq[t];
-            yq_s[lane + 32 * t] = sn * yp[t] + cs * yq[t];
+            for (int t = 0; t < JC_RL; ++t) {
+              yp_s[lane + 32 * t] = cs * yp[t] - sn * yq[t];
+              yq_s[lane + 32 * t] = sn * yp[t] + cs * yq[t];
+            }
+            const float tc = tf * cf;
+            if (lane == 0) { nrm[ps][pc] = a - tc; nrm[qs][qc] = b + tc; }
+            above |= cf * cf > exit_cos2 * (a * b);
           }
-          const float tc = tf * cf;
-          if (lane == 0) { nrm[ps][pc] = a - tc; nrm[qs][qc] = b + tc; }
-          above |= cf * cf > exit_cos2 * (a * b);
+          __syncthreads();
         }
+      } else {
+        // every pair of one column of each block: warp w keeps column w of the first block in registers for all
+        // JC_W rounds (nobody else touches it) and meets the columns of the second block one after the other
+        double* yp_s = col_ptr(cur, 0, warp);
+        double yp[JC_RL];
+#pragma unroll
+        for (int t = 0; t < JC_RL; ++t) yp[t] = yp_s[lane + 32 * t];
+        float a = nrm[0][warp];
+        for (int r = 0; r < JC_W; ++r) {
+          const int qc = (warp + r) % JC_W;
+          double* yq_s = col_ptr(cur, 1, qc);
+          double yq[JC_RL];
+          double c = 0.0;
+#pragma unroll
+          for (int t = 0; t < JC_RL; ++t) { yq[t] = yq_s[lane + 32 * t]; c += yp[t] * yq[t]; }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+          const float b = nrm[1][qc], cf = (float)c;
+          if (cf * cf > 1e-26f * (a * b)) {
+            double cs, sn; float tf;
+            jc_rotation(a, b, cf, cs, sn, tf);
+#pragma unroll
+            for (int t = 0; t < JC_RL; ++t) {
+              const double np_ = cs * yp[t] - sn * yq[t];
+              yq_s[lane + 32 * t] = sn * yp[t] + cs * yq[t];
+              yp[t] = np_;
+            }
+            const float tc = tf * cf;
+            above |= cf * cf > exit_cos2 * (a * b);
+            if (lane == 0) nrm[1][qc] = b + tc;
+            a -= tc;
+          }
+          __syncthreads();
+        }
+#pragma unroll
+        for (int t = 0; t < JC_RL; ++t) yp_s[lane + 32 * t] = yp[t];
         __syncthreads();
       }
       const bool last = orr == 2 * JC_P - 2;

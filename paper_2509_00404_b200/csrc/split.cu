@@ -1563,7 +1563,7 @@ int jacobi_threads(int n) {
 // rows gathered once (SAMPLED) - so that sketch and projection both run on the tcgen05 kernel of the broadcast
 // pass, in groups of sketch columns.
 struct WideWs {
-  size_t amax, idx, xs, omt, zp, z, z2, gram, gram1, l, linv, evals, evecs, ycm, scale, hsp, mp, m, basis, bs, coef, part,
+  size_t amax, idx, xs, omt, zp, z, gram, gram1, l, linv, evals, evecs, ycm, scale, hsp, mp, m, basis, bs, coef, part,
       a6, b6, sign, evals2, evecs2, total;
 };
 constexpr int WIDE_GRAM_PARTS = 32;
@@ -1585,11 +1585,10 @@ WideWs wide_ws_layout(int64_t rows, int64_t cols, int k, int p, int64_t n_s, boo
   w.omt = take(sizeof(__nv_bfloat16) * (size_t)nbq * cols);
   w.zp = take(sizeof(float) * (size_t)metis_coeff_slices(n_r, cols, nullptr) * n_r * WIDE_SK);
   w.z = take(sizeof(float) * (size_t)n_r * q);
-  w.z2 = take(sizeof(float) * (size_t)n_r * q);
   w.gram = take(sizeof(double) * (size_t)WIDE_GRAM_PARTS * q * q);
   w.gram1 = take(sizeof(double) * (size_t)q * q);
   w.l = take(sizeof(double) * (size_t)q * q);
-  w.linv = take(sizeof(double) * (size_t)q * q);
+  w.linv = take(sizeof(double) * (size_t)q * q);                 // inverses of the factor's diagonal blocks (fewer than q * q entries)
   w.evals = take(sizeof(double) * (size_t)q);
   w.evecs = take(sizeof(double) * (size_t)q * q);
   w.ycm = take(sizeof(double) * (size_t)metis_wide::MAXQ_WIDE * q);
@@ -1633,7 +1632,7 @@ metis_status_t launch_gram64(cudaStream_t s, const float* v, int64_t n_rows, int
 
 // eigen-decomposition of the n x n Gram matrix gram1: Cholesky factor, cluster Jacobi on its columns, collection
 metis_status_t launch_eig_wide(cudaStream_t s, const double* gram1, int n, float exit_cos2, double* l, double* ycm, double* evals, double* evecs) {
-  METIS_CUDA_TRY(metis_launch_pdl(metis_wide::chol_wide_kernel, dim3(1), dim3(1024), (size_t)0, s, gram1, n, 1e-14, l, (double*)nullptr, (const int*)nullptr,
+  METIS_CUDA_TRY(metis_launch_pdl(metis_wide::chol_wide_kernel, dim3(1), dim3(1024), metis_wide::CW_SMEM, s, gram1, n, 1e-14, l, (double*)nullptr, (const int*)nullptr,
                                   (int*)nullptr)); METIS_COUNT_LAUNCH();
   metis_wide::jacobi_cluster_kernel<<<metis_wide::JC_P, metis_wide::JC_THREADS, metis_wide::JC_SMEM, s>>>(l, n, exit_cos2, ycm); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(cudaGetLastError());
@@ -1656,7 +1655,6 @@ metis_status_t split_wide(metis_context* ctx, const __nv_bfloat16* x, int64_t ro
   __nv_bfloat16* omt = reinterpret_cast<__nv_bfloat16*>(wsb + L.omt);
   float* zp = reinterpret_cast<float*>(wsb + L.zp);
   float* z = reinterpret_cast<float*>(wsb + L.z);
-  float* z2 = reinterpret_cast<float*>(wsb + L.z2);
   double* gram = reinterpret_cast<double*>(wsb + L.gram);
   double* gram1 = reinterpret_cast<double*>(wsb + L.gram1);
   double* lf = reinterpret_cast<double*>(wsb + L.l);
@@ -1699,19 +1697,17 @@ metis_status_t split_wide(metis_context* ctx, const __nv_bfloat16* x, int64_t ro
                                       z + j0, q)); METIS_COUNT_LAUNCH();
     }
   }
-  // (3) CholeskyQR2: both passes always (FP64 Gram matrix, factor and inverse factor; H = Z L^-T as a product)
+  // (3) CholeskyQR2: both passes always (FP64 Gram matrix, blocked factorisation, blocked triangular solve)
   {
-    float* src = z; float* dst = z2;
+    float* src = z;
     for (int pass = 0; pass < 2; ++pass) {
       METIS_TRY(launch_gram64(s, src, n_r, q, q, 1, gram, gram1));
-      METIS_CUDA_TRY(metis_launch_pdl(metis_wide::chol_wide_kernel, dim3(1), dim3(1024), (size_t)0, s, (const double*)gram1, q, 1e-13, lf, linv, (const int*)nullptr,
+      METIS_CUDA_TRY(metis_launch_pdl(metis_wide::chol_wide_kernel, dim3(1), dim3(1024), metis_wide::CW_SMEM, s, (const double*)gram1, q, 1e-13, lf, linv, (const int*)nullptr,
                                       (int*)nullptr)); METIS_COUNT_LAUNCH();
-      Gemm64Args g{};
-      g.a = src; g.a_m = q; g.a_k = 1; g.b = linv; g.b_k = 1; g.b_n = q; g.c = dst; g.c_m = q; g.c_n = 1; g.M = n_r; g.N = q; g.K = q;
-      METIS_TRY(launch_gemm64(s, g));
-      float* t = src; src = dst; dst = t;
+      METIS_CUDA_TRY(metis_launch_pdl(metis_wide::trsm_wide_kernel, dim3((unsigned)metis_ceil_div(n_r, metis_wide::TW_ROWS)), dim3(256), metis_wide::TW_SMEM, s, src, n_r, q,
+                                      (const double*)lf, (const double*)linv)); METIS_COUNT_LAUNCH();
     }
-  }                                                      // H is in z again
+  }                                                      // H = Z L^-T, in place
   // (4) M = H^T xr on the tensor cores, WIDE_PJ sketch columns per launch; eigen-decomposition of M M^T
   {
     const int slices = metis_project_slices(n_r, cols);
@@ -1822,6 +1818,8 @@ metis_status_t metis_split_set_attrs() {
   METIS_CUDA_TRY(cudaFuncSetAttribute(residual_quant_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(true)));
   METIS_CUDA_TRY(cudaFuncSetAttribute(gram_chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GC_MAX_SMEM));
   METIS_CUDA_TRY(cudaFuncSetAttribute(metis_wide::jacobi_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)metis_wide::JC_SMEM));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(metis_wide::chol_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)metis_wide::CW_SMEM));
+  METIS_CUDA_TRY(cudaFuncSetAttribute(metis_wide::trsm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)metis_wide::TW_SMEM));
 #define METIS_PP_ATTR(MTV) METIS_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<MTV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
       (int)((size_t)PP_STAGES * (PP_K * PP_XP * 2 + 3 * (MTV) * 16 * PP_HP * 2))))
   METIS_PP_ATTR(1); METIS_PP_ATTR(2); METIS_PP_ATTR(3); METIS_PP_ATTR(4); METIS_PP_ATTR(5);
