@@ -199,6 +199,10 @@ metis_status_t metis_quantize_rht_nvfp4(metis_handle_t h, const void* x, int32_t
  * scale amax(x)/2688 of the SOURCE tensor; factors with their own.  `residual_axes` selects which
  * residual orientations are produced.  `residual_dense` (optional, rows x cols FP32) receives the
  * unquantized residual the quantizer saw.  k == 0 quantizes x itself.
+ * src_amax (optional device scalar): amax|x| as the producer of x already knows it (e.g. from the epilogue of the
+ * kernel that wrote x).  NULL: the library finds it - for k > 0 inside a pass it makes anyway, for k == 0 with a
+ * reduction of its own, i.e. a second read of x that a supplied value saves.  The value is trusted: a value below
+ * the true maximum makes the largest elements saturate.
  * Requires rows % 16 == 0, cols % 64 == 0 (tiled scales), k % 4 == 0, k <= 256 and k + p <= 272.
  * Up to k = 64 and k + p = 72 the orthonormalisation and the two small eigen-solvers each run in one CTA's
  * shared memory; above that (the 1.5 % rank of an 8192-wide layer is 128) they run on FP64 kernels tiled over the
@@ -208,7 +212,7 @@ metis_status_t metis_quantize_rht_nvfp4(metis_handle_t h, const void* x, int32_t
  * a larger n_sample may need more and is then refused with METIS_ERR_WORKSPACE). */
 metis_status_t metis_split(metis_handle_t h, const void* x, int64_t rows, int64_t cols, int32_t k, int32_t p,
                            int32_t sketch, int64_t n_sample, uint64_t seed, int32_t rounding,
-                           int32_t residual_axes, metis_operand_t* out, float* residual_dense,
+                           int32_t residual_axes, const float* src_amax, metis_operand_t* out, float* residual_dense,
                            void* ws, size_t ws_bytes, metis_stream_t stream);
 
 /* Re-quantization of a stored operand (Section 3.2: a weight is kept as separately stored U, S, V and W_R, which the

@@ -79,7 +79,7 @@ def lib():
     l.metis_quantize_nvfp4.argtypes = [vp, vp, i32, i64, i64, i64, i32, u64, u32, i32, P(NvFp4Struct), P(NvFp4Struct),
                                        vp, sz, vp]
     l.metis_quantize_rht_nvfp4.argtypes = [vp, vp, i32, i64, i64, i64, i32, u64, u32, P(NvFp4Struct), vp, sz, vp]
-    l.metis_split.argtypes = [vp, vp, i64, i64, i32, i32, i32, i64, u64, i32, i32, P(OperandStruct), vp, vp, sz, vp]
+    l.metis_split.argtypes = [vp, vp, i64, i64, i32, i32, i32, i64, u64, i32, i32, vp, P(OperandStruct), vp, vp, sz, vp]
     l.metis_requantize_operand.argtypes = [vp, vp, i32, i64, i32, u64, i32, i32, P(OperandStruct), vp, sz, vp]
     l.metis_linear_fwd.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp, sz, vp]
     l.metis_linear_fwd_static_ws.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp]
@@ -260,7 +260,8 @@ class Handle:
 
     # -- metis_split ---------------------------------------------------------------------------
     def split(self, x, k, p, sketch=SKETCH_SAMPLED, n_sample=0, seed=0, rounding=ROUND_RNE, axes=BLOCKS_BOTH,
-              out=None, want_residual=False, stream=None):
+              out=None, want_residual=False, stream=None, src_amax=None):
+        """metis_split.  src_amax: optional one-element float32 CUDA tensor holding amax|x| (saves the library's own reduction)."""
         rows, cols = x.shape
         op = out if out is not None else Operand(rows, cols, k, axes)
         dense = torch.empty((rows, cols), dtype=torch.float32, device=x.device) if want_residual else None
@@ -268,7 +269,7 @@ class Handle:
         ws = self.workspace(need)
         st = op.struct()
         _check("metis_split", lib().metis_split(self._h, _ptr(x), rows, cols, k, p, sketch, n_sample, seed, rounding,
-                                                axes, ctypes.byref(st), _ptr(dense), _ptr(ws), ws.numel(),
+                                                axes, _ptr(src_amax), ctypes.byref(st), _ptr(dense), _ptr(ws), ws.numel(),
                                                 _stream_ptr(stream)))
         return (op, dense) if want_residual else op
 

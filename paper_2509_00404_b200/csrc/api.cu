@@ -181,6 +181,7 @@ metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dty
                                     int64_t ld, int32_t rounding, uint64_t seed, uint32_t stream_id, int32_t tscale,
                                     metis_nvfp4_t* out_by_cols, metis_nvfp4_t* out_by_rows, void* ws, size_t ws_bytes,
                                     metis_stream_t stream) {
+  METIS_NVTX("metis_quantize_nvfp4");
   if (!h || !x || (!out_by_cols && !out_by_rows)) return METIS_ERR_INVALID_ARG;
   if (dtype != METIS_BF16 && dtype != METIS_FP32) return METIS_ERR_INVALID_ARG;
   if (rounding != METIS_ROUND_RNE && rounding != METIS_ROUND_SR) return METIS_ERR_INVALID_ARG;
@@ -220,6 +221,7 @@ metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dty
 metis_status_t metis_quantize_rht_nvfp4(metis_handle_t h, const void* x, int32_t dtype, int64_t rows, int64_t cols, int64_t ld,
                                         int32_t rounding, uint64_t seed, uint32_t stream_id, metis_nvfp4_t* out, void* ws,
                                         size_t ws_bytes, metis_stream_t stream) {
+  METIS_NVTX("metis_quantize_rht_nvfp4");
   if (!h || !x || !out || !out->codes || !out->scales || !out->tensor_scale) return METIS_ERR_INVALID_ARG;
   if (dtype != METIS_BF16 && dtype != METIS_FP32) return METIS_ERR_INVALID_ARG;
   if (rounding != METIS_ROUND_RNE && rounding != METIS_ROUND_SR) return METIS_ERR_INVALID_ARG;
@@ -235,6 +237,7 @@ metis_status_t metis_quantize_rht_nvfp4(metis_handle_t h, const void* x, int32_t
 metis_status_t metis_requantize_operand(metis_handle_t h, const void* residual, int32_t res_dtype, int64_t ld_res,
                                         int32_t rounding, uint64_t seed, int32_t residual_axes, int32_t res_tscale,
                                         metis_operand_t* op, void* ws, size_t ws_bytes, metis_stream_t stream) {
+  METIS_NVTX("metis_requantize_operand");
   if (!h || !residual || !op) return METIS_ERR_INVALID_ARG;
   if (res_dtype != METIS_BF16 && res_dtype != METIS_FP32) return METIS_ERR_INVALID_ARG;
   if (rounding != METIS_ROUND_RNE && rounding != METIS_ROUND_SR) return METIS_ERR_INVALID_ARG;
@@ -280,6 +283,7 @@ metis_status_t metis_requantize_operand(metis_handle_t h, const void* residual, 
 
 metis_status_t metis_gemm_nvfp4(metis_handle_t h, const metis_nvfp4_t* a, const metis_nvfp4_t* b, void* d,
                                 int32_t d_dtype, int64_t ldd, int32_t impl, metis_stream_t stream) {
+  METIS_NVTX("metis_gemm_nvfp4");
   if (!h || !a || !b || !d) return METIS_ERR_INVALID_ARG;
   if (!a->codes || !b->codes || !a->scales || !b->scales || !a->tensor_scale || !b->tensor_scale) return METIS_ERR_INVALID_ARG;
   if (a->k_len != b->k_len || a->k_len % 16) return METIS_ERR_SHAPE;

@@ -4,7 +4,16 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/metis.h"
+
+// One NVTX range per entry point of the C ABI (visible in a timeline tool; a no-op when no tool is attached).
+struct metis_nvtx_range {
+  explicit metis_nvtx_range(const char* name) { nvtxRangePushA(name); }
+  ~metis_nvtx_range() { nvtxRangePop(); }
+};
+#define METIS_NVTX(name) metis_nvtx_range nvtx_range_(name)
 
 constexpr int METIS_N_SIDE = 5;                        // side streams per handle (the backward pass uses all five)
 struct metis_context {

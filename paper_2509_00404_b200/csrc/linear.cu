@@ -542,6 +542,7 @@ size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k) {
 
 metis_status_t metis_linear_fwd(metis_handle_t h, const metis_operand_t* x, const metis_operand_t* w, void* y,
                                 int32_t y_dtype, int64_t ldy, void* ws, size_t ws_bytes, metis_stream_t stream) {
+  METIS_NVTX("metis_linear_fwd");
   if (!h || !x || !w || !y) return METIS_ERR_INVALID_ARG;
   if (y_dtype != METIS_BF16 && y_dtype != METIS_FP32) return METIS_ERR_INVALID_ARG;
   if (x->cols != w->cols || ldy < w->rows) return METIS_ERR_SHAPE;
@@ -555,6 +556,7 @@ metis_status_t metis_linear_bwd(metis_handle_t h, const metis_operand_t* dy, con
                                 const metis_operand_t* w, void* dx, int32_t dx_dtype, int64_t lddx, void* dw,
                                 int32_t dw_dtype, int64_t lddw, float* d_left, float* d_sigma, float* d_right,
                                 void* ws, size_t ws_bytes, metis_stream_t stream) {
+  METIS_NVTX("metis_linear_bwd");
   if (!h || !dy) return METIS_ERR_INVALID_ARG;
   if ((d_left || d_sigma || d_right) && (!dw || !w)) return METIS_ERR_INVALID_ARG;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);

@@ -1642,7 +1642,7 @@ metis_status_t launch_eig_wide(cudaStream_t s, const double* gram1, int n, float
 }
 
 metis_status_t split_wide(metis_context* ctx, const __nv_bfloat16* x, int64_t rows, int64_t cols, int k, int p, bool full, int64_t n_s,
-                          uint64_t seed, int rounding, bool want_c, bool want_r, metis_operand_t* out, float* residual_dense,
+                          uint64_t seed, int rounding, bool want_c, bool want_r, const float* src_amax, metis_operand_t* out, float* residual_dense,
                           unsigned char* wsb, const WideWs& L, cudaStream_t s) {
   using namespace metis_qt;
   using metis_wide::Gemm64Args;
@@ -1677,6 +1677,7 @@ metis_status_t split_wide(metis_context* ctx, const __nv_bfloat16* x, int64_t ro
   double* evecs2 = reinterpret_cast<double*>(wsb + L.evecs2);
 
   METIS_CUDA_TRY(cudaMemsetAsync(amax, 0, 64, s));
+  if (src_amax != nullptr) METIS_CUDA_TRY(cudaMemcpyAsync(amax, src_amax, sizeof(float), cudaMemcpyDeviceToDevice, s));
   const __nv_bfloat16* xr = x;
   if (!full) {
     METIS_CUDA_TRY(metis_launch_pdl((sample_rows_kernel), dim3((unsigned)metis_ceil_div(n_s, 256)), dim3(256), (size_t)(0), s, idx, (int)n_s, rows, seed, 0)); METIS_COUNT_LAUNCH();
@@ -1850,8 +1851,9 @@ size_t metis_split_ws_bytes(int64_t rows, int64_t cols, int k, int p) {
 
 metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64_t cols, int32_t k, int32_t p,
                            int32_t sketch, int64_t n_sample, uint64_t seed, int32_t rounding, int32_t residual_axes,
-                           metis_operand_t* out, float* residual_dense, void* ws, size_t ws_bytes,
+                           const float* src_amax, metis_operand_t* out, float* residual_dense, void* ws, size_t ws_bytes,
                            metis_stream_t stream) {
+  METIS_NVTX("metis_split");
   using namespace metis_qt;
   if (!h || !xv || !out || !ws) return METIS_ERR_INVALID_ARG;
   if (rows <= 0 || cols <= 0 || rows % 16 || cols % 16 || k < 0 || p < 0) return METIS_ERR_SHAPE;
@@ -1879,7 +1881,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
     if (!out->left || !out->sigma || !out->right || !out->left_q.codes || !out->right_q.codes || !out->left_q.scales ||
         !out->right_q.scales || !out->left_q.tensor_scale || !out->right_q.tensor_scale)
       return METIS_ERR_INVALID_ARG;
-    return split_wide(h, reinterpret_cast<const __nv_bfloat16*>(xv), rows, cols, k, p, full, n_s, seed, rounding, want_c, want_r, out,
+    return split_wide(h, reinterpret_cast<const __nv_bfloat16*>(xv), rows, cols, k, p, full, n_s, seed, rounding, want_c, want_r, src_amax, out,
                       residual_dense, reinterpret_cast<unsigned char*>(ws), W, reinterpret_cast<cudaStream_t>(stream));
   }
   const SplitWs L = split_ws_layout(rows, cols, k, p, n_s);
@@ -1892,7 +1894,8 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   metis_nvfp4_t rc = out->res_by_cols, rr = out->res_by_rows;
   rc.rows = rows; rc.k_len = cols; rr.rows = cols; rr.k_len = rows;
   if (k == 0) {
-    METIS_TRY(metis_launch_amax(x, METIS_BF16, rows, cols, cols, amax, s));
+    if (src_amax != nullptr) METIS_CUDA_TRY(cudaMemcpyAsync(amax, src_amax, sizeof(float), cudaMemcpyDeviceToDevice, s));
+    else METIS_TRY(metis_launch_amax(x, METIS_BF16, rows, cols, cols, amax, s));
     METIS_TRY(metis_launch_quantize(x, METIS_BF16, rows, cols, cols, rounding, seed, METIS_STREAM_RESIDUAL, cols, 1, amax,
                                     1, want_c ? &rc : nullptr, want_r ? &rr : nullptr, s));
     METIS_CUDA_TRY(metis_launch_pdl((split_status_kernel), dim3(1), dim3(32), (size_t)(0), s, amax, (const double*)nullptr, 0, h->dev_status)); METIS_COUNT_LAUNCH();
@@ -1940,6 +1943,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   const int kp = (k + 15) / 16 * 16;
   // amax|x| for the residual's tensor scale: fused into the sketch pass (FULL) or the broadcast pass (SAMPLED)
   METIS_CUDA_TRY(cudaMemsetAsync(amax, 0, 64, s));       // amax slots of x, left, right and the condition flag
+  if (src_amax != nullptr) METIS_CUDA_TRY(cudaMemcpyAsync(amax, src_amax, sizeof(float), cudaMemcpyDeviceToDevice, s));
 
   // (1) row sample, (2) sketch (tensor cores; Omega generated per CTA into shared memory)
   METIS_CUDA_TRY(metis_launch_pdl((sample_rows_kernel), dim3((unsigned)metis_ceil_div(n_s, 256)), dim3(256), (size_t)(0), s, idx, (int)n_s, rows, seed, full ? 1 : 0)); METIS_COUNT_LAUNCH();

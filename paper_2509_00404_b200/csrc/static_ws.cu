@@ -38,6 +38,7 @@ metis_status_t static_ws_address(int device, void** out) {
 
 extern "C" metis_status_t metis_linear_fwd_static_ws(metis_handle_t h, const metis_operand_t* x, const metis_operand_t* w,
                                                      void* y, int32_t y_dtype, int64_t ldy, metis_stream_t stream) {
+  METIS_NVTX("metis_linear_fwd_static_ws");
   if (!h || !x || !w || !y) return METIS_ERR_INVALID_ARG;
   int current = -1;
   if (cudaGetDevice(&current) != cudaSuccess) return METIS_ERR_CUDA;

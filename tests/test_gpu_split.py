@@ -275,6 +275,24 @@ def test_rank_zero_is_plain_quantization(ctx):
         assert ts == ots and np.array_equal(sg, os_) and np.array_equal(cg, oc)
 
 
+@pytest.mark.parametrize("k", [0, 8])
+def test_supplied_source_amax_gives_the_same_bytes(ctx, k):
+    """metis_split with the producer's amax|x| handed in (no reduction pass of its own for k = 0) against the default."""
+    from gpu_util import to_dev_bf16, nv_to_numpy
+    B, h = ctx
+    x, _ = synth.llama_like(384, 512, 1.0, 71, rank=8)
+    xd = to_dev_bf16(x)
+    a = h.split(xd, k, 8 if k else 0, seed=5)
+    amax = xd.float().abs().max().reshape(1)
+    b = h.split(xd, k, 8 if k else 0, seed=5, src_amax=amax)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    for name in ("res_by_cols", "res_by_rows"):
+        ca, sa, ta = nv_to_numpy(getattr(a, name))
+        cb, sb, tb = nv_to_numpy(getattr(b, name))
+        assert ta == tb and np.array_equal(ca, cb) and np.array_equal(sa, sb)
+
+
 def test_workspace_and_shape_errors(ctx):
     B, h = ctx
     x = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
