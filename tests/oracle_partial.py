@@ -19,6 +19,7 @@ class PartialOperand:
         if k:
             sp = osp.split(x32.astype(np.float64), k, p, mode=mode, seed=seed)
             self.sigma = sp.sigma
+            self.right = sp.right
             self.res = sp.residual.astype(np.float32)
             lq = onv.quantize(np.ascontiguousarray(sp.left.T).astype(np.float32), onv.AXIS_COLS, rounding, seed, philox.STREAM_LEFT)
             rq = onv.quantize(np.ascontiguousarray(sp.right.T).astype(np.float32), onv.AXIS_COLS, rounding, seed, philox.STREAM_RIGHT)

@@ -217,3 +217,32 @@ def test_requantizing_the_stored_pieces_of_a_split_reproduces_the_split_operand(
     i, j = np.unravel_index(np.argmax(np.abs(res32)), res32.shape)
     assert np.isclose(own.res_by_cols[i, j], res32[i, j], rtol=1e-6)
     assert metrics.rel_fro(own.res_by_cols, res32) <= metrics.rel_fro(xq.res_by_cols, res32) * 1.05
+
+
+def test_conditioning_of_the_end_to_end_value_when_the_rank_cut_falls_inside_the_bulk():
+    """How far the oracle's OWN split-FP4 output moves when its input is perturbed by 1e-6 relative - the size of an
+    FP32 accumulation over a few thousand terms, which any FP32 pipeline carries in its sketch and projection.
+    With k at most the planted rank every kept singular vector is well separated and the output moves by about 1e-3;
+    with k above it the extra vectors are singular vectors of the Gaussian bulk (neighbouring singular values a
+    fraction of a percent apart), they turn by ~1e-4, the NVFP4 encoder re-rounds a few blocks per thousand, and the
+    output moves by more than the 2e-3 that the end-to-end comparisons allow.  This is why the GPU parity tests treat
+    the cases with k above the planted rank (the rank-128 and rank-256 points of the 70B-shaped sweep) as
+    conditioning-limited and check what is unique there instead."""
+    def moved(k, rank, n=512, pert=1e-6):
+        x, _ = synth.llama_like(n, n, 1.0, 5, rank=rank)
+        w, _ = synth.llama_like(n, n, 0.02, 6, rank=rank)
+        rng = np.random.default_rng(0)
+
+        def forward(noise):
+            ops = []
+            for t, seed in ((x, 1), (w, 2)):
+                t64 = t.astype(np.float64) * (1.0 + noise * rng.standard_normal(t.shape)) if noise else t.astype(np.float64)
+                sp = split.split(t64, k, 8, split.MODE_FULL, seed)
+                ops.append(layer.requantize_operand(sp.left, sp.sigma, sp.right, sp.residual,
+                                                    residual_scale=nvfp4.tensor_scale_from_amax(np.max(np.abs(t)))))
+            return layer.linear_fwd(*ops)
+        y0, y1 = forward(0.0), forward(pert)
+        return np.linalg.norm(y1 - y0) / np.linalg.norm(y0)
+    assert moved(16, 16) < 2e-3 and moved(32, 32) < 2e-3
+    assert moved(64, 16) > 2e-3 and moved(128, 16) > 2e-3
+    assert moved(64, 16, pert=3e-6) > 1e-2                 # a few 1e-6 are enough for differences of a few per cent
