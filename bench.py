@@ -400,7 +400,7 @@ def main():
                 ref_out = [t.clone() for t in (wl.y[0], wl.dx[0], wl.dw_sets[0][0])]
                 graphs[(0, 0)].replay()
                 barrier()
-                assert all(torch.equal(a_, b_) for a_, b_ in zip(ref_out, (wl.y[0], wl.dx[0], wl.dw_sets[0][0]))), "graph replay differs from host launches"
+                assert all(torch.equal(a_, b_) for a_, b_ in zip(ref_out, (wl.y[0], wl.dx[0], wl.dw_sets[0][0]))), "graph replay differs from host launches (%s)" % name
                 del ref_out
             except AssertionError:
                 raise

@@ -135,6 +135,7 @@ coeff_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
           }
         }
       }
+      fence_proxy_async();                                // the box was read through the generic proxy; a tensor copy refills it
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_bar(s));
       if (++s == STAGES) { s = 0; ph ^= 1u; }

@@ -221,8 +221,12 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
           }
         }
       }
-      // accumulator and x tile read: hand both back
+      // accumulator and x tile read: hand both back.  The x box was read with ordinary shared-memory loads (generic
+      // proxy) and is refilled by a tensor copy (async proxy): the proxy fence orders those reads before the copy
+      // that the arrival permits.  Without it the refill could land - rarely - before the warp's last load had been
+      // performed, and 8 columns of 32 rows came out with the next tile's values.
       tc_fence_before();
+      fence_proxy_async();
       __syncwarp();
       if (lane == 0) { mbar_arrive(tempty_bar(acc)); mbar_arrive(xempty_bar(xb)); }
       const bool step_ok = FAST || c0 < p.cols;                                      // false: the warp's columns lie outside the matrix
