@@ -259,3 +259,61 @@ def test_repeated_calls_are_bit_identical(ctx):
         again = run()
         assert all(torch.equal(a, b) for a, b in zip(first, again))
     assert h.device_status() == 0
+
+
+def test_concurrent_step_replayed_many_times_is_bit_identical():
+    """The whole step of a 4096-token layer - three decompositions on three streams, forward and backward - captured
+    once and replayed 1500 times: every replay must reproduce the first one bit for bit.  Kernels of different
+    operands overlap differently from replay to replay, which is what exposes a missing ordering between a buffer's
+    readers and the copy that refills it (such a gap once let one step in a few hundred through with a 32 x 8 patch of
+    wrong residual values)."""
+    from paper_2509_00404_b200 import binding as B
+    l = m = n = 4096
+    k, p = 32, 8
+    x, w, d = synth.planted_device(l, m, 32, 1.0, 11), synth.planted_device(n, m, 32, 0.02, 12), synth.planted_device(l, n, 32, 1e-4, 13)
+    hx, hw, hd = B.Handle(0), B.Handle(0), B.Handle(0)
+    try:
+        xo, wo, do = B.Operand(l, m, k), B.Operand(n, m, k), B.Operand(l, n, k)
+        y = torch.empty((l, n), dtype=torch.bfloat16, device="cuda")
+        dx, dw = torch.empty((l, m), dtype=torch.bfloat16, device="cuda"), torch.empty((n, m), dtype=torch.bfloat16, device="cuda")
+        sw, sd = torch.cuda.Stream(), torch.cuda.Stream()
+        e0, ew, ex, eb = (torch.cuda.Event() for _ in range(4))
+
+        def step():
+            main = torch.cuda.current_stream()
+            e0.record(main); sw.wait_event(e0); sd.wait_event(e0)
+            with torch.cuda.stream(sw):
+                hw.split(w, k, p, sketch=B.SKETCH_FULL, seed=2, out=wo, stream=sw)
+                ew.record(sw)
+            hx.split(x, k, p, sketch=B.SKETCH_SAMPLED, seed=1, out=xo)
+            ex.record(main)
+            main.wait_event(ew)
+            hx.linear_fwd(xo, wo, out=y)
+            with torch.cuda.stream(sd):
+                hd.split(d, k, p, sketch=B.SKETCH_SAMPLED, seed=3, rounding=B.ROUND_SR, out=do, stream=sd)
+                sd.wait_event(ex); sd.wait_event(ew)
+                hd.linear_bwd(do, xo, wo, out=(dx, dw), stream=sd)
+                eb.record(sd)
+            main.wait_event(eb)
+
+        for _ in range(2):
+            step()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step()
+        g.replay()
+        torch.cuda.synchronize()
+        watched = [y, dx, dw, xo.res_by_cols.codes, xo.res_by_rows.codes, wo.res_by_cols.codes, wo.res_by_rows.codes,
+                   do.res_by_cols.codes, do.res_by_rows.codes, xo.res_by_cols.scales, do.res_by_rows.scales]
+        first = [t.clone() for t in watched]
+        bad = 0
+        for _ in range(1500):
+            g.replay()
+            bad += int(not all(torch.equal(a, b) for a, b in zip(first, watched)))
+        torch.cuda.synchronize()
+        assert bad == 0, "%d of 1500 replays differ from the first" % bad
+        assert (hx.device_status() | hw.device_status() | hd.device_status()) == 0
+    finally:
+        for h in (hx, hw, hd):
+            h.close()
