@@ -39,6 +39,15 @@ FP4_OVER_BF16 = 4.0           # nominal dense FP4 : bf16 tensor throughput ratio
 BYTES_PER_ELEM_BOTH = 3.125   # split / quantize: 2 B read + 2 x 0.5625 B written per operand element
 
 
+# DRAM bytes of ONE launch of the two-CTA GEMM (dram__bytes_read.sum + dram__bytes_write.sum), per (M, N, K), from an
+# ncu capture of this program's block workload (a profiler cannot run inside the timed program).  Reads are 4.7 x the
+# operand bytes at K = 4096 (the B panels are fetched once per group of eight tile rows); the bf16 output is written once.
+NCU_DRAM_BYTES = {(16384, 14336, 4096): 330.1e6 + 417.5e6, (16384, 4096, 14336): 331.9e6 + 111.9e6,
+                  (14336, 4096, 16384): 376.2e6 + 98.9e6}
+NCU_DRAM_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum -k regex:gemm_nvfp4_2cta on "
+                   "`bench.py --workloads block_16384tok --no-graph`, one launch of this shape")
+
+
 def layer(name, d_in, d_out, x_group):
     return {"name": name, "d_in": d_in, "d_out": d_out, "x": x_group}
 
@@ -484,8 +493,9 @@ def main():
         big_bytes = 0.5625 * (big[0].rows + big[1].rows) * big[0].k_len + big[2].element_size() * big[0].rows * big[1].rows
 
         # ---- split + quantize of each operand kind alone, at the workload's largest operand --------------------
-        def alone(fn, reps=6):
-            fn(0)
+        def alone(fn, reps=12):
+            for w_i in range(3):
+                fn(w_i)
             torch.cuda.synchronize()
             return timed_ms(torch, fn, reps)
         k, p = wl.k, wl.p
@@ -496,8 +506,8 @@ def main():
         ms_sw = alone(lambda i: h_x.split(wl.w_in[jw], k, p, sketch=B.SKETCH_FULL, seed=i + 2, out=wl.wo[jw]))
         ms_sd = alone(lambda i: h_x.split(wl.d_in[jd], k, p, sketch=B.SKETCH_SAMPLED, seed=i + 3, rounding=B.ROUND_SR, out=wl.do[jd]))
         xq = wl.xo[gx]
-        ms_q = alone(lambda i: h_x.quantize_nvfp4(wl.x_in[gx], B.BLOCKS_BOTH, B.ROUND_RNE, seed=1, tensor_scale=1.0, out=(xq.res_by_cols, xq.res_by_rows)))
-        ms_qsr = alone(lambda i: h_x.quantize_nvfp4(wl.x_in[gx], B.BLOCKS_BOTH, B.ROUND_SR, seed=1, tensor_scale=1.0, out=(xq.res_by_cols, xq.res_by_rows)))
+        ms_q = alone(lambda i: h_x.quantize_nvfp4(wl.x_in[gx], B.BLOCKS_BOTH, B.ROUND_RNE, seed=1, tensor_scale=1.0, out=(xq.res_by_cols, xq.res_by_rows)), reps=30)
+        ms_qsr = alone(lambda i: h_x.quantize_nvfp4(wl.x_in[gx], B.BLOCKS_BOTH, B.ROUND_SR, seed=1, tensor_scale=1.0, out=(xq.res_by_cols, xq.res_by_rows)), reps=30)
         gbs = lambda elems, t_ms: BYTES_PER_ELEM_BOTH * elems / (t_ms * 1e-3) / 1e9
         ex, ew, ed = wl.x_in[gx].numel(), wl.w_in[jw].numel(), wl.d_in[jd].numel()
         hbm = peaks["hbm_gbs"]
@@ -622,7 +632,8 @@ def main():
         "clocks": hd["rec"]["clocks"],
         "roofline": {"bound": "tensor", "kernel": "two_cta::gemm_nvfp4_2cta_kernel, the largest residual GEMM of the block (M, N, K = %s), bf16 out" % hd["big_shape"],
                      "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak,
-                     "traffic": None, "algorithmic_bytes": hd["big_bytes"],
+                     "traffic": NCU_DRAM_BYTES.get(tuple(hd["big_shape"])), "traffic_source": NCU_DRAM_SOURCE,
+                     "algorithmic_bytes": hd["big_bytes"],
                      "peak_source": "bf16 burst peak (%s) x %.0f nominal FP4:bf16 ratio" % (peaks["source"], FP4_OVER_BF16),
                      "ms_per_launch": hd["ms_big"]},
         "rooflines_hbm": {"peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "algorithmic_bytes_per_element": BYTES_PER_ELEM_BOTH,

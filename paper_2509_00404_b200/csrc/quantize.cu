@@ -48,19 +48,30 @@ __global__ void amax_kernel(const void* __restrict__ x, int dtype, int64_t rows,
 //          the stochastic-rounding draws go to shared memory for pass 2
 //  pass 2  blocks along the rows: a thread reads 16 values down a column from shared memory, encodes them and
 //          stages the bytes; the transposed codes and both scale tiles are then written out coalesced
+constexpr int QK_CP = metis_qt::TILE / 2 + 8;                     // pitch of a staged row of row-block codes, bytes
 template <typename T, bool SR>   // T = __nv_bfloat16 or float: element type of the shared tile (= input type)
 __global__ void __launch_bounds__(metis_qt::THREADS, SR ? 3 : 4)
 quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, const float* __restrict__ tscale_src,
                 int tscale_is_amax, float* ts_out0, float* ts_out1) {
   using namespace metis_qt;
-  constexpr int TP = TILE + (sizeof(T) == 2 ? 2 : 1);            // tile pitch in elements (odd word stride)
+  // Shared-memory layouts, chosen so that every access of a warp touches each bank once.
+  //   BF16 tile and draws: rows of 256 bytes = 16 chunks of 16 bytes, chunk ch stored at ch ^ (ch >> 3): the eight
+  //     lanes of a quarter warp store the even (or odd) chunks of one row, which the swizzle spreads over all banks;
+  //     pass 2 reads 32 consecutive words of a row, a permutation of the chunks inside one 128-byte window.
+  //   FP32 tile: pitch 129 words.
+  //   staged row-block codes: 72-byte rows; a BF16 thread owns two adjacent columns, so column c is staged in row
+  //     (c >> 1) + 64 (c & 1) and the 32 lanes of a store write 32 consecutive rows (18 words apart: 16 lanes cover
+  //     the 32 banks with their 8 bytes each).
+  constexpr int TP = sizeof(T) == 2 ? TILE : TILE + 1;           // tile pitch in elements
   extern __shared__ __align__(16) unsigned char smem[];
   T* tile = reinterpret_cast<T*>(smem);                                        // [TILE][TP]
-  Stage* stage = reinterpret_cast<Stage*>(smem + ((sizeof(T) * TILE * TP + 15) & ~(size_t)15));
-  uint8_t* sfc = reinterpret_cast<uint8_t*>(stage + 1);                        // [TILE][8] scales of the column blocks
+  uint8_t* codes_s = smem + ((sizeof(T) * TILE * TP + 15) & ~(size_t)15);      // [TILE][QK_CP] row-block codes
+  uint8_t* sfr = codes_s + TILE * QK_CP;                                       // [TILE][8] scales of the row blocks
+  uint8_t* sfc = sfr + TILE * 8;                                               // [TILE][8] scales of the column blocks
   float* r_tab = reinterpret_cast<float*>(sfc + TILE * 8);                     // multiplier per scale byte
   uint16_t* rnd = reinterpret_cast<uint16_t*>(r_tab + R_TABLE);                // [TILE][TILE] draws (SR only)
 
+  auto staged_row = [](int c) { return sizeof(T) == 2 ? (c >> 1) + 64 * (c & 1) : c; };
   const int tid = threadIdx.x;
   const int64_t row0 = (int64_t)blockIdx.y * TILE, col0 = (int64_t)blockIdx.x * TILE;
   const float s_T = tscale_is_amax ? metis_tensor_scale(*tscale_src) : *tscale_src;
@@ -74,6 +85,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
   const bool want_c = p.c_codes != nullptr, want_r = p.r_codes != nullptr;
   const int vrows = (int)min((int64_t)TILE, p.rows - row0), vcols = (int)min((int64_t)TILE, p.cols - col0);
   const bool fast_draws = p.e_stride_c == 1 && (p.e_stride_r & 7) == 0;
+  const bool wide_ld = sizeof(T) == 2 && (ld & 15) == 0 && (reinterpret_cast<uintptr_t>(x) & 31) == 0;   // 32-byte aligned blocks
 
   // ---- pass 1 ----
   // all global loads of the tile are issued before the first block is encoded: 128 bytes per thread in flight
@@ -85,7 +97,14 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
       raw[2 * it] = raw[2 * it + 1] = make_uint4(0u, 0u, 0u, 0u);
       if (r < vrows && b * 16 < vcols) {
         const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(x) + (row0 + r) * ld + col0 + b * 16);
-        raw[2 * it] = src[0]; raw[2 * it + 1] = src[1];
+        if (wide_ld) {                                     // one 32-byte load per block: consecutive lanes, consecutive 32 bytes
+          asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                       : "=r"(raw[2 * it].x), "=r"(raw[2 * it].y), "=r"(raw[2 * it].z), "=r"(raw[2 * it].w),
+                         "=r"(raw[2 * it + 1].x), "=r"(raw[2 * it + 1].y), "=r"(raw[2 * it + 1].z), "=r"(raw[2 * it + 1].w)
+                       : "l"(src));
+        } else {
+          raw[2 * it] = src[0]; raw[2 * it + 1] = src[1];
+        }
       }
     }
   }
@@ -103,9 +122,9 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
 #pragma unroll
       for (int j = 0; j < 8; ++j) { v[2 * j] = __uint_as_float(w[j] << 16); v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u); }
       if (want_r) {
-        uint32_t* dst = reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(tile) + r * TP + b * 16);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) dst[j] = w[j];
+        uint4* trow = reinterpret_cast<uint4*>(smem + r * 256);
+        trow[(2 * b) ^ (b >> 2)] = q0;
+        trow[(2 * b + 1) ^ (b >> 2)] = q1;
       }
     } else if (in) {
       const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(x) + gr * ld + gc);
@@ -138,9 +157,15 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
           u[j] = in ? metis_draw_u16((uint64_t)gr * (uint64_t)p.e_stride_r + (uint64_t)(gc + j) * (uint64_t)p.e_stride_c, p.seed, p.stream_id) << 16 : 0u;
       }
       if (want_r) {
-        uint32_t* dst = reinterpret_cast<uint32_t*>(rnd + r * TILE + b * 16);
+        if (sizeof(T) == 2) {
+          uint4* drow = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(rnd) + r * 256);
+          drow[(2 * b) ^ (b >> 2)] = make_uint4((u[0] >> 16) | u[1], (u[2] >> 16) | u[3], (u[4] >> 16) | u[5], (u[6] >> 16) | u[7]);
+          drow[(2 * b + 1) ^ (b >> 2)] = make_uint4((u[8] >> 16) | u[9], (u[10] >> 16) | u[11], (u[12] >> 16) | u[13], (u[14] >> 16) | u[15]);
+        } else {
+          uint32_t* dst = reinterpret_cast<uint32_t*>(rnd + r * TILE + b * 16);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) dst[j] = (u[2 * j] >> 16) | u[2 * j + 1];
+          for (int j = 0; j < 8; ++j) dst[j] = (u[2 * j] >> 16) | u[2 * j + 1];
+        }
       }
     }
     if (want_c) {
@@ -158,28 +183,29 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
       // row blocks, i.e. eight blocks in two rounds of four
 #pragma unroll 1
       for (int it = 0; it < 2; ++it) {
-        const int c = (tid & 63) * 2, b = (tid >> 6) + 4 * it;
+        const int wd = tid & 63, b = (tid >> 6) + 4 * it;         // columns 2 wd, 2 wd + 1: word wd of a tile row
+        const int pw = ((((wd >> 2) ^ (wd >> 5)) << 2) | (wd & 3));    // its swizzled position
         float v0[16], v1[16];
         uint32_t u0[16], u1[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const uint32_t w = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const __nv_bfloat16*>(tile) + (b * 16 + i) * TP + c);
+          const uint32_t w = reinterpret_cast<const uint32_t*>(smem)[(b * 16 + i) * 64 + pw];
           v0[i] = __uint_as_float(w << 16); v1[i] = __uint_as_float(w & 0xFFFF0000u);
         }
         if (sr) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const uint32_t w = *reinterpret_cast<const uint32_t*>(rnd + (b * 16 + i) * TILE + c);
+            const uint32_t w = reinterpret_cast<const uint32_t*>(rnd)[(b * 16 + i) * 64 + pw];
             u0[i] = w << 16; u1[i] = w & 0xFFFF0000u;
           }
         }
         uint32_t packed[2];
         uint32_t byte = encode_block_tab(v0, u0, sr, six_s_T, r_tab, packed);
-        *reinterpret_cast<uint2*>(&stage->codes[c][b * 8]) = make_uint2(packed[0], packed[1]);
-        stage->sf[c][b] = (uint8_t)byte;
+        *reinterpret_cast<uint2*>(codes_s + wd * QK_CP + b * 8) = make_uint2(packed[0], packed[1]);
+        sfr[wd * 8 + b] = (uint8_t)byte;
         byte = encode_block_tab(v1, u1, sr, six_s_T, r_tab, packed);
-        *reinterpret_cast<uint2*>(&stage->codes[c + 1][b * 8]) = make_uint2(packed[0], packed[1]);
-        stage->sf[c + 1][b] = (uint8_t)byte;
+        *reinterpret_cast<uint2*>(codes_s + (64 + wd) * QK_CP + b * 8) = make_uint2(packed[0], packed[1]);
+        sfr[(64 + wd) * 8 + b] = (uint8_t)byte;
       }
     } else {
 #pragma unroll 1
@@ -195,8 +221,8 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
       }
       uint32_t packed[2];
       const uint32_t byte = encode_block_tab(v, u, sr, six_s_T, r_tab, packed);
-      *reinterpret_cast<uint2*>(&stage->codes[c][b * 8]) = make_uint2(packed[0], packed[1]);
-      stage->sf[c][b] = (uint8_t)byte;
+      *reinterpret_cast<uint2*>(codes_s + c * QK_CP + b * 8) = make_uint2(packed[0], packed[1]);
+      sfr[c * 8 + b] = (uint8_t)byte;
     }
     }
     __syncthreads();
@@ -204,7 +230,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
     for (int i = tid; i < TILE * 8; i += THREADS) {
       const int c = i >> 3, seg = i & 7;
       if (c < vcols && seg * 16 < vrows)
-        *reinterpret_cast<uint2*>(p.r_codes + (col0 + c) * kbytes + row0 / 2 + seg * 8) = *reinterpret_cast<const uint2*>(&stage->codes[c][seg * 8]);
+        *reinterpret_cast<uint2*>(p.r_codes + (col0 + c) * kbytes + row0 / 2 + seg * 8) = *reinterpret_cast<const uint2*>(codes_s + staged_row(c) * QK_CP + seg * 8);
     }
     const int64_t bpr = p.rows / 16;
     for (int i = tid; i < TILE * 8; i += THREADS) {
@@ -212,7 +238,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
       if (p.r_layout == METIS_SF_TILED) { const int atom = i >> 9, w = i & 511; c = (w >> 4) + 32 * ((w >> 2) & 3); b = atom * 4 + (w & 3); }
       else { c = i >> 3; b = i & 7; }
       if (b * 16 < vrows && (c < vcols || p.r_layout == METIS_SF_TILED))
-        p.r_scales[metis_sf_offset(col0 + c, row0 / 16 + b, bpr, p.r_layout)] = c < vcols ? stage->sf[c][b] : (uint8_t)0;
+        p.r_scales[metis_sf_offset(col0 + c, row0 / 16 + b, bpr, p.r_layout)] = c < vcols ? sfr[staged_row(c) * 8 + b] : (uint8_t)0;
     }
   }
   if (want_c) {
@@ -229,8 +255,8 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
 
 template <typename T>
 constexpr size_t quantize_smem(bool sr) {
-  return ((sizeof(T) * metis_qt::TILE * (metis_qt::TILE + (sizeof(T) == 2 ? 2 : 1)) + 15) & ~(size_t)15) + sizeof(metis_qt::Stage) +
-         metis_qt::TILE * 8 + sizeof(float) * metis_qt::R_TABLE + (sr ? sizeof(uint16_t) * metis_qt::TILE * metis_qt::TILE : 0);
+  return ((sizeof(T) * metis_qt::TILE * (metis_qt::TILE + (sizeof(T) == 2 ? 0 : 1)) + 15) & ~(size_t)15) + metis_qt::TILE * QK_CP +
+         2 * metis_qt::TILE * 8 + sizeof(float) * metis_qt::R_TABLE + (sr ? sizeof(uint16_t) * metis_qt::TILE * metis_qt::TILE : 0);
 }
 
 }  // namespace
