@@ -72,6 +72,30 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
   uint16_t* rnd = reinterpret_cast<uint16_t*>(r_tab + R_TABLE);                // [TILE][TILE] draws (SR only)
 
   auto staged_row = [](int c) { return sizeof(T) == 2 ? (c >> 1) + 64 * (c & 1) : c; };
+  // Scale bytes of the tile, from their staging area [stored row][8] to global memory.  The four blocks of a 64-element
+  // K group are adjacent in both layouts, so they go out as one word per thread (256 words per tile and orientation;
+  // in the tiled layout consecutive threads write consecutive words of a 512-byte atom, and blocks or rows of the atom
+  // that lie outside the matrix are its zero padding); an unaligned linear layout takes the byte path.
+  auto write_scales = [&](uint8_t* dst, int layout, int64_t bpr, const uint8_t* src, bool staged, int v_rows, int v_k, int64_t g_row0, int64_t g_blk0) {
+    const bool tiled = layout == METIS_SF_TILED;
+    if ((tiled || (bpr & 3) == 0) && (reinterpret_cast<uintptr_t>(dst) & 3) == 0) {
+      const int i = threadIdx.x;                                          // THREADS == 2 * TILE words
+      const int atom = tiled ? i >> 7 : i & 1;
+      const int r = tiled ? ((i & 127) >> 2) + 32 * (i & 3) : i >> 1;
+      if (atom * 64 < v_k && (r < v_rows || tiled)) {
+        const uint32_t w = r < v_rows ? *reinterpret_cast<const uint32_t*>(src + (staged ? staged_row(r) : r) * 8 + atom * 4) : 0u;
+        *reinterpret_cast<uint32_t*>(dst + metis_sf_offset(g_row0 + r, g_blk0 + atom * 4, bpr, layout)) = w;
+      }
+    } else {
+      for (int i = threadIdx.x; i < TILE * 8; i += THREADS) {
+        int r, b;
+        if (tiled) { const int atom = i >> 9, w = i & 511; r = (w >> 4) + 32 * ((w >> 2) & 3); b = atom * 4 + (w & 3); }
+        else { r = i >> 3; b = i & 7; }
+        if (b * 16 < v_k && (r < v_rows || tiled))
+          dst[metis_sf_offset(g_row0 + r, g_blk0 + b, bpr, layout)] = r < v_rows ? src[(staged ? staged_row(r) : r) * 8 + b] : (uint8_t)0;
+      }
+    }
+  };
   const int tid = threadIdx.x;
   const int64_t row0 = (int64_t)blockIdx.y * TILE, col0 = (int64_t)blockIdx.x * TILE;
   const float s_T = tscale_is_amax ? metis_tensor_scale(*tscale_src) : *tscale_src;
@@ -232,25 +256,9 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
       if (c < vcols && seg * 16 < vrows)
         *reinterpret_cast<uint2*>(p.r_codes + (col0 + c) * kbytes + row0 / 2 + seg * 8) = *reinterpret_cast<const uint2*>(codes_s + staged_row(c) * QK_CP + seg * 8);
     }
-    const int64_t bpr = p.rows / 16;
-    for (int i = tid; i < TILE * 8; i += THREADS) {
-      int c, b;
-      if (p.r_layout == METIS_SF_TILED) { const int atom = i >> 9, w = i & 511; c = (w >> 4) + 32 * ((w >> 2) & 3); b = atom * 4 + (w & 3); }
-      else { c = i >> 3; b = i & 7; }
-      if (b * 16 < vrows && (c < vcols || p.r_layout == METIS_SF_TILED))
-        p.r_scales[metis_sf_offset(col0 + c, row0 / 16 + b, bpr, p.r_layout)] = c < vcols ? sfr[staged_row(c) * 8 + b] : (uint8_t)0;
-    }
+    write_scales(p.r_scales, p.r_layout, p.rows / 16, sfr, true, vcols, vrows, col0, row0 / 16);
   }
-  if (want_c) {
-    const int64_t bpr = p.cols / 16;
-    for (int i = tid; i < TILE * 8; i += THREADS) {
-      int r, b;
-      if (p.c_layout == METIS_SF_TILED) { const int atom = i >> 9, w = i & 511; r = (w >> 4) + 32 * ((w >> 2) & 3); b = atom * 4 + (w & 3); }
-      else { r = i >> 3; b = i & 7; }
-      if (b * 16 < vcols && (r < vrows || p.c_layout == METIS_SF_TILED))
-        p.c_scales[metis_sf_offset(row0 + r, col0 / 16 + b, bpr, p.c_layout)] = r < vrows ? sfc[r * 8 + b] : (uint8_t)0;
-    }
-  }
+  if (want_c) write_scales(p.c_scales, p.c_layout, p.cols / 16, sfc, false, vrows, vcols, row0, col0 / 16);
 }
 
 template <typename T>
