@@ -315,6 +315,7 @@ def main():
                          "its stored residual and factors are re-quantized every step (the paper's per-step work for weights)")
     ap.add_argument("--workloads", default="all", help="comma-separated workload names (default: all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-fp4-probe", action="store_true", help="skip the 16384^3 product that measures the GEMM kernel's own best rate")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying CUDA graphs")
     ap.add_argument("--side-streams", type=int, default=2, help="streams (and library handles) per operand kind for the weight and gradient decompositions")
     ap.add_argument("--sustain-seconds", type=float, default=1.0, help="length of the sustained timing loop of every workload")
@@ -643,6 +644,22 @@ def main():
         "sustained": hd["rec"]["sustained"],
         "workloads": records,
     }
+    if rank == 0 and not args.no_fp4_probe:
+        # the kernel's own best rate: one 16384^3 product (221 tiles of 256 x 256 per CTA pair and 64 K blocks per tile), random codes
+        n_p = 16384
+        src = torch.randn((n_p, n_p), dtype=torch.bfloat16, device="cuda")
+        qa, qb = B.NvFp4(n_p, n_p), B.NvFp4(n_p, n_p)
+        handles[0].quantize_nvfp4(src, B.BLOCKS_BOTH, B.ROUND_RNE, seed=1, out=(qa, qb))
+        del src
+        out_p = torch.empty((n_p, n_p), dtype=torch.bfloat16, device="cuda")
+        for _ in range(3):
+            handles[0].gemm_nvfp4(qa, qb, out=out_p)
+        torch.cuda.synchronize()
+        ms_p = timed_ms(torch, lambda i: handles[0].gemm_nvfp4(qa, qb, out=out_p), 10)
+        tf_p = 2.0 * n_p ** 3 / (ms_p * 1e-3) / 1e12
+        line["roofline"]["same_kernel_16384_cubed"] = {"ms": ms_p, "tflops": tf_p, "frac_of_peak": tf_p / fp4_peak,
+                                                       "frac_of_nominal_9000": tf_p / 9000.0}
+        del qa, qb, out_p
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample = 1024
         dt, f = oracle_sample_step(sample, 4242)
