@@ -187,8 +187,10 @@ chol_wide_kernel(const double* __restrict__ g, int n, double tol_rel, double* l_
 constexpr int TW_ROWS = 32, TW_HP = MAXQ_WIDE + 1;
 constexpr size_t TW_SMEM = sizeof(double) * ((size_t)TW_ROWS * TW_HP + 3 * CW_NB * CW_P);
 __global__ void __launch_bounds__(256)
-trsm_wide_kernel(float* __restrict__ z, int64_t n_rows, int n, const double* __restrict__ l, const double* __restrict__ dinv) {
+trsm_wide_kernel(float* __restrict__ z, int64_t n_rows, int n, const double* __restrict__ l, const double* __restrict__ dinv,
+                 const int* __restrict__ skip) {
   metis_pdl_wait();
+  if (skip != nullptr && *skip) return;
   extern __shared__ __align__(16) unsigned char tw_sm[];
   double (*Hs)[TW_HP] = reinterpret_cast<double (*)[TW_HP]>(tw_sm);
   double (*Ls)[CW_P] = reinterpret_cast<double (*)[CW_P]>(tw_sm + sizeof(double) * TW_ROWS * TW_HP);

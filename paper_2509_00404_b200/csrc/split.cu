@@ -1618,15 +1618,16 @@ metis_status_t launch_gemm64(cudaStream_t s, const metis_wide::Gemm64Args& g) {
 }
 
 // FP64 Gram matrix of n vectors (element (r, i) at v[r * sr + i * sv]) into gram1 (n x n), by slabs of rows
-metis_status_t launch_gram64(cudaStream_t s, const float* v, int64_t n_rows, int n, int64_t sr, int64_t sv, double* parts, double* gram1) {
+metis_status_t launch_gram64(cudaStream_t s, const float* v, int64_t n_rows, int n, int64_t sr, int64_t sv, double* parts, double* gram1,
+                             const int* skip = nullptr) {
   int64_t rpp = metis_ceil_div(metis_ceil_div(n_rows, WIDE_GRAM_PARTS), metis_wide::G64_R) * metis_wide::G64_R;
   if (rpp < 64) rpp = 64;
   const int n_parts = (int)metis_ceil_div(n_rows, rpp);
   const unsigned t = (unsigned)metis_ceil_div(n, metis_wide::G64_T);
   METIS_CUDA_TRY(metis_launch_pdl(metis_wide::gram64_kernel, dim3(t, t, (unsigned)n_parts), dim3(256), (size_t)0, s, v, n_rows, n, sr, sv, rpp, parts,
-                                  (const int*)nullptr)); METIS_COUNT_LAUNCH();
+                                  skip)); METIS_COUNT_LAUNCH();
   METIS_CUDA_TRY(metis_launch_pdl((reduce_gram_kernel), dim3((unsigned)metis_ceil_div(n * n, 32)), dim3(128), (size_t)(0), s, (const double*)parts, n_parts, n * n, gram1,
-                                  (const int*)nullptr)); METIS_COUNT_LAUNCH();
+                                  skip)); METIS_COUNT_LAUNCH();
   return METIS_OK;
 }
 
@@ -1698,15 +1699,19 @@ metis_status_t split_wide(metis_context* ctx, const __nv_bfloat16* x, int64_t ro
                                       z + j0, q)); METIS_COUNT_LAUNCH();
     }
   }
-  // (3) CholeskyQR2: both passes always (FP64 Gram matrix, blocked factorisation, blocked triangular solve)
+  // (3) CholeskyQR (FP64 Gram matrix, blocked factorisation, blocked triangular solve).  The first factorisation
+  // reports whether its smallest pivot is above 1e-8 of the largest diagonal entry; if so H is orthonormal to FP32
+  // rounding already and the kernels of the second pass return at once.
   {
     float* src = z;
+    int* cond_flag = reinterpret_cast<int*>(amax + 8);
     for (int pass = 0; pass < 2; ++pass) {
-      METIS_TRY(launch_gram64(s, src, n_r, q, q, 1, gram, gram1));
-      METIS_CUDA_TRY(metis_launch_pdl(metis_wide::chol_wide_kernel, dim3(1), dim3(1024), metis_wide::CW_SMEM, s, (const double*)gram1, q, 1e-13, lf, linv, (const int*)nullptr,
-                                      (int*)nullptr)); METIS_COUNT_LAUNCH();
+      const int* skip = pass ? cond_flag : nullptr;
+      METIS_TRY(launch_gram64(s, src, n_r, q, q, 1, gram, gram1, skip));
+      METIS_CUDA_TRY(metis_launch_pdl(metis_wide::chol_wide_kernel, dim3(1), dim3(1024), metis_wide::CW_SMEM, s, (const double*)gram1, q, 1e-13, lf, linv, skip,
+                                      pass ? (int*)nullptr : cond_flag)); METIS_COUNT_LAUNCH();
       METIS_CUDA_TRY(metis_launch_pdl(metis_wide::trsm_wide_kernel, dim3((unsigned)metis_ceil_div(n_r, metis_wide::TW_ROWS)), dim3(256), metis_wide::TW_SMEM, s, src, n_r, q,
-                                      (const double*)lf, (const double*)linv)); METIS_COUNT_LAUNCH();
+                                      (const double*)lf, (const double*)linv, skip)); METIS_COUNT_LAUNCH();
     }
   }                                                      // H = Z L^-T, in place
   // (4) M = H^T xr on the tensor cores, WIDE_PJ sketch columns per launch; eigen-decomposition of M M^T
