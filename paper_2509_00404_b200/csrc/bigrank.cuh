@@ -87,97 +87,141 @@ gram64_kernel(const float* __restrict__ v, int64_t n_rows, int n, int64_t sr, in
 //             what the triangular solve H = Z L^-T needs besides L itself (trsm_wide_kernel)
 //   well_conditioned  (optional) 1 when every pivot is above 1e-8 of the largest diagonal entry
 constexpr int CW_NB = 32, CW_P = CW_NB + 1;
-constexpr size_t CW_SMEM = sizeof(double) * ((size_t)2 * MAXQ_WIDE * CW_P + CW_NB * CW_P + MAXQ_WIDE);
+constexpr int CW_ROWS = (MAXQ_WIDE + 15) / 16 * 16 + 16;   // rows of the shared panels: every row a thread's 4 x 4 tile may read exists
+constexpr size_t CW_SMEM = sizeof(double) * ((size_t)2 * CW_ROWS * CW_P + CW_NB * CW_P + MAXQ_WIDE);
+
+// acc[a][b] += sum over kk < 32 of  A[row0 + a][kk] * Bm[col0 + 8 b][kk]:  the 4 x 4 register tile of the panel products.
+// The rows of a warp's four row groups and the columns col0 + 8 b of its eight column groups fall on distinct banks
+// (pitch 33 doubles), so a step costs 8 shared-memory wavefronts per 16 multiply-adds of a warp.
+__device__ __forceinline__ void cw_tile_mac(const double (*A)[CW_P], const double (*Bm)[CW_P], int row0, int col0, double (&acc)[4][4]) {
+#pragma unroll 4
+  for (int kk = 0; kk < CW_NB; ++kk) {
+    double av[4], bv[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) { av[t] = A[row0 + t][kk]; bv[t] = Bm[col0 + 8 * t][kk]; }
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b2 = 0; b2 < 4; ++b2) acc[a][b2] += av[a] * bv[b2];
+  }
+}
+
+// Blocked (left-looking) Cholesky factor of the n x n matrix g (symmetrised on the fly), one CTA, panels of 32 columns:
+//   1. the panel (rows j0 .. n-1) minus the products with the finished columns, in 4 x 4 register tiles, the finished
+//      columns streamed from global memory (L2) in chunks of 32;
+//   2. the 32 x 32 diagonal block factorised by one warp (lane = row, column by column, one warp barrier per column);
+//   3. the inverse of that factor by the same warp (lane = column);
+//   4. the rows below the block:  L = A X^T  with X the inverse, again in register tiles.
+// A pivot at or below tol_rel * max diag gives a zero column.  l_out: the factor (lower triangle, zeros above);
+// dinv_out: the inverses of the diagonal blocks (32 x 32 each) for the blocked triangular solve.
 __global__ void __launch_bounds__(1024, 1)
 chol_wide_kernel(const double* __restrict__ g, int n, double tol_rel, double* l_out, double* dinv_out,
                  const int* __restrict__ skip, int* __restrict__ well_conditioned) {
   metis_pdl_wait();
   if (skip != nullptr && *skip) return;
   extern __shared__ __align__(16) unsigned char cw_sm[];
-  double (*P)[CW_P] = reinterpret_cast<double (*)[CW_P]>(cw_sm);                                   // the panel, rows j0 .. n-1
-  double (*As)[CW_P] = reinterpret_cast<double (*)[CW_P]>(cw_sm + sizeof(double) * MAXQ_WIDE * CW_P);    // a chunk of finished columns of those rows
-  double (*Dv)[CW_P] = reinterpret_cast<double (*)[CW_P]>(cw_sm + sizeof(double) * 2 * MAXQ_WIDE * CW_P);
-  double* rinv = reinterpret_cast<double*>(cw_sm + sizeof(double) * (2 * MAXQ_WIDE * CW_P + CW_NB * CW_P));
+  double (*P)[CW_P] = reinterpret_cast<double (*)[CW_P]>(cw_sm);                                      // the panel, rows j0 .. n-1
+  double (*As)[CW_P] = reinterpret_cast<double (*)[CW_P]>(cw_sm + sizeof(double) * CW_ROWS * CW_P);   // a chunk of finished columns of those rows
+  double (*Dv)[CW_P] = reinterpret_cast<double (*)[CW_P]>(cw_sm + sizeof(double) * 2 * CW_ROWS * CW_P);
+  double* rinv = reinterpret_cast<double*>(cw_sm + sizeof(double) * (2 * CW_ROWS * CW_P + CW_NB * CW_P));
   __shared__ double red[32];
-  __shared__ double gmax_s, dmin_s;
+  __shared__ double gmax_s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   for (int o = tid; o < n * n; o += 1024) l_out[o] = 0.0;
+  for (int o = tid; o < 2 * CW_ROWS * CW_P; o += 1024) reinterpret_cast<double*>(cw_sm)[o] = 0.0;   // rows past the matrix read as zeros
   double gm = 0.0;
   for (int i = tid; i < n; i += 1024) gm = fmax(gm, g[(int64_t)i * n + i]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) gm = fmax(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, o));
   if (lane == 0) red[warp] = gm;
   __syncthreads();
-  if (tid == 0) { double m = 0.0; for (int w = 0; w < 32; ++w) m = fmax(m, red[w]); gmax_s = m; dmin_s = 1e300; }
+  if (tid == 0) { double m = 0.0; for (int w2 = 0; w2 < 32; ++w2) m = fmax(m, red[w2]); gmax_s = m; }
   __syncthreads();
   const double tol = tol_rel * gmax_s;
-  const int tr = warp, tc = lane;                           // thread: panel column tc, rows tr + 32 m
-  constexpr int RM = (MAXQ_WIDE + 31) / 32;
+  double dmin = 1e300;                                     // smallest accepted pivot (warp 0 keeps it)
+  const int row0 = 4 * (tid >> 3), col0 = tid & 7;         // this thread's tile: rows row0 .. row0 + 3, columns col0 + 8 b
   for (int j0 = 0; j0 < n; j0 += CW_NB) {
     const int w = min(CW_NB, n - j0), nr = n - j0;
+    const bool mine = row0 < nr;
+    __syncthreads();                                       // the previous panel is stored
     for (int o = tid; o < nr * CW_NB; o += 1024) {
       const int i = o / CW_NB, c = o % CW_NB;
       P[i][c] = c < w ? 0.5 * (g[(int64_t)(j0 + i) * n + j0 + c] + g[(int64_t)(j0 + c) * n + j0 + i]) : 0.0;
     }
-    double acc[RM];
+    // ---- 1. minus the products with the finished columns ----
+    double acc[4][4];
 #pragma unroll
-    for (int m = 0; m < RM; ++m) acc[m] = 0.0;
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b2 = 0; b2 < 4; ++b2) acc[a][b2] = 0.0;
     for (int k0 = 0; k0 < j0; k0 += CW_NB) {
       __syncthreads();
       for (int o = tid; o < nr * CW_NB; o += 1024) { const int i = o / CW_NB, kk = o % CW_NB; As[i][kk] = l_out[(int64_t)(j0 + i) * n + k0 + kk]; }
       __syncthreads();
-      if (tc < w) {
-#pragma unroll 4
-        for (int kk = 0; kk < CW_NB; ++kk) {
-          const double b = As[tc][kk];                      // rows j0 .. j0 + w - 1 of L are the first rows of the chunk
+      if (mine) cw_tile_mac(As, As, row0, col0, acc);      // rows j0 .. j0 + 31 of L are the first rows of the chunk
+    }
+    __syncthreads();
+    if (mine) {
 #pragma unroll
-          for (int m = 0; m < RM; ++m) if (tr + 32 * m < nr) acc[m] += As[tr + 32 * m][kk] * b;
-        }
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b2 = 0; b2 < 4; ++b2)
+          if (row0 + a < nr && col0 + 8 * b2 < w) P[row0 + a][col0 + 8 * b2] -= acc[a][b2];
+    }
+    __syncthreads();
+    // ---- 2. and 3.: the diagonal block and its inverse, warp 0 ----
+    if (warp == 0) {
+      for (int c = 0; c < w; ++c) {
+        double s0 = 0.0, s1 = 0.0;
+        int k = 0;
+        for (; k + 1 < c; k += 2) { s0 += P[lane][k] * P[c][k]; s1 += P[lane][k + 1] * P[c][k + 1]; }
+        if (k < c) s0 += P[lane][k] * P[c][k];
+        const double sv = P[lane][c] - (s0 + s1);
+        const double d = __shfl_sync(0xFFFFFFFFu, sv, c);
+        const double r = d > tol ? 1.0 / sqrt(d) : 0.0;
+        if (lane >= c && lane < w) P[lane][c] = lane == c ? d * r : sv * r;
+        if (lane == 0) { rinv[j0 + c] = r; if (d > tol) dmin = fmin(dmin, d); }
+        __syncwarp();
+      }
+      // X = L^-1, lane = column:  X[i][j] = -r_i sum_{k < i} L[i][k] X[k][j]  (X[k][j] = 0 for k < j),  X[j][j] = r_j
+      for (int i = 0; i < CW_NB; ++i) Dv[i][lane] = 0.0;
+      __syncwarp();
+      for (int i = 0; i < w; ++i) {
+        double s0 = 0.0, s1 = 0.0;
+        int k = 0;
+        for (; k + 1 < i; k += 2) { s0 += P[i][k] * Dv[k][lane]; s1 += P[i][k + 1] * Dv[k + 1][lane]; }
+        if (k < i) s0 += P[i][k] * Dv[k][lane];
+        const double ri = rinv[j0 + i];
+        Dv[i][lane] = i == lane ? ri : (i > lane ? -ri * (s0 + s1) : 0.0);
       }
     }
     __syncthreads();
-    if (tc < w) {
+    // ---- 4. rows below the block: L = A X^T (X[c][cp] = Dv[c][cp], zero for cp > c) ----
+    if (nr > CW_NB) {
 #pragma unroll
-      for (int m = 0; m < RM; ++m) if (tr + 32 * m < nr) P[tr + 32 * m][tc] -= acc[m];
-    }
-    __syncthreads();
-    for (int c = 0; c < w; ++c) {
-      const double d = P[c][c];
-      const double r = d > tol ? 1.0 / sqrt(d) : 0.0;
-      __syncthreads();                                     // everybody has read the pivot
-      for (int i = c + tid; i < nr; i += 1024) P[i][c] = i == c ? d * r : P[i][c] * r;
-      if (tid == 0) { rinv[j0 + c] = r; if (d > tol) dmin_s = fmin(dmin_s, d); }
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b2 = 0; b2 < 4; ++b2) acc[a][b2] = 0.0;
+      const bool below = mine && row0 >= CW_NB;            // a tile lies wholly inside or wholly below the block
+      if (below) cw_tile_mac(P, Dv, row0, col0, acc);
+      __syncthreads();                                     // every tile has read its rows
+      if (below) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int b2 = 0; b2 < 4; ++b2)
+            if (row0 + a < nr) P[row0 + a][col0 + 8 * b2] = acc[a][b2];
+      }
       __syncthreads();
-      const int rest = w - c - 1;
-      for (int o = tid; o < (nr - c - 1) * rest; o += 1024) {
-        const int i = c + 1 + o / rest, cp = c + 1 + o % rest;
-        if (i >= cp) P[i][cp] -= P[i][c] * P[cp][c];
-      }
-      __syncthreads();                                     // the next pivot is final
     }
     for (int o = tid; o < nr * w; o += 1024) {
       const int i = o / w, c = o % w;
       if (i >= c) l_out[(int64_t)(j0 + i) * n + j0 + c] = P[i][c];
     }
-    if (dinv_out != nullptr) {
-      // inverse of the diagonal block, one lane per column: X[j][j] = 1 / L[j][j], X[i][j] = -X[i][i] sum_{k=j}^{i-1} L[i][k] X[k][j]
-      if (warp == 0) {
-        for (int i = 0; i < CW_NB; ++i) Dv[i][lane] = 0.0;
-        if (lane < w) {
-          Dv[lane][lane] = rinv[j0 + lane];
-          for (int i = lane + 1; i < w; ++i) {
-            double sacc = 0.0;
-            for (int k = lane; k < i; ++k) sacc += P[i][k] * Dv[k][lane];
-            Dv[i][lane] = -rinv[j0 + i] * sacc;
-          }
-        }
-      }
-      __syncthreads();
+    if (dinv_out != nullptr)
       for (int o = tid; o < CW_NB * CW_NB; o += 1024) dinv_out[(int64_t)(j0 / CW_NB) * CW_NB * CW_NB + o] = Dv[o / CW_NB][o % CW_NB];
-    }
-    __syncthreads();
   }
-  if (tid == 0 && well_conditioned != nullptr) *well_conditioned = (dmin_s > 1e-8 * gmax_s) ? 1 : 0;
+  if (tid == 0 && well_conditioned != nullptr) *well_conditioned = (dmin > 1e-8 * gmax_s) ? 1 : 0;
 }
 
 // H = Z L^-T by blocked forward substitution, in place: for panel J of CW_NB columns
