@@ -54,6 +54,24 @@ def test_quantizer_bit_exact_both_axes(ctx, rounding, layout):
     _compare(B, h, x, to_dev_bf16(x), B.BLOCKS_BOTH, rounding, layout)
 
 
+@pytest.mark.parametrize("rounding", [0, 1])
+def test_quantizer_strided_views_and_unaligned_scale_rows(ctx, rounding):
+    """The paths beside the fast one: a BF16 operand that is a column slice of a wider tensor (leading dimension larger
+    than the width, rows starting 16 bytes off a 32-byte boundary: no 32-byte loads), and a linear scale layout whose
+    rows are not a multiple of four blocks (scale bytes written one by one)."""
+    from gpu_util import to_dev_bf16
+    B, h = ctx
+    rng = np.random.default_rng(40 + rounding)
+    x = _adversarial(rng, 336, 400)                              # 25 and 21 blocks per stored row
+    wide = torch.zeros((336, 400 + 24), dtype=torch.bfloat16, device="cuda")
+    wide[:, 8:408] = to_dev_bf16(x)
+    view = wide[:, 8:408]
+    assert view.data_ptr() % 32 == 16 and view.stride(0) == 424
+    _compare(B, h, x, view, B.BLOCKS_BOTH, rounding, B.SF_LINEAR)
+    _compare(B, h, np.ascontiguousarray(x[:320, :384]), wide[:320, 8:392], B.BLOCKS_BOTH, rounding, B.SF_TILED)   # tiled scales want multiples of 64
+    _compare(B, h, x, to_dev_bf16(x), B.BLOCKS_BOTH, rounding, B.SF_LINEAR)
+
+
 def test_quantizer_fp32_input_given_scale_and_single_axis(ctx):
     B, h = ctx
     rng = np.random.default_rng(3)
