@@ -147,7 +147,8 @@ uint64_t metis_debug_launch_count(void);
 /* Bytes of scale storage for a stored rows x k_len NVFP4 tensor (host-only helper, no handle). */
 size_t metis_sf_bytes(int64_t rows, int64_t k_len, int32_t sf_layout);
 
-/* Workspace sizes (host-only helpers).  op: 0 quantize, 1 split, 2 linear_fwd, 3 linear_bwd.
+/* Workspace sizes (host-only helpers).  op: 0 quantize, 1 split, 2 linear_fwd, 3 linear_bwd, 4 split of an
+ * FP32 or strided operand (op 1 plus a contiguous BF16 copy of the operand).
  * rows/cols describe the largest operand (for the linear ops: rows = max(l, n), cols = max(m, n)). */
 metis_status_t metis_workspace_bytes(int32_t op, int64_t rows, int64_t cols, int32_t k, int32_t p, size_t* bytes);
 
@@ -186,8 +187,12 @@ metis_status_t metis_quantize_rht_nvfp4(metis_handle_t h, const void* x, int32_t
 
 /* ---- split (Sections 3.1, 3.2) ------------------------------------------------------------ */
 
-/* Splits x (rows x cols BF16, contiguous) into rank-k factors and a residual and quantizes all of
- * them into `out` (whose buffers the caller has allocated; out->k, rows, cols are checked).
+/* Splits x (rows x cols, leading dimension ld elements, BF16 or FP32) into rank-k factors and a residual and
+ * quantizes all of them into `out` (whose buffers the caller has allocated; out->k, rows, cols are checked).
+ * The decomposition runs on BF16 tensor-core passes over a contiguous operand: an FP32 operand is rounded to BF16
+ * (nearest even) and a strided one (ld > cols) is gathered, in one extra pass into the workspace, before anything
+ * else - ask metis_workspace_bytes for op 4 instead of 1 in those cases; ld % 8 == 0 (BF16) or ld % 4 == 0 (FP32).
+ * With k == 0 nothing is packed or rounded: x is quantized as metis_quantize_nvfp4 would.
  *  sketch = METIS_SKETCH_FULL:    Z = x Omega, thin QR, M = H^T x, small SVD, top k, residual
  *                                 x - A Lambda B^T.
  *  sketch = METIS_SKETCH_SAMPLED: the same on n_sample sampled rows (0 = default rule) to get the
@@ -199,7 +204,7 @@ metis_status_t metis_quantize_rht_nvfp4(metis_handle_t h, const void* x, int32_t
  * scale amax(x)/2688 of the SOURCE tensor; factors with their own.  `residual_axes` selects which
  * residual orientations are produced.  `residual_dense` (optional, rows x cols FP32) receives the
  * unquantized residual the quantizer saw.  k == 0 quantizes x itself.
- * src_amax (optional device scalar): amax|x| as the producer of x already knows it (e.g. from the epilogue of the
+ * src_amax (optional device scalar): amax|x| (of the BF16-rounded values, for an FP32 operand with k > 0) as the producer of x already knows it (e.g. from the epilogue of the
  * kernel that wrote x).  NULL: the library finds it - for k > 0 inside a pass it makes anyway, for k == 0 with a
  * reduction of its own, i.e. a second read of x that a supplied value saves.  The value is trusted: a value below
  * the true maximum makes the largest elements saturate.
@@ -210,8 +215,8 @@ metis_status_t metis_quantize_rht_nvfp4(metis_handle_t h, const void* x, int32_t
  * METIS_ERR_SHAPE.
  * Workspace: metis_workspace_bytes(1, rows, cols, k, p) (for the wide ranks: sized for the default sample count;
  * a larger n_sample may need more and is then refused with METIS_ERR_WORKSPACE). */
-metis_status_t metis_split(metis_handle_t h, const void* x, int64_t rows, int64_t cols, int32_t k, int32_t p,
-                           int32_t sketch, int64_t n_sample, uint64_t seed, int32_t rounding,
+metis_status_t metis_split(metis_handle_t h, const void* x, int32_t dtype, int64_t rows, int64_t cols, int64_t ld,
+                           int32_t k, int32_t p, int32_t sketch, int64_t n_sample, uint64_t seed, int32_t rounding,
                            int32_t residual_axes, const float* src_amax, metis_operand_t* out, float* residual_dense,
                            void* ws, size_t ws_bytes, metis_stream_t stream);
 

@@ -79,7 +79,7 @@ def lib():
     l.metis_quantize_nvfp4.argtypes = [vp, vp, i32, i64, i64, i64, i32, u64, u32, i32, P(NvFp4Struct), P(NvFp4Struct),
                                        vp, sz, vp]
     l.metis_quantize_rht_nvfp4.argtypes = [vp, vp, i32, i64, i64, i64, i32, u64, u32, P(NvFp4Struct), vp, sz, vp]
-    l.metis_split.argtypes = [vp, vp, i64, i64, i32, i32, i32, i64, u64, i32, i32, vp, P(OperandStruct), vp, vp, sz, vp]
+    l.metis_split.argtypes = [vp, vp, i32, i64, i64, i64, i32, i32, i32, i64, u64, i32, i32, vp, P(OperandStruct), vp, vp, sz, vp]
     l.metis_requantize_operand.argtypes = [vp, vp, i32, i64, i32, u64, i32, i32, P(OperandStruct), vp, sz, vp]
     l.metis_linear_fwd.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp, sz, vp]
     l.metis_linear_fwd_static_ws.argtypes = [vp, P(OperandStruct), P(OperandStruct), vp, i32, i64, vp]
@@ -265,10 +265,11 @@ class Handle:
         rows, cols = x.shape
         op = out if out is not None else Operand(rows, cols, k, axes)
         dense = torch.empty((rows, cols), dtype=torch.float32, device=x.device) if want_residual else None
-        need = workspace_bytes(1, rows, cols, k, p)
+        plain = x.dtype == torch.bfloat16 and x.stride(0) == cols
+        need = workspace_bytes(1 if plain else 4, rows, cols, k, p)
         ws = self.workspace(need)
         st = op.struct()
-        _check("metis_split", lib().metis_split(self._h, _ptr(x), rows, cols, k, p, sketch, n_sample, seed, rounding,
+        _check("metis_split", lib().metis_split(self._h, _ptr(x), _dtype_code(x), rows, cols, x.stride(0), k, p, sketch, n_sample, seed, rounding,
                                                 axes, _ptr(src_amax), ctypes.byref(st), _ptr(dense), _ptr(ws), ws.numel(),
                                                 _stream_ptr(stream)))
         return (op, dense) if want_residual else op

@@ -130,6 +130,8 @@ metis_status_t metis_workspace_bytes(int32_t op, int64_t rows, int64_t cols, int
     case 1: *bytes = metis_split_ws_bytes(rows, cols, k, p); return METIS_OK;
     case 2: *bytes = metis_linear_ws_bytes(rows, cols, k); return METIS_OK;
     case 3: *bytes = 2 * metis_linear_ws_bytes(rows, cols, k); return METIS_OK;    // two products' intermediates side by side
+    case 4: *bytes = ((metis_split_ws_bytes(rows, cols, k, p) + 255) & ~(size_t)255) +      // split of an FP32 or strided operand:
+                     (((size_t)rows * (size_t)cols * 2 + 255) & ~(size_t)255); return METIS_OK;   // plus its contiguous BF16 copy
     default: return METIS_ERR_INVALID_ARG;
   }
 }

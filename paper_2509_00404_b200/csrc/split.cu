@@ -1840,6 +1840,34 @@ metis_status_t metis_launch_amax_check(metis_context* ctx, const float* amax, cu
   return METIS_OK;
 }
 
+namespace {
+// contiguous BF16 copy of a strided BF16 or FP32 operand (FP32 rounded to nearest even), eight elements per thread
+__global__ void __launch_bounds__(256)
+pack_bf16_kernel(const void* __restrict__ x, int dtype, int64_t rows, int64_t cols, int64_t ld, __nv_bfloat16* __restrict__ out) {
+  metis_pdl_wait();
+  const int64_t g = (int64_t)blockIdx.x * 256 + threadIdx.x, per_row = cols / 8;
+  if (g >= rows * per_row) return;
+  const int64_t r = g / per_row, c = (g - r * per_row) * 8;
+  uint4 o;
+  if (dtype == METIS_BF16) {
+    o = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(x) + r * ld + c);
+  } else {
+    const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(x) + r * ld + c);
+    const float4 a = src[0], b = src[1];
+    __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x, a.y), h1 = __floats2bfloat162_rn(a.z, a.w);
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(b.x, b.y), h3 = __floats2bfloat162_rn(b.z, b.w);
+    o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+    o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+  }
+  *reinterpret_cast<uint4*>(out + r * cols + c) = o;
+}
+metis_status_t launch_pack_bf16(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, __nv_bfloat16* out, cudaStream_t s) {
+  METIS_CUDA_TRY(metis_launch_pdl(pack_bf16_kernel, dim3((unsigned)metis_ceil_div(rows * (cols / 8), 256)), dim3(256), (size_t)0, s, x, dtype, rows, cols, ld, out));
+  METIS_COUNT_LAUNCH();
+  return METIS_OK;
+}
+}  // namespace
+
 size_t metis_split_ws_bytes(int64_t rows, int64_t cols, int k, int p) {
   if (k > 0 && split_is_wide(k, p)) {
     // the larger of the FULL layout and the SAMPLED layout with the default sample count
@@ -1854,14 +1882,19 @@ size_t metis_split_ws_bytes(int64_t rows, int64_t cols, int k, int p) {
   return full > narrow ? full : narrow;
 }
 
-metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64_t cols, int32_t k, int32_t p,
+metis_status_t metis_split(metis_handle_t h, const void* xv, int32_t dtype, int64_t rows, int64_t cols, int64_t ld, int32_t k, int32_t p,
                            int32_t sketch, int64_t n_sample, uint64_t seed, int32_t rounding, int32_t residual_axes,
                            const float* src_amax, metis_operand_t* out, float* residual_dense, void* ws, size_t ws_bytes,
                            metis_stream_t stream) {
   METIS_NVTX("metis_split");
   using namespace metis_qt;
   if (!h || !xv || !out || !ws) return METIS_ERR_INVALID_ARG;
-  if (rows <= 0 || cols <= 0 || rows % 16 || cols % 16 || k < 0 || p < 0) return METIS_ERR_SHAPE;
+  if (dtype != METIS_BF16 && dtype != METIS_FP32) return METIS_ERR_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || rows % 16 || cols % 16 || k < 0 || p < 0 || ld < cols) return METIS_ERR_SHAPE;
+  if (ld % (dtype == METIS_BF16 ? 8 : 4)) return METIS_ERR_ALIGNMENT;          // every row starts on a 16-byte boundary
+  // anything but a contiguous BF16 operand is packed (and rounded) into the tail of the workspace first
+  const bool packed = k > 0 && (dtype != METIS_BF16 || ld != cols);
+  const size_t pack_bytes = packed ? (((size_t)rows * (size_t)cols * sizeof(__nv_bfloat16) + 255) & ~(size_t)255) : 0;
   if (k > 0 && (k > metis_wide::MAXK_WIDE || k + p > metis_wide::MAXQ_WIDE || k % 4)) return METIS_ERR_SHAPE;
   const bool wide = k > 0 && split_is_wide(k, p);
   if (out->k != k || out->rows != rows || out->cols != cols) return METIS_ERR_INVALID_ARG;
@@ -1880,28 +1913,39 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int64_t rows, int64
   if (k == 0) n_s = 16;
   if (wide) {
     // the tensor-core passes carry the wide path: 16-byte aligned rows of x, whole 64-column chunks
-    if (cols % 64 || rows % 64 || !metis_residual_tc_usable(xv, cols)) return METIS_ERR_SHAPE;
+    if (cols % 64 || rows % 64 || (!packed && !metis_residual_tc_usable(xv, cols))) return METIS_ERR_SHAPE;
     const WideWs W = wide_ws_layout(rows, cols, k, p, n_s, full);
-    if (ws_bytes < W.total) return METIS_ERR_WORKSPACE;
+    if (ws_bytes < W.total + pack_bytes) return METIS_ERR_WORKSPACE;
     if (!out->left || !out->sigma || !out->right || !out->left_q.codes || !out->right_q.codes || !out->left_q.scales ||
         !out->right_q.scales || !out->left_q.tensor_scale || !out->right_q.tensor_scale)
       return METIS_ERR_INVALID_ARG;
-    return split_wide(h, reinterpret_cast<const __nv_bfloat16*>(xv), rows, cols, k, p, full, n_s, seed, rounding, want_c, want_r, src_amax, out,
+    const __nv_bfloat16* xw = reinterpret_cast<const __nv_bfloat16*>(xv);
+    if (packed) {
+      __nv_bfloat16* xp = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<unsigned char*>(ws) + ((W.total + 255) & ~(size_t)255));
+      METIS_TRY(launch_pack_bf16(xv, dtype, rows, cols, ld, xp, reinterpret_cast<cudaStream_t>(stream)));
+      xw = xp;
+    }
+    return split_wide(h, xw, rows, cols, k, p, full, n_s, seed, rounding, want_c, want_r, src_amax, out,
                       residual_dense, reinterpret_cast<unsigned char*>(ws), W, reinterpret_cast<cudaStream_t>(stream));
   }
   const SplitWs L = split_ws_layout(rows, cols, k, p, n_s);
-  if (ws_bytes < L.total) return METIS_ERR_WORKSPACE;
+  if (ws_bytes < L.total + pack_bytes) return METIS_ERR_WORKSPACE;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   unsigned char* wsb = reinterpret_cast<unsigned char*>(ws);
   const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(xv);
+  if (packed) {
+    __nv_bfloat16* xp = reinterpret_cast<__nv_bfloat16*>(wsb + ((L.total + 255) & ~(size_t)255));
+    METIS_TRY(launch_pack_bf16(xv, dtype, rows, cols, ld, xp, s));
+    x = xp;
+  }
   float* amax = reinterpret_cast<float*>(wsb + L.amax);
 
   metis_nvfp4_t rc = out->res_by_cols, rr = out->res_by_rows;
   rc.rows = rows; rc.k_len = cols; rr.rows = cols; rr.k_len = rows;
   if (k == 0) {
     if (src_amax != nullptr) METIS_CUDA_TRY(cudaMemcpyAsync(amax, src_amax, sizeof(float), cudaMemcpyDeviceToDevice, s));
-    else METIS_TRY(metis_launch_amax(x, METIS_BF16, rows, cols, cols, amax, s));
-    METIS_TRY(metis_launch_quantize(x, METIS_BF16, rows, cols, cols, rounding, seed, METIS_STREAM_RESIDUAL, cols, 1, amax,
+    else METIS_TRY(metis_launch_amax(xv, dtype, rows, cols, ld, amax, s));
+    METIS_TRY(metis_launch_quantize(xv, dtype, rows, cols, ld, rounding, seed, METIS_STREAM_RESIDUAL, cols, 1, amax,
                                     1, want_c ? &rc : nullptr, want_r ? &rr : nullptr, s));
     METIS_CUDA_TRY(metis_launch_pdl((split_status_kernel), dim3(1), dim3(32), (size_t)(0), s, amax, (const double*)nullptr, 0, h->dev_status)); METIS_COUNT_LAUNCH();
     return METIS_OK;

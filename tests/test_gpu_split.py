@@ -293,6 +293,48 @@ def test_supplied_source_amax_gives_the_same_bytes(ctx, k):
         assert ta == tb and np.array_equal(ca, cb) and np.array_equal(sa, sb)
 
 
+def _same_operand(a, b):
+    from gpu_util import nv_to_numpy
+    for name in ("left_q", "right_q", "res_by_cols", "res_by_rows"):
+        ca, sa, ta = nv_to_numpy(getattr(a, name))
+        cb, sb, tb = nv_to_numpy(getattr(b, name))
+        assert ta == tb and np.array_equal(ca, cb) and np.array_equal(sa, sb), name
+    for name in ("left", "sigma", "right"):
+        assert torch.equal(getattr(a, name), getattr(b, name)), name
+
+
+@pytest.mark.parametrize("k", [0, 8, 80])
+def test_strided_and_fp32_operands_give_the_bytes_of_the_contiguous_bf16_operand(ctx, k):
+    """metis_split takes a leading dimension and FP32 input: the operand is gathered / rounded to BF16 once and the
+    decomposition is that of the contiguous BF16 tensor, byte for byte (k = 0 quantizes the FP32 values themselves)."""
+    from gpu_util import to_dev_bf16, nv_to_numpy
+    B, h = ctx
+    rows, cols, p = 512, 768, (8 if k else 0)
+    x, _ = synth.llama_like(rows, cols, 1.0, 73, rank=16)
+    xd = to_dev_bf16(x)
+    ref = h.split(xd, k, p, seed=5)
+    wide = torch.zeros((rows, cols + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, 24:24 + cols] = xd
+    view = wide[:, 24:24 + cols]
+    assert view.stride(0) == cols + 64 and view.data_ptr() % 16 == 0
+    _same_operand(ref, h.split(view, k, p, seed=5))
+    _same_operand(ref, h.split(xd.float(), k, p, seed=5))                      # BF16 values held in FP32
+    noisy = xd.float() * (1.0 + 1e-3 * torch.randn((rows, cols), device="cuda"))   # not representable in BF16
+    got = h.split(noisy, k, p, seed=5)
+    if k:
+        _same_operand(h.split(noisy.bfloat16(), k, p, seed=5), got)
+    else:
+        qc, qr = h.quantize_nvfp4(noisy, B.BLOCKS_BOTH, B.ROUND_RNE, seed=5)
+        for mine, theirs in ((got.res_by_cols, qc), (got.res_by_rows, qr)):
+            ca, sa, ta = nv_to_numpy(mine)
+            cb, sb, tb = nv_to_numpy(theirs)
+            assert ta == tb and np.array_equal(ca, cb) and np.array_equal(sa, sb)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    with pytest.raises(B.MetisError):
+        h.split(wide[:, 4:4 + cols], k, p, seed=5)                             # rows not 16-byte aligned
+
+
 def test_workspace_and_shape_errors(ctx):
     B, h = ctx
     x = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
