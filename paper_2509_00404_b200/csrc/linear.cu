@@ -141,82 +141,109 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
   }
 }
 
-// The same finishing step for ranks above 64 (up to 256 per operand), in two kernels.  First the FP32 operands:
-// one warp per row, the k_a x k_b matrix P staged through shared memory in slabs of 32 rows shared by the CTA's
-// eight rows.
+// Ranks above 64: the same finishing step as three kernels that tile over the rank.
+//   lowrank_deq_wide_kernel    Lcat[:, kb:] = Fo_a sa and Rcat[:, :kb] = Fo_b from the NVFP4 factors (a thread
+//                              dequantizes eight consecutive rows of one vector from one 32-bit load)
+//   lowrank_gemm_wide_kernel   Lcat[:, :kb] = (G1 + Lcat[:, kb:] P) sb, a 64 x 64 x 16 tiled FP32 product, 4 x 4 per thread
+//   lowrank_bf16_kernel        the BF16 correction operands, eight columns per thread
 constexpr int LW_MAXK = 256;
 __global__ void __launch_bounds__(256)
-lowrank_finish_wide_kernel(int64_t M, int64_t N, int ka, int kb,
-                           const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts, const float* sa,
-                           const uint8_t* fob_codes, const uint8_t* fob_sf, int fob_layout, const float* fob_ts, const float* sb,
-                           const float* __restrict__ pm, float* __restrict__ lcat, float* __restrict__ rcat) {
-  __shared__ float ps[32][LW_MAXK];
-  __shared__ float fa[8][LW_MAXK];
+lowrank_deq_wide_kernel(int64_t M, int64_t N, int ka, int kb,
+                        const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts, const float* sa,
+                        const uint8_t* fob_codes, const uint8_t* fob_sf, int fob_layout, const float* fob_ts,
+                        float* __restrict__ lcat, float* __restrict__ rcat) {
   metis_pdl_wait();
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int kc = ka + kb;
-  const int64_t i = (int64_t)blockIdx.x * 8 + warp;
+  const int tid = threadIdx.x, kc = ka + kb;
+  const int64_t i0 = (int64_t)blockIdx.x * 32 + 8 * (tid & 3);      // this thread's eight rows (M, N are multiples of 16)
   const float tsa = ka ? *foa_ts : 0.0f, tsb = kb ? *fob_ts : 0.0f;
-  if (i < M)
-    for (int u = lane; u < ka; u += 32) {
-      const float v = deq_of(foa_codes[(int64_t)u * (M / 2) + i / 2], foa_sf[metis_sf_offset(u, i / 16, M / 16, foa_layout)], i) * tsa * sa[u];
-      fa[warp][u] = v;
-      lcat[i * kc + kb + u] = v;
+  for (int u = tid >> 2; u < ka; u += 64) {
+    if (i0 >= M) break;
+    const uint32_t word = *reinterpret_cast<const uint32_t*>(foa_codes + (int64_t)u * (M / 2) + i0 / 2);
+    const float sc = metis_e4m3_value(foa_sf[metis_sf_offset(u, i0 / 16, M / 16, foa_layout)]), su = sa[u];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) lcat[(i0 + j) * kc + kb + u] = metis_e2m1_value((word >> (4 * j)) & 15u) * sc * tsa * su;
+  }
+  for (int t = tid >> 2; t < kb; t += 64) {
+    if (i0 >= N) break;
+    const uint32_t word = *reinterpret_cast<const uint32_t*>(fob_codes + (int64_t)t * (N / 2) + i0 / 2);
+    const float sc = metis_e4m3_value(fob_sf[metis_sf_offset(t, i0 / 16, N / 16, fob_layout)]);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) rcat[(i0 + j) * kc + t] = metis_e2m1_value((word >> (4 * j)) & 15u) * sc * tsb;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+lowrank_gemm_wide_kernel(int64_t M, int ka, int kb, const float* __restrict__ sb, const float* __restrict__ pm, float* __restrict__ lcat) {
+  metis_pdl_wait();
+  constexpr int KT = 16;
+  __shared__ __align__(16) float as[KT][68], bs[KT][68];   // [u][row], [u][column]
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15, kc = ka + kb;
+  const int64_t m0 = (int64_t)blockIdx.y * 64;
+  const int n0 = blockIdx.x * 64;
+  float acc[4][4] = {};
+  for (int u0 = 0; u0 < ka; u0 += KT) {
+    __syncthreads();
+    for (int o = tid; o < 64 * KT; o += 256) {
+      const int uu = o % KT, r = o / KT;                    // consecutive threads: consecutive u of one row (contiguous in Lcat)
+      as[uu][r] = (m0 + r < M && u0 + uu < ka) ? lcat[(m0 + r) * kc + kb + u0 + uu] : 0.0f;
+      const int t = o % 64, u2 = o / 64;                    // consecutive threads: consecutive columns of one row of P
+      bs[u2][t] = (u0 + u2 < ka && n0 + t < kb) ? pm[(int64_t)(u0 + u2) * kb + n0 + t] : 0.0f;
     }
-  if (i < N)
-    for (int t = lane; t < kb; t += 32)
-      rcat[i * kc + t] = deq_of(fob_codes[(int64_t)t * (N / 2) + i / 2], fob_sf[metis_sf_offset(t, i / 16, N / 16, fob_layout)], i) * tsb;
-  float acc[LW_MAXK / 32];
-#pragma unroll
-  for (int j = 0; j < LW_MAXK / 32; ++j) { const int t = lane + 32 * j; acc[j] = (i < M && t < kb) ? lcat[i * kc + t] : 0.0f; }
-  for (int u0 = 0; u0 < ka; u0 += 32) {
     __syncthreads();
-    for (int o = tid; o < 32 * kb; o += 256) { const int uu = o / kb, t = o % kb; ps[uu][t] = u0 + uu < ka ? pm[(int64_t)(u0 + uu) * kb + t] : 0.0f; }
-    __syncthreads();
-    if (i < M) {
-      const int nu = min(32, ka - u0);
-      for (int uu = 0; uu < nu; ++uu) {
-        const float f = fa[warp][u0 + uu];
 #pragma unroll
-        for (int j = 0; j < LW_MAXK / 32; ++j) { const int t = lane + 32 * j; if (t < kb) acc[j] = fmaf(f, ps[uu][t], acc[j]); }
-      }
+    for (int uu = 0; uu < KT; ++uu) {
+      const float4 a = *reinterpret_cast<const float4*>(&as[uu][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&bs[uu][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
     }
   }
-  if (i < M) {
 #pragma unroll
-    for (int j = 0; j < LW_MAXK / 32; ++j) { const int t = lane + 32 * j; if (t < kb) lcat[i * kc + t] = acc[j] * sb[t]; }
+  for (int i = 0; i < 4; ++i) {
+    const int64_t r = m0 + ty * 4 + i;
+    if (r >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int t = n0 + tx * 4 + j;
+      if (t < kb) lcat[r * kc + t] = (lcat[r * kc + t] + acc[i][j]) * sb[t];
+    }
   }
 }
 
 // Then the BF16 operands of the in-accumulator correction from the finished FP32 ones:
-// Lx = [Lh | Lh | Ll] / alpha,  Rx = [Rh | Rl | Rh], zero padded to kx columns.  One thread per (row, column).
+// Lx = [Lh | Lh | Ll] / alpha,  Rx = [Rh | Rl | Rh], zero padded to kx columns.  One thread per row and eight columns.
 __global__ void __launch_bounds__(256)
 lowrank_bf16_kernel(int64_t M, int64_t N, int kc, int kx, const float* __restrict__ lcat, const float* __restrict__ rcat,
                     __nv_bfloat16* __restrict__ lx, __nv_bfloat16* __restrict__ rx, const float* res_a_ts, const float* res_b_ts) {
   metis_pdl_wait();
   const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
   const int64_t mx = M > N ? M : N;
-  if (idx >= mx * kx) return;
-  const int64_t i = idx / kx;
-  const int c = (int)(idx % kx), seg = c / kc, t = c - seg * kc;
+  const int per_row = kx / 8;
+  if (idx >= mx * per_row) return;
+  const int64_t i = idx / per_row;
+  const int c0 = (int)(idx - i * per_row) * 8;
   const float inv_alpha = 1.0f / ((*res_a_ts) * (*res_b_ts));
-  if (i < M) {
-    float out = 0.0f;
-    if (seg < 3) {
-      const float v = lcat[i * kc + t] * inv_alpha;
-      const float h = __bfloat162float(__float2bfloat16_rn(v));
-      out = seg == 2 ? v - h : h;
+#pragma unroll
+  for (int side = 0; side < 2; ++side) {
+    if (i >= (side ? N : M)) continue;
+    const float* src = side ? rcat : lcat;
+    const int lo_seg = side ? 1 : 2;                        // the segment that carries the low parts
+    __align__(16) __nv_bfloat16 o[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int c = c0 + e, seg = c / kc, t = c - seg * kc;
+      float out = 0.0f;
+      if (seg < 3) {
+        const float v = side ? src[i * kc + t] : src[i * kc + t] * inv_alpha;
+        const float h = __bfloat162float(__float2bfloat16_rn(v));
+        out = seg == lo_seg ? v - h : h;
+      }
+      o[e] = __float2bfloat16_rn(out);
     }
-    lx[i * kx + c] = __float2bfloat16_rn(out);
-  }
-  if (i < N) {
-    float out = 0.0f;
-    if (seg < 3) {
-      const float v = rcat[i * kc + t];
-      const float h = __bfloat162float(__float2bfloat16_rn(v));
-      out = seg == 1 ? v - h : h;
-    }
-    rx[i * kx + c] = __float2bfloat16_rn(out);
+    *reinterpret_cast<uint4*>((side ? rx : lx) + i * kx + c0) = *reinterpret_cast<const uint4*>(o);
   }
 }
 
@@ -479,12 +506,16 @@ metis_status_t split_gemm_prologue(metis_context* ctx, const Side& a, const Side
   METIS_TRY(metis_join(ctx, s, side0 + 1));
   const int64_t mx = M > N ? M : N;
   if (ka > 64 || kb > 64) {
-    METIS_CUDA_TRY(metis_launch_pdl(lowrank_finish_wide_kernel, dim3((unsigned)metis_ceil_div(mx, 8)), dim3(256), 0, s,
+    METIS_CUDA_TRY(metis_launch_pdl(lowrank_deq_wide_kernel, dim3((unsigned)metis_ceil_div(mx, 32)), dim3(256), 0, s,
         M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
         ka ? a.fo->tensor_scale : nullptr, a.sigma, kb ? b.fo->codes : nullptr, kb ? b.fo->scales : nullptr,
-        kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, b.sigma, (const float*)pl.pm, pl.lcat, pl.rcat)); METIS_COUNT_LAUNCH();
+        kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, pl.lcat, pl.rcat)); METIS_COUNT_LAUNCH();
+    if (kb) {
+      METIS_CUDA_TRY(metis_launch_pdl(lowrank_gemm_wide_kernel, dim3((unsigned)metis_ceil_div(kb, 64), (unsigned)metis_ceil_div(M, 64)), dim3(256), 0, s,
+          M, ka, kb, b.sigma, (const float*)pl.pm, pl.lcat)); METIS_COUNT_LAUNCH();
+    }
     if (pl.lx != nullptr) {
-      METIS_CUDA_TRY(metis_launch_pdl(lowrank_bf16_kernel, dim3((unsigned)metis_ceil_div(mx * pl.kx, 256)), dim3(256), 0, s, M, N, kc, pl.kx,
+      METIS_CUDA_TRY(metis_launch_pdl(lowrank_bf16_kernel, dim3((unsigned)metis_ceil_div(mx * (pl.kx / 8), 256)), dim3(256), 0, s, M, N, kc, pl.kx,
           (const float*)pl.lcat, (const float*)pl.rcat, pl.lx, pl.rx, (const float*)a.res->tensor_scale, (const float*)b.res->tensor_scale)); METIS_COUNT_LAUNCH();
     }
     METIS_CUDA_TRY(cudaGetLastError());
