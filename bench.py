@@ -661,7 +661,7 @@ def main():
                                                        "frac_of_nominal_9000": tf_p / 9000.0}
         del qa, qb, out_p
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        sample = 1024
+        sample = 4096
         dt, f = oracle_sample_step(sample, 4242)
         line["cpu_baseline"] = {"value": f / dt / 1e12, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle",
                                 "sample": "the q projection of the block (4096->4096) on %d of 16384 tokens, one pass (%.1f s)" % (sample, dt)}
