@@ -31,7 +31,8 @@ constexpr int RING = 3;
 constexpr int SLOT_BYTES = 2 * TM * BK * 2;               // A6 chunk + B6 chunk, 16 KiB each
 constexpr int X_BYTES = TM * TN * 2;                      // two 64-column boxes of 16 KiB
 constexpr int N_EW = 16;                                  // epilogue warps: four TMEM lane quarters x four column quarters
-constexpr int PATCH_F = 32 * 17;                          // floats per warp patch (32 rows x 16 columns, odd pitch)
+constexpr int PATCH_HALF = 16 * 20 + 16;                   // 16 rows of 20 floats; the second half starts 16 banks further
+constexpr int PATCH_F = 2 * PATCH_HALF;                   // floats per warp patch (32 rows x 16 columns)
 constexpr int PATCH_U = 32 * 18;                          // 16-bit draws per warp patch
 constexpr int NUM_THREADS = 64 + 32 * N_EW;               // producer, MMA issuer, epilogue warps
 constexpr size_t SMEM_BYTES = (size_t)RING * SLOT_BYTES + 2 * X_BYTES + N_EW * (PATCH_F * 4 + PATCH_U * 2) + 1024 + 256 + metis_qt::R_TABLE * 4;
@@ -279,8 +280,12 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         const bool rb_ok = FAST || slab_row0 + 16 * rb < p.rows;
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
+          {
+            // one row of 16 values per lane as four 16-byte stores (rows 80 bytes apart: a quarter warp covers all banks)
+            float4* dst = reinterpret_cast<float4*>(patch + (lane >> 4) * PATCH_HALF + (lane & 15) * 20);
 #pragma unroll
-          for (int i = 0; i < 16; ++i) patch[lane * 17 + i] = v[16 * hf + i];
+            for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[16 * hf + 4 * j], v[16 * hf + 4 * j + 1], v[16 * hf + 4 * j + 2], v[16 * hf + 4 * j + 3]);
+          }
           if (sr) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) upatch[lane * 18 + i] = (uint16_t)(u[16 * hf + i] >> 16);
@@ -292,7 +297,7 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
           uint32_t d[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            t[i] = patch[(16 * rb + i) * 17 + cb];
+            t[i] = patch[rb * PATCH_HALF + i * 20 + cb];
             d[i] = sr ? (uint32_t)upatch[(16 * rb + i) * 18 + cb] << 16 : 0u;
           }
           uint32_t pk[2];
