@@ -319,6 +319,10 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying CUDA graphs")
     ap.add_argument("--side-streams", type=int, default=2, help="streams (and library handles) per operand kind for the weight and gradient decompositions")
     ap.add_argument("--sustain-seconds", type=float, default=1.0, help="length of the sustained timing loop of every workload")
+    ap.add_argument("--dry-run-ranks-on-one-gpu", action="store_true",
+                    help="control-flow check of the multi-rank path on a one-GPU box: every rank uses device 0 and the weight "
+                         "gradients are summed over gloo (host-staged, so no kernel of one rank waits for another); "
+                         "the line is marked and its numbers mean nothing")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -336,9 +340,14 @@ def main():
     if world != args.gpus:
         sys.stderr.write("bench.py: --gpus %d does not match WORLD_SIZE %d\n" % (args.gpus, world))
         sys.exit(2)
+    if args.dry_run_ranks_on_one_gpu:
+        local_rank = 0
     torch.cuda.set_device(local_rank)
     if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        if args.dry_run_ranks_on_one_gpu:
+            dist.init_process_group("gloo")
+        else:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     n_side = max(1, args.side_streams)
     handles = (B.Handle(local_rank), [B.Handle(local_rank) for _ in range(n_side)], [B.Handle(local_rank) for _ in range(n_side)])   # one workspace owner per stream
     streams = ([torch.cuda.Stream() for _ in range(n_side)], [torch.cuda.Stream() for _ in range(n_side)])
@@ -665,6 +674,8 @@ def main():
         dt, f = oracle_sample_step(sample, 4242)
         line["cpu_baseline"] = {"value": f / dt / 1e12, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle",
                                 "sample": "the q projection of the block (4096->4096) on %d of 16384 tokens, one pass (%.1f s)" % (sample, dt)}
+    if args.dry_run_ranks_on_one_gpu:
+        line["dry_run"] = "%d ranks on one GPU, gloo: control flow only, not a measurement" % world
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
