@@ -194,9 +194,10 @@ def spawn_ranks(n):
 class Workload:
     """Device buffers and the enqueue order of one workload on one rank."""
 
-    def __init__(self, name, spec, B, synth, handles, streams, weights_mode, world, rank, dw_sets=1):
+    def __init__(self, name, spec, B, synth, handles, streams, weights_mode, world, rank, dw_sets=1, act_sketch=None):
         import torch
         self.torch, self.B, self.name, self.spec = torch, B, name, spec
+        self.act_sketch = B.SKETCH_SAMPLED if act_sketch is None else act_sketch      # sketch mode of the activation and gradient operands
         # handles / streams: one for the activations and the forward products (the caller's current stream), N_SIDE
         # for the weights and N_SIDE for the output gradients and the backward products (layer j uses side j % N_SIDE,
         # so that the latency-bound start of one layer's decomposition runs beside the previous layer's big kernels)
@@ -267,7 +268,7 @@ class Workload:
         for j, ly in enumerate(self.layers):
             g = ly["x"]
             if g not in done_x:
-                self.h_x.split(x_in[g], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 1, rounding=B.ROUND_RNE, out=self.xo[g])
+                self.h_x.split(x_in[g], k, p, sketch=self.act_sketch, seed=3 * i + 1, rounding=B.ROUND_RNE, out=self.xo[g])
                 self.ev_x[g].record(main)
                 done_x.add(g)
             main.wait_event(self.ev_w[j])
@@ -276,7 +277,7 @@ class Workload:
             # its stream
             sd, hd = self.side_ds[j % n_d], self.h_ds[j % n_d]
             with torch.cuda.stream(sd):
-                hd.split(d_in[j], k, p, sketch=B.SKETCH_SAMPLED, seed=3 * i + 3, rounding=B.ROUND_SR, out=self.do[j], stream=sd)
+                hd.split(d_in[j], k, p, sketch=self.act_sketch, seed=3 * i + 3, rounding=B.ROUND_SR, out=self.do[j], stream=sd)
                 sd.wait_event(self.ev_x[g])
                 sd.wait_event(self.ev_w[j])
                 hd.linear_bwd(self.do[j], self.xo[g], self.wo[j], out=(dx[j], dw[j]), stream=sd)
@@ -564,6 +565,17 @@ def main():
                                                     "split_overhead_vs_plain_gemms": ms_r / ms_gemm - 1.0,
                                                     "stored_residual": "float32, re-quantized with its own amax/2688"}
             del wr, g_r
+            torch.cuda.empty_cache()
+            # The same block with every operand decomposed from all of its rows (the paper's "without sparse random
+            # sampling" ablation, Section 4 / Table 2): sketch, orthonormalisation and projection run over 16384 rows.
+            wf = Workload(name, spec, B, synth, handles, streams, args.weights, world, rank, dw_sets=1, act_sketch=B.SKETCH_FULL)
+            for i in range(args.warmup):
+                wf.step(i)
+            barrier()
+            ms_f = max_over_ranks([timed_ms(torch, wf.step, max(3, args.steps // 4))])[0]
+            rec["every_operand_full_sketch"] = {"ms_per_step": ms_f, "effective_tflops": world * wf.flops / (ms_f * 1e-3) / 1e12,
+                                                "split_overhead_vs_plain_gemms": ms_f / ms_gemm - 1.0, "cuda_graph": False}
+            del wf
             torch.cuda.empty_cache()
 
         if is_head:
