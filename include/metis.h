@@ -68,6 +68,7 @@ typedef enum {
 #define METIS_DEV_TIMEOUT 1u     /* a bounded wait inside a kernel expired                      */
 #define METIS_DEV_NUMERIC 2u     /* the small eigen-decomposition of a split produced a non-finite value */
 #define METIS_DEV_NONFINITE 4u   /* the operand of a split or of an amax-scaled quantization holds a NaN or an infinity */
+#define METIS_DEV_INDEX 8u       /* debug build only: a kernel was about to store outside an output buffer (the store was skipped) */
 
 typedef enum { METIS_BF16 = 0, METIS_FP32 = 1 } metis_dtype_t;
 typedef enum { METIS_ROUND_RNE = 0, METIS_ROUND_SR = 1 } metis_round_t;
@@ -140,6 +141,14 @@ metis_status_t metis_debug_timestamp(metis_handle_t h, uint64_t* device_slot, me
  * (device, two words) hold, per warp, bit 0 = "my wait expired", bit 1 = "the give-up flag was set".  The kernel
  * returns normally; the context stays usable. */
 metis_status_t metis_debug_wait_timeout(metis_handle_t h, uint32_t polls, uint32_t* device_seen, metis_stream_t stream);
+
+/* Debug build (compiled with METIS_DEBUG_BUILD; the Python binding loads it when METIS_DEBUG=1): the quantizing kernels
+ * check every global store of codes and scales against the extent of its output buffer and, instead of storing out
+ * of range, skip the store and set METIS_DEV_INDEX in the device status word.  metis_debug_build() tells which
+ * library this is (1 = debug).  metis_debug_index_check runs the same check in a one-thread kernel on a made-up
+ * store of nbytes at `offset` into a buffer of `extent` bytes (nothing is accessed): the self-test of the mechanism. */
+int32_t metis_debug_build(void);
+metis_status_t metis_debug_index_check(metis_handle_t h, int64_t offset, int64_t nbytes, int64_t extent, metis_stream_t stream);
 
 /* Test / benchmark hook: kernels launched by the library in this process so far (host counter, atomic). */
 uint64_t metis_debug_launch_count(void);

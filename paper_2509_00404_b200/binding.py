@@ -9,7 +9,8 @@ import os
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libmetis_b200.so")
+# METIS_DEBUG=1 selects the debug build of the same sources (index checks on every output store of the quantizing kernels)
+LIB_PATH = os.path.join(_PKG, "libmetis_b200_debug.so" if os.environ.get("METIS_DEBUG") == "1" else "libmetis_b200.so")
 
 OK = 0
 BF16, FP32 = 0, 1
@@ -19,13 +20,13 @@ TSCALE_AMAX_SELF, TSCALE_GIVEN = 0, 1
 SKETCH_FULL, SKETCH_SAMPLED = 0, 1
 SF_LINEAR, SF_TILED = 0, 1
 STREAM_RESIDUAL, STREAM_LEFT, STREAM_RIGHT = 0x10, 0x11, 0x12
-DEV_TIMEOUT, DEV_NUMERIC, DEV_NONFINITE = 1, 2, 4
+DEV_TIMEOUT, DEV_NUMERIC, DEV_NONFINITE, DEV_INDEX = 1, 2, 4, 8
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "ALIGNMENT", 4: "WORKSPACE", 5: "ARCH", 6: "CUDA",
                 7: "NONFINITE", 8: "NUMERIC", 9: "TIMEOUT"}
 
 EXPORTED = ["metis_create", "metis_destroy", "metis_last_device_status", "metis_debug_quantile_table",
-            "metis_debug_launch_count", "metis_debug_timestamp", "metis_debug_wait_timeout",
+            "metis_debug_launch_count", "metis_debug_timestamp", "metis_debug_wait_timeout", "metis_debug_build", "metis_debug_index_check",
             "metis_sf_bytes", "metis_workspace_bytes", "metis_default_sample_count", "metis_quantize_nvfp4", "metis_quantize_rht_nvfp4",
             "metis_split", "metis_requantize_operand", "metis_linear_fwd", "metis_linear_fwd_static_ws", "metis_linear_bwd", "metis_gemm_nvfp4"]
 
@@ -71,6 +72,9 @@ def lib():
     l.metis_debug_timestamp.argtypes = [vp, vp, vp]
     l.metis_debug_wait_timeout.argtypes = [vp, u32, vp, vp]
     l.metis_debug_launch_count.restype = u64
+    l.metis_debug_build.argtypes = []
+    l.metis_debug_build.restype = i32
+    l.metis_debug_index_check.argtypes = [vp, i64, i64, i64, vp]
     l.metis_sf_bytes.argtypes = [i64, i64, i32]
     l.metis_sf_bytes.restype = sz
     l.metis_workspace_bytes.argtypes = [i32, i64, i64, i32, i32, P(sz)]
@@ -87,7 +91,7 @@ def lib():
                                    i64, vp, vp, vp, vp, sz, vp]
     l.metis_gemm_nvfp4.argtypes = [vp, P(NvFp4Struct), P(NvFp4Struct), vp, i32, i64, i32, vp]
     for name in EXPORTED:
-        if name not in ("metis_sf_bytes", "metis_default_sample_count", "metis_debug_launch_count"):
+        if name not in ("metis_sf_bytes", "metis_default_sample_count", "metis_debug_launch_count", "metis_debug_build"):
             getattr(l, name).restype = ctypes.c_int
     _lib = l
     return l
@@ -113,6 +117,11 @@ def _dtype_code(t):
     if t.dtype == torch.float32:
         return FP32
     raise TypeError("expected a bfloat16 or float32 tensor")
+
+
+def debug_build():
+    """True when the loaded library is the debug build (METIS_DEBUG=1)."""
+    return bool(lib().metis_debug_build())
 
 
 def launch_count():
@@ -339,6 +348,10 @@ class Handle:
     def timestamp(self, slot, stream=None):
         """Enqueues a kernel that writes the GPU nanosecond timer into the int64 CUDA tensor element `slot`."""
         _check("metis_debug_timestamp", lib().metis_debug_timestamp(self._h, _ptr(slot), _stream_ptr(stream)))
+
+    def index_check(self, offset, nbytes, extent, stream=None):
+        """metis_debug_index_check: the debug build's store check on a made-up store (nothing is accessed)."""
+        _check("metis_debug_index_check", lib().metis_debug_index_check(self._h, offset, nbytes, extent, _stream_ptr(stream)))
 
     def wait_timeout(self, polls=256, stream=None):
         """metis_debug_wait_timeout: runs the bounded-wait hook; returns the two per-warp words as a CUDA int32 tensor."""

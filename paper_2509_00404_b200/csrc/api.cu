@@ -115,6 +115,27 @@ metis_status_t metis_debug_quantile_table(metis_handle_t h, uint16_t* host_out) 
   return METIS_OK;
 }
 
+namespace {
+__global__ void index_check_kernel(uint32_t* status, int64_t off, int64_t n, int64_t extent) {
+  (void)metis_dbg_ok(status, off, n, extent);
+}
+}  // namespace
+
+int32_t metis_debug_build(void) {
+#ifdef METIS_DEBUG_BUILD
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+metis_status_t metis_debug_index_check(metis_handle_t h, int64_t offset, int64_t nbytes, int64_t extent, metis_stream_t stream) {
+  if (!h || nbytes <= 0 || extent < 0) return METIS_ERR_INVALID_ARG;
+  index_check_kernel<<<1, 1, 0, reinterpret_cast<cudaStream_t>(stream)>>>(h->dev_status, offset, nbytes, extent); METIS_COUNT_LAUNCH();
+  METIS_CUDA_TRY(cudaGetLastError());
+  return METIS_OK;
+}
+
 uint64_t metis_debug_launch_count(void) { return g_metis_launch_count.load(std::memory_order_relaxed); }
 
 size_t metis_sf_bytes(int64_t rows, int64_t k_len, int32_t sf_layout) {
@@ -217,7 +238,7 @@ metis_status_t metis_quantize_nvfp4(metis_handle_t h, const void* x, int32_t dty
     ts_src = out_by_cols ? out_by_cols->tensor_scale : out_by_rows->tensor_scale;
   }
   return metis_launch_quantize(x, dtype, rows, cols, ld, rounding, seed, stream_id, cols, 1, ts_src, is_amax,
-                               out_by_cols, out_by_rows, s);
+                               out_by_cols, out_by_rows, s, h->dev_status);
 }
 
 metis_status_t metis_quantize_rht_nvfp4(metis_handle_t h, const void* x, int32_t dtype, int64_t rows, int64_t cols, int64_t ld,
@@ -274,7 +295,7 @@ metis_status_t metis_requantize_operand(metis_handle_t h, const void* residual, 
     ts_src = want_c ? rc.tensor_scale : rr.tensor_scale;
   }
   METIS_TRY(metis_launch_quantize(residual, res_dtype, rows, cols, ld_res, rounding, seed, METIS_STREAM_RESIDUAL, cols, 1, ts_src, is_amax,
-                                  want_c ? &rc : nullptr, want_r ? &rr : nullptr, s));
+                                  want_c ? &rc : nullptr, want_r ? &rr : nullptr, s, h->dev_status));
   if (k > 0) {
     METIS_TRY(metis_launch_amax(op->left, METIS_FP32, k, rows, rows, amax + 1, s));
     METIS_TRY(metis_launch_amax(op->right, METIS_FP32, k, cols, cols, amax + 2, s));

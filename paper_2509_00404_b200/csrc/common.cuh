@@ -212,13 +212,28 @@ __device__ __forceinline__ void metis_split3x8(const float (&v)[8], uint4& h, ui
 }
 
 
+// ---- debug-build index checks ----------------------------------------------------------------
+// metis_dbg_ok: is a store of n bytes at byte offset off inside a buffer of extent bytes?  If not, the status word gets
+// METIS_DEV_INDEX and the caller skips the store.  METIS_DBG_GUARD(...) stmt;  compiles to the bare statement in a
+// release build.
+__device__ __forceinline__ bool metis_dbg_ok(uint32_t* status, int64_t off, int64_t n, int64_t extent) {
+  if (off >= 0 && off + n <= extent) return true;
+  if (status != nullptr) atomicOr(status, METIS_DEV_INDEX);
+  return false;
+}
+#ifdef METIS_DEBUG_BUILD
+#define METIS_DBG_GUARD(status, off, n, extent) if (!metis_dbg_ok((status), (int64_t)(off), (int64_t)(n), (int64_t)(extent))) {} else
+#else
+#define METIS_DBG_GUARD(status, off, n, extent)
+#endif
+
 // ---- internal entry points shared between translation units --------------------------------
 metis_status_t metis_launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* amax_out,
                                  cudaStream_t s);
 metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int rounding,
                                      uint64_t seed, uint32_t stream_id, int64_t e_stride_r, int64_t e_stride_c,
                                      const float* tscale_src, int tscale_is_amax, const metis_nvfp4_t* by_cols,
-                                     const metis_nvfp4_t* by_rows, cudaStream_t s);
+                                     const metis_nvfp4_t* by_rows, cudaStream_t s, uint32_t* dbg_status = nullptr);
 int metis_coeff_slices(int64_t rows, int64_t cols, int* chunks_per_slice);
 bool metis_coeff_tc_usable(const void* x, const void* bs, int64_t cols, int kp);
 metis_status_t metis_launch_coeff_tc(metis_context* ctx, const void* x, int64_t rows, int64_t cols, const void* bs, int kp,

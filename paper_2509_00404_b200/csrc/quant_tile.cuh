@@ -19,6 +19,9 @@ struct QuantParams {
   // outputs (either may be absent: codes == nullptr)
   uint8_t* c_codes; uint8_t* c_scales; int c_layout;    // blocks along columns: stored rows x cols
   uint8_t* r_codes; uint8_t* r_scales; int r_layout;    // blocks along rows:    stored cols x rows
+  // debug build: extents of the scale buffers (the code buffers hold rows * cols / 2 bytes) and the status word
+  int64_t c_sf_bytes, r_sf_bytes;
+  uint32_t* dbg;
 };
 
 struct __align__(16) Stage {

@@ -76,7 +76,8 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
   // K group are adjacent in both layouts, so they go out as one word per thread (256 words per tile and orientation;
   // in the tiled layout consecutive threads write consecutive words of a 512-byte atom, and blocks or rows of the atom
   // that lie outside the matrix are its zero padding); an unaligned linear layout takes the byte path.
-  auto write_scales = [&](uint8_t* dst, int layout, int64_t bpr, const uint8_t* src, bool staged, int v_rows, int v_k, int64_t g_row0, int64_t g_blk0) {
+  auto write_scales = [&](uint8_t* dst, int64_t extent, int layout, int64_t bpr, const uint8_t* src, bool staged, int v_rows, int v_k, int64_t g_row0, int64_t g_blk0) {
+    (void)extent;
     const bool tiled = layout == METIS_SF_TILED;
     if ((tiled || (bpr & 3) == 0) && (reinterpret_cast<uintptr_t>(dst) & 3) == 0) {
       const int i = threadIdx.x;                                          // THREADS == 2 * TILE words
@@ -84,7 +85,8 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
       const int r = tiled ? ((i & 127) >> 2) + 32 * (i & 3) : i >> 1;
       if (atom * 64 < v_k && (r < v_rows || tiled)) {
         const uint32_t w = r < v_rows ? *reinterpret_cast<const uint32_t*>(src + (staged ? staged_row(r) : r) * 8 + atom * 4) : 0u;
-        *reinterpret_cast<uint32_t*>(dst + metis_sf_offset(g_row0 + r, g_blk0 + atom * 4, bpr, layout)) = w;
+        const int64_t off = metis_sf_offset(g_row0 + r, g_blk0 + atom * 4, bpr, layout);
+        METIS_DBG_GUARD(p.dbg, off, 4, extent) *reinterpret_cast<uint32_t*>(dst + off) = w;
       }
     } else {
       for (int i = threadIdx.x; i < TILE * 8; i += THREADS) {
@@ -92,7 +94,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
         if (tiled) { const int atom = i >> 9, w = i & 511; r = (w >> 4) + 32 * ((w >> 2) & 3); b = atom * 4 + (w & 3); }
         else { r = i >> 3; b = i & 7; }
         if (b * 16 < v_k && (r < v_rows || tiled))
-          dst[metis_sf_offset(g_row0 + r, g_blk0 + b, bpr, layout)] = r < v_rows ? src[(staged ? staged_row(r) : r) * 8 + b] : (uint8_t)0;
+          METIS_DBG_GUARD(p.dbg, metis_sf_offset(g_row0 + r, g_blk0 + b, bpr, layout), 1, extent) dst[metis_sf_offset(g_row0 + r, g_blk0 + b, bpr, layout)] = r < v_rows ? src[(staged ? staged_row(r) : r) * 8 + b] : (uint8_t)0;
       }
     }
   };
@@ -195,7 +197,7 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
     if (want_c) {
       uint32_t packed[2];
       const uint32_t byte = encode_block_tab(v, u, sr, six_s_T, r_tab, packed);
-      if (in) *reinterpret_cast<uint2*>(p.c_codes + gr * (p.cols / 2) + gc / 2) = make_uint2(packed[0], packed[1]);
+      if (in) METIS_DBG_GUARD(p.dbg, gr * (p.cols / 2) + gc / 2, 8, p.rows * p.cols / 2) *reinterpret_cast<uint2*>(p.c_codes + gr * (p.cols / 2) + gc / 2) = make_uint2(packed[0], packed[1]);
       sfc[r * 8 + b] = in ? (uint8_t)byte : (uint8_t)0;
     }
   }
@@ -254,11 +256,11 @@ quantize_kernel(const T* __restrict__ x, int64_t ld, metis_qt::QuantParams p, co
     for (int i = tid; i < TILE * 8; i += THREADS) {
       const int c = i >> 3, seg = i & 7;
       if (c < vcols && seg * 16 < vrows)
-        *reinterpret_cast<uint2*>(p.r_codes + (col0 + c) * kbytes + row0 / 2 + seg * 8) = *reinterpret_cast<const uint2*>(codes_s + staged_row(c) * QK_CP + seg * 8);
+        METIS_DBG_GUARD(p.dbg, (col0 + c) * kbytes + row0 / 2 + seg * 8, 8, p.rows * p.cols / 2) *reinterpret_cast<uint2*>(p.r_codes + (col0 + c) * kbytes + row0 / 2 + seg * 8) = *reinterpret_cast<const uint2*>(codes_s + staged_row(c) * QK_CP + seg * 8);
     }
-    write_scales(p.r_scales, p.r_layout, p.rows / 16, sfr, true, vcols, vrows, col0, row0 / 16);
+    write_scales(p.r_scales, p.r_sf_bytes, p.r_layout, p.rows / 16, sfr, true, vcols, vrows, col0, row0 / 16);
   }
-  if (want_c) write_scales(p.c_scales, p.c_layout, p.cols / 16, sfc, false, vrows, vcols, row0, col0 / 16);
+  if (want_c) write_scales(p.c_scales, p.c_sf_bytes, p.c_layout, p.cols / 16, sfc, false, vrows, vcols, row0, col0 / 16);
 }
 
 template <typename T>
@@ -437,7 +439,7 @@ quantize_rowblocks_pair_kernel(RowblocksJob a, RowblocksJob b) {
 metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int rounding,
                                      uint64_t seed, uint32_t stream_id, int64_t e_stride_r, int64_t e_stride_c,
                                      const float* tscale_src, int tscale_is_amax, const metis_nvfp4_t* by_cols,
-                                     const metis_nvfp4_t* by_rows, cudaStream_t s) {
+                                     const metis_nvfp4_t* by_rows, cudaStream_t s, uint32_t* dbg_status) {
   using namespace metis_qt;
   if (rows == 0 || cols == 0) return METIS_OK;
   // vector loads of 16 elements per thread: the rows must start on 16-byte boundaries
@@ -445,8 +447,9 @@ metis_status_t metis_launch_quantize(const void* x, int dtype, int64_t rows, int
   QuantParams p{};
   p.rows = rows; p.cols = cols; p.rounding = rounding; p.seed = seed; p.stream_id = stream_id;
   p.e_stride_r = e_stride_r; p.e_stride_c = e_stride_c;
-  if (by_cols) { p.c_codes = by_cols->codes; p.c_scales = by_cols->scales; p.c_layout = by_cols->sf_layout; }
-  if (by_rows) { p.r_codes = by_rows->codes; p.r_scales = by_rows->scales; p.r_layout = by_rows->sf_layout; }
+  if (by_cols) { p.c_codes = by_cols->codes; p.c_scales = by_cols->scales; p.c_layout = by_cols->sf_layout; p.c_sf_bytes = (int64_t)metis_sf_bytes(rows, cols, p.c_layout); }
+  if (by_rows) { p.r_codes = by_rows->codes; p.r_scales = by_rows->scales; p.r_layout = by_rows->sf_layout; p.r_sf_bytes = (int64_t)metis_sf_bytes(cols, rows, p.r_layout); }
+  p.dbg = dbg_status;
   if (dtype == METIS_FP32 && by_cols && !by_rows && rows <= 64) {
     const int64_t rows_pad = p.c_layout == METIS_SF_TILED ? (rows + 127) / 128 * 128 : rows;
     quantize_rowblocks_kernel<<<(unsigned)metis_ceil_div(rows_pad * (cols / 16), 256), 256, 0, s>>>(

@@ -247,6 +247,7 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 #pragma unroll
         for (int j = 0; j < 8; ++j)
           if (c0 + 4 * j < p.cols)
+            METIS_DBG_GUARD(g.dev_status, (row * p.cols + c0 + 4 * j) * 4, 16, p.rows * p.cols * 4)
             *reinterpret_cast<float4*>(g.dense + row * p.cols + c0 + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
       }
       if (p.c_codes != nullptr && step_ok) {
@@ -260,11 +261,14 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         const uint32_t sb1 = encode_block_tab(v1, u1, sr, six_s_T, r_tab, pk1);
         if (row_ok) {
           uint8_t* cp = p.c_codes + row * c_kbytes + c0 / 2;
-          if (blk1_ok) *reinterpret_cast<uint4*>(cp) = make_uint4(pk0[0], pk0[1], pk1[0], pk1[1]);
-          else *reinterpret_cast<uint2*>(cp) = make_uint2(pk0[0], pk0[1]);
+          METIS_DBG_GUARD(g.dev_status, row * c_kbytes + c0 / 2, blk1_ok ? 16 : 8, p.rows * c_kbytes) {
+            if (blk1_ok) *reinterpret_cast<uint4*>(cp) = make_uint4(pk0[0], pk0[1], pk1[0], pk1[1]);
+            else *reinterpret_cast<uint2*>(cp) = make_uint2(pk0[0], pk0[1]);
+          }
         }
         if (row_ok || c_layout == METIS_SF_TILED) {                         // padded rows of a 128-row slab get zero scales
           const int64_t o = metis_sf_offset(row, c0 / 16, c_bpr, c_layout);
+          METIS_DBG_GUARD(g.dev_status, o, 2, p.c_sf_bytes)
           if (FAST) {
             *reinterpret_cast<uint16_t*>(p.c_scales + o) = (uint16_t)(sb0 | (sb1 << 8));   // c0 / 16 is even: an aligned pair
           } else {
@@ -302,8 +306,10 @@ residual_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
           }
           uint32_t pk[2];
           const uint32_t sb = encode_block_tab(t, d, sr, six_s_T, r_tab, pk);
-          if (col_ok && rb_ok) *reinterpret_cast<uint2*>(p.r_codes + col * r_kbytes + (slab_row0 + 16 * rb) / 2) = make_uint2(pk[0], pk[1]);
+          if (col_ok && rb_ok) METIS_DBG_GUARD(g.dev_status, col * r_kbytes + (slab_row0 + 16 * rb) / 2, 8, p.cols * r_kbytes)
+            *reinterpret_cast<uint2*>(p.r_codes + col * r_kbytes + (slab_row0 + 16 * rb) / 2) = make_uint2(pk[0], pk[1]);
           if (rb_ok && (col_ok || r_layout == METIS_SF_TILED))               // padded columns of a 128-slab get zero scales
+            METIS_DBG_GUARD(g.dev_status, metis_sf_offset(col, slab_row0 / 16 + rb, r_bpr, r_layout), 1, p.r_sf_bytes)
             p.r_scales[metis_sf_offset(col, slab_row0 / 16 + rb, r_bpr, r_layout)] = col_ok ? (uint8_t)sb : (uint8_t)0;
           __syncwarp();
         }
@@ -356,7 +362,10 @@ metis_status_t metis_launch_residual_tc(metis_context* ctx, const void* x, const
   METIS_TRY(make_map_bf16(ctx, &ma, a6, rows, kx, kx, TM));
   METIS_TRY(make_map_bf16(ctx, &mb, b6, cols, kx, kx, TN));
   ResidArgs g{};
-  g.p = qp; g.amax_src = amax_src; g.ts_out0 = ts_out0; g.ts_out1 = ts_out1; g.dense = dense;
+  g.p = qp;
+  g.p.c_sf_bytes = qp.c_codes ? (int64_t)metis_sf_bytes(rows, cols, qp.c_layout) : 0;
+  g.p.r_sf_bytes = qp.r_codes ? (int64_t)metis_sf_bytes(cols, rows, qp.r_layout) : 0;
+  g.amax_src = amax_src; g.ts_out0 = ts_out0; g.ts_out1 = ts_out1; g.dense = dense;
   g.k_chunks = kx / BK;
   g.dev_status = ctx->dev_status;
   const bool fast = rows % TM == 0 && cols % TN == 0 && dense == nullptr &&

@@ -1946,7 +1946,7 @@ metis_status_t metis_split(metis_handle_t h, const void* xv, int32_t dtype, int6
     if (src_amax != nullptr) METIS_CUDA_TRY(cudaMemcpyAsync(amax, src_amax, sizeof(float), cudaMemcpyDeviceToDevice, s));
     else METIS_TRY(metis_launch_amax(xv, dtype, rows, cols, ld, amax, s));
     METIS_TRY(metis_launch_quantize(xv, dtype, rows, cols, ld, rounding, seed, METIS_STREAM_RESIDUAL, cols, 1, amax,
-                                    1, want_c ? &rc : nullptr, want_r ? &rr : nullptr, s));
+                                    1, want_c ? &rc : nullptr, want_r ? &rr : nullptr, s, h->dev_status));
     METIS_CUDA_TRY(metis_launch_pdl((split_status_kernel), dim3(1), dim3(32), (size_t)(0), s, amax, (const double*)nullptr, 0, h->dev_status)); METIS_COUNT_LAUNCH();
     return METIS_OK;
   }

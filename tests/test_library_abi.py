@@ -23,6 +23,14 @@ def test_library_builds_loads_and_exports_every_declared_symbol():
     for n in names:
         assert hasattr(lib, n), n
     assert sorted(binding.EXPORTED) == names
+    # the debug build (index checks on every output store) is the same sources with one macro: same symbols
+    import ctypes
+    dbg = ctypes.CDLL(build.LIB_DEBUG)
+    for n in names:
+        assert hasattr(dbg, n), n
+    dbg.metis_debug_build.restype = ctypes.c_int32
+    lib.metis_debug_build.restype = ctypes.c_int32
+    assert dbg.metis_debug_build() == 1 and lib.metis_debug_build() == 0
 
 
 def test_host_only_helpers():
