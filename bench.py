@@ -138,11 +138,13 @@ def oracle_sample_step(sample_tokens, seed, d_in=4096, d_out=4096, k=32, p=8):
     xq = olay.quantize_operand(x, k, p, osp.MODE_SAMPLED, seed)
     wq = olay.quantize_operand(w, k, p, osp.MODE_FULL, seed + 1)
     dq = olay.quantize_operand(d, k, p, osp.MODE_SAMPLED, seed + 2, onv.ROUND_SR)
+    t1 = time.perf_counter()
     y = olay.linear_fwd(xq, wq)
     dx = olay.linear_dgrad(dq, wq)
     dw = olay.linear_wgrad(dq, xq)
     dt = time.perf_counter() - t0
     assert np.isfinite(y).all() and np.isfinite(dx).all() and np.isfinite(dw).all()
+    oracle_sample_step.phases = {"split_and_quantize_s": t1 - t0, "three_products_s": dt - (t1 - t0)}
     return dt, 6.0 * sample_tokens * d_in * d_out
 
 
@@ -685,7 +687,8 @@ def main():
         sample = 4096
         dt, f = oracle_sample_step(sample, 4242)
         line["cpu_baseline"] = {"value": f / dt / 1e12, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle",
-                                "sample": "the q projection of the block (4096->4096) on %d of 16384 tokens, one pass (%.1f s)" % (sample, dt)}
+                                "sample": "the q projection of the block (4096->4096) on %d of 16384 tokens, one pass (%.1f s)" % (sample, dt),
+                                "phases": oracle_sample_step.phases}
     if args.dry_run_ranks_on_one_gpu:
         line["dry_run"] = "%d ranks on one GPU, gloo: control flow only, not a measurement" % world
     if rank == 0:
