@@ -320,7 +320,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fp4-probe", action="store_true", help="skip the 16384^3 product that measures the GEMM kernel's own best rate")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying CUDA graphs")
-    ap.add_argument("--side-streams", type=int, default=2, help="streams (and library handles) per operand kind for the weight and gradient decompositions")
+    ap.add_argument("--side-streams", type=int, default=4, help="streams (and library handles) per operand kind for the weight and gradient decompositions")
     ap.add_argument("--sustain-seconds", type=float, default=1.0, help="length of the sustained timing loop of every workload")
     ap.add_argument("--dry-run-ranks-on-one-gpu", action="store_true",
                     help="control-flow check of the multi-rank path on a one-GPU box: every rank uses device 0 and the weight "
