@@ -1348,7 +1348,7 @@ right_rotate_kernel(const float* __restrict__ basis, int64_t cols, int k, const 
       for (int i = 0; i < MAXQ; ++i) if (i == j) v = bv[i];
     }
     if (col < cols) right[(int64_t)j * cols + col] = v;
-    float av = col < cols ? fabsf(v) : -1.0f, sv = v;            // magnitude for the contest, signed value for the verdict
+    float av = col < cols ? fabsf(v) : -1.0f, sv = v;            // magnitude for the contest, signed value for the decision
     int ai = (int)min(col, (int64_t)0x7FFFFFFF);
 #pragma unroll
     for (int sft = 16; sft > 0; sft >>= 1) {
@@ -1373,7 +1373,7 @@ right_rotate_kernel(const float* __restrict__ basis, int64_t cols, int k, const 
 
 // Sign convention: the largest-magnitude entry of each right vector (lowest index on ties) is made positive.
 // grid (column chunks, k).  Every CTA re-derives the winner of its vector from the per-chunk candidates, whose
-// signed values were recorded before any flipping (the flips of other CTAs must not influence the verdict).
+// signed values were recorded before any flipping (the flips of other CTAs must not influence the decision).
 __global__ void __launch_bounds__(256)
 sign_fix_kernel(float* __restrict__ right, int64_t cols, int k, const float* __restrict__ cand_v,
                 const int* __restrict__ cand_i, int n_cand, float* __restrict__ sign_out, float* __restrict__ amax_out) {
