@@ -200,6 +200,7 @@ class Workload:
         import torch
         self.torch, self.B, self.name, self.spec = torch, B, name, spec
         self.act_sketch = B.SKETCH_SAMPLED if act_sketch is None else act_sketch      # sketch mode of the activation and gradient operands
+        self.amax = None                                     # optional: amax|operand| as its producer would hand it over
         # handles / streams: one for the activations and the forward products (the caller's current stream), N_SIDE
         # for the weights and N_SIDE for the output gradients and the backward products (layer j uses side j % N_SIDE,
         # so that the latency-bound start of one layer's decomposition runs beside the previous layer's big kernels)
@@ -247,6 +248,13 @@ class Workload:
         self.output_bytes = sum(t.numel() * t.element_size() for t in self.y + self.dx + self.dw_sets[0])
         del n_x
 
+    def with_producer_amax(self):
+        """amax|x| of every operand, found once outside any timed region: what the kernel that wrote the operand would
+        pass along (the split then runs no reduction of its own when k = 0)."""
+        am = lambda t: t.float().abs().max().reshape(1)
+        self.amax = ({g: am(t) for g, t in self.x_in.items()}, [am(t) for t in self.w_in], [am(t) for t in self.d_in])
+        return self
+
     def step(self, i, inputs=None, outs=None, dw_set=0):
         """Enqueues one step on the current stream and the two side streams (joined before it returns)."""
         torch, B = self.torch, self.B
@@ -264,13 +272,15 @@ class Workload:
                 if self.w_stored is not None:
                     hw.requantize_operand(self.wo[j], self.w_stored[j], seed=3 * i + 2, stream=sw)
                 else:
-                    hw.split(w_in[j], k, p, sketch=B.SKETCH_FULL, seed=3 * i + 2, rounding=B.ROUND_RNE, out=self.wo[j], stream=sw)
+                    hw.split(w_in[j], k, p, sketch=B.SKETCH_FULL, seed=3 * i + 2, rounding=B.ROUND_RNE, out=self.wo[j], stream=sw,
+                             src_amax=self.amax[1][j] if self.amax else None)
                 self.ev_w[j].record(sw)
         done_x = set()
         for j, ly in enumerate(self.layers):
             g = ly["x"]
             if g not in done_x:
-                self.h_x.split(x_in[g], k, p, sketch=self.act_sketch, seed=3 * i + 1, rounding=B.ROUND_RNE, out=self.xo[g])
+                self.h_x.split(x_in[g], k, p, sketch=self.act_sketch, seed=3 * i + 1, rounding=B.ROUND_RNE, out=self.xo[g],
+                                 src_amax=self.amax[0][g] if self.amax else None)
                 self.ev_x[g].record(main)
                 done_x.add(g)
             main.wait_event(self.ev_w[j])
@@ -279,7 +289,8 @@ class Workload:
             # its stream
             sd, hd = self.side_ds[j % n_d], self.h_ds[j % n_d]
             with torch.cuda.stream(sd):
-                hd.split(d_in[j], k, p, sketch=self.act_sketch, seed=3 * i + 3, rounding=B.ROUND_SR, out=self.do[j], stream=sd)
+                hd.split(d_in[j], k, p, sketch=self.act_sketch, seed=3 * i + 3, rounding=B.ROUND_SR, out=self.do[j], stream=sd,
+                         src_amax=self.amax[2][j] if self.amax else None)
                 sd.wait_event(self.ev_x[g])
                 sd.wait_event(self.ev_w[j])
                 hd.linear_bwd(self.do[j], self.xo[g], self.wo[j], out=(dx[j], dw[j]), stream=sd)
@@ -544,6 +555,18 @@ def main():
             "device_status": int(status),
         }
         records[name] = rec
+
+        if wl.k == 0:
+            # plain quantization with amax|x| supplied by the producer of each operand: no reduction pass inside the step
+            wa = Workload(name, spec, B, synth, handles, streams, args.weights, world, rank, dw_sets=1).with_producer_amax()
+            for i in range(args.warmup):
+                wa.step(i)
+            barrier()
+            ms_a = max_over_ranks([timed_ms(torch, wa.step, args.steps)])[0]
+            rec["amax_supplied_by_the_producer"] = {"ms_per_step": ms_a, "effective_tflops": world * wa.flops / (ms_a * 1e-3) / 1e12,
+                                                    "split_overhead_vs_plain_gemms": ms_a / ms_gemm - 1.0, "cuda_graph": False}
+            del wa
+            torch.cuda.empty_cache()
 
         if is_head and args.weights == "split" and wl.k:
             # The same block with the weights held as stored factors + residual and only re-quantized each step (the
