@@ -46,6 +46,7 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
   __shared__ float fa[8][64];
   __shared__ float lrow[8][128];
   __shared__ float rrow[8][128];
+  __shared__ float lraw[8][64], rraw[8][64];                // the factors as E2M1 x E4M3 products, before any FP32 scale
   metis_pdl_wait();
   metis_pdl_trigger();                                      // the large GEMM behind this kernel sets itself up meanwhile
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -83,7 +84,9 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
     for (int j = 0; j < 2; ++j) {
       const int u = lane + 32 * j;
       if (u < ka) {
-        const float v = deq_of(a_byte[j], a_sfb[j], i) * tsa * sa_v[j];
+        const float raw = deq_of(a_byte[j], a_sfb[j], i);
+        const float v = raw * tsa * sa_v[j];
+        lraw[warp][u] = raw;
         fa[warp][u] = v;
         lrow[warp][kb + u] = v;
         lcat[i * kc + kb + u] = v;
@@ -107,7 +110,9 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
     for (int j = 0; j < 2; ++j) {
       const int t = lane + 32 * j;
       if (t < kb) {
-        const float v = deq_of(b_byte[j], b_sfb[j], i) * tsb;
+        const float raw = deq_of(b_byte[j], b_sfb[j], i);
+        const float v = raw * tsb;
+        rraw[warp][t] = raw;
         rrow[warp][t] = v;
         rcat[i * kc + t] = v;
       }
@@ -115,29 +120,34 @@ lowrank_finish_kernel(int64_t M, int64_t N, int ka, int kb,
     }
   }
   if (lx == nullptr) return;
-  // BF16 operands of the in-accumulator correction:  Lx = [Lh | Lh | Ll] / alpha,  Rx = [Rh | Rl | Rh]
-  // (hi/lo two-term splits, three cross products), zero padded to kx columns.
+  // BF16 operands of the in-accumulator correction, zero padded to kx columns.  A dequantized factor entry is an
+  // E2M1 x E4M3 product (six significant bits): with its FP32 scales moved to the other operand it is exact in BF16
+  // and needs no low part, so each of the two rank-k terms costs two column groups instead of three:
+  //   Lx = [ A hi | A lo | Fa | Fa ],  A  = (G1 + Fo_a sa P) sb ts_b / alpha     (k_b columns), Fa = Fo_a / ts_a (k_a)
+  //   Rx = [ Fb   | Fb   | B hi | B lo ],  Fb = Fo_b / ts_b (k_b),  B = Wt sa ts_a / alpha          (k_a columns)
   __syncwarp();
+  const float l_scale = tsb * inv_alpha, r_scale = tsa * inv_alpha;
   for (int c = lane; c < kx; c += 32) {
-    const int seg = c / kc, t = c - seg * kc;
-    if (i < M) {
-      float out = 0.0f;
-      if (seg < 3) {
-        const float v = lrow[warp][t] * inv_alpha;
+    float lo_ = 0.0f, ro_ = 0.0f;
+    if (c < 2 * kb) {
+      const int t = c < kb ? c : c - kb;
+      if (i < M) {
+        const float v = lrow[warp][t] * l_scale;
         const float h = __bfloat162float(__float2bfloat16_rn(v));
-        out = seg == 2 ? v - h : h;
+        lo_ = c < kb ? h : v - h;
       }
-      lx[i * kx + c] = __float2bfloat16_rn(out);
-    }
-    if (i < N) {
-      float out = 0.0f;
-      if (seg < 3) {
-        const float v = rrow[warp][t];
+      if (i < N) ro_ = rraw[warp][t];
+    } else if (c < 2 * kc) {
+      const int u0 = c - 2 * kb, u = u0 < ka ? u0 : u0 - ka;
+      if (i < M) lo_ = lraw[warp][u];
+      if (i < N) {
+        const float v = rrow[warp][kb + u] * sa[u] * r_scale;
         const float h = __bfloat162float(__float2bfloat16_rn(v));
-        out = seg == 1 ? v - h : h;
+        ro_ = u0 < ka ? h : v - h;
       }
-      rx[i * kx + c] = __float2bfloat16_rn(out);
     }
+    if (i < M) lx[i * kx + c] = __float2bfloat16_rn(lo_);
+    if (i < N) rx[i * kx + c] = __float2bfloat16_rn(ro_);
   }
 }
 
@@ -213,38 +223,49 @@ lowrank_gemm_wide_kernel(int64_t M, int ka, int kb, const float* __restrict__ sb
   }
 }
 
-// Then the BF16 operands of the in-accumulator correction from the finished FP32 ones:
-// Lx = [Lh | Lh | Ll] / alpha,  Rx = [Rh | Rl | Rh], zero padded to kx columns.  One thread per row and eight columns.
+// Then the BF16 operands of the in-accumulator correction (the layout of lowrank_finish_kernel: the dequantized factors
+// exact in BF16, two column groups per rank-k term), zero padded to kx columns.  One thread per row and eight columns.
 __global__ void __launch_bounds__(256)
-lowrank_bf16_kernel(int64_t M, int64_t N, int kc, int kx, const float* __restrict__ lcat, const float* __restrict__ rcat,
+lowrank_bf16_kernel(int64_t M, int64_t N, int ka, int kb, int kx, const float* __restrict__ lcat, const float* __restrict__ rcat,
+                    const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts, const float* __restrict__ sa,
+                    const uint8_t* fob_codes, const uint8_t* fob_sf, int fob_layout, const float* fob_ts,
                     __nv_bfloat16* __restrict__ lx, __nv_bfloat16* __restrict__ rx, const float* res_a_ts, const float* res_b_ts) {
   metis_pdl_wait();
   const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
   const int64_t mx = M > N ? M : N;
-  const int per_row = kx / 8;
+  const int per_row = kx / 8, kc = ka + kb;
   if (idx >= mx * per_row) return;
   const int64_t i = idx / per_row;
   const int c0 = (int)(idx - i * per_row) * 8;
   const float inv_alpha = 1.0f / ((*res_a_ts) * (*res_b_ts));
+  const float l_scale = (kb ? *fob_ts : 0.0f) * inv_alpha, r_scale = (ka ? *foa_ts : 0.0f) * inv_alpha;
+  __align__(16) __nv_bfloat16 lo_[8], ro_[8];
 #pragma unroll
-  for (int side = 0; side < 2; ++side) {
-    if (i >= (side ? N : M)) continue;
-    const float* src = side ? rcat : lcat;
-    const int lo_seg = side ? 1 : 2;                        // the segment that carries the low parts
-    __align__(16) __nv_bfloat16 o[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int c = c0 + e, seg = c / kc, t = c - seg * kc;
-      float out = 0.0f;
-      if (seg < 3) {
-        const float v = side ? src[i * kc + t] : src[i * kc + t] * inv_alpha;
+  for (int e = 0; e < 8; ++e) {
+    const int c = c0 + e;
+    float lv = 0.0f, rv = 0.0f;
+    if (c < 2 * kb) {
+      const int t = c < kb ? c : c - kb;
+      if (i < M) {
+        const float v = lcat[i * kc + t] * l_scale;
         const float h = __bfloat162float(__float2bfloat16_rn(v));
-        out = seg == lo_seg ? v - h : h;
+        lv = c < kb ? h : v - h;
       }
-      o[e] = __float2bfloat16_rn(out);
+      if (i < N) rv = deq_of(fob_codes[(int64_t)t * (N / 2) + i / 2], fob_sf[metis_sf_offset(t, i / 16, N / 16, fob_layout)], i);
+    } else if (c < 2 * kc) {
+      const int u0 = c - 2 * kb, u = u0 < ka ? u0 : u0 - ka;
+      if (i < M) lv = deq_of(foa_codes[(int64_t)u * (M / 2) + i / 2], foa_sf[metis_sf_offset(u, i / 16, M / 16, foa_layout)], i);
+      if (i < N) {
+        const float v = rcat[i * kc + kb + u] * sa[u] * r_scale;
+        const float h = __bfloat162float(__float2bfloat16_rn(v));
+        rv = u0 < ka ? h : v - h;
+      }
     }
-    *reinterpret_cast<uint4*>((side ? rx : lx) + i * kx + c0) = *reinterpret_cast<const uint4*>(o);
+    lo_[e] = __float2bfloat16_rn(lv);
+    ro_[e] = __float2bfloat16_rn(rv);
   }
+  if (i < M) *reinterpret_cast<uint4*>(lx + i * kx + c0) = *reinterpret_cast<const uint4*>(lo_);
+  if (i < N) *reinterpret_cast<uint4*>(rx + i * kx + c0) = *reinterpret_cast<const uint4*>(ro_);
 }
 
 // out = y0 + Lcat Rcat^T, 64 x 64 tile per CTA
@@ -476,7 +497,7 @@ metis_status_t make_plan(const Side& a, const Side& b, void* ws, size_t ws_bytes
   auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
   pl->fuse = metis_gemm_tc_can_fuse(a.res, b.res);
   if (!pl->fuse && kc > 128) return METIS_ERR_SHAPE;    // layers below 256 rows hold the update operands in shared memory
-  pl->kx = (3 * kc + 63) / 64 * 64;
+  pl->kx = (2 * kc + 63) / 64 * 64;          // two BF16 column groups per rank-k term (see lowrank_finish_kernel)
   const size_t o_pm = take(sizeof(float) * (size_t)(ka * kb > 64 * 64 ? ka * kb : 64 * 64)), o_l = take(sizeof(float) * M * kc), o_r = take(sizeof(float) * N * kc);
   const size_t o_lx = pl->fuse ? take(sizeof(__nv_bfloat16) * M * pl->kx) : 0, o_rx = pl->fuse ? take(sizeof(__nv_bfloat16) * N * pl->kx) : 0;
   const size_t o_y0 = pl->fuse ? 0 : take(sizeof(float) * M * N);
@@ -515,8 +536,13 @@ metis_status_t split_gemm_prologue(metis_context* ctx, const Side& a, const Side
           M, ka, kb, b.sigma, (const float*)pl.pm, pl.lcat)); METIS_COUNT_LAUNCH();
     }
     if (pl.lx != nullptr) {
-      METIS_CUDA_TRY(metis_launch_pdl(lowrank_bf16_kernel, dim3((unsigned)metis_ceil_div(mx * (pl.kx / 8), 256)), dim3(256), 0, s, M, N, kc, pl.kx,
-          (const float*)pl.lcat, (const float*)pl.rcat, pl.lx, pl.rx, (const float*)a.res->tensor_scale, (const float*)b.res->tensor_scale)); METIS_COUNT_LAUNCH();
+      METIS_CUDA_TRY(metis_launch_pdl(lowrank_bf16_kernel, dim3((unsigned)metis_ceil_div(mx * (pl.kx / 8), 256)), dim3(256), 0, s, M, N, ka, kb, pl.kx,
+          (const float*)pl.lcat, (const float*)pl.rcat,
+          (const uint8_t*)(ka ? a.fo->codes : nullptr), (const uint8_t*)(ka ? a.fo->scales : nullptr), ka ? a.fo->sf_layout : 0,
+          (const float*)(ka ? a.fo->tensor_scale : nullptr), (const float*)a.sigma,
+          (const uint8_t*)(kb ? b.fo->codes : nullptr), (const uint8_t*)(kb ? b.fo->scales : nullptr), kb ? b.fo->sf_layout : 0,
+          (const float*)(kb ? b.fo->tensor_scale : nullptr),
+          pl.lx, pl.rx, (const float*)a.res->tensor_scale, (const float*)b.res->tensor_scale)); METIS_COUNT_LAUNCH();
     }
     METIS_CUDA_TRY(cudaGetLastError());
     return METIS_OK;
@@ -562,7 +588,7 @@ metis_status_t metis_linear_set_attrs() {
 
 size_t metis_linear_ws_bytes(int64_t M, int64_t N, int k) {
   const int kc = 2 * k;
-  const int kx = (3 * kc + 63) / 64 * 64;
+  const int kx = (2 * kc + 63) / 64 * 64;
   // sized for either path: FP32 staging of the main product (small shapes) or the BF16 correction operands
   const size_t pm_elems = (size_t)k * k > 64 * 64 ? (size_t)k * k : 64 * 64;
   return align256(sizeof(float) * M * N) + align256(sizeof(float) * pm_elems) +
