@@ -40,10 +40,10 @@ BYTES_PER_ELEM_BOTH = 3.125   # split / quantize: 2 B read + 2 x 0.5625 B writte
 
 
 # DRAM bytes of ONE launch of the two-CTA GEMM (dram__bytes_read.sum + dram__bytes_write.sum), per (M, N, K), from an
-# ncu capture of this program's block workload (a profiler cannot run inside the timed program).  Reads are 4.7 x the
+# ncu capture of this program's block workload (a profiler cannot run inside the timed program).  Reads are 4.3 x the
 # operand bytes at K = 4096 (the B panels are fetched once per group of eight tile rows); the bf16 output is written once.
-NCU_DRAM_BYTES = {(16384, 14336, 4096): 330.1e6 + 417.5e6, (16384, 4096, 14336): 331.9e6 + 111.9e6,
-                  (14336, 4096, 16384): 376.2e6 + 98.9e6}
+NCU_DRAM_BYTES = {(16384, 14336, 4096): 304.8e6 + 416.3e6, (16384, 4096, 14336): 321.3e6 + 113.2e6,
+                  (14336, 4096, 16384): 374.7e6 + 98.3e6}
 NCU_DRAM_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum -k regex:gemm_nvfp4_2cta on "
                    "`bench.py --workloads block_16384tok --no-graph`, one launch of this shape")
 
