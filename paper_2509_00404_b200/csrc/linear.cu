@@ -161,7 +161,8 @@ __global__ void __launch_bounds__(256)
 lowrank_deq_wide_kernel(int64_t M, int64_t N, int ka, int kb,
                         const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts, const float* sa,
                         const uint8_t* fob_codes, const uint8_t* fob_sf, int fob_layout, const float* fob_ts,
-                        float* __restrict__ lcat, float* __restrict__ rcat) {
+                        float* __restrict__ lcat, float* __restrict__ rcat,
+                        __nv_bfloat16* __restrict__ lx, __nv_bfloat16* __restrict__ rx, int kx) {
   metis_pdl_wait();
   const int tid = threadIdx.x, kc = ka + kb;
   const int64_t i0 = (int64_t)blockIdx.x * 32 + 8 * (tid & 3);      // this thread's eight rows (M, N are multiples of 16)
@@ -171,14 +172,30 @@ lowrank_deq_wide_kernel(int64_t M, int64_t N, int ka, int kb,
     const uint32_t word = *reinterpret_cast<const uint32_t*>(foa_codes + (int64_t)u * (M / 2) + i0 / 2);
     const float sc = metis_e4m3_value(foa_sf[metis_sf_offset(u, i0 / 16, M / 16, foa_layout)]), su = sa[u];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) lcat[(i0 + j) * kc + kb + u] = metis_e2m1_value((word >> (4 * j)) & 15u) * sc * tsa * su;
+    for (int j = 0; j < 8; ++j) {
+      const float raw = metis_e2m1_value((word >> (4 * j)) & 15u) * sc;
+      lcat[(i0 + j) * kc + kb + u] = raw * tsa * su;
+      if (lx != nullptr) {                                  // the exact factor entry, both of its column groups
+        const __nv_bfloat16 e = __float2bfloat16_rn(raw);
+        lx[(i0 + j) * kx + 2 * kb + u] = e;
+        lx[(i0 + j) * kx + 2 * kb + ka + u] = e;
+      }
+    }
   }
   for (int t = tid >> 2; t < kb; t += 64) {
     if (i0 >= N) break;
     const uint32_t word = *reinterpret_cast<const uint32_t*>(fob_codes + (int64_t)t * (N / 2) + i0 / 2);
     const float sc = metis_e4m3_value(fob_sf[metis_sf_offset(t, i0 / 16, N / 16, fob_layout)]);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) rcat[(i0 + j) * kc + t] = metis_e2m1_value((word >> (4 * j)) & 15u) * sc * tsb;
+    for (int j = 0; j < 8; ++j) {
+      const float raw = metis_e2m1_value((word >> (4 * j)) & 15u) * sc;
+      rcat[(i0 + j) * kc + t] = raw * tsb;
+      if (rx != nullptr) {
+        const __nv_bfloat16 e = __float2bfloat16_rn(raw);
+        rx[(i0 + j) * kx + t] = e;
+        rx[(i0 + j) * kx + kb + t] = e;
+      }
+    }
   }
 }
 
@@ -223,12 +240,13 @@ lowrank_gemm_wide_kernel(int64_t M, int ka, int kb, const float* __restrict__ sb
   }
 }
 
-// Then the BF16 operands of the in-accumulator correction (the layout of lowrank_finish_kernel: the dequantized factors
-// exact in BF16, two column groups per rank-k term), zero padded to kx columns.  One thread per row and eight columns.
+// Then the general halves of the BF16 correction operands (the layout of lowrank_finish_kernel): [A hi | A lo] of Lx and
+// [B hi | B lo] of Rx from the finished FP32 operands, and the zero padding up to kx columns; the exact factor groups
+// were written by lowrank_deq_wide_kernel.  One thread per row and eight columns (the group boundaries 2 k_b and
+// 2 (k_a + k_b) are multiples of eight).
 __global__ void __launch_bounds__(256)
 lowrank_bf16_kernel(int64_t M, int64_t N, int ka, int kb, int kx, const float* __restrict__ lcat, const float* __restrict__ rcat,
-                    const uint8_t* foa_codes, const uint8_t* foa_sf, int foa_layout, const float* foa_ts, const float* __restrict__ sa,
-                    const uint8_t* fob_codes, const uint8_t* fob_sf, int fob_layout, const float* fob_ts,
+                    const float* foa_ts, const float* __restrict__ sa, const float* fob_ts,
                     __nv_bfloat16* __restrict__ lx, __nv_bfloat16* __restrict__ rx, const float* res_a_ts, const float* res_b_ts) {
   metis_pdl_wait();
   const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
@@ -239,33 +257,34 @@ lowrank_bf16_kernel(int64_t M, int64_t N, int ka, int kb, int kx, const float* _
   const int c0 = (int)(idx - i * per_row) * 8;
   const float inv_alpha = 1.0f / ((*res_a_ts) * (*res_b_ts));
   const float l_scale = (kb ? *fob_ts : 0.0f) * inv_alpha, r_scale = (ka ? *foa_ts : 0.0f) * inv_alpha;
-  __align__(16) __nv_bfloat16 lo_[8], ro_[8];
+  __align__(16) __nv_bfloat16 o[8];
+  if (c0 < 2 * kb) {                                        // [A hi | A lo]
+    if (i < M) {
 #pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    const int c = c0 + e;
-    float lv = 0.0f, rv = 0.0f;
-    if (c < 2 * kb) {
-      const int t = c < kb ? c : c - kb;
-      if (i < M) {
+      for (int e = 0; e < 8; ++e) {
+        const int c = c0 + e, t = c < kb ? c : c - kb;
         const float v = lcat[i * kc + t] * l_scale;
         const float h = __bfloat162float(__float2bfloat16_rn(v));
-        lv = c < kb ? h : v - h;
+        o[e] = __float2bfloat16_rn(c < kb ? h : v - h);
       }
-      if (i < N) rv = deq_of(fob_codes[(int64_t)t * (N / 2) + i / 2], fob_sf[metis_sf_offset(t, i / 16, N / 16, fob_layout)], i);
-    } else if (c < 2 * kc) {
-      const int u0 = c - 2 * kb, u = u0 < ka ? u0 : u0 - ka;
-      if (i < M) lv = deq_of(foa_codes[(int64_t)u * (M / 2) + i / 2], foa_sf[metis_sf_offset(u, i / 16, M / 16, foa_layout)], i);
-      if (i < N) {
+      *reinterpret_cast<uint4*>(lx + i * kx + c0) = *reinterpret_cast<const uint4*>(o);
+    }
+  } else if (c0 < 2 * kc) {                                 // [B hi | B lo]
+    if (i < N) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int u0 = c0 + e - 2 * kb, u = u0 < ka ? u0 : u0 - ka;
         const float v = rcat[i * kc + kb + u] * sa[u] * r_scale;
         const float h = __bfloat162float(__float2bfloat16_rn(v));
-        rv = u0 < ka ? h : v - h;
+        o[e] = __float2bfloat16_rn(u0 < ka ? h : v - h);
       }
+      *reinterpret_cast<uint4*>(rx + i * kx + c0) = *reinterpret_cast<const uint4*>(o);
     }
-    lo_[e] = __float2bfloat16_rn(lv);
-    ro_[e] = __float2bfloat16_rn(rv);
+  } else {                                                  // padding of both operands
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    if (i < M) *reinterpret_cast<uint4*>(lx + i * kx + c0) = z;
+    if (i < N) *reinterpret_cast<uint4*>(rx + i * kx + c0) = z;
   }
-  if (i < M) *reinterpret_cast<uint4*>(lx + i * kx + c0) = *reinterpret_cast<const uint4*>(lo_);
-  if (i < N) *reinterpret_cast<uint4*>(rx + i * kx + c0) = *reinterpret_cast<const uint4*>(ro_);
 }
 
 // out = y0 + Lcat Rcat^T, 64 x 64 tile per CTA
@@ -530,17 +549,14 @@ metis_status_t split_gemm_prologue(metis_context* ctx, const Side& a, const Side
     METIS_CUDA_TRY(metis_launch_pdl(lowrank_deq_wide_kernel, dim3((unsigned)metis_ceil_div(mx, 32)), dim3(256), 0, s,
         M, N, ka, kb, ka ? a.fo->codes : nullptr, ka ? a.fo->scales : nullptr, ka ? a.fo->sf_layout : 0,
         ka ? a.fo->tensor_scale : nullptr, a.sigma, kb ? b.fo->codes : nullptr, kb ? b.fo->scales : nullptr,
-        kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, pl.lcat, pl.rcat)); METIS_COUNT_LAUNCH();
+        kb ? b.fo->sf_layout : 0, kb ? b.fo->tensor_scale : nullptr, pl.lcat, pl.rcat, pl.lx, pl.rx, pl.kx)); METIS_COUNT_LAUNCH();
     if (kb) {
       METIS_CUDA_TRY(metis_launch_pdl(lowrank_gemm_wide_kernel, dim3((unsigned)metis_ceil_div(kb, 64), (unsigned)metis_ceil_div(M, 64)), dim3(256), 0, s,
           M, ka, kb, b.sigma, (const float*)pl.pm, pl.lcat)); METIS_COUNT_LAUNCH();
     }
     if (pl.lx != nullptr) {
       METIS_CUDA_TRY(metis_launch_pdl(lowrank_bf16_kernel, dim3((unsigned)metis_ceil_div(mx * (pl.kx / 8), 256)), dim3(256), 0, s, M, N, ka, kb, pl.kx,
-          (const float*)pl.lcat, (const float*)pl.rcat,
-          (const uint8_t*)(ka ? a.fo->codes : nullptr), (const uint8_t*)(ka ? a.fo->scales : nullptr), ka ? a.fo->sf_layout : 0,
-          (const float*)(ka ? a.fo->tensor_scale : nullptr), (const float*)a.sigma,
-          (const uint8_t*)(kb ? b.fo->codes : nullptr), (const uint8_t*)(kb ? b.fo->scales : nullptr), kb ? b.fo->sf_layout : 0,
+          (const float*)pl.lcat, (const float*)pl.rcat, (const float*)(ka ? a.fo->tensor_scale : nullptr), (const float*)a.sigma,
           (const float*)(kb ? b.fo->tensor_scale : nullptr),
           pl.lx, pl.rx, (const float*)a.res->tensor_scale, (const float*)b.res->tensor_scale)); METIS_COUNT_LAUNCH();
     }
