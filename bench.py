@@ -128,7 +128,7 @@ class ClockSampler(threading.Thread):
 
 # ------------------------------------------------------------------------------------------------
 def oracle_sample_step(sample_tokens, seed, d_in=4096, d_out=4096, k=32, p=8):
-    """One pass of the oracle over a token sample of one q_proj-shaped layer.  Returns (seconds, flops credited)."""
+    """One pass of the oracle over a token sample of one q_proj-shaped layer.  Returns (seconds, flops credited, seconds per phase)."""
     from oracle import layer as olay, nvfp4 as onv, split as osp
     from paper_2509_00404_b200 import synth
     x, _ = synth.llama_like(sample_tokens, d_in, 1.0, seed)
@@ -144,8 +144,7 @@ def oracle_sample_step(sample_tokens, seed, d_in=4096, d_out=4096, k=32, p=8):
     dw = olay.linear_wgrad(dq, xq)
     dt = time.perf_counter() - t0
     assert np.isfinite(y).all() and np.isfinite(dx).all() and np.isfinite(dw).all()
-    oracle_sample_step.phases = {"split_and_quantize_s": t1 - t0, "three_products_s": dt - (t1 - t0)}
-    return dt, 6.0 * sample_tokens * d_in * d_out
+    return dt, 6.0 * sample_tokens * d_in * d_out, {"split_and_quantize_s": t1 - t0, "three_products_s": dt - (t1 - t0)}
 
 
 def cpu_threads():
@@ -163,7 +162,7 @@ def run_reference(args):
         oracle_sample_step(sample, 900)
     times, flops = [], 0.0
     for i in range(args.steps):
-        dt, f = oracle_sample_step(sample, 1000 + 10 * i)
+        dt, f, _ = oracle_sample_step(sample, 1000 + 10 * i)
         times.append(dt)
         flops = f
     ms = 1e3 * sum(times) / len(times)
@@ -725,10 +724,10 @@ def main():
         del qa, qb, out_p
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample = 4096
-        dt, f = oracle_sample_step(sample, 4242)
+        dt, f, phases = oracle_sample_step(sample, 4242)
         line["cpu_baseline"] = {"value": f / dt / 1e12, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle",
                                 "sample": "the q projection of the block (4096->4096) on %d of 16384 tokens, one pass (%.1f s)" % (sample, dt),
-                                "phases": oracle_sample_step.phases}
+                                "phases": phases}
     if args.dry_run_ranks_on_one_gpu:
         line["dry_run"] = "%d ranks on one GPU, gloo: control flow only, not a measurement" % world
     if rank == 0:
